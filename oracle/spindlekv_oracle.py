@@ -1,0 +1,335 @@
+"""CPU checker for the SpindleKV prefill KV-cache reduction pass.
+
+TEST INFRASTRUCTURE ONLY.  This file is the slow, plain restatement of what
+the paper defines, in numpy float64.  It shares no code with the CUDA library
+and must never be imported by it; only the tests, the smoke check and the
+benchmark's CPU-baseline leg may call it.
+
+Every function names the passage it follows.  Equations are numbered in print
+order: (1) masked softmax attention, (2) accumulated attention score, (3) GQA
+group mean, (4) cosine similarity, (5) first/last-layer retain ratios,
+(6) per-layer interpolation, (7) argTopK selection, (8) magnitudes,
+(9) thresholded adjacency, (10) node degree, (11) greedy centre pick,
+(12) reference assignment, (13) graph clean-up, (14) reconstruction.
+"Algorithm 1" is the CodeBook-generation listing.
+
+Readings taken where the text is silent, garbled or inconsistent:
+
+* Eq. (2): ``A[i, a, b]`` is the weight query ``b`` puts on key ``a``; the
+  denominator is ``l - a`` exactly as printed.
+* Eq. (3): the sum runs over ``g = 0 .. h_n - 1`` and the printed ``n - a`` is
+  ``l - a``.
+* Eq. (1): causal mask; each window query ``b`` is normalised over keys
+  ``0..b`` (window keys included); scale ``1 / sqrt(d_h)``.
+* Eq. (5): the printed ``0.05`` is ``beta`` and the last case is
+  ``2 r_c - 1`` (this is the only reading that is continuous at ``alpha`` and
+  keeps the mean over layers equal to ``r_c``).
+* Eq. (7): ties go to the lower index; the kept indices are returned in
+  ascending position followed by the window positions.
+* Eq. (9): strict ``>``; the diagonal of ``G`` is 1 (a token is similar to
+  itself, which is what lets the loop end and gives isolated tokens an entry).
+* Eq. (10) / Algorithm 1: the degree is the row sum of ``G`` (the listing
+  prints ``S``).
+* Eq. (11): ``argmax`` ties go to the lower index; a CodeBook entry is the
+  unit vector of the centre token (no averaging).
+* Zero vectors get ``gamma_hat = 0`` and therefore an entry of their own.
+* The shallow/deep split is an argument: layers ``< n_shallow`` build
+  CodeBooks over all tokens, layers ``>= n_shallow`` evict, with the pyramid
+  of Eq. (5)(6) laid over the evicting layers only.
+"""
+from __future__ import annotations
+
+import math
+from typing import Dict, List, Optional, Sequence, Tuple
+
+import numpy as np
+
+MODE_EVICT = 1
+MODE_CODEBOOK = 2
+
+
+class BudgetError(ValueError):
+    """The context reserve ratio falls outside ``(beta, 1]`` where Eq. (5) is defined."""
+
+
+# --------------------------------------------------------------------------
+# Budget planner: the unnumbered r_c definition, Eq. (5), Eq. (6), Eq. (7)'s k
+# --------------------------------------------------------------------------
+
+def context_reserve_ratio(reserved_tokens: float, l: int, l_w: int) -> float:
+    """``r_c = (r*l - l_w) / l_c`` with ``l_c = l - l_w`` (Section 3.3).
+
+    ``reserved_tokens`` is the product ``r * l``: tokens kept per head, the
+    observation window included.
+    """
+    l_c = l - l_w
+    if l_c <= 0:
+        raise BudgetError("sequence not longer than the observation window")
+    return (float(reserved_tokens) - float(l_w)) / float(l_c)
+
+
+def pyramid_endpoints(r_c: float, beta: float) -> Tuple[float, float]:
+    """Retain ratios of the first and last evicting layer, Eq. (5)."""
+    alpha = 0.5 * (1.0 + beta)
+    if beta < r_c <= alpha:
+        return 2.0 * r_c - beta, beta
+    if alpha < r_c <= 1.0:
+        return 1.0, 2.0 * r_c - 1.0
+    raise BudgetError(f"r_c={r_c} outside (beta, 1]")
+
+
+def layer_ratio(r_first: float, r_last: float, m: int, lam: int, r_c: float) -> float:
+    """Eq. (6): linear interpolation over ``m`` evicting layers (``m == 1``: flat ``r_c``)."""
+    if m == 1:
+        return r_c
+    return r_first + (r_last - r_first) / float(m - 1) * float(lam)
+
+
+def plan_layers(n_layers: int, n_shallow: int, seq_lens: Sequence[int], l_w: int, beta: float,
+                reserve_ratio: Optional[float] = None, budget_tokens: Optional[float] = None):
+    """Per-layer mode, retain ratio and top-k size for every sequence.
+
+    Returns ``(mode[m], r_c_layer[m, B], k_ctx[m, B])``; shallow layers carry
+    ratio 1 and ``k = l_c`` (nothing is evicted there).  ``k`` follows Eq. (7):
+    ``floor(r_c(lambda) * l_c)``.
+    """
+    B = len(seq_lens)
+    m_deep = n_layers - n_shallow
+    mode = np.array([MODE_CODEBOOK if lam < n_shallow else MODE_EVICT for lam in range(n_layers)],
+                    dtype=np.int32)
+    ratio = np.ones((n_layers, B), dtype=np.float64)
+    k_ctx = np.zeros((n_layers, B), dtype=np.int32)
+    for s, l in enumerate(seq_lens):
+        l_c = l - l_w
+        if l_c <= 0:
+            raise BudgetError("sequence not longer than the observation window")
+        k_ctx[:n_shallow, s] = l_c
+        if m_deep == 0:
+            continue
+        rl = float(budget_tokens) if budget_tokens is not None else float(reserve_ratio) * float(l)
+        r_c = context_reserve_ratio(rl, l, l_w)
+        r0, r1 = pyramid_endpoints(r_c, beta)
+        for lam in range(m_deep):
+            r = layer_ratio(r0, r1, m_deep, lam, r_c)
+            ratio[n_shallow + lam, s] = r
+            k_ctx[n_shallow + lam, s] = min(l_c, int(math.floor(r * float(l_c))))
+    return mode, ratio, k_ctx
+
+
+# --------------------------------------------------------------------------
+# Deep layers: Eq. (1), (2), (3), (7)
+# --------------------------------------------------------------------------
+
+def window_attention(q_win: np.ndarray, k: np.ndarray) -> np.ndarray:
+    """Eq. (1) restricted to the last ``w`` queries of one head.
+
+    ``q_win`` is ``[w, d]`` (queries at positions ``l-w .. l-1``), ``k`` is
+    ``[l, d]``.  Returns ``A[t, a]``: the weight window query ``t`` (position
+    ``b = l - w + t``) puts on key ``a``; zero where ``a > b``.
+    """
+    q_win = np.asarray(q_win, dtype=np.float64)
+    k = np.asarray(k, dtype=np.float64)
+    w, d = q_win.shape
+    l = k.shape[0]
+    s = (q_win @ k.T) / math.sqrt(d)
+    pos_b = (l - w) + np.arange(w)[:, None]
+    allowed = np.arange(l)[None, :] <= pos_b
+    s = np.where(allowed, s, -np.inf)
+    s = s - s.max(axis=1, keepdims=True)
+    e = np.exp(s)
+    return e / e.sum(axis=1, keepdims=True)
+
+
+def accumulated_scores(q_win: np.ndarray, k: np.ndarray, divide_by_distance: bool = True) -> np.ndarray:
+    """Eq. (2): ``ac[a] = sum_b A[b, a] / (l - a)`` over the window queries, for all ``a < l``.
+
+    With ``divide_by_distance=False`` the raw window sum is returned (an
+    extension outside the paper, used only to pin the tie-break).
+    """
+    A = window_attention(q_win, k)
+    l = k.shape[0]
+    ac = A.sum(axis=0)
+    if divide_by_distance:
+        ac = ac / (l - np.arange(l, dtype=np.float64))
+    return ac
+
+
+def group_scores(q_win_heads: np.ndarray, k_heads: np.ndarray, divide_by_distance: bool = True) -> np.ndarray:
+    """Eq. (3): mean of Eq. (2) over the ``h_n`` query heads that share each KV head.
+
+    ``q_win_heads`` is ``[H_q, w, d]``, ``k_heads`` is ``[H_kv, l, d]``;
+    query head ``h_n * j + g`` reads KV head ``j``.  Returns ``[H_kv, l]``.
+    """
+    H_q, H_kv = q_win_heads.shape[0], k_heads.shape[0]
+    h_n = H_q // H_kv
+    l = k_heads.shape[1]
+    out = np.zeros((H_kv, l), dtype=np.float64)
+    for j in range(H_kv):
+        for g in range(h_n):
+            out[j] += accumulated_scores(q_win_heads[h_n * j + g], k_heads[j], divide_by_distance)
+        out[j] /= float(h_n)
+    return out
+
+
+def arg_topk(scores: np.ndarray, k: int) -> np.ndarray:
+    """Eq. (7): indices of the ``k`` largest scores, ties to the lower index, ascending."""
+    scores = np.asarray(scores, dtype=np.float64)
+    idx = np.arange(scores.shape[0])
+    order = np.lexsort((idx, -scores))  # primary: score descending; secondary: index ascending
+    return np.sort(order[:k]).astype(np.int32)
+
+
+def evict_deep(q_win_heads: np.ndarray, k_heads: np.ndarray, k_ctx: int,
+               divide_by_distance: bool = True) -> Dict[str, np.ndarray]:
+    """Eq. (1)(2)(3)(7) for one (layer, sequence).
+
+    Returns ``keep[H_kv, k_ctx + w]`` (selected context positions ascending,
+    then the window positions, which are always reserved) and the context
+    scores ``[H_kv, l_c]``.
+    """
+    w = q_win_heads.shape[1]
+    H_kv, l, _ = k_heads.shape
+    l_c = l - w
+    sc = group_scores(q_win_heads, k_heads, divide_by_distance)[:, :l_c]
+    keep = np.empty((H_kv, k_ctx + w), dtype=np.int32)
+    for j in range(H_kv):
+        keep[j, :k_ctx] = arg_topk(sc[j], k_ctx)
+        keep[j, k_ctx:] = np.arange(l_c, l)
+    return {"keep": keep, "scores": sc}
+
+
+def topk_margin_mask(scores: np.ndarray, k: int, rel: float = 1e-4) -> np.ndarray:
+    """Positions whose score lies within ``rel`` (relative) of the k-th largest score.
+
+    Membership of such positions in the kept set may legitimately differ
+    between two correct implementations that round differently.
+    """
+    scores = np.asarray(scores, dtype=np.float64)
+    if k <= 0 or k >= scores.shape[0]:
+        return np.zeros(scores.shape[0], dtype=bool)
+    kth = np.sort(scores)[::-1][k - 1]
+    return np.abs(scores - kth) < rel * abs(kth)
+
+
+# --------------------------------------------------------------------------
+# Shallow layers: Eq. (4), (8)-(13), Algorithm 1
+# --------------------------------------------------------------------------
+
+def magnitudes(gamma: np.ndarray) -> np.ndarray:
+    """Eq. (8): ``m_a = sqrt(gamma_a . gamma_a)``."""
+    gamma = np.asarray(gamma, dtype=np.float64)
+    return np.sqrt((gamma * gamma).sum(axis=1))
+
+
+def normalise(gamma: np.ndarray, m: np.ndarray) -> np.ndarray:
+    """Eq. (8): ``gamma_hat = gamma / m``; a zero vector stays zero."""
+    gamma = np.asarray(gamma, dtype=np.float64)
+    safe = np.where(m > 0.0, m, 1.0)
+    return np.where(m[:, None] > 0.0, gamma / safe[:, None], 0.0)
+
+
+def cosine_similarity(gamma: np.ndarray) -> np.ndarray:
+    """Eq. (4): ``S[a, b] = gamma_a . gamma_b / (|gamma_a| |gamma_b|)`` for all pairs of one head."""
+    g = normalise(gamma, magnitudes(gamma))
+    return g @ g.T
+
+
+def adjacency(S: np.ndarray, theta: float) -> np.ndarray:
+    """Eq. (9): ``G = where(S > theta, 1, 0)`` as a symmetric boolean matrix with unit diagonal.
+
+    The pair ``(a, b)`` with ``a < b`` is decided once, from ``S[a, b]``, and
+    mirrored, so that ``G`` is an undirected graph whatever the rounding of
+    the two triangles of ``S``.
+    """
+    up = np.triu(S > theta, k=1)
+    G = up | up.T
+    np.fill_diagonal(G, True)
+    return G
+
+
+def codebook_alg1_dense(G: np.ndarray) -> Tuple[np.ndarray, np.ndarray]:
+    """Algorithm 1's loop, statement by statement, on a dense 0/1 matrix.
+
+    Degrees are recomputed as row sums each round (Eq. (10)), the centre is
+    the first arg-max (Eq. (11)), all of its current neighbours take the new
+    entry's number (Eq. (12)), and the graph is cleaned with the outer product
+    of the negated centre row (Eq. (13)), until ``G`` is all zero.
+    Cubic cost: for small ``N`` only.  Returns ``(centres, ref)``.
+    """
+    G = np.array(G, dtype=np.int64)
+    n = G.shape[0]
+    ref = -np.ones(n, dtype=np.int32)
+    centres: List[int] = []
+    while G.any():
+        s = G.sum(axis=1)
+        iota = int(np.argmax(s))
+        centres.append(iota)
+        eta = np.argwhere(G[iota] == 1)[:, 0]
+        ref[eta] = len(centres) - 1
+        not_row = 1 - G[iota]
+        mask = np.matmul(not_row[:, None], not_row[None, :])
+        G = G & mask
+    return np.array(centres, dtype=np.int32), ref
+
+
+def codebook_greedy(G: np.ndarray) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
+    """Eq. (10)-(13) on a set of live nodes, usable at full sequence length.
+
+    The same steps as Algorithm 1, in the same order; the only difference is
+    bookkeeping: removed nodes leave a ``live`` set instead of having their
+    rows and columns zeroed, and the degree vector of Eq. (10) is kept current
+    by subtracting, for every removed node, its row of ``G`` (``G`` is
+    symmetric, so that row is exactly what the node contributed to the other
+    degrees).  Returns ``(centres, ref, pick_degree)``.
+    """
+    G = np.asarray(G, dtype=bool)
+    n = G.shape[0]
+    live = np.ones(n, dtype=bool)
+    s = G.sum(axis=1).astype(np.int64)
+    ref = -np.ones(n, dtype=np.int32)
+    centres: List[int] = []
+    degs: List[int] = []
+    n_live = n
+    while n_live > 0:
+        iota = int(np.argmax(np.where(live, s, -1)))
+        eta = np.flatnonzero(G[iota] & live)
+        ref[eta] = len(centres)
+        centres.append(iota)
+        degs.append(int(s[iota]))
+        live[eta] = False
+        n_live -= eta.shape[0]
+        s -= G[eta].sum(axis=0)
+    return np.array(centres, dtype=np.int32), ref, np.array(degs, dtype=np.int64)
+
+
+def codebook_shallow(gamma: np.ndarray, theta: float, G_override: Optional[np.ndarray] = None) -> Dict[str, np.ndarray]:
+    """Algorithm 1 for one (layer, sequence, KV head, Gamma in {K, V}).
+
+    Returns magnitudes ``mag[N]``, references ``ref[N]``, centre token indices
+    ``centres[|C|]``, the CodeBook ``C[|C|, d]`` (unit vectors of the centres)
+    and the similarity matrix ``S``.  ``G_override`` replaces the adjacency
+    (used by tests to settle pairs that sit on the threshold).
+    """
+    gamma = np.asarray(gamma, dtype=np.float64)
+    mag = magnitudes(gamma)
+    ghat = normalise(gamma, mag)
+    S = ghat @ ghat.T
+    G = adjacency(S, theta) if G_override is None else np.asarray(G_override, dtype=bool)
+    centres, ref, degs = codebook_greedy(G)
+    return {"mag": mag, "ref": ref, "centres": centres, "C": ghat[centres], "S": S, "G": G,
+            "pick_degree": degs}
+
+
+def threshold_margin_mask(S: np.ndarray, theta: float, rel: float = 1e-4) -> np.ndarray:
+    """Pairs whose similarity lies within ``rel`` (relative) of the threshold."""
+    return np.abs(S - theta) < rel * abs(theta)
+
+
+def reconstruct(C: np.ndarray, ref: np.ndarray, mag: np.ndarray) -> np.ndarray:
+    """Eq. (14): ``Gamma_r = C[r] (x) m``."""
+    return np.asarray(C, dtype=np.float64)[ref] * np.asarray(mag, dtype=np.float64)[:, None]
+
+
+def gather_rows(gamma: np.ndarray, idx: np.ndarray) -> np.ndarray:
+    """Eq. (7), second line: ``Gamma_r = Gamma[eta]``."""
+    return np.asarray(gamma)[np.asarray(idx, dtype=np.int64)]
