@@ -1,0 +1,191 @@
+/*
+ * spindlekv.h -- C ABI of the B200 (sm_100a) SpindleKV prefill KV-cache reduction pass.
+ *
+ * The pass runs once per layer after prompt encoding (Section 3 of the paper):
+ *   deep layers    : attention-weight based token eviction  (Section 3.3, Eq. (1)(2)(3)(7));
+ *   shallow layers : similarity based token replacement by a CodeBook (Section 3.4, Eq. (4), (8)-(13),
+ *                    Algorithm 1).
+ * Layers do not interact, so every call takes a batch of layers.
+ *
+ * Conventions shared by all entry points
+ *   - Plain C: pointers, sizes, two small structs.  No allocation inside the library: the caller
+ *     owns every buffer, including the scratch workspace (size from spindlekv_workspace_bytes).
+ *   - "device" pointers are CUDA global memory of the current device; "host" pointers are ordinary
+ *     host memory.  `stream` is a cudaStream_t passed as void*.
+ *   - Device work is only enqueued; the functions return as soon as the launches are issued.  The
+ *     return value reports argument / launch errors.  Conditions detected on the device (a bounded
+ *     wait that gave up) land in a status word at the start of the workspace, read back with
+ *     spindlekv_poll_status after the caller has synchronised the stream.
+ *   - Tensors are addressed as
+ *         ptr + layer*stride_layer + seq*stride_seq + head*stride_head + row*stride_tok   (+ 0..head_dim-1)
+ *     with strides in ELEMENTS and head_dim contiguous.  When `cu_seqlens` is given (packed,
+ *     variable-length batch) token t of sequence s lives at row cu_seqlens[s] + t and stride_seq
+ *     is ignored for that tensor; otherwise every sequence has max_len tokens.
+ *   - Per-token outputs (scores, keep_idx, mag, ref, centre_idx) are laid out [n_layers][n_kv_heads][T]
+ *     where T = cu_seqlens[B] (packed) or B*max_len, and sequence s starts at column
+ *     tok_base(s) = cu_seqlens[s] (packed) or s*max_len.  Per-unit counts are [n_layers][B][n_kv_heads].
+ *   - head_dim must be 64 or 128; dtype fp32 or bf16; base pointers 16-byte aligned and
+ *     strides multiples of 8 elements.
+ *   - Nothing is written out of bounds on any error; outputs are undefined after a non-OK status.
+ */
+#ifndef SPINDLEKV_H_
+#define SPINDLEKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int32_t spindlekv_status;
+enum {
+  SPINDLEKV_OK = 0,
+  SPINDLEKV_INVALID_ARG = 1,         /* null pointer, non-positive size, bad stride or alignment */
+  SPINDLEKV_BUDGET = 2,              /* context reserve ratio outside (beta, 1], where Eq. (5) is undefined */
+  SPINDLEKV_WORKSPACE_TOO_SMALL = 3,
+  SPINDLEKV_CAPACITY = 4,            /* an output row is too short for what must be written */
+  SPINDLEKV_UNSUPPORTED = 5,         /* head_dim, dtype, sequence length or device not supported */
+  SPINDLEKV_CUDA = 6,                /* a CUDA runtime call failed */
+  SPINDLEKV_TIMEOUT = 7              /* a bounded device-side wait gave up (device status word only) */
+};
+
+enum { SPINDLEKV_F32 = 0, SPINDLEKV_BF16 = 1 };
+enum { SPINDLEKV_MODE_EVICT = 1, SPINDLEKV_MODE_CODEBOOK = 2 };
+enum { SPINDLEKV_WS_EVICT = 0, SPINDLEKV_WS_CODEBOOK = 1 };
+
+typedef struct {
+  void* ptr;            /* device */
+  int32_t dtype;        /* SPINDLEKV_F32 or SPINDLEKV_BF16 */
+  int64_t stride_layer; /* elements */
+  int64_t stride_seq;
+  int64_t stride_head;
+  int64_t stride_tok;
+} spindlekv_tensor;
+
+/* Hyper-parameters of the method (Table 3: theta_K 0.98, theta_V 0.95, beta 0.05) and model shape. */
+typedef struct {
+  int32_t n_layers;
+  int32_t n_q_heads;      /* h   */
+  int32_t n_kv_heads;     /* h_g; query head h_n*j+g reads KV head j, h_n = h / h_g */
+  int32_t head_dim;       /* d_h */
+  int32_t window;         /* l_w: the last l_w tokens are the observation window and are always reserved */
+  int32_t n_shallow;      /* layers [0, n_shallow) build CodeBooks; layers [n_shallow, n_layers) evict */
+  double reserve_ratio;   /* r of Section 3.3 (used when budget_tokens < 0) */
+  double budget_tokens;   /* r*l given directly: tokens kept per head, window included; < 0: use reserve_ratio */
+  double beta;            /* minimal retain ratio of any layer */
+  float theta_k;          /* similarity thresholds of Eq. (9) */
+  float theta_v;
+  int32_t score_norm;     /* 0: divide by (l - a) as Eq. (2) prints; 1: plain window sum (not in the paper) */
+} spindlekv_config;
+
+/* Which layers and sequences one device call covers. */
+typedef struct {
+  int32_t n_layers;            /* layers in this call (tensor strides step through them) */
+  int32_t n_seqs;              /* B */
+  int32_t max_len;             /* longest sequence, l */
+  int32_t total_len;           /* cu_seqlens[B] when packed, else B*max_len */
+  const int32_t* cu_seqlens;   /* device [B+1], or NULL when all sequences have max_len tokens */
+} spindlekv_batch;
+
+/*
+ * Budget planner, host only (Section 3.3: r_c = (r*l - l_w)/l_c; Eq. (5) with alpha = (1+beta)/2, read
+ * as r_c(0) = 2 r_c - beta | 1 and r_c(m-1) = beta | 2 r_c - 1; Eq. (6); k = floor(r_c(lambda) * l_c), Eq. (7)).
+ * The pyramid is laid over the evicting layers [n_shallow, n_layers); all arithmetic in IEEE double
+ * in the order the equations print.
+ *   seq_lens   host [B]
+ *   layer_mode host out [n_layers]      SPINDLEKV_MODE_*
+ *   r_c_layer  host out [n_layers][B]   retain ratio of the context (1 for CodeBook layers)
+ *   k_ctx      host out [n_layers][B]   context tokens kept per head (l_c for CodeBook layers)
+ * Returns BUDGET when some sequence has r_c <= beta or r_c > 1, INVALID_ARG when l <= l_w.
+ */
+spindlekv_status spindlekv_plan_layers(const spindlekv_config* cfg, int32_t n_seqs, const int32_t* seq_lens,
+                                       int32_t* layer_mode, double* r_c_layer, int32_t* k_ctx);
+
+/* Bytes of device scratch the given call kind (SPINDLEKV_WS_*) needs for `batch`.  0 on bad arguments. */
+size_t spindlekv_workspace_bytes(const spindlekv_config* cfg, const spindlekv_batch* batch, int32_t which);
+
+/*
+ * Eviction of deep layers (Eq. (1): causal softmax of the window queries over keys 0..b, scale 1/sqrt(d_h);
+ * Eq. (2): per-key sum over the l_w window queries divided by (l - a); Eq. (3): mean over the h_n query
+ * heads of a group; Eq. (7): argTopK with k = k_ctx, ties to the lower index).
+ *   K        device, [layer][seq][kv head][token][d]
+ *   Qwin     device, [layer][seq][q head][window row][d] (rows are the queries at positions l-l_w .. l-1;
+ *            never packed: stride_seq always applies)
+ *   k_ctx    device [n_layers][B]
+ *   keep_idx device out [n_layers][n_kv_heads][T]: per unit, from tok_base(s): the k selected context
+ *            positions ascending, then the l_w window positions
+ *   keep_cnt device out [n_layers][B][n_kv_heads] = k + l_w
+ *   scores   device out [n_layers][n_kv_heads][T] fp32: ac' of Eq. (3) for context positions
+ *            (window columns are left untouched); may not be NULL
+ */
+spindlekv_status spindlekv_evict_deep(const spindlekv_config* cfg, const spindlekv_batch* batch,
+                                      spindlekv_tensor K, spindlekv_tensor Qwin, const int32_t* k_ctx,
+                                      int32_t* keep_idx, int32_t* keep_cnt, float* scores,
+                                      void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * CodeBook construction for shallow layers, one call per Gamma in {K, V} (Algorithm 1):
+ * magnitudes (Eq. (8)); cosine similarity of all token pairs of a head (Eq. (4)); adjacency
+ * G = [S > theta] with unit diagonal (Eq. (9)); then repeatedly: degrees (Eq. (10)), centre = arg-max
+ * degree with ties to the lower index (Eq. (11)), every live neighbour of the centre refers to the new
+ * entry (Eq. (12)), centre and neighbours leave the graph (Eq. (13)), until the graph is empty.
+ * The decision S > theta is taken in fp32 as  dot(a,b) > theta * (|a| * |b|).
+ *   Gamma      device, [layer][seq][kv head][token][d]
+ *   mag        device out [n_layers][n_kv_heads][T] fp32   |gamma_a|
+ *   ref        device out [n_layers][n_kv_heads][T] int32  CodeBook entry of each token
+ *   centre_idx device out [n_layers][n_kv_heads][T] int32  per unit, from tok_base(s): token position of
+ *              entry 0, 1, ... (the CodeBook itself is these rows divided by their magnitude: see
+ *              spindlekv_compact)
+ *   n_entries  device out [n_layers][B][n_kv_heads]
+ *   adj_bits   device out, optional (NULL: kept in the workspace): the adjacency as a bit matrix,
+ *              [n_layers*B*n_kv_heads][max_len][row_words] uint32, row_words = 4*ceil(max_len/128);
+ *              bit (b & 31) of word b >> 5 of row a is G[a][b]
+ */
+spindlekv_status spindlekv_codebook_shallow(const spindlekv_config* cfg, const spindlekv_batch* batch,
+                                            spindlekv_tensor Gamma, float theta,
+                                            float* mag, int32_t* ref, int32_t* centre_idx, int32_t* n_entries,
+                                            uint32_t* adj_bits, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Gather rows into the output cache (Eq. (7), Gamma_r = Gamma[eta]; Eq. (11), C <- C + [gamma_hat_iota]).
+ * For every (layer, seq, head) copies rows idx[0..cnt) of `src` to rows 0..cnt of `dst`.
+ *   idx        device [n_layers][n_heads][T] as written by the two calls above
+ *   cnt        device [n_layers][B][n_heads]
+ *   divide_by  device, optional [n_layers][n_heads][T] fp32: when given, source row a is divided by
+ *              divide_by[a] (a zero divisor yields a zero row); pass `mag` to obtain unit CodeBook vectors
+ *   dst        device, same addressing rules as src; when dst_cu_seqlens is given, unit s starts at row
+ *              dst_cu_seqlens[s] of dst, else rows are addressed like src (batch->cu_seqlens or stride_seq)
+ * src and dst must have the same dtype and may not overlap.
+ */
+spindlekv_status spindlekv_compact(const spindlekv_batch* batch, int32_t n_heads, int32_t head_dim,
+                                   spindlekv_tensor src, const int32_t* idx, const int32_t* cnt,
+                                   const float* divide_by, spindlekv_tensor dst, const int32_t* dst_cu_seqlens,
+                                   void* stream);
+
+/*
+ * Reads the device status word of a workspace (blocking copy; synchronise the stream first).
+ *   device_status host out: SPINDLEKV_OK or SPINDLEKV_TIMEOUT
+ *   detail        host out, optional [4]: {greedy rounds used, live tokens left, 0, 0}
+ */
+spindlekv_status spindlekv_poll_status(const void* ws, int32_t* device_status, int32_t* detail);
+
+/* Number of kernels this library has launched since load (or since the last reset). */
+int64_t spindlekv_launch_count(int32_t reset);
+
+/*
+ * Optional per-kernel timing with CUDA events recorded on the caller's stream around each launch.
+ * spindlekv_timing_enable(1) starts collecting (costs two event records per launch);
+ * spindlekv_timing_read synchronises the recorded events and returns, for kernel class `which`
+ * (0 window-score, 1 top-k, 2 norms, 3 similarity, 4 degree, 5 greedy, 6 finalise, 7 gather),
+ * the summed milliseconds and the number of launches since the last spindlekv_timing_enable call.
+ */
+void spindlekv_timing_enable(int32_t on);
+spindlekv_status spindlekv_timing_read(int32_t which, double* ms_total, int64_t* launches);
+
+const char* spindlekv_status_string(spindlekv_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPINDLEKV_H_ */

@@ -1,0 +1,228 @@
+"""Thin ctypes binding of ``libspindlekv.so``: same names as the C ABI, argument marshalling only.
+
+Every step of the reduction pass runs in the library's CUDA kernels; torch is used for device
+memory and streams.  Loading fails loudly when the library is missing and cannot be built.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import dataclasses
+import os
+from typing import Optional, Sequence
+
+import numpy as np
+import torch
+
+from . import build as _build
+
+OK, INVALID_ARG, BUDGET, WORKSPACE_TOO_SMALL, CAPACITY, UNSUPPORTED, CUDA_ERROR, TIMEOUT = range(8)
+F32, BF16 = 0, 1
+MODE_EVICT, MODE_CODEBOOK = 1, 2
+WS_EVICT, WS_CODEBOOK = 0, 1
+KERNEL_CLASSES = ("window_score", "topk", "norms", "similarity", "degree", "greedy", "finalise", "gather")
+
+
+class SpindleKVError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {_lib.spindlekv_status_string(status).decode()} (status {status})")
+
+
+class _Tensor(C.Structure):
+    _fields_ = [("ptr", C.c_void_p), ("dtype", C.c_int32), ("stride_layer", C.c_int64),
+                ("stride_seq", C.c_int64), ("stride_head", C.c_int64), ("stride_tok", C.c_int64)]
+
+
+class _Config(C.Structure):
+    _fields_ = [("n_layers", C.c_int32), ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32),
+                ("head_dim", C.c_int32), ("window", C.c_int32), ("n_shallow", C.c_int32),
+                ("reserve_ratio", C.c_double), ("budget_tokens", C.c_double), ("beta", C.c_double),
+                ("theta_k", C.c_float), ("theta_v", C.c_float), ("score_norm", C.c_int32)]
+
+
+class _Batch(C.Structure):
+    _fields_ = [("n_layers", C.c_int32), ("n_seqs", C.c_int32), ("max_len", C.c_int32),
+                ("total_len", C.c_int32), ("cu_seqlens", C.c_void_p)]
+
+
+def _load() -> C.CDLL:
+    path = _build.LIB
+    if not os.path.exists(path):
+        path = _build.build()
+    lib = C.CDLL(path)
+    lib.spindlekv_status_string.restype = C.c_char_p
+    lib.spindlekv_status_string.argtypes = [C.c_int32]
+    lib.spindlekv_plan_layers.restype = C.c_int32
+    lib.spindlekv_plan_layers.argtypes = [C.POINTER(_Config), C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+    lib.spindlekv_workspace_bytes.restype = C.c_size_t
+    lib.spindlekv_workspace_bytes.argtypes = [C.POINTER(_Config), C.POINTER(_Batch), C.c_int32]
+    lib.spindlekv_evict_deep.restype = C.c_int32
+    lib.spindlekv_evict_deep.argtypes = [C.POINTER(_Config), C.POINTER(_Batch), _Tensor, _Tensor, C.c_void_p,
+                                         C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+    lib.spindlekv_codebook_shallow.restype = C.c_int32
+    lib.spindlekv_codebook_shallow.argtypes = [C.POINTER(_Config), C.POINTER(_Batch), _Tensor, C.c_float,
+                                               C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                               C.c_void_p, C.c_size_t, C.c_void_p]
+    lib.spindlekv_compact.restype = C.c_int32
+    lib.spindlekv_compact.argtypes = [C.POINTER(_Batch), C.c_int32, C.c_int32, _Tensor, C.c_void_p, C.c_void_p,
+                                      C.c_void_p, _Tensor, C.c_void_p, C.c_void_p]
+    lib.spindlekv_poll_status.restype = C.c_int32
+    lib.spindlekv_poll_status.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
+    lib.spindlekv_launch_count.restype = C.c_int64
+    lib.spindlekv_launch_count.argtypes = [C.c_int32]
+    lib.spindlekv_timing_enable.restype = None
+    lib.spindlekv_timing_enable.argtypes = [C.c_int32]
+    lib.spindlekv_timing_read.restype = C.c_int32
+    lib.spindlekv_timing_read.argtypes = [C.c_int32, C.c_void_p, C.c_void_p]
+    return lib
+
+
+_lib = _load()
+LIBRARY_PATH = _build.LIB
+
+
+@dataclasses.dataclass
+class Config:
+    n_layers: int
+    n_q_heads: int
+    n_kv_heads: int
+    head_dim: int
+    window: int
+    n_shallow: int
+    reserve_ratio: float = -1.0
+    budget_tokens: float = -1.0
+    beta: float = 0.05
+    theta_k: float = 0.98
+    theta_v: float = 0.95
+    score_norm: int = 0
+
+    def c(self) -> _Config:
+        return _Config(self.n_layers, self.n_q_heads, self.n_kv_heads, self.head_dim, self.window, self.n_shallow,
+                       self.reserve_ratio, self.budget_tokens, self.beta, self.theta_k, self.theta_v, self.score_norm)
+
+
+@dataclasses.dataclass
+class Batch:
+    n_layers: int
+    n_seqs: int
+    max_len: int
+    total_len: int
+    cu_seqlens: Optional[torch.Tensor] = None  # device int32 [B+1]
+
+    def c(self) -> _Batch:
+        ptr = self.cu_seqlens.data_ptr() if self.cu_seqlens is not None else None
+        return _Batch(self.n_layers, self.n_seqs, self.max_len, self.total_len, ptr)
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise TypeError(f"unsupported dtype {t.dtype}")
+
+
+def desc_bhnd(t: torch.Tensor) -> _Tensor:
+    """Descriptor of a ``[layers, B, heads, rows, d]`` tensor (any strides, ``d`` contiguous)."""
+    assert t.dim() == 5 and t.stride(4) == 1
+    return _Tensor(t.data_ptr(), _dtype_code(t), t.stride(0), t.stride(1), t.stride(2), t.stride(3))
+
+
+def desc_thd(t: torch.Tensor) -> _Tensor:
+    """Descriptor of a packed ``[layers, total_tokens, heads, d]`` tensor (used with cu_seqlens)."""
+    assert t.dim() == 4 and t.stride(3) == 1
+    return _Tensor(t.data_ptr(), _dtype_code(t), t.stride(0), 0, t.stride(2), t.stride(1))
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else t.data_ptr()
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def _check(status: int, where: str) -> None:
+    if status != OK:
+        raise SpindleKVError(status, where)
+
+
+def spindlekv_plan_layers(cfg: Config, seq_lens: Sequence[int]):
+    """Host planner: returns ``(layer_mode[m], r_c_layer[m, B], k_ctx[m, B])`` as numpy arrays."""
+    B = len(seq_lens)
+    lens = np.ascontiguousarray(seq_lens, dtype=np.int32)
+    mode = np.zeros(cfg.n_layers, dtype=np.int32)
+    ratio = np.zeros((cfg.n_layers, B), dtype=np.float64)
+    k_ctx = np.zeros((cfg.n_layers, B), dtype=np.int32)
+    cc = cfg.c()
+    st = _lib.spindlekv_plan_layers(C.byref(cc), B, lens.ctypes.data, mode.ctypes.data, ratio.ctypes.data,
+                                    k_ctx.ctypes.data)
+    _check(st, "spindlekv_plan_layers")
+    return mode, ratio, k_ctx
+
+
+def spindlekv_workspace_bytes(cfg: Config, batch: Batch, which: int) -> int:
+    cc, bb = cfg.c(), batch.c()
+    return int(_lib.spindlekv_workspace_bytes(C.byref(cc), C.byref(bb), which))
+
+
+def spindlekv_evict_deep(cfg: Config, batch: Batch, K: _Tensor, Qwin: _Tensor, k_ctx: torch.Tensor,
+                         keep_idx: torch.Tensor, keep_cnt: torch.Tensor, scores: torch.Tensor,
+                         ws: torch.Tensor, stream=None) -> None:
+    cc, bb = cfg.c(), batch.c()
+    st = _lib.spindlekv_evict_deep(C.byref(cc), C.byref(bb), K, Qwin, _ptr(k_ctx), _ptr(keep_idx), _ptr(keep_cnt),
+                                   _ptr(scores), _ptr(ws), ws.numel() * ws.element_size(), _stream(stream))
+    _check(st, "spindlekv_evict_deep")
+
+
+def spindlekv_codebook_shallow(cfg: Config, batch: Batch, Gamma: _Tensor, theta: float, mag: torch.Tensor,
+                               ref: torch.Tensor, centre_idx: torch.Tensor, n_entries: torch.Tensor,
+                               ws: torch.Tensor, adj_bits: Optional[torch.Tensor] = None, stream=None) -> None:
+    cc, bb = cfg.c(), batch.c()
+    st = _lib.spindlekv_codebook_shallow(C.byref(cc), C.byref(bb), Gamma, theta, _ptr(mag), _ptr(ref),
+                                         _ptr(centre_idx), _ptr(n_entries), _ptr(adj_bits), _ptr(ws),
+                                         ws.numel() * ws.element_size(), _stream(stream))
+    _check(st, "spindlekv_codebook_shallow")
+
+
+def spindlekv_compact(batch: Batch, n_heads: int, head_dim: int, src: _Tensor, idx: torch.Tensor,
+                      cnt: torch.Tensor, dst: _Tensor, divide_by: Optional[torch.Tensor] = None,
+                      dst_cu_seqlens: Optional[torch.Tensor] = None, stream=None) -> None:
+    bb = batch.c()
+    st = _lib.spindlekv_compact(C.byref(bb), n_heads, head_dim, src, _ptr(idx), _ptr(cnt), _ptr(divide_by), dst,
+                                _ptr(dst_cu_seqlens), _stream(stream))
+    _check(st, "spindlekv_compact")
+
+
+def spindlekv_poll_status(ws: torch.Tensor):
+    """Device status word of a workspace and ``[greedy rounds, live tokens left, 0, 0]``."""
+    status = C.c_int32(0)
+    detail = (C.c_int32 * 4)()
+    st = _lib.spindlekv_poll_status(_ptr(ws), C.byref(status), detail)
+    _check(st, "spindlekv_poll_status")
+    return int(status.value), [int(x) for x in detail]
+
+
+def spindlekv_launch_count(reset: bool = False) -> int:
+    return int(_lib.spindlekv_launch_count(1 if reset else 0))
+
+
+def spindlekv_timing_enable(on: bool) -> None:
+    _lib.spindlekv_timing_enable(1 if on else 0)
+
+
+def spindlekv_timing_read():
+    """``{kernel class: (milliseconds, launches)}`` since timing was enabled."""
+    out = {}
+    for i, name in enumerate(KERNEL_CLASSES):
+        ms, n = C.c_double(0.0), C.c_int64(0)
+        _check(_lib.spindlekv_timing_read(i, C.byref(ms), C.byref(n)), "spindlekv_timing_read")
+        out[name] = (float(ms.value), int(n.value))
+    return out
+
+
+def row_words(max_len: int) -> int:
+    """Words per row of the adjacency bit matrix."""
+    return 4 * ((max_len + 127) // 128)

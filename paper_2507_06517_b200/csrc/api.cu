@@ -1,0 +1,221 @@
+// C ABI of the SpindleKV reduction library: argument checks, the host-side budget planner,
+// launch counting and optional per-kernel event timing.  Every device step lives in the kernels
+// of evict.cu / codebook.cu / compact.cu.
+#include <math.h>
+
+#include <mutex>
+#include <vector>
+
+#include "common.cuh"
+
+namespace skv {
+size_t evict_workspace_bytes(const spindlekv_config& cfg, const spindlekv_batch& b);
+size_t codebook_workspace_bytes(const spindlekv_config& cfg, const spindlekv_batch& b);
+spindlekv_status evict_deep_impl(const spindlekv_config& cfg, const spindlekv_batch& b, const spindlekv_tensor& K,
+                                 const spindlekv_tensor& Q, const int32_t* k_ctx, int32_t* keep_idx,
+                                 int32_t* keep_cnt, float* scores, void* ws, size_t ws_bytes, cudaStream_t st);
+spindlekv_status codebook_shallow_impl(const spindlekv_config& cfg, const spindlekv_batch& b,
+                                       const spindlekv_tensor& Gamma, float theta, float* mag, int32_t* ref,
+                                       int32_t* centre_idx, int32_t* n_entries, uint32_t* adj_bits, void* ws,
+                                       size_t ws_bytes, cudaStream_t st);
+spindlekv_status compact_impl(const spindlekv_batch& b, int n_heads, int head_dim, const spindlekv_tensor& src,
+                              const int32_t* idx, const int32_t* cnt, const float* divide_by,
+                              const spindlekv_tensor& dst, const int32_t* dst_cu, cudaStream_t st);
+
+// ---- launch counting and timing ---------------------------------------------------------------
+static std::mutex g_mu;
+static int64_t g_launches = 0;
+static bool g_timing = false;
+struct TimedLaunch { int kc; cudaEvent_t a, b; };
+static std::vector<TimedLaunch> g_timed;
+static std::vector<cudaEvent_t> g_pool;
+
+static cudaEvent_t get_event() {
+  if (!g_pool.empty()) { cudaEvent_t e = g_pool.back(); g_pool.pop_back(); return e; }
+  cudaEvent_t e = nullptr;
+  cudaEventCreate(&e);
+  return e;
+}
+
+void note_launch(int kclass, cudaStream_t st, bool before) {
+  std::lock_guard<std::mutex> lk(g_mu);
+  if (before) {
+    ++g_launches;
+    if (g_timing) {
+      TimedLaunch t{kclass, get_event(), get_event()};
+      cudaEventRecord(t.a, st);
+      g_timed.push_back(t);
+    }
+  } else if (g_timing && !g_timed.empty()) {
+    cudaEventRecord(g_timed.back().b, st);
+  }
+}
+}  // namespace skv
+
+using namespace skv;
+
+static bool tensor_ok(const spindlekv_tensor& t) {
+  if (!t.ptr) return false;
+  if (t.dtype != SPINDLEKV_F32 && t.dtype != SPINDLEKV_BF16) return false;
+  if (reinterpret_cast<uintptr_t>(t.ptr) % 16) return false;
+  if (t.stride_layer % 8 || t.stride_seq % 8 || t.stride_head % 8 || t.stride_tok % 8) return false;
+  return true;
+}
+
+static bool cfg_ok(const spindlekv_config* c) {
+  if (!c) return false;
+  if (c->n_layers <= 0 || c->n_q_heads <= 0 || c->n_kv_heads <= 0 || c->window <= 0) return false;
+  if (c->n_q_heads % c->n_kv_heads) return false;
+  return true;
+}
+
+static bool batch_ok(const spindlekv_batch* b, int window) {
+  if (!b) return false;
+  if (b->n_layers <= 0 || b->n_seqs <= 0 || b->max_len <= window || b->total_len < b->max_len) return false;
+  if (!b->cu_seqlens && (int64_t)b->total_len != (int64_t)b->n_seqs * b->max_len) return false;
+  return true;
+}
+
+extern "C" {
+
+const char* spindlekv_status_string(spindlekv_status s) {
+  switch (s) {
+    case SPINDLEKV_OK: return "ok";
+    case SPINDLEKV_INVALID_ARG: return "invalid argument";
+    case SPINDLEKV_BUDGET: return "context reserve ratio outside (beta, 1]";
+    case SPINDLEKV_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case SPINDLEKV_CAPACITY: return "output capacity exceeded";
+    case SPINDLEKV_UNSUPPORTED: return "unsupported shape, dtype or device";
+    case SPINDLEKV_CUDA: return "CUDA runtime error";
+    case SPINDLEKV_TIMEOUT: return "bounded device wait gave up";
+    default: return "unknown status";
+  }
+}
+
+spindlekv_status spindlekv_plan_layers(const spindlekv_config* cfg, int32_t n_seqs, const int32_t* seq_lens,
+                                       int32_t* layer_mode, double* r_c_layer, int32_t* k_ctx) {
+  if (!cfg_ok(cfg) || n_seqs <= 0 || !seq_lens || !layer_mode || !r_c_layer || !k_ctx) return SPINDLEKV_INVALID_ARG;
+  const int m = cfg->n_layers;
+  if (cfg->n_shallow < 0 || cfg->n_shallow > m) return SPINDLEKV_INVALID_ARG;
+  const int m_deep = m - cfg->n_shallow;
+  const double beta = cfg->beta;
+  const double alpha = 0.5 * (1.0 + beta);
+  for (int lam = 0; lam < m; ++lam) layer_mode[lam] = lam < cfg->n_shallow ? SPINDLEKV_MODE_CODEBOOK : SPINDLEKV_MODE_EVICT;
+  for (int s = 0; s < n_seqs; ++s) {
+    const int l = seq_lens[s];
+    const int l_c = l - cfg->window;
+    if (l_c <= 0) return SPINDLEKV_INVALID_ARG;
+    for (int lam = 0; lam < cfg->n_shallow; ++lam) {
+      r_c_layer[(size_t)lam * n_seqs + s] = 1.0;
+      k_ctx[(size_t)lam * n_seqs + s] = l_c;
+    }
+    if (m_deep == 0) continue;
+    const double rl = cfg->budget_tokens >= 0.0 ? cfg->budget_tokens : cfg->reserve_ratio * (double)l;
+    const double r_c = (rl - (double)cfg->window) / (double)l_c;
+    double r_first, r_last;
+    if (beta < r_c && r_c <= alpha) {
+      r_first = 2.0 * r_c - beta;
+      r_last = beta;
+    } else if (alpha < r_c && r_c <= 1.0) {
+      r_first = 1.0;
+      r_last = 2.0 * r_c - 1.0;
+    } else {
+      return SPINDLEKV_BUDGET;
+    }
+    for (int lam = 0; lam < m_deep; ++lam) {
+      const double r = m_deep == 1 ? r_c : r_first + (r_last - r_first) / (double)(m_deep - 1) * (double)lam;
+      int k = (int)floor(r * (double)l_c);
+      if (k > l_c) k = l_c;
+      r_c_layer[(size_t)(cfg->n_shallow + lam) * n_seqs + s] = r;
+      k_ctx[(size_t)(cfg->n_shallow + lam) * n_seqs + s] = k;
+    }
+  }
+  return SPINDLEKV_OK;
+}
+
+size_t spindlekv_workspace_bytes(const spindlekv_config* cfg, const spindlekv_batch* batch, int32_t which) {
+  if (!cfg_ok(cfg) || !batch_ok(batch, cfg->window)) return 0;
+  if (which == SPINDLEKV_WS_EVICT) return evict_workspace_bytes(*cfg, *batch);
+  if (which == SPINDLEKV_WS_CODEBOOK) return codebook_workspace_bytes(*cfg, *batch);
+  return 0;
+}
+
+spindlekv_status spindlekv_evict_deep(const spindlekv_config* cfg, const spindlekv_batch* batch, spindlekv_tensor K,
+                                      spindlekv_tensor Qwin, const int32_t* k_ctx, int32_t* keep_idx,
+                                      int32_t* keep_cnt, float* scores, void* ws, size_t ws_bytes, void* stream) {
+  if (!cfg_ok(cfg) || !batch_ok(batch, cfg->window)) return SPINDLEKV_INVALID_ARG;
+  if (!tensor_ok(K) || !tensor_ok(Qwin) || !k_ctx || !keep_idx || !keep_cnt || !scores || !ws) return SPINDLEKV_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(ws) % 256) return SPINDLEKV_INVALID_ARG;
+  if (K.dtype != Qwin.dtype) return SPINDLEKV_UNSUPPORTED;
+  if (cfg->head_dim != 64 && cfg->head_dim != 128) return SPINDLEKV_UNSUPPORTED;
+  if ((int64_t)batch->n_layers * batch->n_seqs * cfg->n_kv_heads > 65535) return SPINDLEKV_UNSUPPORTED;
+  return evict_deep_impl(*cfg, *batch, K, Qwin, k_ctx, keep_idx, keep_cnt, scores, ws, ws_bytes, (cudaStream_t)stream);
+}
+
+spindlekv_status spindlekv_codebook_shallow(const spindlekv_config* cfg, const spindlekv_batch* batch,
+                                            spindlekv_tensor Gamma, float theta, float* mag, int32_t* ref,
+                                            int32_t* centre_idx, int32_t* n_entries, uint32_t* adj_bits, void* ws,
+                                            size_t ws_bytes, void* stream) {
+  if (!cfg_ok(cfg) || !batch) return SPINDLEKV_INVALID_ARG;
+  if (batch->n_layers <= 0 || batch->n_seqs <= 0 || batch->max_len <= 0 || batch->total_len < batch->max_len) return SPINDLEKV_INVALID_ARG;
+  if (!batch->cu_seqlens && (int64_t)batch->total_len != (int64_t)batch->n_seqs * batch->max_len) return SPINDLEKV_INVALID_ARG;
+  if (!tensor_ok(Gamma) || !mag || !ref || !centre_idx || !n_entries || !ws) return SPINDLEKV_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(ws) % 256) return SPINDLEKV_INVALID_ARG;
+  if (cfg->head_dim != 64 && cfg->head_dim != 128) return SPINDLEKV_UNSUPPORTED;
+  return codebook_shallow_impl(*cfg, *batch, Gamma, theta, mag, ref, centre_idx, n_entries, adj_bits, ws, ws_bytes,
+                               (cudaStream_t)stream);
+}
+
+spindlekv_status spindlekv_compact(const spindlekv_batch* batch, int32_t n_heads, int32_t head_dim,
+                                   spindlekv_tensor src, const int32_t* idx, const int32_t* cnt,
+                                   const float* divide_by, spindlekv_tensor dst, const int32_t* dst_cu_seqlens,
+                                   void* stream) {
+  if (!batch || batch->n_layers <= 0 || batch->n_seqs <= 0 || batch->max_len <= 0 || n_heads <= 0) return SPINDLEKV_INVALID_ARG;
+  if (!tensor_ok(src) || !tensor_ok(dst) || !idx || !cnt) return SPINDLEKV_INVALID_ARG;
+  if (src.dtype != dst.dtype) return SPINDLEKV_UNSUPPORTED;
+  if (head_dim != 64 && head_dim != 128) return SPINDLEKV_UNSUPPORTED;
+  return compact_impl(*batch, n_heads, head_dim, src, idx, cnt, divide_by, dst, dst_cu_seqlens, (cudaStream_t)stream);
+}
+
+spindlekv_status spindlekv_poll_status(const void* ws, int32_t* device_status, int32_t* detail) {
+  if (!ws || !device_status) return SPINDLEKV_INVALID_ARG;
+  int32_t h[4];
+  if (cudaMemcpy(h, ws, sizeof(h), cudaMemcpyDeviceToHost) != cudaSuccess) return SPINDLEKV_CUDA;
+  *device_status = h[kHdrStatus];
+  if (detail) { detail[0] = h[kHdrRounds]; detail[1] = h[kHdrLive]; detail[2] = 0; detail[3] = 0; }
+  return SPINDLEKV_OK;
+}
+
+int64_t spindlekv_launch_count(int32_t reset) {
+  std::lock_guard<std::mutex> lk(g_mu);
+  int64_t v = g_launches;
+  if (reset) g_launches = 0;
+  return v;
+}
+
+void spindlekv_timing_enable(int32_t on) {
+  std::lock_guard<std::mutex> lk(g_mu);
+  for (auto& t : g_timed) { g_pool.push_back(t.a); g_pool.push_back(t.b); }
+  g_timed.clear();
+  g_timing = on != 0;
+}
+
+spindlekv_status spindlekv_timing_read(int32_t which, double* ms_total, int64_t* launches) {
+  if (!ms_total || !launches || which < 0 || which >= KC_COUNT) return SPINDLEKV_INVALID_ARG;
+  std::lock_guard<std::mutex> lk(g_mu);
+  double tot = 0.0;
+  int64_t n = 0;
+  for (auto& t : g_timed) {
+    if (t.kc != which) continue;
+    if (cudaEventSynchronize(t.b) != cudaSuccess) return SPINDLEKV_CUDA;
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, t.a, t.b) != cudaSuccess) return SPINDLEKV_CUDA;
+    tot += ms;
+    ++n;
+  }
+  *ms_total = tot;
+  *launches = n;
+  return SPINDLEKV_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,482 @@
+// Shallow-layer CodeBook construction (Algorithm 1): magnitudes (Eq. (8)), thresholded cosine
+// similarity as a bit matrix (Eq. (4)(9)), exact parallel form of the greedy cover (Eq. (10)-(13)),
+// and the numbering of the entries.
+//
+// Greedy cover in parallel.  Algorithm 1 picks one centre per iteration: the live node with the
+// largest live degree, lowest index on ties, i.e. the largest key (degree, -index).  A live node whose
+// key is the largest among all live nodes within graph distance 2 can be picked at once with its
+// current degree and neighbours: a pick elsewhere changes this node's degree only if it lies within
+// distance 2, and any such node has a smaller key now and a key that can only fall later, so the
+// sequential arg-max reaches this node first.  Every round picks all such nodes together; neighbours
+// of two picks of one round cannot coincide (the picks would be within distance 2 of each other).
+// Pick-time keys equal those of the sequential run and strictly decrease along it, so entry numbers
+// are the ranks of the picks by key.  The result is bit-identical to the one-at-a-time loop.
+#include "common.cuh"
+#include "simt_tile.cuh"
+
+namespace skv {
+
+struct CodebookParams {
+  View G;                // Gamma
+  Batch batch;
+  int n_kv_heads, n_units, row_words;
+  float theta;
+  float* mag;            // [layers][H][T]
+  uint32_t* adj;         // [units][max_len][row_words]
+  int32_t* deg;          // [units][max_len]
+  unsigned long long* key;  // [units][max_len]
+  unsigned long long* m1;   // [units][max_len]
+  uint32_t* live0;       // [units][row_words]
+  uint32_t* live1;
+  int32_t* owner;        // [units][max_len]
+  int32_t* pickdeg;      // [units][max_len], -1 = not a centre
+  int32_t* rank;         // [units][max_len] entry number of a centre
+  uint32_t* hdr;
+  int32_t* ref;          // [layers][H][T]
+  int32_t* centre_idx;   // [layers][H][T]
+  int32_t* n_entries;    // [layers][B][H]
+};
+
+__device__ __forceinline__ void cb_decode(const CodebookParams& p, int unit, int& layer, int& s, int& j) {
+  j = unit % p.n_kv_heads;
+  int ls = unit / p.n_kv_heads;
+  s = ls % p.batch.n_seqs;
+  layer = ls / p.batch.n_seqs;
+}
+__device__ __forceinline__ int64_t cb_out_row(const CodebookParams& p, int layer, int s, int j) {
+  return ((int64_t)layer * p.n_kv_heads + j) * p.batch.total_len + tok_base(p.batch, s);
+}
+
+// ---- Eq. (8): magnitudes.  8 lanes per row of 64 elements, 16 lanes per row of 128. -----------
+template <typename T, int D>
+__global__ void __launch_bounds__(256) norms_kernel(CodebookParams p) {
+  constexpr int LPR = D / 8;  // lanes per row
+  constexpr int RPB = 256 / LPR;
+  int layer, s, j;
+  cb_decode(p, blockIdx.y, layer, s, j);
+  const int l = seq_len(p.batch, s);
+  int row = blockIdx.x * RPB + threadIdx.x / LPR;
+  int seg = threadIdx.x % LPR;
+  float ss = 0.f;
+  if (row < l) {
+    const T* src = reinterpret_cast<const T*>(p.G.ptr) + unit_offset(p.G, p.batch, layer, s, j) + (int64_t)row * p.G.st;
+    float v[8];
+    load8(src + seg * 8, v);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) ss = fmaf(v[i], v[i], ss);
+  }
+#pragma unroll
+  for (int o = LPR / 2; o >= 1; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+  if (row < l && seg == 0) p.mag[cb_out_row(p, layer, s, j) + row] = sqrtf(ss);
+}
+
+// ---- Eq. (4)(9) on CUDA cores: 64x64 tiles, decision dot > theta * (|a| * |b|) ------------------
+template <typename T, int D>
+__global__ void __launch_bounds__(256) sim_simt_kernel(CodebookParams p) {
+  __shared__ TileSmem sm;
+  int layer, s, j;
+  cb_decode(p, blockIdx.z, layer, s, j);
+  const int l = seq_len(p.batch, s);
+  const int r0 = blockIdx.y * kTile, c0 = blockIdx.x * kTile;
+  if (r0 >= l || c0 >= row_words_for(p.batch.max_len) * 32) return;
+  const T* base = reinterpret_cast<const T*>(p.G.ptr) + unit_offset(p.G, p.batch, layer, s, j);
+  const float* mag = p.mag + cb_out_row(p, layer, s, j);
+  const int ty = threadIdx.x >> 4, tx = threadIdx.x & 15;
+  uint32_t bits[4] = {0, 0, 0, 0};
+  if (c0 < l) {
+    float acc[4][4];
+    auto row_a = [&](int r) -> const T* { return r0 + r < l ? base + (int64_t)(r0 + r) * p.G.st : nullptr; };
+    auto row_b = [&](int r) -> const T* { return c0 + r < l ? base + (int64_t)(c0 + r) * p.G.st : nullptr; };
+    dot_tile_64x64<T, D>(sm, row_a, row_b, acc);
+    float mr[4], mc[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      int a = r0 + ty * 4 + i, b = c0 + tx * 4 + i;
+      mr[i] = a < l ? mag[a] : 0.f;
+      mc[i] = b < l ? mag[b] : 0.f;
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        int a = r0 + ty * 4 + i, b = c0 + tx * 4 + c;
+        bool on = (a < l && b < l) && (a == b || acc[i][c] > p.theta * (mr[i] * mc[c]));
+        bits[i] |= (on ? 1u : 0u) << ((tx & 7) * 4 + c);
+      }
+  }
+  // eight neighbouring threads hold the 32 columns of one word
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+#pragma unroll
+    for (int o = 1; o <= 4; o <<= 1) bits[i] |= __shfl_xor_sync(0xffffffffu, bits[i], o);
+    int a = r0 + ty * 4 + i;
+    if ((tx & 7) == 0 && a < l)
+      p.adj[((int64_t)blockIdx.z * p.batch.max_len + a) * p.row_words + (c0 >> 5) + (tx >> 3)] = bits[i];
+  }
+}
+
+// ---- greedy cover, cooperative kernel over all units of the call --------------------------------
+
+constexpr uint32_t kSpinLimit = 4u << 20;
+
+// Grid-wide barrier on a monotonically increasing counter.  Every wait is bounded: when it gives up
+// it raises the TIMEOUT status, and every block that sees a non-zero status leaves the kernel.
+__device__ __forceinline__ bool grid_barrier(uint32_t* hdr, uint32_t& target) {
+  __shared__ int ok_sh;
+  __syncthreads();
+  target += gridDim.x;
+  if (threadIdx.x == 0) {
+    int ok = 1;
+    __threadfence();
+    atomicAdd(&hdr[kHdrBarrier], 1u);
+    uint32_t spins = 0;
+    while (true) {
+      uint32_t v = *reinterpret_cast<volatile uint32_t*>(&hdr[kHdrBarrier]);
+      if (v >= target) break;
+      if (*reinterpret_cast<volatile uint32_t*>(&hdr[kHdrStatus]) != 0u || ++spins > kSpinLimit) {
+        atomicExch(&hdr[kHdrStatus], (uint32_t)SPINDLEKV_TIMEOUT);
+        ok = 0;
+        break;
+      }
+      __nanosleep(64);
+    }
+    __threadfence();
+    ok_sh = ok;
+  }
+  __syncthreads();
+  return ok_sh != 0;
+}
+
+__device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long v) {
+#pragma unroll
+  for (int o = 16; o >= 1; o >>= 1) {
+    unsigned long long n = __shfl_xor_sync(0xffffffffu, v, o);
+    v = n > v ? n : v;
+  }
+  return v;
+}
+
+__global__ void __launch_bounds__(512) greedy_kernel(CodebookParams p) {
+  const int lane = threadIdx.x & 31;
+  const int warps_per_block = blockDim.x >> 5;
+  const int64_t gwarp = (int64_t)blockIdx.x * warps_per_block + (threadIdx.x >> 5);
+  const int64_t nwarps = (int64_t)gridDim.x * warps_per_block;
+  const int64_t gthread = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int64_t nthreads = (int64_t)gridDim.x * blockDim.x;
+  const int ML = p.batch.max_len, RW = p.row_words;
+  const int64_t n_rows = (int64_t)p.n_units * ML;
+  uint32_t target = 0;
+
+  // all tokens start live
+  for (int64_t i = gthread; i < (int64_t)p.n_units * RW; i += nthreads) {
+    int unit = (int)(i / RW), w = (int)(i % RW);
+    int layer, s, j;
+    cb_decode(p, unit, layer, s, j);
+    int l = seq_len(p.batch, s);
+    uint32_t m = 0;
+    if (w * 32 + 32 <= l) m = 0xFFFFFFFFu;
+    else if (w * 32 < l) m = (1u << (l - w * 32)) - 1u;
+    p.live0[i] = m;
+  }
+  if (!grid_barrier(p.hdr, target)) return;
+
+  int round = 0;
+  for (; round <= ML; ++round) {
+    uint32_t* live = (round & 1) ? p.live1 : p.live0;
+    uint32_t* next = (round & 1) ? p.live0 : p.live1;
+    const int slot = (round & 1) ? kHdrLiveCnt1 : kHdrLiveCnt0;
+    const int other = (round & 1) ? kHdrLiveCnt0 : kHdrLiveCnt1;
+    // phase 1: live degrees (Eq. (10)) and keys; `next` starts as a copy of `live`
+    for (int64_t i = gthread; i < (int64_t)p.n_units * RW; i += nthreads) next[i] = live[i];
+    if (gthread == 0) p.hdr[other] = 0;
+    int my_live = 0;
+    for (int64_t idx = gwarp; idx < n_rows; idx += nwarps) {
+      int unit = (int)(idx / ML), u = (int)(idx % ML);
+      const uint32_t* lv = live + (int64_t)unit * RW;
+      bool alive = (lv[u >> 5] >> (u & 31)) & 1u;  // bits beyond the sequence length are never set
+      if (!alive) {
+        if (lane == 0) p.key[idx] = 0ull;
+        continue;
+      }
+      const uint32_t* row = p.adj + idx * RW;
+      int cnt = 0;
+      for (int w = lane; w < RW; w += 32) cnt += __popc(row[w] & lv[w]);
+#pragma unroll
+      for (int o = 16; o >= 1; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+      if (lane == 0) {
+        p.deg[idx] = cnt;
+        p.key[idx] = ((unsigned long long)(uint32_t)cnt << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)u);
+        ++my_live;
+      }
+    }
+    if (lane == 0 && my_live) atomicAdd(&p.hdr[slot], (uint32_t)my_live);
+    if (!grid_barrier(p.hdr, target)) return;
+    const uint32_t total_live = *reinterpret_cast<volatile uint32_t*>(&p.hdr[slot]);
+    if (total_live == 0) break;
+
+    // phase 2: largest key in each closed live neighbourhood
+    for (int64_t idx = gwarp; idx < n_rows; idx += nwarps) {
+      int unit = (int)(idx / ML), u = (int)(idx % ML);
+      const uint32_t* lv = live + (int64_t)unit * RW;
+      if (!((lv[u >> 5] >> (u & 31)) & 1u)) continue;
+      const uint32_t* row = p.adj + idx * RW;
+      const unsigned long long* key = p.key + (int64_t)unit * ML;
+      unsigned long long best = 0ull;
+      for (int w = lane; w < RW; w += 32) {
+        uint32_t m = row[w] & lv[w];
+        while (m) {
+          int b = __ffs(m) - 1;
+          m &= m - 1;
+          unsigned long long kv = key[w * 32 + b];
+          best = kv > best ? kv : best;
+        }
+      }
+      best = warp_max_u64(best);
+      if (lane == 0) p.m1[idx] = best;
+    }
+    if (!grid_barrier(p.hdr, target)) return;
+
+    // phase 3: a node that is the maximum of every neighbour's neighbourhood is a centre (Eq. (11));
+    // its live neighbours take it as owner (Eq. (12)) and leave the graph (Eq. (13))
+    for (int64_t idx = gwarp; idx < n_rows; idx += nwarps) {
+      int unit = (int)(idx / ML), u = (int)(idx % ML);
+      const uint32_t* lv = live + (int64_t)unit * RW;
+      if (!((lv[u >> 5] >> (u & 31)) & 1u)) continue;
+      const unsigned long long mykey = p.key[idx];
+      if (p.m1[idx] != mykey) continue;
+      const uint32_t* row = p.adj + idx * RW;
+      const unsigned long long* m1 = p.m1 + (int64_t)unit * ML;
+      bool ok = true;
+      for (int w = lane; w < RW; w += 32) {
+        uint32_t m = row[w] & lv[w];
+        while (m) {
+          int b = __ffs(m) - 1;
+          m &= m - 1;
+          if (m1[w * 32 + b] != mykey) ok = false;
+        }
+      }
+      if (!__all_sync(0xffffffffu, ok)) continue;
+      if (lane == 0) p.pickdeg[idx] = p.deg[idx];
+      int32_t* owner = p.owner + (int64_t)unit * ML;
+      uint32_t* nx = next + (int64_t)unit * RW;
+      for (int w = lane; w < RW; w += 32) {
+        uint32_t m = row[w] & lv[w];
+        if (m) atomicAnd(&nx[w], ~m);
+        while (m) {
+          int b = __ffs(m) - 1;
+          m &= m - 1;
+          owner[w * 32 + b] = u;
+        }
+      }
+    }
+    if (!grid_barrier(p.hdr, target)) return;
+  }
+  if (gthread == 0) {
+    p.hdr[kHdrRounds] = (uint32_t)round;
+    uint32_t left = *reinterpret_cast<volatile uint32_t*>(&p.hdr[(round & 1) ? kHdrLiveCnt1 : kHdrLiveCnt0]);
+    p.hdr[kHdrLive] = round > ML ? 1u : left;
+    if (round > ML) atomicExch(&p.hdr[kHdrStatus], (uint32_t)SPINDLEKV_TIMEOUT);
+  }
+}
+
+// ---- entry numbering ------------------------------------------------------------------------------
+// One block per unit.  Entries are numbered by decreasing pick-time key (degree, then lower index):
+// a counting sort on the degree, stable in the index.  hist[] lives in dynamic shared memory.
+constexpr int kFinalThreads = 1024;
+
+__global__ void __launch_bounds__(kFinalThreads) finalize_kernel(CodebookParams p) {
+  extern __shared__ int hist[];  // [l + 2]
+  __shared__ int warp_sums[33];
+  __shared__ int carry_sh;
+  const int unit = blockIdx.x;
+  int layer, s, j;
+  cb_decode(p, unit, layer, s, j);
+  const int l = seq_len(p.batch, s);
+  const int ML = p.batch.max_len;
+  const int32_t* pickdeg = p.pickdeg + (int64_t)unit * ML;
+  const int32_t* owner = p.owner + (int64_t)unit * ML;
+  int32_t* rank = p.rank + (int64_t)unit * ML;
+  const int64_t orow = cb_out_row(p, layer, s, j);
+  const int tid = threadIdx.x, lane = tid & 31;
+
+  for (int d = tid; d <= l + 1; d += kFinalThreads) hist[d] = 0;
+  __syncthreads();
+  for (int u = tid; u < l; u += kFinalThreads) {
+    int d = pickdeg[u];
+    if (d >= 0) atomicAdd(&hist[d], 1);
+  }
+  __syncthreads();
+  // start[d] = number of centres with a larger degree: exclusive scan from the top, in place
+  if (tid == 0) carry_sh = 0;
+  __syncthreads();
+  for (int top = l; top >= 0; top -= kFinalThreads) {
+    int d = top - tid;
+    int v = d >= 0 ? hist[d] : 0;
+    // inclusive-to-exclusive scan within the block via warp shuffles
+    int inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      int n = __shfl_up_sync(0xffffffffu, inc, o);
+      if (lane >= o) inc += n;
+    }
+    if (lane == 31) warp_sums[tid >> 5] = inc;
+    __syncthreads();
+    if (tid < 32) {
+      int ws = warp_sums[tid], winc = ws;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        int n = __shfl_up_sync(0xffffffffu, winc, o);
+        if (lane >= o) winc += n;
+      }
+      warp_sums[tid] = winc - ws;
+      if (tid == 31) warp_sums[32] = winc;
+    }
+    __syncthreads();
+    int excl = warp_sums[tid >> 5] + inc - v + carry_sh;
+    int tot = warp_sums[32];
+    if (d >= 0) hist[d] = excl;
+    __syncthreads();
+    if (tid == 0) carry_sh += tot;
+    __syncthreads();
+  }
+  const int n_entries = carry_sh;
+  // stable placement in index order by one warp, eight chunks of 32 tokens in flight
+  if (tid < 32) {
+    for (int base = 0; base < l; base += 256) {
+      int dv[8];
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        int u = base + c * 32 + lane;
+        dv[c] = u < l ? pickdeg[u] : -1;
+      }
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        int u = base + c * 32 + lane;
+        int d = dv[c];
+        uint32_t peers = __match_any_sync(0xffffffffu, d);
+        if (d >= 0) {
+          int before = __popc(peers & ((1u << lane) - 1u));
+          int pos = hist[d] + before;
+          rank[u] = pos;
+          p.centre_idx[orow + pos] = u;
+        }
+        __syncwarp();
+        if (d >= 0 && lane == (31 - __clz(peers))) hist[d] += __popc(peers);
+        __syncwarp();
+      }
+    }
+  }
+  __syncthreads();
+  for (int b = tid; b < l; b += kFinalThreads) p.ref[orow + b] = rank[owner[b]];
+  if (tid == 0) p.n_entries[(layer * p.batch.n_seqs + s) * p.n_kv_heads + j] = n_entries;
+}
+
+// ---- host side ----------------------------------------------------------------------------------
+
+struct CodebookLayout {
+  size_t adj, deg, key, m1, live0, live1, owner, pickdeg, rank, total;
+};
+
+static CodebookLayout codebook_layout(const spindlekv_config& cfg, const spindlekv_batch& b, bool adj_in_ws) {
+  size_t units = (size_t)b.n_layers * b.n_seqs * cfg.n_kv_heads;
+  size_t ML = b.max_len, RW = row_words_for(b.max_len);
+  CodebookLayout L;
+  size_t off = kHeaderBytes;
+  auto take = [&](size_t bytes) { size_t o = off; off += align_up(bytes, 256); return o; };
+  L.deg = take(units * ML * 4);
+  L.key = take(units * ML * 8);
+  L.m1 = take(units * ML * 8);
+  L.live0 = take(units * RW * 4);
+  L.live1 = take(units * RW * 4);
+  L.owner = take(units * ML * 4);
+  L.pickdeg = take(units * ML * 4);
+  L.rank = take(units * ML * 4);
+  L.adj = off;
+  if (adj_in_ws) take(units * ML * RW * 4);
+  L.total = off;
+  return L;
+}
+
+size_t codebook_workspace_bytes(const spindlekv_config& cfg, const spindlekv_batch& b) {
+  return codebook_layout(cfg, b, true).total;
+}
+
+template <typename T, int D>
+static void launch_norms_sim(const CodebookParams& p, const spindlekv_batch& b, cudaStream_t st) {
+  constexpr int RPB = 256 / (D / 8);
+  { LaunchScope ls(KC_NORMS, st); norms_kernel<T, D><<<dim3(ceil_div(b.max_len, RPB), p.n_units), 256, 0, st>>>(p); }
+  int ct = ceil_div(p.row_words * 32, kTile), rt = ceil_div(b.max_len, kTile);
+  { LaunchScope ls(KC_SIM, st); sim_simt_kernel<T, D><<<dim3(ct, rt, p.n_units), 256, 0, st>>>(p); }
+}
+
+spindlekv_status codebook_shallow_impl(const spindlekv_config& cfg, const spindlekv_batch& b,
+                                       const spindlekv_tensor& Gamma, float theta, float* mag, int32_t* ref,
+                                       int32_t* centre_idx, int32_t* n_entries, uint32_t* adj_bits, void* ws,
+                                       size_t ws_bytes, cudaStream_t st) {
+  const bool adj_in_ws = adj_bits == nullptr;
+  CodebookLayout L = codebook_layout(cfg, b, adj_in_ws);
+  if (ws_bytes < L.total) return SPINDLEKV_WORKSPACE_TOO_SMALL;
+  if ((size_t)(b.max_len + 2) * 4 > 200 * 1024) return SPINDLEKV_UNSUPPORTED;
+  const int units = b.n_layers * b.n_seqs * cfg.n_kv_heads;
+  if (units > 65535) return SPINDLEKV_UNSUPPORTED;
+  char* w = reinterpret_cast<char*>(ws);
+  CodebookParams p;
+  p.G = make_view(Gamma);
+  p.batch = make_batch(b);
+  p.n_kv_heads = cfg.n_kv_heads;
+  p.n_units = units;
+  p.row_words = row_words_for(b.max_len);
+  p.theta = theta;
+  p.mag = mag;
+  p.adj = adj_in_ws ? reinterpret_cast<uint32_t*>(w + L.adj) : adj_bits;
+  p.deg = reinterpret_cast<int32_t*>(w + L.deg);
+  p.key = reinterpret_cast<unsigned long long*>(w + L.key);
+  p.m1 = reinterpret_cast<unsigned long long*>(w + L.m1);
+  p.live0 = reinterpret_cast<uint32_t*>(w + L.live0);
+  p.live1 = reinterpret_cast<uint32_t*>(w + L.live1);
+  p.owner = reinterpret_cast<int32_t*>(w + L.owner);
+  p.pickdeg = reinterpret_cast<int32_t*>(w + L.pickdeg);
+  p.rank = reinterpret_cast<int32_t*>(w + L.rank);
+  p.hdr = reinterpret_cast<uint32_t*>(w);
+  p.ref = ref;
+  p.centre_idx = centre_idx;
+  p.n_entries = n_entries;
+  if (cudaMemsetAsync(w, 0, kHeaderBytes, st) != cudaSuccess) return SPINDLEKV_CUDA;
+  if (cudaMemsetAsync(p.pickdeg, 0xFF, (size_t)units * b.max_len * 4, st) != cudaSuccess) return SPINDLEKV_CUDA;
+  const bool bf = Gamma.dtype == SPINDLEKV_BF16;
+  if (cfg.head_dim == 64) {
+    if (bf) launch_norms_sim<__nv_bfloat16, 64>(p, b, st); else launch_norms_sim<float, 64>(p, b, st);
+  } else {
+    if (bf) launch_norms_sim<__nv_bfloat16, 128>(p, b, st); else launch_norms_sim<float, 128>(p, b, st);
+  }
+  // cooperative launch: as many blocks as can be resident at once
+  static int coop_blocks = 0;
+  if (coop_blocks == 0) {
+    int dev = 0, sms = 0, per_sm = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return SPINDLEKV_CUDA;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return SPINDLEKV_CUDA;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, greedy_kernel, 512, 0) != cudaSuccess) return SPINDLEKV_CUDA;
+    if (per_sm < 1) return SPINDLEKV_CUDA;
+    coop_blocks = sms * per_sm;
+  }
+  {
+    LaunchScope ls(KC_GREEDY, st);
+    void* args[] = {&p};
+    if (cudaLaunchCooperativeKernel((const void*)greedy_kernel, dim3(coop_blocks), dim3(512), args, 0, st) != cudaSuccess)
+      return SPINDLEKV_CUDA;
+  }
+  {
+    size_t smem = (size_t)(b.max_len + 2) * 4;
+    static bool attr_set = false;
+    if (!attr_set) {
+      if (cudaFuncSetAttribute(finalize_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess)
+        return SPINDLEKV_CUDA;
+      attr_set = true;
+    }
+    LaunchScope ls(KC_FINAL, st);
+    finalize_kernel<<<units, kFinalThreads, smem, st>>>(p);
+  }
+  return cudaGetLastError() == cudaSuccess ? SPINDLEKV_OK : SPINDLEKV_CUDA;
+}
+
+}  // namespace skv

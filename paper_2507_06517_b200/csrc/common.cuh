@@ -1,0 +1,82 @@
+// Shared device/host helpers of the SpindleKV reduction library (sm_100a).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "spindlekv.h"
+
+namespace skv {
+
+// ---- status block at the start of every workspace -------------------------------------------
+// word 0: device status, 1: greedy rounds used, 2: live tokens left, 3: unused,
+// words 8..: barrier and counters of the cooperative greedy kernel.
+constexpr int kHeaderBytes = 256;
+constexpr int kHdrStatus = 0;
+constexpr int kHdrRounds = 1;
+constexpr int kHdrLive = 2;
+constexpr int kHdrBarrier = 8;
+constexpr int kHdrLiveCnt0 = 9;   // two slots, alternated by round parity
+constexpr int kHdrLiveCnt1 = 10;
+
+// kernel classes for launch counting / timing
+enum KernelClass { KC_WINDOW = 0, KC_TOPK, KC_NORMS, KC_SIM, KC_DEGREE, KC_GREEDY, KC_FINAL, KC_GATHER, KC_COUNT };
+
+struct View {  // device-side copy of spindlekv_tensor
+  const void* ptr;
+  int64_t sl, ss, sh, st;
+};
+
+inline View make_view(const spindlekv_tensor& t) { return View{t.ptr, t.stride_layer, t.stride_seq, t.stride_head, t.stride_tok}; }
+
+struct Batch {  // device-side copy of spindlekv_batch
+  int n_layers, n_seqs, max_len, total_len;
+  const int32_t* cu;
+};
+
+inline Batch make_batch(const spindlekv_batch& b) { return Batch{b.n_layers, b.n_seqs, b.max_len, b.total_len, b.cu_seqlens}; }
+
+__device__ __forceinline__ int seq_len(const Batch& b, int s) { return b.cu ? (b.cu[s + 1] - b.cu[s]) : b.max_len; }
+__device__ __forceinline__ int tok_base(const Batch& b, int s) { return b.cu ? b.cu[s] : s * b.max_len; }
+
+// element offset of row 0 of (layer, seq, head)
+__device__ __forceinline__ int64_t unit_offset(const View& v, const Batch& b, int layer, int s, int h) {
+  int64_t off = (int64_t)layer * v.sl + (int64_t)h * v.sh;
+  off += b.cu ? (int64_t)b.cu[s] * v.st : (int64_t)s * v.ss;
+  return off;
+}
+
+__device__ __forceinline__ float to_f32(float x) { return x; }
+__device__ __forceinline__ float to_f32(__nv_bfloat16 x) { return __bfloat162float(x); }
+
+// 8 consecutive elements -> 8 floats (16-byte aligned source for bf16, 32-byte for fp32)
+__device__ __forceinline__ void load8(const float* p, float* out) {
+  float4 a = *reinterpret_cast<const float4*>(p);
+  float4 b = *reinterpret_cast<const float4*>(p + 4);
+  out[0] = a.x; out[1] = a.y; out[2] = a.z; out[3] = a.w;
+  out[4] = b.x; out[5] = b.y; out[6] = b.z; out[7] = b.w;
+}
+__device__ __forceinline__ void load8(const __nv_bfloat16* p, float* out) {
+  uint4 r = *reinterpret_cast<const uint4*>(p);
+  uint32_t w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    out[2 * i] = __uint_as_float(w[i] << 16);
+    out[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+  }
+}
+
+inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+__host__ __device__ inline int row_words_for(int max_len) { return 4 * ((max_len + 127) / 128); }
+
+// ---- launch bookkeeping (host) ---------------------------------------------------------------
+void note_launch(int kclass, cudaStream_t st, bool before);
+struct LaunchScope {
+  int kc; cudaStream_t st;
+  LaunchScope(int k, cudaStream_t s) : kc(k), st(s) { note_launch(kc, st, true); }
+  ~LaunchScope() { note_launch(kc, st, false); }
+};
+
+}  // namespace skv

@@ -1,0 +1,88 @@
+// Gather of kept tokens / CodeBook centres into the output cache (Eq. (7) second line, Eq. (11)):
+// 16-byte loads and stores, one row per group of head_dim*elem/16 threads, rows of a unit contiguous
+// in the destination.
+#include "common.cuh"
+
+namespace skv {
+
+struct CompactParams {
+  View src, dst;
+  Batch batch;
+  int n_heads;
+  const int32_t* idx;     // [layers][H][T]
+  const int32_t* cnt;     // [layers][B][H]
+  const float* divide_by; // optional [layers][H][T]
+  const int32_t* dst_cu;  // optional [B+1]
+};
+
+template <typename T, int D>
+__global__ void __launch_bounds__(256) compact_kernel(CompactParams p) {
+  constexpr int EPT = 16 / sizeof(T);       // elements per thread
+  constexpr int TPR = D / EPT;              // threads per row
+  constexpr int RPB = 256 / TPR;            // rows per block
+  const int unit = blockIdx.y;
+  const int h = unit % p.n_heads;
+  const int ls = unit / p.n_heads;
+  const int s = ls % p.batch.n_seqs;
+  const int layer = ls / p.batch.n_seqs;
+  const int n = p.cnt[(layer * p.batch.n_seqs + s) * p.n_heads + h];
+  const int64_t orow = ((int64_t)layer * p.n_heads + h) * p.batch.total_len + tok_base(p.batch, s);
+  const T* sbase = reinterpret_cast<const T*>(p.src.ptr) + unit_offset(p.src, p.batch, layer, s, h);
+  T* dbase = reinterpret_cast<T*>(const_cast<void*>(p.dst.ptr)) + (int64_t)layer * p.dst.sl + (int64_t)h * p.dst.sh;
+  if (p.dst_cu) dbase += (int64_t)p.dst_cu[s] * p.dst.st;
+  else if (p.batch.cu) dbase += (int64_t)p.batch.cu[s] * p.dst.st;
+  else dbase += (int64_t)s * p.dst.ss;
+  const int seg = threadIdx.x % TPR;
+  for (int r = blockIdx.x * RPB + threadIdx.x / TPR; r < n; r += gridDim.x * RPB) {
+    const int a = p.idx[orow + r];
+    uint4 v = *reinterpret_cast<const uint4*>(sbase + (int64_t)a * p.src.st + seg * EPT);
+    if (p.divide_by) {
+      const float m = p.divide_by[orow + a];
+      if (sizeof(T) == 4) {
+        float* f = reinterpret_cast<float*>(&v);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) f[i] = m > 0.f ? f[i] / m : 0.f;
+      } else {
+        uint32_t* w = reinterpret_cast<uint32_t*>(&v);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          float lo = __uint_as_float(w[i] << 16), hi = __uint_as_float(w[i] & 0xFFFF0000u);
+          lo = m > 0.f ? lo / m : 0.f;
+          hi = m > 0.f ? hi / m : 0.f;
+          __nv_bfloat162 pk = __floats2bfloat162_rn(lo, hi);
+          w[i] = *reinterpret_cast<uint32_t*>(&pk);
+        }
+      }
+    }
+    *reinterpret_cast<uint4*>(dbase + (int64_t)r * p.dst.st + seg * EPT) = v;
+  }
+}
+
+spindlekv_status compact_impl(const spindlekv_batch& b, int n_heads, int head_dim, const spindlekv_tensor& src,
+                              const int32_t* idx, const int32_t* cnt, const float* divide_by,
+                              const spindlekv_tensor& dst, const int32_t* dst_cu, cudaStream_t st) {
+  CompactParams p;
+  p.src = make_view(src);
+  p.dst = make_view(dst);
+  p.batch = make_batch(b);
+  p.n_heads = n_heads;
+  p.idx = idx;
+  p.cnt = cnt;
+  p.divide_by = divide_by;
+  p.dst_cu = dst_cu;
+  const int units = b.n_layers * b.n_seqs * n_heads;
+  if (units > 65535) return SPINDLEKV_UNSUPPORTED;
+  // enough blocks along x to cover the longest possible row list once at 16 rows per block
+  const int gx = ceil_div(b.max_len, 64);
+  dim3 grid(gx, units);
+  LaunchScope ls(KC_GATHER, st);
+  const bool bf = src.dtype == SPINDLEKV_BF16;
+  if (head_dim == 64) {
+    if (bf) compact_kernel<__nv_bfloat16, 64><<<grid, 256, 0, st>>>(p); else compact_kernel<float, 64><<<grid, 256, 0, st>>>(p);
+  } else {
+    if (bf) compact_kernel<__nv_bfloat16, 128><<<grid, 256, 0, st>>>(p); else compact_kernel<float, 128><<<grid, 256, 0, st>>>(p);
+  }
+  return cudaGetLastError() == cudaSuccess ? SPINDLEKV_OK : SPINDLEKV_CUDA;
+}
+
+}  // namespace skv

@@ -1,0 +1,164 @@
+"""CUDA path against the CPU checker, through the C ABI, element by element on seeded inputs.
+
+Bars: index sets, references, centres and counts bit-exact, except where the checker's own margin
+to the k-th score or to the similarity threshold is below 1e-4 relative (those positions are counted
+and the remaining structure must still be exactly what the checker derives from the GPU's decision);
+magnitudes 2e-6 relative; scores 1e-4 relative; kept rows exact copies; CodeBook vectors 1e-5 (fp32)
+or 1e-2 (bf16).
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import spindlekv_oracle as O
+from paper_2507_06517_b200 import synth
+
+from gpu_util import (check_codebook_unit, check_evict_unit, generate, make_config, stack_layers, tok_base,
+                      torch_dtype, unit_rows, value_tol)
+
+pytestmark = pytest.mark.gpu
+
+
+def _pass(wl, **kw):
+    from paper_2507_06517_b200.pipeline import SpindleKVPass
+    return SpindleKVPass(make_config(wl, **kw.pop("cfg", {})), wl.seq_lens, torch_dtype(wl), **kw)
+
+
+def run_and_check(wl, cfg_kw=None):
+    """Runs every layer of ``wl`` and checks every unit.  Returns margin counters."""
+    cfg_kw = cfg_kw or {}
+    host = generate(wl)
+    p = _pass(wl, cfg=cfg_kw, keep_adjacency=True)
+    ns, H = wl.n_shallow, wl.n_kv_heads
+    stats = {"topk_margin": 0, "adj_margin": 0, "units": 0}
+    deep = list(range(ns, wl.n_layers))
+    shallow = list(range(ns))
+    if deep:
+        K = stack_layers(wl, host, deep, "K")
+        V = stack_layers(wl, host, deep, "V")
+        Q = stack_layers(wl, host, deep, "Q")
+        p.evict(K, V, Q)
+        assert p.device_status()["evict"][0] == 0
+        scores = p.scores.cpu().numpy()
+        keep = p.keep_idx.cpu().numpy()
+        cnt = p.keep_cnt.cpu().numpy()
+        Kk = p.K_kept.float().cpu().numpy()
+        Vk = p.V_kept.float().cpu().numpy()
+        _, _, k_plan = O.plan_layers(wl.n_layers, ns, wl.seq_lens, wl.window, wl.beta,
+                                     reserve_ratio=wl.budget_frac, budget_tokens=wl.budget_tokens)
+        assert np.array_equal(k_plan, p.k_ctx_host)
+        for li, lam in enumerate(deep):
+            for s, l in enumerate(wl.seq_lens):
+                tb = tok_base(wl, s)
+                Ks = np.stack([unit_rows(wl, host[lam][0], s, j) for j in range(H)])
+                Vs = np.stack([unit_rows(wl, host[lam][1], s, j) for j in range(H)])
+                k_ctx = int(k_plan[lam, s])
+                stats["topk_margin"] += check_evict_unit(
+                    wl, host[lam][2][s], Ks, k_ctx, scores[li, :, tb:tb + l], keep[li, :, tb:tb + l], cnt[li, s],
+                    score_norm=cfg_kw.get("score_norm", 0))
+                for j in range(H):
+                    kg = keep[li, j, tb:tb + k_ctx + wl.window]
+                    got_k = unit_rows(wl, Kk[li], s, j)[: kg.size]
+                    got_v = unit_rows(wl, Vk[li], s, j)[: kg.size]
+                    assert np.array_equal(got_k, Ks[j][kg]) and np.array_equal(got_v, Vs[j][kg])
+                    stats["units"] += 1
+    if shallow:
+        for which, idx, theta in (("K", 0, wl.theta_k), ("V", 1, wl.theta_v)):
+            G = stack_layers(wl, host, shallow, which)
+            p.codebook(G, which)
+            st = p.device_status()["codebook"]
+            assert st[0] == 0 and st[1][1] == 0
+            out = {k: v.float().cpu().numpy() if k == "C" else v.cpu().numpy() for k, v in p.cb[which].items()}
+            adj = p.adj.cpu().numpy()
+            for li, lam in enumerate(shallow):
+                for s, l in enumerate(wl.seq_lens):
+                    tb = tok_base(wl, s)
+                    for j in range(H):
+                        unit = (li * wl.batch + s) * H + j
+                        gamma = unit_rows(wl, host[lam][idx], s, j)
+                        stats["adj_margin"] += check_codebook_unit(
+                            gamma, theta, adj[unit], out["mag"][li, j, tb:tb + l], out["ref"][li, j, tb:tb + l],
+                            out["centre_idx"][li, j, tb:tb + l], int(out["n_entries"][li, s, j]),
+                            unit_rows(wl, out["C"][li], s, j), value_tol(wl))
+                        stats["units"] += 1
+    return stats
+
+
+def test_tiny_fp32_config():
+    stats = run_and_check(synth.workload("C1"))
+    assert stats["units"] == 2 + 4
+
+
+def test_ragged_bf16_d128():
+    wl = synth.Workload("ragged", 2, 1, 8, 2, 128, "bf16", 32, (1000,), 40, (0.05, 0.3), 4, "recency",
+                        budget_tokens=200.0, seed=11)
+    run_and_check(wl)
+
+
+def test_packed_varlen_bf16_d64_pyramid():
+    wl = synth.Workload("packed", 3, 1, 4, 2, 64, "bf16", 16, (300, 777, 512), 24, (0.05, 0.3), 2, "recency",
+                        budget_frac=0.2, seed=12)
+    run_and_check(wl)
+
+
+def test_mha_fp32_d128_two_sequences():
+    wl = synth.Workload("mha", 2, 1, 2, 2, 128, "f32", 32, (200, 200), 10, 0.15, 2, "gauss",
+                        budget_tokens=100.0, seed=13)
+    run_and_check(wl)
+
+
+def test_plain_window_sum_extension():
+    wl = synth.Workload("rawsum", 1, 0, 4, 2, 64, "f32", 32, (333,), 8, 0.1, 2, "gauss", budget_tokens=80.0, seed=14)
+    run_and_check(wl, {"score_norm": 1})
+
+
+def test_keep_everything_and_minimum_budget():
+    wl = synth.Workload("all", 1, 0, 4, 2, 64, "f32", 32, (160,), 8, 0.1, 2, "gauss", budget_tokens=160.0, seed=15)
+    run_and_check(wl)  # r_c = 1: every context token kept
+    wl = wl.replace(budget_tokens=32 + 0.051 * 128)  # just above beta: k = floor(0.051 * 128) = 6
+    run_and_check(wl)
+
+
+def _single_layer_codebook(gamma_np, theta, dtype="f32"):
+    """Runs the CodeBook path on one hand-made ``[l, d]`` array; returns outputs as numpy."""
+    l, d = gamma_np.shape
+    wl = synth.Workload("hand", 1, 1, 1, 1, d, dtype, 1, (l,), 1, 0.1, 0, "gauss", budget_tokens=float(l),
+                        theta_k=theta, theta_v=theta)
+    p = _pass(wl, keep_adjacency=True)
+    G = torch.from_numpy(gamma_np.astype(np.float32)).to(torch_dtype(wl)).cuda().reshape(1, 1, 1, l, d)
+    p.codebook(G, "K")
+    assert p.device_status()["codebook"][0] == 0
+    o = p.cb["K"]
+    return (p.adj.cpu().numpy()[0], o["mag"].cpu().numpy()[0, 0], o["ref"].cpu().numpy()[0, 0],
+            o["centre_idx"].cpu().numpy()[0, 0], int(o["n_entries"].cpu().numpy()[0, 0, 0]),
+            o["C"].float().cpu().numpy()[0, 0, 0])
+
+
+def test_degenerate_thresholds_duplicates_and_zero_rows():
+    rng = np.random.default_rng(21)
+    g = rng.standard_normal((150, 64)).astype(np.float32)
+    adj, mag, ref, cen, n, C = _single_layer_codebook(g, 1.5)  # nobody similar: identity CodeBook
+    assert n == 150 and list(cen[:150]) == list(range(150)) and list(ref[:150]) == list(range(150))
+    adj, mag, ref, cen, n, C = _single_layer_codebook(g, -1.5)  # everybody similar: one entry, centre 0
+    assert n == 1 and cen[0] == 0 and np.all(ref[:150] == 0)
+    base = rng.standard_normal((50, 64)).astype(np.float32)
+    g = np.concatenate([base, 2.0 * base, base])  # exact copies (cosine 1) collapse
+    g[7] = 0.0  # a zero vector keeps an entry of its own
+    out = _single_layer_codebook(g, 0.999)
+    check_codebook_unit(g, 0.999, *out, 1e-5)
+    assert out[4] == 50 + 1 + 0  # 49 shared entries + the zero row + row 57/107 pair still shares one
+
+
+def test_all_scores_tie_goes_to_lowest_positions():
+    # zero queries: plain window sums tie everywhere -> the first k context tokens; with the division
+    # by (l - a) scores rise with position -> the last k
+    wl = synth.Workload("tie", 1, 0, 2, 1, 64, "f32", 16, (200,), 4, 0.1, 0, "gauss", budget_tokens=56.0, seed=16)
+    host = generate(wl)
+    l_c, k = 200 - 16, 40
+    for norm, want in ((1, list(range(k))), (0, list(range(l_c - k, l_c)))):
+        p = _pass(wl, cfg={"score_norm": norm})
+        K = stack_layers(wl, host, [0], "K")
+        Q = torch.zeros((1, 1, 2, 16, 64), dtype=torch.float32, device="cuda")
+        p.evict(K, K, Q)
+        keep = p.keep_idx.cpu().numpy()[0, 0]
+        assert list(keep[:k]) == want and list(keep[k:k + 16]) == list(range(l_c, 200))
