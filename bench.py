@@ -1,0 +1,365 @@
+#!/usr/bin/env python
+"""Throughput of the SpindleKV prefill reduction pass (all layers of one prompt) on B200.
+
+One "step" = the whole hot path over one synthetic prompt batch: plan, evict every deep layer
+(window scores, top-k, gather of K and V), build K and V CodeBooks for every shallow layer
+(magnitudes, similarity, greedy cover, numbering, gather of the centres).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload C3] [--impl reference]
+
+Prints one JSON line.  With N > 1 (under torchrun) every rank compresses its own prompt: the units
+of this pass are independent, so more GPUs means more prompts and no data-path collective.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2507_06517_b200 import synth
+
+METRIC = "prompt tokens compressed/s (all layers)"
+UNIT = "tokens/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the similarity kernel, from the ncu
+# capture summarised under profiles/ (None until one exists for the current kernel)
+SIMILARITY_TRAFFIC_BYTES_PER_UNIT = None
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="C3")
+    ap.add_argument("--impl", default="native", choices=["native", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    return ap.parse_args()
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {k: float(p[k]) for k in FALLBACK_PEAKS if k in p}, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+def workload_config(wl, extra=None):
+    cfg = {"workload": f"{wl.name}: B{wl.batch} x {wl.n_layers} layers ({wl.n_shallow} CodeBook + "
+                       f"{wl.n_layers - wl.n_shallow} evict), {wl.n_q_heads}/{wl.n_kv_heads} heads, d{wl.head_dim}, "
+                       f"N={'/'.join(map(str, wl.seq_lens)) if wl.packed else wl.max_len}, {wl.dtype}, w{wl.window}",
+           "tokens_per_step": wl.total_tokens,
+           "l2": "inputs larger than L2 (K and V of all layers are read once per step)"}
+    if extra:
+        cfg.update(extra)
+    return cfg
+
+
+# ---- CPU baseline: the checker, as it stands, on a bounded sample ------------------------------
+
+def oracle_sample_seconds(wl):
+    """Times the CPU checker on (shallow layer 0, head 0: K and V CodeBooks) and on one deep layer
+    (all heads) of sequence 0, and scales by unit counts to one whole step."""
+    from oracle import spindlekv_oracle as O
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([int(x.get("num_threads", 1)) for x in threadpool_info()] + [1])
+    except Exception:
+        cores = os.cpu_count() or 1
+    ns, nd = wl.n_shallow, wl.n_layers - wl.n_shallow
+    units = wl.batch * wl.n_kv_heads
+    total = 0.0
+    parts = []
+    scale_len = wl.total_tokens / (wl.seq_lens[0])  # sequences other than 0: scaled by length
+    if ns:
+        k, v = synth.unit_kv(wl, 0, 0, 0)
+        t0 = time.perf_counter()
+        O.codebook_shallow(k.astype(np.float64), wl.theta_k)
+        t1 = time.perf_counter()
+        O.codebook_shallow(v.astype(np.float64), wl.theta_v)
+        t2 = time.perf_counter()
+        # cost grows with the square of the length; other sequences are scaled accordingly
+        sq = sum(float(l) ** 2 for l in wl.seq_lens) / float(wl.seq_lens[0]) ** 2
+        total += ((t1 - t0) + (t2 - t1)) * ns * wl.n_kv_heads * sq
+        parts.append(f"layer 0 head 0 K+V CodeBooks ({t2 - t0:.1f} s)")
+    if nd:
+        lam = ns
+        ks = np.stack([synth.unit_kv(wl, lam, 0, j)[0] for j in range(wl.n_kv_heads)])
+        q = synth.window_queries(wl, lam, 0, list(ks))
+        _, _, kplan = O.plan_layers(wl.n_layers, ns, wl.seq_lens, wl.window, wl.beta,
+                                    reserve_ratio=wl.budget_frac, budget_tokens=wl.budget_tokens)
+        t0 = time.perf_counter()
+        res = O.evict_deep(q.astype(np.float64), ks.astype(np.float64), int(kplan[lam, 0]))
+        for j in range(wl.n_kv_heads):
+            O.gather_rows(ks[j], res["keep"][j])
+        t1 = time.perf_counter()
+        total += (t1 - t0) * nd * scale_len
+        parts.append(f"layer {lam} all heads eviction ({t1 - t0:.1f} s)")
+    return total, cores, "extrapolated by unit count from: " + "; ".join(parts)
+
+
+def run_reference(args, wl):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    times = []
+    sample = ""
+    cores = 1
+    for i in range(args.warmup + args.steps):
+        t, cores, sample = oracle_sample_seconds(wl)
+        if i >= args.warmup:
+            times.append(t)
+        if sum(times) > 0 and (time.perf_counter() - T_START) > 240:
+            break
+    sec = statistics.median(times)
+    val = wl.total_tokens / sec
+    line = {"metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": len(times),
+            "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic", "impl": "reference",
+            "config": workload_config(wl),
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# ---- clocks ---------------------------------------------------------------------------------------
+
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index: int):
+        self.rows = []
+        self.proc = None
+        try:
+            uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+            if not uuid.startswith("GPU-"):
+                uuid = "GPU-" + uuid
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", uuid, f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.perf_counter(), line.strip()))
+
+    def stop(self, t0, t1):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        sm, mx, reasons = [], [], set()
+        for t, line in self.rows:
+            if t < t0 or t > t1 + 0.2:
+                continue
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 6:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), parts[2:6]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ---- native arm -------------------------------------------------------------------------------------
+
+def host_inputs(wl):
+    """Pinned host tensors K, V [m, ...] and Q [deep layers, B, H_q, w, d] in the storage dtype."""
+    from concurrent.futures import ThreadPoolExecutor
+    dt = torch.float32 if wl.dtype == "f32" else torch.bfloat16
+    ns = wl.n_shallow
+
+    def one(lam):
+        K, V, Q = synth.layer_arrays(wl, lam, need_q=lam >= ns)
+        return (torch.from_numpy(K).to(dt), torch.from_numpy(V).to(dt), None if Q is None else torch.from_numpy(Q).to(dt))
+
+    with ThreadPoolExecutor(max_workers=min(16, os.cpu_count() or 1)) as ex:
+        layers = list(ex.map(one, range(wl.n_layers)))
+    K = torch.stack([x[0] for x in layers]).pin_memory()
+    V = torch.stack([x[1] for x in layers]).pin_memory()
+    Q = torch.stack([x[2] for x in layers[ns:]]).pin_memory() if wl.n_layers > ns else None
+    return K, V, Q
+
+
+def run_native(args, wl):
+    from paper_2507_06517_b200 import binding as B
+    from paper_2507_06517_b200.pipeline import SpindleKVPass
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the reduction pass has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    # every rank compresses its own prompt (different seed)
+    wl = wl.replace(seed=wl.seed + rank)
+    dev = torch.device("cuda", local_rank)
+    cfg = B.Config(n_layers=wl.n_layers, n_q_heads=wl.n_q_heads, n_kv_heads=wl.n_kv_heads, head_dim=wl.head_dim,
+                   window=wl.window, n_shallow=wl.n_shallow, beta=wl.beta, theta_k=wl.theta_k, theta_v=wl.theta_v,
+                   budget_tokens=wl.budget_tokens if wl.budget_tokens is not None else -1.0,
+                   reserve_ratio=wl.budget_frac if wl.budget_frac is not None else -1.0)
+    hK, hV, hQ = host_inputs(wl)
+    dtype = hK.dtype
+    p = SpindleKVPass(cfg, wl.seq_lens, dtype, device=dev)
+    dK = torch.empty_like(hK, device=dev)
+    dV = torch.empty_like(hV, device=dev)
+    dQ = torch.empty_like(hQ, device=dev) if hQ is not None else None
+
+    def upload():
+        dK.copy_(hK, non_blocking=True)
+        dV.copy_(hV, non_blocking=True)
+        if dQ is not None:
+            dQ.copy_(hQ, non_blocking=True)
+
+    # results read back by the end-to-end arm: index maps, counts, magnitudes, and the compacted rows
+    # that can hold data (kept rows up to the largest k + w; CodeBook rows in full)
+    max_keep = int(p.k_ctx_host[wl.n_shallow:].max()) + wl.window if p.n_deep else 0
+    outs = []
+    if p.n_deep:
+        outs += [p.keep_idx, p.keep_cnt]
+        if wl.packed:
+            outs += [p.K_kept, p.V_kept]
+        else:
+            outs += [p.K_kept[:, :, :, :max_keep], p.V_kept[:, :, :, :max_keep]]
+    if p.n_shallow:
+        for g in ("K", "V"):
+            outs += [p.cb[g]["ref"], p.cb[g]["mag"], p.cb[g]["n_entries"], p.cb[g]["C"]]
+    host_out = [torch.empty(o.shape, dtype=o.dtype, pin_memory=True) for o in outs]
+    h2d = sum(t.numel() * t.element_size() for t in (hK, hV) + ((hQ,) if hQ is not None else ()))
+    d2h = sum(t.numel() * t.element_size() for t in host_out)
+
+    def download():
+        for o, h in zip(outs, host_out):
+            h.copy_(o, non_blocking=True)
+
+    def barrier():
+        torch.cuda.synchronize(dev)
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    def timed(fn, steps):
+        barrier()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev0.record()
+        for _ in range(steps):
+            fn()
+        ev1.record()
+        barrier()
+        ms = ev0.elapsed_time(ev1)
+        if dist is not None:
+            t = torch.tensor([ms], device=dev, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms
+
+    upload()
+    step = lambda: p.run(dK, dV, dQ)
+    for _ in range(max(args.warmup, 3)):
+        step()
+    st = p.device_status()
+    for k, v in st.items():
+        if v[0] != 0:
+            raise RuntimeError(f"device status {v} in {k}")
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    B.spindlekv_launch_count(True)
+    t0 = time.perf_counter()
+    ms = timed(step, args.steps)
+    t1 = time.perf_counter()
+    launches = B.spindlekv_launch_count(True)
+    clocks = sampler.stop(t0, t1) if sampler else None
+
+    e2e = None
+    if not args.no_e2e:
+        def step_e2e():
+            upload()
+            p.run(dK, dV, dQ)
+            download()
+        step_e2e()
+        ms_e2e = timed(step_e2e, args.steps)
+        e2e = {"value": world * wl.total_tokens * args.steps / (ms_e2e * 1e-3), "unit": UNIT,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / args.steps}
+
+    # per-kernel times: one more pass with event pairs around every launch
+    B.spindlekv_timing_enable(True)
+    for _ in range(args.steps):
+        step()
+    torch.cuda.synchronize(dev)
+    kt = B.spindlekv_timing_read()
+    B.spindlekv_timing_enable(False)
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+    pk, pk_src = peaks()
+    total_ms = sum(v[0] for v in kt.values()) or 1.0
+    kernels = {k: {"ms_per_step": v[0] / args.steps, "launches_per_step": v[1] / args.steps,
+                   "share": v[0] / total_ms} for k, v in kt.items() if v[1]}
+    roof = None
+    if p.n_shallow and kt["similarity"][1]:
+        sim_ms, sim_n = kt["similarity"]
+        units_per_launch = 2 * wl.n_shallow * wl.n_kv_heads * wl.batch / (sim_n / args.steps)
+        flops_per_step = sum(float(l) * (l - 1) * wl.head_dim for l in wl.seq_lens) * 2 * wl.n_shallow * wl.n_kv_heads
+        achieved = flops_per_step * args.steps / (sim_ms * 1e-3) / 1e12
+        peak = pk["bf16_tflops_sustained"] if wl.dtype == "bf16" else pk["bf16_tflops_sustained"] / 32.0
+        traffic = None
+        if SIMILARITY_TRAFFIC_BYTES_PER_UNIT is not None:
+            traffic = SIMILARITY_TRAFFIC_BYTES_PER_UNIT * units_per_launch
+        roof = {"kernel": "similarity (Eq. 4, 9)", "bound": "tensor", "achieved": achieved, "peak": peak,
+                "unit": "TFLOP/s", "frac": achieved / peak, "traffic": traffic, "peak_source": pk_src,
+                "avg_launch_ms": sim_ms / sim_n, "algorithmic_flops_per_launch": flops_per_step * args.steps / sim_n}
+    line = {"metric": METRIC, "value": world * wl.total_tokens * args.steps / (ms * 1e-3), "unit": UNIT,
+            "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": wl.dtype,
+            "data": "synthetic", "config": workload_config(wl, {"parallelism": f"replicas x{world}"}),
+            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roof, "kernels": kernels,
+            "greedy_rounds": st.get("codebook", (0, [0]))[1][0]}
+    if not args.no_cpu_baseline and world == 1:
+        sec, cores, sample = oracle_sample_seconds(wl)
+        line["cpu_baseline"] = {"value": wl.total_tokens / sec, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                "sample": sample}
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+T_START = time.perf_counter()
+
+if __name__ == "__main__":
+    a = parse_args()
+    w = synth.workload(a.workload)
+    if a.impl == "reference":
+        run_reference(a, w)
+    else:
+        run_native(a, w)
