@@ -10,8 +10,8 @@ ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libspindlekv.so")
 
-SOURCES = ["api.cu", "evict.cu", "codebook.cu", "compact.cu"]
-HEADERS = ["common.cuh", "simt_tile.cuh"]
+SOURCES = ["api.cu", "evict.cu", "codebook.cu", "compact.cu", "sim_tc.cu"]
+HEADERS = ["common.cuh", "simt_tile.cuh", "sm100_ptx.cuh"]
 
 
 def _nvcc() -> str:

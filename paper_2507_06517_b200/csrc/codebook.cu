@@ -22,6 +22,7 @@ struct CodebookParams {
   int n_kv_heads, n_units, row_words;
   float theta;
   float* mag;            // [layers][H][T]
+  float* rinv;           // [units][row_words*32]: 1/|gamma|, 0 for zero vectors and beyond the sequence
   uint32_t* adj;         // [units][max_len][row_words]
   int32_t* deg;          // [units][max_len]
   unsigned long long* key;  // [units][max_len]
@@ -67,7 +68,11 @@ __global__ void __launch_bounds__(256) norms_kernel(CodebookParams p) {
   }
 #pragma unroll
   for (int o = LPR / 2; o >= 1; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-  if (row < l && seg == 0) p.mag[cb_out_row(p, layer, s, j) + row] = sqrtf(ss);
+  if (seg == 0) {
+    const float m = sqrtf(ss);
+    if (row < l) p.mag[cb_out_row(p, layer, s, j) + row] = m;
+    if (row < p.row_words * 32) p.rinv[(int64_t)blockIdx.y * p.row_words * 32 + row] = (row < l && m > 0.f) ? 1.0f / m : 0.f;
+  }
 }
 
 // ---- Eq. (4)(9) on CUDA cores: 64x64 tiles, decision dot > theta * (|a| * |b|) ------------------
@@ -374,7 +379,7 @@ __global__ void __launch_bounds__(kFinalThreads) finalize_kernel(CodebookParams 
 // ---- host side ----------------------------------------------------------------------------------
 
 struct CodebookLayout {
-  size_t adj, deg, key, m1, live0, live1, owner, pickdeg, rank, total;
+  size_t rinv, adj, deg, key, m1, live0, live1, owner, pickdeg, rank, total;
 };
 
 static CodebookLayout codebook_layout(const spindlekv_config& cfg, const spindlekv_batch& b, bool adj_in_ws) {
@@ -391,6 +396,7 @@ static CodebookLayout codebook_layout(const spindlekv_config& cfg, const spindle
   L.owner = take(units * ML * 4);
   L.pickdeg = take(units * ML * 4);
   L.rank = take(units * ML * 4);
+  L.rinv = take(units * RW * 32 * 4);
   L.adj = off;
   if (adj_in_ws) take(units * ML * RW * 4);
   L.total = off;
@@ -401,10 +407,19 @@ size_t codebook_workspace_bytes(const spindlekv_config& cfg, const spindlekv_bat
   return codebook_layout(cfg, b, true).total;
 }
 
+bool sim_tc_available();
+spindlekv_status launch_sim_tc(const spindlekv_tensor& Gamma, const spindlekv_batch& b, int n_kv_heads, int head_dim,
+                               float theta, const float* rinv, uint32_t* adj, uint32_t* hdr, cudaStream_t st);
+
 template <typename T, int D>
-static void launch_norms_sim(const CodebookParams& p, const spindlekv_batch& b, cudaStream_t st) {
+static void launch_norms(const CodebookParams& p, cudaStream_t st) {
   constexpr int RPB = 256 / (D / 8);
-  { LaunchScope ls(KC_NORMS, st); norms_kernel<T, D><<<dim3(ceil_div(b.max_len, RPB), p.n_units), 256, 0, st>>>(p); }
+  LaunchScope ls(KC_NORMS, st);
+  norms_kernel<T, D><<<dim3(ceil_div(p.row_words * 32, RPB), p.n_units), 256, 0, st>>>(p);
+}
+
+template <typename T, int D>
+static void launch_sim_simt(const CodebookParams& p, const spindlekv_batch& b, cudaStream_t st) {
   int ct = ceil_div(p.row_words * 32, kTile), rt = ceil_div(b.max_len, kTile);
   { LaunchScope ls(KC_SIM, st); sim_simt_kernel<T, D><<<dim3(ct, rt, p.n_units), 256, 0, st>>>(p); }
 }
@@ -428,6 +443,7 @@ spindlekv_status codebook_shallow_impl(const spindlekv_config& cfg, const spindl
   p.row_words = row_words_for(b.max_len);
   p.theta = theta;
   p.mag = mag;
+  p.rinv = reinterpret_cast<float*>(w + L.rinv);
   p.adj = adj_in_ws ? reinterpret_cast<uint32_t*>(w + L.adj) : adj_bits;
   p.deg = reinterpret_cast<int32_t*>(w + L.deg);
   p.key = reinterpret_cast<unsigned long long*>(w + L.key);
@@ -445,9 +461,18 @@ spindlekv_status codebook_shallow_impl(const spindlekv_config& cfg, const spindl
   if (cudaMemsetAsync(p.pickdeg, 0xFF, (size_t)units * b.max_len * 4, st) != cudaSuccess) return SPINDLEKV_CUDA;
   const bool bf = Gamma.dtype == SPINDLEKV_BF16;
   if (cfg.head_dim == 64) {
-    if (bf) launch_norms_sim<__nv_bfloat16, 64>(p, b, st); else launch_norms_sim<float, 64>(p, b, st);
+    if (bf) launch_norms<__nv_bfloat16, 64>(p, st); else launch_norms<float, 64>(p, st);
   } else {
-    if (bf) launch_norms_sim<__nv_bfloat16, 128>(p, b, st); else launch_norms_sim<float, 128>(p, b, st);
+    if (bf) launch_norms<__nv_bfloat16, 128>(p, st); else launch_norms<float, 128>(p, st);
+  }
+  if (bf && sim_tc_available()) {
+    // bf16: tensor-core similarity (TMA + tcgen05)
+    spindlekv_status rs = launch_sim_tc(Gamma, b, cfg.n_kv_heads, cfg.head_dim, theta, p.rinv, p.adj, p.hdr, st);
+    if (rs != SPINDLEKV_OK) return rs;
+  } else if (cfg.head_dim == 64) {
+    if (bf) launch_sim_simt<__nv_bfloat16, 64>(p, b, st); else launch_sim_simt<float, 64>(p, b, st);
+  } else {
+    if (bf) launch_sim_simt<__nv_bfloat16, 128>(p, b, st); else launch_sim_simt<float, 128>(p, b, st);
   }
   // cooperative launch: as many blocks as can be resident at once
   static int coop_blocks = 0;
