@@ -45,6 +45,8 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="C3")
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
+    ap.add_argument("--layers", type=int, default=None, help="override the layer count (profiling on a small case)")
+    ap.add_argument("--shallow", type=int, default=None, help="override the number of CodeBook layers")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     return ap.parse_args()
@@ -359,6 +361,9 @@ T_START = time.perf_counter()
 if __name__ == "__main__":
     a = parse_args()
     w = synth.workload(a.workload)
+    if a.layers is not None:
+        w = w.replace(n_layers=a.layers, n_shallow=a.shallow if a.shallow is not None else a.layers // 2,
+                      name=f"{w.name}[{a.layers} layers]")
     if a.impl == "reference":
         run_reference(a, w)
     else:

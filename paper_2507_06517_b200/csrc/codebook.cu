@@ -32,6 +32,8 @@ struct CodebookParams {
   int32_t* owner;        // [units][max_len]
   int32_t* pickdeg;      // [units][max_len], -1 = not a centre
   int32_t* rank;         // [units][max_len] entry number of a centre
+  int32_t* ell;          // [units][max_len][kEll] neighbour lists of rows with few neighbours
+  int32_t* ell_cnt;      // [units][max_len] list length, -1: use the bit row
   uint32_t* hdr;
   int32_t* ref;          // [layers][H][T]
   int32_t* centre_idx;   // [layers][H][T]
@@ -161,6 +163,67 @@ __device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long v)
   return v;
 }
 
+// ---- neighbour lists ------------------------------------------------------------------------------
+// One pass over the bit matrix: initial degrees (Eq. (10)), keys, and for every row with at most
+// kEll neighbours (itself not counted) the ascending list of those neighbours.  Rows with more
+// neighbours keep using their bit row.  One warp per row, 16-byte loads.
+constexpr int kEll = 32;
+
+__global__ void __launch_bounds__(256) extract_kernel(CodebookParams p) {
+  const int lane = threadIdx.x & 31;
+  const int64_t gwarp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int ML = p.batch.max_len, RW = p.row_words, RW4 = RW >> 2;
+  if (gwarp >= (int64_t)p.n_units * ML) return;
+  const int unit = (int)(gwarp / ML), u = (int)(gwarp % ML);
+  int layer, s, j;
+  cb_decode(p, unit, layer, s, j);
+  if (u >= seq_len(p.batch, s)) return;
+  const uint4* row4 = reinterpret_cast<const uint4*>(p.adj + gwarp * RW);
+  int cnt = 0;
+  for (int w4 = lane; w4 < RW4; w4 += 32) {
+    uint4 a = row4[w4];
+    cnt += __popc(a.x) + __popc(a.y) + __popc(a.z) + __popc(a.w);
+  }
+#pragma unroll
+  for (int o = 16; o >= 1; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+  if (lane == 0) {
+    p.deg[gwarp] = cnt;
+    p.key[gwarp] = ((unsigned long long)(uint32_t)cnt << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)u);
+    p.ell_cnt[gwarp] = cnt - 1 <= kEll ? cnt - 1 : -1;
+  }
+  if (cnt - 1 > kEll) return;
+  int32_t* ell = p.ell + gwarp * kEll;
+  int base = 0;
+  for (int w0 = 0; w0 < RW4; w0 += 32) {
+    const int w4 = w0 + lane;
+    uint32_t wd[4] = {0, 0, 0, 0};
+    if (w4 < RW4) {
+      uint4 a = row4[w4];
+      wd[0] = a.x; wd[1] = a.y; wd[2] = a.z; wd[3] = a.w;
+      if ((u >> 7) == w4) wd[(u >> 5) & 3] &= ~(1u << (u & 31));  // the token itself is not listed
+    }
+    const int c = __popc(wd[0]) + __popc(wd[1]) + __popc(wd[2]) + __popc(wd[3]);
+    int inc = c;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      int n = __shfl_up_sync(0xffffffffu, inc, o);
+      if (lane >= o) inc += n;
+    }
+    int pos = base + inc - c;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      uint32_t m = wd[k];
+      while (m) {
+        int b = __ffs(m) - 1;
+        m &= m - 1;
+        ell[pos++] = w4 * 128 + k * 32 + b;
+      }
+    }
+    base += __shfl_sync(0xffffffffu, inc, 31);
+  }
+}
+
+// ---- greedy cover, cooperative kernel over all units of the call --------------------------------
 __global__ void __launch_bounds__(512) greedy_kernel(CodebookParams p) {
   const int lane = threadIdx.x & 31;
   const int warps_per_block = blockDim.x >> 5;
@@ -168,11 +231,11 @@ __global__ void __launch_bounds__(512) greedy_kernel(CodebookParams p) {
   const int64_t nwarps = (int64_t)gridDim.x * warps_per_block;
   const int64_t gthread = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   const int64_t nthreads = (int64_t)gridDim.x * blockDim.x;
-  const int ML = p.batch.max_len, RW = p.row_words;
+  const int ML = p.batch.max_len, RW = p.row_words, RW4 = RW >> 2;
   const int64_t n_rows = (int64_t)p.n_units * ML;
   uint32_t target = 0;
 
-  // all tokens start live
+  // all tokens start live (both copies of the mask)
   for (int64_t i = gthread; i < (int64_t)p.n_units * RW; i += nthreads) {
     int unit = (int)(i / RW), w = (int)(i % RW);
     int layer, s, j;
@@ -182,6 +245,7 @@ __global__ void __launch_bounds__(512) greedy_kernel(CodebookParams p) {
     if (w * 32 + 32 <= l) m = 0xFFFFFFFFu;
     else if (w * 32 < l) m = (1u << (l - w * 32)) - 1u;
     p.live0[i] = m;
+    p.live1[i] = m;
   }
   if (!grid_barrier(p.hdr, target)) return;
 
@@ -191,49 +255,79 @@ __global__ void __launch_bounds__(512) greedy_kernel(CodebookParams p) {
     uint32_t* next = (round & 1) ? p.live0 : p.live1;
     const int slot = (round & 1) ? kHdrLiveCnt1 : kHdrLiveCnt0;
     const int other = (round & 1) ? kHdrLiveCnt0 : kHdrLiveCnt1;
-    // phase 1: live degrees (Eq. (10)) and keys; `next` starts as a copy of `live`
-    for (int64_t i = gthread; i < (int64_t)p.n_units * RW; i += nthreads) next[i] = live[i];
-    if (gthread == 0) p.hdr[other] = 0;
-    int my_live = 0;
-    for (int64_t idx = gwarp; idx < n_rows; idx += nwarps) {
-      int unit = (int)(idx / ML), u = (int)(idx % ML);
-      const uint32_t* lv = live + (int64_t)unit * RW;
-      bool alive = (lv[u >> 5] >> (u & 31)) & 1u;  // bits beyond the sequence length are never set
-      if (!alive) {
-        if (lane == 0) p.key[idx] = 0ull;
-        continue;
-      }
-      const uint32_t* row = p.adj + idx * RW;
-      int cnt = 0;
-      for (int w = lane; w < RW; w += 32) cnt += __popc(row[w] & lv[w]);
+    if (round > 0) {
+      // phase 1: live degrees (Eq. (10)) and keys; `next` becomes a copy of `live`.
+      // (Round 0 uses the degrees and keys written with the neighbour lists.)
+      for (int64_t i = gthread; i < (int64_t)p.n_units * RW; i += nthreads) next[i] = live[i];
+      if (gthread == 0) p.hdr[other] = 0;
+      int my_live = 0;
+      for (int64_t idx = gwarp; idx < n_rows; idx += nwarps) {
+        int unit = (int)(idx / ML), u = (int)(idx - (int64_t)unit * ML);
+        const uint32_t* lv = live + (int64_t)unit * RW;
+        bool alive = (lv[u >> 5] >> (u & 31)) & 1u;  // bits beyond the sequence length are never set
+        if (!alive) {
+          if (lane == 0) p.key[idx] = 0ull;
+          continue;
+        }
+        const int ec = p.ell_cnt[idx];
+        int cnt;
+        if (ec >= 0) {
+          bool on = false;
+          if (lane < ec) {
+            int v = p.ell[idx * kEll + lane];
+            on = (lv[v >> 5] >> (v & 31)) & 1u;
+          }
+          cnt = 1 + __popc(__ballot_sync(0xffffffffu, on));
+        } else {
+          const uint4* row4 = reinterpret_cast<const uint4*>(p.adj + idx * RW);
+          const uint4* lv4 = reinterpret_cast<const uint4*>(lv);
+          cnt = 0;
+          for (int w4 = lane; w4 < RW4; w4 += 32) {
+            uint4 a = row4[w4], b = lv4[w4];
+            cnt += __popc(a.x & b.x) + __popc(a.y & b.y) + __popc(a.z & b.z) + __popc(a.w & b.w);
+          }
 #pragma unroll
-      for (int o = 16; o >= 1; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
-      if (lane == 0) {
-        p.deg[idx] = cnt;
-        p.key[idx] = ((unsigned long long)(uint32_t)cnt << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)u);
-        ++my_live;
+          for (int o = 16; o >= 1; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+        }
+        if (lane == 0) {
+          p.deg[idx] = cnt;
+          p.key[idx] = ((unsigned long long)(uint32_t)cnt << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)u);
+          ++my_live;
+        }
       }
+      if (lane == 0 && my_live) atomicAdd(&p.hdr[slot], (uint32_t)my_live);
+      if (!grid_barrier(p.hdr, target)) return;
+      const uint32_t total_live = *reinterpret_cast<volatile uint32_t*>(&p.hdr[slot]);
+      if (total_live == 0) break;
     }
-    if (lane == 0 && my_live) atomicAdd(&p.hdr[slot], (uint32_t)my_live);
-    if (!grid_barrier(p.hdr, target)) return;
-    const uint32_t total_live = *reinterpret_cast<volatile uint32_t*>(&p.hdr[slot]);
-    if (total_live == 0) break;
 
     // phase 2: largest key in each closed live neighbourhood
     for (int64_t idx = gwarp; idx < n_rows; idx += nwarps) {
-      int unit = (int)(idx / ML), u = (int)(idx % ML);
+      int unit = (int)(idx / ML), u = (int)(idx - (int64_t)unit * ML);
       const uint32_t* lv = live + (int64_t)unit * RW;
       if (!((lv[u >> 5] >> (u & 31)) & 1u)) continue;
-      const uint32_t* row = p.adj + idx * RW;
       const unsigned long long* key = p.key + (int64_t)unit * ML;
+      const int ec = p.ell_cnt[idx];
       unsigned long long best = 0ull;
-      for (int w = lane; w < RW; w += 32) {
-        uint32_t m = row[w] & lv[w];
-        while (m) {
-          int b = __ffs(m) - 1;
-          m &= m - 1;
-          unsigned long long kv = key[w * 32 + b];
-          best = kv > best ? kv : best;
+      if (ec >= 0) {
+        if (lane < ec) {
+          int v = p.ell[idx * kEll + lane];
+          if ((lv[v >> 5] >> (v & 31)) & 1u) best = key[v];
+        }
+        if (lane == 0) {  // the token itself belongs to its closed neighbourhood
+          unsigned long long own = key[u];
+          best = own > best ? own : best;
+        }
+      } else {
+        const uint32_t* row = p.adj + idx * RW;
+        for (int w = lane; w < RW; w += 32) {
+          uint32_t m = row[w] & lv[w];
+          while (m) {
+            int b = __ffs(m) - 1;
+            m &= m - 1;
+            unsigned long long kv = key[w * 32 + b];
+            best = kv > best ? kv : best;
+          }
         }
       }
       best = warp_max_u64(best);
@@ -244,33 +338,53 @@ __global__ void __launch_bounds__(512) greedy_kernel(CodebookParams p) {
     // phase 3: a node that is the maximum of every neighbour's neighbourhood is a centre (Eq. (11));
     // its live neighbours take it as owner (Eq. (12)) and leave the graph (Eq. (13))
     for (int64_t idx = gwarp; idx < n_rows; idx += nwarps) {
-      int unit = (int)(idx / ML), u = (int)(idx % ML);
+      int unit = (int)(idx / ML), u = (int)(idx - (int64_t)unit * ML);
       const uint32_t* lv = live + (int64_t)unit * RW;
       if (!((lv[u >> 5] >> (u & 31)) & 1u)) continue;
       const unsigned long long mykey = p.key[idx];
       if (p.m1[idx] != mykey) continue;
-      const uint32_t* row = p.adj + idx * RW;
       const unsigned long long* m1 = p.m1 + (int64_t)unit * ML;
-      bool ok = true;
-      for (int w = lane; w < RW; w += 32) {
-        uint32_t m = row[w] & lv[w];
-        while (m) {
-          int b = __ffs(m) - 1;
-          m &= m - 1;
-          if (m1[w * 32 + b] != mykey) ok = false;
-        }
-      }
-      if (!__all_sync(0xffffffffu, ok)) continue;
-      if (lane == 0) p.pickdeg[idx] = p.deg[idx];
       int32_t* owner = p.owner + (int64_t)unit * ML;
       uint32_t* nx = next + (int64_t)unit * RW;
-      for (int w = lane; w < RW; w += 32) {
-        uint32_t m = row[w] & lv[w];
-        if (m) atomicAnd(&nx[w], ~m);
-        while (m) {
-          int b = __ffs(m) - 1;
-          m &= m - 1;
-          owner[w * 32 + b] = u;
+      const int ec = p.ell_cnt[idx];
+      if (ec >= 0) {
+        int v = -1;
+        if (lane < ec) {
+          v = p.ell[idx * kEll + lane];
+          if (!((lv[v >> 5] >> (v & 31)) & 1u)) v = -1;
+        }
+        bool ok = v < 0 || m1[v] == mykey;
+        if (!__all_sync(0xffffffffu, ok)) continue;
+        if (v >= 0) {
+          owner[v] = u;
+          atomicAnd(&nx[v >> 5], ~(1u << (v & 31)));
+        }
+        if (lane == 0) {
+          p.pickdeg[idx] = p.deg[idx];
+          owner[u] = u;
+          atomicAnd(&nx[u >> 5], ~(1u << (u & 31)));
+        }
+      } else {
+        const uint32_t* row = p.adj + idx * RW;
+        bool ok = true;
+        for (int w = lane; w < RW; w += 32) {
+          uint32_t m = row[w] & lv[w];
+          while (m) {
+            int b = __ffs(m) - 1;
+            m &= m - 1;
+            if (m1[w * 32 + b] != mykey) ok = false;
+          }
+        }
+        if (!__all_sync(0xffffffffu, ok)) continue;
+        if (lane == 0) p.pickdeg[idx] = p.deg[idx];
+        for (int w = lane; w < RW; w += 32) {
+          uint32_t m = row[w] & lv[w];
+          if (m) atomicAnd(&nx[w], ~m);
+          while (m) {
+            int b = __ffs(m) - 1;
+            m &= m - 1;
+            owner[w * 32 + b] = u;
+          }
         }
       }
     }
@@ -278,7 +392,7 @@ __global__ void __launch_bounds__(512) greedy_kernel(CodebookParams p) {
   }
   if (gthread == 0) {
     p.hdr[kHdrRounds] = (uint32_t)round;
-    uint32_t left = *reinterpret_cast<volatile uint32_t*>(&p.hdr[(round & 1) ? kHdrLiveCnt1 : kHdrLiveCnt0]);
+    uint32_t left = round == 0 ? 0u : *reinterpret_cast<volatile uint32_t*>(&p.hdr[(round & 1) ? kHdrLiveCnt1 : kHdrLiveCnt0]);
     p.hdr[kHdrLive] = round > ML ? 1u : left;
     if (round > ML) atomicExch(&p.hdr[kHdrStatus], (uint32_t)SPINDLEKV_TIMEOUT);
   }
@@ -379,7 +493,7 @@ __global__ void __launch_bounds__(kFinalThreads) finalize_kernel(CodebookParams 
 // ---- host side ----------------------------------------------------------------------------------
 
 struct CodebookLayout {
-  size_t rinv, adj, deg, key, m1, live0, live1, owner, pickdeg, rank, total;
+  size_t rinv, ell, ell_cnt, adj, deg, key, m1, live0, live1, owner, pickdeg, rank, total;
 };
 
 static CodebookLayout codebook_layout(const spindlekv_config& cfg, const spindlekv_batch& b, bool adj_in_ws) {
@@ -397,6 +511,8 @@ static CodebookLayout codebook_layout(const spindlekv_config& cfg, const spindle
   L.pickdeg = take(units * ML * 4);
   L.rank = take(units * ML * 4);
   L.rinv = take(units * RW * 32 * 4);
+  L.ell = take(units * ML * 32 * 4);
+  L.ell_cnt = take(units * ML * 4);
   L.adj = off;
   if (adj_in_ws) take(units * ML * RW * 4);
   L.total = off;
@@ -453,6 +569,8 @@ spindlekv_status codebook_shallow_impl(const spindlekv_config& cfg, const spindl
   p.owner = reinterpret_cast<int32_t*>(w + L.owner);
   p.pickdeg = reinterpret_cast<int32_t*>(w + L.pickdeg);
   p.rank = reinterpret_cast<int32_t*>(w + L.rank);
+  p.ell = reinterpret_cast<int32_t*>(w + L.ell);
+  p.ell_cnt = reinterpret_cast<int32_t*>(w + L.ell_cnt);
   p.hdr = reinterpret_cast<uint32_t*>(w);
   p.ref = ref;
   p.centre_idx = centre_idx;
@@ -473,6 +591,10 @@ spindlekv_status codebook_shallow_impl(const spindlekv_config& cfg, const spindl
     if (bf) launch_sim_simt<__nv_bfloat16, 64>(p, b, st); else launch_sim_simt<float, 64>(p, b, st);
   } else {
     if (bf) launch_sim_simt<__nv_bfloat16, 128>(p, b, st); else launch_sim_simt<float, 128>(p, b, st);
+  }
+  {
+    LaunchScope ls(KC_DEGREE, st);
+    extract_kernel<<<(unsigned)(((size_t)units * b.max_len * 32 + 255) / 256), 256, 0, st>>>(p);
   }
   // cooperative launch: as many blocks as can be resident at once
   static int coop_blocks = 0;

@@ -107,6 +107,17 @@ def test_mha_fp32_d128_two_sequences():
     run_and_check(wl)
 
 
+def test_dense_and_sparse_rows_mixed():
+    # three big clusters (rows with far more than 32 neighbours use their bit row) next to
+    # noisy tokens with few or no neighbours (rows that use neighbour lists)
+    wl = synth.Workload("dense", 1, 1, 2, 2, 64, "bf16", 8, (700,), 3, (0.02, 0.6), 2, "gauss",
+                        budget_tokens=700.0, seed=17)
+    run_and_check(wl)
+    wl = synth.Workload("dense32", 1, 1, 2, 2, 128, "f32", 8, (520,), 12, (0.05, 0.2), 2, "gauss",
+                        budget_tokens=520.0, seed=18)
+    run_and_check(wl)
+
+
 def test_plain_window_sum_extension():
     wl = synth.Workload("rawsum", 1, 0, 4, 2, 64, "f32", 32, (333,), 8, 0.1, 2, "gauss", budget_tokens=80.0, seed=14)
     run_and_check(wl, {"score_norm": 1})
