@@ -1,15 +1,19 @@
 // Thresholded cosine similarity (Eq. (4)(9)) on the 5th-generation tensor cores, bf16 inputs.
 //
-// One CTA owns a block of 128 token rows of one (layer, sequence, head) unit: the block is loaded
-// once by TMA and stays in shared memory as operand A; tiles of 256 token rows stream through a
-// two-stage ring as operand B.  One elected thread issues tcgen05.mma (128 x 256 x 16, fp32
-// accumulation in TMEM) for the raw bf16 dot products; eight epilogue warps read the accumulators
-// back with tcgen05.ld, apply the fp32 inverse norms, compare with theta and pack one bit per pair,
-// while the tensor cores work on the other TMEM stage.  Nothing but bits leaves the SM:
-// N*N/8 bytes per unit.
+// The adjacency is symmetric, so only pairs (a, b) with a < b are computed and each decision is
+// written twice: into row a and, mirrored, into row b.
 //
-// Decision per pair (symmetric in a and b by construction of the arithmetic):
-//     dot(a,b) * (rinv_a * rinv_b) > theta,   rinv = 1/|gamma| (0 for a zero vector).
+// One CTA owns a block of 128 token rows of one (layer, sequence, head) unit: the block is loaded
+// once by TMA and stays in shared memory as operand A; tiles of 256 token rows, from the tile that
+// holds the diagonal onwards, stream through a two-stage ring as operand B.  One elected thread
+// issues tcgen05.mma (128 x 256 x 16, fp32 accumulation in TMEM) for the raw bf16 dot products.
+// Eight epilogue warps read the accumulators back with tcgen05.ld while the tensor cores work on
+// the other TMEM stage.  A thread owns one row a; per pair it evaluates
+//     x = fma(-dot, rinv_b, theta * |a|)        (rinv = 1/|gamma|, 0 for a zero vector)
+// whose sign bit is the decision dot/(|a||b|) > theta, and shifts that bit into a 32-bit word.
+// The word goes to row a as is; a 32x32 bit transpose across the warp turns the 32 words of a
+// sub-block into the words of the mirrored rows, which are staged in shared memory and written
+// 16 bytes per row.  Nothing but bits leaves the SM: N*N/8 bytes per unit.
 #include "common.cuh"
 #include "sm100_ptx.cuh"
 
@@ -27,7 +31,10 @@ struct SimTcParams {
 constexpr int kBM = 128;          // rows of the resident block (UMMA M)
 constexpr int kBN = 256;          // rows of a streamed tile (UMMA N)
 constexpr int kStages = 2;
-constexpr int kEpiWarps = 8;
+constexpr int kEpiWarps = 16;
+constexpr int kColsPerWarp = kBN / (kEpiWarps / 4);   // tile columns handled by one epilogue warp
+constexpr int kChunks = kColsPerWarp / 32;
+constexpr int kEpiThreads = 32 * kEpiWarps;
 constexpr int kSimThreads = 32 * (2 + kEpiWarps);
 
 template <int D>
@@ -35,10 +42,48 @@ struct SimSmem {
   static constexpr int KH = D / 64;                  // 64-element (128-byte) swizzle atoms along head_dim
   static constexpr int A_BYTES = KH * kBM * 128;
   static constexpr int B_BYTES = KH * kBN * 128;
-  static constexpr int USED = A_BYTES + kStages * B_BYTES + 256 /*barriers*/ + 1024 /*alignment slack*/;
+  static constexpr int RC_BYTES = 2 * kBN * 4;       // inverse norms of the tile's 256 tokens, two slots
+  static constexpr int T_BYTES = 2 * 4 * kBN * 4;    // mirrored words [slot][row quarter][tile column]
+  static constexpr int USED = A_BYTES + kStages * B_BYTES + RC_BYTES + T_BYTES + 256 /*barriers*/ + 1024 /*alignment*/;
   // at least 120 KB so that two blocks never share an SM: each block allocates all 512 TMEM columns
   static constexpr int TOTAL = USED > 120 * 1024 ? USED : 120 * 1024;
 };
+
+// 32x32 bit transpose across a warp: in: lane r holds bits (r, c) at bit c; out: lane c holds bit r
+__device__ __forceinline__ uint32_t warp_transpose32(uint32_t x, int lane) {
+  uint32_t m = 0x0000FFFFu;
+#pragma unroll
+  for (int j = 16; j >= 1; j >>= 1) {
+    const uint32_t y = __shfl_xor_sync(0xffffffffu, x, j);
+    const bool hi = (lane & j) != 0;
+    const uint32_t keep = hi ? ~m : m;
+    const uint32_t sh = hi ? (y >> j) : (y << j);
+    x = (x & keep) | (sh & ~keep);
+    m ^= m << (j >> 1);
+  }
+  return x;
+}
+
+// four transposes at once: the shuffles of one stage are independent of each other
+__device__ __forceinline__ void warp_transpose32x4(uint32_t (&x)[4], int lane) {
+  uint32_t m = 0x0000FFFFu;
+#pragma unroll
+  for (int j = 16; j >= 1; j >>= 1) {
+    const bool hi = (lane & j) != 0;
+    const uint32_t keep = hi ? ~m : m;
+    uint32_t y[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) y[i] = __shfl_xor_sync(0xffffffffu, x[i], j);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const uint32_t sh = hi ? (y[i] >> j) : (y[i] << j);
+      x[i] = (x[i] & keep) | (sh & ~keep);
+    }
+    m ^= m << (j >> 1);
+  }
+}
+
+__device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory"); }
 
 template <int D>
 __global__ void __launch_bounds__(kSimThreads, 1) sim_tc_kernel(const __grid_constant__ CUtensorMap tmap, SimTcParams p) {
@@ -52,12 +97,15 @@ __global__ void __launch_bounds__(kSimThreads, 1) sim_tc_kernel(const __grid_con
   const int row0 = blockIdx.x * kBM;
   if (row0 >= l) return;
   const int n_tiles = (p.row_words * 32 + kBN - 1) / kBN;
+  const int tile0 = row0 / kBN;   // the tile that holds this block's diagonal; earlier tiles are mirrored by other blocks
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint8_t* sA = smem;
   uint8_t* sB = smem + L::A_BYTES;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::A_BYTES + kStages * L::B_BYTES);
+  float* sRC = reinterpret_cast<float*>(smem + L::A_BYTES + kStages * L::B_BYTES);
+  uint32_t* sT = reinterpret_cast<uint32_t*>(smem + L::A_BYTES + kStages * L::B_BYTES + L::RC_BYTES);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::A_BYTES + kStages * L::B_BYTES + L::RC_BYTES + L::T_BYTES);
   uint64_t* a_full = bars + 0;
   uint64_t* b_full = bars + 1;      // [kStages]
   uint64_t* b_empty = bars + 3;     // [kStages]
@@ -92,7 +140,7 @@ __global__ void __launch_bounds__(kSimThreads, 1) sim_tc_kernel(const __grid_con
       ptx::mbar_expect_tx(a_full, L::A_BYTES);
       for (int kh = 0; kh < L::KH; ++kh)
         ptx::tma_load_5d(sA + kh * kBM * 128, &tmap, a_full, kh * 64, tok0 + row0, j, sdim, layer);
-      for (int it = 0; it < n_tiles; ++it) {
+      for (int it = 0; tile0 + it < n_tiles; ++it) {
         const int st = it & 1;
         if (!ptx::mbar_wait(b_empty + st, ((it >> 1) & 1) ^ 1, abort_flag)) break;
         ptx::mbar_expect_tx(b_full + st, L::B_BYTES);
@@ -100,7 +148,7 @@ __global__ void __launch_bounds__(kSimThreads, 1) sim_tc_kernel(const __grid_con
         for (int kh = 0; kh < L::KH; ++kh)
           for (int half = 0; half < 2; ++half)
             ptx::tma_load_5d(dst + kh * kBN * 128 + half * 128 * 128, &tmap, b_full + st, kh * 64,
-                             tok0 + it * kBN + half * 128, j, sdim, layer);
+                             tok0 + (tile0 + it) * kBN + half * 128, j, sdim, layer);
       }
     }
   } else if (warp == 1) {
@@ -108,7 +156,7 @@ __global__ void __launch_bounds__(kSimThreads, 1) sim_tc_kernel(const __grid_con
       constexpr uint32_t idesc = ptx::idesc_bf16_f32(kBM, kBN);
       const uint32_t a_addr = ptx::smem_u32(sA);
       bool ok = ptx::mbar_wait(a_full, 0, abort_flag);
-      for (int it = 0; ok && it < n_tiles; ++it) {
+      for (int it = 0; ok && tile0 + it < n_tiles; ++it) {
         const int st = it & 1;
         const uint32_t ph = (it >> 1) & 1;
         if (!ptx::mbar_wait(b_full + st, ph, abort_flag)) break;
@@ -128,50 +176,110 @@ __global__ void __launch_bounds__(kSimThreads, 1) sim_tc_kernel(const __grid_con
     }
   } else {
     const int q = warp & 3;               // TMEM lane quarter this warp may read
-    const int hc = (warp - 2) >> 2;       // which 128-column half of the tile
-    const int row = row0 + q * 32 + lane;
+    const int cg = (warp - 2) >> 2;       // which group of kColsPerWarp tile columns
+    const int et = threadIdx.x - 64;      // index within the epilogue group
+    const int R = row0 + q * 32;          // first row of this warp's 32-row strip
+    const int row = R + lane;
     const float* rinv = p.rinv + (int64_t)unit * p.row_words * 32;
-    const float rr = row < l ? rinv[row] : 0.f;
-    uint32_t* out = p.adj + ((int64_t)unit * p.batch.max_len + row) * p.row_words;
-    for (int it = 0; it < n_tiles; ++it) {
+    const int ncols = p.row_words * 32;
+    // threshold scaled by this row's norm; a zero row has similarity 0 with everything
+    float thr;
+    {
+      const float rr = row < l ? rinv[row] : 0.f;
+      thr = rr > 0.f ? p.theta / rr : p.theta;
+    }
+    uint32_t* adj_unit = p.adj + (int64_t)unit * p.batch.max_len * p.row_words;
+    uint32_t* out = adj_unit + (int64_t)row * p.row_words;
+    if (et < kBN) {
+      const int c = tile0 * kBN + et;
+      sRC[et] = c < ncols ? rinv[c] : 0.f;
+    }
+    epi_bar_sync();
+    for (int it = 0; tile0 + it < n_tiles; ++it) {
       const int st = it & 1;
-      if (!ptx::mbar_wait(acc_full + st, (it >> 1) & 1, abort_flag)) break;
+      const int c0 = (tile0 + it) * kBN;
+      const bool fast = c0 >= row0 + kBM;      // whole tile strictly above the diagonal
+      float rc_next = 0.f;
+      if (et < kBN) {
+        const int c = c0 + kBN + et;
+        if (tile0 + it + 1 < n_tiles && c < ncols) rc_next = __ldg(rinv + c);
+      }
+      // one lane polls, the warp follows
+      int ok = 1;
+      if (lane == 0) ok = ptx::mbar_wait(acc_full + st, (it >> 1) & 1, abort_flag) ? 1 : 0;
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+      if (!ok) break;
       ptx::tc_fence_after();
-      uint32_t words[4];
+      const float* rcs = sRC + st * kBN + cg * kColsPerWarp;
+      const uint32_t tbase = tmem_base + ((uint32_t)(q * 32) << 16) + st * kBN + cg * kColsPerWarp;
+      uint32_t words[kChunks];
 #pragma unroll
-      for (int ch = 0; ch < 4; ++ch) {
-        const int col0 = it * kBN + hc * 128 + ch * 32;
+      for (int ch = 0; ch < kChunks; ++ch) {
+        const int col0 = c0 + cg * kColsPerWarp + ch * 32;
         uint32_t acc[32];
-        ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + st * kBN + hc * 128 + ch * 32, acc);
-        float rc[32];
-        if (col0 < p.row_words * 32) {
+        ptx::tmem_ld_32x32(tbase + ch * 32, acc);
+        ptx::tmem_ld_wait(acc);
+        // four independent 8-bit groups keep the shift chains short
+        uint32_t wg[4] = {0, 0, 0, 0};
 #pragma unroll
-          for (int v = 0; v < 8; ++v) {
-            float4 t = __ldg(reinterpret_cast<const float4*>(rinv + col0) + v);
-            rc[4 * v] = t.x; rc[4 * v + 1] = t.y; rc[4 * v + 2] = t.z; rc[4 * v + 3] = t.w;
+        for (int v = 7; v >= 0; --v) {
+          float4 t = *reinterpret_cast<const float4*>(rcs + ch * 32 + v * 4);
+          const float rc4[4] = {t.x, t.y, t.z, t.w};
+#pragma unroll
+          for (int e = 3; e >= 0; --e) {
+            const int c = v * 4 + e;
+            float x = fmaf(-__uint_as_float(acc[c]), rc4[e], thr);
+            wg[c >> 3] = __funnelshift_l(__float_as_uint(x), wg[c >> 3], 1);
           }
-        } else {
-#pragma unroll
-          for (int v = 0; v < 32; ++v) rc[v] = 0.f;
         }
-        ptx::tmem_ld_wait();
-        uint32_t w = 0;
-#pragma unroll
-        for (int c = 31; c >= 0; --c) {
-          // negative exactly when dot * (rinv_a * rinv_b) > theta; the sign bit is shifted into the word
-          float x = fmaf(-__uint_as_float(acc[c]), rr * rc[c], p.theta);
-          w = __funnelshift_l(__float_as_uint(x), w, 1);
-        }
+        uint32_t w = __byte_perm(__byte_perm(wg[0], wg[1], 0x0040), __byte_perm(wg[2], wg[3], 0x0040), 0x5410);
         const int nvalid = l - col0;  // columns of this word that exist
         if (nvalid < 32) w &= nvalid > 0 ? ((1u << nvalid) - 1u) : 0u;
-        if (row >= col0 && row < col0 + 32) w |= 1u << (row - col0);  // unit diagonal
+        if (row >= l) w = 0;
         words[ch] = w;
       }
       ptx::tc_fence_before();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(acc_empty + st);
-      const int widx = it * (kBN / 32) + hc * 4;
-      if (row < l && widx < p.row_words) *reinterpret_cast<uint4*>(out + widx) = make_uint4(words[0], words[1], words[2], words[3]);
+      const int widx = (c0 >> 5) + cg * kChunks;
+      if (fast) {
+        if (row < l && widx < p.row_words) {
+          if (kChunks == 2) *reinterpret_cast<uint2*>(out + widx) = make_uint2(words[0], words[kChunks - 1]);
+          else
+#pragma unroll
+            for (int ch = 0; ch < kChunks; ++ch) out[widx + ch] = words[ch];
+        }
+        uint32_t* tq = sT + (st * 4 + q) * kBN + cg * kColsPerWarp;
+#pragma unroll
+        for (int ch = 0; ch < kChunks; ++ch) tq[ch * 32 + lane] = warp_transpose32(words[ch], lane);
+      } else {
+#pragma unroll
+        for (int ch = 0; ch < kChunks; ++ch) {
+          const int col0 = c0 + cg * kColsPerWarp + ch * 32;
+          if (col0 + 32 <= R) continue;                      // below the diagonal: another block mirrors it
+          if (col0 == R) {
+            // diagonal sub-block: upper triangle as computed, lower triangle mirrored from it, unit diagonal
+            const uint32_t upper = lane == 31 ? 0u : (0xFFFFFFFFu << (lane + 1));
+            const uint32_t wu = words[ch] & upper;
+            const uint32_t wt = warp_transpose32(wu, lane);
+            if (row < l) out[widx + ch] = wu | wt | (1u << lane);
+          } else {
+            if (row < l && widx + ch < p.row_words) out[widx + ch] = words[ch];
+            const uint32_t wt = warp_transpose32(words[ch], lane);
+            if (col0 + lane < l) adj_unit[(int64_t)(col0 + lane) * p.row_words + (R >> 5)] = wt;
+          }
+        }
+      }
+      if (et < kBN) sRC[(st ^ 1) * kBN + et] = rc_next;
+      epi_bar_sync();  // mirrored words of this tile and the next tile's inverse norms are in shared memory
+      if (fast && et < kBN) {
+        const int b = c0 + et;
+        if (b < l) {
+          const uint32_t* t0 = sT + st * 4 * kBN + et;
+          *reinterpret_cast<uint4*>(adj_unit + (int64_t)b * p.row_words + (row0 >> 5)) =
+              make_uint4(t0[0], t0[kBN], t0[2 * kBN], t0[3 * kBN]);
+        }
+      }
     }
   }
   // teardown: every role ends here, also after a wait that gave up

@@ -160,6 +160,24 @@ def test_degenerate_thresholds_duplicates_and_zero_rows():
     assert out[4] == 50 + 1 + 0  # 49 shared entries + the zero row + row 57/107 pair still shares one
 
 
+def test_degenerate_cases_on_the_tensor_core_path():
+    rng = np.random.default_rng(22)
+    from paper_2507_06517_b200.synth import round_to_dtype
+    for d, n in ((128, 700), (64, 300)):
+        g = round_to_dtype(rng.standard_normal((n, d)).astype(np.float32), "bf16")
+        adj, mag, ref, cen, cnt, C = _single_layer_codebook(g, 1.5, "bf16")
+        assert cnt == n and list(cen[:n]) == list(range(n)) and list(ref[:n]) == list(range(n))
+        g[5] = 0.0
+        g[n - 1] = 0.0
+        out = _single_layer_codebook(g, -1.5, "bf16")  # zero rows have similarity 0 > theta with everybody
+        assert out[4] == 1 and np.all(out[2][:n] == 0)
+        base = round_to_dtype(rng.standard_normal((n // 3, d)).astype(np.float32), "bf16")
+        g = np.concatenate([base, 2.0 * base, base, base[: n - 3 * (n // 3)]])
+        g[7] = 0.0
+        out = _single_layer_codebook(g, 0.999, "bf16")
+        check_codebook_unit(g, 0.999, *out, 1e-2)
+
+
 def test_all_scores_tie_goes_to_lowest_positions():
     # zero queries: plain window sums tie everywhere -> the first k context tokens; with the division
     # by (l - a) scores rise with position -> the last k
