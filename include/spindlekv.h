@@ -125,6 +125,29 @@ spindlekv_status spindlekv_evict_deep(const spindlekv_config* cfg, const spindle
                                       void* ws, size_t ws_bytes, void* stream);
 
 /*
+ * The same eviction as spindlekv_evict_deep for callers that cannot allocate device memory (the paper
+ * has no counterpart: this is a deployment convenience).  Typical callers: an inference server whose
+ * own pool has claimed the whole GPU, code running under another framework's allocator lock, or a
+ * latency-critical thread that must not trigger the implicit synchronisation of an allocation.  The
+ * scratch the kernels need is a fixed array of SPINDLEKV_NOALLOC_SCRATCH_BYTES inside the library
+ * image (present on every GPU that loads the library, until the process exits), so no workspace is
+ * passed and the function never calls cudaMalloc/cudaFree or any allocating routine.
+ *   - Arguments as spindlekv_evict_deep, minus the workspace.
+ *   - Returns WORKSPACE_TOO_SMALL when spindlekv_workspace_bytes(cfg, batch, SPINDLEKV_WS_EVICT) exceeds
+ *     SPINDLEKV_NOALLOC_SCRATCH_BYTES (e.g. more than about four 8B-shaped layers of 16k tokens at once):
+ *     split the layers over several calls.
+ *   - The first call on each device looks up the array's device address (with that device current);
+ *     make that first call outside any stream capture.
+ *   - All calls share the one array, which keeps the previous call's contents; what must start at
+ *     zero is cleared by the call itself.  Two calls whose kernels overlap on the GPU (different
+ *     streams, no ordering between them) race on it: order them.
+ */
+#define SPINDLEKV_NOALLOC_SCRATCH_BYTES (8 * 1024 * 1024)
+spindlekv_status spindlekv_evict_deep_noalloc(const spindlekv_config* cfg, const spindlekv_batch* batch,
+                                              spindlekv_tensor K, spindlekv_tensor Qwin, const int32_t* k_ctx,
+                                              int32_t* keep_idx, int32_t* keep_cnt, float* scores, void* stream);
+
+/*
  * CodeBook construction for shallow layers, one call per Gamma in {K, V} (Algorithm 1):
  * magnitudes (Eq. (8)); cosine similarity of all token pairs of a head (Eq. (4)); adjacency
  * G = [S > theta] with unit diagonal (Eq. (9)); then repeatedly: degrees (Eq. (10)), centre = arg-max

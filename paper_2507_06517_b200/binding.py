@@ -59,6 +59,9 @@ def _load() -> C.CDLL:
     lib.spindlekv_evict_deep.restype = C.c_int32
     lib.spindlekv_evict_deep.argtypes = [C.POINTER(_Config), C.POINTER(_Batch), _Tensor, _Tensor, C.c_void_p,
                                          C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+    lib.spindlekv_evict_deep_noalloc.restype = C.c_int32
+    lib.spindlekv_evict_deep_noalloc.argtypes = [C.POINTER(_Config), C.POINTER(_Batch), _Tensor, _Tensor, C.c_void_p,
+                                                 C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
     lib.spindlekv_codebook_shallow.restype = C.c_int32
     lib.spindlekv_codebook_shallow.argtypes = [C.POINTER(_Config), C.POINTER(_Batch), _Tensor, C.c_float,
                                                C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
@@ -175,6 +178,22 @@ def spindlekv_evict_deep(cfg: Config, batch: Batch, K: _Tensor, Qwin: _Tensor, k
     st = _lib.spindlekv_evict_deep(C.byref(cc), C.byref(bb), K, Qwin, _ptr(k_ctx), _ptr(keep_idx), _ptr(keep_cnt),
                                    _ptr(scores), _ptr(ws), ws.numel() * ws.element_size(), _stream(stream))
     _check(st, "spindlekv_evict_deep")
+
+
+NOALLOC_SCRATCH_BYTES = 8 * 1024 * 1024
+
+
+def spindlekv_evict_deep_noalloc(cfg: Config, batch: Batch, K: _Tensor, Qwin: _Tensor, k_ctx: torch.Tensor,
+                                 keep_idx: torch.Tensor, keep_cnt: torch.Tensor, scores: torch.Tensor,
+                                 stream=None) -> None:
+    """Eviction without a workspace, for callers that may not allocate device memory (a server whose
+    pool owns the GPU, code under another allocator's lock): the kernels' scratch is a fixed 8 MiB
+    array inside the library.  Raises ``WORKSPACE_TOO_SMALL`` when the batch needs more than that.
+    Calls share the array, so calls that could overlap on the GPU must be ordered by the caller."""
+    cc, bb = cfg.c(), batch.c()
+    st = _lib.spindlekv_evict_deep_noalloc(C.byref(cc), C.byref(bb), K, Qwin, _ptr(k_ctx), _ptr(keep_idx),
+                                           _ptr(keep_cnt), _ptr(scores), _stream(stream))
+    _check(st, "spindlekv_evict_deep_noalloc")
 
 
 def spindlekv_codebook_shallow(cfg: Config, batch: Batch, Gamma: _Tensor, theta: float, mag: torch.Tensor,
