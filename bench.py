@@ -224,7 +224,8 @@ def run_native(args, wl):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     # every rank compresses its own prompt (different seed)
-    wl = wl.replace(seed=wl.seed + rank)
+    from paper_2507_06517_b200 import sharding
+    wl = sharding.rank_workload(wl, rank)
     dev = torch.device("cuda", local_rank)
     cfg = B.Config(n_layers=wl.n_layers, n_q_heads=wl.n_q_heads, n_kv_heads=wl.n_kv_heads, head_dim=wl.head_dim,
                    window=wl.window, n_shallow=wl.n_shallow, beta=wl.beta, theta_k=wl.theta_k, theta_v=wl.theta_v,
@@ -278,11 +279,8 @@ def run_native(args, wl):
             fn()
         ev1.record()
         barrier()
-        ms = ev0.elapsed_time(ev1)
-        if dist is not None:
-            t = torch.tensor([ms], device=dev, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
+        tokens, ms = sharding.aggregate(wl.total_tokens, ev0.elapsed_time(ev1), dist, dev)
+        timed.tokens = tokens
         return ms
 
     upload()
@@ -298,6 +296,7 @@ def run_native(args, wl):
     t0 = time.perf_counter()
     ms = timed(step, args.steps)
     t1 = time.perf_counter()
+    job_tokens = timed.tokens
     launches = B.spindlekv_launch_count(True)
     clocks = sampler.stop(t0, t1) if sampler else None
 
@@ -309,7 +308,7 @@ def run_native(args, wl):
             download()
         step_e2e()
         ms_e2e = timed(step_e2e, args.steps)
-        e2e = {"value": world * wl.total_tokens * args.steps / (ms_e2e * 1e-3), "unit": UNIT,
+        e2e = {"value": sharding.throughput(timed.tokens, args.steps, ms_e2e), "unit": UNIT,
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / args.steps}
 
     # per-kernel times: one more pass with event pairs around every launch
@@ -341,7 +340,7 @@ def run_native(args, wl):
         roof = {"kernel": "similarity (Eq. 4, 9)", "bound": "tensor", "achieved": achieved, "peak": peak,
                 "unit": "TFLOP/s", "frac": achieved / peak, "traffic": traffic, "peak_source": pk_src,
                 "avg_launch_ms": sim_ms / sim_n, "algorithmic_flops_per_launch": flops_per_step * args.steps / sim_n}
-    line = {"metric": METRIC, "value": world * wl.total_tokens * args.steps / (ms * 1e-3), "unit": UNIT,
+    line = {"metric": METRIC, "value": sharding.throughput(job_tokens, args.steps, ms), "unit": UNIT,
             "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": wl.dtype,
             "data": "synthetic", "config": workload_config(wl, {"parallelism": f"replicas x{world}"}),
