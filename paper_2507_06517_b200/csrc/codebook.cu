@@ -22,7 +22,8 @@ struct CodebookParams {
   int n_kv_heads, n_units, row_words;
   float theta;
   float* mag;            // [layers][H][T]
-  float* rinv;           // [units][row_words*32]: 1/|gamma|, 0 for zero vectors and beyond the sequence
+  __nv_bfloat16* ext;    // [2][units][row_words*32][16]: the extra K-step of the tensor-core similarity
+                         // ([0]: theta*|gamma|, [1]: |gamma|, each in three bf16 pieces; zero beyond the sequence)
   uint32_t* adj;         // [units][max_len][row_words]
   int32_t* deg;          // [units][max_len]
   unsigned long long* key;  // [units][max_len]
@@ -51,6 +52,15 @@ __device__ __forceinline__ int64_t cb_out_row(const CodebookParams& p, int layer
 }
 
 // ---- Eq. (8): magnitudes.  8 lanes per row of 64 elements, 16 lanes per row of 128. -----------
+// x = p0 + p1 + p2 exactly, each piece a bf16 (8 significant bits each, 24 in all)
+__device__ __forceinline__ void split3_bf16(float x, __nv_bfloat16 (&pc)[3]) {
+#pragma unroll
+  for (int i = 0; i < 3; ++i) {
+    pc[i] = __float2bfloat16_rn(x);
+    x -= __bfloat162float(pc[i]);
+  }
+}
+
 template <typename T, int D>
 __global__ void __launch_bounds__(256) norms_kernel(CodebookParams p) {
   constexpr int LPR = D / 8;  // lanes per row
@@ -70,10 +80,25 @@ __global__ void __launch_bounds__(256) norms_kernel(CodebookParams p) {
   }
 #pragma unroll
   for (int o = LPR / 2; o >= 1; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-  if (seg == 0) {
-    const float m = sqrtf(ss);
-    if (row < l) p.mag[cb_out_row(p, layer, s, j) + row] = m;
-    if (row < p.row_words * 32) p.rinv[(int64_t)blockIdx.y * p.row_words * 32 + row] = (row < l && m > 0.f) ? 1.0f / m : 0.f;
+  const float m = sqrtf(ss);
+  if (seg == 0 && row < l) p.mag[cb_out_row(p, layer, s, j) + row] = m;
+  if (p.ext && seg < 2 && row < p.row_words * 32) {
+    // Row `row` of operand [seg] of the extra K-step: slots 0..8 hold the pieces so that the nine
+    // products of an A row with a B row add up to theta*|a| * |b|.  A zero vector takes magnitude 1:
+    // its dot products are 0, so the accumulator keeps the sign of theta, as "0 > theta" demands.
+    const float n = m > 0.f ? m : 1.f;
+    __nv_bfloat16 pc[3];
+    split3_bf16(seg == 0 ? p.theta * n : n, pc);
+    __align__(16) __nv_bfloat16 out[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) out[i] = __float2bfloat16_rn(0.f);
+    if (row < l) {
+#pragma unroll
+      for (int i = 0; i < 9; ++i) out[i] = seg == 0 ? pc[i / 3] : pc[i % 3];
+    }
+    uint4* dst = reinterpret_cast<uint4*>(p.ext + (((int64_t)seg * p.n_units + blockIdx.y) * p.row_words * 32 + row) * 16);
+    dst[0] = *reinterpret_cast<const uint4*>(out);
+    dst[1] = *reinterpret_cast<const uint4*>(out + 8);
   }
 }
 
@@ -493,7 +518,7 @@ __global__ void __launch_bounds__(kFinalThreads) finalize_kernel(CodebookParams 
 // ---- host side ----------------------------------------------------------------------------------
 
 struct CodebookLayout {
-  size_t rinv, ell, ell_cnt, adj, deg, key, m1, live0, live1, owner, pickdeg, rank, total;
+  size_t ext, ell, ell_cnt, adj, deg, key, m1, live0, live1, owner, pickdeg, rank, total;
 };
 
 static CodebookLayout codebook_layout(const spindlekv_config& cfg, const spindlekv_batch& b, bool adj_in_ws) {
@@ -510,7 +535,7 @@ static CodebookLayout codebook_layout(const spindlekv_config& cfg, const spindle
   L.owner = take(units * ML * 4);
   L.pickdeg = take(units * ML * 4);
   L.rank = take(units * ML * 4);
-  L.rinv = take(units * RW * 32 * 4);
+  L.ext = take(2 * units * RW * 32 * 16 * 2);
   L.ell = take(units * ML * 32 * 4);
   L.ell_cnt = take(units * ML * 4);
   L.adj = off;
@@ -525,7 +550,7 @@ size_t codebook_workspace_bytes(const spindlekv_config& cfg, const spindlekv_bat
 
 bool sim_tc_available();
 spindlekv_status launch_sim_tc(const spindlekv_tensor& Gamma, const spindlekv_batch& b, int n_kv_heads, int head_dim,
-                               float theta, const float* rinv, uint32_t* adj, uint32_t* hdr, cudaStream_t st);
+                               const void* ext, uint32_t* adj, uint32_t* hdr, cudaStream_t st);
 
 template <typename T, int D>
 static void launch_norms(const CodebookParams& p, cudaStream_t st) {
@@ -559,7 +584,6 @@ spindlekv_status codebook_shallow_impl(const spindlekv_config& cfg, const spindl
   p.row_words = row_words_for(b.max_len);
   p.theta = theta;
   p.mag = mag;
-  p.rinv = reinterpret_cast<float*>(w + L.rinv);
   p.adj = adj_in_ws ? reinterpret_cast<uint32_t*>(w + L.adj) : adj_bits;
   p.deg = reinterpret_cast<int32_t*>(w + L.deg);
   p.key = reinterpret_cast<unsigned long long*>(w + L.key);
@@ -578,14 +602,15 @@ spindlekv_status codebook_shallow_impl(const spindlekv_config& cfg, const spindl
   if (cudaMemsetAsync(w, 0, kHeaderBytes, st) != cudaSuccess) return SPINDLEKV_CUDA;
   if (cudaMemsetAsync(p.pickdeg, 0xFF, (size_t)units * b.max_len * 4, st) != cudaSuccess) return SPINDLEKV_CUDA;
   const bool bf = Gamma.dtype == SPINDLEKV_BF16;
+  const bool tc = bf && sim_tc_available();   // bf16: tensor-core similarity (TMA + tcgen05)
+  p.ext = tc ? reinterpret_cast<__nv_bfloat16*>(w + L.ext) : nullptr;
   if (cfg.head_dim == 64) {
     if (bf) launch_norms<__nv_bfloat16, 64>(p, st); else launch_norms<float, 64>(p, st);
   } else {
     if (bf) launch_norms<__nv_bfloat16, 128>(p, st); else launch_norms<float, 128>(p, st);
   }
-  if (bf && sim_tc_available()) {
-    // bf16: tensor-core similarity (TMA + tcgen05)
-    spindlekv_status rs = launch_sim_tc(Gamma, b, cfg.n_kv_heads, cfg.head_dim, theta, p.rinv, p.adj, p.hdr, st);
+  if (tc) {
+    spindlekv_status rs = launch_sim_tc(Gamma, b, cfg.n_kv_heads, cfg.head_dim, p.ext, p.adj, p.hdr, st);
     if (rs != SPINDLEKV_OK) return rs;
   } else if (cfg.head_dim == 64) {
     if (bf) launch_sim_simt<__nv_bfloat16, 64>(p, b, st); else launch_sim_simt<float, 64>(p, b, st);

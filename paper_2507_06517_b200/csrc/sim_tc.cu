@@ -6,14 +6,22 @@
 // One CTA owns a block of 128 token rows of one (layer, sequence, head) unit: the block is loaded
 // once by TMA and stays in shared memory as operand A; tiles of 256 token rows, from the tile that
 // holds the diagonal onwards, stream through a two-stage ring as operand B.  One elected thread
-// issues tcgen05.mma (128 x 256 x 16, fp32 accumulation in TMEM) for the raw bf16 dot products.
-// Eight epilogue warps read the accumulators back with tcgen05.ld while the tensor cores work on
-// the other TMEM stage.  A thread owns one row a; per pair it evaluates
-//     x = fma(-dot, rinv_b, theta * |a|)        (rinv = 1/|gamma|, 0 for a zero vector)
-// whose sign bit is the decision dot/(|a||b|) > theta, and shifts that bit into a 32-bit word.
-// The word goes to row a as is; a 32x32 bit transpose across the warp turns the 32 words of a
-// sub-block into the words of the mirrored rows, which are staged in shared memory and written
-// 16 bytes per row.  Nothing but bits leaves the SM: N*N/8 bytes per unit.
+// issues tcgen05.mma (128 x 256 x 16, fp32 accumulation in TMEM).
+//
+// The threshold is part of the contraction.  The main K-steps run with the negate-A flag and
+// accumulate -gamma_a . gamma_b; one more K-step multiplies two 16-element rows prepared by the
+// magnitude kernel: theta*|gamma_a| and |gamma_b|, each split into three bf16 pieces, laid out so
+// that the nine cross products add up to theta*|gamma_a|*|gamma_b| (exact up to the fp32
+// accumulation).  The accumulator then holds  theta*|a||b| - a.b , whose sign bit is the decision
+// a.b / (|a||b|) > theta.  The epilogue therefore only collects sign bits: no per-column operand,
+// no floating-point instruction.
+//
+// Sixteen epilogue warps read the accumulators back with tcgen05.ld while the tensor cores work on
+// the other TMEM stage.  A thread owns one row a and shifts the sign bits of 32 columns into a word.
+// Direct words are staged in shared memory and leave in 128-byte row segments once every four
+// tiles; a 32x32 bit transpose across the warp turns the words of a sub-block into the words of the
+// mirrored rows, which are staged too and written 16 bytes per row.  Nothing but bits leaves the SM:
+// N*N/8 bytes per unit.
 #include "common.cuh"
 #include "sm100_ptx.cuh"
 
@@ -22,8 +30,6 @@ namespace skv {
 struct SimTcParams {
   Batch batch;
   int n_kv_heads, row_words;
-  float theta;
-  const float* rinv;   // [units][row_words*32], zero beyond the sequence
   uint32_t* adj;       // [units][max_len][row_words]
   uint32_t* hdr;
 };
@@ -36,57 +42,89 @@ constexpr int kColsPerWarp = kBN / (kEpiWarps / 4);   // tile columns handled by
 constexpr int kChunks = kColsPerWarp / 32;
 constexpr int kEpiThreads = 32 * kEpiWarps;
 constexpr int kSimThreads = 32 * (2 + kEpiWarps);
+constexpr int kGroupTiles = 4;                        // direct rows are flushed once per this many tiles
+constexpr int kGroupWords = kGroupTiles * kBN / 32;   // 32 words = 128 bytes of a row
+constexpr int kDPitch = kGroupWords + 2;              // row pitch of the staging buffer in words
+static_assert(kChunks == 2 && kGroupWords == 32, "epilogue layout assumes 64 columns per warp and 128-byte flushes");
 
 template <int D>
 struct SimSmem {
   static constexpr int KH = D / 64;                  // 64-element (128-byte) swizzle atoms along head_dim
   static constexpr int A_BYTES = KH * kBM * 128;
   static constexpr int B_BYTES = KH * kBN * 128;
-  static constexpr int RC_BYTES = 2 * kBN * 4;       // inverse norms of the tile's 256 tokens, two slots
+  static constexpr int EA_BYTES = kBM * 32;          // threshold rows of the block (one 16-element K-step)
+  static constexpr int EB_BYTES = kBN * 32;          // magnitude rows of a tile
   static constexpr int T_BYTES = 2 * 4 * kBN * 4;    // mirrored words [slot][row quarter][tile column]
-  static constexpr int USED = A_BYTES + kStages * B_BYTES + RC_BYTES + T_BYTES + 256 /*barriers*/ + 1024 /*alignment*/;
+  static constexpr int D_BYTES = 2 * kBM * kDPitch * 4;  // direct words [slot][row][word of the group]
+  static constexpr int OFF_B = A_BYTES;
+  static constexpr int OFF_EA = OFF_B + kStages * B_BYTES;
+  static constexpr int OFF_EB = OFF_EA + EA_BYTES;
+  static constexpr int OFF_T = OFF_EB + kStages * EB_BYTES;
+  static constexpr int OFF_D = OFF_T + T_BYTES;
+  static constexpr int OFF_BAR = OFF_D + D_BYTES;
+  static constexpr int USED = OFF_BAR + 256 /*barriers*/ + 1024 /*alignment*/;
   // at least 120 KB so that two blocks never share an SM: each block allocates all 512 TMEM columns
   static constexpr int TOTAL = USED > 120 * 1024 ? USED : 120 * 1024;
+  static_assert(TOTAL <= 227 * 1024, "shared memory budget");
 };
 
-// 32x32 bit transpose across a warp: in: lane r holds bits (r, c) at bit c; out: lane c holds bit r
-__device__ __forceinline__ uint32_t warp_transpose32(uint32_t x, int lane) {
-  uint32_t m = 0x0000FFFFu;
+// 32x32 bit transpose across a warp: in: lane r holds bits (r, c) at bit c; out: lane c holds bit r.
+// Five butterfly stages (j = 16, 8, 4, 2, 1): a lane takes from its partner the half of every 2j-bit
+// group that it does not keep, moved by j positions.  The move is a rotation (the bits that wrap
+// around fall outside the kept mask), so a stage is one shuffle, one funnel shift and one logic op;
+// rotation amounts and masks depend on the lane only and are set up once.
+struct TransposeLane {
+  uint32_t rot[5], keep[5];
+  __device__ __forceinline__ void init(int lane) {
+    uint32_t m = 0x0000FFFFu;
 #pragma unroll
-  for (int j = 16; j >= 1; j >>= 1) {
-    const uint32_t y = __shfl_xor_sync(0xffffffffu, x, j);
-    const bool hi = (lane & j) != 0;
-    const uint32_t keep = hi ? ~m : m;
-    const uint32_t sh = hi ? (y >> j) : (y << j);
-    x = (x & keep) | (sh & ~keep);
-    m ^= m << (j >> 1);
-  }
-  return x;
-}
-
-// four transposes at once: the shuffles of one stage are independent of each other
-__device__ __forceinline__ void warp_transpose32x4(uint32_t (&x)[4], int lane) {
-  uint32_t m = 0x0000FFFFu;
-#pragma unroll
-  for (int j = 16; j >= 1; j >>= 1) {
-    const bool hi = (lane & j) != 0;
-    const uint32_t keep = hi ? ~m : m;
-    uint32_t y[4];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) y[i] = __shfl_xor_sync(0xffffffffu, x[i], j);
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const uint32_t sh = hi ? (y[i] >> j) : (y[i] << j);
-      x[i] = (x[i] & keep) | (sh & ~keep);
+    for (int k = 0; k < 5; ++k) {
+      const int j = 16 >> k;
+      const bool hi = (lane & j) != 0;
+      keep[k] = hi ? ~m : m;
+      rot[k] = hi ? 32 - j : j;
+      m ^= m << (j >> 1);
     }
-    m ^= m << (j >> 1);
   }
+  __device__ __forceinline__ uint32_t apply(uint32_t x) const {
+#pragma unroll
+    for (int k = 0; k < 5; ++k) {
+      const uint32_t y = __shfl_xor_sync(0xffffffffu, x, 16 >> k);
+      const uint32_t r = __funnelshift_l(y, y, rot[k]);
+      x = (x & keep[k]) | (r & ~keep[k]);
+    }
+    return x;
+  }
+};
+
+// Barrier over the epilogue warps that also agrees on whether everybody is still fine: returns
+// the AND of `ok` over all of them, so that they leave the tile loop together.
+__device__ __forceinline__ bool epi_bar_all(bool ok) {
+  uint32_t r;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.u32 q, %1, 0;\n\t"
+      "bar.red.and.pred p, 1, %2, q;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(r)
+      : "r"((uint32_t)ok), "n"(kEpiThreads)
+      : "memory");
+  return r != 0;
 }
 
-__device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory"); }
+// sign bits of 32 accumulators -> one word, bit c = sign of column c
+__device__ __forceinline__ uint32_t sign_word(const uint32_t (&acc)[32]) {
+  // four independent 8-bit groups keep the shift chains short
+  uint32_t wg[4] = {0, 0, 0, 0};
+#pragma unroll
+  for (int c = 31; c >= 0; --c) wg[c >> 3] = __funnelshift_l(acc[c], wg[c >> 3], 1);
+  return __byte_perm(__byte_perm(wg[0], wg[1], 0x0040), __byte_perm(wg[2], wg[3], 0x0040), 0x5410);
+}
 
 template <int D>
-__global__ void __launch_bounds__(kSimThreads, 1) sim_tc_kernel(const __grid_constant__ CUtensorMap tmap, SimTcParams p) {
+__global__ void __launch_bounds__(kSimThreads, 1) sim_tc_kernel(const __grid_constant__ CUtensorMap tmap,
+                                                                const __grid_constant__ CUtensorMap emap,
+                                                                SimTcParams p) {
   using L = SimSmem<D>;
   const int unit = blockIdx.y;
   const int j = unit % p.n_kv_heads;
@@ -102,10 +140,12 @@ __global__ void __launch_bounds__(kSimThreads, 1) sim_tc_kernel(const __grid_con
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint8_t* sA = smem;
-  uint8_t* sB = smem + L::A_BYTES;
-  float* sRC = reinterpret_cast<float*>(smem + L::A_BYTES + kStages * L::B_BYTES);
-  uint32_t* sT = reinterpret_cast<uint32_t*>(smem + L::A_BYTES + kStages * L::B_BYTES + L::RC_BYTES);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::A_BYTES + kStages * L::B_BYTES + L::RC_BYTES + L::T_BYTES);
+  uint8_t* sB = smem + L::OFF_B;
+  uint8_t* sEA = smem + L::OFF_EA;
+  uint8_t* sEB = smem + L::OFF_EB;
+  uint32_t* sT = reinterpret_cast<uint32_t*>(smem + L::OFF_T);
+  uint32_t* sD = reinterpret_cast<uint32_t*>(smem + L::OFF_D);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::OFF_BAR);
   uint64_t* a_full = bars + 0;
   uint64_t* b_full = bars + 1;      // [kStages]
   uint64_t* b_empty = bars + 3;     // [kStages]
@@ -137,24 +177,31 @@ __global__ void __launch_bounds__(kSimThreads, 1) sim_tc_kernel(const __grid_con
   if (warp == 0) {
     if (lane == 0) {
       ptx::prefetch_tensormap(&tmap);
-      ptx::mbar_expect_tx(a_full, L::A_BYTES);
+      ptx::prefetch_tensormap(&emap);
+      ptx::mbar_expect_tx(a_full, L::A_BYTES + L::EA_BYTES);
       for (int kh = 0; kh < L::KH; ++kh)
         ptx::tma_load_5d(sA + kh * kBM * 128, &tmap, a_full, kh * 64, tok0 + row0, j, sdim, layer);
+      ptx::tma_load_4d(sEA, &emap, a_full, 0, row0, unit, 0);
       for (int it = 0; tile0 + it < n_tiles; ++it) {
         const int st = it & 1;
         if (!ptx::mbar_wait(b_empty + st, ((it >> 1) & 1) ^ 1, abort_flag)) break;
-        ptx::mbar_expect_tx(b_full + st, L::B_BYTES);
+        ptx::mbar_expect_tx(b_full + st, L::B_BYTES + L::EB_BYTES);
         uint8_t* dst = sB + st * L::B_BYTES;
         for (int kh = 0; kh < L::KH; ++kh)
           for (int half = 0; half < 2; ++half)
             ptx::tma_load_5d(dst + kh * kBN * 128 + half * 128 * 128, &tmap, b_full + st, kh * 64,
                              tok0 + (tile0 + it) * kBN + half * 128, j, sdim, layer);
+        for (int half = 0; half < 2; ++half)
+          ptx::tma_load_4d(sEB + st * L::EB_BYTES + half * 128 * 32, &emap, b_full + st, 0,
+                           (tile0 + it) * kBN + half * 128, unit, 1);
       }
     }
   } else if (warp == 1) {
     if (lane == 0) {
-      constexpr uint32_t idesc = ptx::idesc_bf16_f32(kBM, kBN);
+      constexpr uint32_t idesc_neg = ptx::idesc_bf16_f32(kBM, kBN, true);
+      constexpr uint32_t idesc_pos = ptx::idesc_bf16_f32(kBM, kBN, false);
       const uint32_t a_addr = ptx::smem_u32(sA);
+      const uint64_t dea = ptx::smem_desc_sw32(ptx::smem_u32(sEA));
       bool ok = ptx::mbar_wait(a_full, 0, abort_flag);
       for (int it = 0; ok && tile0 + it < n_tiles; ++it) {
         const int st = it & 1;
@@ -168,8 +215,10 @@ __global__ void __launch_bounds__(kSimThreads, 1) sim_tc_kernel(const __grid_con
           const int kh = k >> 2, kk = k & 3;
           uint64_t da = ptx::smem_desc_sw128(a_addr + kh * kBM * 128 + kk * 32);
           uint64_t db = ptx::smem_desc_sw128(b_addr + kh * kBN * 128 + kk * 32);
-          ptx::umma_bf16(tmem_base + st * kBN, da, db, idesc, k > 0 ? 1u : 0u);
+          ptx::umma_bf16(tmem_base + st * kBN, da, db, idesc_neg, k > 0 ? 1u : 0u);
         }
+        // + theta * |a| * |b|
+        ptx::umma_bf16(tmem_base + st * kBN, dea, ptx::smem_desc_sw32(ptx::smem_u32(sEB + st * L::EB_BYTES)), idesc_pos, 1u);
         ptx::umma_commit(b_empty + st);   // shared-memory stage may be refilled
         ptx::umma_commit(acc_full + st);  // accumulator ready for the epilogue
       }
@@ -177,107 +226,101 @@ __global__ void __launch_bounds__(kSimThreads, 1) sim_tc_kernel(const __grid_con
   } else {
     const int q = warp & 3;               // TMEM lane quarter this warp may read
     const int cg = (warp - 2) >> 2;       // which group of kColsPerWarp tile columns
+    const int ew = warp - 2;              // index among the epilogue warps
     const int et = threadIdx.x - 64;      // index within the epilogue group
+    const int rl = q * 32 + lane;         // row within the block
     const int R = row0 + q * 32;          // first row of this warp's 32-row strip
     const int row = R + lane;
-    const float* rinv = p.rinv + (int64_t)unit * p.row_words * 32;
-    const int ncols = p.row_words * 32;
-    // threshold scaled by this row's norm; a zero row has similarity 0 with everything
-    float thr;
-    {
-      const float rr = row < l ? rinv[row] : 0.f;
-      thr = rr > 0.f ? p.theta / rr : p.theta;
-    }
-    uint32_t* adj_unit = p.adj + (int64_t)unit * p.batch.max_len * p.row_words;
-    uint32_t* out = adj_unit + (int64_t)row * p.row_words;
-    if (et < kBN) {
-      const int c = tile0 * kBN + et;
-      sRC[et] = c < ncols ? rinv[c] : 0.f;
-    }
-    epi_bar_sync();
-    for (int it = 0; tile0 + it < n_tiles; ++it) {
+    const int RW = p.row_words;
+    uint32_t* adj_unit = p.adj + (int64_t)unit * p.batch.max_len * RW;
+    TransposeLane tr;
+    tr.init(lane);
+    // where this thread stages its direct words (advances by one tile's words, wraps per group)
+    uint32_t* sd_mine = sD + rl * kDPitch + cg * kChunks;
+    // mirrored rows: thread et writes row c0 + et, 16 bytes at the block's column
+    uint32_t* mir = adj_unit + (int64_t)(tile0 * kBN + et) * RW + (row0 >> 5);
+    const int64_t mir_step = (int64_t)kBN * RW;
+    const uint32_t tcol = tmem_base + ((uint32_t)(q * 32) << 16) + cg * kColsPerWarp;
+    uint32_t* tq = sT + q * kBN + cg * kColsPerWarp + lane;
+    for (int it = 0; tile0 + it < n_tiles; ++it, mir += mir_step) {
       const int st = it & 1;
-      const int c0 = (tile0 + it) * kBN;
+      const int tile = tile0 + it;
+      const int c0 = tile * kBN;
       const bool fast = c0 >= row0 + kBM;      // whole tile strictly above the diagonal
-      float rc_next = 0.f;
-      if (et < kBN) {
-        const int c = c0 + kBN + et;
-        if (tile0 + it + 1 < n_tiles && c < ncols) rc_next = __ldg(rinv + c);
-      }
+      const int gslot = (tile & (kGroupTiles - 1)) * (kBN / 32);
+      uint32_t* sdbuf = sD + ((tile / kGroupTiles) & 1) * (kBM * kDPitch);
+      uint32_t* sdw = sd_mine + ((tile / kGroupTiles) & 1) * (kBM * kDPitch) + gslot;
       // one lane polls, the warp follows
       int ok = 1;
       if (lane == 0) ok = ptx::mbar_wait(acc_full + st, (it >> 1) & 1, abort_flag) ? 1 : 0;
       ok = __shfl_sync(0xffffffffu, ok, 0);
-      if (!ok) break;
-      ptx::tc_fence_after();
-      const float* rcs = sRC + st * kBN + cg * kColsPerWarp;
-      const uint32_t tbase = tmem_base + ((uint32_t)(q * 32) << 16) + st * kBN + cg * kColsPerWarp;
-      uint32_t words[kChunks];
-#pragma unroll
-      for (int ch = 0; ch < kChunks; ++ch) {
-        const int col0 = c0 + cg * kColsPerWarp + ch * 32;
-        uint32_t acc[32];
-        ptx::tmem_ld_32x32(tbase + ch * 32, acc);
-        ptx::tmem_ld_wait(acc);
-        // four independent 8-bit groups keep the shift chains short
-        uint32_t wg[4] = {0, 0, 0, 0};
-#pragma unroll
-        for (int v = 7; v >= 0; --v) {
-          float4 t = *reinterpret_cast<const float4*>(rcs + ch * 32 + v * 4);
-          const float rc4[4] = {t.x, t.y, t.z, t.w};
-#pragma unroll
-          for (int e = 3; e >= 0; --e) {
-            const int c = v * 4 + e;
-            float x = fmaf(-__uint_as_float(acc[c]), rc4[e], thr);
-            wg[c >> 3] = __funnelshift_l(__float_as_uint(x), wg[c >> 3], 1);
-          }
-        }
-        uint32_t w = __byte_perm(__byte_perm(wg[0], wg[1], 0x0040), __byte_perm(wg[2], wg[3], 0x0040), 0x5410);
-        const int nvalid = l - col0;  // columns of this word that exist
-        if (nvalid < 32) w &= nvalid > 0 ? ((1u << nvalid) - 1u) : 0u;
-        if (row >= l) w = 0;
-        words[ch] = w;
-      }
-      ptx::tc_fence_before();
-      __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(acc_empty + st);
-      const int widx = (c0 >> 5) + cg * kChunks;
-      if (fast) {
-        if (row < l && widx < p.row_words) {
-          if (kChunks == 2) *reinterpret_cast<uint2*>(out + widx) = make_uint2(words[0], words[kChunks - 1]);
-          else
-#pragma unroll
-            for (int ch = 0; ch < kChunks; ++ch) out[widx + ch] = words[ch];
-        }
-        uint32_t* tq = sT + (st * 4 + q) * kBN + cg * kColsPerWarp;
-#pragma unroll
-        for (int ch = 0; ch < kChunks; ++ch) tq[ch * 32 + lane] = warp_transpose32(words[ch], lane);
-      } else {
+      if (ok) {
+        ptx::tc_fence_after();
+        uint32_t words[kChunks];
 #pragma unroll
         for (int ch = 0; ch < kChunks; ++ch) {
-          const int col0 = c0 + cg * kColsPerWarp + ch * 32;
-          if (col0 + 32 <= R) continue;                      // below the diagonal: another block mirrors it
-          if (col0 == R) {
-            // diagonal sub-block: upper triangle as computed, lower triangle mirrored from it, unit diagonal
-            const uint32_t upper = lane == 31 ? 0u : (0xFFFFFFFFu << (lane + 1));
-            const uint32_t wu = words[ch] & upper;
-            const uint32_t wt = warp_transpose32(wu, lane);
-            if (row < l) out[widx + ch] = wu | wt | (1u << lane);
-          } else {
-            if (row < l && widx + ch < p.row_words) out[widx + ch] = words[ch];
-            const uint32_t wt = warp_transpose32(words[ch], lane);
-            if (col0 + lane < l) adj_unit[(int64_t)(col0 + lane) * p.row_words + (R >> 5)] = wt;
+          uint32_t acc[32];
+          ptx::tmem_ld_32x32(tcol + st * kBN + ch * 32, acc);
+          ptx::tmem_ld_wait(acc);
+          words[ch] = sign_word(acc);
+        }
+        ptx::tc_fence_before();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(acc_empty + st);
+        if (c0 + kBN > l || R + 32 > l) {
+          // ragged edge: columns and rows that do not exist carry no bits
+#pragma unroll
+          for (int ch = 0; ch < kChunks; ++ch) {
+            const int nvalid = l - (c0 + cg * kColsPerWarp + ch * 32);
+            if (nvalid < 32) words[ch] &= nvalid > 0 ? ((1u << nvalid) - 1u) : 0u;
+            if (row >= l) words[ch] = 0;
+          }
+        }
+        if (fast) {
+          if (kChunks == 2) *reinterpret_cast<uint2*>(sdw) = make_uint2(words[0], words[kChunks - 1]);
+          else
+#pragma unroll
+            for (int ch = 0; ch < kChunks; ++ch) sdw[ch] = words[ch];
+          // most 32 x 32 sub-blocks of a sparse graph are empty: their mirror image is too
+#pragma unroll
+          for (int ch = 0; ch < kChunks; ++ch)
+            tq[st * 4 * kBN + ch * 32] = __any_sync(0xffffffffu, words[ch] != 0u) ? tr.apply(words[ch]) : 0u;
+        } else {
+#pragma unroll
+          for (int ch = 0; ch < kChunks; ++ch) {
+            const int col0 = c0 + cg * kColsPerWarp + ch * 32;
+            if (col0 + 32 <= R) continue;                      // below the diagonal: another block mirrors it
+            if (col0 == R) {
+              // diagonal sub-block: upper triangle as computed, lower triangle mirrored from it, unit diagonal
+              const uint32_t upper = lane == 31 ? 0u : (0xFFFFFFFFu << (lane + 1));
+              const uint32_t wu = words[ch] & upper;
+              const uint32_t wt = tr.apply(wu);
+              sdw[ch] = row < l ? (wu | wt | (1u << lane)) : 0u;
+            } else {
+              sdw[ch] = words[ch];
+              const uint32_t wt = tr.apply(words[ch]);
+              if (col0 + lane < l) adj_unit[(int64_t)(col0 + lane) * RW + (R >> 5)] = wt;
+            }
           }
         }
       }
-      if (et < kBN) sRC[(st ^ 1) * kBN + et] = rc_next;
-      epi_bar_sync();  // mirrored words of this tile and the next tile's inverse norms are in shared memory
-      if (fast && et < kBN) {
-        const int b = c0 + et;
-        if (b < l) {
-          const uint32_t* t0 = sT + st * 4 * kBN + et;
-          *reinterpret_cast<uint4*>(adj_unit + (int64_t)b * p.row_words + (row0 >> 5)) =
-              make_uint4(t0[0], t0[kBN], t0[2 * kBN], t0[3 * kBN]);
+      // mirrored and direct words of this tile are in shared memory; everybody agrees to go on
+      if (!epi_bar_all(ok != 0)) break;
+      if (fast && et < kBN && c0 + et < l) {
+        const uint32_t* t0 = sT + st * 4 * kBN + et;
+        *reinterpret_cast<uint4*>(mir) = make_uint4(t0[0], t0[kBN], t0[2 * kBN], t0[3 * kBN]);
+      }
+      if (gslot == (kGroupTiles - 1) * (kBN / 32) || tile == n_tiles - 1) {
+        // direct rows of the last (up to) four tiles: one 128-byte segment per row, eight rows per warp;
+        // words left of a row's diagonal sub-block belong to other blocks' mirrored writes
+        const int wi = (tile & ~(kGroupTiles - 1)) * (kBN / 32) + lane;
+        const int r0 = ew * (kBM / kEpiWarps);
+        if (wi >= ((row0 + (r0 & ~31)) >> 5) && wi < RW) {
+          uint32_t* dst = adj_unit + (int64_t)(row0 + r0) * RW + wi;
+          const uint32_t* src = sdbuf + r0 * kDPitch + lane;
+#pragma unroll
+          for (int i = 0; i < kBM / kEpiWarps; ++i)
+            if (row0 + r0 + i < l) dst[(int64_t)i * RW] = src[i * kDPitch];
         }
       }
     }
@@ -338,6 +381,20 @@ bool make_tensor_map_bf16(CUtensorMap* map, const spindlekv_tensor& t, const spi
   return r == CUDA_SUCCESS;
 }
 
+// threshold / magnitude rows [2][units][rows_padded][16] bf16 -> 4-D map, box 16 x 128 rows, 32-byte swizzle
+static bool make_ext_map(CUtensorMap* map, const void* ext, int units, int rows_padded) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[4] = {16, (cuuint64_t)rows_padded, (cuuint64_t)units, 2};
+  cuuint64_t strides[3] = {32, (cuuint64_t)rows_padded * 32, (cuuint64_t)units * rows_padded * 32};
+  cuuint32_t box[4] = {16, 128, 1, 1};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ext), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_32B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
 bool sim_tc_available() {
   static int ok = -1;
   if (ok < 0) {
@@ -352,18 +409,17 @@ bool sim_tc_available() {
 }
 
 spindlekv_status launch_sim_tc(const spindlekv_tensor& Gamma, const spindlekv_batch& b, int n_kv_heads, int head_dim,
-                               float theta, const float* rinv, uint32_t* adj, uint32_t* hdr, cudaStream_t st) {
-  CUtensorMap map;
+                               const void* ext, uint32_t* adj, uint32_t* hdr, cudaStream_t st) {
+  const int units = b.n_layers * b.n_seqs * n_kv_heads;
+  CUtensorMap map, emap;
   if (!make_tensor_map_bf16(&map, Gamma, b, n_kv_heads, head_dim, 128)) return SPINDLEKV_CUDA;
+  if (!make_ext_map(&emap, ext, units, row_words_for(b.max_len) * 32)) return SPINDLEKV_CUDA;
   SimTcParams p;
   p.batch = make_batch(b);
   p.n_kv_heads = n_kv_heads;
   p.row_words = row_words_for(b.max_len);
-  p.theta = theta;
-  p.rinv = rinv;
   p.adj = adj;
   p.hdr = hdr;
-  const int units = b.n_layers * b.n_seqs * n_kv_heads;
   dim3 grid(ceil_div(b.max_len, kBM), units);
   LaunchScope ls(KC_SIM, st);
   if (head_dim == 128) {
@@ -373,7 +429,7 @@ spindlekv_status launch_sim_tc(const spindlekv_tensor& Gamma, const spindlekv_ba
         return SPINDLEKV_CUDA;
       set = true;
     }
-    sim_tc_kernel<128><<<grid, kSimThreads, SimSmem<128>::TOTAL, st>>>(map, p);
+    sim_tc_kernel<128><<<grid, kSimThreads, SimSmem<128>::TOTAL, st>>>(map, emap, p);
   } else {
     static bool set = false;
     if (!set) {
@@ -381,7 +437,7 @@ spindlekv_status launch_sim_tc(const spindlekv_tensor& Gamma, const spindlekv_ba
         return SPINDLEKV_CUDA;
       set = true;
     }
-    sim_tc_kernel<64><<<grid, kSimThreads, SimSmem<64>::TOTAL, st>>>(map, p);
+    sim_tc_kernel<64><<<grid, kSimThreads, SimSmem<64>::TOTAL, st>>>(map, emap, p);
   }
   return cudaGetLastError() == cudaSuccess ? SPINDLEKV_OK : SPINDLEKV_CUDA;
 }
