@@ -112,6 +112,11 @@ __device__ __forceinline__ bool epi_bar_all(bool ok) {
   return r != 0;
 }
 
+// Barrier over the four epilogue warps (one per TMEM lane quarter) that share a column group.
+__device__ __forceinline__ void epi_bar_group(int cg) {
+  asm volatile("bar.sync %0, %1;" ::"r"(2 + cg), "n"(128) : "memory");
+}
+
 // sign bits of 32 accumulators -> one word, bit c = sign of column c
 __device__ __forceinline__ uint32_t sign_word(const uint32_t (&acc)[32]) {
   // four independent 8-bit groups keep the shift chains short
@@ -227,7 +232,6 @@ __global__ void __launch_bounds__(kSimThreads, 1) sim_tc_kernel(const __grid_con
     const int q = warp & 3;               // TMEM lane quarter this warp may read
     const int cg = (warp - 2) >> 2;       // which group of kColsPerWarp tile columns
     const int ew = warp - 2;              // index among the epilogue warps
-    const int et = threadIdx.x - 64;      // index within the epilogue group
     const int rl = q * 32 + lane;         // row within the block
     const int R = row0 + q * 32;          // first row of this warp's 32-row strip
     const int row = R + lane;
@@ -237,11 +241,13 @@ __global__ void __launch_bounds__(kSimThreads, 1) sim_tc_kernel(const __grid_con
     tr.init(lane);
     // where this thread stages its direct words (advances by one tile's words, wraps per group)
     uint32_t* sd_mine = sD + rl * kDPitch + cg * kChunks;
-    // mirrored rows: thread et writes row c0 + et, 16 bytes at the block's column
-    uint32_t* mir = adj_unit + (int64_t)(tile0 * kBN + et) * RW + (row0 >> 5);
+    // mirrored rows: the first kColsPerWarp threads of a column group write one row each, 16 bytes at
+    // the block's column
+    uint32_t* mir = adj_unit + (int64_t)(tile0 * kBN + cg * kColsPerWarp + rl) * RW + (row0 >> 5);
     const int64_t mir_step = (int64_t)kBN * RW;
     const uint32_t tcol = tmem_base + ((uint32_t)(q * 32) << 16) + cg * kColsPerWarp;
     uint32_t* tq = sT + q * kBN + cg * kColsPerWarp + lane;
+    int ok_all = 1;
     for (int it = 0; tile0 + it < n_tiles; ++it, mir += mir_step) {
       const int st = it & 1;
       const int tile = tile0 + it;
@@ -250,10 +256,12 @@ __global__ void __launch_bounds__(kSimThreads, 1) sim_tc_kernel(const __grid_con
       const int gslot = (tile & (kGroupTiles - 1)) * (kBN / 32);
       uint32_t* sdbuf = sD + ((tile / kGroupTiles) & 1) * (kBM * kDPitch);
       uint32_t* sdw = sd_mine + ((tile / kGroupTiles) & 1) * (kBM * kDPitch) + gslot;
-      // one lane polls, the warp follows
+      // one lane polls, the warp follows; after a wait that gave up the warp keeps pace with the
+      // barriers below and everybody leaves together at the next flush
       int ok = 1;
       if (lane == 0) ok = ptx::mbar_wait(acc_full + st, (it >> 1) & 1, abort_flag) ? 1 : 0;
       ok = __shfl_sync(0xffffffffu, ok, 0);
+      ok_all &= ok;
       if (ok) {
         ptx::tc_fence_after();
         uint32_t words[kChunks];
@@ -304,13 +312,15 @@ __global__ void __launch_bounds__(kSimThreads, 1) sim_tc_kernel(const __grid_con
           }
         }
       }
-      // mirrored and direct words of this tile are in shared memory; everybody agrees to go on
-      if (!epi_bar_all(ok != 0)) break;
-      if (fast && et < kBN && c0 + et < l) {
-        const uint32_t* t0 = sT + st * 4 * kBN + et;
+      // the mirrored words of this column group are in shared memory
+      epi_bar_group(cg);
+      if (fast && rl < kColsPerWarp && c0 + cg * kColsPerWarp + rl < l) {
+        const uint32_t* t0 = sT + st * 4 * kBN + cg * kColsPerWarp + rl;
         *reinterpret_cast<uint4*>(mir) = make_uint4(t0[0], t0[kBN], t0[2 * kBN], t0[3 * kBN]);
       }
       if (gslot == (kGroupTiles - 1) * (kBN / 32) || tile == n_tiles - 1) {
+        // all column groups have staged their direct words; everybody agrees to go on
+        if (!epi_bar_all(ok_all != 0)) break;
         // direct rows of the last (up to) four tiles: one 128-byte segment per row, eight rows per warp;
         // words left of a row's diagonal sub-block belong to other blocks' mirrored writes
         const int wi = (tile & ~(kGroupTiles - 1)) * (kBN / 32) + lane;
