@@ -256,11 +256,10 @@ __global__ void __launch_bounds__(kSimThreads, 1) sim_tc_kernel(const __grid_con
       const int gslot = (tile & (kGroupTiles - 1)) * (kBN / 32);
       uint32_t* sdbuf = sD + ((tile / kGroupTiles) & 1) * (kBM * kDPitch);
       uint32_t* sdw = sd_mine + ((tile / kGroupTiles) & 1) * (kBM * kDPitch) + gslot;
-      // one lane polls, the warp follows; after a wait that gave up the warp keeps pace with the
-      // barriers below and everybody leaves together at the next flush
-      int ok = 1;
-      if (lane == 0) ok = ptx::mbar_wait(acc_full + st, (it >> 1) & 1, abort_flag) ? 1 : 0;
-      ok = __shfl_sync(0xffffffffu, ok, 0);
+      // after a wait that gave up the warp keeps pace with the barriers below and everybody leaves
+      // together at the next flush
+      int ok = ptx::mbar_wait(acc_full + st, (it >> 1) & 1, abort_flag) ? 1 : 0;
+      ok = __all_sync(0xffffffffu, ok);
       ok_all &= ok;
       if (ok) {
         ptx::tc_fence_after();
