@@ -306,6 +306,10 @@ static void launch_window(const EvictParams& p, int units, cudaStream_t st) {
   { LaunchScope ls(KC_WINDOW, st); win_colsum_kernel<T, D><<<grid, 256, 0, st>>>(p); }
 }
 
+bool win_tc_supported(const spindlekv_config& cfg, int dtype);
+spindlekv_status launch_win_tc(const spindlekv_config& cfg, const spindlekv_batch& b, const spindlekv_tensor& K,
+                               const spindlekv_tensor& Q, float* scores, uint32_t* hdr, cudaStream_t st);
+
 spindlekv_status evict_deep_impl(const spindlekv_config& cfg, const spindlekv_batch& b, const spindlekv_tensor& K,
                                  const spindlekv_tensor& Q, const int32_t* k_ctx, int32_t* keep_idx,
                                  int32_t* keep_cnt, float* scores, void* ws, size_t ws_bytes, cudaStream_t st) {
@@ -330,7 +334,11 @@ spindlekv_status evict_deep_impl(const spindlekv_config& cfg, const spindlekv_ba
   p.rowstat = reinterpret_cast<float2*>(w + kHeaderBytes + align_up((size_t)units * M * p.n_tiles * sizeof(float2), 256));
   p.scores = scores;
   const bool bf = K.dtype == SPINDLEKV_BF16;
-  if (cfg.head_dim == 64) {
+  if (win_tc_supported(cfg, K.dtype)) {
+    // bf16 with a window that tiles 128 rows: both passes on the tensor cores, one launch
+    spindlekv_status rs = launch_win_tc(cfg, b, K, Q, scores, reinterpret_cast<uint32_t*>(w), st);
+    if (rs != SPINDLEKV_OK) return rs;
+  } else if (cfg.head_dim == 64) {
     if (bf) launch_window<__nv_bfloat16, 64>(p, units, st); else launch_window<float, 64>(p, units, st);
   } else {
     if (bf) launch_window<__nv_bfloat16, 128>(p, units, st); else launch_window<float, 128>(p, units, st);

@@ -390,6 +390,26 @@ bool make_tensor_map_bf16(CUtensorMap* map, const spindlekv_tensor& t, const spi
   return r == CUDA_SUCCESS;
 }
 
+// bf16 window queries [layer][seq][q head][window row][d] -> 5-D map (d, row, head, seq, layer); one box is
+// 64 elements x `window` rows x 128/window heads: 128 operand rows (head-major) of 128 bytes
+bool make_query_map_bf16(CUtensorMap* map, const spindlekv_tensor& q, const spindlekv_batch& b, int n_q_heads,
+                         int head_dim, int window) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn || window <= 0 || 128 % window) return false;
+  auto bytes = [](int64_t elems) { return (cuuint64_t)(elems > 0 ? elems : 8) * 2; };
+  cuuint64_t dims[5] = {(cuuint64_t)head_dim, (cuuint64_t)window, (cuuint64_t)n_q_heads, (cuuint64_t)b.n_seqs,
+                        (cuuint64_t)b.n_layers};
+  cuuint64_t strides[4] = {bytes(q.stride_tok), bytes(q.stride_head), bytes(q.stride_seq), bytes(q.stride_layer)};
+  const int64_t st_el[5] = {1, q.stride_tok, q.stride_head, q.stride_seq, q.stride_layer};
+  for (int i = 1; i < 5; ++i)
+    if (dims[i] > 1 && st_el[i] <= 0) return false;
+  cuuint32_t box[5] = {64, (cuuint32_t)window, (cuuint32_t)(128 / window), 1, 1};
+  cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, q.ptr, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                  CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
 // threshold / magnitude rows [2][units][rows_padded][16] bf16 -> 4-D map, box 16 x 128 rows, 32-byte swizzle
 static bool make_ext_map(CUtensorMap* map, const void* ext, int units, int rows_padded) {
   EncodeTiledFn fn = encode_fn();

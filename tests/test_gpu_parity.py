@@ -118,6 +118,33 @@ def test_dense_and_sparse_rows_mixed():
     run_and_check(wl)
 
 
+def test_window_scores_on_tensor_cores_shapes():
+    # evicting layers only; every case takes the tensor-core window-score path (bf16, window divides 128)
+    cases = [
+        # 256 query rows per KV head (two 128-row blocks): 4 x 64 and 8 x 32; several tiles and a ragged tail
+        synth.Workload("qb2_w64", 2, 0, 8, 2, 128, "bf16", 64, (1100,), 30, (0.05, 0.3), 4, "recency",
+                       budget_tokens=300.0, seed=31),
+        synth.Workload("qb2_h8", 1, 0, 16, 2, 64, "bf16", 32, (700,), 30, (0.05, 0.3), 4, "recency",
+                       budget_tokens=200.0, seed=32),
+        # 192 rows: the second block is half padding; head_dim 64, window 16
+        synth.Workload("rows192", 1, 0, 12, 2, 128, "bf16", 32, (515,), 20, 0.2, 2, "gauss",
+                       budget_tokens=150.0, seed=33),
+        synth.Workload("d64_w16", 2, 0, 16, 4, 64, "bf16", 16, (640,), 20, 0.2, 2, "recency",
+                       budget_tokens=100.0, seed=34),
+        # fewer rows than one block (rows of the next group's heads are loaded and ignored); window 128
+        synth.Workload("rows64", 1, 0, 8, 4, 128, "bf16", 32, (400,), 20, 0.2, 2, "recency",
+                       budget_tokens=100.0, seed=35),
+        synth.Workload("w128", 1, 0, 2, 2, 64, "bf16", 128, (900,), 20, 0.2, 2, "gauss",
+                       budget_tokens=300.0, seed=36),
+        # packed sequences of very different lengths, one shorter than a tile, one a single tile plus one key
+        synth.Workload("packed_tc", 2, 0, 8, 2, 128, "bf16", 32, (100, 129, 1500, 128), 16, (0.05, 0.3), 2,
+                       "recency", budget_frac=0.5, seed=37),
+    ]
+    for wl in cases:
+        stats = run_and_check(wl)
+        assert stats["units"] == (wl.n_layers - wl.n_shallow) * wl.batch * wl.n_kv_heads
+
+
 def test_plain_window_sum_extension():
     wl = synth.Workload("rawsum", 1, 0, 4, 2, 64, "f32", 32, (333,), 8, 0.1, 2, "gauss", budget_tokens=80.0, seed=14)
     run_and_check(wl, {"score_norm": 1})
