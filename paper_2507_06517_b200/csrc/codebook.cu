@@ -33,8 +33,10 @@ struct CodebookParams {
   int32_t* owner;        // [units][max_len]
   int32_t* pickdeg;      // [units][max_len], -1 = not a centre
   int32_t* rank;         // [units][max_len] entry number of a centre
-  int32_t* ell;          // [units][max_len][kEll] neighbour lists of rows with few neighbours
+  int32_t* ell;          // [kEll][units][max_len] neighbour lists of rows with few neighbours, entry-major
   int32_t* ell_cnt;      // [units][max_len] list length, -1: use the bit row
+  int32_t* dense_rows;   // rows (unit * max_len + token) that use their bit row; count in the header
+  uint8_t* flags;        // [units][row_words/4][row_words*32] 0: that 128-column chunk of the row is empty
   uint32_t* hdr;
   int32_t* ref;          // [layers][H][T]
   int32_t* centre_idx;   // [layers][H][T]
@@ -189,90 +191,96 @@ __device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long v)
 }
 
 // ---- neighbour lists ------------------------------------------------------------------------------
-// One pass over the bit matrix: initial degrees (Eq. (10)), keys, and for every row with at most
-// kEll neighbours (itself not counted) the ascending list of those neighbours.  Rows with more
-// neighbours keep using their bit row.  One warp per row, 16-byte loads.
+// One thread per row.  The similarity kernel left one byte per (row, 128-column chunk) that says
+// whether the chunk may hold a set bit; only those chunks of the bit row are read.  Written per row:
+// the initial degree (Eq. (10)) and key, and, for rows with at most kEll neighbours (the row itself
+// not counted), the ascending list of those neighbours, stored entry-major (`ell[k][row]`) so that
+// the threads of a warp read consecutive words.  Rows with more neighbours keep using their bit row
+// and are appended to a list of dense rows.  A token with no neighbour at all is settled here: it is
+// a centre with pick degree 1 (Algorithm 1 reaches it with exactly that degree, whenever it does).
 constexpr int kEll = 32;
 
 __global__ void __launch_bounds__(256) extract_kernel(CodebookParams p) {
   const int lane = threadIdx.x & 31;
-  const int64_t gwarp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-  const int ML = p.batch.max_len, RW = p.row_words, RW4 = RW >> 2;
-  if (gwarp >= (int64_t)p.n_units * ML) return;
-  const int unit = (int)(gwarp / ML), u = (int)(gwarp % ML);
+  const int RW = p.row_words, NP = RW * 32, NB = RW >> 2, ML = p.batch.max_len;
+  const int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;   // over units x padded rows
+  if (g >= (int64_t)p.n_units * NP) return;
+  const int unit = (int)(g / NP), u = (int)(g - (int64_t)unit * NP);
   int layer, s, j;
   cb_decode(p, unit, layer, s, j);
-  if (u >= seq_len(p.batch, s)) return;
-  const uint4* row4 = reinterpret_cast<const uint4*>(p.adj + gwarp * RW);
-  int cnt = 0;
-  for (int w4 = lane; w4 < RW4; w4 += 32) {
-    uint4 a = row4[w4];
-    cnt += __popc(a.x) + __popc(a.y) + __popc(a.z) + __popc(a.w);
-  }
+  const int l = seq_len(p.batch, s);
+  bool live = false;
+  if (u < l) {
+    const int64_t idx = (int64_t)unit * ML + u;
+    const int64_t n_rows = (int64_t)p.n_units * ML;
+    const int blk = u >> 7;
+    const uint8_t* fl = p.flags + (int64_t)unit * NB * NP + u;
+    const uint4* row4 = reinterpret_cast<const uint4*>(p.adj + idx * RW);
+    int cnt = 1, k = 0;
+    for (int c0 = 0; c0 < NB; c0 += 32) {
+      // 32 flags at a time (independent loads), then only the occupied chunks
+      uint8_t f[32];
 #pragma unroll
-  for (int o = 16; o >= 1; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
-  if (lane == 0) {
-    p.deg[gwarp] = cnt;
-    p.key[gwarp] = ((unsigned long long)(uint32_t)cnt << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)u);
-    p.ell_cnt[gwarp] = cnt - 1 <= kEll ? cnt - 1 : -1;
-  }
-  if (cnt - 1 > kEll) return;
-  int32_t* ell = p.ell + gwarp * kEll;
-  int base = 0;
-  for (int w0 = 0; w0 < RW4; w0 += 32) {
-    const int w4 = w0 + lane;
-    uint32_t wd[4] = {0, 0, 0, 0};
-    if (w4 < RW4) {
-      uint4 a = row4[w4];
-      wd[0] = a.x; wd[1] = a.y; wd[2] = a.z; wd[3] = a.w;
-      if ((u >> 7) == w4) wd[(u >> 5) & 3] &= ~(1u << (u & 31));  // the token itself is not listed
-    }
-    const int c = __popc(wd[0]) + __popc(wd[1]) + __popc(wd[2]) + __popc(wd[3]);
-    int inc = c;
+      for (int c = 0; c < 32; ++c) f[c] = fl[(int64_t)min(c0 + c, NB - 1) * NP];
+      uint32_t occ = 0;
 #pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      int n = __shfl_up_sync(0xffffffffu, inc, o);
-      if (lane >= o) inc += n;
-    }
-    int pos = base + inc - c;
+      for (int c = 0; c < 32; ++c)
+        if (f[c]) occ |= 1u << c;
+      if (c0 + 32 > NB) occ &= (1u << (NB - c0)) - 1u;
+      while (occ) {
+      const int c = c0 + __ffs(occ) - 1;
+      occ &= occ - 1;
+      const uint4 a = row4[c];
+      uint32_t wd[4] = {a.x, a.y, a.z, a.w};
+      if (c == blk) wd[(u >> 5) & 3] &= ~(1u << (u & 31));   // the token itself is not listed
 #pragma unroll
-    for (int k = 0; k < 4; ++k) {
-      uint32_t m = wd[k];
-      while (m) {
-        int b = __ffs(m) - 1;
-        m &= m - 1;
-        ell[pos++] = w4 * 128 + k * 32 + b;
+      for (int q = 0; q < 4; ++q) {
+        uint32_t m = wd[q];
+        cnt += __popc(m);
+        while (m && k < kEll) {
+          const int b = __ffs(m) - 1;
+          m &= m - 1;
+          p.ell[(int64_t)k * n_rows + idx] = c * 128 + q * 32 + b;
+          ++k;
+        }
+      }
       }
     }
-    base += __shfl_sync(0xffffffffu, inc, 31);
+    p.deg[idx] = cnt;
+    p.key[idx] = ((unsigned long long)(uint32_t)cnt << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)u);
+    p.ell_cnt[idx] = cnt - 1 <= kEll ? cnt - 1 : -1;
+    if (cnt == 1) {
+      p.pickdeg[idx] = 1;
+      p.owner[idx] = u;
+    } else {
+      live = true;
+      if (cnt - 1 > kEll) p.dense_rows[atomicAdd(&p.hdr[kHdrDenseCnt], 1u)] = (int32_t)idx;
+    }
+  }
+  // all tokens that still have a neighbour start live (both copies of the mask)
+  const uint32_t word = __ballot_sync(0xffffffffu, live);
+  if (lane == 0) {
+    p.live0[(int64_t)unit * RW + (u >> 5)] = word;
+    p.live1[(int64_t)unit * RW + (u >> 5)] = word;
   }
 }
 
 // ---- greedy cover, cooperative kernel over all units of the call --------------------------------
+// Rows with a neighbour list are handled one per thread (a warp takes the 32 rows of one word of the
+// live mask and skips words that are empty), dense rows one per warp from their list.
+__device__ __forceinline__ bool is_live(const uint32_t* lv, int v) { return (lv[v >> 5] >> (v & 31)) & 1u; }
+
 __global__ void __launch_bounds__(512) greedy_kernel(CodebookParams p) {
   const int lane = threadIdx.x & 31;
   const int warps_per_block = blockDim.x >> 5;
   const int64_t gwarp = (int64_t)blockIdx.x * warps_per_block + (threadIdx.x >> 5);
   const int64_t nwarps = (int64_t)gridDim.x * warps_per_block;
   const int64_t gthread = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  const int64_t nthreads = (int64_t)gridDim.x * blockDim.x;
   const int ML = p.batch.max_len, RW = p.row_words, RW4 = RW >> 2;
   const int64_t n_rows = (int64_t)p.n_units * ML;
+  const int64_t n_words = (int64_t)p.n_units * RW;
+  const int n_dense = (int)*reinterpret_cast<volatile uint32_t*>(&p.hdr[kHdrDenseCnt]);
   uint32_t target = 0;
-
-  // all tokens start live (both copies of the mask)
-  for (int64_t i = gthread; i < (int64_t)p.n_units * RW; i += nthreads) {
-    int unit = (int)(i / RW), w = (int)(i % RW);
-    int layer, s, j;
-    cb_decode(p, unit, layer, s, j);
-    int l = seq_len(p.batch, s);
-    uint32_t m = 0;
-    if (w * 32 + 32 <= l) m = 0xFFFFFFFFu;
-    else if (w * 32 < l) m = (1u << (l - w * 32)) - 1u;
-    p.live0[i] = m;
-    p.live1[i] = m;
-  }
-  if (!grid_barrier(p.hdr, target)) return;
 
   int round = 0;
   for (; round <= ML; ++round) {
@@ -283,41 +291,41 @@ __global__ void __launch_bounds__(512) greedy_kernel(CodebookParams p) {
     if (round > 0) {
       // phase 1: live degrees (Eq. (10)) and keys; `next` becomes a copy of `live`.
       // (Round 0 uses the degrees and keys written with the neighbour lists.)
-      for (int64_t i = gthread; i < (int64_t)p.n_units * RW; i += nthreads) next[i] = live[i];
       if (gthread == 0) p.hdr[other] = 0;
       int my_live = 0;
-      for (int64_t idx = gwarp; idx < n_rows; idx += nwarps) {
-        int unit = (int)(idx / ML), u = (int)(idx - (int64_t)unit * ML);
-        const uint32_t* lv = live + (int64_t)unit * RW;
-        bool alive = (lv[u >> 5] >> (u & 31)) & 1u;  // bits beyond the sequence length are never set
-        if (!alive) {
-          if (lane == 0) p.key[idx] = 0ull;
-          continue;
-        }
+      for (int64_t w = gwarp; w < n_words; w += nwarps) {
+        const uint32_t lvw = live[w];
+        if (lane == 0) next[w] = lvw;
+        if (!lvw) continue;
+        my_live += __popc(lvw);
+        if (!((lvw >> lane) & 1u)) continue;
+        const int unit = (int)(w / RW), u = (int)(w - (int64_t)unit * RW) * 32 + lane;
+        const int64_t idx = (int64_t)unit * ML + u;
         const int ec = p.ell_cnt[idx];
-        int cnt;
-        if (ec >= 0) {
-          bool on = false;
-          if (lane < ec) {
-            int v = p.ell[idx * kEll + lane];
-            on = (lv[v >> 5] >> (v & 31)) & 1u;
-          }
-          cnt = 1 + __popc(__ballot_sync(0xffffffffu, on));
-        } else {
-          const uint4* row4 = reinterpret_cast<const uint4*>(p.adj + idx * RW);
-          const uint4* lv4 = reinterpret_cast<const uint4*>(lv);
-          cnt = 0;
-          for (int w4 = lane; w4 < RW4; w4 += 32) {
-            uint4 a = row4[w4], b = lv4[w4];
-            cnt += __popc(a.x & b.x) + __popc(a.y & b.y) + __popc(a.z & b.z) + __popc(a.w & b.w);
-          }
-#pragma unroll
-          for (int o = 16; o >= 1; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+        if (ec < 0) continue;                       // dense rows: below
+        const uint32_t* lv = live + (int64_t)unit * RW;
+        int cnt = 1;
+        for (int k = 0; k < ec; ++k) cnt += is_live(lv, p.ell[(int64_t)k * n_rows + idx]) ? 1 : 0;
+        p.deg[idx] = cnt;
+        p.key[idx] = ((unsigned long long)(uint32_t)cnt << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)u);
+      }
+      for (int64_t d = gwarp; d < n_dense; d += nwarps) {
+        const int64_t idx = p.dense_rows[d];
+        const int unit = (int)(idx / ML), u = (int)(idx - (int64_t)unit * ML);
+        const uint32_t* lv = live + (int64_t)unit * RW;
+        if (!is_live(lv, u)) continue;
+        const uint4* row4 = reinterpret_cast<const uint4*>(p.adj + idx * RW);
+        const uint4* lv4 = reinterpret_cast<const uint4*>(lv);
+        int cnt = 0;
+        for (int w4 = lane; w4 < RW4; w4 += 32) {
+          uint4 a = row4[w4], b = lv4[w4];
+          cnt += __popc(a.x & b.x) + __popc(a.y & b.y) + __popc(a.z & b.z) + __popc(a.w & b.w);
         }
+#pragma unroll
+        for (int o = 16; o >= 1; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
         if (lane == 0) {
           p.deg[idx] = cnt;
           p.key[idx] = ((unsigned long long)(uint32_t)cnt << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)u);
-          ++my_live;
         }
       }
       if (lane == 0 && my_live) atomicAdd(&p.hdr[slot], (uint32_t)my_live);
@@ -327,32 +335,40 @@ __global__ void __launch_bounds__(512) greedy_kernel(CodebookParams p) {
     }
 
     // phase 2: largest key in each closed live neighbourhood
-    for (int64_t idx = gwarp; idx < n_rows; idx += nwarps) {
-      int unit = (int)(idx / ML), u = (int)(idx - (int64_t)unit * ML);
-      const uint32_t* lv = live + (int64_t)unit * RW;
-      if (!((lv[u >> 5] >> (u & 31)) & 1u)) continue;
-      const unsigned long long* key = p.key + (int64_t)unit * ML;
+    for (int64_t w = gwarp; w < n_words; w += nwarps) {
+      const uint32_t lvw = live[w];
+      if (!((lvw >> lane) & 1u)) continue;
+      const int unit = (int)(w / RW), u = (int)(w - (int64_t)unit * RW) * 32 + lane;
+      const int64_t idx = (int64_t)unit * ML + u;
       const int ec = p.ell_cnt[idx];
+      if (ec < 0) continue;
+      const uint32_t* lv = live + (int64_t)unit * RW;
+      const unsigned long long* key = p.key + (int64_t)unit * ML;
+      unsigned long long best = key[u];             // the token itself belongs to its closed neighbourhood
+      for (int k = 0; k < ec; ++k) {
+        const int v = p.ell[(int64_t)k * n_rows + idx];
+        if (is_live(lv, v)) {
+          const unsigned long long kv = key[v];
+          best = kv > best ? kv : best;
+        }
+      }
+      p.m1[idx] = best;
+    }
+    for (int64_t d = gwarp; d < n_dense; d += nwarps) {
+      const int64_t idx = p.dense_rows[d];
+      const int unit = (int)(idx / ML), u = (int)(idx - (int64_t)unit * ML);
+      const uint32_t* lv = live + (int64_t)unit * RW;
+      if (!is_live(lv, u)) continue;
+      const unsigned long long* key = p.key + (int64_t)unit * ML;
+      const uint32_t* row = p.adj + idx * RW;
       unsigned long long best = 0ull;
-      if (ec >= 0) {
-        if (lane < ec) {
-          int v = p.ell[idx * kEll + lane];
-          if ((lv[v >> 5] >> (v & 31)) & 1u) best = key[v];
-        }
-        if (lane == 0) {  // the token itself belongs to its closed neighbourhood
-          unsigned long long own = key[u];
-          best = own > best ? own : best;
-        }
-      } else {
-        const uint32_t* row = p.adj + idx * RW;
-        for (int w = lane; w < RW; w += 32) {
-          uint32_t m = row[w] & lv[w];
-          while (m) {
-            int b = __ffs(m) - 1;
-            m &= m - 1;
-            unsigned long long kv = key[w * 32 + b];
-            best = kv > best ? kv : best;
-          }
+      for (int w = lane; w < RW; w += 32) {
+        uint32_t m = row[w] & lv[w];
+        while (m) {
+          int b = __ffs(m) - 1;
+          m &= m - 1;
+          unsigned long long kv = key[w * 32 + b];
+          best = kv > best ? kv : best;
         }
       }
       best = warp_max_u64(best);
@@ -362,54 +378,65 @@ __global__ void __launch_bounds__(512) greedy_kernel(CodebookParams p) {
 
     // phase 3: a node that is the maximum of every neighbour's neighbourhood is a centre (Eq. (11));
     // its live neighbours take it as owner (Eq. (12)) and leave the graph (Eq. (13))
-    for (int64_t idx = gwarp; idx < n_rows; idx += nwarps) {
-      int unit = (int)(idx / ML), u = (int)(idx - (int64_t)unit * ML);
+    for (int64_t w = gwarp; w < n_words; w += nwarps) {
+      const uint32_t lvw = live[w];
+      if (!((lvw >> lane) & 1u)) continue;
+      const int unit = (int)(w / RW), u = (int)(w - (int64_t)unit * RW) * 32 + lane;
+      const int64_t idx = (int64_t)unit * ML + u;
+      const int ec = p.ell_cnt[idx];
+      if (ec < 0) continue;
+      const unsigned long long mykey = p.key[idx];
+      if (p.m1[idx] != mykey) continue;
       const uint32_t* lv = live + (int64_t)unit * RW;
-      if (!((lv[u >> 5] >> (u & 31)) & 1u)) continue;
+      const unsigned long long* m1 = p.m1 + (int64_t)unit * ML;
+      bool ok = true;
+      for (int k = 0; k < ec && ok; ++k) {
+        const int v = p.ell[(int64_t)k * n_rows + idx];
+        if (is_live(lv, v) && m1[v] != mykey) ok = false;
+      }
+      if (!ok) continue;
+      int32_t* owner = p.owner + (int64_t)unit * ML;
+      uint32_t* nx = next + (int64_t)unit * RW;
+      for (int k = 0; k < ec; ++k) {
+        const int v = p.ell[(int64_t)k * n_rows + idx];
+        if (is_live(lv, v)) {
+          owner[v] = u;
+          atomicAnd(&nx[v >> 5], ~(1u << (v & 31)));
+        }
+      }
+      p.pickdeg[idx] = p.deg[idx];
+      owner[u] = u;
+      atomicAnd(&nx[u >> 5], ~(1u << (u & 31)));
+    }
+    for (int64_t d = gwarp; d < n_dense; d += nwarps) {
+      const int64_t idx = p.dense_rows[d];
+      const int unit = (int)(idx / ML), u = (int)(idx - (int64_t)unit * ML);
+      const uint32_t* lv = live + (int64_t)unit * RW;
+      if (!is_live(lv, u)) continue;
       const unsigned long long mykey = p.key[idx];
       if (p.m1[idx] != mykey) continue;
       const unsigned long long* m1 = p.m1 + (int64_t)unit * ML;
       int32_t* owner = p.owner + (int64_t)unit * ML;
       uint32_t* nx = next + (int64_t)unit * RW;
-      const int ec = p.ell_cnt[idx];
-      if (ec >= 0) {
-        int v = -1;
-        if (lane < ec) {
-          v = p.ell[idx * kEll + lane];
-          if (!((lv[v >> 5] >> (v & 31)) & 1u)) v = -1;
+      const uint32_t* row = p.adj + idx * RW;
+      bool ok = true;
+      for (int w = lane; w < RW; w += 32) {
+        uint32_t m = row[w] & lv[w];
+        while (m) {
+          int b = __ffs(m) - 1;
+          m &= m - 1;
+          if (m1[w * 32 + b] != mykey) ok = false;
         }
-        bool ok = v < 0 || m1[v] == mykey;
-        if (!__all_sync(0xffffffffu, ok)) continue;
-        if (v >= 0) {
-          owner[v] = u;
-          atomicAnd(&nx[v >> 5], ~(1u << (v & 31)));
-        }
-        if (lane == 0) {
-          p.pickdeg[idx] = p.deg[idx];
-          owner[u] = u;
-          atomicAnd(&nx[u >> 5], ~(1u << (u & 31)));
-        }
-      } else {
-        const uint32_t* row = p.adj + idx * RW;
-        bool ok = true;
-        for (int w = lane; w < RW; w += 32) {
-          uint32_t m = row[w] & lv[w];
-          while (m) {
-            int b = __ffs(m) - 1;
-            m &= m - 1;
-            if (m1[w * 32 + b] != mykey) ok = false;
-          }
-        }
-        if (!__all_sync(0xffffffffu, ok)) continue;
-        if (lane == 0) p.pickdeg[idx] = p.deg[idx];
-        for (int w = lane; w < RW; w += 32) {
-          uint32_t m = row[w] & lv[w];
-          if (m) atomicAnd(&nx[w], ~m);
-          while (m) {
-            int b = __ffs(m) - 1;
-            m &= m - 1;
-            owner[w * 32 + b] = u;
-          }
+      }
+      if (!__all_sync(0xffffffffu, ok)) continue;
+      if (lane == 0) p.pickdeg[idx] = p.deg[idx];
+      for (int w = lane; w < RW; w += 32) {
+        uint32_t m = row[w] & lv[w];
+        if (m) atomicAnd(&nx[w], ~m);
+        while (m) {
+          int b = __ffs(m) - 1;
+          m &= m - 1;
+          owner[w * 32 + b] = u;
         }
       }
     }
@@ -518,7 +545,7 @@ __global__ void __launch_bounds__(kFinalThreads) finalize_kernel(CodebookParams 
 // ---- host side ----------------------------------------------------------------------------------
 
 struct CodebookLayout {
-  size_t ext, ell, ell_cnt, adj, deg, key, m1, live0, live1, owner, pickdeg, rank, total;
+  size_t ext, ell, ell_cnt, dense_rows, flags, adj, deg, key, m1, live0, live1, owner, pickdeg, rank, total;
 };
 
 static CodebookLayout codebook_layout(const spindlekv_config& cfg, const spindlekv_batch& b, bool adj_in_ws) {
@@ -538,6 +565,8 @@ static CodebookLayout codebook_layout(const spindlekv_config& cfg, const spindle
   L.ext = take(2 * units * RW * 32 * 16 * 2);
   L.ell = take(units * ML * 32 * 4);
   L.ell_cnt = take(units * ML * 4);
+  L.dense_rows = take(units * ML * 4);
+  L.flags = take(units * (RW / 4) * RW * 32);
   L.adj = off;
   if (adj_in_ws) take(units * ML * RW * 4);
   L.total = off;
@@ -550,7 +579,7 @@ size_t codebook_workspace_bytes(const spindlekv_config& cfg, const spindlekv_bat
 
 bool sim_tc_available();
 spindlekv_status launch_sim_tc(const spindlekv_tensor& Gamma, const spindlekv_batch& b, int n_kv_heads, int head_dim,
-                               const void* ext, uint32_t* adj, uint32_t* hdr, cudaStream_t st);
+                               const void* ext, uint32_t* adj, uint8_t* flags, uint32_t* hdr, cudaStream_t st);
 
 template <typename T, int D>
 static void launch_norms(const CodebookParams& p, cudaStream_t st) {
@@ -595,6 +624,8 @@ spindlekv_status codebook_shallow_impl(const spindlekv_config& cfg, const spindl
   p.rank = reinterpret_cast<int32_t*>(w + L.rank);
   p.ell = reinterpret_cast<int32_t*>(w + L.ell);
   p.ell_cnt = reinterpret_cast<int32_t*>(w + L.ell_cnt);
+  p.dense_rows = reinterpret_cast<int32_t*>(w + L.dense_rows);
+  p.flags = reinterpret_cast<uint8_t*>(w + L.flags);
   p.hdr = reinterpret_cast<uint32_t*>(w);
   p.ref = ref;
   p.centre_idx = centre_idx;
@@ -610,16 +641,21 @@ spindlekv_status codebook_shallow_impl(const spindlekv_config& cfg, const spindl
     if (bf) launch_norms<__nv_bfloat16, 128>(p, st); else launch_norms<float, 128>(p, st);
   }
   if (tc) {
-    spindlekv_status rs = launch_sim_tc(Gamma, b, cfg.n_kv_heads, cfg.head_dim, p.ext, p.adj, p.hdr, st);
+    spindlekv_status rs = launch_sim_tc(Gamma, b, cfg.n_kv_heads, cfg.head_dim, p.ext, p.adj, p.flags, p.hdr, st);
     if (rs != SPINDLEKV_OK) return rs;
   } else if (cfg.head_dim == 64) {
     if (bf) launch_sim_simt<__nv_bfloat16, 64>(p, b, st); else launch_sim_simt<float, 64>(p, b, st);
   } else {
     if (bf) launch_sim_simt<__nv_bfloat16, 128>(p, b, st); else launch_sim_simt<float, 128>(p, b, st);
   }
+  if (!tc) {
+    // the CUDA-core similarity kernel writes no occupancy flags: every chunk counts as occupied
+    if (cudaMemsetAsync(p.flags, 1, (size_t)units * (p.row_words / 4) * p.row_words * 32, st) != cudaSuccess)
+      return SPINDLEKV_CUDA;
+  }
   {
     LaunchScope ls(KC_DEGREE, st);
-    extract_kernel<<<(unsigned)(((size_t)units * b.max_len * 32 + 255) / 256), 256, 0, st>>>(p);
+    extract_kernel<<<(unsigned)(((size_t)units * p.row_words * 32 + 255) / 256), 256, 0, st>>>(p);
   }
   // cooperative launch: as many blocks as can be resident at once
   static int coop_blocks = 0;

@@ -19,6 +19,7 @@ constexpr int kHdrLive = 2;
 constexpr int kHdrBarrier = 8;
 constexpr int kHdrLiveCnt0 = 9;   // two slots, alternated by round parity
 constexpr int kHdrLiveCnt1 = 10;
+constexpr int kHdrDenseCnt = 11;  // rows with too many neighbours for a list
 
 // kernel classes for launch counting / timing
 enum KernelClass { KC_WINDOW = 0, KC_TOPK, KC_NORMS, KC_SIM, KC_DEGREE, KC_GREEDY, KC_FINAL, KC_GATHER, KC_COUNT };

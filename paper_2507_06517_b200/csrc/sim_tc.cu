@@ -21,7 +21,10 @@
 // Direct words are staged in shared memory and leave in 128-byte row segments once every four
 // tiles; a 32x32 bit transpose across the warp turns the words of a sub-block into the words of the
 // mirrored rows, which are staged too and written 16 bytes per row.  Nothing but bits leaves the SM:
-// N*N/8 bytes per unit.
+// N*N/8 bytes per unit, plus one byte per (row, 128-column chunk) that says whether the chunk may hold
+// a set bit (0: certainly empty), so that the next kernel reads only the occupied part of a sparse
+// graph.  A chunk's flag (`flags[chunk][row]`) has exactly one writer: the row's own block for chunks at
+// or right of the diagonal, the block that mirrors into the row for chunks left of it.
 #include "common.cuh"
 #include "sm100_ptx.cuh"
 
@@ -31,6 +34,7 @@ struct SimTcParams {
   Batch batch;
   int n_kv_heads, row_words;
   uint32_t* adj;       // [units][max_len][row_words]
+  uint8_t* flags;      // [units][row_words / 4][row_words * 32]
   uint32_t* hdr;
 };
 
@@ -237,6 +241,16 @@ __global__ void __launch_bounds__(kSimThreads, 1) sim_tc_kernel(const __grid_con
     const int row = R + lane;
     const int RW = p.row_words;
     uint32_t* adj_unit = p.adj + (int64_t)unit * p.batch.max_len * RW;
+    const int NB = RW >> 2;               // 128-column chunks per row
+    const int blk = blockIdx.x;           // the chunk that holds this block's diagonal
+    uint8_t* funit = p.flags + (int64_t)unit * NB * (RW * 32);
+    uint8_t* fmir = funit + (int64_t)blk * (RW * 32);   // chunk `blk` of the rows this block mirrors into
+    if (!(blk & 1) && cg == 0) {
+      // an even block mirrors into the next block from its diagonal tile, sub-block by sub-block: those
+      // chunks are flagged as possibly occupied without looking
+      const int b = row0 + kBM + rl;
+      if (b < l) fmir[b] = 1;
+    }
     TransposeLane tr;
     tr.init(lane);
     // where this thread stages its direct words (advances by one tile's words, wraps per group)
@@ -315,7 +329,9 @@ __global__ void __launch_bounds__(kSimThreads, 1) sim_tc_kernel(const __grid_con
       epi_bar_group(cg);
       if (fast && rl < kColsPerWarp && c0 + cg * kColsPerWarp + rl < l) {
         const uint32_t* t0 = sT + st * 4 * kBN + cg * kColsPerWarp + rl;
-        *reinterpret_cast<uint4*>(mir) = make_uint4(t0[0], t0[kBN], t0[2 * kBN], t0[3 * kBN]);
+        const uint4 mv = make_uint4(t0[0], t0[kBN], t0[2 * kBN], t0[3 * kBN]);
+        *reinterpret_cast<uint4*>(mir) = mv;
+        fmir[c0 + cg * kColsPerWarp + rl] = (mv.x | mv.y | mv.z | mv.w) != 0u;
       }
       if (gslot == (kGroupTiles - 1) * (kBN / 32) || tile == n_tiles - 1) {
         // all column groups have staged their direct words; everybody agrees to go on
@@ -330,6 +346,18 @@ __global__ void __launch_bounds__(kSimThreads, 1) sim_tc_kernel(const __grid_con
 #pragma unroll
           for (int i = 0; i < kBM / kEpiWarps; ++i)
             if (row0 + r0 + i < l) dst[(int64_t)i * RW] = src[i * kDPitch];
+        }
+        // occupancy of the group's eight chunks: thread (row, chunk pair) reads the row's staged words
+        const int fr = (ew & 3) * 32 + lane;                       // row within the block
+        const int jc = (tile & ~(kGroupTiles - 1)) * (kBN / 128) + (ew >> 2) * 2;   // first chunk of the pair
+        if (row0 + fr < l) {
+          const uint2* sw = reinterpret_cast<const uint2*>(sdbuf + fr * kDPitch + (ew >> 2) * 8);
+#pragma unroll
+          for (int c = 0; c < 2; ++c) {
+            const uint2 x = sw[2 * c], y = sw[2 * c + 1];
+            if (jc + c >= blk && jc + c < NB)   // the chunk of the diagonal always holds the diagonal bit
+              funit[(int64_t)(jc + c) * (RW * 32) + row0 + fr] = jc + c == blk ? 1 : (x.x | x.y | y.x | y.y) != 0u;
+          }
         }
       }
     }
@@ -438,7 +466,7 @@ bool sim_tc_available() {
 }
 
 spindlekv_status launch_sim_tc(const spindlekv_tensor& Gamma, const spindlekv_batch& b, int n_kv_heads, int head_dim,
-                               const void* ext, uint32_t* adj, uint32_t* hdr, cudaStream_t st) {
+                               const void* ext, uint32_t* adj, uint8_t* flags, uint32_t* hdr, cudaStream_t st) {
   const int units = b.n_layers * b.n_seqs * n_kv_heads;
   CUtensorMap map, emap;
   if (!make_tensor_map_bf16(&map, Gamma, b, n_kv_heads, head_dim, 128)) return SPINDLEKV_CUDA;
@@ -448,6 +476,7 @@ spindlekv_status launch_sim_tc(const spindlekv_tensor& Gamma, const spindlekv_ba
   p.n_kv_heads = n_kv_heads;
   p.row_words = row_words_for(b.max_len);
   p.adj = adj;
+  p.flags = flags;
   p.hdr = hdr;
   dim3 grid(ceil_div(b.max_len, kBM), units);
   LaunchScope ls(KC_SIM, st);
