@@ -36,7 +36,7 @@ struct CodebookParams {
   int32_t* ell;          // [kEll][units][max_len] neighbour lists of rows with few neighbours, entry-major
   int32_t* ell_cnt;      // [units][max_len] list length, -1: use the bit row
   int32_t* dense_rows;   // rows (unit * max_len + token) that use their bit row; count in the header
-  uint8_t* flags;        // [units][row_words/4][row_words*32] 0: that 128-column chunk of the row is empty
+  uint32_t* flags;       // [units][row_words/2][row_words] bit r of word w: the 64-column chunk of row 32w+r may hold a bit
   uint32_t* hdr;
   int32_t* ref;          // [layers][H][T]
   int32_t* centre_idx;   // [layers][H][T]
@@ -149,7 +149,7 @@ __global__ void __launch_bounds__(256) sim_simt_kernel(CodebookParams p) {
   }
 }
 
-// ---- greedy cover, cooperative kernel over all units of the call --------------------------------
+// ---- grid-wide barrier and warp helpers of the cooperative greedy kernel ------------------------
 
 constexpr uint32_t kSpinLimit = 4u << 20;
 
@@ -191,8 +191,9 @@ __device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long v)
 }
 
 // ---- neighbour lists ------------------------------------------------------------------------------
-// One thread per row.  The similarity kernel left one byte per (row, 128-column chunk) that says
-// whether the chunk may hold a set bit; only those chunks of the bit row are read.  Written per row:
+// One thread per row.  The similarity kernel left one bit per (row, 64-column chunk) that says
+// whether the chunk may hold a set bit (a word holds the bits of 32 rows: a warp reads the words of 32
+// chunks and transposes them); only those chunks of the bit row are read.  Written per row:
 // the initial degree (Eq. (10)) and key, and, for rows with at most kEll neighbours (the row itself
 // not counted), the ascending list of those neighbours, stored entry-major (`ell[k][row]`) so that
 // the threads of a warp read consecutive words.  Rows with more neighbours keep using their bit row
@@ -202,50 +203,59 @@ constexpr int kEll = 32;
 
 __global__ void __launch_bounds__(256) extract_kernel(CodebookParams p) {
   const int lane = threadIdx.x & 31;
-  const int RW = p.row_words, NP = RW * 32, NB = RW >> 2, ML = p.batch.max_len;
+  const int RW = p.row_words, NP = RW * 32, NC = RW >> 1, ML = p.batch.max_len;
   const int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;   // over units x padded rows
-  if (g >= (int64_t)p.n_units * NP) return;
+  if (g >= (int64_t)p.n_units * NP) return;                           // whole warps: NP is a multiple of 32
   const int unit = (int)(g / NP), u = (int)(g - (int64_t)unit * NP);
   int layer, s, j;
   cb_decode(p, unit, layer, s, j);
   const int l = seq_len(p.batch, s);
-  bool live = false;
-  if (u < l) {
-    const int64_t idx = (int64_t)unit * ML + u;
-    const int64_t n_rows = (int64_t)p.n_units * ML;
-    const int blk = u >> 7;
-    const uint8_t* fl = p.flags + (int64_t)unit * NB * NP + u;
-    const uint4* row4 = reinterpret_cast<const uint4*>(p.adj + idx * RW);
-    int cnt = 1, k = 0;
-    for (int c0 = 0; c0 < NB; c0 += 32) {
-      // 32 flags at a time (independent loads), then only the occupied chunks
-      uint8_t f[32];
+  const bool exists = u < l;
+  const int64_t idx = (int64_t)unit * ML + (exists ? u : 0);
+  const int64_t n_rows = (int64_t)p.n_units * ML;
+  const int own = u >> 6;   // the chunk that holds the token's own bit
+  const uint32_t* fl = p.flags + (int64_t)unit * NC * RW + (u >> 5);
+  const uint2* row2 = reinterpret_cast<const uint2*>(p.adj + idx * RW);
+  TransposeLane tr;
+  tr.init(lane);
+  int cnt = 1, k = 0;
+  for (int c0 = 0; c0 < NC; c0 += 32) {
+    // lane c holds the flags of chunk c0 + c for the warp's 32 rows; after the transpose lane r holds
+    // the flags of its own row for these 32 chunks
+    uint32_t occ = tr.apply(c0 + lane < NC ? fl[(int64_t)(c0 + lane) * RW] : 0u);
+    if (!exists) occ = 0;
+    while (occ) {
+      // up to four occupied chunks at a time, loaded before any of them is looked at
+      int cs[4];
+      uint2 av[4];
 #pragma unroll
-      for (int c = 0; c < 32; ++c) f[c] = fl[(int64_t)min(c0 + c, NB - 1) * NP];
-      uint32_t occ = 0;
+      for (int i = 0; i < 4; ++i) {
+        cs[i] = occ ? c0 + __ffs(occ) - 1 : -1;
+        occ &= occ - 1;   // 0 stays 0
+      }
 #pragma unroll
-      for (int c = 0; c < 32; ++c)
-        if (f[c]) occ |= 1u << c;
-      if (c0 + 32 > NB) occ &= (1u << (NB - c0)) - 1u;
-      while (occ) {
-      const int c = c0 + __ffs(occ) - 1;
-      occ &= occ - 1;
-      const uint4 a = row4[c];
-      uint32_t wd[4] = {a.x, a.y, a.z, a.w};
-      if (c == blk) wd[(u >> 5) & 3] &= ~(1u << (u & 31));   // the token itself is not listed
+      for (int i = 0; i < 4; ++i) av[i] = cs[i] >= 0 ? row2[cs[i]] : make_uint2(0, 0);
 #pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        uint32_t m = wd[q];
-        cnt += __popc(m);
-        while (m && k < kEll) {
-          const int b = __ffs(m) - 1;
-          m &= m - 1;
-          p.ell[(int64_t)k * n_rows + idx] = c * 128 + q * 32 + b;
-          ++k;
+      for (int i = 0; i < 4; ++i) {
+        if (cs[i] < 0) continue;
+        const uint32_t wd[2] = {av[i].x, av[i].y};
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+          uint32_t m = wd[q];
+          if (cs[i] == own && q == ((u >> 5) & 1)) m &= ~(1u << (u & 31));   // the token itself is not listed
+          cnt += __popc(m);
+          while (m && k < kEll) {
+            const int b = __ffs(m) - 1;
+            m &= m - 1;
+            p.ell[(int64_t)k * n_rows + idx] = cs[i] * 64 + q * 32 + b;
+            ++k;
+          }
         }
       }
-      }
     }
+  }
+  bool live = false;
+  if (exists) {
     p.deg[idx] = cnt;
     p.key[idx] = ((unsigned long long)(uint32_t)cnt << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)u);
     p.ell_cnt[idx] = cnt - 1 <= kEll ? cnt - 1 : -1;
@@ -269,6 +279,23 @@ __global__ void __launch_bounds__(256) extract_kernel(CodebookParams p) {
 // Rows with a neighbour list are handled one per thread (a warp takes the 32 rows of one word of the
 // live mask and skips words that are empty), dense rows one per warp from their list.
 __device__ __forceinline__ bool is_live(const uint32_t* lv, int v) { return (lv[v >> 5] >> (v & 31)) & 1u; }
+
+// Eight entries of a row's neighbour list at a time: the loads of one batch do not depend on each
+// other, so a row costs a few memory round trips instead of one per neighbour.
+constexpr int kBatch = 8;
+__device__ __forceinline__ void load_batch(const int32_t* ell_row, int64_t n_rows, int k0, int ec, int (&v)[kBatch]) {
+#pragma unroll
+  for (int i = 0; i < kBatch; ++i) v[i] = k0 + i < ec ? ell_row[(int64_t)(k0 + i) * n_rows] : -1;
+}
+// keeps only the entries that are live (others become -1)
+__device__ __forceinline__ void keep_live(const uint32_t* lv, int (&v)[kBatch]) {
+  uint32_t w[kBatch];
+#pragma unroll
+  for (int i = 0; i < kBatch; ++i) w[i] = v[i] >= 0 ? lv[v[i] >> 5] : 0u;
+#pragma unroll
+  for (int i = 0; i < kBatch; ++i)
+    if (!((w[i] >> (v[i] & 31)) & 1u)) v[i] = -1;
+}
 
 __global__ void __launch_bounds__(512) greedy_kernel(CodebookParams p) {
   const int lane = threadIdx.x & 31;
@@ -305,7 +332,13 @@ __global__ void __launch_bounds__(512) greedy_kernel(CodebookParams p) {
         if (ec < 0) continue;                       // dense rows: below
         const uint32_t* lv = live + (int64_t)unit * RW;
         int cnt = 1;
-        for (int k = 0; k < ec; ++k) cnt += is_live(lv, p.ell[(int64_t)k * n_rows + idx]) ? 1 : 0;
+        for (int k0 = 0; k0 < ec; k0 += kBatch) {
+          int v[kBatch];
+          load_batch(p.ell + idx, n_rows, k0, ec, v);
+          keep_live(lv, v);
+#pragma unroll
+          for (int i = 0; i < kBatch; ++i) cnt += v[i] >= 0 ? 1 : 0;
+        }
         p.deg[idx] = cnt;
         p.key[idx] = ((unsigned long long)(uint32_t)cnt << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)u);
       }
@@ -345,12 +378,15 @@ __global__ void __launch_bounds__(512) greedy_kernel(CodebookParams p) {
       const uint32_t* lv = live + (int64_t)unit * RW;
       const unsigned long long* key = p.key + (int64_t)unit * ML;
       unsigned long long best = key[u];             // the token itself belongs to its closed neighbourhood
-      for (int k = 0; k < ec; ++k) {
-        const int v = p.ell[(int64_t)k * n_rows + idx];
-        if (is_live(lv, v)) {
-          const unsigned long long kv = key[v];
-          best = kv > best ? kv : best;
-        }
+      for (int k0 = 0; k0 < ec; k0 += kBatch) {
+        int v[kBatch];
+        load_batch(p.ell + idx, n_rows, k0, ec, v);
+        keep_live(lv, v);
+        unsigned long long kv[kBatch];
+#pragma unroll
+        for (int i = 0; i < kBatch; ++i) kv[i] = v[i] >= 0 ? key[v[i]] : 0ull;
+#pragma unroll
+        for (int i = 0; i < kBatch; ++i) best = kv[i] > best ? kv[i] : best;
       }
       p.m1[idx] = best;
     }
@@ -390,19 +426,29 @@ __global__ void __launch_bounds__(512) greedy_kernel(CodebookParams p) {
       const uint32_t* lv = live + (int64_t)unit * RW;
       const unsigned long long* m1 = p.m1 + (int64_t)unit * ML;
       bool ok = true;
-      for (int k = 0; k < ec && ok; ++k) {
-        const int v = p.ell[(int64_t)k * n_rows + idx];
-        if (is_live(lv, v) && m1[v] != mykey) ok = false;
+      for (int k0 = 0; k0 < ec && ok; k0 += kBatch) {
+        int v[kBatch];
+        load_batch(p.ell + idx, n_rows, k0, ec, v);
+        keep_live(lv, v);
+        unsigned long long mv[kBatch];
+#pragma unroll
+        for (int i = 0; i < kBatch; ++i) mv[i] = v[i] >= 0 ? m1[v[i]] : mykey;
+#pragma unroll
+        for (int i = 0; i < kBatch; ++i) ok = ok && mv[i] == mykey;
       }
       if (!ok) continue;
       int32_t* owner = p.owner + (int64_t)unit * ML;
       uint32_t* nx = next + (int64_t)unit * RW;
-      for (int k = 0; k < ec; ++k) {
-        const int v = p.ell[(int64_t)k * n_rows + idx];
-        if (is_live(lv, v)) {
-          owner[v] = u;
-          atomicAnd(&nx[v >> 5], ~(1u << (v & 31)));
-        }
+      for (int k0 = 0; k0 < ec; k0 += kBatch) {
+        int v[kBatch];
+        load_batch(p.ell + idx, n_rows, k0, ec, v);
+        keep_live(lv, v);
+#pragma unroll
+        for (int i = 0; i < kBatch; ++i)
+          if (v[i] >= 0) {
+            owner[v[i]] = u;
+            atomicAnd(&nx[v[i] >> 5], ~(1u << (v[i] & 31)));
+          }
       }
       p.pickdeg[idx] = p.deg[idx];
       owner[u] = u;
@@ -566,7 +612,7 @@ static CodebookLayout codebook_layout(const spindlekv_config& cfg, const spindle
   L.ell = take(units * ML * 32 * 4);
   L.ell_cnt = take(units * ML * 4);
   L.dense_rows = take(units * ML * 4);
-  L.flags = take(units * (RW / 4) * RW * 32);
+  L.flags = take(units * (RW / 2) * RW * 4);
   L.adj = off;
   if (adj_in_ws) take(units * ML * RW * 4);
   L.total = off;
@@ -579,7 +625,7 @@ size_t codebook_workspace_bytes(const spindlekv_config& cfg, const spindlekv_bat
 
 bool sim_tc_available();
 spindlekv_status launch_sim_tc(const spindlekv_tensor& Gamma, const spindlekv_batch& b, int n_kv_heads, int head_dim,
-                               const void* ext, uint32_t* adj, uint8_t* flags, uint32_t* hdr, cudaStream_t st);
+                               const void* ext, uint32_t* adj, uint32_t* flags, uint32_t* hdr, cudaStream_t st);
 
 template <typename T, int D>
 static void launch_norms(const CodebookParams& p, cudaStream_t st) {
@@ -625,7 +671,7 @@ spindlekv_status codebook_shallow_impl(const spindlekv_config& cfg, const spindl
   p.ell = reinterpret_cast<int32_t*>(w + L.ell);
   p.ell_cnt = reinterpret_cast<int32_t*>(w + L.ell_cnt);
   p.dense_rows = reinterpret_cast<int32_t*>(w + L.dense_rows);
-  p.flags = reinterpret_cast<uint8_t*>(w + L.flags);
+  p.flags = reinterpret_cast<uint32_t*>(w + L.flags);
   p.hdr = reinterpret_cast<uint32_t*>(w);
   p.ref = ref;
   p.centre_idx = centre_idx;
@@ -650,7 +696,7 @@ spindlekv_status codebook_shallow_impl(const spindlekv_config& cfg, const spindl
   }
   if (!tc) {
     // the CUDA-core similarity kernel writes no occupancy flags: every chunk counts as occupied
-    if (cudaMemsetAsync(p.flags, 1, (size_t)units * (p.row_words / 4) * p.row_words * 32, st) != cudaSuccess)
+    if (cudaMemsetAsync(p.flags, 0xFF, (size_t)units * (p.row_words / 2) * p.row_words * 4, st) != cudaSuccess)
       return SPINDLEKV_CUDA;
   }
   {

@@ -72,6 +72,35 @@ inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 __host__ __device__ inline int row_words_for(int max_len) { return 4 * ((max_len + 127) / 128); }
 
+// 32x32 bit transpose across a warp: in: lane r holds bits (r, c) at bit c; out: lane c holds bit r.
+// Five butterfly stages (j = 16, 8, 4, 2, 1): a lane takes from its partner the half of every 2j-bit
+// group that it does not keep, moved by j positions.  The move is a rotation (the bits that wrap
+// around fall outside the kept mask), so a stage is one shuffle, one funnel shift and one logic op;
+// rotation amounts and masks depend on the lane only and are set up once.
+struct TransposeLane {
+  uint32_t rot[5], keep[5];
+  __device__ __forceinline__ void init(int lane) {
+    uint32_t m = 0x0000FFFFu;
+#pragma unroll
+    for (int k = 0; k < 5; ++k) {
+      const int j = 16 >> k;
+      const bool hi = (lane & j) != 0;
+      keep[k] = hi ? ~m : m;
+      rot[k] = hi ? 32 - j : j;
+      m ^= m << (j >> 1);
+    }
+  }
+  __device__ __forceinline__ uint32_t apply(uint32_t x) const {
+#pragma unroll
+    for (int k = 0; k < 5; ++k) {
+      const uint32_t y = __shfl_xor_sync(0xffffffffu, x, 16 >> k);
+      const uint32_t r = __funnelshift_l(y, y, rot[k]);
+      x = (x & keep[k]) | (r & ~keep[k]);
+    }
+    return x;
+  }
+};
+
 // ---- launch bookkeeping (host) ---------------------------------------------------------------
 void note_launch(int kclass, cudaStream_t st, bool before);
 struct LaunchScope {

@@ -19,12 +19,13 @@
 // Sixteen epilogue warps read the accumulators back with tcgen05.ld while the tensor cores work on
 // the other TMEM stage.  A thread owns one row a and shifts the sign bits of 32 columns into a word.
 // Direct words are staged in shared memory and leave in 128-byte row segments once every four
-// tiles; a 32x32 bit transpose across the warp turns the words of a sub-block into the words of the
+// tiles (the four warps of a 32-row strip meet for that); a 32x32 bit transpose across the warp turns the words of a sub-block into the words of the
 // mirrored rows, which are staged too and written 16 bytes per row.  Nothing but bits leaves the SM:
-// N*N/8 bytes per unit, plus one byte per (row, 128-column chunk) that says whether the chunk may hold
+// N*N/8 bytes per unit, plus one bit per (row, 64-column chunk) that says whether the chunk may hold
 // a set bit (0: certainly empty), so that the next kernel reads only the occupied part of a sparse
-// graph.  A chunk's flag (`flags[chunk][row]`) has exactly one writer: the row's own block for chunks at
-// or right of the diagonal, the block that mirrors into the row for chunks left of it.
+// graph.  The flags of 32 consecutive rows and one chunk form a word (`flags[chunk][row / 32]`) with
+// exactly one writer: the rows' own block for chunks at or right of the block's own columns, the
+// block that mirrors into the rows for chunks left of them.
 #include "common.cuh"
 #include "sm100_ptx.cuh"
 
@@ -34,7 +35,7 @@ struct SimTcParams {
   Batch batch;
   int n_kv_heads, row_words;
   uint32_t* adj;       // [units][max_len][row_words]
-  uint8_t* flags;      // [units][row_words / 4][row_words * 32]
+  uint32_t* flags;     // [units][row_words / 2][row_words]
   uint32_t* hdr;
 };
 
@@ -72,53 +73,10 @@ struct SimSmem {
   static_assert(TOTAL <= 227 * 1024, "shared memory budget");
 };
 
-// 32x32 bit transpose across a warp: in: lane r holds bits (r, c) at bit c; out: lane c holds bit r.
-// Five butterfly stages (j = 16, 8, 4, 2, 1): a lane takes from its partner the half of every 2j-bit
-// group that it does not keep, moved by j positions.  The move is a rotation (the bits that wrap
-// around fall outside the kept mask), so a stage is one shuffle, one funnel shift and one logic op;
-// rotation amounts and masks depend on the lane only and are set up once.
-struct TransposeLane {
-  uint32_t rot[5], keep[5];
-  __device__ __forceinline__ void init(int lane) {
-    uint32_t m = 0x0000FFFFu;
-#pragma unroll
-    for (int k = 0; k < 5; ++k) {
-      const int j = 16 >> k;
-      const bool hi = (lane & j) != 0;
-      keep[k] = hi ? ~m : m;
-      rot[k] = hi ? 32 - j : j;
-      m ^= m << (j >> 1);
-    }
-  }
-  __device__ __forceinline__ uint32_t apply(uint32_t x) const {
-#pragma unroll
-    for (int k = 0; k < 5; ++k) {
-      const uint32_t y = __shfl_xor_sync(0xffffffffu, x, 16 >> k);
-      const uint32_t r = __funnelshift_l(y, y, rot[k]);
-      x = (x & keep[k]) | (r & ~keep[k]);
-    }
-    return x;
-  }
-};
-
-// Barrier over the epilogue warps that also agrees on whether everybody is still fine: returns
-// the AND of `ok` over all of them, so that they leave the tile loop together.
-__device__ __forceinline__ bool epi_bar_all(bool ok) {
-  uint32_t r;
-  asm volatile(
-      "{\n\t.reg .pred p, q;\n\t"
-      "setp.ne.u32 q, %1, 0;\n\t"
-      "bar.red.and.pred p, 1, %2, q;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(r)
-      : "r"((uint32_t)ok), "n"(kEpiThreads)
-      : "memory");
-  return r != 0;
-}
-
-// Barrier over the four epilogue warps (one per TMEM lane quarter) that share a column group.
-__device__ __forceinline__ void epi_bar_group(int cg) {
-  asm volatile("bar.sync %0, %1;" ::"r"(2 + cg), "n"(128) : "memory");
+// Barrier over four epilogue warps (128 threads): ids 2.. for the warps that share a column group,
+// ids 2 + kEpiWarps/4 .. for the warps that share a 32-row strip.
+__device__ __forceinline__ void epi_bar_named(int id) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "n"(128) : "memory");
 }
 
 // sign bits of 32 accumulators -> one word, bit c = sign of column c
@@ -235,21 +193,21 @@ __global__ void __launch_bounds__(kSimThreads, 1) sim_tc_kernel(const __grid_con
   } else {
     const int q = warp & 3;               // TMEM lane quarter this warp may read
     const int cg = (warp - 2) >> 2;       // which group of kColsPerWarp tile columns
-    const int ew = warp - 2;              // index among the epilogue warps
     const int rl = q * 32 + lane;         // row within the block
     const int R = row0 + q * 32;          // first row of this warp's 32-row strip
     const int row = R + lane;
     const int RW = p.row_words;
     uint32_t* adj_unit = p.adj + (int64_t)unit * p.batch.max_len * RW;
-    const int NB = RW >> 2;               // 128-column chunks per row
-    const int blk = blockIdx.x;           // the chunk that holds this block's diagonal
-    uint8_t* funit = p.flags + (int64_t)unit * NB * (RW * 32);
-    uint8_t* fmir = funit + (int64_t)blk * (RW * 32);   // chunk `blk` of the rows this block mirrors into
-    if (!(blk & 1) && cg == 0) {
-      // an even block mirrors into the next block from its diagonal tile, sub-block by sub-block: those
-      // chunks are flagged as possibly occupied without looking
-      const int b = row0 + kBM + rl;
-      if (b < l) fmir[b] = 1;
+    const int NC = RW >> 1;               // 64-column chunks per row
+    const int blk = blockIdx.x;
+    uint32_t* funit = p.flags + (int64_t)unit * NC * RW;
+    if (lane == 0) {
+      // The two chunks that hold the block's own 128 columns are flagged as occupied without looking:
+      // for the block's rows (diagonal bit, and words mirrored inside the block), and, from an even
+      // block, for the rows of the next block, which its diagonal tile mirrors into piecemeal.
+      const int chunk = 2 * blk + (cg & 1);
+      const int wb = (row0 >> 5) + (cg >> 1) * 4 + q;   // cg 0,1: own rows; cg 2,3: the next block's rows
+      if (chunk < NC && wb < RW && (cg < 2 || !(blk & 1))) funit[(int64_t)chunk * RW + wb] = 0xFFFFFFFFu;
     }
     TransposeLane tr;
     tr.init(lane);
@@ -261,7 +219,8 @@ __global__ void __launch_bounds__(kSimThreads, 1) sim_tc_kernel(const __grid_con
     const int64_t mir_step = (int64_t)kBN * RW;
     const uint32_t tcol = tmem_base + ((uint32_t)(q * 32) << 16) + cg * kColsPerWarp;
     uint32_t* tq = sT + q * kBN + cg * kColsPerWarp + lane;
-    int ok_all = 1;
+    // No early exit from this loop: after a wait that gave up (every later wait then returns at once)
+    // the warp still meets its partners at each barrier, with nothing to do in between.
     for (int it = 0; tile0 + it < n_tiles; ++it, mir += mir_step) {
       const int st = it & 1;
       const int tile = tile0 + it;
@@ -270,11 +229,7 @@ __global__ void __launch_bounds__(kSimThreads, 1) sim_tc_kernel(const __grid_con
       const int gslot = (tile & (kGroupTiles - 1)) * (kBN / 32);
       uint32_t* sdbuf = sD + ((tile / kGroupTiles) & 1) * (kBM * kDPitch);
       uint32_t* sdw = sd_mine + ((tile / kGroupTiles) & 1) * (kBM * kDPitch) + gslot;
-      // after a wait that gave up the warp keeps pace with the barriers below and everybody leaves
-      // together at the next flush
-      int ok = ptx::mbar_wait(acc_full + st, (it >> 1) & 1, abort_flag) ? 1 : 0;
-      ok = __all_sync(0xffffffffu, ok);
-      ok_all &= ok;
+      const bool ok = __all_sync(0xffffffffu, ptx::mbar_wait(acc_full + st, (it >> 1) & 1, abort_flag));
       if (ok) {
         ptx::tc_fence_after();
         uint32_t words[kChunks];
@@ -297,11 +252,14 @@ __global__ void __launch_bounds__(kSimThreads, 1) sim_tc_kernel(const __grid_con
             if (row >= l) words[ch] = 0;
           }
         }
+        if (c0 + cg * kColsPerWarp >= row0 + kBM) {
+          // this warp's 64 columns are one chunk right of the block's own columns: its flags for the strip
+          const uint32_t fw = __ballot_sync(0xffffffffu, (words[0] | words[kChunks - 1]) != 0u);
+          const int chunk = tile * (kBN / kColsPerWarp) + cg;
+          if (lane == 0 && chunk < NC) funit[(int64_t)chunk * RW + (R >> 5)] = fw;
+        }
         if (fast) {
-          if (kChunks == 2) *reinterpret_cast<uint2*>(sdw) = make_uint2(words[0], words[kChunks - 1]);
-          else
-#pragma unroll
-            for (int ch = 0; ch < kChunks; ++ch) sdw[ch] = words[ch];
+          *reinterpret_cast<uint2*>(sdw) = make_uint2(words[0], words[kChunks - 1]);
           // most 32 x 32 sub-blocks of a sparse graph are empty: their mirror image is too
 #pragma unroll
           for (int ch = 0; ch < kChunks; ++ch)
@@ -326,38 +284,33 @@ __global__ void __launch_bounds__(kSimThreads, 1) sim_tc_kernel(const __grid_con
         }
       }
       // the mirrored words of this column group are in shared memory
-      epi_bar_group(cg);
-      if (fast && rl < kColsPerWarp && c0 + cg * kColsPerWarp + rl < l) {
-        const uint32_t* t0 = sT + st * 4 * kBN + cg * kColsPerWarp + rl;
-        const uint4 mv = make_uint4(t0[0], t0[kBN], t0[2 * kBN], t0[3 * kBN]);
-        *reinterpret_cast<uint4*>(mir) = mv;
-        fmir[c0 + cg * kColsPerWarp + rl] = (mv.x | mv.y | mv.z | mv.w) != 0u;
+      epi_bar_named(2 + cg);
+      if (ok && fast && rl < kColsPerWarp) {   // whole warps: rl / 32 = q
+        const int b = c0 + cg * kColsPerWarp + rl;
+        bool occ_lo = false, occ_hi = false;
+        if (b < l) {
+          const uint32_t* t0 = sT + st * 4 * kBN + cg * kColsPerWarp + rl;
+          const uint4 mv = make_uint4(t0[0], t0[kBN], t0[2 * kBN], t0[3 * kBN]);
+          *reinterpret_cast<uint4*>(mir) = mv;
+          occ_lo = (mv.x | mv.y) != 0u;
+          occ_hi = (mv.z | mv.w) != 0u;
+        }
+        const uint32_t flo = __ballot_sync(0xffffffffu, occ_lo), fhi = __ballot_sync(0xffffffffu, occ_hi);
+        if (lane < 2 && (b >> 5) < RW) funit[(int64_t)(2 * blk + lane) * RW + (b >> 5)] = lane ? fhi : flo;
       }
       if (gslot == (kGroupTiles - 1) * (kBN / 32) || tile == n_tiles - 1) {
-        // all column groups have staged their direct words; everybody agrees to go on
-        if (!epi_bar_all(ok_all != 0)) break;
-        // direct rows of the last (up to) four tiles: one 128-byte segment per row, eight rows per warp;
-        // words left of a row's diagonal sub-block belong to other blocks' mirrored writes
+        // the four warps of this 32-row strip have staged their direct words of the last (up to) four
+        // tiles: one 128-byte segment per row, eight rows per warp; words left of the strip's diagonal
+        // sub-block belong to mirrored writes
+        epi_bar_named(2 + kEpiWarps / 4 + q);
         const int wi = (tile & ~(kGroupTiles - 1)) * (kBN / 32) + lane;
-        const int r0 = ew * (kBM / kEpiWarps);
-        if (wi >= ((row0 + (r0 & ~31)) >> 5) && wi < RW) {
+        const int r0 = q * 32 + cg * (32 / (kEpiWarps / 4));
+        if (wi >= (R >> 5) && wi < RW) {
           uint32_t* dst = adj_unit + (int64_t)(row0 + r0) * RW + wi;
           const uint32_t* src = sdbuf + r0 * kDPitch + lane;
 #pragma unroll
-          for (int i = 0; i < kBM / kEpiWarps; ++i)
+          for (int i = 0; i < 32 / (kEpiWarps / 4); ++i)
             if (row0 + r0 + i < l) dst[(int64_t)i * RW] = src[i * kDPitch];
-        }
-        // occupancy of the group's eight chunks: thread (row, chunk pair) reads the row's staged words
-        const int fr = (ew & 3) * 32 + lane;                       // row within the block
-        const int jc = (tile & ~(kGroupTiles - 1)) * (kBN / 128) + (ew >> 2) * 2;   // first chunk of the pair
-        if (row0 + fr < l) {
-          const uint2* sw = reinterpret_cast<const uint2*>(sdbuf + fr * kDPitch + (ew >> 2) * 8);
-#pragma unroll
-          for (int c = 0; c < 2; ++c) {
-            const uint2 x = sw[2 * c], y = sw[2 * c + 1];
-            if (jc + c >= blk && jc + c < NB)   // the chunk of the diagonal always holds the diagonal bit
-              funit[(int64_t)(jc + c) * (RW * 32) + row0 + fr] = jc + c == blk ? 1 : (x.x | x.y | y.x | y.y) != 0u;
-          }
         }
       }
     }
@@ -466,7 +419,7 @@ bool sim_tc_available() {
 }
 
 spindlekv_status launch_sim_tc(const spindlekv_tensor& Gamma, const spindlekv_batch& b, int n_kv_heads, int head_dim,
-                               const void* ext, uint32_t* adj, uint8_t* flags, uint32_t* hdr, cudaStream_t st) {
+                               const void* ext, uint32_t* adj, uint32_t* flags, uint32_t* hdr, cudaStream_t st) {
   const int units = b.n_layers * b.n_seqs * n_kv_heads;
   CUtensorMap map, emap;
   if (!make_tensor_map_bf16(&map, Gamma, b, n_kv_heads, head_dim, 128)) return SPINDLEKV_CUDA;
