@@ -16,11 +16,14 @@
 // a.b / (|a||b|) > theta.  The epilogue therefore only collects sign bits: no per-column operand,
 // no floating-point instruction.
 //
-// Sixteen epilogue warps read the accumulators back with tcgen05.ld while the tensor cores work on
-// the other TMEM stage.  A thread owns one row a and shifts the sign bits of 32 columns into a word.
-// Direct words are staged in shared memory and leave in 128-byte row segments once every four
-// tiles (the four warps of a 32-row strip meet for that); a 32x32 bit transpose across the warp turns the words of a sub-block into the words of the
-// mirrored rows, which are staged too and written 16 bytes per row.  Nothing but bits leaves the SM:
+// Sixteen epilogue warps in two teams of eight read the accumulators back with tcgen05.ld; team e
+// serves TMEM stage e, i.e. every other tile, so that two tiles are in the epilogue at once while the
+// tensor cores fill the stage that was released first.  Inside a team a warp owns a 32-row strip and
+// half of the tile's columns; a thread owns one row a and shifts the sign bits of 32 columns into a
+// word.  Direct words are staged in shared memory and leave in 32-byte pieces, two per row, after the
+// team's two tiles of a four-tile span (the two warps of a strip meet for that); a 32x32 bit transpose
+// across the warp turns the words of a sub-block into the words of the mirrored rows, which are
+// staged too and written 16 bytes per row by the whole team.  Nothing but bits leaves the SM:
 // N*N/8 bytes per unit, plus one bit per (row, 64-column chunk) that says whether the chunk may hold
 // a set bit (0: certainly empty), so that the next kernel reads only the occupied part of a sparse
 // graph.  The flags of 32 consecutive rows and one chunk form a word (`flags[chunk][row / 32]`) with
@@ -42,15 +45,14 @@ struct SimTcParams {
 constexpr int kBM = 128;          // rows of the resident block (UMMA M)
 constexpr int kBN = 256;          // rows of a streamed tile (UMMA N)
 constexpr int kStages = 2;
-constexpr int kEpiWarps = 16;
-constexpr int kColsPerWarp = kBN / (kEpiWarps / 4);   // tile columns handled by one epilogue warp
+constexpr int kEpiWarps = 16;                         // two teams of eight; team e serves TMEM stage e
+constexpr int kTeamWarps = kEpiWarps / 2;
+constexpr int kColsPerWarp = kBN / (kTeamWarps / 4);  // tile columns handled by one epilogue warp
 constexpr int kChunks = kColsPerWarp / 32;
-constexpr int kEpiThreads = 32 * kEpiWarps;
 constexpr int kSimThreads = 32 * (2 + kEpiWarps);
-constexpr int kGroupTiles = 4;                        // direct rows are flushed once per this many tiles
-constexpr int kGroupWords = kGroupTiles * kBN / 32;   // 32 words = 128 bytes of a row
-constexpr int kDPitch = kGroupWords + 2;              // row pitch of the staging buffer in words
-static_assert(kChunks == 2 && kGroupWords == 32, "epilogue layout assumes 64 columns per warp and 128-byte flushes");
+constexpr int kTileWords = kBN / 32;                  // words of a row per tile
+constexpr int kDPitch = 2 * kTileWords + 2;           // staging pitch: a team's two tiles of a four-tile span
+static_assert(kChunks == 4 && kTileWords == 8, "epilogue layout assumes 128 columns per warp");
 
 template <int D>
 struct SimSmem {
@@ -60,7 +62,7 @@ struct SimSmem {
   static constexpr int EA_BYTES = kBM * 32;          // threshold rows of the block (one 16-element K-step)
   static constexpr int EB_BYTES = kBN * 32;          // magnitude rows of a tile
   static constexpr int T_BYTES = 2 * 4 * kBN * 4;    // mirrored words [slot][row quarter][tile column]
-  static constexpr int D_BYTES = 2 * kBM * kDPitch * 4;  // direct words [slot][row][word of the group]
+  static constexpr int D_BYTES = 2 * 2 * kBM * kDPitch * 4;  // direct words [team][slot][row][word]
   static constexpr int OFF_B = A_BYTES;
   static constexpr int OFF_EA = OFF_B + kStages * B_BYTES;
   static constexpr int OFF_EB = OFF_EA + EA_BYTES;
@@ -73,10 +75,10 @@ struct SimSmem {
   static_assert(TOTAL <= 227 * 1024, "shared memory budget");
 };
 
-// Barrier over four epilogue warps (128 threads): ids 2.. for the warps that share a column group,
-// ids 2 + kEpiWarps/4 .. for the warps that share a 32-row strip.
-__device__ __forceinline__ void epi_bar_named(int id) {
-  asm volatile("bar.sync %0, %1;" ::"r"(id), "n"(128) : "memory");
+// Named barrier over some of the epilogue warps: ids 2, 3 for a whole team (256 threads), ids 4..11 for
+// the two warps of a team that share a 32-row strip (64 threads).
+__device__ __forceinline__ void epi_bar_n(int id, int nthreads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
 }
 
 // sign bits of 32 accumulators -> one word, bit c = sign of column c
@@ -125,7 +127,7 @@ __global__ void __launch_bounds__(kSimThreads, 1) sim_tc_kernel(const __grid_con
   if (threadIdx.x == 0) {
     ptx::mbar_init(a_full, 1);
     for (int i = 0; i < kStages; ++i) { ptx::mbar_init(b_full + i, 1); ptx::mbar_init(b_empty + i, 1); }
-    for (int i = 0; i < 2; ++i) { ptx::mbar_init(acc_full + i, 1); ptx::mbar_init(acc_empty + i, kEpiWarps); }
+    for (int i = 0; i < 2; ++i) { ptx::mbar_init(acc_full + i, 1); ptx::mbar_init(acc_empty + i, kTeamWarps); }
     *abort_flag = 0;
     ptx::fence_barrier_init();
   }
@@ -192,7 +194,9 @@ __global__ void __launch_bounds__(kSimThreads, 1) sim_tc_kernel(const __grid_con
     }
   } else {
     const int q = warp & 3;               // TMEM lane quarter this warp may read
-    const int cg = (warp - 2) >> 2;       // which group of kColsPerWarp tile columns
+    const int team = (warp - 2) >> 3;     // which TMEM stage this warp serves
+    const int cg = ((warp - 2) >> 2) & 1; // which half of the tile's columns
+    const int tt = ((warp - 2) & 7) * 32 + lane;   // thread index within the team
     const int rl = q * 32 + lane;         // row within the block
     const int R = row0 + q * 32;          // first row of this warp's 32-row strip
     const int row = R + lane;
@@ -205,44 +209,40 @@ __global__ void __launch_bounds__(kSimThreads, 1) sim_tc_kernel(const __grid_con
       // The two chunks that hold the block's own 128 columns are flagged as occupied without looking:
       // for the block's rows (diagonal bit, and words mirrored inside the block), and, from an even
       // block, for the rows of the next block, which its diagonal tile mirrors into piecemeal.
-      const int chunk = 2 * blk + (cg & 1);
-      const int wb = (row0 >> 5) + (cg >> 1) * 4 + q;   // cg 0,1: own rows; cg 2,3: the next block's rows
-      if (chunk < NC && wb < RW && (cg < 2 || !(blk & 1))) funit[(int64_t)chunk * RW + wb] = 0xFFFFFFFFu;
+      const int chunk = 2 * blk + cg;
+      const int wb = (row0 >> 5) + team * 4 + q;   // team 0: own rows; team 1: the next block's rows
+      if (chunk < NC && wb < RW && (team == 0 || !(blk & 1))) funit[(int64_t)chunk * RW + wb] = 0xFFFFFFFFu;
     }
     TransposeLane tr;
     tr.init(lane);
-    // where this thread stages its direct words (advances by one tile's words, wraps per group)
-    uint32_t* sd_mine = sD + rl * kDPitch + cg * kChunks;
-    // mirrored rows: the first kColsPerWarp threads of a column group write one row each, 16 bytes at
-    // the block's column
-    uint32_t* mir = adj_unit + (int64_t)(tile0 * kBN + cg * kColsPerWarp + rl) * RW + (row0 >> 5);
-    const int64_t mir_step = (int64_t)kBN * RW;
-    const uint32_t tcol = tmem_base + ((uint32_t)(q * 32) << 16) + cg * kColsPerWarp;
-    uint32_t* tq = sT + q * kBN + cg * kColsPerWarp + lane;
+    uint32_t* sD_team = sD + team * (2 * kBM * kDPitch);
+    // mirrored rows: thread tt of the team writes row c0 + tt, 16 bytes at the block's column
+    const uint32_t tcol = tmem_base + ((uint32_t)(q * 32) << 16) + team * kBN + cg * kColsPerWarp;
+    uint32_t* tq = sT + (team * 4 + q) * kBN + cg * kColsPerWarp + lane;
+    const uint32_t* tr0 = sT + team * 4 * kBN + tt;
     // No early exit from this loop: after a wait that gave up (every later wait then returns at once)
     // the warp still meets its partners at each barrier, with nothing to do in between.
-    for (int it = 0; tile0 + it < n_tiles; ++it, mir += mir_step) {
-      const int st = it & 1;
+    for (int it = team; tile0 + it < n_tiles; it += 2) {
       const int tile = tile0 + it;
       const int c0 = tile * kBN;
       const bool fast = c0 >= row0 + kBM;      // whole tile strictly above the diagonal
-      const int gslot = (tile & (kGroupTiles - 1)) * (kBN / 32);
-      uint32_t* sdbuf = sD + ((tile / kGroupTiles) & 1) * (kBM * kDPitch);
-      uint32_t* sdw = sd_mine + ((tile / kGroupTiles) & 1) * (kBM * kDPitch) + gslot;
-      const bool ok = __all_sync(0xffffffffu, ptx::mbar_wait(acc_full + st, (it >> 1) & 1, abort_flag));
+      const int slot = (tile >> 1) & 1;        // which of the team's two tiles of the four-tile span
+      uint32_t* sdbuf = sD_team + ((tile >> 2) & 1) * (kBM * kDPitch);
+      uint32_t* sdw = sdbuf + rl * kDPitch + slot * kTileWords + cg * kChunks;
+      const bool ok = __all_sync(0xffffffffu, ptx::mbar_wait(acc_full + team, (it >> 1) & 1, abort_flag));
       if (ok) {
         ptx::tc_fence_after();
         uint32_t words[kChunks];
 #pragma unroll
         for (int ch = 0; ch < kChunks; ++ch) {
           uint32_t acc[32];
-          ptx::tmem_ld_32x32(tcol + st * kBN + ch * 32, acc);
+          ptx::tmem_ld_32x32(tcol + ch * 32, acc);
           ptx::tmem_ld_wait(acc);
           words[ch] = sign_word(acc);
         }
         ptx::tc_fence_before();
         __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(acc_empty + st);
+        if (lane == 0) ptx::mbar_arrive(acc_empty + team);
         if (c0 + kBN > l || R + 32 > l) {
           // ragged edge: columns and rows that do not exist carry no bits
 #pragma unroll
@@ -253,17 +253,19 @@ __global__ void __launch_bounds__(kSimThreads, 1) sim_tc_kernel(const __grid_con
           }
         }
         if (c0 + cg * kColsPerWarp >= row0 + kBM) {
-          // this warp's 64 columns are one chunk right of the block's own columns: its flags for the strip
-          const uint32_t fw = __ballot_sync(0xffffffffu, (words[0] | words[kChunks - 1]) != 0u);
-          const int chunk = tile * (kBN / kColsPerWarp) + cg;
-          if (lane == 0 && chunk < NC) funit[(int64_t)chunk * RW + (R >> 5)] = fw;
+          // this warp's two 64-column chunks lie right of the block's own columns: their flags for the strip
+          const uint32_t f0 = __ballot_sync(0xffffffffu, (words[0] | words[1]) != 0u);
+          const uint32_t f1 = __ballot_sync(0xffffffffu, (words[2] | words[3]) != 0u);
+          const int chunk = tile * 4 + cg * 2 + lane;
+          if (lane < 2 && chunk < NC) funit[(int64_t)chunk * RW + (R >> 5)] = lane ? f1 : f0;
         }
         if (fast) {
-          *reinterpret_cast<uint2*>(sdw) = make_uint2(words[0], words[kChunks - 1]);
+          *reinterpret_cast<uint2*>(sdw) = make_uint2(words[0], words[1]);
+          *reinterpret_cast<uint2*>(sdw + 2) = make_uint2(words[2], words[3]);
           // most 32 x 32 sub-blocks of a sparse graph are empty: their mirror image is too
 #pragma unroll
           for (int ch = 0; ch < kChunks; ++ch)
-            tq[st * 4 * kBN + ch * 32] = __any_sync(0xffffffffu, words[ch] != 0u) ? tr.apply(words[ch]) : 0u;
+            tq[ch * 32] = __any_sync(0xffffffffu, words[ch] != 0u) ? tr.apply(words[ch]) : 0u;
         } else {
 #pragma unroll
           for (int ch = 0; ch < kChunks; ++ch) {
@@ -283,33 +285,34 @@ __global__ void __launch_bounds__(kSimThreads, 1) sim_tc_kernel(const __grid_con
           }
         }
       }
-      // the mirrored words of this column group are in shared memory
-      epi_bar_named(2 + cg);
-      if (ok && fast && rl < kColsPerWarp) {   // whole warps: rl / 32 = q
-        const int b = c0 + cg * kColsPerWarp + rl;
+      // the team's mirrored words of this tile are in shared memory
+      epi_bar_n(2 + team, 32 * kTeamWarps);
+      if (ok && fast) {
+        const int b = c0 + tt;
         bool occ_lo = false, occ_hi = false;
         if (b < l) {
-          const uint32_t* t0 = sT + st * 4 * kBN + cg * kColsPerWarp + rl;
-          const uint4 mv = make_uint4(t0[0], t0[kBN], t0[2 * kBN], t0[3 * kBN]);
-          *reinterpret_cast<uint4*>(mir) = mv;
+          const uint4 mv = make_uint4(tr0[0], tr0[kBN], tr0[2 * kBN], tr0[3 * kBN]);
+          *reinterpret_cast<uint4*>(adj_unit + (int64_t)b * RW + (row0 >> 5)) = mv;
           occ_lo = (mv.x | mv.y) != 0u;
           occ_hi = (mv.z | mv.w) != 0u;
         }
         const uint32_t flo = __ballot_sync(0xffffffffu, occ_lo), fhi = __ballot_sync(0xffffffffu, occ_hi);
         if (lane < 2 && (b >> 5) < RW) funit[(int64_t)(2 * blk + lane) * RW + (b >> 5)] = lane ? fhi : flo;
       }
-      if (gslot == (kGroupTiles - 1) * (kBN / 32) || tile == n_tiles - 1) {
-        // the four warps of this 32-row strip have staged their direct words of the last (up to) four
-        // tiles: one 128-byte segment per row, eight rows per warp; words left of the strip's diagonal
-        // sub-block belong to mirrored writes
-        epi_bar_named(2 + kEpiWarps / 4 + q);
-        const int wi = (tile & ~(kGroupTiles - 1)) * (kBN / 32) + lane;
-        const int r0 = q * 32 + cg * (32 / (kEpiWarps / 4));
+      if (slot == 1 || tile + 2 >= n_tiles) {
+        // the two warps of the team that share this 32-row strip have staged their direct words of the
+        // team's (up to) two tiles of this four-tile span: two 32-byte pieces per row, sixteen rows per
+        // warp, two rows per store; words left of the strip's diagonal sub-block belong to mirrored writes
+        epi_bar_n(4 + team * 4 + q, 64);
+        const int half = lane >> 4, wl = lane & 15;           // row of the pair, word of the row's 16
+        const int wtile = (tile & ~3) + (tile & 1) + 2 * (wl >> 3);   // the tile this word belongs to
+        const int wi = wtile * kTileWords + (wl & 7);
+        const int r0 = q * 32 + cg * 16 + half;
         if (wi >= (R >> 5) && wi < RW) {
           uint32_t* dst = adj_unit + (int64_t)(row0 + r0) * RW + wi;
-          const uint32_t* src = sdbuf + r0 * kDPitch + lane;
+          const uint32_t* src = sdbuf + r0 * kDPitch + wl;
 #pragma unroll
-          for (int i = 0; i < 32 / (kEpiWarps / 4); ++i)
+          for (int i = 0; i < 16; i += 2)
             if (row0 + r0 + i < l) dst[(int64_t)i * RW] = src[i * kDPitch];
         }
       }
