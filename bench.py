@@ -327,6 +327,26 @@ def run_native(args, wl):
     total_ms = sum(v[0] for v in kt.values()) or 1.0
     kernels = {k: {"ms_per_step": v[0] / args.steps, "launches_per_step": v[1] / args.steps,
                    "share": v[0] / total_ms} for k, v in kt.items() if v[1]}
+    # algorithmic bytes per step of the bandwidth-bound kernels (what must move at least once) against
+    # the measured HBM copy rate
+    e = 4 if wl.dtype == "f32" else 2
+    tok, Hk, d = wl.total_tokens, wl.n_kv_heads, wl.head_dim
+    nd, ns = wl.n_layers - wl.n_shallow, wl.n_shallow
+    alg = {}
+    if nd:
+        kept = int(p.keep_cnt.sum().item())
+        alg["window_score"] = nd * (tok * Hk * d * e + wl.batch * wl.n_q_heads * wl.window * d * e + 4 * Hk * tok)
+        alg["topk"] = nd * Hk * 4 * tok + 4 * kept
+        alg["gather"] = 2 * 2 * kept * d * e
+    if ns:
+        entries = sum(int(p.cb[g]["n_entries"].sum().item()) for g in ("K", "V"))
+        alg["norms"] = 2 * ns * (tok * Hk * d * e + 4 * Hk * tok)
+        alg["gather"] = alg.get("gather", 0) + 2 * entries * d * e
+    for k, nbytes in alg.items():
+        if k in kernels and kernels[k]["ms_per_step"] > 0:
+            gbs = nbytes / (kernels[k]["ms_per_step"] * 1e-3) / 1e9
+            kernels[k].update({"bound": "hbm", "algorithmic_bytes": nbytes, "achieved_gbs": gbs,
+                               "frac_of_hbm_peak": gbs / pk["hbm_gbs"]})
     roof = None
     if p.n_shallow and kt["similarity"][1]:
         sim_ms, sim_n = kt["similarity"]

@@ -63,6 +63,8 @@ __device__ __forceinline__ void split3_bf16(float x, __nv_bfloat16 (&pc)[3]) {
   }
 }
 
+constexpr int kNormRows = 4;   // rows per thread group: their loads are all in flight before any is used
+
 template <typename T, int D>
 __global__ void __launch_bounds__(256) norms_kernel(CodebookParams p) {
   constexpr int LPR = D / 8;  // lanes per row
@@ -70,37 +72,47 @@ __global__ void __launch_bounds__(256) norms_kernel(CodebookParams p) {
   int layer, s, j;
   cb_decode(p, blockIdx.y, layer, s, j);
   const int l = seq_len(p.batch, s);
-  int row = blockIdx.x * RPB + threadIdx.x / LPR;
-  int seg = threadIdx.x % LPR;
-  float ss = 0.f;
-  if (row < l) {
-    const T* src = reinterpret_cast<const T*>(p.G.ptr) + unit_offset(p.G, p.batch, layer, s, j) + (int64_t)row * p.G.st;
-    float v[8];
-    load8(src + seg * 8, v);
+  const int seg = threadIdx.x % LPR;
+  const int row_first = blockIdx.x * (RPB * kNormRows) + threadIdx.x / LPR;
+  const T* base = reinterpret_cast<const T*>(p.G.ptr) + unit_offset(p.G, p.batch, layer, s, j) + seg * 8;
+  float v[kNormRows][8];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) ss = fmaf(v[i], v[i], ss);
+  for (int r = 0; r < kNormRows; ++r) {
+    const int row = row_first + r * RPB;
+    if (row < l) load8(base + (int64_t)row * p.G.st, v[r]);
+    else {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) v[r][i] = 0.f;
+    }
   }
 #pragma unroll
-  for (int o = LPR / 2; o >= 1; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-  const float m = sqrtf(ss);
-  if (seg == 0 && row < l) p.mag[cb_out_row(p, layer, s, j) + row] = m;
-  if (p.ext && seg < 2 && row < p.row_words * 32) {
-    // Row `row` of operand [seg] of the extra K-step: slots 0..8 hold the pieces so that the nine
-    // products of an A row with a B row add up to theta*|a| * |b|.  A zero vector takes magnitude 1:
-    // its dot products are 0, so the accumulator keeps the sign of theta, as "0 > theta" demands.
-    const float n = m > 0.f ? m : 1.f;
-    __nv_bfloat16 pc[3];
-    split3_bf16(seg == 0 ? p.theta * n : n, pc);
-    __align__(16) __nv_bfloat16 out[16];
+  for (int r = 0; r < kNormRows; ++r) {
+    const int row = row_first + r * RPB;
+    float ss = 0.f;
 #pragma unroll
-    for (int i = 0; i < 16; ++i) out[i] = __float2bfloat16_rn(0.f);
-    if (row < l) {
+    for (int i = 0; i < 8; ++i) ss = fmaf(v[r][i], v[r][i], ss);
 #pragma unroll
-      for (int i = 0; i < 9; ++i) out[i] = seg == 0 ? pc[i / 3] : pc[i % 3];
+    for (int o = LPR / 2; o >= 1; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+    const float m = sqrtf(ss);
+    if (seg == 0 && row < l) p.mag[cb_out_row(p, layer, s, j) + row] = m;
+    if (p.ext && seg < 2 && row < p.row_words * 32) {
+      // Row `row` of operand [seg] of the extra K-step: slots 0..8 hold the pieces so that the nine
+      // products of an A row with a B row add up to theta*|a| * |b|.  A zero vector takes magnitude 1:
+      // its dot products are 0, so the accumulator keeps the sign of theta, as "0 > theta" demands.
+      const float n = m > 0.f ? m : 1.f;
+      __nv_bfloat16 pc[3];
+      split3_bf16(seg == 0 ? p.theta * n : n, pc);
+      __align__(16) __nv_bfloat16 out[16];
+#pragma unroll
+      for (int i = 0; i < 16; ++i) out[i] = __float2bfloat16_rn(0.f);
+      if (row < l) {
+#pragma unroll
+        for (int i = 0; i < 9; ++i) out[i] = seg == 0 ? pc[i / 3] : pc[i % 3];
+      }
+      uint4* dst = reinterpret_cast<uint4*>(p.ext + (((int64_t)seg * p.n_units + blockIdx.y) * p.row_words * 32 + row) * 16);
+      dst[0] = *reinterpret_cast<const uint4*>(out);
+      dst[1] = *reinterpret_cast<const uint4*>(out + 8);
     }
-    uint4* dst = reinterpret_cast<uint4*>(p.ext + (((int64_t)seg * p.n_units + blockIdx.y) * p.row_words * 32 + row) * 16);
-    dst[0] = *reinterpret_cast<const uint4*>(out);
-    dst[1] = *reinterpret_cast<const uint4*>(out + 8);
   }
 }
 
@@ -631,7 +643,7 @@ template <typename T, int D>
 static void launch_norms(const CodebookParams& p, cudaStream_t st) {
   constexpr int RPB = 256 / (D / 8);
   LaunchScope ls(KC_NORMS, st);
-  norms_kernel<T, D><<<dim3(ceil_div(p.row_words * 32, RPB), p.n_units), 256, 0, st>>>(p);
+  norms_kernel<T, D><<<dim3(ceil_div(p.row_words * 32, RPB * kNormRows), p.n_units), 256, 0, st>>>(p);
 }
 
 template <typename T, int D>
