@@ -49,6 +49,7 @@ def parse_args():
     ap.add_argument("--shallow", type=int, default=None, help="override the number of CodeBook layers")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--e2e-chunk", type=int, default=4, help="CodeBook layers per upload/compute/download group")
     return ap.parse_args()
 
 
@@ -244,27 +245,6 @@ def run_native(args, wl):
         if dQ is not None:
             dQ.copy_(hQ, non_blocking=True)
 
-    # results read back by the end-to-end arm: index maps, counts, magnitudes, and the compacted rows
-    # that can hold data (kept rows up to the largest k + w; CodeBook rows in full)
-    max_keep = int(p.k_ctx_host[wl.n_shallow:].max()) + wl.window if p.n_deep else 0
-    outs = []
-    if p.n_deep:
-        outs += [p.keep_idx, p.keep_cnt]
-        if wl.packed:
-            outs += [p.K_kept, p.V_kept]
-        else:
-            outs += [p.K_kept[:, :, :, :max_keep], p.V_kept[:, :, :, :max_keep]]
-    if p.n_shallow:
-        for g in ("K", "V"):
-            outs += [p.cb[g]["ref"], p.cb[g]["mag"], p.cb[g]["n_entries"], p.cb[g]["C"]]
-    host_out = [torch.empty(o.shape, dtype=o.dtype, pin_memory=True) for o in outs]
-    h2d = sum(t.numel() * t.element_size() for t in (hK, hV) + ((hQ,) if hQ is not None else ()))
-    d2h = sum(t.numel() * t.element_size() for t in host_out)
-
-    def download():
-        for o, h in zip(outs, host_out):
-            h.copy_(o, non_blocking=True)
-
     def barrier():
         torch.cuda.synchronize(dev)
         if dist is not None:
@@ -302,14 +282,26 @@ def run_native(args, wl):
 
     e2e = None
     if not args.no_e2e:
-        def step_e2e():
-            upload()
-            p.run(dK, dV, dQ)
-            download()
+        # the same pass through the host-buffer call: K, V, Q start in pinned host memory and every result
+        # (index maps, counts, magnitudes, kept rows, CodeBook rows) ends there, each step
+        p2 = SpindleKVPass(cfg, wl.seq_lens, dtype, device=dev, layers_per_codebook_call=args.e2e_chunk)
+        host_out = p2.host_outputs()
+        h2d = sum(t.numel() * t.element_size() for t in (hK, hV) + ((hQ,) if hQ is not None else ()))
+        d2h = sum(t.numel() * t.element_size() for t in host_out.values())
+        step_e2e = lambda: p2.run_from_host(hK, hV, hQ, host_out)
         step_e2e()
+        torch.cuda.synchronize(dev)
+        for g in ("K", "V") if p.n_shallow else ():
+            for k in ("ref", "n_entries"):
+                if not torch.equal(host_out[f"{g}.{k}"], p.cb[g][k].cpu()):
+                    raise RuntimeError(f"host-fed pass disagrees with the resident pass on {g}.{k}")
+        if p.n_deep and not torch.equal(host_out["keep_cnt"], p.keep_cnt.cpu()):
+            raise RuntimeError("host-fed pass disagrees with the resident pass on keep_cnt")
         ms_e2e = timed(step_e2e, args.steps)
         e2e = {"value": sharding.throughput(timed.tokens, args.steps, ms_e2e), "unit": UNIT,
-               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / args.steps}
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / args.steps,
+               "codebook_layers_per_group": args.e2e_chunk}
+        del p2
 
     # per-kernel times: one more pass with event pairs around every launch
     B.spindlekv_timing_enable(True)

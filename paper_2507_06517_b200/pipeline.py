@@ -90,21 +90,24 @@ class SpindleKVPass:
             B.spindlekv_compact(self.deep_batch, cfg.n_kv_heads, cfg.head_dim, self._desc(src), self.keep_idx,
                                 self.keep_cnt, self._desc(dst), None, None, stream)
 
-    def codebook(self, G: torch.Tensor, which: str, stream=None) -> None:
-        """Shallow layers: ``G`` holds only the CodeBook layers of ``which`` in {"K", "V"}."""
+    def _codebook_chunk(self, G: torch.Tensor, which: str, l0: int, stream=None) -> None:
+        """CodeBooks of ``G.shape[0]`` consecutive shallow layers starting at layer ``l0``."""
         cfg = self.cfg
+        n = G.shape[0]
         theta = cfg.theta_k if which == "K" else cfg.theta_v
         out = self.cb[which]
+        batch = self.cb_batch if n == self.cb_layers_per_call else B.Batch(n, self.n_seqs, self.max_len, self.total, self.cu)
+        sl = slice(l0, l0 + n)
+        B.spindlekv_codebook_shallow(cfg, batch, self._desc(G), theta, out["mag"][sl], out["ref"][sl],
+                                     out["centre_idx"][sl], out["n_entries"][sl], self.ws_codebook, self.adj, stream)
+        B.spindlekv_compact(batch, cfg.n_kv_heads, cfg.head_dim, self._desc(G), out["centre_idx"][sl],
+                            out["n_entries"][sl], self._desc(out["C"][sl]), out["mag"][sl], None, stream)
+
+    def codebook(self, G: torch.Tensor, which: str, stream=None) -> None:
+        """Shallow layers: ``G`` holds only the CodeBook layers of ``which`` in {"K", "V"}."""
         step = self.cb_layers_per_call
         for l0 in range(0, self.n_shallow, step):
-            n = min(step, self.n_shallow - l0)
-            batch = self.cb_batch if n == step else B.Batch(n, self.n_seqs, self.max_len, self.total, self.cu)
-            sl = slice(l0, l0 + n)
-            B.spindlekv_codebook_shallow(cfg, batch, self._desc(G[sl]), theta, out["mag"][sl], out["ref"][sl],
-                                         out["centre_idx"][sl], out["n_entries"][sl], self.ws_codebook, self.adj,
-                                         stream)
-            B.spindlekv_compact(batch, cfg.n_kv_heads, cfg.head_dim, self._desc(G[sl]), out["centre_idx"][sl],
-                                out["n_entries"][sl], self._desc(out["C"][sl]), out["mag"][sl], None, stream)
+            self._codebook_chunk(G[l0:l0 + min(step, self.n_shallow - l0)], which, l0, stream)
 
     def run(self, K: torch.Tensor, V: torch.Tensor, Q: torch.Tensor, stream=None) -> None:
         """All layers of one prompt batch (``K``/``V`` hold every layer)."""
@@ -114,6 +117,101 @@ class SpindleKVPass:
         if ns:
             self.codebook(K[:ns], "K", stream)
             self.codebook(V[:ns], "V", stream)
+
+    # -- the same pass fed from host memory ----------------------------------------------------
+    def host_outputs(self) -> Dict[str, torch.Tensor]:
+        """Pinned host tensors for everything ``run_from_host`` brings back: index maps, counts,
+        magnitudes, kept rows (up to the largest ``k + w`` of any layer) and CodeBook rows."""
+        out: Dict[str, torch.Tensor] = {}
+
+        def pin(name, t):
+            out[name] = torch.empty(t.shape, dtype=t.dtype, pin_memory=True)
+
+        if self.n_deep:
+            pin("keep_idx", self.keep_idx)
+            pin("keep_cnt", self.keep_cnt)
+            pin("K_kept", self._kept_view(self.K_kept))
+            pin("V_kept", self._kept_view(self.V_kept))
+        if self.n_shallow:
+            for g in ("K", "V"):
+                for k in ("ref", "mag", "n_entries", "C"):
+                    pin(f"{g}.{k}", self.cb[g][k])
+        return out
+
+    def _kept_view(self, t: torch.Tensor) -> torch.Tensor:
+        if self.packed:
+            return t
+        return t[:, :, :, : int(self.k_ctx_host[self.n_shallow:].max()) + self.cfg.window]
+
+    def run_from_host(self, hK: torch.Tensor, hV: torch.Tensor, hQ: Optional[torch.Tensor],
+                      host_out: Dict[str, torch.Tensor]) -> None:
+        """All layers of one prompt batch whose K, V (every layer) and Q (evicting layers) sit in pinned
+        host memory.  Uploads, kernels and downloads run on three streams: while the CodeBooks of one
+        group of layers are built, the next group is on its way in and the previous results are on
+        their way out.  Returns once everything is enqueued; work that follows on the current stream
+        is ordered after the last download."""
+        dev, cfg, ns = self.device, self.cfg, self.n_shallow
+        cur = torch.cuda.current_stream(dev)
+        if not hasattr(self, "_s_in"):
+            self._s_in, self._s_out = torch.cuda.Stream(dev), torch.cuda.Stream(dev)
+            c = self.cb_layers_per_call if ns else 0
+            self._stage = [self._alloc_like_input(c, self.dtype) for _ in range(2)] if ns else []
+            if self.n_deep:
+                self._dK = self._alloc_like_input(self.n_deep, self.dtype)
+                self._dV = self._alloc_like_input(self.n_deep, self.dtype)
+                self._dQ = torch.empty(hQ.shape, dtype=hQ.dtype, device=dev)
+        s_in, s_out = self._s_in, self._s_out
+        s_in.wait_stream(cur)
+        s_out.wait_stream(cur)
+        free = [None, None]   # event after the kernels that last read a staging buffer
+
+        def send(dst, src, after=None):
+            with torch.cuda.stream(s_in):
+                if after is not None:
+                    s_in.wait_event(after)
+                dst.copy_(src, non_blocking=True)
+                ev = torch.cuda.Event()
+                ev.record(s_in)
+            return ev
+
+        def fetch(pairs):
+            ev = torch.cuda.Event()
+            ev.record(cur)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(ev)
+                for h, d in pairs:
+                    h.copy_(d, non_blocking=True)
+
+        slot = 0
+        step = self.cb_layers_per_call if ns else 1
+        for l0 in range(0, ns, step):
+            n = min(step, ns - l0)
+            for which, h in (("K", hK), ("V", hV)):
+                buf = self._stage[slot & 1][:n]
+                cur.wait_event(send(buf, h[l0:l0 + n], free[slot & 1]))
+                self._codebook_chunk(buf, which, l0)
+                free[slot & 1] = torch.cuda.Event()
+                free[slot & 1].record(cur)
+                o = self.cb[which]
+                fetch([(host_out[f"{which}.{k}"][l0:l0 + n], o[k][l0:l0 + n]) for k in ("ref", "mag", "n_entries", "C")])
+                slot += 1
+        if self.n_deep:
+            ev_k = send(self._dK, hK[ns:])
+            ev_q = send(self._dQ, hQ)
+            ev_v = send(self._dV, hV[ns:])
+            cur.wait_event(ev_k)
+            cur.wait_event(ev_q)
+            B.spindlekv_evict_deep(cfg, self.deep_batch, self._desc(self._dK), B.desc_bhnd(self._dQ), self.k_ctx,
+                                   self.keep_idx, self.keep_cnt, self.scores, self.ws_evict)
+            B.spindlekv_compact(self.deep_batch, cfg.n_kv_heads, cfg.head_dim, self._desc(self._dK), self.keep_idx,
+                                self.keep_cnt, self._desc(self.K_kept), None, None)
+            fetch([(host_out["keep_idx"], self.keep_idx), (host_out["keep_cnt"], self.keep_cnt),
+                   (host_out["K_kept"], self._kept_view(self.K_kept))])
+            cur.wait_event(ev_v)
+            B.spindlekv_compact(self.deep_batch, cfg.n_kv_heads, cfg.head_dim, self._desc(self._dV), self.keep_idx,
+                                self.keep_cnt, self._desc(self.V_kept), None, None)
+            fetch([(host_out["V_kept"], self._kept_view(self.V_kept))])
+        cur.wait_stream(s_out)
 
     def device_status(self):
         """Status words of both workspaces (synchronises the device)."""

@@ -145,6 +145,43 @@ def test_window_scores_on_tensor_cores_shapes():
         assert stats["units"] == (wl.n_layers - wl.n_shallow) * wl.batch * wl.n_kv_heads
 
 
+def test_host_fed_pass_equals_resident_pass():
+    # the streamed call (pinned host buffers in, pinned host buffers out, CodeBook layers in groups) must
+    # return exactly what the resident call leaves on the device
+    wl = synth.Workload("hostfed", 5, 3, 8, 2, 128, "bf16", 32, (600,), 20, (0.05, 0.3), 2, "recency",
+                        budget_tokens=200.0, seed=41)
+    host = generate(wl)
+    layers = list(range(wl.n_layers))
+    K, V = stack_layers(wl, host, layers, "K"), stack_layers(wl, host, layers, "V")
+    Q = stack_layers(wl, host, layers[wl.n_shallow:], "Q")
+    p = _pass(wl)
+    p.run(K, V, Q)
+    p2 = _pass(wl, layers_per_codebook_call=2)
+    out = p2.host_outputs()
+    hK, hV, hQ = K.cpu().pin_memory(), V.cpu().pin_memory(), Q.cpu().pin_memory()
+    for _ in range(2):   # the second call reuses the staging buffers
+        p2.run_from_host(hK, hV, hQ, out)
+        torch.cuda.synchronize()
+        for g in ("K", "V"):
+            n = p.cb[g]["n_entries"].cpu()
+            assert torch.equal(out[f"{g}.n_entries"], n)
+            assert torch.equal(out[f"{g}.ref"], p.cb[g]["ref"].cpu())
+            assert torch.equal(out[f"{g}.mag"], p.cb[g]["mag"].cpu())
+            C = p.cb[g]["C"].cpu()
+            for li in range(wl.n_shallow):
+                for j in range(wl.n_kv_heads):
+                    m = int(n[li, 0, j])
+                    assert torch.equal(out[f"{g}.C"][li, 0, j, :m], C[li, 0, j, :m])
+        assert torch.equal(out["keep_cnt"], p.keep_cnt.cpu())
+        cnt = p.keep_cnt.cpu()
+        for li in range(wl.n_layers - wl.n_shallow):
+            for j in range(wl.n_kv_heads):
+                m = int(cnt[li, 0, j])
+                assert torch.equal(out["keep_idx"][li, j, :m], p.keep_idx.cpu()[li, j, :m])
+                assert torch.equal(out["K_kept"][li, 0, j, :m], p.K_kept.cpu()[li, 0, j, :m])
+                assert torch.equal(out["V_kept"][li, 0, j, :m], p.V_kept.cpu()[li, 0, j, :m])
+
+
 def test_plain_window_sum_extension():
     wl = synth.Workload("rawsum", 1, 0, 4, 2, 64, "f32", 32, (333,), 8, 0.1, 2, "gauss", budget_tokens=80.0, seed=14)
     run_and_check(wl, {"score_norm": 1})
