@@ -33,9 +33,10 @@ from paper_2507_06517_b200 import synth
 METRIC = "prompt tokens compressed/s (all layers)"
 UNIT = "tokens/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the similarity kernel, from the ncu
-# capture summarised under profiles/ (None until one exists for the current kernel)
-SIMILARITY_TRAFFIC_BYTES_PER_UNIT = None
+# dram__bytes_read.sum + dram__bytes_write.sum of the similarity kernel per unit (one head's K or V of one
+# layer), by sequence length, from the ncu capture summarised under profiles/ (8 units per launch there;
+# traffic grows in proportion to the units of a launch).  Lengths without a capture report null.
+SIMILARITY_TRAFFIC_BYTES_PER_UNIT = {16384: 32.6e6}
 
 
 def parse_args():
@@ -347,8 +348,8 @@ def run_native(args, wl):
         achieved = flops_per_step * args.steps / (sim_ms * 1e-3) / 1e12
         peak = pk["bf16_tflops_sustained"] if wl.dtype == "bf16" else pk["bf16_tflops_sustained"] / 32.0
         traffic = None
-        if SIMILARITY_TRAFFIC_BYTES_PER_UNIT is not None:
-            traffic = SIMILARITY_TRAFFIC_BYTES_PER_UNIT * units_per_launch
+        if not wl.packed and wl.max_len in SIMILARITY_TRAFFIC_BYTES_PER_UNIT and wl.head_dim == 128:
+            traffic = SIMILARITY_TRAFFIC_BYTES_PER_UNIT[wl.max_len] * units_per_launch
         roof = {"kernel": "similarity (Eq. 4, 9)", "bound": "tensor", "achieved": achieved, "peak": peak,
                 "unit": "TFLOP/s", "frac": achieved / peak, "traffic": traffic, "peak_source": pk_src,
                 "avg_launch_ms": sim_ms / sim_n, "algorithmic_flops_per_launch": flops_per_step * args.steps / sim_n}
