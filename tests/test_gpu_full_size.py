@@ -1,0 +1,116 @@
+"""The headline configuration at full size, launched the way ``bench.py`` launches it (all 16 evicting
+layers in one call, all 16 CodeBook layers of K, then of V, in one call each, N = 16384).
+
+The CPU checker needs seconds per unit at this size, so a few units are compared with it element by
+element (under the same bars as the small cases) and every unit is checked through properties that hold
+at any size: exact counts, the window always kept, ascending kept positions, kept rows equal to the
+source rows, every token referring to an existing entry, every centre referring to itself, unit-norm
+CodeBook rows, magnitudes equal to a float64 recomputation.
+"""
+from concurrent.futures import ThreadPoolExecutor
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import spindlekv_oracle as O
+from paper_2507_06517_b200 import synth
+
+from gpu_util import check_codebook_unit, check_evict_unit, make_config, torch_dtype, value_tol
+
+pytestmark = pytest.mark.gpu
+
+
+def _device_layers(wl):
+    dt = torch_dtype(wl)
+
+    def one(lam):
+        K, V, Q = synth.layer_arrays(wl, lam, need_q=lam >= wl.n_shallow)
+        return (torch.from_numpy(K).to(dt), torch.from_numpy(V).to(dt), None if Q is None else torch.from_numpy(Q).to(dt))
+
+    with ThreadPoolExecutor(max_workers=16) as ex:
+        layers = list(ex.map(one, range(wl.n_layers)))
+    K = torch.stack([x[0] for x in layers]).cuda()
+    V = torch.stack([x[1] for x in layers]).cuda()
+    Q = torch.stack([x[2] for x in layers[wl.n_shallow:]]).cuda()
+    return K, V, Q
+
+
+def _single_unit_codebook(wl, gamma_dev, theta):
+    """CodeBook of one [N, d] device array through a one-unit call that also returns the adjacency."""
+    from paper_2507_06517_b200.pipeline import SpindleKVPass
+    l, d = gamma_dev.shape
+    one = synth.Workload("one", 1, 1, 1, 1, d, wl.dtype, 1, (l,), 1, 0.1, 0, "gauss", budget_tokens=float(l),
+                         theta_k=theta, theta_v=theta)
+    p = SpindleKVPass(make_config(one), one.seq_lens, torch_dtype(one), keep_adjacency=True)
+    p.codebook(gamma_dev.reshape(1, 1, 1, l, d), "K")
+    assert p.device_status()["codebook"][0] == 0
+    o = p.cb["K"]
+    return (p.adj.cpu().numpy()[0], o["mag"].cpu().numpy()[0, 0], o["ref"].cpu().numpy()[0, 0],
+            o["centre_idx"].cpu().numpy()[0, 0], int(o["n_entries"].cpu().numpy()[0, 0, 0]),
+            o["C"].float().cpu().numpy()[0, 0, 0])
+
+
+def test_headline_configuration_full_size():
+    from paper_2507_06517_b200.pipeline import SpindleKVPass
+    wl = synth.workload("C3")
+    ns, nd, H, N, w = wl.n_shallow, wl.n_layers - wl.n_shallow, wl.n_kv_heads, wl.max_len, wl.window
+    K, V, Q = _device_layers(wl)
+    p = SpindleKVPass(make_config(wl), wl.seq_lens, torch_dtype(wl))
+    p.run(K, V, Q)
+    st = p.device_status()
+    assert st["evict"][0] == 0 and st["codebook"][0] == 0 and st["codebook"][1][1] == 0
+
+    # ---- every evicting unit: properties ----
+    _, _, k_plan = O.plan_layers(wl.n_layers, ns, wl.seq_lens, w, wl.beta, budget_tokens=wl.budget_tokens)
+    assert np.array_equal(k_plan, p.k_ctx_host)
+    keep = p.keep_idx.cpu().numpy()
+    cnt = p.keep_cnt.cpu().numpy()
+    for li in range(nd):
+        k = int(k_plan[ns + li, 0])
+        assert np.all(cnt[li] == k + w)
+        rows = keep[li, :, : k + w]
+        assert np.all(np.diff(rows, axis=1) > 0) and np.all(rows[:, k:] == np.arange(N - w, N))
+        idx = torch.from_numpy(rows.astype(np.int64)).cuda()
+        for src, dst in ((K, p.K_kept), (V, p.V_kept)):
+            want = torch.gather(src[ns + li, 0], 1, idx[:, :, None].expand(-1, -1, wl.head_dim))
+            assert torch.equal(dst[li, 0, :, : k + w], want)
+    # ---- two evicting layers against the checker (first and last of the pyramid) ----
+    scores = p.scores.cpu().numpy()
+    margin = 0
+    for li in (0, nd - 1):
+        lam = ns + li
+        margin += check_evict_unit(wl, Q[li, 0].float().cpu().numpy(), K[lam, 0].float().cpu().numpy(),
+                                   int(k_plan[lam, 0]), scores[li], keep[li], cnt[li, 0])
+
+    # ---- every CodeBook unit: properties ----
+    for g, G in (("K", K), ("V", V)):
+        o = p.cb[g]
+        n_ent = o["n_entries"].cpu().numpy()[:, 0]
+        ref = o["ref"].cpu().numpy()
+        cen = o["centre_idx"].cpu().numpy()
+        mag = o["mag"].cpu().numpy()
+        want_mag = torch.linalg.vector_norm(G[:ns, 0].double(), dim=-1).cpu().numpy()
+        np.testing.assert_allclose(mag, want_mag, rtol=2e-6)
+        for li in range(ns):
+            for j in range(H):
+                n = int(n_ent[li, j])
+                assert 1 <= n <= N
+                r, c = ref[li, j], cen[li, j, :n]
+                assert r.min() >= 0 and r.max() == n - 1                 # every token has an entry; every entry is used
+                assert np.array_equal(r[c], np.arange(n))                 # a centre refers to its own entry
+                assert len(np.unique(c)) == n
+                Cn = torch.linalg.vector_norm(o["C"][li, 0, j, :n].float(), dim=-1)
+                assert torch.all((Cn - 1).abs() < 1e-2)                   # unit vectors up to bf16 rounding
+    # ---- sampled CodeBook units against the checker; the one-unit call must reproduce the batched one ----
+    flips = 0
+    for g, G, theta, (li, j) in (("K", K, wl.theta_k, (3, 5)), ("V", V, wl.theta_v, (12, 0))):
+        gamma = G[li, 0, j]
+        adj, mag1, ref1, cen1, n1, C1 = _single_unit_codebook(wl, gamma, theta)
+        o = p.cb[g]
+        assert n1 == int(o["n_entries"][li, 0, j])
+        assert np.array_equal(ref1, o["ref"][li, j].cpu().numpy())
+        assert np.array_equal(cen1[:n1], o["centre_idx"][li, j, :n1].cpu().numpy())
+        assert np.array_equal(C1[:n1], o["C"][li, 0, j, :n1].float().cpu().numpy())
+        flips += check_codebook_unit(gamma.float().cpu().numpy(), theta, adj, mag1, ref1, cen1, n1, C1, value_tol(wl))
+    print(f"full size: {margin} kept positions and {flips} adjacency bits decided inside the 1e-4 margin")
