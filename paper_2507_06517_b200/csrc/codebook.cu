@@ -231,10 +231,11 @@ __global__ void __launch_bounds__(256) extract_kernel(CodebookParams p) {
   TransposeLane tr;
   tr.init(lane);
   int cnt = 1, k = 0;
-  for (int c0 = 0; c0 < NC; c0 += 32) {
+  const int nc = (l + 63) >> 6;   // chunks of this sequence (flags and bit rows beyond it are not written)
+  for (int c0 = 0; c0 < nc; c0 += 32) {
     // lane c holds the flags of chunk c0 + c for the warp's 32 rows; after the transpose lane r holds
     // the flags of its own row for these 32 chunks
-    uint32_t occ = tr.apply(c0 + lane < NC ? fl[(int64_t)(c0 + lane) * RW] : 0u);
+    uint32_t occ = tr.apply(c0 + lane < nc ? fl[(int64_t)(c0 + lane) * RW] : 0u);
     if (!exists) occ = 0;
     while (occ) {
       // up to four occupied chunks at a time, loaded before any of them is looked at

@@ -103,7 +103,7 @@ __global__ void __launch_bounds__(kSimThreads, 1) sim_tc_kernel(const __grid_con
   const int l = seq_len(p.batch, s);
   const int row0 = blockIdx.x * kBM;
   if (row0 >= l) return;
-  const int n_tiles = (p.row_words * 32 + kBN - 1) / kBN;
+  const int n_tiles = (l + kBN - 1) / kBN;   // tiles of this sequence: columns beyond its end are never produced
   const int tile0 = row0 / kBN;   // the tile that holds this block's diagonal; earlier tiles are mirrored by other blocks
 
   extern __shared__ uint8_t smem_raw[];
