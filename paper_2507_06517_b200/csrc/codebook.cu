@@ -36,7 +36,7 @@ struct CodebookParams {
   int32_t* ell;          // [kEll][units][max_len] neighbour lists of rows with few neighbours, entry-major
   int32_t* ell_cnt;      // [units][max_len] list length, -1: use the bit row
   int32_t* dense_rows;   // rows (unit * max_len + token) that use their bit row; count in the header
-  uint32_t* flags;       // [units][row_words/2][row_words] bit r of word w: the 64-column chunk of row 32w+r may hold a bit
+  uint32_t* flags;       // [units][row_words][row_words/2] bit r of word [w][c]: chunk c (64 columns) of row 32w+r may hold a bit
   uint32_t* hdr;
   int32_t* ref;          // [layers][H][T]
   int32_t* centre_idx;   // [layers][H][T]
@@ -226,16 +226,27 @@ __global__ void __launch_bounds__(256) extract_kernel(CodebookParams p) {
   const int64_t idx = (int64_t)unit * ML + (exists ? u : 0);
   const int64_t n_rows = (int64_t)p.n_units * ML;
   const int own = u >> 6;   // the chunk that holds the token's own bit
-  const uint32_t* fl = p.flags + (int64_t)unit * NC * RW + (u >> 5);
+  const uint32_t* fl = p.flags + ((int64_t)unit * RW + (u >> 5)) * NC;
   const uint2* row2 = reinterpret_cast<const uint2*>(p.adj + idx * RW);
   TransposeLane tr;
   tr.init(lane);
   int cnt = 1, k = 0;
   const int nc = (l + 63) >> 6;   // chunks of this sequence (flags and bit rows beyond it are not written)
-  for (int c0 = 0; c0 < nc; c0 += 32) {
-    // lane c holds the flags of chunk c0 + c for the warp's 32 rows; after the transpose lane r holds
+  constexpr int kFlagGroup = 8;   // flag words fetched together (256 chunks = 16384 columns)
+  for (int cb = 0; cb < nc; cb += 32 * kFlagGroup) {
+  uint32_t fw[kFlagGroup];
+#pragma unroll
+  for (int i = 0; i < kFlagGroup; ++i) {
+    const int c = cb + 32 * i + lane;
+    fw[i] = c < nc ? fl[c] : 0u;
+  }
+#pragma unroll
+  for (int i = 0; i < kFlagGroup; ++i) {
+    const int c0 = cb + 32 * i;
+    if (c0 >= nc) break;
+    // lane c held the flags of chunk c0 + c for the warp's 32 rows; after the transpose lane r holds
     // the flags of its own row for these 32 chunks
-    uint32_t occ = tr.apply(c0 + lane < nc ? fl[(int64_t)(c0 + lane) * RW] : 0u);
+    uint32_t occ = tr.apply(fw[i]);
     if (!exists) occ = 0;
     while (occ) {
       // up to four occupied chunks at a time, loaded before any of them is looked at
@@ -266,6 +277,7 @@ __global__ void __launch_bounds__(256) extract_kernel(CodebookParams p) {
         }
       }
     }
+  }
   }
   bool live = false;
   if (exists) {
@@ -310,6 +322,164 @@ __device__ __forceinline__ void keep_live(const uint32_t* lv, int (&v)[kBatch]) 
     if (!((w[i] >> (v[i] & 31)) & 1u)) v[i] = -1;
 }
 
+// Phase 2 for the 32 rows of live-mask word w: largest key in each closed live neighbourhood.
+// `kAllLive`: every listed neighbour is known to be live (round 0: a token with a neighbour is live),
+// so the live mask need not be consulted per neighbour.
+template <bool kAllLive>
+__device__ __forceinline__ void max_of_listed_rows(const CodebookParams& p, const uint32_t* live, int64_t w, int lane) {
+  const int ML = p.batch.max_len, RW = p.row_words;
+  const int64_t n_rows = (int64_t)p.n_units * ML;
+  const uint32_t lvw = live[w];
+  if (!((lvw >> lane) & 1u)) return;
+  const int unit = (int)(w / RW), u = (int)(w - (int64_t)unit * RW) * 32 + lane;
+  const int64_t idx = (int64_t)unit * ML + u;
+  const int ec = p.ell_cnt[idx];
+  if (ec < 0) return;                             // dense rows: separately
+  const uint32_t* lv = live + (int64_t)unit * RW;
+  const unsigned long long* key = p.key + (int64_t)unit * ML;
+  unsigned long long best = key[u];               // the token itself belongs to its closed neighbourhood
+  for (int k0 = 0; k0 < ec; k0 += kBatch) {
+    int v[kBatch];
+    load_batch(p.ell + idx, n_rows, k0, ec, v);
+    if (!kAllLive) keep_live(lv, v);
+    unsigned long long kv[kBatch];
+#pragma unroll
+    for (int i = 0; i < kBatch; ++i) kv[i] = v[i] >= 0 ? key[v[i]] : 0ull;
+#pragma unroll
+    for (int i = 0; i < kBatch; ++i) best = kv[i] > best ? kv[i] : best;
+  }
+  p.m1[idx] = best;
+}
+
+// Phase 2 for one dense row, a warp on its bit row.
+__device__ __forceinline__ void max_of_dense_row(const CodebookParams& p, const uint32_t* live, int64_t idx, int lane) {
+  const int ML = p.batch.max_len, RW = p.row_words;
+  const int unit = (int)(idx / ML), u = (int)(idx - (int64_t)unit * ML);
+  const uint32_t* lv = live + (int64_t)unit * RW;
+  if (!is_live(lv, u)) return;
+  const unsigned long long* key = p.key + (int64_t)unit * ML;
+  const uint32_t* row = p.adj + idx * RW;
+  unsigned long long best = 0ull;
+  for (int w = lane; w < RW; w += 32) {
+    uint32_t m = row[w] & lv[w];
+    while (m) {
+      int b = __ffs(m) - 1;
+      m &= m - 1;
+      unsigned long long kv = key[w * 32 + b];
+      best = kv > best ? kv : best;
+    }
+  }
+  best = warp_max_u64(best);
+  if (lane == 0) p.m1[idx] = best;
+}
+
+// Phase 3 for the 32 rows of live-mask word w: a node that is the maximum of every neighbour's
+// neighbourhood is a centre (Eq. (11)); its live neighbours take it as owner (Eq. (12)) and leave the
+// graph (Eq. (13)).
+template <bool kAllLive>
+__device__ __forceinline__ void pick_listed_rows(const CodebookParams& p, const uint32_t* live, uint32_t* next, int64_t w,
+                                                 int lane) {
+  const int ML = p.batch.max_len, RW = p.row_words;
+  const int64_t n_rows = (int64_t)p.n_units * ML;
+  const uint32_t lvw = live[w];
+  if (!((lvw >> lane) & 1u)) return;
+  const int unit = (int)(w / RW), u = (int)(w - (int64_t)unit * RW) * 32 + lane;
+  const int64_t idx = (int64_t)unit * ML + u;
+  const int ec = p.ell_cnt[idx];
+  if (ec < 0) return;
+  const unsigned long long mykey = p.key[idx];
+  if (p.m1[idx] != mykey) return;
+  const uint32_t* lv = live + (int64_t)unit * RW;
+  const unsigned long long* m1 = p.m1 + (int64_t)unit * ML;
+  bool ok = true;
+  for (int k0 = 0; k0 < ec && ok; k0 += kBatch) {
+    int v[kBatch];
+    load_batch(p.ell + idx, n_rows, k0, ec, v);
+    if (!kAllLive) keep_live(lv, v);
+    unsigned long long mv[kBatch];
+#pragma unroll
+    for (int i = 0; i < kBatch; ++i) mv[i] = v[i] >= 0 ? m1[v[i]] : mykey;
+#pragma unroll
+    for (int i = 0; i < kBatch; ++i) ok = ok && mv[i] == mykey;
+  }
+  if (!ok) return;
+  int32_t* owner = p.owner + (int64_t)unit * ML;
+  uint32_t* nx = next + (int64_t)unit * RW;
+  for (int k0 = 0; k0 < ec; k0 += kBatch) {
+    int v[kBatch];
+    load_batch(p.ell + idx, n_rows, k0, ec, v);
+    if (!kAllLive) keep_live(lv, v);
+#pragma unroll
+    for (int i = 0; i < kBatch; ++i)
+      if (v[i] >= 0) {
+        owner[v[i]] = u;
+        atomicAnd(&nx[v[i] >> 5], ~(1u << (v[i] & 31)));
+      }
+  }
+  p.pickdeg[idx] = p.deg[idx];
+  owner[u] = u;
+  atomicAnd(&nx[u >> 5], ~(1u << (u & 31)));
+}
+
+// Phase 3 for one dense row.
+__device__ __forceinline__ void pick_dense_row(const CodebookParams& p, const uint32_t* live, uint32_t* next, int64_t idx,
+                                               int lane) {
+  const int ML = p.batch.max_len, RW = p.row_words;
+  const int unit = (int)(idx / ML), u = (int)(idx - (int64_t)unit * ML);
+  const uint32_t* lv = live + (int64_t)unit * RW;
+  if (!is_live(lv, u)) return;
+  const unsigned long long mykey = p.key[idx];
+  if (p.m1[idx] != mykey) return;
+  const unsigned long long* m1 = p.m1 + (int64_t)unit * ML;
+  int32_t* owner = p.owner + (int64_t)unit * ML;
+  uint32_t* nx = next + (int64_t)unit * RW;
+  const uint32_t* row = p.adj + idx * RW;
+  bool ok = true;
+  for (int w = lane; w < RW; w += 32) {
+    uint32_t m = row[w] & lv[w];
+    while (m) {
+      int b = __ffs(m) - 1;
+      m &= m - 1;
+      if (m1[w * 32 + b] != mykey) ok = false;
+    }
+  }
+  if (!__all_sync(0xffffffffu, ok)) return;
+  if (lane == 0) p.pickdeg[idx] = p.deg[idx];
+  for (int w = lane; w < RW; w += 32) {
+    uint32_t m = row[w] & lv[w];
+    if (m) atomicAnd(&nx[w], ~m);
+    while (m) {
+      int b = __ffs(m) - 1;
+      m &= m - 1;
+      owner[w * 32 + b] = u;
+    }
+  }
+}
+
+// Round 0 as two ordinary launches: every row is still live, so the phases run with one warp per word of
+// the live mask over the whole grid (far more threads in flight than the cooperative kernel can keep
+// resident); the last kDenseBlocks blocks walk the list of dense rows.  `phase` 2: neighbourhood maxima,
+// 3: picks.
+constexpr int kDenseBlocks = 148;
+
+__global__ void __launch_bounds__(256) greedy_first_round_kernel(CodebookParams p, int phase, int word_blocks) {
+  const int lane = threadIdx.x & 31;
+  if ((int)blockIdx.x < word_blocks) {
+    const int64_t w = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    if (w >= (int64_t)p.n_units * p.row_words) return;
+    if (phase == 2) max_of_listed_rows<true>(p, p.live0, w, lane);
+    else pick_listed_rows<true>(p, p.live0, p.live1, w, lane);
+  } else {
+    const int n_dense = (int)p.hdr[kHdrDenseCnt];
+    const int nw = kDenseBlocks * (blockDim.x >> 5);
+    for (int d = ((int)blockIdx.x - word_blocks) * (blockDim.x >> 5) + (threadIdx.x >> 5); d < n_dense; d += nw) {
+      if (phase == 2) max_of_dense_row(p, p.live0, p.dense_rows[d], lane);
+      else pick_dense_row(p, p.live0, p.live1, p.dense_rows[d], lane);
+    }
+  }
+}
+
+// Rounds 1, 2, ...: few rows are left, one cooperative launch runs them to the end.
 __global__ void __launch_bounds__(512) greedy_kernel(CodebookParams p) {
   const int lane = threadIdx.x & 31;
   const int warps_per_block = blockDim.x >> 5;
@@ -322,15 +492,14 @@ __global__ void __launch_bounds__(512) greedy_kernel(CodebookParams p) {
   const int n_dense = (int)*reinterpret_cast<volatile uint32_t*>(&p.hdr[kHdrDenseCnt]);
   uint32_t target = 0;
 
-  int round = 0;
+  int round = 1;
   for (; round <= ML; ++round) {
     uint32_t* live = (round & 1) ? p.live1 : p.live0;
     uint32_t* next = (round & 1) ? p.live0 : p.live1;
     const int slot = (round & 1) ? kHdrLiveCnt1 : kHdrLiveCnt0;
     const int other = (round & 1) ? kHdrLiveCnt0 : kHdrLiveCnt1;
-    if (round > 0) {
+    {
       // phase 1: live degrees (Eq. (10)) and keys; `next` becomes a copy of `live`.
-      // (Round 0 uses the degrees and keys written with the neighbour lists.)
       if (gthread == 0) p.hdr[other] = 0;
       int my_live = 0;
       for (int64_t w = gwarp; w < n_words; w += nwarps) {
@@ -381,129 +550,18 @@ __global__ void __launch_bounds__(512) greedy_kernel(CodebookParams p) {
     }
 
     // phase 2: largest key in each closed live neighbourhood
-    for (int64_t w = gwarp; w < n_words; w += nwarps) {
-      const uint32_t lvw = live[w];
-      if (!((lvw >> lane) & 1u)) continue;
-      const int unit = (int)(w / RW), u = (int)(w - (int64_t)unit * RW) * 32 + lane;
-      const int64_t idx = (int64_t)unit * ML + u;
-      const int ec = p.ell_cnt[idx];
-      if (ec < 0) continue;
-      const uint32_t* lv = live + (int64_t)unit * RW;
-      const unsigned long long* key = p.key + (int64_t)unit * ML;
-      unsigned long long best = key[u];             // the token itself belongs to its closed neighbourhood
-      for (int k0 = 0; k0 < ec; k0 += kBatch) {
-        int v[kBatch];
-        load_batch(p.ell + idx, n_rows, k0, ec, v);
-        keep_live(lv, v);
-        unsigned long long kv[kBatch];
-#pragma unroll
-        for (int i = 0; i < kBatch; ++i) kv[i] = v[i] >= 0 ? key[v[i]] : 0ull;
-#pragma unroll
-        for (int i = 0; i < kBatch; ++i) best = kv[i] > best ? kv[i] : best;
-      }
-      p.m1[idx] = best;
-    }
-    for (int64_t d = gwarp; d < n_dense; d += nwarps) {
-      const int64_t idx = p.dense_rows[d];
-      const int unit = (int)(idx / ML), u = (int)(idx - (int64_t)unit * ML);
-      const uint32_t* lv = live + (int64_t)unit * RW;
-      if (!is_live(lv, u)) continue;
-      const unsigned long long* key = p.key + (int64_t)unit * ML;
-      const uint32_t* row = p.adj + idx * RW;
-      unsigned long long best = 0ull;
-      for (int w = lane; w < RW; w += 32) {
-        uint32_t m = row[w] & lv[w];
-        while (m) {
-          int b = __ffs(m) - 1;
-          m &= m - 1;
-          unsigned long long kv = key[w * 32 + b];
-          best = kv > best ? kv : best;
-        }
-      }
-      best = warp_max_u64(best);
-      if (lane == 0) p.m1[idx] = best;
-    }
+    for (int64_t w = gwarp; w < n_words; w += nwarps) max_of_listed_rows<false>(p, live, w, lane);
+    for (int64_t d = gwarp; d < n_dense; d += nwarps) max_of_dense_row(p, live, p.dense_rows[d], lane);
     if (!grid_barrier(p.hdr, target)) return;
 
-    // phase 3: a node that is the maximum of every neighbour's neighbourhood is a centre (Eq. (11));
-    // its live neighbours take it as owner (Eq. (12)) and leave the graph (Eq. (13))
-    for (int64_t w = gwarp; w < n_words; w += nwarps) {
-      const uint32_t lvw = live[w];
-      if (!((lvw >> lane) & 1u)) continue;
-      const int unit = (int)(w / RW), u = (int)(w - (int64_t)unit * RW) * 32 + lane;
-      const int64_t idx = (int64_t)unit * ML + u;
-      const int ec = p.ell_cnt[idx];
-      if (ec < 0) continue;
-      const unsigned long long mykey = p.key[idx];
-      if (p.m1[idx] != mykey) continue;
-      const uint32_t* lv = live + (int64_t)unit * RW;
-      const unsigned long long* m1 = p.m1 + (int64_t)unit * ML;
-      bool ok = true;
-      for (int k0 = 0; k0 < ec && ok; k0 += kBatch) {
-        int v[kBatch];
-        load_batch(p.ell + idx, n_rows, k0, ec, v);
-        keep_live(lv, v);
-        unsigned long long mv[kBatch];
-#pragma unroll
-        for (int i = 0; i < kBatch; ++i) mv[i] = v[i] >= 0 ? m1[v[i]] : mykey;
-#pragma unroll
-        for (int i = 0; i < kBatch; ++i) ok = ok && mv[i] == mykey;
-      }
-      if (!ok) continue;
-      int32_t* owner = p.owner + (int64_t)unit * ML;
-      uint32_t* nx = next + (int64_t)unit * RW;
-      for (int k0 = 0; k0 < ec; k0 += kBatch) {
-        int v[kBatch];
-        load_batch(p.ell + idx, n_rows, k0, ec, v);
-        keep_live(lv, v);
-#pragma unroll
-        for (int i = 0; i < kBatch; ++i)
-          if (v[i] >= 0) {
-            owner[v[i]] = u;
-            atomicAnd(&nx[v[i] >> 5], ~(1u << (v[i] & 31)));
-          }
-      }
-      p.pickdeg[idx] = p.deg[idx];
-      owner[u] = u;
-      atomicAnd(&nx[u >> 5], ~(1u << (u & 31)));
-    }
-    for (int64_t d = gwarp; d < n_dense; d += nwarps) {
-      const int64_t idx = p.dense_rows[d];
-      const int unit = (int)(idx / ML), u = (int)(idx - (int64_t)unit * ML);
-      const uint32_t* lv = live + (int64_t)unit * RW;
-      if (!is_live(lv, u)) continue;
-      const unsigned long long mykey = p.key[idx];
-      if (p.m1[idx] != mykey) continue;
-      const unsigned long long* m1 = p.m1 + (int64_t)unit * ML;
-      int32_t* owner = p.owner + (int64_t)unit * ML;
-      uint32_t* nx = next + (int64_t)unit * RW;
-      const uint32_t* row = p.adj + idx * RW;
-      bool ok = true;
-      for (int w = lane; w < RW; w += 32) {
-        uint32_t m = row[w] & lv[w];
-        while (m) {
-          int b = __ffs(m) - 1;
-          m &= m - 1;
-          if (m1[w * 32 + b] != mykey) ok = false;
-        }
-      }
-      if (!__all_sync(0xffffffffu, ok)) continue;
-      if (lane == 0) p.pickdeg[idx] = p.deg[idx];
-      for (int w = lane; w < RW; w += 32) {
-        uint32_t m = row[w] & lv[w];
-        if (m) atomicAnd(&nx[w], ~m);
-        while (m) {
-          int b = __ffs(m) - 1;
-          m &= m - 1;
-          owner[w * 32 + b] = u;
-        }
-      }
-    }
+    // phase 3: picks
+    for (int64_t w = gwarp; w < n_words; w += nwarps) pick_listed_rows<false>(p, live, next, w, lane);
+    for (int64_t d = gwarp; d < n_dense; d += nwarps) pick_dense_row(p, live, next, p.dense_rows[d], lane);
     if (!grid_barrier(p.hdr, target)) return;
   }
   if (gthread == 0) {
     p.hdr[kHdrRounds] = (uint32_t)round;
-    uint32_t left = round == 0 ? 0u : *reinterpret_cast<volatile uint32_t*>(&p.hdr[(round & 1) ? kHdrLiveCnt1 : kHdrLiveCnt0]);
+    uint32_t left = *reinterpret_cast<volatile uint32_t*>(&p.hdr[(round & 1) ? kHdrLiveCnt1 : kHdrLiveCnt0]);
     p.hdr[kHdrLive] = round > ML ? 1u : left;
     if (round > ML) atomicExch(&p.hdr[kHdrStatus], (uint32_t)SPINDLEKV_TIMEOUT);
   }
@@ -725,6 +783,11 @@ spindlekv_status codebook_shallow_impl(const spindlekv_config& cfg, const spindl
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, greedy_kernel, 512, 0) != cudaSuccess) return SPINDLEKV_CUDA;
     if (per_sm < 1) return SPINDLEKV_CUDA;
     coop_blocks = sms * per_sm;
+  }
+  for (int phase = 2; phase <= 3; ++phase) {
+    const int word_blocks = (int)(((size_t)units * p.row_words * 32 + 255) / 256);
+    LaunchScope ls(KC_GREEDY, st);
+    greedy_first_round_kernel<<<word_blocks + kDenseBlocks, 256, 0, st>>>(p, phase, word_blocks);
   }
   {
     LaunchScope ls(KC_GREEDY, st);

@@ -26,7 +26,7 @@
 // staged too and written 16 bytes per row by the whole team.  Nothing but bits leaves the SM:
 // N*N/8 bytes per unit, plus one bit per (row, 64-column chunk) that says whether the chunk may hold
 // a set bit (0: certainly empty), so that the next kernel reads only the occupied part of a sparse
-// graph.  The flags of 32 consecutive rows and one chunk form a word (`flags[chunk][row / 32]`) with
+// graph.  The flags of 32 consecutive rows and one chunk form a word (`flags[row / 32][chunk]`) with
 // exactly one writer: the rows' own block for chunks at or right of the block's own columns, the
 // block that mirrors into the rows for chunks left of them.
 #include "common.cuh"
@@ -38,7 +38,7 @@ struct SimTcParams {
   Batch batch;
   int n_kv_heads, row_words;
   uint32_t* adj;       // [units][max_len][row_words]
-  uint32_t* flags;     // [units][row_words / 2][row_words]
+  uint32_t* flags;     // [units][row_words][row_words / 2]
   uint32_t* hdr;
 };
 
@@ -211,7 +211,7 @@ __global__ void __launch_bounds__(kSimThreads, 1) sim_tc_kernel(const __grid_con
       // block, for the rows of the next block, which its diagonal tile mirrors into piecemeal.
       const int chunk = 2 * blk + cg;
       const int wb = (row0 >> 5) + team * 4 + q;   // team 0: own rows; team 1: the next block's rows
-      if (chunk < NC && wb < RW && (team == 0 || !(blk & 1))) funit[(int64_t)chunk * RW + wb] = 0xFFFFFFFFu;
+      if (chunk < NC && wb < RW && (team == 0 || !(blk & 1))) funit[(int64_t)wb * NC + chunk] = 0xFFFFFFFFu;
     }
     TransposeLane tr;
     tr.init(lane);
@@ -257,7 +257,7 @@ __global__ void __launch_bounds__(kSimThreads, 1) sim_tc_kernel(const __grid_con
           const uint32_t f0 = __ballot_sync(0xffffffffu, (words[0] | words[1]) != 0u);
           const uint32_t f1 = __ballot_sync(0xffffffffu, (words[2] | words[3]) != 0u);
           const int chunk = tile * 4 + cg * 2 + lane;
-          if (lane < 2 && chunk < NC) funit[(int64_t)chunk * RW + (R >> 5)] = lane ? f1 : f0;
+          if (lane < 2 && chunk < NC) funit[(int64_t)(R >> 5) * NC + chunk] = lane ? f1 : f0;
         }
         if (fast) {
           *reinterpret_cast<uint2*>(sdw) = make_uint2(words[0], words[1]);
@@ -297,7 +297,7 @@ __global__ void __launch_bounds__(kSimThreads, 1) sim_tc_kernel(const __grid_con
           occ_hi = (mv.z | mv.w) != 0u;
         }
         const uint32_t flo = __ballot_sync(0xffffffffu, occ_lo), fhi = __ballot_sync(0xffffffffu, occ_hi);
-        if (lane < 2 && (b >> 5) < RW) funit[(int64_t)(2 * blk + lane) * RW + (b >> 5)] = lane ? fhi : flo;
+        if (lane < 2 && (b >> 5) < RW) funit[(int64_t)(b >> 5) * NC + 2 * blk + lane] = lane ? fhi : flo;
       }
       if (slot == 1 || tile + 2 >= n_tiles) {
         // the two warps of the team that share this 32-row strip have staged their direct words of the
