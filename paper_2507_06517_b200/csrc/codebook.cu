@@ -69,16 +69,19 @@ template <typename T, int D>
 __global__ void __launch_bounds__(256) norms_kernel(CodebookParams p) {
   constexpr int LPR = D / 8;  // lanes per row
   constexpr int RPB = 256 / LPR;
+  constexpr int ROWS = RPB * kNormRows;   // consecutive rows of one block
+  __shared__ float sm_m[ROWS];
   int layer, s, j;
   cb_decode(p, blockIdx.y, layer, s, j);
   const int l = seq_len(p.batch, s);
   const int seg = threadIdx.x % LPR;
-  const int row_first = blockIdx.x * (RPB * kNormRows) + threadIdx.x / LPR;
+  const int block_row0 = blockIdx.x * ROWS;
+  const int local_first = threadIdx.x / LPR;
   const T* base = reinterpret_cast<const T*>(p.G.ptr) + unit_offset(p.G, p.batch, layer, s, j) + seg * 8;
   float v[kNormRows][8];
 #pragma unroll
   for (int r = 0; r < kNormRows; ++r) {
-    const int row = row_first + r * RPB;
+    const int row = block_row0 + local_first + r * RPB;
     if (row < l) load8(base + (int64_t)row * p.G.st, v[r]);
     else {
 #pragma unroll
@@ -87,31 +90,37 @@ __global__ void __launch_bounds__(256) norms_kernel(CodebookParams p) {
   }
 #pragma unroll
   for (int r = 0; r < kNormRows; ++r) {
-    const int row = row_first + r * RPB;
     float ss = 0.f;
 #pragma unroll
     for (int i = 0; i < 8; ++i) ss = fmaf(v[r][i], v[r][i], ss);
 #pragma unroll
     for (int o = LPR / 2; o >= 1; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-    const float m = sqrtf(ss);
-    if (seg == 0 && row < l) p.mag[cb_out_row(p, layer, s, j) + row] = m;
-    if (p.ext && seg < 2 && row < p.row_words * 32) {
-      // Row `row` of operand [seg] of the extra K-step: slots 0..8 hold the pieces so that the nine
-      // products of an A row with a B row add up to theta*|a| * |b|.  A zero vector takes magnitude 1:
-      // its dot products are 0, so the accumulator keeps the sign of theta, as "0 > theta" demands.
+    if (seg == 0) sm_m[local_first + r * RPB] = sqrtf(ss);
+  }
+  __syncthreads();
+  // magnitudes and operand rows leave in whole lines: consecutive threads, consecutive addresses
+  if (threadIdx.x < ROWS && block_row0 + threadIdx.x < l)
+    p.mag[cb_out_row(p, layer, s, j) + block_row0 + threadIdx.x] = sm_m[threadIdx.x];
+  if (p.ext) {
+    // Operand [op] of the extra K-step, row `row`: slots 0..8 hold the pieces so that the nine products of
+    // an A row with a B row add up to theta*|a| * |b|.  A zero vector takes magnitude 1: its dot
+    // products are 0, so the accumulator keeps the sign of theta, as "0 > theta" demands.
+    for (int t = threadIdx.x; t < ROWS * 4; t += 256) {
+      const int op = t / (ROWS * 2), r = (t % (ROWS * 2)) >> 1, hi = t & 1;
+      const int row = block_row0 + r;
+      if (row >= p.row_words * 32) continue;
+      const float m = sm_m[r];
       const float n = m > 0.f ? m : 1.f;
       __nv_bfloat16 pc[3];
-      split3_bf16(seg == 0 ? p.theta * n : n, pc);
-      __align__(16) __nv_bfloat16 out[16];
+      split3_bf16(op == 0 ? p.theta * n : n, pc);
+      __align__(16) __nv_bfloat16 out[8];
 #pragma unroll
-      for (int i = 0; i < 16; ++i) out[i] = __float2bfloat16_rn(0.f);
-      if (row < l) {
-#pragma unroll
-        for (int i = 0; i < 9; ++i) out[i] = seg == 0 ? pc[i / 3] : pc[i % 3];
+      for (int i = 0; i < 8; ++i) {
+        const int slot = hi * 8 + i;
+        out[i] = (row < l && slot < 9) ? (op == 0 ? pc[slot / 3] : pc[slot % 3]) : __float2bfloat16_rn(0.f);
       }
-      uint4* dst = reinterpret_cast<uint4*>(p.ext + (((int64_t)seg * p.n_units + blockIdx.y) * p.row_words * 32 + row) * 16);
-      dst[0] = *reinterpret_cast<const uint4*>(out);
-      dst[1] = *reinterpret_cast<const uint4*>(out + 8);
+      uint4* dst = reinterpret_cast<uint4*>(p.ext + (((int64_t)op * p.n_units + blockIdx.y) * p.row_words * 32 + row) * 16);
+      dst[hi] = *reinterpret_cast<const uint4*>(out);
     }
   }
 }
