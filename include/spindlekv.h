@@ -70,7 +70,9 @@ typedef struct {
   int32_t n_kv_heads;     /* h_g; query head h_n*j+g reads KV head j, h_n = h / h_g */
   int32_t head_dim;       /* d_h */
   int32_t window;         /* l_w: the last l_w tokens are the observation window and are always reserved */
-  int32_t n_shallow;      /* layers [0, n_shallow) build CodeBooks; layers [n_shallow, n_layers) evict */
+  int32_t n_shallow;      /* layers [0, n_shallow) build CodeBooks; layers [n_shallow, n_layers) evict;
+                             -1: the composition of Section 3 as written: every layer evicts under the pyramid
+                             of Eq. (5)(6) laid over all layers and then builds CodeBooks of what it kept */
   double reserve_ratio;   /* r of Section 3.3 (used when budget_tokens < 0) */
   double budget_tokens;   /* r*l given directly: tokens kept per head, window included; < 0: use reserve_ratio */
   double beta;            /* minimal retain ratio of any layer */
@@ -86,6 +88,10 @@ typedef struct {
   int32_t max_len;             /* longest sequence, l */
   int32_t total_len;           /* cu_seqlens[B] when packed, else B*max_len */
   const int32_t* cu_seqlens;   /* device [B+1], or NULL when all sequences have max_len tokens */
+  const int32_t* layer_lens;   /* device [n_layers][B], or NULL.  When given (only without cu_seqlens): sequence s
+                                  has layer_lens[layer*B + s] <= max_len tokens in layer `layer` of the call, rows
+                                  still max_len apart.  This is how the CodeBook call takes the tokens that
+                                  eviction kept, whose number differs from layer to layer (Eq. (5)(6)). */
 } spindlekv_batch;
 
 /*

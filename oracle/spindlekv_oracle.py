@@ -91,9 +91,16 @@ def plan_layers(n_layers: int, n_shallow: int, seq_lens: Sequence[int], l_w: int
 
     Returns ``(mode[m], r_c_layer[m, B], k_ctx[m, B])``; shallow layers carry
     ratio 1 and ``k = l_c`` (nothing is evicted there).  ``k`` follows Eq. (7):
-    ``floor(r_c(lambda) * l_c)``.
+    ``floor(r_c(lambda) * l_c)``.  ``n_shallow = -1`` is the paper's own
+    composition: all layers evict (pyramid over all ``m`` layers) and all build
+    CodeBooks of the kept tokens.
     """
     B = len(seq_lens)
+    if n_shallow == -1:
+        # Section 3 as written: every layer evicts under the pyramid laid over all layers and then
+        # builds CodeBooks of what it kept
+        mode, ratio, k_ctx = plan_layers(n_layers, 0, seq_lens, l_w, beta, reserve_ratio, budget_tokens)
+        return np.full(n_layers, MODE_EVICT | MODE_CODEBOOK, dtype=np.int32), ratio, k_ctx
     m_deep = n_layers - n_shallow
     mode = np.array([MODE_CODEBOOK if lam < n_shallow else MODE_EVICT for lam in range(n_layers)],
                     dtype=np.int32)
@@ -333,3 +340,33 @@ def reconstruct(C: np.ndarray, ref: np.ndarray, mag: np.ndarray) -> np.ndarray:
 def gather_rows(gamma: np.ndarray, idx: np.ndarray) -> np.ndarray:
     """Eq. (7), second line: ``Gamma_r = Gamma[eta]``."""
     return np.asarray(gamma)[np.asarray(idx, dtype=np.int64)]
+
+
+# --------------------------------------------------------------------------
+# The composition of Section 3 as written, and the reserve ratio of Eq. (15)
+# --------------------------------------------------------------------------
+
+def spindle_layer(q_win_heads: np.ndarray, k_heads: np.ndarray, v_heads: np.ndarray, k_ctx: int,
+                  theta_k: float, theta_v: float) -> Dict[str, object]:
+    """One layer of one sequence as Section 3 composes it: Eq. (1)(2)(3)(7) pick the tokens to keep
+    per KV head; Algorithm 1 then builds a K and a V CodeBook from the kept rows of each head.
+
+    Returns the kept positions ``keep[H_kv, k + w]`` and, per head, the CodeBook results of
+    ``K[keep]`` and ``V[keep]`` (lists ``cb_k``, ``cb_v`` of ``codebook_shallow`` dictionaries).
+    """
+    ev = evict_deep(q_win_heads, k_heads, k_ctx)
+    cb_k, cb_v = [], []
+    for j in range(k_heads.shape[0]):
+        cb_k.append(codebook_shallow(gather_rows(k_heads[j], ev["keep"][j]), theta_k))
+        cb_v.append(codebook_shallow(gather_rows(v_heads[j], ev["keep"][j]), theta_v))
+    return {"keep": ev["keep"], "scores": ev["scores"], "cb_k": cb_k, "cb_v": cb_v}
+
+
+def reserve_ratio_layer(l: int, kept: int, entries_k: Sequence[int], entries_v: Sequence[int]) -> Tuple[float, float]:
+    """Eq. (15) for one layer: ``r1`` = kept K and V tokens over all K and V tokens (summed over the
+    KV heads), ``r2`` = CodeBook entries of K and V over kept K and V tokens.  The dtype factor
+    ``r3`` is left to the caller."""
+    h = len(entries_k)
+    r1 = (2.0 * h * kept) / (2.0 * h * l)
+    r2 = (float(sum(entries_k)) + float(sum(entries_v))) / (2.0 * h * kept)
+    return r1, r2

@@ -42,7 +42,7 @@ class _Config(C.Structure):
 
 class _Batch(C.Structure):
     _fields_ = [("n_layers", C.c_int32), ("n_seqs", C.c_int32), ("max_len", C.c_int32),
-                ("total_len", C.c_int32), ("cu_seqlens", C.c_void_p)]
+                ("total_len", C.c_int32), ("cu_seqlens", C.c_void_p), ("layer_lens", C.c_void_p)]
 
 
 def _load() -> C.CDLL:
@@ -111,10 +111,12 @@ class Batch:
     max_len: int
     total_len: int
     cu_seqlens: Optional[torch.Tensor] = None  # device int32 [B+1]
+    layer_lens: Optional[torch.Tensor] = None  # device int32 [n_layers, B]: per-layer lengths (not with cu_seqlens)
 
     def c(self) -> _Batch:
         ptr = self.cu_seqlens.data_ptr() if self.cu_seqlens is not None else None
-        return _Batch(self.n_layers, self.n_seqs, self.max_len, self.total_len, ptr)
+        ll = self.layer_lens.data_ptr() if self.layer_lens is not None else None
+        return _Batch(self.n_layers, self.n_seqs, self.max_len, self.total_len, ptr, ll)
 
 
 def _dtype_code(t: torch.Tensor) -> int:

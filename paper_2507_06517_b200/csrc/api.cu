@@ -71,6 +71,7 @@ static bool cfg_ok(const spindlekv_config* c) {
 
 static bool batch_ok(const spindlekv_batch* b, int window) {
   if (!b) return false;
+  if (b->layer_lens && b->cu_seqlens) return false;
   if (b->n_layers <= 0 || b->n_seqs <= 0 || b->max_len <= window || b->total_len < b->max_len) return false;
   if (!b->cu_seqlens && (int64_t)b->total_len != (int64_t)b->n_seqs * b->max_len) return false;
   return true;
@@ -96,16 +97,20 @@ spindlekv_status spindlekv_plan_layers(const spindlekv_config* cfg, int32_t n_se
                                        int32_t* layer_mode, double* r_c_layer, int32_t* k_ctx) {
   if (!cfg_ok(cfg) || n_seqs <= 0 || !seq_lens || !layer_mode || !r_c_layer || !k_ctx) return SPINDLEKV_INVALID_ARG;
   const int m = cfg->n_layers;
-  if (cfg->n_shallow < 0 || cfg->n_shallow > m) return SPINDLEKV_INVALID_ARG;
-  const int m_deep = m - cfg->n_shallow;
+  if (cfg->n_shallow < -1 || cfg->n_shallow > m) return SPINDLEKV_INVALID_ARG;
+  const bool literal = cfg->n_shallow == -1;   // every layer evicts, then builds CodeBooks of what it kept
+  const int n_shallow = literal ? 0 : cfg->n_shallow;
+  const int m_deep = m - n_shallow;
   const double beta = cfg->beta;
   const double alpha = 0.5 * (1.0 + beta);
-  for (int lam = 0; lam < m; ++lam) layer_mode[lam] = lam < cfg->n_shallow ? SPINDLEKV_MODE_CODEBOOK : SPINDLEKV_MODE_EVICT;
+  for (int lam = 0; lam < m; ++lam)
+    layer_mode[lam] = literal ? (SPINDLEKV_MODE_EVICT | SPINDLEKV_MODE_CODEBOOK)
+                              : (lam < n_shallow ? SPINDLEKV_MODE_CODEBOOK : SPINDLEKV_MODE_EVICT);
   for (int s = 0; s < n_seqs; ++s) {
     const int l = seq_lens[s];
     const int l_c = l - cfg->window;
     if (l_c <= 0) return SPINDLEKV_INVALID_ARG;
-    for (int lam = 0; lam < cfg->n_shallow; ++lam) {
+    for (int lam = 0; lam < n_shallow; ++lam) {
       r_c_layer[(size_t)lam * n_seqs + s] = 1.0;
       k_ctx[(size_t)lam * n_seqs + s] = l_c;
     }
@@ -126,8 +131,8 @@ spindlekv_status spindlekv_plan_layers(const spindlekv_config* cfg, int32_t n_se
       const double r = m_deep == 1 ? r_c : r_first + (r_last - r_first) / (double)(m_deep - 1) * (double)lam;
       int k = (int)floor(r * (double)l_c);
       if (k > l_c) k = l_c;
-      r_c_layer[(size_t)(cfg->n_shallow + lam) * n_seqs + s] = r;
-      k_ctx[(size_t)(cfg->n_shallow + lam) * n_seqs + s] = k;
+      r_c_layer[(size_t)(n_shallow + lam) * n_seqs + s] = r;
+      k_ctx[(size_t)(n_shallow + lam) * n_seqs + s] = k;
     }
   }
   return SPINDLEKV_OK;
@@ -159,6 +164,7 @@ spindlekv_status spindlekv_codebook_shallow(const spindlekv_config* cfg, const s
   if (!cfg_ok(cfg) || !batch) return SPINDLEKV_INVALID_ARG;
   if (batch->n_layers <= 0 || batch->n_seqs <= 0 || batch->max_len <= 0 || batch->total_len < batch->max_len) return SPINDLEKV_INVALID_ARG;
   if (!batch->cu_seqlens && (int64_t)batch->total_len != (int64_t)batch->n_seqs * batch->max_len) return SPINDLEKV_INVALID_ARG;
+  if (batch->layer_lens && batch->cu_seqlens) return SPINDLEKV_INVALID_ARG;
   if (!tensor_ok(Gamma) || !mag || !ref || !centre_idx || !n_entries || !ws) return SPINDLEKV_INVALID_ARG;
   if (reinterpret_cast<uintptr_t>(ws) % 256) return SPINDLEKV_INVALID_ARG;
   if (cfg->head_dim != 64 && cfg->head_dim != 128) return SPINDLEKV_UNSUPPORTED;

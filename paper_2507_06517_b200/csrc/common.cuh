@@ -34,11 +34,18 @@ inline View make_view(const spindlekv_tensor& t) { return View{t.ptr, t.stride_l
 struct Batch {  // device-side copy of spindlekv_batch
   int n_layers, n_seqs, max_len, total_len;
   const int32_t* cu;
+  const int32_t* ll;   // per-layer lengths [n_layers][n_seqs], or null
 };
 
-inline Batch make_batch(const spindlekv_batch& b) { return Batch{b.n_layers, b.n_seqs, b.max_len, b.total_len, b.cu_seqlens}; }
+inline Batch make_batch(const spindlekv_batch& b) {
+  return Batch{b.n_layers, b.n_seqs, b.max_len, b.total_len, b.cu_seqlens, b.layer_lens};
+}
 
-__device__ __forceinline__ int seq_len(const Batch& b, int s) { return b.cu ? (b.cu[s + 1] - b.cu[s]) : b.max_len; }
+// tokens of sequence s in layer `layer` of the call
+__device__ __forceinline__ int seq_len(const Batch& b, int layer, int s) {
+  if (b.ll) return min(b.ll[layer * b.n_seqs + s], b.max_len);
+  return b.cu ? (b.cu[s + 1] - b.cu[s]) : b.max_len;
+}
 __device__ __forceinline__ int tok_base(const Batch& b, int s) { return b.cu ? b.cu[s] : s * b.max_len; }
 
 // element offset of row 0 of (layer, seq, head)

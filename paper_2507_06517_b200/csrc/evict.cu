@@ -63,7 +63,7 @@ __global__ void __launch_bounds__(256) win_stats_kernel(EvictParams p) {
   __shared__ TileSmem sm;
   int layer, s, j;
   decode_unit(p, blockIdx.y, layer, s, j);
-  const int l = seq_len(p.batch, s);
+  const int l = seq_len(p.batch, layer, s);
   const int key0 = blockIdx.x * kTile;
   if (key0 >= l) return;
   const int l_c = l - p.window;
@@ -106,7 +106,7 @@ __global__ void win_combine_kernel(EvictParams p, int n_units) {
   int unit = gw / M;
   int layer, s, j;
   decode_unit(p, unit, layer, s, j);
-  int nt = (seq_len(p.batch, s) + kTile - 1) / kTile;
+  int nt = (seq_len(p.batch, layer, s) + kTile - 1) / kTile;
   const float2* src = p.part + (int64_t)gw * p.n_tiles;
   float mx = -CUDART_INF_F;
   for (int t = lane; t < nt; t += 32) mx = fmaxf(mx, src[t].x);
@@ -128,7 +128,7 @@ __global__ void __launch_bounds__(256) win_colsum_kernel(EvictParams p) {
   __shared__ float colred[16][kTile];
   int layer, s, j;
   decode_unit(p, blockIdx.y, layer, s, j);
-  const int l = seq_len(p.batch, s);
+  const int l = seq_len(p.batch, layer, s);
   const int l_c = l - p.window;
   const int key0 = blockIdx.x * kTile;
   if (key0 >= l_c) return;  // only context columns are scored
@@ -226,7 +226,7 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(TopkParams p) {
   const int ls = unit / p.n_kv_heads;
   const int s = ls % p.batch.n_seqs;
   const int layer = ls / p.batch.n_seqs;
-  const int l = seq_len(p.batch, s);
+  const int l = seq_len(p.batch, layer, s);
   const int l_c = l - p.window;
   int k = p.k_ctx[layer * p.batch.n_seqs + s];
   k = max(0, min(k, l_c));

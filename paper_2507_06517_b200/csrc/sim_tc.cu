@@ -100,7 +100,7 @@ __global__ void __launch_bounds__(kSimThreads, 1) sim_tc_kernel(const __grid_con
   const int ls = unit / p.n_kv_heads;
   const int s = ls % p.batch.n_seqs;
   const int layer = ls / p.batch.n_seqs;
-  const int l = seq_len(p.batch, s);
+  const int l = seq_len(p.batch, layer, s);
   const int row0 = blockIdx.x * kBM;
   if (row0 >= l) return;
   const int n_tiles = (l + kBN - 1) / kBN;   // tiles of this sequence: columns beyond its end are never produced

@@ -4,6 +4,7 @@ layers, compact).  No arithmetic happens here; this is buffer ownership and call
 """
 from __future__ import annotations
 
+import dataclasses
 from typing import Dict, Optional, Sequence
 
 import numpy as np
@@ -222,3 +223,64 @@ class SpindleKVPass:
         if self.n_shallow:
             out["codebook"] = B.spindlekv_poll_status(self.ws_codebook)
         return out
+
+
+class SpindleKVLiteralPass:
+    """The composition of Section 3 as the paper writes it: every layer evicts under the pyramid of
+    Eq. (5)(6) laid over all layers (Eq. (7)), then K and V CodeBooks are built from the tokens the layer
+    kept (Algorithm 1), whose number differs from layer to layer.  ``cfg.n_shallow`` must be -1; all
+    sequences have the same length.  ``K``, ``V``: ``[n_layers, B, H_kv, N, d]``; ``Q``:
+    ``[n_layers, B, H_q, w, d]``.  No arithmetic happens here: buffers and call order only.
+    """
+
+    def __init__(self, cfg: B.Config, seq_lens: Sequence[int], dtype: torch.dtype, device="cuda",
+                 keep_adjacency: bool = False):
+        if cfg.n_shallow != -1:
+            raise ValueError("SpindleKVLiteralPass needs cfg.n_shallow == -1")
+        if len(set(int(x) for x in seq_lens)) != 1:
+            raise ValueError("SpindleKVLiteralPass needs sequences of equal length")
+        self.cfg = cfg
+        self.device = torch.device(device)
+        self.ev = SpindleKVPass(dataclasses.replace(cfg, n_shallow=0), seq_lens, dtype, device)
+        self.mode, self.ratio, self.k_ctx_host = B.spindlekv_plan_layers(cfg, list(seq_lens))
+        L, nB, H, d = cfg.n_layers, len(seq_lens), cfg.n_kv_heads, cfg.head_dim
+        self.kept_host = (self.k_ctx_host + cfg.window).astype(np.int32)          # [L, B] tokens kept per head
+        self.max_keep = int(self.kept_host.max())
+        self.layer_lens = torch.from_numpy(np.ascontiguousarray(self.kept_host)).to(self.device)
+        T = nB * self.max_keep
+        self.cb_batch = B.Batch(L, nB, self.max_keep, T, None, self.layer_lens)
+        nb = B.spindlekv_workspace_bytes(cfg, self.cb_batch, B.WS_CODEBOOK)
+        self.ws_codebook = torch.empty(nb, dtype=torch.uint8, device=self.device)
+        i32 = dict(dtype=torch.int32, device=self.device)
+        self.cb: Dict[str, Dict[str, torch.Tensor]] = {}
+        for g in ("K", "V"):
+            self.cb[g] = {
+                "mag": torch.zeros((L, H, T), dtype=torch.float32, device=self.device),
+                "ref": torch.zeros((L, H, T), **i32),
+                "centre_idx": torch.zeros((L, H, T), **i32),
+                "n_entries": torch.zeros((L, nB, H), **i32),
+                "C": torch.zeros((L, nB, H, self.max_keep, d), dtype=dtype, device=self.device),
+            }
+        self.adj = None
+        if keep_adjacency:
+            self.adj = torch.zeros((L * nB * H, self.max_keep, B.row_words(self.max_keep)), **i32)
+
+    def run(self, K: torch.Tensor, V: torch.Tensor, Q: torch.Tensor, which=("K", "V"), stream=None) -> None:
+        cfg = self.cfg
+        self.ev.evict(K, V, Q, stream)
+        for g in which:
+            kept = (self.ev.K_kept if g == "K" else self.ev.V_kept)[:, :, :, : self.max_keep]
+            o = self.cb[g]
+            B.spindlekv_codebook_shallow(cfg, self.cb_batch, B.desc_bhnd(kept), cfg.theta_k if g == "K" else cfg.theta_v,
+                                         o["mag"], o["ref"], o["centre_idx"], o["n_entries"], self.ws_codebook,
+                                         self.adj, stream)
+            B.spindlekv_compact(self.cb_batch, cfg.n_kv_heads, cfg.head_dim, B.desc_bhnd(kept), o["centre_idx"],
+                                o["n_entries"], B.desc_bhnd(o["C"]), o["mag"], None, stream)
+
+    def entry_counts(self):
+        """Host copies of the CodeBook sizes ``[L, B, H]`` for K and V (synchronises)."""
+        return self.cb["K"]["n_entries"].cpu().numpy(), self.cb["V"]["n_entries"].cpu().numpy()
+
+    def device_status(self):
+        torch.cuda.synchronize(self.device)
+        return {"evict": B.spindlekv_poll_status(self.ev.ws_evict), "codebook": B.spindlekv_poll_status(self.ws_codebook)}

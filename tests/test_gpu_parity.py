@@ -182,6 +182,48 @@ def test_host_fed_pass_equals_resident_pass():
                 assert torch.equal(out["V_kept"][li, 0, j, :m], p.V_kept.cpu()[li, 0, j, :m])
 
 
+def test_composition_as_written_evict_then_codebooks_of_the_kept_tokens():
+    # every layer evicts under the pyramid over all layers, then builds K and V CodeBooks of what it kept
+    # (different counts per layer, passed to the CodeBook call as per-layer lengths)
+    from paper_2507_06517_b200.pipeline import SpindleKVLiteralPass
+    wl = synth.Workload("literal", 3, -1, 8, 2, 128, "bf16", 32, (700,), 12, (0.03, 0.3), 2, "recency",
+                        budget_tokens=260.0, seed=51)
+    layers = list(range(wl.n_layers))
+    host = {lam: synth.layer_arrays(wl, lam, need_q=True) for lam in layers}
+    K, V, Q = (stack_layers(wl, host, layers, x) for x in ("K", "V", "Q"))
+    p = SpindleKVLiteralPass(make_config(wl), wl.seq_lens, torch_dtype(wl), keep_adjacency=True)
+    _, _, k_plan = O.plan_layers(wl.n_layers, -1, wl.seq_lens, wl.window, wl.beta, budget_tokens=wl.budget_tokens)
+    assert np.array_equal(k_plan, p.k_ctx_host) and len(set(k_plan[:, 0])) == wl.n_layers
+    H, l, w = wl.n_kv_heads, wl.max_len, wl.window
+    units = 0
+    for g, idx, theta in (("K", 0, wl.theta_k), ("V", 1, wl.theta_v)):
+        p.run(K, V, Q, which=(g,))
+        st = p.device_status()
+        assert st["evict"][0] == 0 and st["codebook"][0] == 0 and st["codebook"][1][1] == 0
+        keep = p.ev.keep_idx.cpu().numpy()
+        cnt = p.ev.keep_cnt.cpu().numpy()
+        scores = p.ev.scores.cpu().numpy()
+        o = {k: (v.float() if k == "C" else v).cpu().numpy() for k, v in p.cb[g].items()}
+        adj = p.adj.cpu().numpy()
+        for lam in layers:
+            k_ctx = int(k_plan[lam, 0])
+            Ks = np.stack([host[lam][0][0, j] for j in range(H)])
+            check_evict_unit(wl, host[lam][2][0], Ks, k_ctx, scores[lam], keep[lam], cnt[lam, 0])
+            n = k_ctx + w
+            for j in range(H):
+                # the checker builds its CodeBook from the rows this layer and head actually kept
+                gamma = host[lam][idx][0, j][keep[lam, j, :n]]
+                check_codebook_unit(gamma, theta, adj[lam * H + j], o["mag"][lam, j, :n],
+                                    o["ref"][lam, j, :n], o["centre_idx"][lam, j, :n], int(o["n_entries"][lam, 0, j]),
+                                    o["C"][lam, 0, j], value_tol(wl))
+                units += 1
+    assert units == 2 * wl.n_layers * H
+    nk, nv = p.entry_counts()
+    for lam in layers:   # Eq. (15)
+        r1, r2 = O.reserve_ratio_layer(l, int(k_plan[lam, 0]) + w, nk[lam, 0], nv[lam, 0])
+        assert 0 < r1 <= 1 and 0 < r2 <= 1
+
+
 def test_plain_window_sum_extension():
     wl = synth.Workload("rawsum", 1, 0, 4, 2, 64, "f32", 32, (333,), 8, 0.1, 2, "gauss", budget_tokens=80.0, seed=14)
     run_and_check(wl, {"score_norm": 1})

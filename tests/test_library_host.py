@@ -32,7 +32,7 @@ def test_planner_matches_checker():
     rng = np.random.default_rng(3)
     for _ in range(200):
         m = int(rng.integers(1, 48))
-        ns = int(rng.integers(0, m + 1))
+        ns = int(rng.integers(-1, m + 1))   # -1: every layer evicts, then builds CodeBooks
         Bn = int(rng.integers(1, 5))
         w = int(rng.choice([16, 32, 64]))
         lens = [int(x) for x in rng.integers(w + 200, 40000, size=Bn)]

@@ -1,0 +1,64 @@
+"""Pins for the checker's composition of Section 3 (every layer evicts, then builds CodeBooks of what it
+kept) and for the reserve ratio of Eq. (15): closed forms and special cases whose answer does not
+depend on the checker's own code."""
+import numpy as np
+import pytest
+
+from oracle import spindlekv_oracle as O
+
+
+def test_literal_plan_is_the_pyramid_over_all_layers():
+    for m, lens, w, budget in ((32, [16384], 32, 1024.0), (5, [600, 900], 16, 200.0)):
+        mode, ratio, k = O.plan_layers(m, -1, lens, w, 0.05, budget_tokens=budget)
+        assert np.all(mode == (O.MODE_EVICT | O.MODE_CODEBOOK))
+        for s, l in enumerate(lens):
+            r_c = (budget - w) / (l - w)
+            assert abs(ratio[:, s].mean() - r_c) < 1e-12            # the pyramid keeps the mean (Eq. (5)(6))
+            assert np.all(np.diff(ratio[:, s]) <= 0) and ratio[-1, s] >= 0.05 - 1e-12
+            assert np.array_equal(k[:, s], np.floor(ratio[:, s] * (l - w)).astype(np.int32))   # Eq. (7)
+
+
+def test_dominant_keys_are_kept_and_their_duplicates_share_entries():
+    # Four context keys are 6x longer copies of one direction that every window query points at: they
+    # take nearly all attention mass, so with k = 4 exactly they are kept (plus the window).  Among the
+    # kept keys those four are parallel (cosine 1) and the window keys are random: K needs 1 + w entries.
+    rng = np.random.default_rng(5)
+    l, w, d, H = 120, 8, 32, 2
+    k = rng.standard_normal((H, l, d)) * 0.1
+    v = rng.standard_normal((H, l, d))
+    dirn = rng.standard_normal(d)
+    dirn /= np.linalg.norm(dirn)
+    hot = [7, 40, 41, 99]
+    for j in range(H):
+        k[j, hot] = 6.0 * dirn * np.array([1.0, 1.5, 2.0, 2.5])[:, None]
+        v[j, hot] = v[j, hot[0]]                                   # identical values: one V entry for the four
+    q = np.tile(8.0 * dirn, (2 * H, w, 1))
+    out = O.spindle_layer(q, k, v, 4, 0.98, 0.95)
+    for j in range(H):
+        assert list(out["keep"][j]) == hot + list(range(l - w, l))
+        ck, cv = out["cb_k"][j], out["cb_v"][j]
+        assert len(ck["centres"]) == 1 + w and len(cv["centres"]) == 1 + w
+        assert len(set(ck["ref"][:4])) == 1 and len(set(cv["ref"][:4])) == 1
+        # the entry is the unit vector of the centre; magnitudes are those of the kept rows (Eq. (8))
+        np.testing.assert_allclose(np.abs(ck["C"][ck["ref"][0]] @ dirn), 1.0, atol=1e-12)
+        np.testing.assert_allclose(ck["mag"][:4], 6.0 * np.array([1.0, 1.5, 2.0, 2.5]), rtol=1e-12)
+
+
+def test_no_merging_and_total_merging():
+    rng = np.random.default_rng(6)
+    l, w, d, H = 90, 6, 16, 2
+    k, v = rng.standard_normal((H, l, d)), rng.standard_normal((H, l, d))
+    q = rng.standard_normal((2 * H, w, d))
+    none = O.spindle_layer(q, k, v, 20, 1.0, 1.0)      # nothing is similar enough: one entry per kept token
+    every = O.spindle_layer(q, k, v, 20, -1.5, -1.5)   # everything is: one entry per head
+    for j in range(H):
+        assert len(none["cb_k"][j]["centres"]) == 26 and list(none["cb_k"][j]["ref"]) == list(range(26))
+        assert len(every["cb_v"][j]["centres"]) == 1 and np.all(every["cb_v"][j]["ref"] == 0)
+    assert np.array_equal(none["keep"], every["keep"])  # eviction does not depend on the thresholds
+    # Eq. (15): r1 = kept / l; r2 = entries / kept tokens
+    r1, r2 = O.reserve_ratio_layer(l, 26, [26] * H, [26] * H)
+    assert r1 == pytest.approx(26 / 90) and r2 == 1.0
+    r1, r2 = O.reserve_ratio_layer(l, 26, [1] * H, [1] * H)
+    assert r2 == pytest.approx(1 / 26)
+    r1, r2 = O.reserve_ratio_layer(100, 40, [10, 30], [20, 20])
+    assert r1 == pytest.approx(0.4) and r2 == pytest.approx(80 / 160)
