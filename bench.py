@@ -48,6 +48,8 @@ def parse_args():
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
     ap.add_argument("--layers", type=int, default=None, help="override the layer count (profiling on a small case)")
     ap.add_argument("--shallow", type=int, default=None, help="override the number of CodeBook layers")
+    ap.add_argument("--literal", action="store_true",
+                    help="the paper's own composition: every layer evicts, then builds CodeBooks of what it kept")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--e2e-chunk", type=int, default=4, help="CodeBook layers per upload/compute/download group")
@@ -209,6 +211,52 @@ def host_inputs(wl):
     V = torch.stack([x[1] for x in layers]).pin_memory()
     Q = torch.stack([x[2] for x in layers[ns:]]).pin_memory() if wl.n_layers > ns else None
     return K, V, Q
+
+
+def run_literal(args, wl):
+    """Every layer evicts under the pyramid over all layers, then builds K and V CodeBooks of the kept
+    tokens (Section 3 as written).  Single GPU; reports throughput and the reserve ratios of Eq. (15)."""
+    from paper_2507_06517_b200 import binding as B
+    from paper_2507_06517_b200.pipeline import SpindleKVLiteralPass
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the reduction pass has no CPU fallback")
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    wl = wl.replace(n_shallow=0)   # window queries for every layer
+    hK, hV, hQ = host_inputs(wl)
+    cfg = B.Config(n_layers=wl.n_layers, n_q_heads=wl.n_q_heads, n_kv_heads=wl.n_kv_heads, head_dim=wl.head_dim,
+                   window=wl.window, n_shallow=-1, beta=wl.beta, theta_k=wl.theta_k, theta_v=wl.theta_v,
+                   budget_tokens=wl.budget_tokens if wl.budget_tokens is not None else -1.0,
+                   reserve_ratio=wl.budget_frac if wl.budget_frac is not None else -1.0)
+    p = SpindleKVLiteralPass(cfg, wl.seq_lens, hK.dtype, device=dev)
+    dK, dV, dQ = hK.to(dev), hV.to(dev), hQ.to(dev)
+    for _ in range(max(args.warmup, 3)):
+        p.run(dK, dV, dQ)
+    st = p.device_status()
+    if st["evict"][0] or st["codebook"][0]:
+        raise RuntimeError(f"device status {st}")
+    B.spindlekv_launch_count(True)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize(dev)
+    ev0.record()
+    for _ in range(args.steps):
+        p.run(dK, dV, dQ)
+    ev1.record()
+    torch.cuda.synchronize(dev)
+    ms = ev0.elapsed_time(ev1)
+    launches = B.spindlekv_launch_count(True)
+    nk, nv = p.entry_counts()
+    kept = p.kept_host[:, 0].astype(np.float64)
+    r1 = kept / wl.max_len
+    r2 = (nk[:, 0].sum(axis=1) + nv[:, 0].sum(axis=1)) / (2.0 * wl.n_kv_heads * kept)
+    line = {"metric": METRIC + ", composition as written", "value": wl.total_tokens * args.steps / (ms * 1e-3),
+            "unit": UNIT, "n_gpus": 1, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic",
+            "config": workload_config(wl, {"composition": "every layer: evict (pyramid over all layers), then CodeBooks of the kept tokens"}),
+            "gpu_launches": int(launches),
+            "reserve_ratio": {"r1_mean": float(r1.mean()), "r2_mean": float(r2.mean()), "r1_r2_mean": float((r1 * r2).mean()),
+                              "kept_first_last": [int(kept[0]), int(kept[-1])]}}
+    print(json.dumps(line))
 
 
 def run_native(args, wl):
@@ -378,5 +426,7 @@ if __name__ == "__main__":
                       name=f"{w.name}[{a.layers} layers]")
     if a.impl == "reference":
         run_reference(a, w)
+    elif a.literal:
+        run_literal(a, w)
     else:
         run_native(a, w)
