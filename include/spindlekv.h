@@ -194,6 +194,18 @@ spindlekv_status spindlekv_compact(const spindlekv_batch* batch, int32_t n_heads
                                    void* stream);
 
 /*
+ * Reconstruction of the replaced cache from a CodeBook (Eq. (14): Gamma_r = C[r] (x) m): for every
+ * (layer, seq, head) and token t of the sequence, dst row t = C row ref[t] times mag[t] (product in fp32,
+ * rounded to the storage type).
+ *   C    device, CodeBook rows as written by spindlekv_compact with divide_by = mag, addressed like a cache tensor
+ *   ref  device [n_layers][n_heads][T], mag device [n_layers][n_heads][T]: outputs of spindlekv_codebook_shallow
+ *   dst  device, same addressing rules and dtype as C; may not overlap C
+ */
+spindlekv_status spindlekv_reconstruct(const spindlekv_batch* batch, int32_t n_heads, int32_t head_dim,
+                                       spindlekv_tensor C, const int32_t* ref, const float* mag, spindlekv_tensor dst,
+                                       void* stream);
+
+/*
  * Reads the device status word of a workspace (blocking copy; synchronise the stream first).
  *   device_status host out: SPINDLEKV_OK or SPINDLEKV_TIMEOUT
  *   detail        host out, optional [4]: {greedy rounds used, live tokens left, 0, 0}

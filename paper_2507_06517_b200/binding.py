@@ -69,6 +69,9 @@ def _load() -> C.CDLL:
     lib.spindlekv_compact.restype = C.c_int32
     lib.spindlekv_compact.argtypes = [C.POINTER(_Batch), C.c_int32, C.c_int32, _Tensor, C.c_void_p, C.c_void_p,
                                       C.c_void_p, _Tensor, C.c_void_p, C.c_void_p]
+    lib.spindlekv_reconstruct.restype = C.c_int32
+    lib.spindlekv_reconstruct.argtypes = [C.POINTER(_Batch), C.c_int32, C.c_int32, _Tensor, C.c_void_p, C.c_void_p,
+                                          _Tensor, C.c_void_p]
     lib.spindlekv_poll_status.restype = C.c_int32
     lib.spindlekv_poll_status.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
     lib.spindlekv_launch_count.restype = C.c_int64
@@ -215,6 +218,13 @@ def spindlekv_compact(batch: Batch, n_heads: int, head_dim: int, src: _Tensor, i
     st = _lib.spindlekv_compact(C.byref(bb), n_heads, head_dim, src, _ptr(idx), _ptr(cnt), _ptr(divide_by), dst,
                                 _ptr(dst_cu_seqlens), _stream(stream))
     _check(st, "spindlekv_compact")
+
+
+def spindlekv_reconstruct(batch: Batch, n_heads: int, head_dim: int, Cb: _Tensor, ref: torch.Tensor,
+                          mag: torch.Tensor, dst: _Tensor, stream=None) -> None:
+    bb = batch.c()
+    st = _lib.spindlekv_reconstruct(C.byref(bb), n_heads, head_dim, Cb, _ptr(ref), _ptr(mag), dst, _stream(stream))
+    _check(st, "spindlekv_reconstruct")
 
 
 def spindlekv_poll_status(ws: torch.Tensor):

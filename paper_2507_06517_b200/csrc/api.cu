@@ -22,6 +22,9 @@ spindlekv_status compact_impl(const spindlekv_batch& b, int n_heads, int head_di
                               const int32_t* idx, const int32_t* cnt, const float* divide_by,
                               const spindlekv_tensor& dst, const int32_t* dst_cu, cudaStream_t st);
 
+spindlekv_status reconstruct_impl(const spindlekv_batch& b, int n_heads, int head_dim, const spindlekv_tensor& C,
+                                  const int32_t* ref, const float* mag, const spindlekv_tensor& dst, cudaStream_t st);
+
 // ---- launch counting and timing ---------------------------------------------------------------
 static std::mutex g_mu;
 static int64_t g_launches = 0;
@@ -181,6 +184,17 @@ spindlekv_status spindlekv_compact(const spindlekv_batch* batch, int32_t n_heads
   if (src.dtype != dst.dtype) return SPINDLEKV_UNSUPPORTED;
   if (head_dim != 64 && head_dim != 128) return SPINDLEKV_UNSUPPORTED;
   return compact_impl(*batch, n_heads, head_dim, src, idx, cnt, divide_by, dst, dst_cu_seqlens, (cudaStream_t)stream);
+}
+
+spindlekv_status spindlekv_reconstruct(const spindlekv_batch* batch, int32_t n_heads, int32_t head_dim,
+                                       spindlekv_tensor C, const int32_t* ref, const float* mag, spindlekv_tensor dst,
+                                       void* stream) {
+  if (!batch || batch->n_layers <= 0 || batch->n_seqs <= 0 || batch->max_len <= 0 || n_heads <= 0) return SPINDLEKV_INVALID_ARG;
+  if (batch->layer_lens && batch->cu_seqlens) return SPINDLEKV_INVALID_ARG;
+  if (!tensor_ok(C) || !tensor_ok(dst) || !ref || !mag) return SPINDLEKV_INVALID_ARG;
+  if (C.dtype != dst.dtype) return SPINDLEKV_UNSUPPORTED;
+  if (head_dim != 64 && head_dim != 128) return SPINDLEKV_UNSUPPORTED;
+  return reconstruct_impl(*batch, n_heads, head_dim, C, ref, mag, dst, (cudaStream_t)stream);
 }
 
 spindlekv_status spindlekv_poll_status(const void* ws, int32_t* device_status, int32_t* detail) {

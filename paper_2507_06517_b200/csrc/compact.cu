@@ -58,6 +58,75 @@ __global__ void __launch_bounds__(256) compact_kernel(CompactParams p) {
   }
 }
 
+// ---- Eq. (14): Gamma_r = C[r] (x) m --------------------------------------------------------------
+// One group of head_dim*elem/16 threads per token: reads the token's entry row, scales it by the
+// token's magnitude in fp32, writes the row.
+struct ReconstructParams {
+  View C, dst;
+  Batch batch;
+  int n_heads;
+  const int32_t* ref;   // [layers][H][T]
+  const float* mag;     // [layers][H][T]
+};
+
+template <typename T, int D>
+__global__ void __launch_bounds__(256) reconstruct_kernel(ReconstructParams p) {
+  constexpr int EPT = 16 / sizeof(T);
+  constexpr int TPR = D / EPT;
+  constexpr int RPB = 256 / TPR;
+  const int unit = blockIdx.y;
+  const int h = unit % p.n_heads;
+  const int ls = unit / p.n_heads;
+  const int s = ls % p.batch.n_seqs;
+  const int layer = ls / p.batch.n_seqs;
+  const int l = seq_len(p.batch, layer, s);
+  const int64_t orow = ((int64_t)layer * p.n_heads + h) * p.batch.total_len + tok_base(p.batch, s);
+  const T* cbase = reinterpret_cast<const T*>(p.C.ptr) + unit_offset(p.C, p.batch, layer, s, h);
+  T* dbase = reinterpret_cast<T*>(const_cast<void*>(p.dst.ptr)) + unit_offset(p.dst, p.batch, layer, s, h);
+  const int seg = threadIdx.x % TPR;
+  for (int t = blockIdx.x * RPB + threadIdx.x / TPR; t < l; t += gridDim.x * RPB) {
+    const int r = p.ref[orow + t];
+    const float m = p.mag[orow + t];
+    uint4 v = *reinterpret_cast<const uint4*>(cbase + (int64_t)r * p.C.st + seg * EPT);
+    if (sizeof(T) == 4) {
+      float* f = reinterpret_cast<float*>(&v);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) f[i] *= m;
+    } else {
+      uint32_t* w = reinterpret_cast<uint32_t*>(&v);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const float lo = __uint_as_float(w[i] << 16) * m, hi = __uint_as_float(w[i] & 0xFFFF0000u) * m;
+        __nv_bfloat162 pk = __floats2bfloat162_rn(lo, hi);
+        w[i] = *reinterpret_cast<uint32_t*>(&pk);
+      }
+    }
+    *reinterpret_cast<uint4*>(dbase + (int64_t)t * p.dst.st + seg * EPT) = v;
+  }
+}
+
+spindlekv_status reconstruct_impl(const spindlekv_batch& b, int n_heads, int head_dim, const spindlekv_tensor& C,
+                                  const int32_t* ref, const float* mag, const spindlekv_tensor& dst, cudaStream_t st) {
+  ReconstructParams p;
+  p.C = make_view(C);
+  p.dst = make_view(dst);
+  p.batch = make_batch(b);
+  p.n_heads = n_heads;
+  p.ref = ref;
+  p.mag = mag;
+  const int units = b.n_layers * b.n_seqs * n_heads;
+  if (units > 65535) return SPINDLEKV_UNSUPPORTED;
+  dim3 grid(ceil_div(b.max_len, 64), units);
+  LaunchScope ls(KC_GATHER, st);
+  const bool bf = C.dtype == SPINDLEKV_BF16;
+  if (head_dim == 64) {
+    if (bf) reconstruct_kernel<__nv_bfloat16, 64><<<grid, 256, 0, st>>>(p); else reconstruct_kernel<float, 64><<<grid, 256, 0, st>>>(p);
+  } else {
+    if (bf) reconstruct_kernel<__nv_bfloat16, 128><<<grid, 256, 0, st>>>(p); else reconstruct_kernel<float, 128><<<grid, 256, 0, st>>>(p);
+  }
+  return cudaGetLastError() == cudaSuccess ? SPINDLEKV_OK : SPINDLEKV_CUDA;
+}
+
 spindlekv_status compact_impl(const spindlekv_batch& b, int n_heads, int head_dim, const spindlekv_tensor& src,
                               const int32_t* idx, const int32_t* cnt, const float* divide_by,
                               const spindlekv_tensor& dst, const int32_t* dst_cu, cudaStream_t st) {

@@ -224,6 +224,36 @@ def test_composition_as_written_evict_then_codebooks_of_the_kept_tokens():
         assert 0 < r1 <= 1 and 0 < r2 <= 1
 
 
+def test_reconstruction_from_the_codebook():
+    # Eq. (14): C[r] (x) m, against the checker's reconstruction from the same CodeBook rows; and the
+    # reconstructed rows keep each token's magnitude and a cosine above the threshold to the original
+    from paper_2507_06517_b200 import binding as B
+    for wl in (synth.Workload("rec32", 2, 2, 2, 2, 64, "f32", 8, (300, 300), 10, 0.1, 2, "gauss", budget_tokens=300.0, seed=61),
+               synth.Workload("rec16", 1, 1, 4, 2, 128, "bf16", 8, (333, 700, 128), 16, (0.03, 0.2), 2, "gauss",
+                              budget_frac=1.0, seed=62)):
+        host = generate(wl)
+        p = _pass(wl)
+        K = stack_layers(wl, host, list(range(wl.n_shallow)), "K")
+        p.codebook(K, "K")
+        o = p.cb["K"]
+        out = torch.zeros_like(K)
+        B.spindlekv_reconstruct(p.cb_batch, wl.n_kv_heads, wl.head_dim, p._desc(o["C"]), o["ref"], o["mag"], p._desc(out))
+        torch.cuda.synchronize()
+        got, Cn, ref, mag = out.float().cpu().numpy(), o["C"].float().cpu().numpy(), o["ref"].cpu().numpy(), o["mag"].cpu().numpy()
+        tol = value_tol(wl)
+        for li in range(wl.n_shallow):
+            for s, l in enumerate(wl.seq_lens):
+                tb = tok_base(wl, s)
+                for j in range(wl.n_kv_heads):
+                    want = O.reconstruct(unit_rows(wl, Cn[li], s, j), ref[li, j, tb:tb + l], mag[li, j, tb:tb + l])
+                    rows = unit_rows(wl, got[li], s, j)[:l]
+                    np.testing.assert_allclose(rows, want, rtol=tol, atol=tol * np.abs(want).max())
+                    orig = unit_rows(wl, host[li][0], s, j).astype(np.float64)
+                    cos = (rows * orig).sum(1) / (np.linalg.norm(rows, axis=1) * np.linalg.norm(orig, axis=1))
+                    assert np.all(cos > wl.theta_k - 2 * tol)
+                    np.testing.assert_allclose(np.linalg.norm(rows, axis=1), mag[li, j, tb:tb + l], rtol=2 * tol)
+
+
 def test_plain_window_sum_extension():
     wl = synth.Workload("rawsum", 1, 0, 4, 2, 64, "f32", 32, (333,), 8, 0.1, 2, "gauss", budget_tokens=80.0, seed=14)
     run_and_check(wl, {"score_norm": 1})
