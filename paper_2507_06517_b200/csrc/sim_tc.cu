@@ -5,8 +5,10 @@
 //
 // One CTA owns a block of 128 token rows of one (layer, sequence, head) unit: the block is loaded
 // once by TMA and stays in shared memory as operand A; tiles of 256 token rows, from the tile that
-// holds the diagonal onwards, stream through a two-stage ring as operand B.  One elected thread
-// issues tcgen05.mma (128 x 256 x 16, fp32 accumulation in TMEM).
+// holds the diagonal onwards, stream through a ring as operand B.  Two CTAs (a cluster) own the two
+// blocks of a 256-row span and share one MMA stream: each loads only its half of every streamed tile,
+// and one elected thread of the first CTA issues tcgen05.mma.cta_group::2 (256 x 256 x 16, fp32
+// accumulation in both CTAs' TMEM, 128 rows each), which halves the operand traffic per SM.
 //
 // The threshold is part of the contraction.  The main K-steps run with the negate-A flag and
 // accumulate -gamma_a . gamma_b; one more K-step multiplies two 16-element rows prepared by the
@@ -44,7 +46,8 @@ struct SimTcParams {
 
 constexpr int kBM = 128;          // rows of the resident block (UMMA M)
 constexpr int kBN = 256;          // rows of a streamed tile (UMMA N)
-constexpr int kStages = 2;
+constexpr int kStages = 4;         // shared-memory ring of streamed half tiles (TMEM ring: 2 accumulators)
+constexpr int kBH = kBN / 2;       // rows of a streamed tile that one CTA of the pair loads
 constexpr int kEpiWarps = 16;                         // two teams of eight; team e serves TMEM stage e
 constexpr int kTeamWarps = kEpiWarps / 2;
 constexpr int kColsPerWarp = kBN / (kTeamWarps / 4);  // tile columns handled by one epilogue warp
@@ -58,9 +61,9 @@ template <int D>
 struct SimSmem {
   static constexpr int KH = D / 64;                  // 64-element (128-byte) swizzle atoms along head_dim
   static constexpr int A_BYTES = KH * kBM * 128;
-  static constexpr int B_BYTES = KH * kBN * 128;
+  static constexpr int B_BYTES = KH * kBH * 128;     // this CTA's half of a streamed tile
   static constexpr int EA_BYTES = kBM * 32;          // threshold rows of the block (one 16-element K-step)
-  static constexpr int EB_BYTES = kBN * 32;          // magnitude rows of a tile
+  static constexpr int EB_BYTES = kBH * 32;          // magnitude rows of this CTA's half tile
   static constexpr int T_BYTES = 2 * 4 * kBN * 4;    // mirrored words [slot][row quarter][tile column]
   static constexpr int D_BYTES = 2 * 2 * kBM * kDPitch * 4;  // direct words [team][slot][row][word]
   static constexpr int OFF_B = A_BYTES;
@@ -90,8 +93,63 @@ __device__ __forceinline__ uint32_t sign_word(const uint32_t (&acc)[32]) {
   return __byte_perm(__byte_perm(wg[0], wg[1], 0x0040), __byte_perm(wg[2], wg[3], 0x0040), 0x5410);
 }
 
+// ---- CTA pairs ------------------------------------------------------------------------------------
+// Two CTAs of a cluster (ranks 0 and 1) own the two 128-row blocks of a 256-row span and run one
+// tcgen05.mma.cta_group::2 stream, issued by rank 0: each CTA holds its own block (operand A) and loads
+// only its half of every streamed tile (operand B), which halves the operand traffic per SM.
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// address of the same shared-memory location in the pair's rank-0 CTA
+__device__ __forceinline__ uint32_t leader_addr(const void* p) { return ptx::smem_u32(p) & 0xFEFFFFFFu; }
+__device__ __forceinline__ void mbar_arrive_leader(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(leader_addr(bar)) : "memory");
+}
+// tiled TMA loads into this CTA's shared memory whose completion is counted on the leader's barrier
+__device__ __forceinline__ void tma_load_5d_pair(void* smem_dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1,
+                                                 int c2, int c3, int c4) {
+  asm volatile(
+      "cp.async.bulk.tensor.5d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+      ::"r"(ptx::smem_u32(smem_dst)), "l"(map), "r"(leader_addr(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_4d_pair(void* smem_dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1,
+                                                 int c2, int c3) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+      ::"r"(ptx::smem_u32(smem_dst)), "l"(map), "r"(leader_addr(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t* smem_result, uint32_t ncols) {  // warp 1 of both CTAs
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(ptx::smem_u32(smem_result)), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish_pair() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// arrive on the same barrier in both CTAs once all MMAs issued so far have completed
+__device__ __forceinline__ void umma_commit_pair(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(ptx::smem_u32(bar)), "h"((uint16_t)3) : "memory");
+}
+
 template <int D>
-__global__ void __launch_bounds__(kSimThreads, 1) sim_tc_kernel(const __grid_constant__ CUtensorMap tmap,
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kSimThreads, 1) sim_tc_kernel(const __grid_constant__ CUtensorMap tmap,
                                                                 const __grid_constant__ CUtensorMap emap,
                                                                 SimTcParams p) {
   using L = SimSmem<D>;
@@ -102,9 +160,10 @@ __global__ void __launch_bounds__(kSimThreads, 1) sim_tc_kernel(const __grid_con
   const int layer = ls / p.batch.n_seqs;
   const int l = seq_len(p.batch, layer, s);
   const int row0 = blockIdx.x * kBM;
-  if (row0 >= l) return;
+  const int rank = (int)cluster_ctarank();   // = blockIdx.x & 1
+  if ((row0 & ~(kBN - 1)) >= l) return;      // both CTAs of a pair: the whole 256-row span lies beyond the sequence
   const int n_tiles = (l + kBN - 1) / kBN;   // tiles of this sequence: columns beyond its end are never produced
-  const int tile0 = row0 / kBN;   // the tile that holds this block's diagonal; earlier tiles are mirrored by other blocks
+  const int tile0 = row0 / kBN;   // the tile that holds the pair's diagonal; earlier tiles are mirrored by other pairs
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -115,28 +174,30 @@ __global__ void __launch_bounds__(kSimThreads, 1) sim_tc_kernel(const __grid_con
   uint32_t* sT = reinterpret_cast<uint32_t*>(smem + L::OFF_T);
   uint32_t* sD = reinterpret_cast<uint32_t*>(smem + L::OFF_D);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::OFF_BAR);
+  // a_full, b_full and acc_empty are used in the leader (rank 0) only: both CTAs' loads and both CTAs'
+  // epilogue warps signal them there; b_empty and acc_full are signalled in both CTAs by the leader's commits
   uint64_t* a_full = bars + 0;
-  uint64_t* b_full = bars + 1;      // [kStages]
-  uint64_t* b_empty = bars + 3;     // [kStages]
-  uint64_t* acc_full = bars + 5;    // [2]
-  uint64_t* acc_empty = bars + 7;   // [2]
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 9);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 10);
+  uint64_t* b_full = bars + 1;                  // [kStages]
+  uint64_t* b_empty = bars + 1 + kStages;       // [kStages]
+  uint64_t* acc_full = bars + 1 + 2 * kStages;  // [2]
+  uint64_t* acc_empty = acc_full + 2;           // [2]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(acc_empty + 3);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
     ptx::mbar_init(a_full, 1);
     for (int i = 0; i < kStages; ++i) { ptx::mbar_init(b_full + i, 1); ptx::mbar_init(b_empty + i, 1); }
-    for (int i = 0; i < 2; ++i) { ptx::mbar_init(acc_full + i, 1); ptx::mbar_init(acc_empty + i, kTeamWarps); }
+    for (int i = 0; i < 2; ++i) { ptx::mbar_init(acc_full + i, 1); ptx::mbar_init(acc_empty + i, 2 * kTeamWarps); }
     *abort_flag = 0;
     ptx::fence_barrier_init();
   }
   if (warp == 1) {
-    ptx::tmem_alloc(tmem_slot, 512);
-    ptx::tmem_relinquish();
+    tmem_alloc_pair(tmem_slot, 512);
+    tmem_relinquish_pair();
   }
   ptx::tc_fence_before();
-  __syncthreads();
+  cluster_sync_all();   // barriers of both CTAs are initialised before either signals the other
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
@@ -147,49 +208,45 @@ __global__ void __launch_bounds__(kSimThreads, 1) sim_tc_kernel(const __grid_con
     if (lane == 0) {
       ptx::prefetch_tensormap(&tmap);
       ptx::prefetch_tensormap(&emap);
-      ptx::mbar_expect_tx(a_full, L::A_BYTES + L::EA_BYTES);
+      if (rank == 0) ptx::mbar_expect_tx(a_full, 2 * (L::A_BYTES + L::EA_BYTES));
       for (int kh = 0; kh < L::KH; ++kh)
-        ptx::tma_load_5d(sA + kh * kBM * 128, &tmap, a_full, kh * 64, tok0 + row0, j, sdim, layer);
-      ptx::tma_load_4d(sEA, &emap, a_full, 0, row0, unit, 0);
+        tma_load_5d_pair(sA + kh * kBM * 128, &tmap, a_full, kh * 64, tok0 + row0, j, sdim, layer);
+      tma_load_4d_pair(sEA, &emap, a_full, 0, row0, unit, 0);
       for (int it = 0; tile0 + it < n_tiles; ++it) {
-        const int st = it & 1;
-        if (!ptx::mbar_wait(b_empty + st, ((it >> 1) & 1) ^ 1, abort_flag)) break;
-        ptx::mbar_expect_tx(b_full + st, L::B_BYTES + L::EB_BYTES);
+        const int st = it % kStages;
+        if (!ptx::mbar_wait(b_empty + st, ((it / kStages) & 1) ^ 1, abort_flag)) break;
+        if (rank == 0) ptx::mbar_expect_tx(b_full + st, 2 * (L::B_BYTES + L::EB_BYTES));
         uint8_t* dst = sB + st * L::B_BYTES;
+        const int brow = (tile0 + it) * kBN + rank * kBH;   // this CTA's half of the tile
         for (int kh = 0; kh < L::KH; ++kh)
-          for (int half = 0; half < 2; ++half)
-            ptx::tma_load_5d(dst + kh * kBN * 128 + half * 128 * 128, &tmap, b_full + st, kh * 64,
-                             tok0 + (tile0 + it) * kBN + half * 128, j, sdim, layer);
-        for (int half = 0; half < 2; ++half)
-          ptx::tma_load_4d(sEB + st * L::EB_BYTES + half * 128 * 32, &emap, b_full + st, 0,
-                           (tile0 + it) * kBN + half * 128, unit, 1);
+          tma_load_5d_pair(dst + kh * kBH * 128, &tmap, b_full + st, kh * 64, tok0 + brow, j, sdim, layer);
+        tma_load_4d_pair(sEB + st * L::EB_BYTES, &emap, b_full + st, 0, brow, unit, 1);
       }
     }
   } else if (warp == 1) {
-    if (lane == 0) {
-      constexpr uint32_t idesc_neg = ptx::idesc_bf16_f32(kBM, kBN, true);
-      constexpr uint32_t idesc_pos = ptx::idesc_bf16_f32(kBM, kBN, false);
+    if (lane == 0 && rank == 0) {
+      constexpr uint32_t idesc_neg = ptx::idesc_bf16_f32(2 * kBM, kBN, true);
+      constexpr uint32_t idesc_pos = ptx::idesc_bf16_f32(2 * kBM, kBN, false);
       const uint32_t a_addr = ptx::smem_u32(sA);
       const uint64_t dea = ptx::smem_desc_sw32(ptx::smem_u32(sEA));
       bool ok = ptx::mbar_wait(a_full, 0, abort_flag);
       for (int it = 0; ok && tile0 + it < n_tiles; ++it) {
-        const int st = it & 1;
-        const uint32_t ph = (it >> 1) & 1;
-        if (!ptx::mbar_wait(b_full + st, ph, abort_flag)) break;
-        if (!ptx::mbar_wait(acc_empty + st, ph ^ 1, abort_flag)) break;
+        const int st = it % kStages, as = it & 1;
+        if (!ptx::mbar_wait(b_full + st, (it / kStages) & 1, abort_flag)) break;
+        if (!ptx::mbar_wait(acc_empty + as, ((it >> 1) & 1) ^ 1, abort_flag)) break;
         ptx::tc_fence_after();
         const uint32_t b_addr = ptx::smem_u32(sB + st * L::B_BYTES);
 #pragma unroll
         for (int k = 0; k < D / 16; ++k) {
           const int kh = k >> 2, kk = k & 3;
           uint64_t da = ptx::smem_desc_sw128(a_addr + kh * kBM * 128 + kk * 32);
-          uint64_t db = ptx::smem_desc_sw128(b_addr + kh * kBN * 128 + kk * 32);
-          ptx::umma_bf16(tmem_base + st * kBN, da, db, idesc_neg, k > 0 ? 1u : 0u);
+          uint64_t db = ptx::smem_desc_sw128(b_addr + kh * kBH * 128 + kk * 32);
+          umma_bf16_pair(tmem_base + as * kBN, da, db, idesc_neg, k > 0 ? 1u : 0u);
         }
         // + theta * |a| * |b|
-        ptx::umma_bf16(tmem_base + st * kBN, dea, ptx::smem_desc_sw32(ptx::smem_u32(sEB + st * L::EB_BYTES)), idesc_pos, 1u);
-        ptx::umma_commit(b_empty + st);   // shared-memory stage may be refilled
-        ptx::umma_commit(acc_full + st);  // accumulator ready for the epilogue
+        umma_bf16_pair(tmem_base + as * kBN, dea, ptx::smem_desc_sw32(ptx::smem_u32(sEB + st * L::EB_BYTES)), idesc_pos, 1u);
+        umma_commit_pair(b_empty + st);   // both CTAs: the stage may be refilled
+        umma_commit_pair(acc_full + as);  // both CTAs: accumulator ready for the epilogue
       }
     }
   } else {
@@ -205,7 +262,10 @@ __global__ void __launch_bounds__(kSimThreads, 1) sim_tc_kernel(const __grid_con
     const int NC = RW >> 1;               // 64-column chunks per row
     const int blk = blockIdx.x;
     uint32_t* funit = p.flags + (int64_t)unit * NC * RW;
-    if (lane == 0) {
+    // the second CTA of a sequence's last pair may own no row at all: it still loads its half tiles and
+    // keeps the barrier protocol going, but reads and writes nothing
+    const bool live_block = row0 < l;
+    if (lane == 0 && live_block) {
       // The two chunks that hold the block's own 128 columns are flagged as occupied without looking:
       // for the block's rows (diagonal bit, and words mirrored inside the block), and, from an even
       // block, for the rows of the next block, which its diagonal tile mirrors into piecemeal.
@@ -229,7 +289,11 @@ __global__ void __launch_bounds__(kSimThreads, 1) sim_tc_kernel(const __grid_con
       const int slot = (tile >> 1) & 1;        // which of the team's two tiles of the four-tile span
       uint32_t* sdbuf = sD_team + ((tile >> 2) & 1) * (kBM * kDPitch);
       uint32_t* sdw = sdbuf + rl * kDPitch + slot * kTileWords + cg * kChunks;
-      const bool ok = __all_sync(0xffffffffu, ptx::mbar_wait(acc_full + team, (it >> 1) & 1, abort_flag));
+      bool ok = __all_sync(0xffffffffu, ptx::mbar_wait(acc_full + team, (it >> 1) & 1, abort_flag));
+      if (ok && !live_block) {
+        if (lane == 0) mbar_arrive_leader(acc_empty + team);
+        ok = false;
+      }
       if (ok) {
         ptx::tc_fence_after();
         uint32_t words[kChunks];
@@ -242,7 +306,7 @@ __global__ void __launch_bounds__(kSimThreads, 1) sim_tc_kernel(const __grid_con
         }
         ptx::tc_fence_before();
         __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(acc_empty + team);
+        if (lane == 0) mbar_arrive_leader(acc_empty + team);
         if (c0 + kBN > l || R + 32 > l) {
           // ragged edge: columns and rows that do not exist carry no bits
 #pragma unroll
@@ -326,9 +390,10 @@ __global__ void __launch_bounds__(kSimThreads, 1) sim_tc_kernel(const __grid_con
     if (threadIdx.x == 0) atomicExch(&p.hdr[kHdrStatus], (uint32_t)SPINDLEKV_TIMEOUT);
     __nanosleep(100000);  // let any bulk copy still in flight land before the block retires
   }
+  cluster_sync_all();   // neither CTA leaves (or frees TMEM) while its partner may still signal it or use its memory
   if (warp == 1) {
     ptx::tc_fence_after();
-    ptx::tmem_dealloc(tmem_base, 512);
+    tmem_dealloc_pair(tmem_base, 512);
   }
 }
 
@@ -434,7 +499,7 @@ spindlekv_status launch_sim_tc(const spindlekv_tensor& Gamma, const spindlekv_ba
   p.adj = adj;
   p.flags = flags;
   p.hdr = hdr;
-  dim3 grid(ceil_div(b.max_len, kBM), units);
+  dim3 grid(2 * ceil_div(b.max_len, 2 * kBM), units);   // whole pairs
   LaunchScope ls(KC_SIM, st);
   if (head_dim == 128) {
     static bool set = false;

@@ -35,13 +35,19 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   return ok != 0;
 }
 // Bounded wait.  `abort_flag` (shared memory) lets one role's failure release the others quickly.
-constexpr uint32_t kMbarSpinLimit = 1u << 24;
+// The bound is in time (about two seconds of SM clock), not in polls: a poll may itself block for a
+// hardware-chosen while.
+constexpr long long kMbarWaitCycles = 4000000000ll;
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
   if (mbar_try_wait(bar, parity)) return true;
   if (*abort_flag) return false;
-  for (uint32_t i = 0; i < kMbarSpinLimit; ++i) {
+  const long long t0 = clock64();
+  for (uint32_t i = 0;; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
-    if ((i & 1023u) == 1023u && *abort_flag) return false;
+    if ((i & 63u) == 63u) {
+      if (*abort_flag) return false;
+      if (clock64() - t0 > kMbarWaitCycles) break;
+    }
   }
   *abort_flag = 1;
   return false;
