@@ -194,6 +194,21 @@ spindlekv_status spindlekv_compact(const spindlekv_batch* batch, int32_t n_heads
                                    void* stream);
 
 /*
+ * Joins the kept-token lists of several eviction passes over the same KV heads (Section 3.3, the GQA
+ * "repeat" alternative: the KV vectors are repeated h_n times, every query head of a group selects on its
+ * own, and the CodeBook of Section 3.4 is built from all selections of the group, where repeated
+ * tokens have cosine similarity 1 and share an entry).  For every (layer, seq, head): out list = list of
+ * pass 0, then of pass 1, ...; out count = sum of the counts (clipped to seq_out).  Equal-length batches only.
+ *   idx_in  device [n_lists][n_layers][n_heads][t_in], sequence s starting at column s * seq_in
+ *   cnt_in  device [n_lists][n_layers][n_seqs][n_heads]
+ *   idx_out device [n_layers][n_heads][t_out], sequence s starting at column s * seq_out
+ *   cnt_out device [n_layers][n_seqs][n_heads]
+ */
+spindlekv_status spindlekv_union_lists(int32_t n_layers, int32_t n_seqs, int32_t n_heads, int32_t n_lists,
+                                       int32_t t_in, int32_t seq_in, const int32_t* idx_in, const int32_t* cnt_in,
+                                       int32_t t_out, int32_t seq_out, int32_t* idx_out, int32_t* cnt_out, void* stream);
+
+/*
  * Reconstruction of the replaced cache from a CodeBook (Eq. (14): Gamma_r = C[r] (x) m): for every
  * (layer, seq, head) and token t of the sequence, dst row t = C row ref[t] times mag[t] (product in fp32,
  * rounded to the storage type).

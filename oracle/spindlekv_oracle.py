@@ -362,6 +362,31 @@ def spindle_layer(q_win_heads: np.ndarray, k_heads: np.ndarray, v_heads: np.ndar
     return {"keep": ev["keep"], "scores": ev["scores"], "cb_k": cb_k, "cb_v": cb_v}
 
 
+def spindle_layer_repeat(q_win_heads: np.ndarray, k_heads: np.ndarray, v_heads: np.ndarray, k_ctx: int,
+                         theta_k: float, theta_v: float) -> Dict[str, object]:
+    """The GQA "repeat" alternative of Section 3.3: the KV vectors are repeated ``h_n`` times, so that
+    every query head ``i`` selects by its own ``ac_i`` of Eq. (2) (no group mean), and the CodeBooks of KV
+    head ``j`` are built (Section 3.4) from the rows kept by its query heads ``h_n*j .. h_n*j + h_n - 1``,
+    one head after the other; a token kept by several heads appears several times (cosine 1).
+
+    Reading (the paper does not say over which tokens the CodeBook of a repeated cache is built): per KV
+    head, over the concatenation above.  Returns ``keep[H_q, k + w]``, ``union[H_kv, h_n (k + w)]`` and the
+    per-KV-head CodeBook results.
+    """
+    H_q, w = q_win_heads.shape[0], q_win_heads.shape[1]
+    H_kv, l, _ = k_heads.shape
+    h_n = H_q // H_kv
+    keep = np.empty((H_q, k_ctx + w), dtype=np.int32)
+    scores = np.empty((H_q, l - w), dtype=np.float64)
+    for i in range(H_q):
+        ev = evict_deep(q_win_heads[i:i + 1], k_heads[i // h_n:i // h_n + 1], k_ctx)
+        keep[i], scores[i] = ev["keep"][0], ev["scores"][0]
+    union = keep.reshape(H_kv, h_n * (k_ctx + w))
+    cb_k = [codebook_shallow(gather_rows(k_heads[j], union[j]), theta_k) for j in range(H_kv)]
+    cb_v = [codebook_shallow(gather_rows(v_heads[j], union[j]), theta_v) for j in range(H_kv)]
+    return {"keep": keep, "scores": scores, "union": union, "cb_k": cb_k, "cb_v": cb_v}
+
+
 def reserve_ratio_layer(l: int, kept: int, entries_k: Sequence[int], entries_v: Sequence[int]) -> Tuple[float, float]:
     """Eq. (15) for one layer: ``r1`` = kept K and V tokens over all K and V tokens (summed over the
     KV heads), ``r2`` = CodeBook entries of K and V over kept K and V tokens.  The dtype factor

@@ -69,6 +69,9 @@ def _load() -> C.CDLL:
     lib.spindlekv_compact.restype = C.c_int32
     lib.spindlekv_compact.argtypes = [C.POINTER(_Batch), C.c_int32, C.c_int32, _Tensor, C.c_void_p, C.c_void_p,
                                       C.c_void_p, _Tensor, C.c_void_p, C.c_void_p]
+    lib.spindlekv_union_lists.restype = C.c_int32
+    lib.spindlekv_union_lists.argtypes = [C.c_int32] * 6 + [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_void_p,
+                                                            C.c_void_p, C.c_void_p]
     lib.spindlekv_reconstruct.restype = C.c_int32
     lib.spindlekv_reconstruct.argtypes = [C.POINTER(_Batch), C.c_int32, C.c_int32, _Tensor, C.c_void_p, C.c_void_p,
                                           _Tensor, C.c_void_p]
@@ -218,6 +221,14 @@ def spindlekv_compact(batch: Batch, n_heads: int, head_dim: int, src: _Tensor, i
     st = _lib.spindlekv_compact(C.byref(bb), n_heads, head_dim, src, _ptr(idx), _ptr(cnt), _ptr(divide_by), dst,
                                 _ptr(dst_cu_seqlens), _stream(stream))
     _check(st, "spindlekv_compact")
+
+
+def spindlekv_union_lists(n_layers: int, n_seqs: int, n_heads: int, idx_in: torch.Tensor, cnt_in: torch.Tensor,
+                          seq_in: int, idx_out: torch.Tensor, cnt_out: torch.Tensor, seq_out: int, stream=None) -> None:
+    """``idx_in [n_lists, L, H, t_in]``, ``cnt_in [n_lists, L, B, H]`` -> ``idx_out [L, H, t_out]``, ``cnt_out [L, B, H]``."""
+    st = _lib.spindlekv_union_lists(n_layers, n_seqs, n_heads, idx_in.shape[0], idx_in.shape[-1], seq_in, _ptr(idx_in),
+                                    _ptr(cnt_in), idx_out.shape[-1], seq_out, _ptr(idx_out), _ptr(cnt_out), _stream(stream))
+    _check(st, "spindlekv_union_lists")
 
 
 def spindlekv_reconstruct(batch: Batch, n_heads: int, head_dim: int, Cb: _Tensor, ref: torch.Tensor,

@@ -284,3 +284,87 @@ class SpindleKVLiteralPass:
     def device_status(self):
         torch.cuda.synchronize(self.device)
         return {"evict": B.spindlekv_poll_status(self.ev.ws_evict), "codebook": B.spindlekv_poll_status(self.ws_codebook)}
+
+
+class SpindleKVRepeatPass:
+    """The GQA "repeat" alternative of Section 3.3 inside the composition as written: the KV vectors of
+    a group are taken once per query head, so every query head selects its own tokens (Eq. (2)(7) without
+    the group mean of Eq. (3)); the K and V CodeBooks of a KV head are then built from the tokens all
+    its query heads kept, listed one head after the other, where a token kept by several heads
+    appears several times and collapses into one entry (cosine similarity 1).  ``cfg.n_shallow`` must
+    be -1; equal-length sequences.  ``K``, ``V``: ``[L, B, H_kv, N, d]``; ``Q``: ``[L, B, H_q, w, d]``.
+    Buffers and call order only.
+    """
+
+    def __init__(self, cfg: B.Config, seq_lens: Sequence[int], dtype: torch.dtype, device="cuda",
+                 keep_adjacency: bool = False):
+        if cfg.n_shallow != -1:
+            raise ValueError("SpindleKVRepeatPass needs cfg.n_shallow == -1")
+        if len(set(int(x) for x in seq_lens)) != 1:
+            raise ValueError("SpindleKVRepeatPass needs sequences of equal length")
+        self.cfg = cfg
+        self.device = dev = torch.device(device)
+        self.h_n = cfg.n_q_heads // cfg.n_kv_heads
+        L, nB, H, d, N = cfg.n_layers, len(seq_lens), cfg.n_kv_heads, cfg.head_dim, int(seq_lens[0])
+        self.n_seqs, self.max_len = nB, N
+        # one eviction call per position g in the group: query heads g, h_n + g, ... against the KV heads
+        self.ecfg = dataclasses.replace(cfg, n_q_heads=H, n_shallow=0)
+        self.mode, self.ratio, self.k_ctx_host = B.spindlekv_plan_layers(cfg, list(seq_lens))
+        self.k_ctx = torch.from_numpy(np.ascontiguousarray(self.k_ctx_host)).to(dev)
+        self.ev_batch = B.Batch(L, nB, N, nB * N)
+        i32 = dict(dtype=torch.int32, device=dev)
+        self.keep_idx = torch.zeros((self.h_n, L, H, nB * N), **i32)
+        self.keep_cnt = torch.zeros((self.h_n, L, nB, H), **i32)
+        self.scores = torch.zeros((self.h_n, L, H, nB * N), dtype=torch.float32, device=dev)
+        self.ws_evict = torch.empty(B.spindlekv_workspace_bytes(self.ecfg, self.ev_batch, B.WS_EVICT), dtype=torch.uint8, device=dev)
+        self.kept_host = (self.k_ctx_host + cfg.window).astype(np.int32)                     # per query head
+        self.union_host = (self.h_n * self.kept_host).astype(np.int32)                       # per KV head
+        self.max_union = int(self.union_host.max())
+        self.layer_lens = torch.from_numpy(np.ascontiguousarray(self.union_host)).to(dev)
+        T = nB * self.max_union
+        self.union_idx = torch.zeros((L, H, T), **i32)
+        self.union_cnt = torch.zeros((L, nB, H), **i32)
+        self.cb_batch = B.Batch(L, nB, self.max_union, T, None, self.layer_lens)
+        self.gather_batch = B.Batch(L, nB, N, nB * N)
+        self.ws_codebook = torch.empty(B.spindlekv_workspace_bytes(cfg, self.cb_batch, B.WS_CODEBOOK), dtype=torch.uint8, device=dev)
+        self.rep = {g: torch.zeros((L, nB, H, self.max_union, d), dtype=dtype, device=dev) for g in ("K", "V")}
+        self.cb: Dict[str, Dict[str, torch.Tensor]] = {}
+        for g in ("K", "V"):
+            self.cb[g] = {
+                "mag": torch.zeros((L, H, T), dtype=torch.float32, device=dev),
+                "ref": torch.zeros((L, H, T), **i32),
+                "centre_idx": torch.zeros((L, H, T), **i32),
+                "n_entries": torch.zeros((L, nB, H), **i32),
+                "C": torch.zeros((L, nB, H, self.max_union, d), dtype=dtype, device=dev),
+            }
+        self.adj = torch.zeros((L * nB * H, self.max_union, B.row_words(self.max_union)), **i32) if keep_adjacency else None
+
+    def run(self, K: torch.Tensor, V: torch.Tensor, Q: torch.Tensor, which=("K", "V"), stream=None) -> None:
+        cfg, H, d = self.cfg, self.cfg.n_kv_heads, self.cfg.head_dim
+        for g in range(self.h_n):
+            B.spindlekv_evict_deep(self.ecfg, self.ev_batch, B.desc_bhnd(K), B.desc_bhnd(Q[:, :, g::self.h_n]), self.k_ctx,
+                                   self.keep_idx[g], self.keep_cnt[g], self.scores[g], self.ws_evict, stream)
+        B.spindlekv_union_lists(cfg.n_layers, self.n_seqs, H, self.keep_idx, self.keep_cnt, self.max_len,
+                                self.union_idx, self.union_cnt, self.max_union, stream)
+        for g in which:
+            src, rep, o = (K if g == "K" else V), self.rep[g], self.cb[g]
+            # rows of the union list, gathered from the KV head (the union list is laid out per max_union tokens,
+            # the source per max_len tokens: two batches describe the two sides)
+            self._gather(src, rep, stream)
+            B.spindlekv_codebook_shallow(cfg, self.cb_batch, B.desc_bhnd(rep), cfg.theta_k if g == "K" else cfg.theta_v,
+                                         o["mag"], o["ref"], o["centre_idx"], o["n_entries"], self.ws_codebook,
+                                         self.adj, stream)
+            B.spindlekv_compact(self.cb_batch, H, d, B.desc_bhnd(rep), o["centre_idx"], o["n_entries"],
+                                B.desc_bhnd(o["C"]), o["mag"], None, stream)
+
+    def _gather(self, src: torch.Tensor, rep: torch.Tensor, stream=None) -> None:
+        # index rows are [L][H][B * max_union]; the compaction call addresses source rows through the batch's
+        # max_len and index rows through total_len, so the batch carries the index layout and the source
+        # tensor descriptor carries its own strides
+        cfg = self.cfg
+        B.spindlekv_compact(self.cb_batch, cfg.n_kv_heads, cfg.head_dim, B.desc_bhnd(src), self.union_idx, self.union_cnt,
+                            B.desc_bhnd(rep), None, None, stream)
+
+    def device_status(self):
+        torch.cuda.synchronize(self.device)
+        return {"evict": B.spindlekv_poll_status(self.ws_evict), "codebook": B.spindlekv_poll_status(self.ws_codebook)}

@@ -224,6 +224,46 @@ def test_composition_as_written_evict_then_codebooks_of_the_kept_tokens():
         assert 0 < r1 <= 1 and 0 < r2 <= 1
 
 
+def test_gqa_repeat_variant():
+    # every query head selects on its own; the CodeBooks of a KV head are built from all its query heads' tokens
+    from paper_2507_06517_b200.pipeline import SpindleKVRepeatPass
+    wl = synth.Workload("repeat", 2, -1, 8, 2, 128, "bf16", 32, (640,), 12, (0.03, 0.3), 2, "recency",
+                        budget_tokens=150.0, seed=71)
+    layers = list(range(wl.n_layers))
+    host = {lam: synth.layer_arrays(wl, lam, need_q=True) for lam in layers}
+    K, V, Q = (stack_layers(wl, host, layers, x) for x in ("K", "V", "Q"))
+    p = SpindleKVRepeatPass(make_config(wl), wl.seq_lens, torch_dtype(wl), keep_adjacency=True)
+    _, _, k_plan = O.plan_layers(wl.n_layers, -1, wl.seq_lens, wl.window, wl.beta, budget_tokens=wl.budget_tokens)
+    H, h_n, l, w = wl.n_kv_heads, wl.group, wl.max_len, wl.window
+    one = wl.replace(n_q_heads=H)   # a group of one query head per KV head, as each eviction call sees it
+    for g, idx, theta in (("K", 0, wl.theta_k), ("V", 1, wl.theta_v)):
+        p.run(K, V, Q, which=(g,))
+        st = p.device_status()
+        assert st["evict"][0] == 0 and st["codebook"][0] == 0 and st["codebook"][1][1] == 0
+        keep, cnt, scores = p.keep_idx.cpu().numpy(), p.keep_cnt.cpu().numpy(), p.scores.cpu().numpy()
+        union, ucnt = p.union_idx.cpu().numpy(), p.union_cnt.cpu().numpy()
+        o = {k: (v.float() if k == "C" else v).cpu().numpy() for k, v in p.cb[g].items()}
+        adj = p.adj.cpu().numpy()
+        for lam in layers:
+            k_ctx = int(k_plan[lam, 0])
+            n = k_ctx + w
+            Ks = np.stack([host[lam][0][0, j] for j in range(H)])
+            for gq in range(h_n):
+                check_evict_unit(one, host[lam][2][0][gq::h_n], Ks, k_ctx, scores[gq, lam], keep[gq, lam], cnt[gq, lam, 0])
+            for j in range(H):
+                assert ucnt[lam, 0, j] == h_n * n
+                want_union = np.concatenate([keep[gq, lam, j, :n] for gq in range(h_n)])
+                assert np.array_equal(union[lam, j, : h_n * n], want_union)
+                gamma = host[lam][idx][0, j][want_union]
+                check_codebook_unit(gamma, theta, adj[lam * H + j], o["mag"][lam, j, : h_n * n], o["ref"][lam, j, : h_n * n],
+                                    o["centre_idx"][lam, j, : h_n * n], int(o["n_entries"][lam, 0, j]), o["C"][lam, 0, j],
+                                    value_tol(wl))
+                # copies of a token share an entry
+                ref = o["ref"][lam, j, : h_n * n]
+                for tok in np.unique(want_union):
+                    assert len(set(ref[want_union == tok])) == 1
+
+
 def test_reconstruction_from_the_codebook():
     # Eq. (14): C[r] (x) m, against the checker's reconstruction from the same CodeBook rows; and the
     # reconstructed rows keep each token's magnitude and a cosine above the threshold to the original

@@ -62,3 +62,33 @@ def test_no_merging_and_total_merging():
     assert r2 == pytest.approx(1 / 26)
     r1, r2 = O.reserve_ratio_layer(100, 40, [10, 30], [20, 20])
     assert r1 == pytest.approx(0.4) and r2 == pytest.approx(80 / 160)
+
+
+def test_repeat_variant_selects_per_query_head_and_collapses_repeats():
+    rng = np.random.default_rng(7)
+    l, w, d, H, h_n = 100, 6, 16, 2, 3
+    k, v = rng.standard_normal((H, l, d)), rng.standard_normal((H, l, d))
+    q = rng.standard_normal((H * h_n, w, d))
+    out = O.spindle_layer_repeat(q, k, v, 10, 0.999, 0.999)
+    for i in range(H * h_n):
+        # a query head's selection is what the group formula gives for a group of one (Eq. (3) with h_n = 1)
+        alone = O.evict_deep(q[i:i + 1], k[i // h_n:i // h_n + 1], 10)
+        assert np.array_equal(out["keep"][i], alone["keep"][0])
+    for j in range(H):
+        u = out["union"][j]
+        assert np.array_equal(u, np.concatenate([out["keep"][h_n * j + g] for g in range(h_n)]))
+        cb = out["cb_k"][j]
+        # random directions: nothing merges except copies of the same token, so entries = distinct tokens,
+        # and copies (the window, kept by every head, among them) share their entry
+        assert len(cb["centres"]) == len(set(u.tolist()))
+        first = {}
+        for pos, tok in enumerate(u):
+            first.setdefault(int(tok), cb["ref"][pos])
+            assert cb["ref"][pos] == first[int(tok)]
+    # identical query heads in a group select identical tokens: the union is h_n copies, entries as without repeat
+    q_same = np.repeat(q[::h_n], h_n, axis=0)
+    rep = O.spindle_layer_repeat(q_same, k, v, 10, 0.999, 0.999)
+    base = O.spindle_layer(q_same, k, v, 10, 0.999, 0.999)   # group mean of equal scores = the score itself
+    for j in range(H):
+        assert np.array_equal(rep["keep"][h_n * j], base["keep"][j])
+        assert len(rep["cb_k"][j]["centres"]) == len(base["cb_k"][j]["centres"])
