@@ -221,6 +221,7 @@ __device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long v)
 // and are appended to a list of dense rows.  A token with no neighbour at all is settled here: it is
 // a centre with pick degree 1 (Algorithm 1 reaches it with exactly that degree, whenever it does).
 constexpr int kEll = 32;
+constexpr int kChunkBatch = 4;
 
 __global__ void __launch_bounds__(256) extract_kernel(CodebookParams p) {
   const int lane = threadIdx.x & 31;
@@ -258,18 +259,18 @@ __global__ void __launch_bounds__(256) extract_kernel(CodebookParams p) {
     uint32_t occ = tr.apply(fw[i]);
     if (!exists) occ = 0;
     while (occ) {
-      // up to four occupied chunks at a time, loaded before any of them is looked at
-      int cs[4];
-      uint2 av[4];
+      // several occupied chunks at a time, loaded before any of them is looked at
+      int cs[kChunkBatch];
+      uint2 av[kChunkBatch];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
+      for (int i = 0; i < kChunkBatch; ++i) {
         cs[i] = occ ? c0 + __ffs(occ) - 1 : -1;
         occ &= occ - 1;   // 0 stays 0
       }
 #pragma unroll
-      for (int i = 0; i < 4; ++i) av[i] = cs[i] >= 0 ? row2[cs[i]] : make_uint2(0, 0);
+      for (int i = 0; i < kChunkBatch; ++i) av[i] = cs[i] >= 0 ? row2[cs[i]] : make_uint2(0, 0);
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
+      for (int i = 0; i < kChunkBatch; ++i) {
         if (cs[i] < 0) continue;
         const uint32_t wd[2] = {av[i].x, av[i].y};
 #pragma unroll
