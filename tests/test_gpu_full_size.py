@@ -114,3 +114,86 @@ def test_headline_configuration_full_size():
         assert np.array_equal(C1[:n1], o["C"][li, 0, j, :n1].float().cpu().numpy())
         flips += check_codebook_unit(gamma.float().cpu().numpy(), theta, adj, mag1, ref1, cen1, n1, C1, value_tol(wl))
     print(f"full size: {margin} kept positions and {flips} adjacency bits decided inside the 1e-4 margin")
+
+
+def _check_workload(wl, sampled_codebooks, sampled_evictions):
+    """Runs ``wl`` as ``bench.py`` would (one call per kind of layer), checks properties on every unit and the
+    sampled units against the checker.  ``sampled_codebooks``: (Gamma, layer, sequence, head);
+    ``sampled_evictions``: (evicting layer index, sequence)."""
+    from paper_2507_06517_b200.pipeline import SpindleKVPass
+    from gpu_util import tok_base, unit_rows
+    ns, nd, H, w, d = wl.n_shallow, wl.n_layers - wl.n_shallow, wl.n_kv_heads, wl.window, wl.head_dim
+    K, V, Q = _device_layers(wl)
+    p = SpindleKVPass(make_config(wl), wl.seq_lens, torch_dtype(wl))
+    p.run(K, V, Q)
+    st = p.device_status()
+    assert st["evict"][0] == 0 and st["codebook"][0] == 0 and st["codebook"][1][1] == 0
+    _, _, k_plan = O.plan_layers(wl.n_layers, ns, wl.seq_lens, w, wl.beta, reserve_ratio=wl.budget_frac,
+                                 budget_tokens=wl.budget_tokens)
+    assert np.array_equal(k_plan, p.k_ctx_host)
+    Kh, Vh = K.float().cpu().numpy(), V.float().cpu().numpy()
+    keep, cnt, scores = p.keep_idx.cpu().numpy(), p.keep_cnt.cpu().numpy(), p.scores.cpu().numpy()
+    Kk, Vk = p.K_kept.float().cpu().numpy(), p.V_kept.float().cpu().numpy()
+    for li in range(nd):
+        for s, l in enumerate(wl.seq_lens):
+            k, tb = int(k_plan[ns + li, s]), tok_base(wl, s)
+            assert np.all(cnt[li, s] == k + w)
+            rows = keep[li, :, tb:tb + k + w]
+            assert np.all(np.diff(rows, axis=1) > 0) and np.all(rows[:, k:] == np.arange(l - w, l))
+            for j in range(H):
+                for src, dst in ((Kh, Kk), (Vh, Vk)):
+                    assert np.array_equal(unit_rows(wl, dst[li], s, j)[: k + w], unit_rows(wl, src[ns + li], s, j)[rows[j]])
+    margin = 0
+    Qh = Q.float().cpu().numpy()
+    for li, s in sampled_evictions:
+        l, tb = wl.seq_lens[s], tok_base(wl, s)
+        Ks = np.stack([unit_rows(wl, Kh[ns + li], s, j) for j in range(H)])
+        margin += check_evict_unit(wl, Qh[li, s], Ks, int(k_plan[ns + li, s]), scores[li, :, tb:tb + l],
+                                   keep[li, :, tb:tb + l], cnt[li, s])
+    for g, Gh in (("K", Kh), ("V", Vh)):
+        o = p.cb[g]
+        n_ent, ref, cen, mag = (o[x].cpu().numpy() for x in ("n_entries", "ref", "centre_idx", "mag"))
+        Cn = o["C"].float().cpu().numpy()
+        for li in range(ns):
+            for s, l in enumerate(wl.seq_lens):
+                tb = tok_base(wl, s)
+                for j in range(H):
+                    n = int(n_ent[li, s, j])
+                    r, c = ref[li, j, tb:tb + l], cen[li, j, tb:tb + n]
+                    assert 1 <= n <= l and r.min() >= 0 and r.max() == n - 1
+                    assert np.array_equal(r[c], np.arange(n)) and len(np.unique(c)) == n
+                    rows = unit_rows(wl, Gh[li], s, j).astype(np.float64)
+                    np.testing.assert_allclose(mag[li, j, tb:tb + l], np.sqrt((rows * rows).sum(1)), rtol=2e-6)
+                    assert np.all(np.abs(np.linalg.norm(unit_rows(wl, Cn[li], s, j)[:n], axis=1) - 1) < 1e-2)
+    flips = 0
+    for g, li, s, j in sampled_codebooks:
+        src, theta = (K, wl.theta_k) if g == "K" else (V, wl.theta_v)
+        l, tb = wl.seq_lens[s], tok_base(wl, s)
+        gamma = (src[li, tb:tb + l, j] if wl.packed else src[li, s, j]).contiguous()
+        adj, mag1, ref1, cen1, n1, C1 = _single_unit_codebook(wl, gamma, theta)
+        o = p.cb[g]
+        assert n1 == int(o["n_entries"][li, s, j])
+        assert np.array_equal(ref1[:l], o["ref"][li, j, tb:tb + l].cpu().numpy())
+        assert np.array_equal(cen1[:n1], o["centre_idx"][li, j, tb:tb + n1].cpu().numpy())
+        flips += check_codebook_unit(gamma.float().cpu().numpy(), theta, adj, mag1, ref1, cen1, n1, C1, value_tol(wl))
+    print(f"{wl.name}: {margin} kept positions and {flips} adjacency bits decided inside the 1e-4 margin")
+
+
+def test_8b_shape_at_4k_full():
+    _check_workload(synth.workload("C2"), [("K", 0, 0, 0), ("V", 7, 0, 3), ("K", 15, 0, 7), ("V", 15, 0, 6)],
+                    [(0, 0), (8, 0), (15, 0)])
+
+
+def test_packed_variable_length_batch():
+    # the packed batch of eight sequences, cut to four layers (two CodeBook, two evicting)
+    wl = synth.workload("C4")
+    wl = wl.replace(n_layers=4, n_shallow=2, name="C4[4 layers]")
+    short, long = int(np.argmin(wl.seq_lens)), int(np.argmax(wl.seq_lens))
+    _check_workload(wl, [("K", 0, short, 1), ("V", 1, long, 6)], [(0, short), (1, long)])
+
+
+def test_70b_shape_at_32k():
+    # 64 query heads on 8 KV heads (256 query rows per KV head), N = 32768, cut to two layers
+    wl = synth.workload("C5")
+    wl = wl.replace(n_layers=2, n_shallow=1, name="C5[2 layers]")
+    _check_workload(wl, [("V", 0, 0, 2)], [(0, 0)])
