@@ -768,6 +768,8 @@ spindlekv_status codebook_shallow_impl(const spindlekv_config& cfg, const spindl
     if (bf) launch_norms<__nv_bfloat16, 128>(p, st); else launch_norms<float, 128>(p, st);
   }
   if (tc) {
+    // the similarity kernel writes only the flag words that hold a set bit
+    if (cudaMemsetAsync(p.flags, 0, (size_t)units * (p.row_words / 2) * p.row_words * 4, st) != cudaSuccess) return SPINDLEKV_CUDA;
     spindlekv_status rs = launch_sim_tc(Gamma, b, cfg.n_kv_heads, cfg.head_dim, p.ext, p.adj, p.flags, p.hdr, st);
     if (rs != SPINDLEKV_OK) return rs;
   } else if (cfg.head_dim == 64) {

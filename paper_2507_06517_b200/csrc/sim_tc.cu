@@ -30,7 +30,8 @@
 // a set bit (0: certainly empty), so that the next kernel reads only the occupied part of a sparse
 // graph.  The flags of 32 consecutive rows and one chunk form a word (`flags[row / 32][chunk]`) with
 // exactly one writer: the rows' own block for chunks at or right of the block's own columns, the
-// block that mirrors into the rows for chunks left of them.
+// block that mirrors into the rows for chunks left of them.  The caller clears the flag words; only
+// words with a set bit are written.
 #include "common.cuh"
 #include "sm100_ptx.cuh"
 
@@ -321,7 +322,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kSimThreads, 1) sim_
           const uint32_t f0 = __ballot_sync(0xffffffffu, (words[0] | words[1]) != 0u);
           const uint32_t f1 = __ballot_sync(0xffffffffu, (words[2] | words[3]) != 0u);
           const int chunk = tile * 4 + cg * 2 + lane;
-          if (lane < 2 && chunk < NC) funit[(int64_t)(R >> 5) * NC + chunk] = lane ? f1 : f0;
+          const uint32_t fw = lane ? f1 : f0;   // the flag words start at zero: only occupied ones are written
+          if (lane < 2 && chunk < NC && fw) funit[(int64_t)(R >> 5) * NC + chunk] = fw;
         }
         if (fast) {
           *reinterpret_cast<uint2*>(sdw) = make_uint2(words[0], words[1]);
@@ -361,7 +363,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kSimThreads, 1) sim_
           occ_hi = (mv.z | mv.w) != 0u;
         }
         const uint32_t flo = __ballot_sync(0xffffffffu, occ_lo), fhi = __ballot_sync(0xffffffffu, occ_hi);
-        if (lane < 2 && (b >> 5) < RW) funit[(int64_t)(b >> 5) * NC + 2 * blk + lane] = lane ? fhi : flo;
+        const uint32_t fw = lane ? fhi : flo;
+        if (lane < 2 && (b >> 5) < RW && fw) funit[(int64_t)(b >> 5) * NC + 2 * blk + lane] = fw;
       }
       if (slot == 1 || tile + 2 >= n_tiles) {
         // the two warps of the team that share this 32-row strip have staged their direct words of the
