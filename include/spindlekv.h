@@ -92,6 +92,9 @@ typedef struct {
                                   has layer_lens[layer*B + s] <= max_len tokens in layer `layer` of the call, rows
                                   still max_len apart.  This is how the CodeBook call takes the tokens that
                                   eviction kept, whose number differs from layer to layer (Eq. (5)(6)). */
+  int32_t layer_lens_heads;    /* 0: layer_lens is indexed [layer][seq].  H > 0: it is indexed [layer][seq][head]
+                                  with H heads per sequence (lengths that differ from head to head, e.g. the new
+                                  tokens that found no CodeBook entry); a length may be 0. */
 } spindlekv_batch;
 
 /*
@@ -207,6 +210,44 @@ spindlekv_status spindlekv_compact(const spindlekv_batch* batch, int32_t n_heads
 spindlekv_status spindlekv_union_lists(int32_t n_layers, int32_t n_seqs, int32_t n_heads, int32_t n_lists,
                                        int32_t t_in, int32_t seq_in, const int32_t* idx_in, const int32_t* cnt_in,
                                        int32_t t_out, int32_t seq_out, int32_t* idx_out, int32_t* cnt_out, void* stream);
+
+/*
+ * Decode-time merging of new tokens into existing CodeBooks (Section 3.4, last paragraph: new entries of the
+ * cache first look for a suitable CodeBook entry, with theta as the threshold; those that find one are
+ * merged into it, for the others the CodeBook construction is repeated).  Three steps:
+ *
+ * spindlekv_codebook_match: for every new token the entry with the largest cosine similarity, if that
+ * exceeds theta (strictly; ties to the lower entry number), else -1; and the ascending list of the tokens
+ * without an entry.
+ *   batch      describes the NEW tokens: sequence s of every (layer, head) has max_len of them, or
+ *              layer_lens of them; equal-length form only (no cu_seqlens)
+ *   Gamma_new  device, [layer][seq][head][new token][d]
+ *   C          device, CodeBook rows [layer][seq][head][entry][d] (as written by spindlekv_compact with
+ *              divide_by = mag); n_entries device [n_layers][B][n_heads]; c_rows: row capacity per unit
+ *   mag_new    device out [n_layers][n_heads][T] fp32, ref_new device out [n_layers][n_heads][T] int32
+ *   left_idx   device out [n_layers][n_heads][T]: per unit the positions of its unmatched tokens, ascending
+ *   left_cnt   device out [n_layers][B][n_heads]
+ *   ws         device scratch of spindlekv_match_workspace_bytes(batch, n_heads) bytes, 256-byte aligned
+ * Then the caller gathers the unmatched rows (spindlekv_compact with left_idx, left_cnt) and builds their
+ * CodeBook (spindlekv_codebook_shallow with layer_lens = left_cnt, layer_lens_heads = n_heads).
+ *
+ * spindlekv_codebook_append: the entries of that CodeBook become entries n_entries, n_entries + 1, ... of C
+ * (unit vectors of their centre rows), the unmatched tokens' ref_new become n_entries + ref_left, and
+ * n_entries grows by n_left_entries.  Entries beyond c_rows are not written: compare n_entries with c_rows
+ * afterwards.
+ *   Gamma_left     device, the gathered unmatched rows; mag_left, ref_left, centre_left, n_left_entries: the
+ *                  outputs of spindlekv_codebook_shallow on them
+ */
+size_t spindlekv_match_workspace_bytes(const spindlekv_batch* batch, int32_t n_heads);
+spindlekv_status spindlekv_codebook_match(const spindlekv_batch* batch, int32_t n_heads, int32_t head_dim,
+                                          spindlekv_tensor Gamma_new, spindlekv_tensor C, const int32_t* n_entries,
+                                          int32_t c_rows, float theta, float* mag_new, int32_t* ref_new,
+                                          int32_t* left_idx, int32_t* left_cnt, void* ws, size_t ws_bytes, void* stream);
+spindlekv_status spindlekv_codebook_append(const spindlekv_batch* batch, int32_t n_heads, int32_t head_dim,
+                                           spindlekv_tensor Gamma_left, const float* mag_left, const int32_t* ref_left,
+                                           const int32_t* centre_left, const int32_t* n_left_entries,
+                                           const int32_t* left_idx, const int32_t* left_cnt, spindlekv_tensor C,
+                                           int32_t c_rows, int32_t* n_entries, int32_t* ref_new, void* stream);
 
 /*
  * Reconstruction of the replaced cache from a CodeBook (Eq. (14): Gamma_r = C[r] (x) m): for every

@@ -395,3 +395,51 @@ def reserve_ratio_layer(l: int, kept: int, entries_k: Sequence[int], entries_v: 
     r1 = (2.0 * h * kept) / (2.0 * h * l)
     r2 = (float(sum(entries_k)) + float(sum(entries_v))) / (2.0 * h * kept)
     return r1, r2
+
+
+# --------------------------------------------------------------------------
+# Decode-time merging of new tokens into a CodeBook (Section 3.4, last paragraph)
+# --------------------------------------------------------------------------
+
+def match_entries(C: np.ndarray, gamma_new: np.ndarray, theta: float) -> Tuple[np.ndarray, np.ndarray]:
+    """For every new token the existing entry it is merged into, or -1.
+
+    "Suitable" entries are those whose cosine similarity with the token exceeds ``theta`` (strictly).
+    Reading: among several, the most similar one, the lower entry number on ties.  The cosine is taken
+    with the entries as stored (their own norm divides, although it is 1 up to the rounding of the
+    storage type).  Returns ``(ref, S)`` with ``S[t, j]`` the similarities.
+    """
+    C = np.asarray(C, dtype=np.float64)
+    g = normalise(gamma_new, magnitudes(gamma_new))
+    S = g @ normalise(C, magnitudes(C)).T if C.shape[0] else np.zeros((g.shape[0], 0))
+    ref = -np.ones(g.shape[0], dtype=np.int32)
+    for t in range(g.shape[0]):
+        if S.shape[1] and S[t].max() > theta:
+            ref[t] = int(np.argmax(S[t]))      # first maximum: lower entry number on ties
+    return ref, S
+
+
+def codebook_extend(C: np.ndarray, gamma_new: np.ndarray, theta: float,
+                    ref_override: Optional[np.ndarray] = None, G_override: Optional[np.ndarray] = None) -> Dict[str, np.ndarray]:
+    """New tokens are merged into suitable entries; for the remaining ones the CodeBook construction is
+    repeated (Algorithm 1 on the unmatched tokens, in their order) and its entries are appended.
+
+    ``ref_override`` replaces the matching decisions and ``G_override`` the adjacency of the unmatched
+    tokens (tests use both to settle decisions that sit on the threshold).  Returns ``ref`` (entry of
+    every new token in the extended CodeBook), ``mag``, the extended ``C``, the similarities ``S`` and
+    the unmatched positions ``left``.
+    """
+    C = np.asarray(C, dtype=np.float64)
+    gamma_new = np.asarray(gamma_new, dtype=np.float64)
+    ref, S = match_entries(C, gamma_new, theta)
+    if ref_override is not None:
+        ref = np.asarray(ref_override, dtype=np.int32).copy()
+    left = np.flatnonzero(ref < 0)
+    out_ref = ref.copy()
+    C_ext = C
+    sub = None
+    if left.size:
+        sub = codebook_shallow(gamma_new[left], theta, G_override=G_override)
+        out_ref[left] = C.shape[0] + sub["ref"]
+        C_ext = np.concatenate([C, sub["C"]], axis=0)
+    return {"ref": out_ref, "mag": magnitudes(gamma_new), "C": C_ext, "S": S, "left": left, "sub": sub}

@@ -42,7 +42,7 @@ class _Config(C.Structure):
 
 class _Batch(C.Structure):
     _fields_ = [("n_layers", C.c_int32), ("n_seqs", C.c_int32), ("max_len", C.c_int32),
-                ("total_len", C.c_int32), ("cu_seqlens", C.c_void_p), ("layer_lens", C.c_void_p)]
+                ("total_len", C.c_int32), ("cu_seqlens", C.c_void_p), ("layer_lens", C.c_void_p), ("layer_lens_heads", C.c_int32)]
 
 
 def _load() -> C.CDLL:
@@ -72,6 +72,15 @@ def _load() -> C.CDLL:
     lib.spindlekv_union_lists.restype = C.c_int32
     lib.spindlekv_union_lists.argtypes = [C.c_int32] * 6 + [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_void_p,
                                                             C.c_void_p, C.c_void_p]
+    lib.spindlekv_match_workspace_bytes.restype = C.c_size_t
+    lib.spindlekv_match_workspace_bytes.argtypes = [C.POINTER(_Batch), C.c_int32]
+    lib.spindlekv_codebook_match.restype = C.c_int32
+    lib.spindlekv_codebook_match.argtypes = [C.POINTER(_Batch), C.c_int32, C.c_int32, _Tensor, _Tensor, C.c_void_p, C.c_int32,
+                                             C.c_float, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                             C.c_size_t, C.c_void_p]
+    lib.spindlekv_codebook_append.restype = C.c_int32
+    lib.spindlekv_codebook_append.argtypes = [C.POINTER(_Batch), C.c_int32, C.c_int32, _Tensor] + [C.c_void_p] * 6 + \
+                                             [_Tensor, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
     lib.spindlekv_reconstruct.restype = C.c_int32
     lib.spindlekv_reconstruct.argtypes = [C.POINTER(_Batch), C.c_int32, C.c_int32, _Tensor, C.c_void_p, C.c_void_p,
                                           _Tensor, C.c_void_p]
@@ -117,12 +126,13 @@ class Batch:
     max_len: int
     total_len: int
     cu_seqlens: Optional[torch.Tensor] = None  # device int32 [B+1]
-    layer_lens: Optional[torch.Tensor] = None  # device int32 [n_layers, B]: per-layer lengths (not with cu_seqlens)
+    layer_lens: Optional[torch.Tensor] = None  # device int32 [n_layers, B] or [n_layers, B, H] (not with cu_seqlens)
 
     def c(self) -> _Batch:
         ptr = self.cu_seqlens.data_ptr() if self.cu_seqlens is not None else None
         ll = self.layer_lens.data_ptr() if self.layer_lens is not None else None
-        return _Batch(self.n_layers, self.n_seqs, self.max_len, self.total_len, ptr, ll)
+        heads = self.layer_lens.shape[2] if self.layer_lens is not None and self.layer_lens.dim() == 3 else 0
+        return _Batch(self.n_layers, self.n_seqs, self.max_len, self.total_len, ptr, ll, heads)
 
 
 def _dtype_code(t: torch.Tensor) -> int:
@@ -229,6 +239,32 @@ def spindlekv_union_lists(n_layers: int, n_seqs: int, n_heads: int, idx_in: torc
     st = _lib.spindlekv_union_lists(n_layers, n_seqs, n_heads, idx_in.shape[0], idx_in.shape[-1], seq_in, _ptr(idx_in),
                                     _ptr(cnt_in), idx_out.shape[-1], seq_out, _ptr(idx_out), _ptr(cnt_out), _stream(stream))
     _check(st, "spindlekv_union_lists")
+
+
+def spindlekv_match_workspace_bytes(batch: Batch, n_heads: int) -> int:
+    bb = batch.c()
+    return int(_lib.spindlekv_match_workspace_bytes(C.byref(bb), n_heads))
+
+
+def spindlekv_codebook_match(batch: Batch, n_heads: int, head_dim: int, G_new: _Tensor, Cb: _Tensor, n_entries: torch.Tensor,
+                             c_rows: int, theta: float, mag_new: torch.Tensor, ref_new: torch.Tensor,
+                             left_idx: torch.Tensor, left_cnt: torch.Tensor, ws: torch.Tensor, stream=None) -> None:
+    bb = batch.c()
+    st = _lib.spindlekv_codebook_match(C.byref(bb), n_heads, head_dim, G_new, Cb, _ptr(n_entries), c_rows, theta,
+                                       _ptr(mag_new), _ptr(ref_new), _ptr(left_idx), _ptr(left_cnt), _ptr(ws),
+                                       ws.numel() * ws.element_size(), _stream(stream))
+    _check(st, "spindlekv_codebook_match")
+
+
+def spindlekv_codebook_append(batch: Batch, n_heads: int, head_dim: int, G_left: _Tensor, mag_left: torch.Tensor,
+                              ref_left: torch.Tensor, centre_left: torch.Tensor, n_left_entries: torch.Tensor,
+                              left_idx: torch.Tensor, left_cnt: torch.Tensor, Cb: _Tensor, c_rows: int,
+                              n_entries: torch.Tensor, ref_new: torch.Tensor, stream=None) -> None:
+    bb = batch.c()
+    st = _lib.spindlekv_codebook_append(C.byref(bb), n_heads, head_dim, G_left, _ptr(mag_left), _ptr(ref_left),
+                                        _ptr(centre_left), _ptr(n_left_entries), _ptr(left_idx), _ptr(left_cnt), Cb,
+                                        c_rows, _ptr(n_entries), _ptr(ref_new), _stream(stream))
+    _check(st, "spindlekv_codebook_append")
 
 
 def spindlekv_reconstruct(batch: Batch, n_heads: int, head_dim: int, Cb: _Tensor, ref: torch.Tensor,

@@ -29,6 +29,15 @@ spindlekv_status union_lists_impl(int n_layers, int n_seqs, int n_heads, int n_l
                                   const int32_t* idx_in, const int32_t* cnt_in, int t_out, int seq_out,
                                   int32_t* idx_out, int32_t* cnt_out, cudaStream_t st);
 
+size_t match_workspace_bytes(const spindlekv_batch& b, int n_heads);
+spindlekv_status match_impl(const spindlekv_batch& b, int n_heads, int head_dim, const spindlekv_tensor& G,
+                            const spindlekv_tensor& C, const int32_t* n_entries, int c_rows, float theta, float* mag,
+                            int32_t* ref, int32_t* left_idx, int32_t* left_cnt, void* ws, size_t ws_bytes, cudaStream_t st);
+spindlekv_status append_impl(const spindlekv_batch& b, int n_heads, int head_dim, const spindlekv_tensor& Lt,
+                             const float* mag_left, const int32_t* ref_left, const int32_t* centre_left,
+                             const int32_t* n_left_entries, const int32_t* left_idx, const int32_t* left_cnt,
+                             const spindlekv_tensor& C, int c_rows, int32_t* n_entries, int32_t* ref_new, cudaStream_t st);
+
 // ---- launch counting and timing ---------------------------------------------------------------
 static std::mutex g_mu;
 static int64_t g_launches = 0;
@@ -199,6 +208,46 @@ spindlekv_status spindlekv_union_lists(int32_t n_layers, int32_t n_seqs, int32_t
   if ((int64_t)n_layers * n_seqs * n_heads > 0x7FFFFFFF) return SPINDLEKV_UNSUPPORTED;
   return union_lists_impl(n_layers, n_seqs, n_heads, n_lists, t_in, seq_in, idx_in, cnt_in, t_out, seq_out, idx_out,
                           cnt_out, (cudaStream_t)stream);
+}
+
+static bool new_batch_ok(const spindlekv_batch* b) {
+  if (!b || b->n_layers <= 0 || b->n_seqs <= 0 || b->max_len <= 0 || b->cu_seqlens) return false;
+  return (int64_t)b->total_len == (int64_t)b->n_seqs * b->max_len;
+}
+
+size_t spindlekv_match_workspace_bytes(const spindlekv_batch* batch, int32_t n_heads) {
+  if (!new_batch_ok(batch) || n_heads <= 0) return 0;
+  return match_workspace_bytes(*batch, n_heads);
+}
+
+spindlekv_status spindlekv_codebook_match(const spindlekv_batch* batch, int32_t n_heads, int32_t head_dim,
+                                          spindlekv_tensor Gamma_new, spindlekv_tensor C, const int32_t* n_entries,
+                                          int32_t c_rows, float theta, float* mag_new, int32_t* ref_new,
+                                          int32_t* left_idx, int32_t* left_cnt, void* ws, size_t ws_bytes, void* stream) {
+  if (!new_batch_ok(batch) || n_heads <= 0 || c_rows <= 0) return SPINDLEKV_INVALID_ARG;
+  if (!tensor_ok(Gamma_new) || !tensor_ok(C) || !n_entries || !mag_new || !ref_new || !left_idx || !left_cnt || !ws)
+    return SPINDLEKV_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(ws) % 256) return SPINDLEKV_INVALID_ARG;
+  if (Gamma_new.dtype != C.dtype) return SPINDLEKV_UNSUPPORTED;
+  if (head_dim != 64 && head_dim != 128) return SPINDLEKV_UNSUPPORTED;
+  return match_impl(*batch, n_heads, head_dim, Gamma_new, C, n_entries, c_rows, theta, mag_new, ref_new, left_idx,
+                    left_cnt, ws, ws_bytes, (cudaStream_t)stream);
+}
+
+spindlekv_status spindlekv_codebook_append(const spindlekv_batch* batch, int32_t n_heads, int32_t head_dim,
+                                           spindlekv_tensor Gamma_left, const float* mag_left, const int32_t* ref_left,
+                                           const int32_t* centre_left, const int32_t* n_left_entries,
+                                           const int32_t* left_idx, const int32_t* left_cnt, spindlekv_tensor C,
+                                           int32_t c_rows, int32_t* n_entries, int32_t* ref_new, void* stream) {
+  if (!new_batch_ok(batch) || n_heads <= 0 || c_rows <= 0) return SPINDLEKV_INVALID_ARG;
+  if (!tensor_ok(Gamma_left) || !tensor_ok(C) || !mag_left || !ref_left || !centre_left || !n_left_entries || !left_idx ||
+      !left_cnt || !n_entries || !ref_new)
+    return SPINDLEKV_INVALID_ARG;
+  if (Gamma_left.dtype != C.dtype) return SPINDLEKV_UNSUPPORTED;
+  if (head_dim != 64 && head_dim != 128) return SPINDLEKV_UNSUPPORTED;
+  if ((int64_t)batch->n_layers * batch->n_seqs * n_heads > 0x7FFFFFFF) return SPINDLEKV_UNSUPPORTED;
+  return append_impl(*batch, n_heads, head_dim, Gamma_left, mag_left, ref_left, centre_left, n_left_entries, left_idx,
+                     left_cnt, C, c_rows, n_entries, ref_new, (cudaStream_t)stream);
 }
 
 spindlekv_status spindlekv_reconstruct(const spindlekv_batch* batch, int32_t n_heads, int32_t head_dim,

@@ -73,7 +73,7 @@ __global__ void __launch_bounds__(256) norms_kernel(CodebookParams p) {
   __shared__ float sm_m[ROWS];
   int layer, s, j;
   cb_decode(p, blockIdx.y, layer, s, j);
-  const int l = seq_len(p.batch, layer, s);
+  const int l = seq_len(p.batch, layer, s, j);
   const int seg = threadIdx.x % LPR;
   const int block_row0 = blockIdx.x * ROWS;
   const int local_first = threadIdx.x / LPR;
@@ -131,7 +131,7 @@ __global__ void __launch_bounds__(256) sim_simt_kernel(CodebookParams p) {
   __shared__ TileSmem sm;
   int layer, s, j;
   cb_decode(p, blockIdx.z, layer, s, j);
-  const int l = seq_len(p.batch, layer, s);
+  const int l = seq_len(p.batch, layer, s, j);
   const int r0 = blockIdx.y * kTile, c0 = blockIdx.x * kTile;
   if (r0 >= l || c0 >= row_words_for(p.batch.max_len) * 32) return;
   const T* base = reinterpret_cast<const T*>(p.G.ptr) + unit_offset(p.G, p.batch, layer, s, j);
@@ -231,7 +231,7 @@ __global__ void __launch_bounds__(256) extract_kernel(CodebookParams p) {
   const int unit = (int)(g / NP), u = (int)(g - (int64_t)unit * NP);
   int layer, s, j;
   cb_decode(p, unit, layer, s, j);
-  const int l = seq_len(p.batch, layer, s);
+  const int l = seq_len(p.batch, layer, s, j);
   const bool exists = u < l;
   const int64_t idx = (int64_t)unit * ML + (exists ? u : 0);
   const int64_t n_rows = (int64_t)p.n_units * ML;
@@ -589,7 +589,7 @@ __global__ void __launch_bounds__(kFinalThreads) finalize_kernel(CodebookParams 
   const int unit = blockIdx.x;
   int layer, s, j;
   cb_decode(p, unit, layer, s, j);
-  const int l = seq_len(p.batch, layer, s);
+  const int l = seq_len(p.batch, layer, s, j);
   const int ML = p.batch.max_len;
   const int32_t* pickdeg = p.pickdeg + (int64_t)unit * ML;
   const int32_t* owner = p.owner + (int64_t)unit * ML;

@@ -34,16 +34,20 @@ inline View make_view(const spindlekv_tensor& t) { return View{t.ptr, t.stride_l
 struct Batch {  // device-side copy of spindlekv_batch
   int n_layers, n_seqs, max_len, total_len;
   const int32_t* cu;
-  const int32_t* ll;   // per-layer lengths [n_layers][n_seqs], or null
+  const int32_t* ll;   // lengths per layer [n_layers][n_seqs], or per unit [n_layers][n_seqs][ll_heads], or null
+  int ll_heads;        // 0: `ll` is per layer and sequence; otherwise the number of heads it is indexed by
 };
 
 inline Batch make_batch(const spindlekv_batch& b) {
-  return Batch{b.n_layers, b.n_seqs, b.max_len, b.total_len, b.cu_seqlens, b.layer_lens};
+  return Batch{b.n_layers, b.n_seqs, b.max_len, b.total_len, b.cu_seqlens, b.layer_lens, b.layer_lens_heads};
 }
 
-// tokens of sequence s in layer `layer` of the call
-__device__ __forceinline__ int seq_len(const Batch& b, int layer, int s) {
-  if (b.ll) return min(b.ll[layer * b.n_seqs + s], b.max_len);
+// tokens of sequence s (head `head`) in layer `layer` of the call
+__device__ __forceinline__ int seq_len(const Batch& b, int layer, int s, int head) {
+  if (b.ll) {
+    const int i = layer * b.n_seqs + s;
+    return max(0, min(b.ll[b.ll_heads ? i * b.ll_heads + head : i], b.max_len));
+  }
   return b.cu ? (b.cu[s + 1] - b.cu[s]) : b.max_len;
 }
 __device__ __forceinline__ int tok_base(const Batch& b, int s) { return b.cu ? b.cu[s] : s * b.max_len; }
@@ -107,6 +111,35 @@ struct TransposeLane {
     return x;
   }
 };
+
+// exclusive prefix sum of one int per thread over the block; returns the block total through `total`
+__device__ __forceinline__ int block_exclusive_scan(int v, int* warp_sums, int& total) {
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  int inc = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    int n = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += n;
+  }
+  if (lane == 31) warp_sums[wid] = inc;
+  __syncthreads();
+  if (wid == 0) {
+    int ws = warp_sums[lane];
+    int winc = ws;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      int n = __shfl_up_sync(0xffffffffu, winc, o);
+      if (lane >= o) winc += n;
+    }
+    warp_sums[lane] = winc - ws;
+    if (lane == 31) warp_sums[32] = winc;
+  }
+  __syncthreads();
+  int res = warp_sums[wid] + inc - v;
+  total = warp_sums[32];
+  __syncthreads();
+  return res;
+}
 
 // ---- launch bookkeeping (host) ---------------------------------------------------------------
 void note_launch(int kclass, cudaStream_t st, bool before);

@@ -79,7 +79,7 @@ __global__ void __launch_bounds__(256) reconstruct_kernel(ReconstructParams p) {
   const int ls = unit / p.n_heads;
   const int s = ls % p.batch.n_seqs;
   const int layer = ls / p.batch.n_seqs;
-  const int l = seq_len(p.batch, layer, s);
+  const int l = seq_len(p.batch, layer, s, h);
   const int64_t orow = ((int64_t)layer * p.n_heads + h) * p.batch.total_len + tok_base(p.batch, s);
   const T* cbase = reinterpret_cast<const T*>(p.C.ptr) + unit_offset(p.C, p.batch, layer, s, h);
   T* dbase = reinterpret_cast<T*>(const_cast<void*>(p.dst.ptr)) + unit_offset(p.dst, p.batch, layer, s, h);

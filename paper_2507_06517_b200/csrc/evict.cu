@@ -63,7 +63,7 @@ __global__ void __launch_bounds__(256) win_stats_kernel(EvictParams p) {
   __shared__ TileSmem sm;
   int layer, s, j;
   decode_unit(p, blockIdx.y, layer, s, j);
-  const int l = seq_len(p.batch, layer, s);
+  const int l = seq_len(p.batch, layer, s, j);
   const int key0 = blockIdx.x * kTile;
   if (key0 >= l) return;
   const int l_c = l - p.window;
@@ -106,7 +106,7 @@ __global__ void win_combine_kernel(EvictParams p, int n_units) {
   int unit = gw / M;
   int layer, s, j;
   decode_unit(p, unit, layer, s, j);
-  int nt = (seq_len(p.batch, layer, s) + kTile - 1) / kTile;
+  int nt = (seq_len(p.batch, layer, s, j) + kTile - 1) / kTile;
   const float2* src = p.part + (int64_t)gw * p.n_tiles;
   float mx = -CUDART_INF_F;
   for (int t = lane; t < nt; t += 32) mx = fmaxf(mx, src[t].x);
@@ -128,7 +128,7 @@ __global__ void __launch_bounds__(256) win_colsum_kernel(EvictParams p) {
   __shared__ float colred[16][kTile];
   int layer, s, j;
   decode_unit(p, blockIdx.y, layer, s, j);
-  const int l = seq_len(p.batch, layer, s);
+  const int l = seq_len(p.batch, layer, s, j);
   const int l_c = l - p.window;
   const int key0 = blockIdx.x * kTile;
   if (key0 >= l_c) return;  // only context columns are scored
@@ -187,35 +187,6 @@ __device__ __forceinline__ uint32_t order_key(float f) {
 
 constexpr int kTopkThreads = 1024;
 
-// exclusive prefix sum of one int per thread over the block; returns the block total through `total`
-__device__ __forceinline__ int block_exclusive_scan(int v, int* warp_sums, int& total) {
-  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-  int inc = v;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    int n = __shfl_up_sync(0xffffffffu, inc, o);
-    if (lane >= o) inc += n;
-  }
-  if (lane == 31) warp_sums[wid] = inc;
-  __syncthreads();
-  if (wid == 0) {
-    int ws = warp_sums[lane];
-    int winc = ws;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      int n = __shfl_up_sync(0xffffffffu, winc, o);
-      if (lane >= o) winc += n;
-    }
-    warp_sums[lane] = winc - ws;
-    if (lane == 31) warp_sums[32] = winc;
-  }
-  __syncthreads();
-  int res = warp_sums[wid] + inc - v;
-  total = warp_sums[32];
-  __syncthreads();
-  return res;
-}
-
 __global__ void __launch_bounds__(kTopkThreads) topk_kernel(TopkParams p) {
   __shared__ int hist[256];
   __shared__ int warp_sums[33];
@@ -226,7 +197,7 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(TopkParams p) {
   const int ls = unit / p.n_kv_heads;
   const int s = ls % p.batch.n_seqs;
   const int layer = ls / p.batch.n_seqs;
-  const int l = seq_len(p.batch, layer, s);
+  const int l = seq_len(p.batch, layer, s, j);
   const int l_c = l - p.window;
   int k = p.k_ctx[layer * p.batch.n_seqs + s];
   k = max(0, min(k, l_c));

@@ -159,7 +159,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kSimThreads, 1) sim_
   const int ls = unit / p.n_kv_heads;
   const int s = ls % p.batch.n_seqs;
   const int layer = ls / p.batch.n_seqs;
-  const int l = seq_len(p.batch, layer, s);
+  const int l = seq_len(p.batch, layer, s, j);
   const int row0 = blockIdx.x * kBM;
   const int rank = (int)cluster_ctarank();   // = blockIdx.x & 1
   if ((row0 & ~(kBN - 1)) >= l) return;      // both CTAs of a pair: the whole 256-row span lies beyond the sequence

@@ -82,7 +82,7 @@ __global__ void __launch_bounds__(kWinThreads, 1) win_tc_kernel(const __grid_con
   const int ls = unit / p.n_kv_heads;
   const int s = ls % p.batch.n_seqs;
   const int layer = ls / p.batch.n_seqs;
-  const int l = seq_len(p.batch, layer, s);
+  const int l = seq_len(p.batch, layer, s, j);
   const int l_c = l - p.window;
   const int T = (l + kWinTile - 1) / kWinTile;      // tiles of pass A (all keys)
   const int Tc = (l_c + kWinTile - 1) / kWinTile;   // tiles of pass B (context keys)

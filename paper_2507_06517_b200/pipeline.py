@@ -368,3 +368,42 @@ class SpindleKVRepeatPass:
     def device_status(self):
         torch.cuda.synchronize(self.device)
         return {"evict": B.spindlekv_poll_status(self.ws_evict), "codebook": B.spindlekv_poll_status(self.ws_codebook)}
+
+
+class SpindleKVDecodeMerge:
+    """Decode-time merging (Section 3.4, last paragraph) of ``t_new`` new tokens per (layer, sequence, head)
+    into existing CodeBooks: match against the entries, build a CodeBook of the unmatched tokens, append
+    it.  ``C``: ``[L, B, H, c_rows, d]`` with ``n_entries [L, B, H]`` (both updated in place); new tokens
+    ``[L, B, H, t_new, d]``.  Results: ``ref_new``, ``mag_new`` ``[L, H, B * t_new]``.  Call order only.
+    """
+
+    def __init__(self, cfg: B.Config, n_layers: int, n_seqs: int, t_new: int, c_rows: int, dtype: torch.dtype,
+                 device="cuda", keep_adjacency: bool = False):
+        self.cfg, self.L, self.nB, self.t_new, self.c_rows = cfg, n_layers, n_seqs, t_new, c_rows
+        self.device = dev = torch.device(device)
+        H, d, T = cfg.n_kv_heads, cfg.head_dim, n_seqs * t_new
+        i32 = dict(dtype=torch.int32, device=dev)
+        self.batch = B.Batch(n_layers, n_seqs, t_new, T)
+        self.ws_match = torch.empty(B.spindlekv_match_workspace_bytes(self.batch, H), dtype=torch.uint8, device=dev)
+        self.ref_new = torch.zeros((n_layers, H, T), **i32)
+        self.mag_new = torch.zeros((n_layers, H, T), dtype=torch.float32, device=dev)
+        self.left_idx = torch.zeros((n_layers, H, T), **i32)
+        self.left_cnt = torch.zeros((n_layers, n_seqs, H), **i32)
+        self.left_rows = torch.zeros((n_layers, n_seqs, H, t_new, d), dtype=dtype, device=dev)
+        self.left_batch = B.Batch(n_layers, n_seqs, t_new, T, None, self.left_cnt)   # lengths per head, on the device
+        self.ws_codebook = torch.empty(B.spindlekv_workspace_bytes(cfg, self.left_batch, B.WS_CODEBOOK), dtype=torch.uint8, device=dev)
+        self.left = {"mag": torch.zeros((n_layers, H, T), dtype=torch.float32, device=dev), "ref": torch.zeros((n_layers, H, T), **i32),
+                     "centre_idx": torch.zeros((n_layers, H, T), **i32), "n_entries": torch.zeros((n_layers, n_seqs, H), **i32)}
+        self.adj = torch.zeros((n_layers * n_seqs * H, t_new, B.row_words(t_new)), **i32) if keep_adjacency else None
+
+    def run(self, G_new: torch.Tensor, C: torch.Tensor, n_entries: torch.Tensor, theta: float, stream=None) -> None:
+        cfg, H, d = self.cfg, self.cfg.n_kv_heads, self.cfg.head_dim
+        gd, cd, ld = B.desc_bhnd(G_new), B.desc_bhnd(C), B.desc_bhnd(self.left_rows)
+        B.spindlekv_codebook_match(self.batch, H, d, gd, cd, n_entries, self.c_rows, theta, self.mag_new, self.ref_new,
+                                   self.left_idx, self.left_cnt, self.ws_match, stream)
+        B.spindlekv_compact(self.batch, H, d, gd, self.left_idx, self.left_cnt, ld, None, None, stream)
+        o = self.left
+        B.spindlekv_codebook_shallow(cfg, self.left_batch, ld, theta, o["mag"], o["ref"], o["centre_idx"], o["n_entries"],
+                                     self.ws_codebook, self.adj, stream)
+        B.spindlekv_codebook_append(self.batch, H, d, ld, o["mag"], o["ref"], o["centre_idx"], o["n_entries"],
+                                    self.left_idx, self.left_cnt, cd, self.c_rows, n_entries, self.ref_new, stream)

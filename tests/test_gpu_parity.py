@@ -13,7 +13,7 @@ import torch
 from oracle import spindlekv_oracle as O
 from paper_2507_06517_b200 import synth
 
-from gpu_util import (check_codebook_unit, check_evict_unit, generate, make_config, stack_layers, tok_base,
+from gpu_util import (REL_MARGIN, check_codebook_unit, check_evict_unit, generate, make_config, stack_layers, tok_base,
                       torch_dtype, unit_rows, value_tol)
 
 pytestmark = pytest.mark.gpu
@@ -262,6 +262,73 @@ def test_gqa_repeat_variant():
                 ref = o["ref"][lam, j, : h_n * n]
                 for tok in np.unique(want_union):
                     assert len(set(ref[want_union == tok])) == 1
+
+
+def test_decode_time_merge_into_existing_codebooks():
+    # CodeBooks of the first tokens of a sequence, then the rest of the sequence arrives as new tokens: some
+    # find an entry, the others get entries of their own, appended
+    from paper_2507_06517_b200 import binding as B
+    from paper_2507_06517_b200.pipeline import SpindleKVDecodeMerge
+    for dtype, d, l0, t_new, tol in (("bf16", 128, 512, 200, 1e-2), ("f32", 64, 300, 90, 1e-5)):
+        wl = synth.Workload("merge", 2, 2, 4, 2, d, dtype, 8, (l0 + t_new,), 24, (0.03, 0.3), 2, "gauss",
+                            budget_tokens=float(l0 + t_new), seed=81)
+        host = generate(wl)
+        full = stack_layers(wl, host, [0, 1], "K")                      # [2, 1, H, l0 + t_new, d]
+        old, new = full[:, :, :, :l0].contiguous(), full[:, :, :, l0:].contiguous()
+        H, theta, c_rows = wl.n_kv_heads, wl.theta_k, l0 + t_new
+        base = synth.Workload("base", 2, 2, 4, 2, d, dtype, 8, (l0,), 24, 0.1, 2, "gauss", budget_tokens=float(l0))
+        p = _pass(base)
+        p.codebook(old, "K")
+        C = torch.zeros((2, 1, H, c_rows, d), dtype=old.dtype, device="cuda")
+        C[:, :, :, :l0] = p.cb["K"]["C"]
+        n_entries = p.cb["K"]["n_entries"].clone()
+        C_before, n_before = C.float().cpu().numpy(), n_entries.cpu().numpy()
+        m = SpindleKVDecodeMerge(make_config(base), 2, 1, t_new, c_rows, old.dtype, keep_adjacency=True)
+        m.run(new, C, n_entries, theta)
+        torch.cuda.synchronize()
+        assert B.spindlekv_poll_status(m.ws_codebook)[0] == 0
+        ref, mag, left_idx, left_cnt = (x.cpu().numpy() for x in (m.ref_new, m.mag_new, m.left_idx, m.left_cnt))
+        C_after, n_after, adj = C.float().cpu().numpy(), n_entries.cpu().numpy(), m.adj.cpu().numpy()
+        sub = {k: v.cpu().numpy() for k, v in m.left.items()}
+        new_h = new.float().cpu().numpy()
+        n_near = n_matched = n_unmatched = 0
+        for li in range(2):
+            for j in range(H):
+                n0 = int(n_before[li, 0, j])
+                gam = new_h[li, 0, j]
+                want_ref, S = O.match_entries(C_before[li, 0, j, :n0], gam, theta)
+                got = ref[li, j]
+                np.testing.assert_allclose(mag[li, j], O.magnitudes(gam), rtol=2e-6)
+                matched = np.array([got[t] if 0 <= got[t] < n0 else -1 for t in range(t_new)])
+                for t in range(t_new):
+                    top = S[t].max()
+                    if matched[t] != want_ref[t]:
+                        n_near += 1   # only on the threshold, or between entries that are equally similar
+                        if matched[t] < 0 or want_ref[t] < 0:
+                            assert abs(top - theta) < REL_MARGIN * theta
+                        else:
+                            assert S[t, matched[t]] > top - REL_MARGIN * abs(top)
+                left = np.flatnonzero(matched < 0)
+                n_matched += t_new - left.size
+                n_unmatched += left.size
+                assert left_cnt[li, 0, j] == left.size and np.array_equal(left_idx[li, j, : left.size], left)
+                # the unmatched tokens' own CodeBook, against the checker on the same rows
+                unit = li * H + j
+                n_add = int(sub["n_entries"][li, 0, j])
+                if left.size:
+                    check_codebook_unit(gam[left], theta, adj[unit], sub["mag"][li, j, : left.size], sub["ref"][li, j, : left.size],
+                                        sub["centre_idx"][li, j, : left.size], n_add, None, tol)
+                    assert np.array_equal(got[left], n0 + sub["ref"][li, j, : left.size])
+                    rows = gam[left][sub["centre_idx"][li, j, :n_add]].astype(np.float64)
+                    np.testing.assert_allclose(C_after[li, 0, j, n0:n0 + n_add], rows / np.linalg.norm(rows, axis=1, keepdims=True),
+                                               rtol=tol, atol=tol)
+                assert n_after[li, 0, j] == n0 + n_add
+                assert np.array_equal(C_after[li, 0, j, :n0], C_before[li, 0, j, :n0])       # old entries untouched
+                # every new token ends up within the threshold of its entry (Eq. (14))
+                ent = C_after[li, 0, j][got].astype(np.float64)
+                cos = (ent * gam).sum(1) / (np.linalg.norm(ent, axis=1) * np.linalg.norm(gam, axis=1))
+                assert np.all(cos > theta - 2 * tol)
+        assert (ref >= 0).all() and n_matched > 0 and n_unmatched > 0   # both branches were exercised
 
 
 def test_reconstruction_from_the_codebook():

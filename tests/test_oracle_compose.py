@@ -92,3 +92,39 @@ def test_repeat_variant_selects_per_query_head_and_collapses_repeats():
     for j in range(H):
         assert np.array_equal(rep["keep"][h_n * j], base["keep"][j])
         assert len(rep["cb_k"][j]["centres"]) == len(base["cb_k"][j]["centres"])
+
+
+def test_decode_time_merge_of_new_tokens():
+    rng = np.random.default_rng(8)
+    d = 24
+    C = rng.standard_normal((5, d))
+    C /= np.linalg.norm(C, axis=1, keepdims=True)
+    far = rng.standard_normal((3, d))
+    far -= (far @ C.T) @ np.linalg.pinv(C.T)            # orthogonal to every entry: cosine 0 with all of them
+    new = np.stack([3.0 * C[2],                          # a copy of entry 2, three times as long
+                    0.5 * (C[0] + 1e-3 * rng.standard_normal(d)),   # entry 0 with a little noise
+                    far[0], 2.0 * far[0],                # two parallel strangers: one new entry for both
+                    far[1],                              # another stranger: its own entry
+                    C[4] + C[3]])                        # 45 degrees from two entries: cos = 0.707.. < theta
+    out = O.codebook_extend(C, new, 0.9)
+    assert list(out["ref"][:2]) == [2, 0] and list(out["left"]) == [2, 3, 4, 5]
+    assert out["ref"][2] == out["ref"][3] and len({out["ref"][2], out["ref"][4], out["ref"][5]}) == 3
+    assert out["C"].shape[0] == 5 + 3 and sorted(out["ref"][2:]) == sorted([5, 5, 6, 7])
+    np.testing.assert_allclose(out["mag"][:2], [3.0, np.linalg.norm(new[1])], rtol=1e-12)
+    # the same answer by brute force: scalar cosines, first maximum
+    for t in range(new.shape[0]):
+        cos = [float(new[t] @ C[j]) / (np.linalg.norm(new[t]) * np.linalg.norm(C[j])) for j in range(5)]
+        best = max(range(5), key=lambda j: (cos[j], -j))
+        assert (out["ref"][t] == best) if cos[best] > 0.9 else (out["ref"][t] >= 5)
+    # every new token's reconstruction points within the threshold of the token (Eq. (14))
+    rec = O.reconstruct(out["C"], out["ref"], out["mag"])
+    cosr = (rec * new).sum(1) / (np.linalg.norm(rec, axis=1) * np.linalg.norm(new, axis=1))
+    assert np.all(cosr > 0.9 - 1e-12)
+    # with the 45-degree threshold lowered, the last token merges: two equally similar entries, lower number wins
+    assert O.codebook_extend(C, new, 0.7)["ref"][5] == 3
+    # nothing is suitable at theta >= 1: the result is the old CodeBook followed by the new tokens' own CodeBook
+    alone = O.codebook_shallow(new, 1.0)
+    ext = O.codebook_extend(C, new, 1.0)
+    assert np.array_equal(ext["ref"], 5 + alone["ref"]) and np.allclose(ext["C"][5:], alone["C"])
+    # an empty CodeBook: plain Algorithm 1
+    assert np.array_equal(O.codebook_extend(np.zeros((0, d)), new, 0.9)["ref"], O.codebook_shallow(new, 0.9)["ref"])
