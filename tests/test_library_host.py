@@ -81,3 +81,38 @@ def test_workspace_bytes_is_zero_on_bad_input_and_monotone():
     assert 0 < a < b and a < c
     # the adjacency bit matrix dominates: N^2/8 bytes per unit
     assert a >= 2 * 1024 * 1024 // 8
+
+
+def test_device_entry_points_reject_bad_arguments_before_touching_the_gpu():
+    # argument checks come first in every entry point, so they can be exercised without a device
+    import ctypes as C
+    from paper_2507_06517_b200 import binding as B
+    lib = B._lib
+    cfg = B.Config(4, 8, 2, 128, 32, 2, budget_tokens=300.0).c()
+    good = B._Tensor(256, B.BF16, 8, 8, 8, 8)          # an aligned, non-null address that is never dereferenced
+    odd = B._Tensor(264, B.BF16, 8, 8, 8, 8)           # not 16-byte aligned
+    f32 = B._Tensor(256, B.F32, 8, 8, 8, 8)
+    batch = B._Batch(1, 1, 1024, 1024, None, None, 0)
+    both = B._Batch(1, 1, 1024, 1024, 256, 256, 0)     # packed and per-layer lengths at once
+    p = C.c_void_p(256)
+    assert lib.spindlekv_evict_deep(C.byref(cfg), C.byref(batch), good, good, None, p, p, p, p, 1 << 20, None) == B.INVALID_ARG
+    assert lib.spindlekv_evict_deep(C.byref(cfg), C.byref(batch), odd, good, p, p, p, p, p, 1 << 20, None) == B.INVALID_ARG
+    assert lib.spindlekv_evict_deep(C.byref(cfg), C.byref(batch), good, f32, p, p, p, p, p, 1 << 20, None) == B.UNSUPPORTED
+    assert lib.spindlekv_evict_deep(C.byref(cfg), C.byref(both), good, good, p, p, p, p, p, 1 << 20, None) == B.INVALID_ARG
+    assert lib.spindlekv_codebook_shallow(C.byref(cfg), C.byref(both), good, 0.98, p, p, p, p, None, p, 1 << 20, None) == B.INVALID_ARG
+    assert lib.spindlekv_codebook_shallow(C.byref(cfg), C.byref(batch), good, 0.98, None, p, p, p, None, p, 1 << 20, None) == B.INVALID_ARG
+    bad_dim = B.Config(4, 8, 2, 96, 32, 2, budget_tokens=300.0).c()
+    assert lib.spindlekv_codebook_shallow(C.byref(bad_dim), C.byref(batch), good, 0.98, p, p, p, p, None, p, 1 << 20, None) == B.UNSUPPORTED
+    assert lib.spindlekv_compact(C.byref(batch), 2, 128, good, None, p, None, good, None, None) == B.INVALID_ARG
+    assert lib.spindlekv_compact(C.byref(batch), 2, 128, good, p, p, None, f32, None, None) == B.UNSUPPORTED
+    assert lib.spindlekv_reconstruct(C.byref(batch), 2, 128, good, None, p, good, None) == B.INVALID_ARG
+    assert lib.spindlekv_reconstruct(C.byref(batch), 2, 96, good, p, p, good, None) == B.UNSUPPORTED
+    assert lib.spindlekv_union_lists(1, 2, 2, 4, 100, 60, p, p, 400, 200, p, p, None) == B.INVALID_ARG   # 2 x 60 > 100
+    assert lib.spindlekv_union_lists(1, 1, 2, 4, 100, 100, None, p, 400, 400, p, p, None) == B.INVALID_ARG
+    assert lib.spindlekv_match_workspace_bytes(C.byref(both), 2) == 0
+    assert lib.spindlekv_match_workspace_bytes(C.byref(batch), 2) >= 8 * 2 * 1024
+    assert lib.spindlekv_codebook_match(C.byref(batch), 2, 128, good, good, p, 0, 0.98, p, p, p, p, p, 1 << 20, None) == B.INVALID_ARG
+    assert lib.spindlekv_codebook_match(C.byref(batch), 2, 128, good, f32, p, 64, 0.98, p, p, p, p, p, 1 << 20, None) == B.UNSUPPORTED
+    assert lib.spindlekv_codebook_append(C.byref(batch), 2, 128, good, p, p, p, p, p, None, good, 64, p, p, None) == B.INVALID_ARG
+    assert lib.spindlekv_evict_deep_noalloc(C.byref(cfg), C.byref(batch), good, good, None, p, p, p, None) == B.INVALID_ARG
+    assert lib.spindlekv_poll_status(None, p, None) == B.INVALID_ARG
