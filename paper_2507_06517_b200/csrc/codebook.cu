@@ -787,15 +787,17 @@ spindlekv_status codebook_shallow_impl(const spindlekv_config& cfg, const spindl
     extract_kernel<<<(unsigned)(((size_t)units * p.row_words * 32 + 255) / 256), 256, 0, st>>>(p);
   }
   // cooperative launch: as many blocks as can be resident at once
-  static int coop_blocks = 0;
-  if (coop_blocks == 0) {
-    int dev = 0, sms = 0, per_sm = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return SPINDLEKV_CUDA;
+  static int coop_blocks_dev[kMaxDevices] = {};
+  const int dev = PerDeviceOnce::current();
+  if (dev < 0) return SPINDLEKV_CUDA;
+  if (coop_blocks_dev[dev] == 0) {
+    int sms = 0, per_sm = 0;
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return SPINDLEKV_CUDA;
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, greedy_kernel, 512, 0) != cudaSuccess) return SPINDLEKV_CUDA;
     if (per_sm < 1) return SPINDLEKV_CUDA;
-    coop_blocks = sms * per_sm;
+    coop_blocks_dev[dev] = sms * per_sm;
   }
+  const int coop_blocks = coop_blocks_dev[dev];
   for (int phase = 2; phase <= 3; ++phase) {
     const int word_blocks = (int)(((size_t)units * p.row_words * 32 + 255) / 256);
     LaunchScope ls(KC_GREEDY, st);
@@ -809,11 +811,11 @@ spindlekv_status codebook_shallow_impl(const spindlekv_config& cfg, const spindl
   }
   {
     size_t smem = (size_t)(b.max_len + 2) * 4;
-    static bool attr_set = false;
-    if (!attr_set) {
+    static PerDeviceOnce once;
+    if (!once.done[dev]) {
       if (cudaFuncSetAttribute(finalize_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess)
         return SPINDLEKV_CUDA;
-      attr_set = true;
+      once.done[dev] = true;
     }
     LaunchScope ls(KC_FINAL, st);
     finalize_kernel<<<units, kFinalThreads, smem, st>>>(p);

@@ -141,6 +141,18 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int* warp_sums, int& 
   return res;
 }
 
+// Per-device "done once" flags for host-side set-up (function attributes, occupancy queries): the
+// library may be used from several devices of one process.
+constexpr int kMaxDevices = 64;
+struct PerDeviceOnce {
+  bool done[kMaxDevices] = {};
+  // index of the current device, or -1
+  static int current() {
+    int dev = -1;
+    return cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < kMaxDevices ? dev : -1;
+  }
+};
+
 // ---- launch bookkeeping (host) ---------------------------------------------------------------
 void note_launch(int kclass, cudaStream_t st, bool before);
 struct LaunchScope {

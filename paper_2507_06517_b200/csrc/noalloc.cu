@@ -21,14 +21,13 @@ spindlekv_status evict_deep_impl(const spindlekv_config& cfg, const spindlekv_ba
 static __device__ __align__(256) unsigned char g_evict_scratch[SPINDLEKV_NOALLOC_SCRATCH_BYTES];
 
 namespace {
-constexpr int kMaxDevices = 64;
 std::mutex g_setup_mu;
-void* g_scratch_ptr[kMaxDevices] = {};
+void* g_scratch_ptr[skv::kMaxDevices] = {};
 
 // Device address of the scratch array on the current device (looked up once per device).
 spindlekv_status scratch_for_current_device(void** out) {
   int dev = -1;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return SPINDLEKV_CUDA;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= skv::kMaxDevices) return SPINDLEKV_CUDA;
   std::lock_guard<std::mutex> lk(g_setup_mu);
   if (!g_scratch_ptr[dev]) {
     void* ptr = nullptr;

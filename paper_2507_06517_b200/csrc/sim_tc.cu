@@ -477,16 +477,15 @@ static bool make_ext_map(CUtensorMap* map, const void* ext, int units, int rows_
 }
 
 bool sim_tc_available() {
-  static int ok = -1;
-  if (ok < 0) {
-    int dev = 0, major = 0;
-    ok = 0;
-    if (cudaGetDevice(&dev) == cudaSuccess &&
-        cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) == cudaSuccess && major == 10 &&
-        encode_fn() != nullptr)
-      ok = 1;
+  static int ok[kMaxDevices] = {};   // 0: not asked yet, 1: yes, 2: no
+  const int dev = PerDeviceOnce::current();
+  if (dev < 0) return false;
+  if (ok[dev] == 0) {
+    int major = 0;
+    ok[dev] = (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) == cudaSuccess && major == 10 &&
+               encode_fn() != nullptr) ? 1 : 2;
   }
-  return ok == 1;
+  return ok[dev] == 1;
 }
 
 spindlekv_status launch_sim_tc(const spindlekv_tensor& Gamma, const spindlekv_batch& b, int n_kv_heads, int head_dim,
@@ -505,19 +504,23 @@ spindlekv_status launch_sim_tc(const spindlekv_tensor& Gamma, const spindlekv_ba
   dim3 grid(2 * ceil_div(b.max_len, 2 * kBM), units);   // whole pairs
   LaunchScope ls(KC_SIM, st);
   if (head_dim == 128) {
-    static bool set = false;
-    if (!set) {
+    static PerDeviceOnce once;
+    const int dev = PerDeviceOnce::current();
+    if (dev < 0) return SPINDLEKV_CUDA;
+    if (!once.done[dev]) {
       if (cudaFuncSetAttribute(sim_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, SimSmem<128>::TOTAL) != cudaSuccess)
         return SPINDLEKV_CUDA;
-      set = true;
+      once.done[dev] = true;
     }
     sim_tc_kernel<128><<<grid, kSimThreads, SimSmem<128>::TOTAL, st>>>(map, emap, p);
   } else {
-    static bool set = false;
-    if (!set) {
+    static PerDeviceOnce once;
+    const int dev = PerDeviceOnce::current();
+    if (dev < 0) return SPINDLEKV_CUDA;
+    if (!once.done[dev]) {
       if (cudaFuncSetAttribute(sim_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, SimSmem<64>::TOTAL) != cudaSuccess)
         return SPINDLEKV_CUDA;
-      set = true;
+      once.done[dev] = true;
     }
     sim_tc_kernel<64><<<grid, kSimThreads, SimSmem<64>::TOTAL, st>>>(map, emap, p);
   }

@@ -346,11 +346,13 @@ template <int D, int QB>
 static spindlekv_status launch_one(const CUtensorMap& kmap, const CUtensorMap& qmap, const WinTcParams& p, int units,
                                    cudaStream_t st) {
   using L = WinSmem<D, QB>;
-  static bool set = false;
-  if (!set) {
+  static PerDeviceOnce once;
+  const int dev = PerDeviceOnce::current();
+  if (dev < 0) return SPINDLEKV_CUDA;
+  if (!once.done[dev]) {
     if (cudaFuncSetAttribute(win_tc_kernel<D, QB>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::TOTAL) != cudaSuccess)
       return SPINDLEKV_CUDA;
-    set = true;
+    once.done[dev] = true;
   }
   win_tc_kernel<D, QB><<<units, kWinThreads, L::TOTAL, st>>>(kmap, qmap, p);
   return SPINDLEKV_OK;
