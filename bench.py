@@ -50,6 +50,8 @@ def parse_args():
     ap.add_argument("--shallow", type=int, default=None, help="override the number of CodeBook layers")
     ap.add_argument("--literal", action="store_true",
                     help="the paper's own composition: every layer evicts, then builds CodeBooks of what it kept")
+    ap.add_argument("--repeat", action="store_true",
+                    help="with --literal: unfold GQA, every query head selects its own tokens (Section 3.3)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--e2e-chunk", type=int, default=4, help="CodeBook layers per upload/compute/download group")
@@ -217,7 +219,7 @@ def run_literal(args, wl):
     """Every layer evicts under the pyramid over all layers, then builds K and V CodeBooks of the kept
     tokens (Section 3 as written).  Single GPU; reports throughput and the reserve ratios of Eq. (15)."""
     from paper_2507_06517_b200 import binding as B
-    from paper_2507_06517_b200.pipeline import SpindleKVLiteralPass
+    from paper_2507_06517_b200.pipeline import SpindleKVLiteralPass, SpindleKVRepeatPass
     if not torch.cuda.is_available():
         raise RuntimeError("bench.py needs a CUDA device: the reduction pass has no CPU fallback")
     dev = torch.device("cuda", 0)
@@ -228,7 +230,7 @@ def run_literal(args, wl):
                    window=wl.window, n_shallow=-1, beta=wl.beta, theta_k=wl.theta_k, theta_v=wl.theta_v,
                    budget_tokens=wl.budget_tokens if wl.budget_tokens is not None else -1.0,
                    reserve_ratio=wl.budget_frac if wl.budget_frac is not None else -1.0)
-    p = SpindleKVLiteralPass(cfg, wl.seq_lens, hK.dtype, device=dev)
+    p = (SpindleKVRepeatPass if args.repeat else SpindleKVLiteralPass)(cfg, wl.seq_lens, hK.dtype, device=dev)
     dK, dV, dQ = hK.to(dev), hV.to(dev), hQ.to(dev)
     for _ in range(max(args.warmup, 3)):
         p.run(dK, dV, dQ)
@@ -245,11 +247,12 @@ def run_literal(args, wl):
     torch.cuda.synchronize(dev)
     ms = ev0.elapsed_time(ev1)
     launches = B.spindlekv_launch_count(True)
-    nk, nv = p.entry_counts()
-    kept = p.kept_host[:, 0].astype(np.float64)
+    nk, nv = p.cb["K"]["n_entries"].cpu().numpy(), p.cb["V"]["n_entries"].cpu().numpy()
+    kept = p.kept_host[:, 0].astype(np.float64)       # tokens kept per head (per query head when unfolded)
+    heads = wl.n_q_heads if args.repeat else wl.n_kv_heads   # Eq. (15): h_g = h after a repeat
     r1 = kept / wl.max_len
-    r2 = (nk[:, 0].sum(axis=1) + nv[:, 0].sum(axis=1)) / (2.0 * wl.n_kv_heads * kept)
-    line = {"metric": METRIC + ", composition as written", "value": wl.total_tokens * args.steps / (ms * 1e-3),
+    r2 = (nk[:, 0].sum(axis=1) + nv[:, 0].sum(axis=1)) / (2.0 * heads * kept)
+    line = {"metric": METRIC + (", composition as written, GQA unfolded" if args.repeat else ", composition as written"), "value": wl.total_tokens * args.steps / (ms * 1e-3),
             "unit": UNIT, "n_gpus": 1, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic",
             "config": workload_config(wl, {"composition": "every layer: evict (pyramid over all layers), then CodeBooks of the kept tokens"}),
