@@ -421,6 +421,20 @@ def test_degenerate_cases_on_the_tensor_core_path():
         check_codebook_unit(g, 0.999, *out, 1e-2)
 
 
+def test_tensor_core_similarity_at_awkward_lengths():
+    # lengths around the 128-row blocks and 256-row spans of the CTA pairs (odd numbers of blocks, a lone block,
+    # two tokens), both head sizes; clustered rows so that the graphs are not empty
+    rng = np.random.default_rng(23)
+    from paper_2507_06517_b200.synth import round_to_dtype
+    for d in (128, 64):
+        for n in (2, 31, 128, 129, 255, 256, 257, 383, 385, 641, 1100):
+            cents = rng.standard_normal((max(2, n // 12), d)).astype(np.float32)
+            g = cents[rng.integers(0, cents.shape[0], size=n)] + 0.12 * rng.standard_normal((n, d)).astype(np.float32)
+            g = round_to_dtype(g, "bf16")
+            out = _single_layer_codebook(g, 0.95, "bf16")
+            check_codebook_unit(g, 0.95, *out, 1e-2)
+
+
 def test_all_scores_tie_goes_to_lowest_positions():
     # zero queries: plain window sums tie everywhere -> the first k context tokens; with the division
     # by (l - a) scores rise with position -> the last k
