@@ -124,6 +124,15 @@ def test_threshold_is_strict_and_diagonal_is_one():
     assert np.array_equal(G, G.T)
 
 
+def test_opposite_vectors_are_not_similar():
+    # Eq. (9) compares the signed cosine: a vector and its negative (cosine -1) share no edge
+    g = np.array([[2.0, 1.0], [-4.0, -2.0], [2.0, 1.1]])
+    G = O.adjacency(O.cosine_similarity(g), 0.9)
+    assert not G[0, 1] and not G[1, 2] and G[0, 2]
+    r = O.codebook_shallow(g, 0.9)
+    assert list(r["centres"]) == [0, 1] and list(r["ref"]) == [0, 1, 0]
+
+
 def test_degenerate_thresholds():
     rng = np.random.default_rng(11)
     g = rng.standard_normal((20, 8))

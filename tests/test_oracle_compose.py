@@ -1,6 +1,8 @@
 """Pins for the checker's composition of Section 3 (every layer evicts, then builds CodeBooks of what it
 kept) and for the reserve ratio of Eq. (15): closed forms and special cases whose answer does not
 depend on the checker's own code."""
+import math
+
 import numpy as np
 import pytest
 
@@ -62,6 +64,19 @@ def test_no_merging_and_total_merging():
     assert r2 == pytest.approx(1 / 26)
     r1, r2 = O.reserve_ratio_layer(100, 40, [10, 30], [20, 20])
     assert r1 == pytest.approx(0.4) and r2 == pytest.approx(80 / 160)
+
+
+def test_each_cache_uses_its_own_threshold():
+    # one threshold merges everything, the other nothing: which cache got which shows in the entry counts
+    rng = np.random.default_rng(16)
+    l, w, d, H = 70, 5, 12, 2
+    k, v = rng.standard_normal((H, l, d)), rng.standard_normal((H, l, d))
+    q = rng.standard_normal((2 * H, w, d))
+    out = O.spindle_layer(q, k, v, 15, 0.999999, -1.5)
+    rep = O.spindle_layer_repeat(q, k, v, 15, 0.999999, -1.5)
+    for j in range(H):
+        assert len(out["cb_k"][j]["centres"]) == 20 and len(out["cb_v"][j]["centres"]) == 1
+        assert len(rep["cb_v"][j]["centres"]) == 1 and len(rep["cb_k"][j]["centres"]) == len(set(rep["union"][j]))
 
 
 def test_repeat_variant_selects_per_query_head_and_collapses_repeats():
@@ -128,3 +143,21 @@ def test_decode_time_merge_of_new_tokens():
     assert np.array_equal(ext["ref"], 5 + alone["ref"]) and np.allclose(ext["C"][5:], alone["C"])
     # an empty CodeBook: plain Algorithm 1
     assert np.array_equal(O.codebook_extend(np.zeros((0, d)), new, 0.9)["ref"], O.codebook_shallow(new, 0.9)["ref"])
+
+
+def test_merge_takes_the_most_similar_entry_and_the_lower_number_on_exact_ties():
+    # unit entries in the plane at 0, 30 and 0 degrees (entries 0 and 2 are the same vector), one at 90 degrees
+    ang = np.deg2rad([0.0, 30.0, 0.0, 90.0])
+    C = np.stack([np.cos(ang), np.sin(ang)], axis=1)
+    deg = np.deg2rad([25.0, 0.0, 12.0, 50.0])
+    new = np.stack([np.cos(deg), np.sin(deg)], axis=1) * np.array([2.0, 0.5, 1.0, 3.0])[:, None]
+    ref, S = O.match_entries(C, new, math.cos(math.radians(28.0)))
+    # 25 degrees: entries 0/2 (25 away) and 1 (5 away) are all suitable, the nearest wins
+    # 0 degrees: entries 0 and 2 tie exactly, the lower number wins
+    # 12 degrees: 12 from entries 0/2, 18 from entry 1: entry 0 again
+    # 50 degrees: 20 from entry 1, suitable; 40 from entry 3, not suitable
+    assert list(ref) == [1, 0, 0, 1]
+    np.testing.assert_allclose(S[0], np.cos(np.deg2rad([25.0, 5.0, 25.0, 65.0])), atol=1e-15)
+    # at a 4-degree threshold only the exact copy is suitable; the others open entries of their own
+    out = O.codebook_extend(C, new, math.cos(math.radians(4.0)))
+    assert list(out["ref"]) == [4, 0, 5, 6] and list(out["left"]) == [0, 2, 3]
