@@ -186,7 +186,8 @@ spindlekv_status spindlekv_codebook_shallow(const spindlekv_config* cfg, const s
  *   idx        device [n_layers][n_heads][T] as written by the two calls above
  *   cnt        device [n_layers][B][n_heads]
  *   divide_by  device, optional [n_layers][n_heads][T] fp32: when given, source row a is divided by
- *              divide_by[a] (a zero divisor yields a zero row); pass `mag` to obtain unit CodeBook vectors
+ *              divide_by[a] (in fp32, as a product with the correctly rounded reciprocal, then rounded to the
+ *              storage type; a zero divisor yields a zero row); pass `mag` to obtain unit CodeBook vectors
  *   dst        device, same addressing rules as src; when dst_cu_seqlens is given, unit s starts at row
  *              dst_cu_seqlens[s] of dst, else rows are addressed like src (batch->cu_seqlens or stride_seq)
  * src and dst must have the same dtype and may not overlap.

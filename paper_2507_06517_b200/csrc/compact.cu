@@ -1,6 +1,6 @@
 // Gather of kept tokens / CodeBook centres into the output cache (Eq. (7) second line, Eq. (11)):
-// 16-byte loads and stores, one row per group of head_dim*elem/16 threads, rows of a unit contiguous
-// in the destination.
+// 16-byte loads and stores, one row per group of head_dim*elem/16 threads, eight rows of every group in
+// flight, rows of a unit contiguous in the destination.
 #include "common.cuh"
 
 namespace skv {
@@ -15,11 +15,13 @@ struct CompactParams {
   const int32_t* dst_cu;  // optional [B+1]
 };
 
+constexpr int kGatherRows = 8;   // rows per thread group, all of their loads in flight before any is used
+
 template <typename T, int D>
 __global__ void __launch_bounds__(256) compact_kernel(CompactParams p) {
   constexpr int EPT = 16 / sizeof(T);       // elements per thread
   constexpr int TPR = D / EPT;              // threads per row
-  constexpr int RPB = 256 / TPR;            // rows per block
+  constexpr int RPB = 256 / TPR;            // rows per sweep of the block
   const int unit = blockIdx.y;
   const int h = unit % p.n_heads;
   const int ls = unit / p.n_heads;
@@ -33,28 +35,44 @@ __global__ void __launch_bounds__(256) compact_kernel(CompactParams p) {
   else if (p.batch.cu) dbase += (int64_t)p.batch.cu[s] * p.dst.st;
   else dbase += (int64_t)s * p.dst.ss;
   const int seg = threadIdx.x % TPR;
-  for (int r = blockIdx.x * RPB + threadIdx.x / TPR; r < n; r += gridDim.x * RPB) {
-    const int a = p.idx[orow + r];
-    uint4 v = *reinterpret_cast<const uint4*>(sbase + (int64_t)a * p.src.st + seg * EPT);
-    if (p.divide_by) {
-      const float m = p.divide_by[orow + a];
-      if (sizeof(T) == 4) {
-        float* f = reinterpret_cast<float*>(&v);
+  // a block owns kGatherRows * RPB consecutive output rows
+  for (int r0 = blockIdx.x * (RPB * kGatherRows) + threadIdx.x / TPR; r0 < n; r0 += gridDim.x * (RPB * kGatherRows)) {
+    int a[kGatherRows];
+    uint4 v[kGatherRows];
+    float rc[kGatherRows];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) f[i] = m > 0.f ? f[i] / m : 0.f;
-      } else {
-        uint32_t* w = reinterpret_cast<uint32_t*>(&v);
+    for (int i = 0; i < kGatherRows; ++i) {
+      const int r = r0 + i * RPB;
+      a[i] = r < n ? p.idx[orow + r] : -1;
+    }
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          float lo = __uint_as_float(w[i] << 16), hi = __uint_as_float(w[i] & 0xFFFF0000u);
-          lo = m > 0.f ? lo / m : 0.f;
-          hi = m > 0.f ? hi / m : 0.f;
-          __nv_bfloat162 pk = __floats2bfloat162_rn(lo, hi);
-          w[i] = *reinterpret_cast<uint32_t*>(&pk);
+    for (int i = 0; i < kGatherRows; ++i) {
+      if (a[i] < 0) continue;
+      v[i] = *reinterpret_cast<const uint4*>(sbase + (int64_t)a[i] * p.src.st + seg * EPT);
+      if (p.divide_by) rc[i] = p.divide_by[orow + a[i]];
+    }
+#pragma unroll
+    for (int i = 0; i < kGatherRows; ++i) {
+      if (a[i] < 0) continue;
+      if (p.divide_by) {
+        // one correctly rounded reciprocal per row, then a product per element; a zero row stays zero
+        const float m = rc[i] > 0.f ? __frcp_rn(rc[i]) : 0.f;
+        if (sizeof(T) == 4) {
+          float* f = reinterpret_cast<float*>(&v[i]);
+#pragma unroll
+          for (int q = 0; q < 4; ++q) f[q] *= m;
+        } else {
+          uint32_t* w = reinterpret_cast<uint32_t*>(&v[i]);
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const float lo = __uint_as_float(w[q] << 16), hi = __uint_as_float(w[q] & 0xFFFF0000u);
+            __nv_bfloat162 pk = __floats2bfloat162_rn(lo * m, hi * m);
+            w[q] = *reinterpret_cast<uint32_t*>(&pk);
+          }
         }
       }
+      *reinterpret_cast<uint4*>(dbase + (int64_t)(r0 + i * RPB) * p.dst.st + seg * EPT) = v[i];
     }
-    *reinterpret_cast<uint4*>(dbase + (int64_t)r * p.dst.st + seg * EPT) = v;
   }
 }
 
@@ -185,8 +203,8 @@ spindlekv_status compact_impl(const spindlekv_batch& b, int n_heads, int head_di
   p.dst_cu = dst_cu;
   const int units = b.n_layers * b.n_seqs * n_heads;
   if (units > 65535) return SPINDLEKV_UNSUPPORTED;
-  // enough blocks along x to cover the longest possible row list once at 16 rows per block
-  const int gx = ceil_div(b.max_len, 64);
+  // enough blocks along x to cover the longest possible row list in one sweep (128 rows per block at 16 threads per row)
+  const int gx = ceil_div(b.max_len, 16 * kGatherRows);
   dim3 grid(gx, units);
   LaunchScope ls(KC_GATHER, st);
   const bool bf = src.dtype == SPINDLEKV_BF16;
