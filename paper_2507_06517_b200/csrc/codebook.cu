@@ -221,7 +221,8 @@ __device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long v)
 // and are appended to a list of dense rows.  A token with no neighbour at all is settled here: it is
 // a centre with pick degree 1 (Algorithm 1 reaches it with exactly that degree, whenever it does).
 constexpr int kEll = 32;
-constexpr int kChunkBatch = 4;
+constexpr int kChunkBatch = 8;    // occupied chunks of a row fetched together
+constexpr int kFlagGroup = 8;     // flag words fetched together (256 chunks = 16384 columns)
 
 __global__ void __launch_bounds__(256) extract_kernel(CodebookParams p) {
   const int lane = threadIdx.x & 31;
@@ -242,31 +243,35 @@ __global__ void __launch_bounds__(256) extract_kernel(CodebookParams p) {
   tr.init(lane);
   int cnt = 1, k = 0;
   const int nc = (l + 63) >> 6;   // chunks of this sequence (flags and bit rows beyond it are not written)
-  constexpr int kFlagGroup = 8;   // flag words fetched together (256 chunks = 16384 columns)
+  __shared__ uint32_t occ_sh[kFlagGroup][256];   // per thread: occupancy of its row, 32 chunks per word
   for (int cb = 0; cb < nc; cb += 32 * kFlagGroup) {
-  uint32_t fw[kFlagGroup];
+    uint32_t fw[kFlagGroup];
 #pragma unroll
-  for (int i = 0; i < kFlagGroup; ++i) {
-    const int c = cb + 32 * i + lane;
-    fw[i] = c < nc ? fl[c] : 0u;
-  }
-#pragma unroll
-  for (int i = 0; i < kFlagGroup; ++i) {
-    const int c0 = cb + 32 * i;
-    if (c0 >= nc) break;
-    // lane c held the flags of chunk c0 + c for the warp's 32 rows; after the transpose lane r holds
+    for (int i = 0; i < kFlagGroup; ++i) {
+      const int c = cb + 32 * i + lane;
+      fw[i] = c < nc ? fl[c] : 0u;
+    }
+    // lane c held the flags of chunk cb + 32 i + c for the warp's 32 rows; after the transpose lane r holds
     // the flags of its own row for these 32 chunks
-    uint32_t occ = tr.apply(fw[i]);
-    if (!exists) occ = 0;
-    while (occ) {
-      // several occupied chunks at a time, loaded before any of them is looked at
+#pragma unroll
+    for (int i = 0; i < kFlagGroup; ++i) {
+      const uint32_t occ = tr.apply(fw[i]);
+      occ_sh[i][threadIdx.x] = exists ? occ : 0u;
+    }
+    // the row's occupied chunks in ascending order, kChunkBatch at a time across all flag words, loaded
+    // before any of them is looked at: a row costs a round trip per batch, not one per flag word
+    int wi = 0;
+    uint32_t cur = occ_sh[0][threadIdx.x];
+    for (;;) {
       int cs[kChunkBatch];
       uint2 av[kChunkBatch];
 #pragma unroll
       for (int i = 0; i < kChunkBatch; ++i) {
-        cs[i] = occ ? c0 + __ffs(occ) - 1 : -1;
-        occ &= occ - 1;   // 0 stays 0
+        while (cur == 0u && wi < kFlagGroup - 1) cur = occ_sh[++wi][threadIdx.x];
+        cs[i] = cur ? cb + 32 * wi + __ffs(cur) - 1 : -1;
+        cur &= cur - 1;   // 0 stays 0
       }
+      if (cs[0] < 0) break;
 #pragma unroll
       for (int i = 0; i < kChunkBatch; ++i) av[i] = cs[i] >= 0 ? row2[cs[i]] : make_uint2(0, 0);
 #pragma unroll
@@ -287,7 +292,6 @@ __global__ void __launch_bounds__(256) extract_kernel(CodebookParams p) {
         }
       }
     }
-  }
   }
   bool live = false;
   if (exists) {
