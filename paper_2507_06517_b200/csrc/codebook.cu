@@ -584,12 +584,18 @@ __global__ void __launch_bounds__(512) greedy_kernel(CodebookParams p) {
 // ---- entry numbering ------------------------------------------------------------------------------
 // One block per unit.  Entries are numbered by decreasing pick-time key (degree, then lower index):
 // a counting sort on the degree, stable in the index.  hist[] lives in dynamic shared memory.
+// Centres of degree 1 are placed by all threads (ballots and a block scan); centres of larger degree by
+// one warp that walks, in index order, only the 32-token chunks that hold one.
 constexpr int kFinalThreads = 1024;
+constexpr int kFinalBatch = 16;        // tokens per thread loaded together
+constexpr int kFinalChunkWords = 64;   // chunk map for 64 * 32 * 32 = 65536 tokens (longer sequences: every chunk is visited)
 
 __global__ void __launch_bounds__(kFinalThreads) finalize_kernel(CodebookParams p) {
   extern __shared__ int hist[];  // [l + 2]
   __shared__ int warp_sums[33];
-  __shared__ int carry_sh;
+  __shared__ uint32_t busy[kFinalChunkWords];   // bit per 32-token chunk: holds a centre of pick degree >= 2
+  __shared__ uint16_t busy_list[kFinalChunkWords * 32];
+  __shared__ int cnt_sh[kFinalBatch * 32];
   const int unit = blockIdx.x;
   int layer, s, j;
   cb_decode(p, unit, layer, s, j);
@@ -602,74 +608,160 @@ __global__ void __launch_bounds__(kFinalThreads) finalize_kernel(CodebookParams 
   const int tid = threadIdx.x, lane = tid & 31;
 
   for (int d = tid; d <= l + 1; d += kFinalThreads) hist[d] = 0;
+  for (int c = tid; c < kFinalChunkWords; c += kFinalThreads) busy[c] = 0u;
   __syncthreads();
-  for (int u = tid; u < l; u += kFinalThreads) {
-    int d = pickdeg[u];
-    if (d >= 0) atomicAdd(&hist[d], 1);
+  // centres of pick degree 1 (tokens without a neighbour, as a rule the bulk) are counted by ballot: one
+  // atomic per warp instead of 32 on one address.  A thread's kFinalBatch tokens are loaded before any is used.
+  for (int base0 = 0; base0 < l; base0 += kFinalBatch * kFinalThreads) {
+    int dr[kFinalBatch];
+#pragma unroll
+    for (int i = 0; i < kFinalBatch; ++i) {
+      const int u = base0 + i * kFinalThreads + tid;
+      dr[i] = u < l ? pickdeg[u] : -1;
+    }
+    int n_ones = 0;
+#pragma unroll
+    for (int i = 0; i < kFinalBatch; ++i) {
+      const int u = base0 + i * kFinalThreads + tid;
+      n_ones += __popc(__ballot_sync(0xffffffffu, dr[i] == 1));
+      if (dr[i] >= 2) atomicAdd(&hist[dr[i]], 1);
+      // 32-token chunks that hold a centre of degree >= 2: the only ones the ordered sweep below visits
+      const uint32_t more = __ballot_sync(0xffffffffu, dr[i] >= 2);
+      if (lane == 0 && more && (u >> 5) < kFinalChunkWords * 32) atomicOr(&busy[u >> 10], 1u << ((u >> 5) & 31));
+    }
+    if (lane == 0 && n_ones) atomicAdd(&hist[1], n_ones);
   }
   __syncthreads();
-  // start[d] = number of centres with a larger degree: exclusive scan from the top, in place
-  if (tid == 0) carry_sh = 0;
-  __syncthreads();
-  for (int top = l; top >= 0; top -= kFinalThreads) {
-    int d = top - tid;
-    int v = d >= 0 ? hist[d] : 0;
-    // inclusive-to-exclusive scan within the block via warp shuffles
-    int inc = v;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      int n = __shfl_up_sync(0xffffffffu, inc, o);
-      if (lane >= o) inc += n;
+  // start[d] = number of centres with a larger degree: exclusive scan from the top, in place; a thread owns
+  // `nb` consecutive degrees
+  int n_entries;
+  {
+    const int nb = (l + 1 + kFinalThreads - 1) / kFinalThreads;
+    const int hi = l - tid * nb;
+    int sum = 0;
+    for (int i = 0; i < nb; ++i) {
+      const int d = hi - i;
+      if (d >= 0) sum += hist[d];
     }
-    if (lane == 31) warp_sums[tid >> 5] = inc;
+    int run = block_exclusive_scan(sum, warp_sums, n_entries);
+    for (int i = 0; i < nb; ++i) {
+      const int d = hi - i;
+      if (d >= 0) {
+        const int v = hist[d];
+        hist[d] = run;
+        run += v;
+      }
+    }
     __syncthreads();
-    if (tid < 32) {
-      int ws = warp_sums[tid], winc = ws;
+  }
+  // degree 1, stable in the index: position = start[1] + number of such centres before the token
+  {
+    int before = hist[1];
+    for (int base0 = 0; base0 < l; base0 += kFinalBatch * kFinalThreads) {
+      uint32_t ones[kFinalBatch];
+      int dr[kFinalBatch];
+#pragma unroll
+      for (int i = 0; i < kFinalBatch; ++i) {
+        const int u = base0 + i * kFinalThreads + tid;
+        dr[i] = u < l ? pickdeg[u] : -1;
+      }
+#pragma unroll
+      for (int i = 0; i < kFinalBatch; ++i) {
+        ones[i] = __ballot_sync(0xffffffffu, dr[i] == 1);
+        if (lane == 0) cnt_sh[i * 32 + (tid >> 5)] = __popc(ones[i]);   // in token order: sweep i, warp w
+      }
+      __syncthreads();
+      int tot;
+      {
+        // exclusive scan of the kFinalBatch * 32 counts (entries beyond them count 0)
+        const int v = tid < kFinalBatch * 32 ? cnt_sh[tid] : 0;
+        const int ex = block_exclusive_scan(v, warp_sums, tot);
+        if (tid < kFinalBatch * 32) cnt_sh[tid] = ex;
+        __syncthreads();
+      }
+#pragma unroll
+      for (int i = 0; i < kFinalBatch; ++i) {
+        if (dr[i] == 1) {
+          const int u = base0 + i * kFinalThreads + tid;
+          const int pos = before + cnt_sh[i * 32 + (tid >> 5)] + __popc(ones[i] & ((1u << lane) - 1u));
+          rank[u] = pos;
+          p.centre_idx[orow + pos] = u;
+        }
+      }
+      before += tot;
+      __syncthreads();
+    }
+  }
+  // larger degrees: stable placement in index order by one warp over the chunks that hold such a centre,
+  // eight chunks in flight
+  if (tid < 32) {
+    const int n_chunks = (l + 31) >> 5;
+    // ascending list of those chunks (beyond the map every chunk is listed by its number at once)
+    int n_busy = 0;
+    for (int cw0 = 0; cw0 < kFinalChunkWords; cw0 += 32) {
+      uint32_t wd = busy[cw0 + lane];
+      const int c = __popc(wd);
+      int inc = c;
 #pragma unroll
       for (int o = 1; o < 32; o <<= 1) {
-        int n = __shfl_up_sync(0xffffffffu, winc, o);
-        if (lane >= o) winc += n;
+        const int n = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += n;
       }
-      warp_sums[tid] = winc - ws;
-      if (tid == 31) warp_sums[32] = winc;
+      int at = n_busy + inc - c;
+      while (wd) {
+        busy_list[at++] = (uint16_t)((cw0 + lane) * 32 + __ffs(wd) - 1);
+        wd &= wd - 1;
+      }
+      n_busy += __shfl_sync(0xffffffffu, inc, 31);
     }
-    __syncthreads();
-    int excl = warp_sums[tid >> 5] + inc - v + carry_sh;
-    int tot = warp_sums[32];
-    if (d >= 0) hist[d] = excl;
-    __syncthreads();
-    if (tid == 0) carry_sh += tot;
-    __syncthreads();
-  }
-  const int n_entries = carry_sh;
-  // stable placement in index order by one warp, eight chunks of 32 tokens in flight
-  if (tid < 32) {
-    for (int base = 0; base < l; base += 256) {
-      int dv[8];
+    __syncwarp();
+    const int extra0 = kFinalChunkWords * 32;   // first chunk that the map does not cover
+    const int n_items = n_busy + (n_chunks > extra0 ? n_chunks - extra0 : 0);
+    for (int i0 = 0; i0 < n_items; i0 += 8) {
+      int cv[8], dv[8];
 #pragma unroll
-      for (int c = 0; c < 8; ++c) {
-        int u = base + c * 32 + lane;
-        dv[c] = u < l ? pickdeg[u] : -1;
+      for (int i = 0; i < 8; ++i) {
+        const int it = i0 + i;
+        cv[i] = it < n_busy ? (int)busy_list[it] : (it < n_items ? extra0 + (it - n_busy) : -1);
+        const int u = cv[i] * 32 + lane;
+        dv[i] = (cv[i] >= 0 && u < l) ? pickdeg[u] : -1;
       }
 #pragma unroll
-      for (int c = 0; c < 8; ++c) {
-        int u = base + c * 32 + lane;
-        int d = dv[c];
-        uint32_t peers = __match_any_sync(0xffffffffu, d);
-        if (d >= 0) {
-          int before = __popc(peers & ((1u << lane) - 1u));
-          int pos = hist[d] + before;
+      for (int i = 0; i < 8; ++i) {
+        if (cv[i] < 0) break;
+        const int u = cv[i] * 32 + lane;
+        const int d = dv[i] >= 2 ? dv[i] : -1;   // others share one value: the match costs a step per distinct value
+        const uint32_t peers = __match_any_sync(0xffffffffu, d);
+        if (d >= 2) {
+          const int pos = hist[d] + __popc(peers & ((1u << lane) - 1u));
           rank[u] = pos;
           p.centre_idx[orow + pos] = u;
         }
         __syncwarp();
-        if (d >= 0 && lane == (31 - __clz(peers))) hist[d] += __popc(peers);
+        if (d >= 2 && lane == (31 - __clz(peers))) hist[d] += __popc(peers);
         __syncwarp();
       }
     }
   }
   __syncthreads();
-  for (int b = tid; b < l; b += kFinalThreads) p.ref[orow + b] = rank[owner[b]];
+  // rank[] was written by this block: make the writes visible to all of its threads, then resolve the references
+  // (eight independent owner -> rank chains per thread)
+  for (int b0 = tid; b0 < l; b0 += 8 * kFinalThreads) {
+    int o[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int b = b0 + i * kFinalThreads;
+      o[i] = b < l ? owner[b] : -1;
+    }
+    int r[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) r[i] = o[i] >= 0 ? rank[o[i]] : 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int b = b0 + i * kFinalThreads;
+      if (b < l) p.ref[orow + b] = r[i];
+    }
+  }
   if (tid == 0) p.n_entries[(layer * p.batch.n_seqs + s) * p.n_kv_heads + j] = n_entries;
 }
 
