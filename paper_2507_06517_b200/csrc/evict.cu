@@ -186,10 +186,16 @@ __device__ __forceinline__ uint32_t order_key(float f) {
 }
 
 constexpr int kTopkThreads = 1024;
+constexpr int kTopkItems = 16;                                // scores per thread loaded together
+constexpr int kTopkChunk = kTopkThreads * kTopkItems;         // scores per sweep of the block
 
+// One block per unit.  Four 8-bit radix passes find the k-th largest key and how many of its equals are
+// taken; one ordered pass writes the kept positions in ascending order (ties to the lower position).
+// A thread loads its kTopkItems scores of a sweep (positions `i * kTopkThreads + tid`) before using any.
 __global__ void __launch_bounds__(kTopkThreads) topk_kernel(TopkParams p) {
   __shared__ int hist[256];
   __shared__ int warp_sums[33];
+  __shared__ int cnt_gt[kTopkItems * 32], cnt_eq[kTopkItems * 32];
   __shared__ uint32_t sh_prefix;
   __shared__ int sh_need;
   const int unit = blockIdx.x;
@@ -204,59 +210,129 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(TopkParams p) {
   const int64_t row = ((int64_t)layer * p.n_kv_heads + j) * p.batch.total_len + tok_base(p.batch, s);
   const float* sc = p.scores + row;
   int32_t* out = p.keep_idx + row;
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
 
   uint32_t prefix = 0, mask = 0;
   int need = k;
   if (k > 0 && k < l_c) {
     for (int shift = 24; shift >= 0; shift -= 8) {
-      if (threadIdx.x < 256) hist[threadIdx.x] = 0;
+      if (tid < 256) hist[tid] = 0;
       __syncthreads();
-      for (int a = threadIdx.x; a < l_c; a += kTopkThreads) {
-        uint32_t key = order_key(sc[a]);
-        if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255], 1);
+      for (int a0 = 0; a0 < l_c; a0 += kTopkChunk) {
+        uint32_t key[kTopkItems];
+#pragma unroll
+        for (int i = 0; i < kTopkItems; ++i) {
+          const int a = a0 + i * kTopkThreads + tid;
+          key[i] = a < l_c ? order_key(sc[a]) : 0u;
+        }
+#pragma unroll
+        for (int i = 0; i < kTopkItems; ++i) {
+          const int a = a0 + i * kTopkThreads + tid;
+          const bool part = a < l_c && (key[i] & mask) == prefix;
+          const int bin = (key[i] >> shift) & 255;
+          if (shift == 24) {
+            // the leading byte (sign and exponent) takes few values: one atomic per value and warp
+            const uint32_t peers = __match_any_sync(0xffffffffu, part ? bin : 256);
+            if (part && lane == __ffs(peers) - 1) atomicAdd(&hist[bin], __popc(peers));
+          } else if (part) {
+            atomicAdd(&hist[bin], 1);
+          }
+        }
       }
       __syncthreads();
-      if (threadIdx.x == 0) {
-        int cum = 0, bin = 255;
-        for (; bin > 0; --bin) {
-          if (cum + hist[bin] >= need) break;
-          cum += hist[bin];
+      if (wid == 0) {
+        // the bin that holds the `need`-th largest: lane t owns bins 8t .. 8t+7
+        int h[8], mine = 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          h[i] = hist[lane * 8 + i];
+          mine += h[i];
         }
-        sh_prefix = prefix | ((uint32_t)bin << shift);
-        sh_need = need - cum;
+        int incl = mine;   // sum over lanes >= this one
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const int n = __shfl_down_sync(0xffffffffu, incl, o);
+          if (lane + o < 32) incl += n;
+        }
+        int above = incl - mine;
+        // the highest lane whose inclusive sum reaches `need` holds the bin; none does only if fewer than
+        // `need` keys carry the prefix, which the previous pass excludes; bin 0 is the guard
+        const uint32_t reach = __ballot_sync(0xffffffffu, incl >= need);
+        const int owner = reach ? 31 - __clz(reach) : 0;
+        if (lane == owner) {
+          int bin = 7;
+          for (; bin > 0; --bin) {
+            if (above + h[bin] >= need) break;
+            above += h[bin];
+          }
+          sh_prefix = prefix | ((uint32_t)(lane * 8 + bin) << shift);
+          sh_need = need - above;
+        }
       }
       __syncthreads();
       prefix = sh_prefix;
       need = sh_need;
       mask |= 0xFFu << shift;
-      __syncthreads();
     }
   }
-  // ordered sweep
-  int base_eq = 0, base_out = 0;
-  for (int a0 = 0; a0 < l_c; a0 += kTopkThreads) {
-    int a = a0 + threadIdx.x;
-    bool in = a < l_c;
-    int gt = 0, eq = 0;
-    if (in) {
-      if (k >= l_c) gt = 1;
-      else if (k > 0) {
-        uint32_t key = order_key(sc[a]);
-        gt = key > prefix;
-        eq = key == prefix;
+  // ordered pass: counts of every (sweep, warp) by ballot, one block scan over them per kTopkChunk positions
+  int base_gt = 0, base_eq = 0;
+  for (int a0 = 0; a0 < l_c; a0 += kTopkChunk) {
+    uint32_t key[kTopkItems], bg[kTopkItems], be[kTopkItems];
+#pragma unroll
+    for (int i = 0; i < kTopkItems; ++i) {
+      const int a = a0 + i * kTopkThreads + tid;
+      key[i] = (a < l_c && k > 0 && k < l_c) ? order_key(sc[a]) : 0u;
+    }
+#pragma unroll
+    for (int i = 0; i < kTopkItems; ++i) {
+      const int a = a0 + i * kTopkThreads + tid;
+      const bool in = a < l_c;
+      bool gt = false, eq = false;
+      if (in) {
+        if (k >= l_c) gt = true;
+        else if (k > 0) {
+          gt = key[i] > prefix;
+          eq = key[i] == prefix;
+        }
+      }
+      bg[i] = __ballot_sync(0xffffffffu, gt);
+      be[i] = __ballot_sync(0xffffffffu, eq);
+      if (lane == 0) {
+        cnt_gt[i * 32 + wid] = __popc(bg[i]);
+        cnt_eq[i * 32 + wid] = __popc(be[i]);
       }
     }
-    int tot_eq;
-    int eq_rank = block_exclusive_scan(eq, warp_sums, tot_eq) + base_eq;
-    int sel = gt | (eq && eq_rank < need);
-    int tot_sel;
-    int pos = block_exclusive_scan(sel, warp_sums, tot_sel) + base_out;
-    if (sel) out[pos] = a;
+    __syncthreads();
+    int tot_gt, tot_eq;
+    {
+      const bool has = tid < kTopkItems * 32;
+      const int vg = has ? cnt_gt[tid] : 0, ve = has ? cnt_eq[tid] : 0;
+      const int eg = block_exclusive_scan(vg, warp_sums, tot_gt);
+      const int ee = block_exclusive_scan(ve, warp_sums, tot_eq);
+      if (has) {
+        cnt_gt[tid] = eg;
+        cnt_eq[tid] = ee;
+      }
+      __syncthreads();
+    }
+    const uint32_t below = (1u << lane) - 1u;
+#pragma unroll
+    for (int i = 0; i < kTopkItems; ++i) {
+      const int a = a0 + i * kTopkThreads + tid;
+      const bool gt = (bg[i] >> lane) & 1u, eq = (be[i] >> lane) & 1u;
+      if (!gt && !eq) continue;
+      // kept before this position: every larger key, and the first `need` of the equal ones
+      const int gt_before = base_gt + cnt_gt[i * 32 + wid] + __popc(bg[i] & below);
+      const int eq_before = base_eq + cnt_eq[i * 32 + wid] + __popc(be[i] & below);
+      if (gt || eq_before < need) out[gt_before + min(eq_before, need)] = a;
+    }
+    base_gt += tot_gt;
     base_eq += tot_eq;
-    base_out += tot_sel;
+    __syncthreads();
   }
-  for (int t = threadIdx.x; t < p.window; t += kTopkThreads) out[k + t] = l_c + t;
-  if (threadIdx.x == 0) p.keep_cnt[(layer * p.batch.n_seqs + s) * p.n_kv_heads + j] = k + p.window;
+  for (int t = tid; t < p.window; t += kTopkThreads) out[k + t] = l_c + t;
+  if (tid == 0) p.keep_cnt[(layer * p.batch.n_seqs + s) * p.n_kv_heads + j] = k + p.window;
 }
 
 // ---- host side ----------------------------------------------------------------------------------
