@@ -319,6 +319,13 @@ __global__ void __launch_bounds__(256) extract_kernel(CodebookParams p) {
 // live mask and skips words that are empty), dense rows one per warp from their list.
 __device__ __forceinline__ bool is_live(const uint32_t* lv, int v) { return (lv[v >> 5] >> (v & 31)) & 1u; }
 
+// The flag words of token u's group of 32 rows, one per 64-column chunk.  A chunk of a bit row whose flag bit is
+// clear holds no set bit and may never have been written: readers of whole bit rows skip it.
+__device__ __forceinline__ const uint32_t* flag_row(const CodebookParams& p, int unit, int u) {
+  return p.flags + ((int64_t)unit * p.row_words + (u >> 5)) * (p.row_words >> 1);
+}
+__device__ __forceinline__ bool chunk_flagged(const uint32_t* fr, int chunk, int u) { return (fr[chunk] >> (u & 31)) & 1u; }
+
 // Eight entries of a row's neighbour list at a time: the loads of one batch do not depend on each
 // other, so a row costs a few memory round trips instead of one per neighbour.
 constexpr int kBatch = 8;
@@ -373,9 +380,10 @@ __device__ __forceinline__ void max_of_dense_row(const CodebookParams& p, const 
   if (!is_live(lv, u)) return;
   const unsigned long long* key = p.key + (int64_t)unit * ML;
   const uint32_t* row = p.adj + idx * RW;
+  const uint32_t* fr = flag_row(p, unit, u);
   unsigned long long best = 0ull;
   for (int w = lane; w < RW; w += 32) {
-    uint32_t m = row[w] & lv[w];
+    uint32_t m = chunk_flagged(fr, w >> 1, u) ? row[w] & lv[w] : 0u;
     while (m) {
       int b = __ffs(m) - 1;
       m &= m - 1;
@@ -448,9 +456,10 @@ __device__ __forceinline__ void pick_dense_row(const CodebookParams& p, const ui
   int32_t* owner = p.owner + (int64_t)unit * ML;
   uint32_t* nx = next + (int64_t)unit * RW;
   const uint32_t* row = p.adj + idx * RW;
+  const uint32_t* fr = flag_row(p, unit, u);
   bool ok = true;
   for (int w = lane; w < RW; w += 32) {
-    uint32_t m = row[w] & lv[w];
+    uint32_t m = chunk_flagged(fr, w >> 1, u) ? row[w] & lv[w] : 0u;
     while (m) {
       int b = __ffs(m) - 1;
       m &= m - 1;
@@ -460,7 +469,7 @@ __device__ __forceinline__ void pick_dense_row(const CodebookParams& p, const ui
   if (!__all_sync(0xffffffffu, ok)) return;
   if (lane == 0) p.pickdeg[idx] = p.deg[idx];
   for (int w = lane; w < RW; w += 32) {
-    uint32_t m = row[w] & lv[w];
+    uint32_t m = chunk_flagged(fr, w >> 1, u) ? row[w] & lv[w] : 0u;
     if (m) atomicAnd(&nx[w], ~m);
     while (m) {
       int b = __ffs(m) - 1;
@@ -545,10 +554,12 @@ __global__ void __launch_bounds__(512) greedy_kernel(CodebookParams p) {
         if (!is_live(lv, u)) continue;
         const uint4* row4 = reinterpret_cast<const uint4*>(p.adj + idx * RW);
         const uint4* lv4 = reinterpret_cast<const uint4*>(lv);
+        const uint32_t* fr = flag_row(p, unit, u);
         int cnt = 0;
         for (int w4 = lane; w4 < RW4; w4 += 32) {
-          uint4 a = row4[w4], b = lv4[w4];
-          cnt += __popc(a.x & b.x) + __popc(a.y & b.y) + __popc(a.z & b.z) + __popc(a.w & b.w);
+          const uint4 a = row4[w4], b = lv4[w4];
+          if (chunk_flagged(fr, 2 * w4, u)) cnt += __popc(a.x & b.x) + __popc(a.y & b.y);
+          if (chunk_flagged(fr, 2 * w4 + 1, u)) cnt += __popc(a.z & b.z) + __popc(a.w & b.w);
         }
 #pragma unroll
         for (int o = 16; o >= 1; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
@@ -802,7 +813,8 @@ size_t codebook_workspace_bytes(const spindlekv_config& cfg, const spindlekv_bat
 
 bool sim_tc_available();
 spindlekv_status launch_sim_tc(const spindlekv_tensor& Gamma, const spindlekv_batch& b, int n_kv_heads, int head_dim,
-                               const void* ext, uint32_t* adj, uint32_t* flags, uint32_t* hdr, cudaStream_t st);
+                               const void* ext, uint32_t* adj, uint32_t* flags, uint32_t* hdr, bool skip_empty,
+                               cudaStream_t st);
 
 template <typename T, int D>
 static void launch_norms(const CodebookParams& p, cudaStream_t st) {
@@ -866,7 +878,7 @@ spindlekv_status codebook_shallow_impl(const spindlekv_config& cfg, const spindl
   if (tc) {
     // the similarity kernel writes only the flag words that hold a set bit
     if (cudaMemsetAsync(p.flags, 0, (size_t)units * (p.row_words / 2) * p.row_words * 4, st) != cudaSuccess) return SPINDLEKV_CUDA;
-    spindlekv_status rs = launch_sim_tc(Gamma, b, cfg.n_kv_heads, cfg.head_dim, p.ext, p.adj, p.flags, p.hdr, st);
+    spindlekv_status rs = launch_sim_tc(Gamma, b, cfg.n_kv_heads, cfg.head_dim, p.ext, p.adj, p.flags, p.hdr, adj_in_ws, st);
     if (rs != SPINDLEKV_OK) return rs;
   } else if (cfg.head_dim == 64) {
     if (bf) launch_sim_simt<__nv_bfloat16, 64>(p, b, st); else launch_sim_simt<float, 64>(p, b, st);

@@ -43,6 +43,7 @@ struct SimTcParams {
   uint32_t* adj;       // [units][max_len][row_words]
   uint32_t* flags;     // [units][row_words][row_words / 2]
   uint32_t* hdr;
+  int skip_empty;      // mirrored chunks without a set bit are not stored (their flag bit stays 0)
 };
 
 constexpr int kBM = 128;          // rows of the resident block (UMMA M)
@@ -358,9 +359,16 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kSimThreads, 1) sim_
         bool occ_lo = false, occ_hi = false;
         if (b < l) {
           const uint4 mv = make_uint4(tr0[0], tr0[kBN], tr0[2 * kBN], tr0[3 * kBN]);
-          *reinterpret_cast<uint4*>(adj_unit + (int64_t)b * RW + (row0 >> 5)) = mv;
           occ_lo = (mv.x | mv.y) != 0u;
           occ_hi = (mv.z | mv.w) != 0u;
+          uint32_t* dst = adj_unit + (int64_t)b * RW + (row0 >> 5);
+          if (!p.skip_empty) {
+            *reinterpret_cast<uint4*>(dst) = mv;
+          } else {
+            // a reader consults the chunk's flag bit first: empty chunks need not reach memory
+            if (occ_lo) *reinterpret_cast<uint2*>(dst) = make_uint2(mv.x, mv.y);
+            if (occ_hi) *reinterpret_cast<uint2*>(dst + 2) = make_uint2(mv.z, mv.w);
+          }
         }
         const uint32_t flo = __ballot_sync(0xffffffffu, occ_lo), fhi = __ballot_sync(0xffffffffu, occ_hi);
         const uint32_t fw = lane ? fhi : flo;
@@ -489,7 +497,8 @@ bool sim_tc_available() {
 }
 
 spindlekv_status launch_sim_tc(const spindlekv_tensor& Gamma, const spindlekv_batch& b, int n_kv_heads, int head_dim,
-                               const void* ext, uint32_t* adj, uint32_t* flags, uint32_t* hdr, cudaStream_t st) {
+                               const void* ext, uint32_t* adj, uint32_t* flags, uint32_t* hdr, bool skip_empty,
+                               cudaStream_t st) {
   const int units = b.n_layers * b.n_seqs * n_kv_heads;
   CUtensorMap map, emap;
   if (!make_tensor_map_bf16(&map, Gamma, b, n_kv_heads, head_dim, 128)) return SPINDLEKV_CUDA;
@@ -501,6 +510,7 @@ spindlekv_status launch_sim_tc(const spindlekv_tensor& Gamma, const spindlekv_ba
   p.adj = adj;
   p.flags = flags;
   p.hdr = hdr;
+  p.skip_empty = skip_empty ? 1 : 0;
   dim3 grid(2 * ceil_div(b.max_len, 2 * kBM), units);   // whole pairs
   LaunchScope ls(KC_SIM, st);
   if (head_dim == 128) {

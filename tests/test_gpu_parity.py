@@ -373,17 +373,20 @@ def test_keep_everything_and_minimum_budget():
     run_and_check(wl)
 
 
-def _single_layer_codebook(gamma_np, theta, dtype="f32"):
-    """Runs the CodeBook path on one hand-made ``[l, d]`` array; returns outputs as numpy."""
+def _single_layer_codebook(gamma_np, theta, dtype="f32", keep_adjacency=True, poison=False):
+    """Runs the CodeBook path on one hand-made ``[l, d]`` array; returns outputs as numpy.  ``poison`` fills the
+    workspace with a byte pattern first (nothing in it may be taken for initialised)."""
     l, d = gamma_np.shape
     wl = synth.Workload("hand", 1, 1, 1, 1, d, dtype, 1, (l,), 1, 0.1, 0, "gauss", budget_tokens=float(l),
                         theta_k=theta, theta_v=theta)
-    p = _pass(wl, keep_adjacency=True)
+    p = _pass(wl, keep_adjacency=keep_adjacency)
+    if poison:
+        p.ws_codebook.fill_(0xA5)
     G = torch.from_numpy(gamma_np.astype(np.float32)).to(torch_dtype(wl)).cuda().reshape(1, 1, 1, l, d)
     p.codebook(G, "K")
     assert p.device_status()["codebook"][0] == 0
     o = p.cb["K"]
-    return (p.adj.cpu().numpy()[0], o["mag"].cpu().numpy()[0, 0], o["ref"].cpu().numpy()[0, 0],
+    return (p.adj.cpu().numpy()[0] if keep_adjacency else None, o["mag"].cpu().numpy()[0, 0], o["ref"].cpu().numpy()[0, 0],
             o["centre_idx"].cpu().numpy()[0, 0], int(o["n_entries"].cpu().numpy()[0, 0, 0]),
             o["C"].float().cpu().numpy()[0, 0, 0])
 
@@ -433,6 +436,28 @@ def test_tensor_core_similarity_at_awkward_lengths():
             g = round_to_dtype(g, "bf16")
             out = _single_layer_codebook(g, 0.95, "bf16")
             check_codebook_unit(g, 0.95, *out, 1e-2)
+
+
+def test_adjacency_in_a_poisoned_workspace_with_dense_rows():
+    # When the adjacency lives in the caller's workspace, chunks of it without a set bit are never written and
+    # must never be read: the workspace is filled with a byte pattern first.  Groups of 40 to 70 exactly parallel
+    # rows (power-of-two multiples: cosine 1) give rows with more than 32 neighbours, which are read as whole bit
+    # rows; everything else is far from the threshold, so the result is the checker's without any margin.
+    rng = np.random.default_rng(24)
+    from paper_2507_06517_b200.synth import round_to_dtype
+    for d, n in ((128, 1500), (64, 900)):
+        dirs = round_to_dtype(rng.standard_normal((40, d)).astype(np.float32), "bf16")
+        sizes = list(rng.integers(40, 71, size=6)) + [1] * 34
+        rows = []
+        for c, sz in enumerate(sizes):
+            rows += [dirs[c] * (2.0 ** int(e)) for e in rng.integers(-2, 3, size=sz)]
+        while len(rows) < n:
+            rows.append(round_to_dtype(rng.standard_normal(d).astype(np.float32), "bf16"))
+        g = np.stack(rows)[rng.permutation(len(rows))][:n]
+        out = _single_layer_codebook(g, 0.9, "bf16", keep_adjacency=False, poison=True)
+        check_codebook_unit(g, 0.9, *out, 1e-2)
+        ref = _single_layer_codebook(g, 0.9, "bf16")
+        assert np.array_equal(out[2], ref[2]) and np.array_equal(out[3], ref[3]) and out[4] == ref[4]
 
 
 def test_all_scores_tie_goes_to_lowest_positions():
