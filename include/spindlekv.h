@@ -173,7 +173,8 @@ spindlekv_status spindlekv_evict_deep_noalloc(const spindlekv_config* cfg, const
  *   adj_bits   device out, optional (NULL: kept in the workspace): the adjacency as a bit matrix,
  *              [n_layers*B*n_kv_heads][max_len][row_words] uint32, row_words = 4*ceil(max_len/128);
  *              bit (b & 31) of word b >> 5 of row a is G[a][b]; rows and words beyond a sequence's own
- *              length are not written
+ *              length are not written; 16-byte aligned, else INVALID_ARG.  With NULL the matrix in the
+ *              workspace is sparse: 64-column chunks of a row without a set bit may be left unwritten
  */
 spindlekv_status spindlekv_codebook_shallow(const spindlekv_config* cfg, const spindlekv_batch* batch,
                                             spindlekv_tensor Gamma, float theta,

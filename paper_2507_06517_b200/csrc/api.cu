@@ -183,6 +183,7 @@ spindlekv_status spindlekv_codebook_shallow(const spindlekv_config* cfg, const s
   if (batch->layer_lens && batch->cu_seqlens) return SPINDLEKV_INVALID_ARG;
   if (!tensor_ok(Gamma) || !mag || !ref || !centre_idx || !n_entries || !ws) return SPINDLEKV_INVALID_ARG;
   if (reinterpret_cast<uintptr_t>(ws) % 256) return SPINDLEKV_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(adj_bits) % 16) return SPINDLEKV_INVALID_ARG;   // rows are moved 16 bytes at a time
   if (cfg->head_dim != 64 && cfg->head_dim != 128) return SPINDLEKV_UNSUPPORTED;
   return codebook_shallow_impl(*cfg, *batch, Gamma, theta, mag, ref, centre_idx, n_entries, adj_bits, ws, ws_bytes,
                                (cudaStream_t)stream);

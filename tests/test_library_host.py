@@ -101,6 +101,7 @@ def test_device_entry_points_reject_bad_arguments_before_touching_the_gpu():
     assert lib.spindlekv_evict_deep(C.byref(cfg), C.byref(both), good, good, p, p, p, p, p, 1 << 20, None) == B.INVALID_ARG
     assert lib.spindlekv_codebook_shallow(C.byref(cfg), C.byref(both), good, 0.98, p, p, p, p, None, p, 1 << 20, None) == B.INVALID_ARG
     assert lib.spindlekv_codebook_shallow(C.byref(cfg), C.byref(batch), good, 0.98, None, p, p, p, None, p, 1 << 20, None) == B.INVALID_ARG
+    assert lib.spindlekv_codebook_shallow(C.byref(cfg), C.byref(batch), good, 0.98, p, p, p, p, C.c_void_p(260), p, 1 << 20, None) == B.INVALID_ARG  # adjacency not 16-byte aligned
     bad_dim = B.Config(4, 8, 2, 96, 32, 2, budget_tokens=300.0).c()
     assert lib.spindlekv_codebook_shallow(C.byref(bad_dim), C.byref(batch), good, 0.98, p, p, p, p, None, p, 1 << 20, None) == B.UNSUPPORTED
     assert lib.spindlekv_compact(C.byref(batch), 2, 128, good, None, p, None, good, None, None) == B.INVALID_ARG
