@@ -218,33 +218,54 @@ __global__ void __launch_bounds__(kWinThreads, 1) win_tc_kernel(const __grid_con
       ptx::tc_fence_after();
       const int key0 = i * kWinTile;
       const bool masked = key0 + kWinTile > l_c;     // window keys or the ragged end are in this tile
+      // 32 columns at a time; the next 32 are on their way from tensor memory while these are worked on
+      auto chunk_a = [&](const uint32_t (&raw)[32], int qb, int ch) {
+        float v[32];
+#pragma unroll
+        for (int e = 0; e < 32; ++e) v[e] = __uint_as_float(raw[e]);
+        if (masked) {
+          const int a0 = key0 + ch * 32;
+#pragma unroll
+          for (int e = 0; e < 32; ++e)
+            if (a0 + e > brow[qb]) v[e] = -CUDART_INF_F;   // causal: query b sees keys 0..b (b < l)
+        }
+        float mx = v[0];
+#pragma unroll
+        for (int e = 1; e < 32; ++e) mx = fmaxf(mx, v[e]);
+        const float m_new = fmaxf(rmax[qb], mx * c);
+        // a row that has seen no visible key yet keeps max = -inf and sum = 0 (exp2(-inf) = 0)
+        const float m_ref = m_new == -CUDART_INF_F ? 0.f : m_new;
+        float acc = rsum[qb] * ex2_approx(rmax[qb] - m_ref);
+#pragma unroll
+        for (int e = 0; e < 32; ++e) acc += ex2_approx(fmaf(v[e], c, -m_ref));
+        rsum[qb] = acc;
+        rmax[qb] = m_new;
+      };
+      constexpr int CPT = kWinTile / 32;   // chunks per 128 query rows
 #pragma unroll
       for (int qb = 0; qb < QB; ++qb) {
-#pragma unroll 1
-        for (int ch = 0; ch < kWinTile / 32; ++ch) {
-          uint32_t raw[32];
-          ptx::tmem_ld_32x32(tlane + qb * 128 + ch * 32, raw);
-          ptx::tmem_ld_wait(raw);
-          float v[32];
+        if constexpr (QB == 1) {
+          uint32_t r0[32], r1[32];
+          ptx::tmem_ld_32x32(tlane + qb * 128, r0);
+          // straight-line code: registers with a load in flight are not carried around a loop edge
 #pragma unroll
-          for (int e = 0; e < 32; ++e) v[e] = __uint_as_float(raw[e]);
-          if (masked) {
-            const int a0 = key0 + ch * 32;
-#pragma unroll
-            for (int e = 0; e < 32; ++e)
-              if (a0 + e > brow[qb]) v[e] = -CUDART_INF_F;   // causal: query b sees keys 0..b (b < l)
+          for (int ch = 0; ch < CPT; ch += 2) {
+            ptx::tmem_ld_wait(r0);
+            ptx::tmem_ld_32x32(tlane + qb * 128 + (ch + 1) * 32, r1);
+            chunk_a(r0, qb, ch);
+            ptx::tmem_ld_wait(r1);
+            if (ch + 2 < CPT) ptx::tmem_ld_32x32(tlane + qb * 128 + (ch + 2) * 32, r0);
+            chunk_a(r1, qb, ch + 1);
           }
-          float mx = v[0];
-#pragma unroll
-          for (int e = 1; e < 32; ++e) mx = fmaxf(mx, v[e]);
-          const float m_new = fmaxf(rmax[qb], mx * c);
-          // a row that has seen no visible key yet keeps max = -inf and sum = 0 (exp2(-inf) = 0)
-          const float m_ref = m_new == -CUDART_INF_F ? 0.f : m_new;
-          float acc = rsum[qb] * ex2_approx(rmax[qb] - m_ref);
-#pragma unroll
-          for (int e = 0; e < 32; ++e) acc += ex2_approx(fmaf(v[e], c, -m_ref));
-          rsum[qb] = acc;
-          rmax[qb] = m_new;
+        } else {
+          // two blocks of query rows: the unrolled form above would not fit the register file
+#pragma unroll 1
+          for (int ch = 0; ch < CPT; ++ch) {
+            uint32_t raw[32];
+            ptx::tmem_ld_32x32(tlane + qb * 128 + ch * 32, raw);
+            ptx::tmem_ld_wait(raw);
+            chunk_a(raw, qb, ch);
+          }
         }
       }
       ptx::tc_fence_before();
@@ -288,15 +309,27 @@ __global__ void __launch_bounds__(kWinThreads, 1) win_tc_kernel(const __grid_con
       if (!__all_sync(0xffffffffu, ptx::mbar_wait(acc_full + eg, (i >> 1) & 1, abort_flag))) break;
       ptx::tc_fence_after();
       float colsum = 0.f;
-#pragma unroll 1
-      for (int ch = 0; ch < NQ / 32; ++ch) {
-        uint32_t raw[32];
-        ptx::tmem_ld_32x32(tlane + ch * 32, raw);
-        ptx::tmem_ld_wait(raw);
+      auto chunk_b = [&](const uint32_t (&raw)[32]) {
         float part = 0.f;
 #pragma unroll
         for (int e = 0; e < 32; ++e) part += ex2_approx(__uint_as_float(raw[e]) * c);
         colsum += part;
+      };
+      // groups of four chunks in straight-line code: registers with a load in flight are not carried around a
+      // loop edge
+#pragma unroll 1
+      for (int g = 0; g < NQ / 128; ++g) {
+        uint32_t r0[32], r1[32];
+        ptx::tmem_ld_32x32(tlane + g * 128, r0);
+#pragma unroll
+        for (int ch = 0; ch < 4; ch += 2) {
+          ptx::tmem_ld_wait(r0);
+          ptx::tmem_ld_32x32(tlane + g * 128 + (ch + 1) * 32, r1);
+          chunk_b(r0);
+          ptx::tmem_ld_wait(r1);
+          if (ch + 2 < 4) ptx::tmem_ld_32x32(tlane + g * 128 + (ch + 2) * 32, r0);
+          chunk_b(r1);
+        }
       }
       ptx::tc_fence_before();
       __syncwarp();
