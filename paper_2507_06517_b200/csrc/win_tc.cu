@@ -84,6 +84,10 @@ __global__ void __launch_bounds__(kWinThreads, 1) win_tc_kernel(const __grid_con
   const int layer = ls / p.batch.n_seqs;
   const int l = seq_len(p.batch, layer, s, j);
   const int l_c = l - p.window;
+  // accumulator ring in tensor memory: four stages of 128 columns when one block of query rows is held, else two
+  // of 256; the epilogue group of tile i is i & 1, so a stage always belongs to one group
+  constexpr int AS = QB == 1 ? 4 : 2;
+  constexpr int AS_COLS = 512 / AS;
   const int T = (l + kWinTile - 1) / kWinTile;      // tiles of pass A (all keys)
   const int Tc = (l_c + kWinTile - 1) / kWinTile;   // tiles of pass B (context keys)
 
@@ -98,9 +102,9 @@ __global__ void __launch_bounds__(kWinThreads, 1) win_tc_kernel(const __grid_con
   uint64_t* q_full = bars + 0;
   uint64_t* k_full = bars + 1;                 // [kWinStages]
   uint64_t* k_empty = bars + 1 + kWinStages;   // [kWinStages]
-  uint64_t* acc_full = bars + 1 + 2 * kWinStages;   // [2]
-  uint64_t* acc_empty = acc_full + 2;               // [2]
-  uint64_t* ext_full = acc_empty + 2;
+  uint64_t* acc_full = bars + 1 + 2 * kWinStages;   // [AS]
+  uint64_t* acc_empty = acc_full + 4;               // [AS]
+  uint64_t* ext_full = acc_empty + 4;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ext_full + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(ext_full + 2);
 
@@ -108,7 +112,7 @@ __global__ void __launch_bounds__(kWinThreads, 1) win_tc_kernel(const __grid_con
   if (threadIdx.x == 0) {
     ptx::mbar_init(q_full, 1);
     for (int i = 0; i < kWinStages; ++i) { ptx::mbar_init(k_full + i, 1); ptx::mbar_init(k_empty + i, 1); }
-    for (int i = 0; i < 2; ++i) { ptx::mbar_init(acc_full + i, 1); ptx::mbar_init(acc_empty + i, kWinEpiWarps / 2); }
+    for (int i = 0; i < AS; ++i) { ptx::mbar_init(acc_full + i, 1); ptx::mbar_init(acc_empty + i, kWinEpiWarps / 2); }
     ptx::mbar_init(ext_full, kWinEpiWarps);
     *abort_flag = 0;
     ptx::fence_barrier_init();
@@ -160,9 +164,9 @@ __global__ void __launch_bounds__(kWinThreads, 1) win_tc_kernel(const __grid_con
       bool ok = ptx::mbar_wait(q_full, 0, abort_flag);
       int i = 0;
       for (; ok && i < T; ++i) {
-        const int st = i % kWinStages, as = i & 1;
+        const int st = i % kWinStages, as = i % AS;
         if (!ptx::mbar_wait(k_full + st, (i / kWinStages) & 1, abort_flag)) { ok = false; break; }
-        if (!ptx::mbar_wait(acc_empty + as, ((i >> 1) & 1) ^ 1, abort_flag)) { ok = false; break; }
+        if (!ptx::mbar_wait(acc_empty + as, ((i / AS) & 1) ^ 1, abort_flag)) { ok = false; break; }
         ptx::tc_fence_after();
         const uint32_t k_addr = ptx::smem_u32(sK + st * L::K_BYTES);
 #pragma unroll
@@ -172,7 +176,7 @@ __global__ void __launch_bounds__(kWinThreads, 1) win_tc_kernel(const __grid_con
             const int kh = k >> 2, kk = k & 3;
             const uint64_t da = ptx::smem_desc_sw128(q_addr + kh * NQ * 128 + qb * 128 * 128 + kk * 32);
             const uint64_t db = ptx::smem_desc_sw128(k_addr + kh * kWinTile * 128 + kk * 32);
-            ptx::umma_bf16(tmem_base + as * 256 + qb * 128, da, db, idesc_a, k > 0 ? 1u : 0u);
+            ptx::umma_bf16(tmem_base + as * AS_COLS + qb * 128, da, db, idesc_a, k > 0 ? 1u : 0u);
           }
         ptx::umma_commit(k_empty + st);
         ptx::umma_commit(acc_full + as);
@@ -181,9 +185,9 @@ __global__ void __launch_bounds__(kWinThreads, 1) win_tc_kernel(const __grid_con
       const uint64_t dea = ptx::smem_desc_interleaved(ptx::smem_u32(sEA), kWinTile * 16, 128);
       const uint64_t deb = ptx::smem_desc_interleaved(ptx::smem_u32(sEB), NQ * 16, 128);
       for (; ok && i < T + Tc; ++i) {
-        const int st = i % kWinStages, as = i & 1;
+        const int st = i % kWinStages, as = i % AS;
         if (!ptx::mbar_wait(k_full + st, (i / kWinStages) & 1, abort_flag)) break;
-        if (!ptx::mbar_wait(acc_empty + as, ((i >> 1) & 1) ^ 1, abort_flag)) break;
+        if (!ptx::mbar_wait(acc_empty + as, ((i / AS) & 1) ^ 1, abort_flag)) break;
         ptx::tc_fence_after();
         const uint32_t k_addr = ptx::smem_u32(sK + st * L::K_BYTES);
 #pragma unroll
@@ -191,9 +195,9 @@ __global__ void __launch_bounds__(kWinThreads, 1) win_tc_kernel(const __grid_con
           const int kh = k >> 2, kk = k & 3;
           const uint64_t da = ptx::smem_desc_sw128(k_addr + kh * kWinTile * 128 + kk * 32);
           const uint64_t db = ptx::smem_desc_sw128(q_addr + kh * NQ * 128 + kk * 32);
-          ptx::umma_bf16(tmem_base + as * 256, da, db, idesc_b, k > 0 ? 1u : 0u);
+          ptx::umma_bf16(tmem_base + as * AS_COLS, da, db, idesc_b, k > 0 ? 1u : 0u);
         }
-        ptx::umma_bf16(tmem_base + as * 256, dea, deb, idesc_b, 1u);   // - L_r on column r
+        ptx::umma_bf16(tmem_base + as * AS_COLS, dea, deb, idesc_b, 1u);   // - L_r on column r
         ptx::umma_commit(k_empty + st);
         ptx::umma_commit(acc_full + as);
       }
@@ -201,7 +205,7 @@ __global__ void __launch_bounds__(kWinThreads, 1) win_tc_kernel(const __grid_con
   } else {
     const int q = warp & 3;                 // TMEM lane quarter of this warp
     const int eg = (warp - 2) >> 2;         // epilogue group = TMEM stage it serves
-    const uint32_t tlane = tmem_base + ((uint32_t)(q * 32) << 16) + eg * 256;
+    const uint32_t tquarter = tmem_base + ((uint32_t)(q * 32) << 16);
     const float c = p.c;
     // ---- pass A: running (max, sum) of this thread's query rows, base-2 domain ----
     float rmax[QB], rsum[QB];
@@ -214,7 +218,9 @@ __global__ void __launch_bounds__(kWinThreads, 1) win_tc_kernel(const __grid_con
     }
     bool ok = true;
     for (int i = eg; i < T; i += 2) {
-      if (!__all_sync(0xffffffffu, ptx::mbar_wait(acc_full + eg, (i >> 1) & 1, abort_flag))) { ok = false; break; }
+      const int as = i % AS;
+      const uint32_t tlane = tquarter + as * AS_COLS;
+      if (!__all_sync(0xffffffffu, ptx::mbar_wait(acc_full + as, (i / AS) & 1, abort_flag))) { ok = false; break; }
       ptx::tc_fence_after();
       const int key0 = i * kWinTile;
       const bool masked = key0 + kWinTile > l_c;     // window keys or the ragged end are in this tile
@@ -270,7 +276,7 @@ __global__ void __launch_bounds__(kWinThreads, 1) win_tc_kernel(const __grid_con
       }
       ptx::tc_fence_before();
       __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(acc_empty + eg);
+      if (lane == 0) ptx::mbar_arrive(acc_empty + as);
     }
     // ---- merge the two groups' statistics; write the -L operand of pass B ----
     if (eg == 1) {
@@ -306,7 +312,9 @@ __global__ void __launch_bounds__(kWinThreads, 1) win_tc_kernel(const __grid_con
     float* out = p.scores + ((int64_t)layer * p.n_kv_heads + j) * p.batch.total_len + tok_base(p.batch, s);
     // the first pass-B item whose stage belongs to this group
     for (int i = T + ((T & 1) ^ eg); ok && i < T + Tc; i += 2) {
-      if (!__all_sync(0xffffffffu, ptx::mbar_wait(acc_full + eg, (i >> 1) & 1, abort_flag))) break;
+      const int as = i % AS;
+      const uint32_t tlane = tquarter + as * AS_COLS;
+      if (!__all_sync(0xffffffffu, ptx::mbar_wait(acc_full + as, (i / AS) & 1, abort_flag))) break;
       ptx::tc_fence_after();
       float colsum = 0.f;
       auto chunk_b = [&](const uint32_t (&raw)[32]) {
@@ -333,7 +341,7 @@ __global__ void __launch_bounds__(kWinThreads, 1) win_tc_kernel(const __grid_con
       }
       ptx::tc_fence_before();
       __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(acc_empty + eg);
+      if (lane == 0) ptx::mbar_arrive(acc_empty + as);
       const int a = (i - T) * kWinTile + q * 32 + lane;
       if (a < l_c) {
         float v = colsum * inv_hn;
