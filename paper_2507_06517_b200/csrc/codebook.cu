@@ -213,8 +213,9 @@ __device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long v)
 
 // ---- neighbour lists ------------------------------------------------------------------------------
 // One thread per row.  The similarity kernel left one bit per (row, 64-column chunk) that says
-// whether the chunk may hold a set bit (a word holds the bits of 32 rows: a warp reads the words of 32
-// chunks and transposes them); only those chunks of the bit row are read.  Written per row:
+// whether the chunk may hold a set bit (a word holds the bits of 32 rows: a warp reads the words of 256
+// chunks, eight per lane, and transposes them into per-row occupancy words); only those chunks of the bit
+// row are read, several at a time.  Written per row:
 // the initial degree (Eq. (10)) and key, and, for rows with at most kEll neighbours (the row itself
 // not counted), the ascending list of those neighbours, stored entry-major (`ell[k][row]`) so that
 // the threads of a warp read consecutive words.  Rows with more neighbours keep using their bit row
