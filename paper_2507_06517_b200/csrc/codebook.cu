@@ -225,7 +225,7 @@ constexpr int kEll = 32;
 constexpr int kChunkBatch = 8;    // occupied chunks of a row fetched together
 constexpr int kFlagGroup = 8;     // flag words fetched together (256 chunks = 16384 columns)
 
-__global__ void __launch_bounds__(256) extract_kernel(CodebookParams p) {
+__global__ void __launch_bounds__(256, 5) extract_kernel(CodebookParams p) {
   const int lane = threadIdx.x & 31;
   const int RW = p.row_words, NP = RW * 32, NC = RW >> 1, ML = p.batch.max_len;
   const int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;   // over units x padded rows
