@@ -37,8 +37,14 @@ struct WinTcParams {
 
 constexpr int kWinTile = 128;                 // keys per tile
 constexpr int kWinStages = 4;                 // K ring
-constexpr int kWinEpiWarps = 8;
-constexpr int kWinThreads = 32 * (2 + kWinEpiWarps);
+// Epilogue groups of four warps (one per lane quarter of tensor memory); group g takes the tiles i with i % G == g.
+// With one block of query rows an accumulator is 128 columns wide: four stages, four groups.  With two blocks it is
+// 256 columns wide: two stages, two groups.
+template <int QB> struct WinShape {
+  static constexpr int G = QB == 1 ? 4 : 2;
+  static constexpr int EPI_WARPS = 4 * G;
+  static constexpr int THREADS = 32 * (2 + EPI_WARPS);
+};
 
 template <int D, int QB>
 struct WinSmem {
@@ -48,7 +54,7 @@ struct WinSmem {
   static constexpr int K_BYTES = KH * kWinTile * 128;
   static constexpr int EA_BYTES = 2 * kWinTile * 16;  // ones operand, two 16-byte column chunks
   static constexpr int EB_BYTES = 2 * NQ * 16;        // -L operand
-  static constexpr int ST_BYTES = NQ * 8;             // (max, sum) of the second epilogue group
+  static constexpr int ST_BYTES = (WinShape<QB>::G - 1) * NQ * 8;   // (max, sum) of the epilogue groups after the first
   static constexpr int OFF_K = Q_BYTES;
   static constexpr int OFF_EA = OFF_K + kWinStages * K_BYTES;
   static constexpr int OFF_EB = OFF_EA + EA_BYTES;
@@ -72,7 +78,7 @@ __device__ __forceinline__ float lg2_approx(float x) {
 }
 
 template <int D, int QB>
-__global__ void __launch_bounds__(kWinThreads, 1) win_tc_kernel(const __grid_constant__ CUtensorMap kmap,
+__global__ void __launch_bounds__(WinShape<QB>::THREADS, 1) win_tc_kernel(const __grid_constant__ CUtensorMap kmap,
                                                                 const __grid_constant__ CUtensorMap qmap,
                                                                 WinTcParams p) {
   using L = WinSmem<D, QB>;
@@ -86,8 +92,11 @@ __global__ void __launch_bounds__(kWinThreads, 1) win_tc_kernel(const __grid_con
   const int l_c = l - p.window;
   // accumulator ring in tensor memory: four stages of 128 columns when one block of query rows is held, else two
   // of 256; the epilogue group of tile i is i & 1, so a stage always belongs to one group
-  constexpr int AS = QB == 1 ? 4 : 2;
+  constexpr int AS = WinShape<QB>::G;
   constexpr int AS_COLS = 512 / AS;
+  constexpr int G = WinShape<QB>::G;
+  constexpr int kWinEpiWarps = WinShape<QB>::EPI_WARPS;
+  constexpr int kWinThreads = WinShape<QB>::THREADS;
   const int T = (l + kWinTile - 1) / kWinTile;      // tiles of pass A (all keys)
   const int Tc = (l_c + kWinTile - 1) / kWinTile;   // tiles of pass B (context keys)
 
@@ -112,7 +121,7 @@ __global__ void __launch_bounds__(kWinThreads, 1) win_tc_kernel(const __grid_con
   if (threadIdx.x == 0) {
     ptx::mbar_init(q_full, 1);
     for (int i = 0; i < kWinStages; ++i) { ptx::mbar_init(k_full + i, 1); ptx::mbar_init(k_empty + i, 1); }
-    for (int i = 0; i < AS; ++i) { ptx::mbar_init(acc_full + i, 1); ptx::mbar_init(acc_empty + i, kWinEpiWarps / 2); }
+    for (int i = 0; i < AS; ++i) { ptx::mbar_init(acc_full + i, 1); ptx::mbar_init(acc_empty + i, 4); }
     ptx::mbar_init(ext_full, kWinEpiWarps);
     *abort_flag = 0;
     ptx::fence_barrier_init();
@@ -217,7 +226,7 @@ __global__ void __launch_bounds__(kWinThreads, 1) win_tc_kernel(const __grid_con
       brow[qb] = l_c + (qb * 128 + q * 32 + lane) % p.window;
     }
     bool ok = true;
-    for (int i = eg; i < T; i += 2) {
+    for (int i = eg; i < T; i += G) {
       const int as = i % AS;
       const uint32_t tlane = tquarter + as * AS_COLS;
       if (!__all_sync(0xffffffffu, ptx::mbar_wait(acc_full + as, (i / AS) & 1, abort_flag))) { ok = false; break; }
@@ -250,47 +259,40 @@ __global__ void __launch_bounds__(kWinThreads, 1) win_tc_kernel(const __grid_con
       constexpr int CPT = kWinTile / 32;   // chunks per 128 query rows
 #pragma unroll
       for (int qb = 0; qb < QB; ++qb) {
-        if constexpr (QB == 1) {
-          uint32_t r0[32], r1[32];
-          ptx::tmem_ld_32x32(tlane + qb * 128, r0);
-          // straight-line code: registers with a load in flight are not carried around a loop edge
-#pragma unroll
-          for (int ch = 0; ch < CPT; ch += 2) {
-            ptx::tmem_ld_wait(r0);
-            ptx::tmem_ld_32x32(tlane + qb * 128 + (ch + 1) * 32, r1);
-            chunk_a(r0, qb, ch);
-            ptx::tmem_ld_wait(r1);
-            if (ch + 2 < CPT) ptx::tmem_ld_32x32(tlane + qb * 128 + (ch + 2) * 32, r0);
-            chunk_a(r1, qb, ch + 1);
-          }
-        } else {
-          // two blocks of query rows: the unrolled form above would not fit the register file
 #pragma unroll 1
-          for (int ch = 0; ch < CPT; ++ch) {
-            uint32_t raw[32];
-            ptx::tmem_ld_32x32(tlane + qb * 128 + ch * 32, raw);
-            ptx::tmem_ld_wait(raw);
-            chunk_a(raw, qb, ch);
-          }
+        for (int ch = 0; ch < CPT; ++ch) {
+          uint32_t raw[32];
+          ptx::tmem_ld_32x32(tlane + qb * 128 + ch * 32, raw);
+          ptx::tmem_ld_wait(raw);
+          chunk_a(raw, qb, ch);
         }
       }
       ptx::tc_fence_before();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(acc_empty + as);
     }
-    // ---- merge the two groups' statistics; write the -L operand of pass B ----
-    if (eg == 1) {
+    // ---- merge the groups' statistics; write the -L operand of pass B ----
+    if (eg > 0) {
 #pragma unroll
-      for (int qb = 0; qb < QB; ++qb) sST[qb * 128 + q * 32 + lane] = make_float2(rmax[qb], rsum[qb]);
+      for (int qb = 0; qb < QB; ++qb) sST[(eg - 1) * NQ + qb * 128 + q * 32 + lane] = make_float2(rmax[qb], rsum[qb]);
     }
     asm volatile("bar.sync 1, %0;" ::"n"(32 * kWinEpiWarps) : "memory");
     if (eg == 0) {
 #pragma unroll
       for (int qb = 0; qb < QB; ++qb) {
         const int r = qb * 128 + q * 32 + lane;
-        const float2 o = sST[r];
-        const float m = fmaxf(rmax[qb], o.x);
-        const float sum = rsum[qb] * ex2_approx(rmax[qb] - m) + o.y * ex2_approx(o.x - m);
+        float m = rmax[qb];
+        float2 o[G - 1];
+#pragma unroll
+        for (int g = 0; g < G - 1; ++g) {
+          o[g] = sST[g * NQ + r];
+          m = fmaxf(m, o[g].x);
+        }
+        // a group that saw no visible key of this row has (max, sum) = (-inf, 0): its term is 0 * exp2(-inf) = 0
+        const float m_ref = m == -CUDART_INF_F ? 0.f : m;
+        float sum = rsum[qb] * ex2_approx(rmax[qb] - m_ref);
+#pragma unroll
+        for (int g = 0; g < G - 1; ++g) sum += o[g].y * ex2_approx(o[g].x - m_ref);
         // rows beyond M (padding, or heads of the next group) get a huge L: their weights vanish
         float Lr = r < p.m_rows ? (m + lg2_approx(sum)) / c : 1e30f;
         uint32_t pc[3];
@@ -311,7 +313,7 @@ __global__ void __launch_bounds__(kWinThreads, 1) win_tc_kernel(const __grid_con
     const float inv_hn = 1.0f / (float)p.h_n;
     float* out = p.scores + ((int64_t)layer * p.n_kv_heads + j) * p.batch.total_len + tok_base(p.batch, s);
     // the first pass-B item whose stage belongs to this group
-    for (int i = T + ((T & 1) ^ eg); ok && i < T + Tc; i += 2) {
+    for (int i = T + ((eg - T % G + G) % G); ok && i < T + Tc; i += G) {
       const int as = i % AS;
       const uint32_t tlane = tquarter + as * AS_COLS;
       if (!__all_sync(0xffffffffu, ptx::mbar_wait(acc_full + as, (i / AS) & 1, abort_flag))) break;
@@ -323,20 +325,31 @@ __global__ void __launch_bounds__(kWinThreads, 1) win_tc_kernel(const __grid_con
         for (int e = 0; e < 32; ++e) part += ex2_approx(__uint_as_float(raw[e]) * c);
         colsum += part;
       };
-      // groups of four chunks in straight-line code: registers with a load in flight are not carried around a
-      // loop edge
+      if constexpr (QB == 1) {
+        // eighteen warps share the register file: one load at a time, the other warps of the scheduler fill in
 #pragma unroll 1
-      for (int g = 0; g < NQ / 128; ++g) {
-        uint32_t r0[32], r1[32];
-        ptx::tmem_ld_32x32(tlane + g * 128, r0);
+        for (int ch = 0; ch < NQ / 32; ++ch) {
+          uint32_t raw[32];
+          ptx::tmem_ld_32x32(tlane + ch * 32, raw);
+          ptx::tmem_ld_wait(raw);
+          chunk_b(raw);
+        }
+      } else {
+        // groups of four chunks in straight-line code, the next 32 columns on their way while these are worked on:
+        // registers with a load in flight are not carried around a loop edge
+#pragma unroll 1
+        for (int g = 0; g < NQ / 128; ++g) {
+          uint32_t r0[32], r1[32];
+          ptx::tmem_ld_32x32(tlane + g * 128, r0);
 #pragma unroll
-        for (int ch = 0; ch < 4; ch += 2) {
-          ptx::tmem_ld_wait(r0);
-          ptx::tmem_ld_32x32(tlane + g * 128 + (ch + 1) * 32, r1);
-          chunk_b(r0);
-          ptx::tmem_ld_wait(r1);
-          if (ch + 2 < 4) ptx::tmem_ld_32x32(tlane + g * 128 + (ch + 2) * 32, r0);
-          chunk_b(r1);
+          for (int ch = 0; ch < 4; ch += 2) {
+            ptx::tmem_ld_wait(r0);
+            ptx::tmem_ld_32x32(tlane + g * 128 + (ch + 1) * 32, r1);
+            chunk_b(r0);
+            ptx::tmem_ld_wait(r1);
+            if (ch + 2 < 4) ptx::tmem_ld_32x32(tlane + g * 128 + (ch + 2) * 32, r0);
+            chunk_b(r1);
+          }
         }
       }
       ptx::tc_fence_before();
@@ -395,7 +408,7 @@ static spindlekv_status launch_one(const CUtensorMap& kmap, const CUtensorMap& q
       return SPINDLEKV_CUDA;
     once.done[dev] = true;
   }
-  win_tc_kernel<D, QB><<<units, kWinThreads, L::TOTAL, st>>>(kmap, qmap, p);
+  win_tc_kernel<D, QB><<<units, WinShape<QB>::THREADS, L::TOTAL, st>>>(kmap, qmap, p);
   return SPINDLEKV_OK;
 }
 
