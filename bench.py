@@ -391,6 +391,16 @@ def run_native(args, wl):
             gbs = nbytes / (kernels[k]["ms_per_step"] * 1e-3) / 1e9
             kernels[k].update({"bound": "hbm", "algorithmic_bytes": nbytes, "achieved_gbs": gbs,
                                "frac_of_hbm_peak": gbs / pk["hbm_gbs"]})
+    if nd and "window_score" in kernels and kernels["window_score"]["ms_per_step"] > 0 and wl.dtype == "bf16":
+        # the window-score kernel takes one exponential per (query row, key) in each of its two passes; the
+        # special-function units deliver 16 per clock and SM (148 SMs, the SM clock sampled during the run)
+        h_n = wl.n_q_heads // wl.n_kv_heads
+        exps = 2.0 * h_n * wl.window * tok * Hk * nd
+        mhz = (clocks or {}).get("sm_mhz") or (clocks or {}).get("sm_max_mhz") or 1965.0
+        peak = 16.0 * 148 * mhz * 1e6
+        rate = exps / (kernels["window_score"]["ms_per_step"] * 1e-3)
+        kernels["window_score"]["exp_unit"] = {"exponentials_per_step": exps, "achieved_per_s": rate,
+                                               "peak_per_s": peak, "frac": rate / peak, "sm_mhz": mhz}
     roof = None
     if p.n_shallow and kt["similarity"][1]:
         sim_ms, sim_n = kt["similarity"]
