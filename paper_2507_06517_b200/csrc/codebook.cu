@@ -299,8 +299,8 @@ __global__ void __launch_bounds__(256, 5) extract_kernel(CodebookParams p) {
     p.deg[idx] = cnt;
     p.key[idx] = ((unsigned long long)(uint32_t)cnt << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)u);
     p.ell_cnt[idx] = cnt - 1 <= kEll ? cnt - 1 : -1;
+    p.pickdeg[idx] = cnt == 1 ? 1 : -1;   // -1: not a centre (until the greedy cover picks it)
     if (cnt == 1) {
-      p.pickdeg[idx] = 1;
       p.owner[idx] = u;
     } else {
       live = true;
@@ -867,7 +867,6 @@ spindlekv_status codebook_shallow_impl(const spindlekv_config& cfg, const spindl
   p.centre_idx = centre_idx;
   p.n_entries = n_entries;
   if (cudaMemsetAsync(w, 0, kHeaderBytes, st) != cudaSuccess) return SPINDLEKV_CUDA;
-  if (cudaMemsetAsync(p.pickdeg, 0xFF, (size_t)units * b.max_len * 4, st) != cudaSuccess) return SPINDLEKV_CUDA;
   const bool bf = Gamma.dtype == SPINDLEKV_BF16;
   const bool tc = bf && sim_tc_available();   // bf16: tensor-core similarity (TMA + tcgen05)
   p.ext = tc ? reinterpret_cast<__nv_bfloat16*>(w + L.ext) : nullptr;
