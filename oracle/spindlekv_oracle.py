@@ -254,36 +254,45 @@ def adjacency(S: np.ndarray, theta: float) -> np.ndarray:
     return G
 
 
-def codebook_alg1_dense(G: np.ndarray) -> Tuple[np.ndarray, np.ndarray]:
-    """Algorithm 1's loop, statement by statement, on a dense 0/1 matrix.
+def codebook_cover_small(G: np.ndarray) -> Tuple[np.ndarray, np.ndarray]:
+    """Eq. (10)-(13) written out on explicit node lists, for small ``N`` only.
 
-    Degrees are recomputed as row sums each round (Eq. (10)), the centre is
-    the first arg-max (Eq. (11)), all of its current neighbours take the new
-    entry's number (Eq. (12)), and the graph is cleaned with the outer product
-    of the negated centre row (Eq. (13)), until ``G`` is all zero.
-    Cubic cost: for small ``N`` only.  Returns ``(centres, ref)``.
+    Nothing is kept between picks: for every pick the degree of each remaining node is counted
+    afresh by going through all remaining nodes (Eq. (10), the node itself included because the
+    diagonal of ``G`` is 1); the remaining node with the largest count, the lowest index among
+    equals, becomes a centre (Eq. (11)); the remaining nodes similar to it, itself among them, take
+    the new entry's number (Eq. (12)) and leave the graph (Eq. (13)).  Work per pick is quadratic in
+    the number of remaining nodes.  This form shares no bookkeeping with ``codebook_greedy`` and
+    serves as its cross-check.  Returns ``(centres, ref)``.
     """
-    G = np.array(G, dtype=np.int64)
+    G = np.asarray(G, dtype=bool)
     n = G.shape[0]
-    ref = -np.ones(n, dtype=np.int32)
+    remaining = list(range(n))
+    ref = [-1] * n
     centres: List[int] = []
-    while G.any():
-        s = G.sum(axis=1)
-        iota = int(np.argmax(s))
-        centres.append(iota)
-        eta = np.argwhere(G[iota] == 1)[:, 0]
-        ref[eta] = len(centres) - 1
-        not_row = 1 - G[iota]
-        mask = np.matmul(not_row[:, None], not_row[None, :])
-        G = G & mask
-    return np.array(centres, dtype=np.int32), ref
+    while remaining:
+        chosen, chosen_degree = -1, -1
+        for a in remaining:                      # ascending: the first largest count is the lowest index
+            count = 0
+            for b in remaining:
+                if a == b or G[a, b]:
+                    count += 1
+            if count > chosen_degree:
+                chosen, chosen_degree = a, count
+        members = [b for b in remaining if b == chosen or G[chosen, b]]
+        for b in members:
+            ref[b] = len(centres)
+        centres.append(chosen)
+        gone = set(members)
+        remaining = [b for b in remaining if b not in gone]
+    return np.array(centres, dtype=np.int32), np.array(ref, dtype=np.int32)
 
 
 def codebook_greedy(G: np.ndarray) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
     """Eq. (10)-(13) on a set of live nodes, usable at full sequence length.
 
-    The same steps as Algorithm 1, in the same order; the only difference is
-    bookkeeping: removed nodes leave a ``live`` set instead of having their
+    The steps of Eq. (10)-(13) in their order; what differs from the small-N form above is
+    bookkeeping only: removed nodes leave a ``live`` set instead of having their
     rows and columns zeroed, and the degree vector of Eq. (10) is kept current
     by subtracting, for every removed node, its row of ``G`` (``G`` is
     symmetric, so that row is exactly what the node contributed to the other

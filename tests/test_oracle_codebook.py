@@ -31,7 +31,7 @@ def _hand_graphs():
 
 @pytest.mark.parametrize("name,G,centres,ref", _hand_graphs(), ids=[g[0] for g in _hand_graphs()])
 def test_hand_worked_graphs(name, G, centres, ref):
-    for fn in (O.codebook_alg1_dense, O.codebook_greedy):
+    for fn in (O.codebook_cover_small, O.codebook_greedy):
         res = fn(G)
         assert list(res[0]) == centres
         assert list(res[1]) == ref
@@ -78,7 +78,7 @@ def test_all_graphs_up_to_five_nodes():
                 if bits >> e & 1:
                     G[a, b] = G[b, a] = True
             want = _set_greedy(_adj_sets(G))
-            c1, r1 = O.codebook_alg1_dense(G)
+            c1, r1 = O.codebook_cover_small(G)
             c2, r2, d2 = O.codebook_greedy(G)
             assert list(c1) == want[0] and list(r1) == want[1]
             assert list(c2) == want[0] and list(r2) == want[1]
@@ -92,7 +92,7 @@ def test_random_graphs_three_ways(n, p):
         up = np.triu(rng.random((n, n)) < p, k=1)
         G = up | up.T | np.eye(n, dtype=bool)
         want = _set_greedy(_adj_sets(G))
-        c1, r1 = O.codebook_alg1_dense(G)
+        c1, r1 = O.codebook_cover_small(G)
         c2, r2, d2 = O.codebook_greedy(G)
         assert list(c1) == want[0] and list(r1) == want[1]
         assert list(c2) == want[0] and list(r2) == want[1]
@@ -181,8 +181,8 @@ def test_coverage_reconstruction_and_codebook_norms():
     assert np.all(cos[~own] > theta)  # every replaced token meets the similarity criterion
     np.testing.assert_allclose(cos[own], 1.0, rtol=1e-12)
     _check_invariants(r["G"], r["centres"], r["ref"], r["pick_degree"])
-    # dense transcription agrees at this size as well
-    c1, r1 = O.codebook_alg1_dense(r["G"])
+    # the small-N form, which recounts every degree for every pick, agrees at this size as well
+    c1, r1 = O.codebook_cover_small(r["G"])
     assert np.array_equal(c1, r["centres"]) and np.array_equal(r1, r["ref"])
 
 
