@@ -141,15 +141,24 @@ spindlekv_status spindlekv_evict_deep(const spindlekv_config* cfg, const spindle
  * scratch the kernels need is a fixed array of SPINDLEKV_NOALLOC_SCRATCH_BYTES inside the library
  * image (present on every GPU that loads the library, until the process exits), so no workspace is
  * passed and the function never calls cudaMalloc/cudaFree or any allocating routine.
- *   - Arguments as spindlekv_evict_deep, minus the workspace.
- *   - Returns WORKSPACE_TOO_SMALL when spindlekv_workspace_bytes(cfg, batch, SPINDLEKV_WS_EVICT) exceeds
- *     SPINDLEKV_NOALLOC_SCRATCH_BYTES (e.g. more than about four 8B-shaped layers of 16k tokens at once):
- *     split the layers over several calls.
+ *   - Arguments as spindlekv_evict_deep, minus the workspace, and checked in the same way (same
+ *     status codes for null pointers, misaligned bases, strides that are not multiples of 8, unknown
+ *     dtypes, inconsistent batches) before anything is enqueued.
+ *   - Returns WORKSPACE_TOO_SMALL when the scratch this call would really use exceeds
+ *     SPINDLEKV_NOALLOC_SCRATCH_BYTES: split the layers over several calls.  bf16 inputs whose window
+ *     is 16, 32, 64 or 128 with at most 256 query rows per KV head run on the tensor-core kernel,
+ *     which needs the status block only, so any batch fits; other inputs need
+ *     spindlekv_workspace_bytes(cfg, batch, SPINDLEKV_WS_EVICT), e.g. about four fp32 layers of
+ *     8 x 16k tokens.
  *   - The first call on each device looks up the array's device address (with that device current);
- *     make that first call outside any stream capture.
+ *     make that first call outside any stream capture.  With lazy module loading the same first call
+ *     is what makes the array resident on the device: let it happen before the host's own pool
+ *     claims the rest of the memory.
  *   - All calls share the one array, which keeps the previous call's contents; what must start at
  *     zero is cleared by the call itself.  Two calls whose kernels overlap on the GPU (different
  *     streams, no ordering between them) race on it: order them.
+ *   - The device status word of the last call (a bounded wait that gave up) is read with
+ *     spindlekv_poll_status(NULL, ...) after synchronising the stream, with the same device current.
  */
 #define SPINDLEKV_NOALLOC_SCRATCH_BYTES (8 * 1024 * 1024)
 spindlekv_status spindlekv_evict_deep_noalloc(const spindlekv_config* cfg, const spindlekv_batch* batch,
@@ -265,6 +274,9 @@ spindlekv_status spindlekv_reconstruct(const spindlekv_batch* batch, int32_t n_h
 
 /*
  * Reads the device status word of a workspace (blocking copy; synchronise the stream first).
+ *   ws            the workspace of the call in question; NULL: the built-in scratch that
+ *                 spindlekv_evict_deep_noalloc uses on the current device (INVALID_ARG before the first
+ *                 such call on this device)
  *   device_status host out: SPINDLEKV_OK or SPINDLEKV_TIMEOUT
  *   detail        host out, optional [4]: {greedy rounds used, live tokens left, 0, 0}
  */

@@ -206,8 +206,10 @@ def spindlekv_evict_deep_noalloc(cfg: Config, batch: Batch, K: _Tensor, Qwin: _T
                                  stream=None) -> None:
     """Eviction without a workspace, for callers that may not allocate device memory (a server whose
     pool owns the GPU, code under another allocator's lock): the kernels' scratch is a fixed 8 MiB
-    array inside the library.  Raises ``WORKSPACE_TOO_SMALL`` when the batch needs more than that.
-    Calls share the array, so calls that could overlap on the GPU must be ordered by the caller."""
+    array inside the library.  Raises ``WORKSPACE_TOO_SMALL`` when the call would use more than that
+    (never on the tensor-core path, which keeps only a status block there).  Calls share the array, so
+    calls that could overlap on the GPU must be ordered by the caller; ``spindlekv_poll_status(None)``
+    reads the device status word of the last call."""
     cc, bb = cfg.c(), batch.c()
     st = _lib.spindlekv_evict_deep_noalloc(C.byref(cc), C.byref(bb), K, Qwin, _ptr(k_ctx), _ptr(keep_idx),
                                            _ptr(keep_cnt), _ptr(scores), _stream(stream))
@@ -274,8 +276,9 @@ def spindlekv_reconstruct(batch: Batch, n_heads: int, head_dim: int, Cb: _Tensor
     _check(st, "spindlekv_reconstruct")
 
 
-def spindlekv_poll_status(ws: torch.Tensor):
-    """Device status word of a workspace and ``[greedy rounds, live tokens left, 0, 0]``."""
+def spindlekv_poll_status(ws: Optional[torch.Tensor]):
+    """Device status word of a workspace and ``[greedy rounds, live tokens left, 0, 0]``.  ``None`` reads the
+    built-in scratch of ``spindlekv_evict_deep_noalloc`` on the current device."""
     status = C.c_int32(0)
     detail = (C.c_int32 * 4)()
     st = _lib.spindlekv_poll_status(_ptr(ws), C.byref(status), detail)

@@ -11,7 +11,7 @@ CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libspindlekv.so")
 
 SOURCES = ["api.cu", "evict.cu", "codebook.cu", "compact.cu", "sim_tc.cu", "win_tc.cu", "extend.cu", "noalloc.cu"]
-HEADERS = ["common.cuh", "simt_tile.cuh", "sm100_ptx.cuh"]
+HEADERS = ["args.cuh", "common.cuh", "simt_tile.cuh", "sm100_ptx.cuh"]
 
 
 def _nvcc() -> str:

@@ -6,6 +6,7 @@
 #include <mutex>
 #include <vector>
 
+#include "args.cuh"
 #include "common.cuh"
 
 namespace skv {
@@ -28,6 +29,8 @@ spindlekv_status reconstruct_impl(const spindlekv_batch& b, int n_heads, int hea
 spindlekv_status union_lists_impl(int n_layers, int n_seqs, int n_heads, int n_lists, int t_in, int seq_in,
                                   const int32_t* idx_in, const int32_t* cnt_in, int t_out, int seq_out,
                                   int32_t* idx_out, int32_t* cnt_out, cudaStream_t st);
+
+const void* noalloc_scratch_of_current_device();
 
 size_t match_workspace_bytes(const spindlekv_batch& b, int n_heads);
 spindlekv_status match_impl(const spindlekv_batch& b, int n_heads, int head_dim, const spindlekv_tensor& G,
@@ -69,29 +72,6 @@ void note_launch(int kclass, cudaStream_t st, bool before) {
 }  // namespace skv
 
 using namespace skv;
-
-static bool tensor_ok(const spindlekv_tensor& t) {
-  if (!t.ptr) return false;
-  if (t.dtype != SPINDLEKV_F32 && t.dtype != SPINDLEKV_BF16) return false;
-  if (reinterpret_cast<uintptr_t>(t.ptr) % 16) return false;
-  if (t.stride_layer % 8 || t.stride_seq % 8 || t.stride_head % 8 || t.stride_tok % 8) return false;
-  return true;
-}
-
-static bool cfg_ok(const spindlekv_config* c) {
-  if (!c) return false;
-  if (c->n_layers <= 0 || c->n_q_heads <= 0 || c->n_kv_heads <= 0 || c->window <= 0) return false;
-  if (c->n_q_heads % c->n_kv_heads) return false;
-  return true;
-}
-
-static bool batch_ok(const spindlekv_batch* b, int window) {
-  if (!b) return false;
-  if (b->layer_lens && b->cu_seqlens) return false;
-  if (b->n_layers <= 0 || b->n_seqs <= 0 || b->max_len <= window || b->total_len < b->max_len) return false;
-  if (!b->cu_seqlens && (int64_t)b->total_len != (int64_t)b->n_seqs * b->max_len) return false;
-  return true;
-}
 
 extern "C" {
 
@@ -164,12 +144,9 @@ size_t spindlekv_workspace_bytes(const spindlekv_config* cfg, const spindlekv_ba
 spindlekv_status spindlekv_evict_deep(const spindlekv_config* cfg, const spindlekv_batch* batch, spindlekv_tensor K,
                                       spindlekv_tensor Qwin, const int32_t* k_ctx, int32_t* keep_idx,
                                       int32_t* keep_cnt, float* scores, void* ws, size_t ws_bytes, void* stream) {
-  if (!cfg_ok(cfg) || !batch_ok(batch, cfg->window)) return SPINDLEKV_INVALID_ARG;
-  if (!tensor_ok(K) || !tensor_ok(Qwin) || !k_ctx || !keep_idx || !keep_cnt || !scores || !ws) return SPINDLEKV_INVALID_ARG;
-  if (reinterpret_cast<uintptr_t>(ws) % 256) return SPINDLEKV_INVALID_ARG;
-  if (K.dtype != Qwin.dtype) return SPINDLEKV_UNSUPPORTED;
-  if (cfg->head_dim != 64 && cfg->head_dim != 128) return SPINDLEKV_UNSUPPORTED;
-  if ((int64_t)batch->n_layers * batch->n_seqs * cfg->n_kv_heads > 65535) return SPINDLEKV_UNSUPPORTED;
+  const spindlekv_status as = evict_args_status(cfg, batch, K, Qwin, k_ctx, keep_idx, keep_cnt, scores);
+  if (as != SPINDLEKV_OK) return as;
+  if (!ws || reinterpret_cast<uintptr_t>(ws) % 256) return SPINDLEKV_INVALID_ARG;
   return evict_deep_impl(*cfg, *batch, K, Qwin, k_ctx, keep_idx, keep_cnt, scores, ws, ws_bytes, (cudaStream_t)stream);
 }
 
@@ -263,7 +240,9 @@ spindlekv_status spindlekv_reconstruct(const spindlekv_batch* batch, int32_t n_h
 }
 
 spindlekv_status spindlekv_poll_status(const void* ws, int32_t* device_status, int32_t* detail) {
-  if (!ws || !device_status) return SPINDLEKV_INVALID_ARG;
+  if (!device_status) return SPINDLEKV_INVALID_ARG;
+  if (!ws) ws = noalloc_scratch_of_current_device();   // NULL: the built-in scratch of the allocation-free entry point
+  if (!ws) return SPINDLEKV_INVALID_ARG;
   int32_t h[4];
   if (cudaMemcpy(h, ws, sizeof(h), cudaMemcpyDeviceToHost) != cudaSuccess) return SPINDLEKV_CUDA;
   *device_status = h[kHdrStatus];

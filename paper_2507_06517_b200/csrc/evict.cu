@@ -344,6 +344,14 @@ size_t evict_workspace_bytes(const spindlekv_config& cfg, const spindlekv_batch&
   return kHeaderBytes + align_up(units * M * nt * sizeof(float2), 256) + align_up(units * M * sizeof(float2), 256);
 }
 
+bool win_tc_supported(const spindlekv_config& cfg, int dtype);
+
+// Scratch the call really uses: the tensor-core window-score kernel keeps its row statistics on chip and
+// needs the status block only; the CUDA-core kernels keep per-tile row statistics in the workspace.
+size_t evict_scratch_needed(const spindlekv_config& cfg, const spindlekv_batch& b, int dtype) {
+  return win_tc_supported(cfg, dtype) ? (size_t)kHeaderBytes : evict_workspace_bytes(cfg, b);
+}
+
 template <typename T, int D>
 static void launch_window(const EvictParams& p, int units, cudaStream_t st) {
   dim3 grid(p.n_tiles, units);
@@ -353,14 +361,13 @@ static void launch_window(const EvictParams& p, int units, cudaStream_t st) {
   { LaunchScope ls(KC_WINDOW, st); win_colsum_kernel<T, D><<<grid, 256, 0, st>>>(p); }
 }
 
-bool win_tc_supported(const spindlekv_config& cfg, int dtype);
 spindlekv_status launch_win_tc(const spindlekv_config& cfg, const spindlekv_batch& b, const spindlekv_tensor& K,
                                const spindlekv_tensor& Q, float* scores, uint32_t* hdr, cudaStream_t st);
 
 spindlekv_status evict_deep_impl(const spindlekv_config& cfg, const spindlekv_batch& b, const spindlekv_tensor& K,
                                  const spindlekv_tensor& Q, const int32_t* k_ctx, int32_t* keep_idx,
                                  int32_t* keep_cnt, float* scores, void* ws, size_t ws_bytes, cudaStream_t st) {
-  if (ws_bytes < evict_workspace_bytes(cfg, b)) return SPINDLEKV_WORKSPACE_TOO_SMALL;
+  if (ws_bytes < evict_scratch_needed(cfg, b, K.dtype)) return SPINDLEKV_WORKSPACE_TOO_SMALL;
   const int units = b.n_layers * b.n_seqs * cfg.n_kv_heads;
   const int h_n = cfg.n_q_heads / cfg.n_kv_heads;
   const size_t M = (size_t)h_n * cfg.window;

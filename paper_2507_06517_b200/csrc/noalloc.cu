@@ -7,13 +7,15 @@
 // fixed array inside the library image instead of a caller-provided workspace.
 #include <mutex>
 
+#include "args.cuh"
 #include "common.cuh"
 
 namespace skv {
-size_t evict_workspace_bytes(const spindlekv_config& cfg, const spindlekv_batch& b);
+size_t evict_scratch_needed(const spindlekv_config& cfg, const spindlekv_batch& b, int dtype);
 spindlekv_status evict_deep_impl(const spindlekv_config& cfg, const spindlekv_batch& b, const spindlekv_tensor& K,
                                  const spindlekv_tensor& Q, const int32_t* k_ctx, int32_t* keep_idx,
                                  int32_t* keep_cnt, float* scores, void* ws, size_t ws_bytes, cudaStream_t st);
+const void* noalloc_scratch_of_current_device();
 }  // namespace skv
 
 // The scratch itself: 8 MiB of global memory on every device that loads the library, held until exit.
@@ -39,18 +41,25 @@ spindlekv_status scratch_for_current_device(void** out) {
 }
 }  // namespace
 
+// For spindlekv_poll_status(NULL, ...): the scratch of the current device, or null before the first
+// allocation-free call on it.
+const void* skv::noalloc_scratch_of_current_device() {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= skv::kMaxDevices) return nullptr;
+  std::lock_guard<std::mutex> lk(g_setup_mu);
+  return g_scratch_ptr[dev];
+}
+
 extern "C" spindlekv_status spindlekv_evict_deep_noalloc(const spindlekv_config* cfg, const spindlekv_batch* batch,
                                                          spindlekv_tensor K, spindlekv_tensor Qwin,
                                                          const int32_t* k_ctx, int32_t* keep_idx, int32_t* keep_cnt,
                                                          float* scores, void* stream) {
-  if (!cfg || !batch || !K.ptr || !Qwin.ptr || !k_ctx || !keep_idx || !keep_cnt || !scores) return SPINDLEKV_INVALID_ARG;
-  if (cfg->n_q_heads <= 0 || cfg->n_kv_heads <= 0 || cfg->n_q_heads % cfg->n_kv_heads || cfg->window <= 0) return SPINDLEKV_INVALID_ARG;
-  if (batch->n_layers <= 0 || batch->n_seqs <= 0 || batch->max_len <= cfg->window) return SPINDLEKV_INVALID_ARG;
-  if (cfg->head_dim != 64 && cfg->head_dim != 128) return SPINDLEKV_UNSUPPORTED;
-  if (K.dtype != Qwin.dtype) return SPINDLEKV_UNSUPPORTED;
-  if ((int64_t)batch->n_layers * batch->n_seqs * cfg->n_kv_heads > 65535) return SPINDLEKV_UNSUPPORTED;
+  // the same checks as spindlekv_evict_deep, all before anything is enqueued
+  const spindlekv_status as = skv::evict_args_status(cfg, batch, K, Qwin, k_ctx, keep_idx, keep_cnt, scores);
+  if (as != SPINDLEKV_OK) return as;
   // the problem must fit the fixed scratch: say so instead of overrunning it
-  if (skv::evict_workspace_bytes(*cfg, *batch) > (size_t)SPINDLEKV_NOALLOC_SCRATCH_BYTES) return SPINDLEKV_WORKSPACE_TOO_SMALL;
+  if (skv::evict_scratch_needed(*cfg, *batch, K.dtype) > (size_t)SPINDLEKV_NOALLOC_SCRATCH_BYTES)
+    return SPINDLEKV_WORKSPACE_TOO_SMALL;
   void* scratch = nullptr;
   spindlekv_status st = scratch_for_current_device(&scratch);
   if (st != SPINDLEKV_OK) return st;

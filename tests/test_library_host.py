@@ -117,3 +117,33 @@ def test_device_entry_points_reject_bad_arguments_before_touching_the_gpu():
     assert lib.spindlekv_codebook_append(C.byref(batch), 2, 128, good, p, p, p, p, p, None, good, 64, p, p, None) == B.INVALID_ARG
     assert lib.spindlekv_evict_deep_noalloc(C.byref(cfg), C.byref(batch), good, good, None, p, p, p, None) == B.INVALID_ARG
     assert lib.spindlekv_poll_status(None, p, None) == B.INVALID_ARG
+
+
+def test_allocation_free_entry_point_checks_its_arguments_like_the_ordinary_one():
+    # every rejection below comes back before anything is enqueued (no device is needed to see it): a
+    # misaligned base or an odd stride would otherwise reach the 16-byte loads of the kernels
+    import ctypes as C
+    from paper_2507_06517_b200 import binding as B
+    lib = B._lib
+    cfg = B.Config(4, 8, 2, 128, 32, 2, budget_tokens=300.0).c()
+    batch = B._Batch(1, 1, 1024, 1024, None, None, 0)
+    p = C.c_void_p(256)
+    good = B._Tensor(256, B.BF16, 8, 8, 8, 8)
+
+    def call(K=good, Q=good, b=batch, c=cfg):
+        return lib.spindlekv_evict_deep_noalloc(C.byref(c), C.byref(b), K, Q, p, p, p, p, None)
+
+    assert call(K=B._Tensor(264, B.BF16, 8, 8, 8, 8)) == B.INVALID_ARG          # base not 16-byte aligned
+    assert call(Q=B._Tensor(256, B.BF16, 8, 8, 8, 12)) == B.INVALID_ARG         # token stride not a multiple of 8
+    assert call(K=B._Tensor(256, 7, 8, 8, 8, 8)) == B.INVALID_ARG               # unknown dtype
+    assert call(Q=B._Tensor(256, B.F32, 8, 8, 8, 8)) == B.UNSUPPORTED           # K and Q of different types
+    assert call(b=B._Batch(1, 2, 1024, 1024, None, None, 0)) == B.INVALID_ARG   # total_len != n_seqs * max_len
+    assert call(b=B._Batch(1, 1, 1024, 1024, 256, 256, 0)) == B.INVALID_ARG     # packed and per-layer lengths at once
+    assert call(b=B._Batch(0, 1, 1024, 1024, None, None, 0)) == B.INVALID_ARG   # no layers
+    assert call(c=B.Config(4, 8, 2, 96, 32, 2, budget_tokens=300.0).c()) == B.UNSUPPORTED
+    # fp32 inputs run on the CUDA-core kernels, whose row statistics must fit the fixed scratch
+    f32 = B._Tensor(256, B.F32, 8, 8, 8, 8)
+    big = B._Batch(16, 1, 16384, 16384, None, None, 0)
+    assert B.spindlekv_workspace_bytes(B.Config(4, 8, 2, 128, 32, 2, budget_tokens=300.0),
+                                       B.Batch(16, 1, 16384, 16384), B.WS_EVICT) > B.NOALLOC_SCRATCH_BYTES
+    assert call(K=f32, Q=f32, b=big) == B.WORKSPACE_TOO_SMALL

@@ -54,15 +54,33 @@ def test_noalloc_matches_workspace_entry_point_twice_in_a_row():
 
 
 def test_noalloc_rejects_what_does_not_fit():
+    # fp32 inputs take the CUDA-core kernels, which keep per-tile row statistics in the scratch: all 16 evicting
+    # layers of the 16k-token shape at once need about 34 MB of it.  The rejection comes before any launch.
     from paper_2507_06517_b200 import binding as B
     wl = synth.workload("C3")
     cfg = make_config(wl)
-    batch = B.Batch(16, 1, wl.max_len, wl.max_len)  # all 16 evicting layers at once need ~34 MB of scratch
+    batch = B.Batch(16, 1, wl.max_len, wl.max_len)
     assert B.spindlekv_workspace_bytes(cfg, batch, B.WS_EVICT) > B.NOALLOC_SCRATCH_BYTES
-    t = torch.zeros(64, dtype=torch.bfloat16, device="cuda")
+    t = torch.zeros(64, dtype=torch.float32, device="cuda")
     i = torch.zeros(64, dtype=torch.int32, device="cuda")
-    f = torch.zeros(64, dtype=torch.float32, device="cuda")
-    d = B._Tensor(t.data_ptr(), B.BF16, 8, 8, 8, 8)
+    d = B._Tensor(t.data_ptr(), B.F32, 8, 8, 8, 8)
     with pytest.raises(B.SpindleKVError) as e:
-        B.spindlekv_evict_deep_noalloc(cfg, batch, d, d, i, i, i, f)
+        B.spindlekv_evict_deep_noalloc(cfg, batch, d, d, i, i, i, t)
     assert e.value.status == B.WORKSPACE_TOO_SMALL
+
+
+def test_noalloc_on_the_tensor_core_kernel_and_its_status_word():
+    # bf16 with 128 query rows per KV head: the TMA / tensor-core window-score kernel, the only one that writes
+    # the device status word.  Its scratch is the status block alone, so a batch that the CUDA-core path could not
+    # hold fits; the status word of the call is read back through the NULL form of spindlekv_poll_status.
+    from paper_2507_06517_b200 import binding as B
+    wl = synth.Workload("noalloc-tc", 2, 0, 32, 8, 128, "bf16", 32, (1500,), 40, (0.05, 0.3), 4, "recency",
+                        budget_tokens=300.0, seed=19)
+    for _ in range(2):
+        _both_ways(wl)
+        status, _ = B.spindlekv_poll_status(None)
+        assert status == B.OK
+    many = wl.replace(n_layers=12, seq_lens=(6000,), name="noalloc-tc-12")   # row statistics of 12 such layers would not fit 8 MiB
+    assert B.spindlekv_workspace_bytes(make_config(many), B.Batch(12, 1, 6000, 6000), B.WS_EVICT) > B.NOALLOC_SCRATCH_BYTES
+    _both_ways(many)
+    assert B.spindlekv_poll_status(None)[0] == B.OK
