@@ -278,7 +278,9 @@ spindlekv_status spindlekv_reconstruct(const spindlekv_batch* batch, int32_t n_h
  *                 spindlekv_evict_deep_noalloc uses on the current device (INVALID_ARG before the first
  *                 such call on this device)
  *   device_status host out: SPINDLEKV_OK or SPINDLEKV_TIMEOUT
- *   detail        host out, optional [4]: {greedy rounds used, live tokens left, 0, 0}
+ *   detail        host out, optional [4]: {greedy rounds used, live tokens left, units of the call whose
+ *                 adjacency was computed as a bit matrix (all of them for fp32 input; for bf16 input only
+ *                 those whose candidate pairs did not fit the record pool), 0}
  */
 spindlekv_status spindlekv_poll_status(const void* ws, int32_t* device_status, int32_t* detail);
 

@@ -86,6 +86,14 @@ def _load() -> C.CDLL:
                                           _Tensor, C.c_void_p]
     lib.spindlekv_poll_status.restype = C.c_int32
     lib.spindlekv_poll_status.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
+    lib.spindlekv_set_tuning.restype = C.c_int32
+    lib.spindlekv_set_tuning.argtypes = [C.c_int32, C.c_int64]
+    lib.spindlekv_get_tuning.restype = C.c_int64
+    lib.spindlekv_get_tuning.argtypes = [C.c_int32]
+    lib.spindlekv_selftest_grid_barrier_timeout.restype = C.c_int32
+    lib.spindlekv_selftest_grid_barrier_timeout.argtypes = [C.c_void_p, C.c_int64, C.c_void_p]
+    lib.spindlekv_selftest_mbarrier_timeout.restype = C.c_int32
+    lib.spindlekv_selftest_mbarrier_timeout.argtypes = [C.c_void_p, C.c_int64, C.c_void_p]
     lib.spindlekv_launch_count.restype = C.c_int64
     lib.spindlekv_launch_count.argtypes = [C.c_int32]
     lib.spindlekv_timing_enable.restype = None
@@ -277,13 +285,35 @@ def spindlekv_reconstruct(batch: Batch, n_heads: int, head_dim: int, Cb: _Tensor
 
 
 def spindlekv_poll_status(ws: Optional[torch.Tensor]):
-    """Device status word of a workspace and ``[greedy rounds, live tokens left, 0, 0]``.  ``None`` reads the
+    """Device status word of a workspace and ``[greedy rounds, live tokens left, units done as a bit matrix, 0]``.  ``None`` reads the
     built-in scratch of ``spindlekv_evict_deep_noalloc`` on the current device."""
     status = C.c_int32(0)
     detail = (C.c_int32 * 4)()
     st = _lib.spindlekv_poll_status(_ptr(ws), C.byref(status), detail)
     _check(st, "spindlekv_poll_status")
     return int(status.value), [int(x) for x in detail]
+
+
+TUNE_RECORDS_PER_TILE, TUNE_SPIN_LIMIT, TUNE_GREEDY_ROUND_CAP, TUNE_MBAR_WAIT_CYCLES = range(4)
+
+
+def spindlekv_set_tuning(key: int, value: int) -> None:
+    """Test hook: tightens one of the library's limits (``value < 0`` restores the default)."""
+    _check(_lib.spindlekv_set_tuning(key, value), "spindlekv_set_tuning")
+
+
+def spindlekv_get_tuning(key: int) -> int:
+    return int(_lib.spindlekv_get_tuning(key))
+
+
+def spindlekv_selftest_grid_barrier_timeout(ws: torch.Tensor, limit: int, stream=None) -> None:
+    """Test hook: a grid-wide barrier that cannot complete; must leave TIMEOUT in the status word of ``ws``."""
+    _check(_lib.spindlekv_selftest_grid_barrier_timeout(_ptr(ws), limit, _stream(stream)), "spindlekv_selftest_grid_barrier_timeout")
+
+
+def spindlekv_selftest_mbarrier_timeout(ws: torch.Tensor, limit: int, stream=None) -> None:
+    """Test hook: a shared-memory barrier nobody arrives on; must leave TIMEOUT in the status word of ``ws``."""
+    _check(_lib.spindlekv_selftest_mbarrier_timeout(_ptr(ws), limit, _stream(stream)), "spindlekv_selftest_mbarrier_timeout")
 
 
 def spindlekv_launch_count(reset: bool = False) -> int:

@@ -11,6 +11,8 @@
 // of two picks of one round cannot coincide (the picks would be within distance 2 of each other).
 // Pick-time keys equal those of the sequential run and strictly decrease along it, so entry numbers
 // are the ranks of the picks by key.  The result is bit-identical to the one-at-a-time loop.
+#include <algorithm>
+
 #include "common.cuh"
 #include "simt_tile.cuh"
 
@@ -34,13 +36,24 @@ struct CodebookParams {
   int32_t* pickdeg;      // [units][max_len], -1 = not a centre
   int32_t* rank;         // [units][max_len] entry number of a centre
   int32_t* ell;          // [kEll][units][max_len] neighbour lists of rows with few neighbours, entry-major
-  int32_t* ell_cnt;      // [units][max_len] list length, -1: use the bit row
-  int32_t* dense_rows;   // rows (unit * max_len + token) that use their bit row; count in the header
+  int32_t* ell_cnt;      // [units][max_len] list length; -1: use the bit row; -1 - n (n > kEll): the n neighbours are in `csr`
+  int32_t* dense_rows;   // rows (unit * max_len + token) with more than kEll neighbours; count in the header
   uint32_t* flags;       // [units][row_words][row_words/2] bit r of word [w][c]: chunk c (64 columns) of row 32w+r may hold a bit
   uint32_t* hdr;
   int32_t* ref;          // [layers][H][T]
   int32_t* centre_idx;   // [layers][H][T]
   int32_t* n_entries;    // [layers][B][H]
+  // candidate records of the tensor-core similarity kernel and what is built from them
+  const uint2* rec;      // [units][unit_rec_cap]
+  const int32_t* rec_cnt;   // [units][n_blocks]
+  int32_t* ovf;          // [units] != 0: the unit goes through the bit matrix (records did not fit, or no records at all)
+  int rec_per_tile, n_blocks;
+  long long unit_rec_cap;
+  int32_t* csr;          // [units][long_cap] neighbour lists of rows with more than kEll neighbours (record path)
+  int32_t* lbase;        // [units][max_len] start of such a row's list within its unit's part of `csr`
+  int long_cap;
+  uint32_t spin_limit;   // polls after which a grid barrier gives up
+  int round_cap;         // rounds after which the greedy cover gives up
 };
 
 __device__ __forceinline__ void cb_decode(const CodebookParams& p, int unit, int& layer, int& s, int& j) {
@@ -172,11 +185,10 @@ __global__ void __launch_bounds__(256) sim_simt_kernel(CodebookParams p) {
 
 // ---- grid-wide barrier and warp helpers of the cooperative greedy kernel ------------------------
 
-constexpr uint32_t kSpinLimit = 4u << 20;
-
 // Grid-wide barrier on a monotonically increasing counter.  Every wait is bounded: when it gives up
-// it raises the TIMEOUT status, and every block that sees a non-zero status leaves the kernel.
-__device__ __forceinline__ bool grid_barrier(uint32_t* hdr, uint32_t& target) {
+// (after `spin_limit` polls) it raises the TIMEOUT status, and every block that sees a non-zero status
+// leaves the kernel.
+__device__ __forceinline__ bool grid_barrier(uint32_t* hdr, uint32_t& target, uint32_t spin_limit) {
   __shared__ int ok_sh;
   __syncthreads();
   target += gridDim.x;
@@ -188,7 +200,7 @@ __device__ __forceinline__ bool grid_barrier(uint32_t* hdr, uint32_t& target) {
     while (true) {
       uint32_t v = *reinterpret_cast<volatile uint32_t*>(&hdr[kHdrBarrier]);
       if (v >= target) break;
-      if (*reinterpret_cast<volatile uint32_t*>(&hdr[kHdrStatus]) != 0u || ++spins > kSpinLimit) {
+      if (*reinterpret_cast<volatile uint32_t*>(&hdr[kHdrStatus]) != 0u || ++spins > spin_limit) {
         atomicExch(&hdr[kHdrStatus], (uint32_t)SPINDLEKV_TIMEOUT);
         ok = 0;
         break;
@@ -200,6 +212,20 @@ __device__ __forceinline__ bool grid_barrier(uint32_t* hdr, uint32_t& target) {
   }
   __syncthreads();
   return ok_sh != 0;
+}
+
+// Self-test of the bounded barrier: the blocks of this launch are one short of the arrivals the barrier
+// expects, so the wait must run out, raise TIMEOUT in the status word and let every block return.
+__global__ void barrier_selftest_kernel(uint32_t* hdr, uint32_t spin_limit) {
+  uint32_t target = 1;   // one arrival more than the grid will ever deliver
+  const bool ok = grid_barrier(hdr, target, spin_limit);
+  if (ok && threadIdx.x == 0) hdr[kHdrLive] = 0xBADu;   // must not happen
+}
+
+spindlekv_status selftest_grid_barrier_impl(uint32_t* hdr, uint32_t spin_limit, cudaStream_t st) {
+  if (cudaMemsetAsync(hdr, 0, kHeaderBytes, st) != cudaSuccess) return SPINDLEKV_CUDA;
+  barrier_selftest_kernel<<<2, 64, 0, st>>>(hdr, spin_limit);
+  return cudaGetLastError() == cudaSuccess ? SPINDLEKV_OK : SPINDLEKV_CUDA;
 }
 
 __device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long v) {
@@ -231,6 +257,8 @@ __global__ void __launch_bounds__(256, 5) extract_kernel(CodebookParams p) {
   const int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;   // over units x padded rows
   if (g >= (int64_t)p.n_units * NP) return;                           // whole warps: NP is a multiple of 32
   const int unit = (int)(g / NP), u = (int)(g - (int64_t)unit * NP);
+  if (!p.ovf[unit]) return;                                           // built from candidate records instead
+  if (u == 0) atomicAdd(&p.hdr[kHdrBitUnits], 1u);
   int layer, s, j;
   cb_decode(p, unit, layer, s, j);
   const int l = seq_len(p.batch, layer, s, j);
@@ -313,6 +341,157 @@ __global__ void __launch_bounds__(256, 5) extract_kernel(CodebookParams p) {
     p.live0[(int64_t)unit * RW + (u >> 5)] = word;
     p.live1[(int64_t)unit * RW + (u >> 5)] = word;
   }
+}
+
+// ---- neighbour lists from candidate records ------------------------------------------------------
+// One block per unit that fitted its record pool.  A record is a non-zero word of the strict upper
+// triangle: every set bit is a pair (a, b), a < b, and is entered into both tokens' lists.  Degrees are
+// counted in shared memory (a word per token: neighbours in the low half, fill cursor in the high half),
+// then the pairs are entered: tokens with at most kEll neighbours into the entry-major lists that the
+// greedy kernels read (`ell`), the others into one contiguous list each (`csr`).  The order of a list
+// depends on the order in which the atomics land; nothing downstream depends on it (maxima, counts and
+// ownership by the single centre within reach are all independent of it).  Everything else the bit-matrix
+// path's extraction pass leaves behind is written here too: degree, key, live masks, settled isolated
+// tokens, the list of rows with many neighbours.  A unit whose long lists do not fit `long_cap` raises its
+// overflow flag and goes through the bit matrix instead.
+constexpr int kBuildThreads = 1024;
+
+template <typename F>
+__device__ __forceinline__ void for_each_record(const CodebookParams& p, int unit, F f) {
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  const int T = p.n_blocks >> 1;
+  const uint2* pool = p.rec + (long long)unit * p.unit_rec_cap;
+  for (int blk = wid; blk < p.n_blocks; blk += kBuildThreads / 32) {
+    const int n = p.rec_cnt[(long long)unit * p.n_blocks + blk];
+    const uint2* r = pool + rec_region_offset(blk, T, p.rec_per_tile);
+    for (int i0 = 0; i0 < n; i0 += 128) {
+      uint2 v[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const int i = i0 + k * 32 + lane;
+        v[k] = i < n ? r[i] : make_uint2(0u, 0u);
+      }
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+        if (v[k].y) f((int)(v[k].x >> kRecRowShift), (int)(v[k].x & ((1u << kRecRowShift) - 1u)) * 32, v[k].y);
+    }
+  }
+}
+
+__global__ void __launch_bounds__(kBuildThreads) build_lists_kernel(CodebookParams p) {
+  extern __shared__ uint32_t cur[];   // [row_words * 32]
+  __shared__ int long_total, long_used;
+  const int unit = blockIdx.x;
+  if (p.ovf[unit]) return;
+  int layer, s, j;
+  cb_decode(p, unit, layer, s, j);
+  const int l = seq_len(p.batch, layer, s, j);
+  const int RW = p.row_words, NP = RW * 32, ML = p.batch.max_len;
+  const int64_t n_rows = (int64_t)p.n_units * ML;
+  const int64_t row0 = (int64_t)unit * ML;
+  const int tid = threadIdx.x, lane = tid & 31;
+  for (int u = tid; u < NP; u += kBuildThreads) cur[u] = 0u;
+  if (tid == 0) { long_total = 0; long_used = 0; }
+  __syncthreads();
+  // Eq. (10) without the token itself: both ends of every pair
+  for_each_record(p, unit, [&](int a, int b0, uint32_t bits) {
+    atomicAdd(&cur[a], (uint32_t)__popc(bits));
+    while (bits) {
+      atomicAdd(&cur[b0 + __ffs(bits) - 1], 1u);
+      bits &= bits - 1;
+    }
+  });
+  __syncthreads();
+  {
+    int mine = 0;
+    for (int u = tid; u < l; u += kBuildThreads) {
+      const int d = (int)cur[u];
+      if (d > kEll) mine += d;
+    }
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1) mine += __shfl_xor_sync(0xffffffffu, mine, o);
+    if (lane == 0 && mine) atomicAdd(&long_total, mine);
+  }
+  __syncthreads();
+  if (long_total > p.long_cap) {
+    if (tid == 0) p.ovf[unit] = 1;
+    return;
+  }
+  for (int u = tid; u < NP; u += kBuildThreads) {
+    const bool exists = u < l;
+    const int d = exists ? (int)cur[u] : 0;
+    const int64_t idx = row0 + u;
+    bool live = false;
+    if (exists) {
+      const int cnt = d + 1;
+      p.deg[idx] = cnt;
+      p.key[idx] = ((unsigned long long)(uint32_t)cnt << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)u);
+      p.ell_cnt[idx] = d <= kEll ? d : -1 - d;
+      p.pickdeg[idx] = cnt == 1 ? 1 : -1;   // a token without a neighbour is a centre of pick degree 1
+      if (cnt == 1) {
+        p.owner[idx] = u;
+      } else {
+        live = true;
+        if (d > kEll) {
+          p.lbase[idx] = atomicAdd(&long_used, d);
+          p.dense_rows[atomicAdd(&p.hdr[kHdrDenseCnt], 1u)] = (int32_t)idx;
+        }
+      }
+    }
+    const uint32_t word = __ballot_sync(0xffffffffu, live);
+    if (lane == 0) {
+      p.live0[(int64_t)unit * RW + (u >> 5)] = word;
+      p.live1[(int64_t)unit * RW + (u >> 5)] = word;
+    }
+  }
+  __syncthreads();   // lbase of this unit's long rows is complete (read back below through L2)
+  int32_t* csr = p.csr + (int64_t)unit * p.long_cap;
+  auto enter = [&](int a, int b, uint32_t old) {
+    const int d = (int)(old & 0xFFFFu), k = (int)(old >> 16);
+    if (d <= kEll) p.ell[(int64_t)k * n_rows + row0 + a] = b;
+    else csr[__ldcg(&p.lbase[row0 + a]) + k] = b;
+  };
+  for_each_record(p, unit, [&](int a, int b0, uint32_t bits) {
+    uint32_t old_a = atomicAdd(&cur[a], (uint32_t)__popc(bits) << 16);
+    while (bits) {
+      const int b = b0 + __ffs(bits) - 1;
+      bits &= bits - 1;
+      enter(a, b, old_a);
+      old_a += 1u << 16;
+      enter(b, a, atomicAdd(&cur[b], 1u << 16));
+    }
+  });
+}
+
+// Flag words of the units that go through the bit matrix start at zero (the similarity kernel writes only
+// the words that hold a set bit).
+__global__ void __launch_bounds__(256) clear_flags_kernel(CodebookParams p) {
+  const int unit = blockIdx.y;
+  if (!p.ovf[unit]) return;
+  const int64_t n = (int64_t)(p.row_words >> 1) * p.row_words;
+  uint32_t* f = p.flags + (int64_t)unit * n;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) f[i] = 0u;
+}
+
+// The adjacency bit matrix of the units that were built from records, for callers that ask for it: unit
+// diagonal, every recorded pair and its mirror image.  The caller has cleared the matrix.
+__global__ void __launch_bounds__(kBuildThreads) expand_records_kernel(CodebookParams p, uint32_t* adj) {
+  const int unit = blockIdx.x;
+  if (p.ovf[unit]) return;
+  int layer, s, j;
+  cb_decode(p, unit, layer, s, j);
+  const int l = seq_len(p.batch, layer, s, j);
+  const int RW = p.row_words;
+  uint32_t* a_unit = adj + (int64_t)unit * p.batch.max_len * RW;
+  for (int u = threadIdx.x; u < l; u += kBuildThreads) atomicOr(&a_unit[(int64_t)u * RW + (u >> 5)], 1u << (u & 31));
+  for_each_record(p, unit, [&](int a, int b0, uint32_t bits) {
+    atomicOr(&a_unit[(int64_t)a * RW + (b0 >> 5)], bits);
+    while (bits) {
+      const int b = b0 + __ffs(bits) - 1;
+      bits &= bits - 1;
+      atomicOr(&a_unit[(int64_t)b * RW + (a >> 5)], 1u << (a & 31));
+    }
+  });
 }
 
 // ---- greedy cover, cooperative kernel over all units of the call --------------------------------
@@ -480,6 +659,91 @@ __device__ __forceinline__ void pick_dense_row(const CodebookParams& p, const ui
   }
 }
 
+// The same three steps for a row whose `n` neighbours (more than kEll) are listed in `csr` (record path): a warp
+// walks the list, 32 entries at a time.
+__device__ __forceinline__ const int32_t* long_list(const CodebookParams& p, int unit, int64_t idx) {
+  return p.csr + (int64_t)unit * p.long_cap + p.lbase[idx];
+}
+
+__device__ __forceinline__ void degree_of_long_row(const CodebookParams& p, const uint32_t* live, int64_t idx, int n, int lane) {
+  const int ML = p.batch.max_len, RW = p.row_words;
+  const int unit = (int)(idx / ML), u = (int)(idx - (int64_t)unit * ML);
+  const uint32_t* lv = live + (int64_t)unit * RW;
+  if (!is_live(lv, u)) return;
+  const int32_t* list = long_list(p, unit, idx);
+  int cnt = 0;
+  for (int k = lane; k < n; k += 32) cnt += is_live(lv, list[k]) ? 1 : 0;
+#pragma unroll
+  for (int o = 16; o >= 1; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+  if (lane == 0) {
+    p.deg[idx] = cnt + 1;
+    p.key[idx] = ((unsigned long long)(uint32_t)(cnt + 1) << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)u);
+  }
+}
+
+__device__ __forceinline__ void max_of_long_row(const CodebookParams& p, const uint32_t* live, int64_t idx, int n, int lane) {
+  const int ML = p.batch.max_len, RW = p.row_words;
+  const int unit = (int)(idx / ML), u = (int)(idx - (int64_t)unit * ML);
+  const uint32_t* lv = live + (int64_t)unit * RW;
+  if (!is_live(lv, u)) return;
+  const unsigned long long* key = p.key + (int64_t)unit * ML;
+  const int32_t* list = long_list(p, unit, idx);
+  unsigned long long best = lane == 0 ? key[u] : 0ull;   // the token itself belongs to its closed neighbourhood
+  for (int k = lane; k < n; k += 32) {
+    const int v = list[k];
+    if (is_live(lv, v)) {
+      const unsigned long long kv = key[v];
+      best = kv > best ? kv : best;
+    }
+  }
+  best = warp_max_u64(best);
+  if (lane == 0) p.m1[idx] = best;
+}
+
+__device__ __forceinline__ void pick_long_row(const CodebookParams& p, const uint32_t* live, uint32_t* next, int64_t idx, int n,
+                                              int lane) {
+  const int ML = p.batch.max_len, RW = p.row_words;
+  const int unit = (int)(idx / ML), u = (int)(idx - (int64_t)unit * ML);
+  const uint32_t* lv = live + (int64_t)unit * RW;
+  if (!is_live(lv, u)) return;
+  const unsigned long long mykey = p.key[idx];
+  if (p.m1[idx] != mykey) return;
+  const unsigned long long* m1 = p.m1 + (int64_t)unit * ML;
+  int32_t* owner = p.owner + (int64_t)unit * ML;
+  uint32_t* nx = next + (int64_t)unit * RW;
+  const int32_t* list = long_list(p, unit, idx);
+  bool ok = true;
+  for (int k = lane; k < n; k += 32) {
+    const int v = list[k];
+    if (is_live(lv, v) && m1[v] != mykey) ok = false;
+  }
+  if (!__all_sync(0xffffffffu, ok)) return;
+  for (int k = lane; k < n; k += 32) {
+    const int v = list[k];
+    if (is_live(lv, v)) {
+      owner[v] = u;
+      atomicAnd(&nx[v >> 5], ~(1u << (v & 31)));
+    }
+  }
+  if (lane == 0) {
+    p.pickdeg[idx] = p.deg[idx];
+    owner[u] = u;
+    atomicAnd(&nx[u >> 5], ~(1u << (u & 31)));
+  }
+}
+
+// A row with more than kEll neighbours: its bit row (ell_cnt == -1) or its list (ell_cnt == -1 - n).
+__device__ __forceinline__ void max_of_big_row(const CodebookParams& p, const uint32_t* live, int64_t idx, int lane) {
+  const int ec = p.ell_cnt[idx];
+  if (ec == -1) max_of_dense_row(p, live, idx, lane);
+  else max_of_long_row(p, live, idx, -1 - ec, lane);
+}
+__device__ __forceinline__ void pick_big_row(const CodebookParams& p, const uint32_t* live, uint32_t* next, int64_t idx, int lane) {
+  const int ec = p.ell_cnt[idx];
+  if (ec == -1) pick_dense_row(p, live, next, idx, lane);
+  else pick_long_row(p, live, next, idx, -1 - ec, lane);
+}
+
 // Round 0 as two ordinary launches: every row is still live, so the phases run with one warp per word of
 // the live mask over the whole grid (far more threads in flight than the cooperative kernel can keep
 // resident); the last kDenseBlocks blocks walk the list of dense rows.  `phase` 2: neighbourhood maxima,
@@ -497,8 +761,8 @@ __global__ void __launch_bounds__(256) greedy_first_round_kernel(CodebookParams 
     const int n_dense = (int)p.hdr[kHdrDenseCnt];
     const int nw = kDenseBlocks * (blockDim.x >> 5);
     for (int d = ((int)blockIdx.x - word_blocks) * (blockDim.x >> 5) + (threadIdx.x >> 5); d < n_dense; d += nw) {
-      if (phase == 2) max_of_dense_row(p, p.live0, p.dense_rows[d], lane);
-      else pick_dense_row(p, p.live0, p.live1, p.dense_rows[d], lane);
+      if (phase == 2) max_of_big_row(p, p.live0, p.dense_rows[d], lane);
+      else pick_big_row(p, p.live0, p.live1, p.dense_rows[d], lane);
     }
   }
 }
@@ -516,8 +780,9 @@ __global__ void __launch_bounds__(512) greedy_kernel(CodebookParams p) {
   const int n_dense = (int)*reinterpret_cast<volatile uint32_t*>(&p.hdr[kHdrDenseCnt]);
   uint32_t target = 0;
 
+  const int round_cap = min(ML, p.round_cap);
   int round = 1;
-  for (; round <= ML; ++round) {
+  for (; round <= round_cap; ++round) {
     uint32_t* live = (round & 1) ? p.live1 : p.live0;
     uint32_t* next = (round & 1) ? p.live0 : p.live1;
     const int slot = (round & 1) ? kHdrLiveCnt1 : kHdrLiveCnt0;
@@ -550,6 +815,11 @@ __global__ void __launch_bounds__(512) greedy_kernel(CodebookParams p) {
       }
       for (int64_t d = gwarp; d < n_dense; d += nwarps) {
         const int64_t idx = p.dense_rows[d];
+        const int ec_big = p.ell_cnt[idx];
+        if (ec_big != -1) {
+          degree_of_long_row(p, live, idx, -1 - ec_big, lane);
+          continue;
+        }
         const int unit = (int)(idx / ML), u = (int)(idx - (int64_t)unit * ML);
         const uint32_t* lv = live + (int64_t)unit * RW;
         if (!is_live(lv, u)) continue;
@@ -570,26 +840,26 @@ __global__ void __launch_bounds__(512) greedy_kernel(CodebookParams p) {
         }
       }
       if (lane == 0 && my_live) atomicAdd(&p.hdr[slot], (uint32_t)my_live);
-      if (!grid_barrier(p.hdr, target)) return;
+      if (!grid_barrier(p.hdr, target, p.spin_limit)) return;
       const uint32_t total_live = *reinterpret_cast<volatile uint32_t*>(&p.hdr[slot]);
       if (total_live == 0) break;
     }
 
     // phase 2: largest key in each closed live neighbourhood
     for (int64_t w = gwarp; w < n_words; w += nwarps) max_of_listed_rows<false>(p, live, w, lane);
-    for (int64_t d = gwarp; d < n_dense; d += nwarps) max_of_dense_row(p, live, p.dense_rows[d], lane);
-    if (!grid_barrier(p.hdr, target)) return;
+    for (int64_t d = gwarp; d < n_dense; d += nwarps) max_of_big_row(p, live, p.dense_rows[d], lane);
+    if (!grid_barrier(p.hdr, target, p.spin_limit)) return;
 
     // phase 3: picks
     for (int64_t w = gwarp; w < n_words; w += nwarps) pick_listed_rows<false>(p, live, next, w, lane);
-    for (int64_t d = gwarp; d < n_dense; d += nwarps) pick_dense_row(p, live, next, p.dense_rows[d], lane);
-    if (!grid_barrier(p.hdr, target)) return;
+    for (int64_t d = gwarp; d < n_dense; d += nwarps) pick_big_row(p, live, next, p.dense_rows[d], lane);
+    if (!grid_barrier(p.hdr, target, p.spin_limit)) return;
   }
   if (gthread == 0) {
     p.hdr[kHdrRounds] = (uint32_t)round;
     uint32_t left = *reinterpret_cast<volatile uint32_t*>(&p.hdr[(round & 1) ? kHdrLiveCnt1 : kHdrLiveCnt0]);
-    p.hdr[kHdrLive] = round > ML ? 1u : left;
-    if (round > ML) atomicExch(&p.hdr[kHdrStatus], (uint32_t)SPINDLEKV_TIMEOUT);
+    p.hdr[kHdrLive] = round > round_cap ? max(left, 1u) : left;
+    if (round > round_cap) atomicExch(&p.hdr[kHdrStatus], (uint32_t)SPINDLEKV_TIMEOUT);
   }
 }
 
@@ -767,7 +1037,7 @@ __global__ void __launch_bounds__(kFinalThreads) finalize_kernel(CodebookParams 
     }
     int r[8];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) r[i] = o[i] >= 0 ? rank[o[i]] : 0;
+    for (int i = 0; i < 8; ++i) r[i] = (o[i] >= 0 && o[i] < l) ? rank[o[i]] : 0;   // a cover that was cut short leaves owners unset
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
       const int b = b0 + i * kFinalThreads;
@@ -781,9 +1051,16 @@ __global__ void __launch_bounds__(kFinalThreads) finalize_kernel(CodebookParams 
 
 struct CodebookLayout {
   size_t ext, ell, ell_cnt, dense_rows, flags, adj, deg, key, m1, live0, live1, owner, pickdeg, rank, total;
+  size_t ovf, rec_cnt, lbase, csr, rec;   // candidate records (tensor-core path)
+  int rec_per_tile, n_blocks, long_cap;
 };
 
-static CodebookLayout codebook_layout(const spindlekv_config& cfg, const spindlekv_batch& b, bool adj_in_ws) {
+// Neighbour-list entries per unit that the record path may spend on rows with more than kEll neighbours.
+static int long_list_capacity(int max_len) { return 64 * max_len; }
+// The record path counts degrees in one 32-bit word per token in shared memory.
+static bool record_path_fits(int max_len) { return row_words_for(max_len) * 32 <= 49152; }
+
+static CodebookLayout codebook_layout(const spindlekv_config& cfg, const spindlekv_batch& b, bool adj_in_ws, int rec_per_tile) {
   size_t units = (size_t)b.n_layers * b.n_seqs * cfg.n_kv_heads;
   size_t ML = b.max_len, RW = row_words_for(b.max_len);
   CodebookLayout L;
@@ -802,6 +1079,15 @@ static CodebookLayout codebook_layout(const spindlekv_config& cfg, const spindle
   L.ell_cnt = take(units * ML * 4);
   L.dense_rows = take(units * ML * 4);
   L.flags = take(units * (RW / 2) * RW * 4);
+  // candidate records: the overflow flags and the per-block counts sit side by side (one clearing pass)
+  L.rec_per_tile = record_path_fits(b.max_len) ? rec_per_tile : 0;
+  L.n_blocks = 2 * ceil_div(b.max_len, 256);
+  L.long_cap = long_list_capacity(b.max_len);
+  L.ovf = take(units * 4);
+  L.rec_cnt = take(units * L.n_blocks * 4);
+  L.lbase = take(units * ML * 4);
+  L.csr = take(L.rec_per_tile ? units * (size_t)L.long_cap * 4 : 0);
+  L.rec = take(L.rec_per_tile ? units * (size_t)rec_unit_capacity(L.n_blocks / 2, L.rec_per_tile) * 8 : 0);
   L.adj = off;
   if (adj_in_ws) take(units * ML * RW * 4);
   L.total = off;
@@ -809,13 +1095,14 @@ static CodebookLayout codebook_layout(const spindlekv_config& cfg, const spindle
 }
 
 size_t codebook_workspace_bytes(const spindlekv_config& cfg, const spindlekv_batch& b) {
-  return codebook_layout(cfg, b, true).total;
+  // sized for the default record pool; tuning can only make the pool of a call smaller
+  return codebook_layout(cfg, b, true, kDefaultRecPerTile).total;
 }
 
 bool sim_tc_available();
 spindlekv_status launch_sim_tc(const spindlekv_tensor& Gamma, const spindlekv_batch& b, int n_kv_heads, int head_dim,
                                const void* ext, uint32_t* adj, uint32_t* flags, uint32_t* hdr, bool skip_empty,
-                               cudaStream_t st);
+                               const SimRecordPool* pool, bool emit, long long wait_cycles, cudaStream_t st);
 
 template <typename T, int D>
 static void launch_norms(const CodebookParams& p, cudaStream_t st) {
@@ -835,11 +1122,15 @@ spindlekv_status codebook_shallow_impl(const spindlekv_config& cfg, const spindl
                                        int32_t* centre_idx, int32_t* n_entries, uint32_t* adj_bits, void* ws,
                                        size_t ws_bytes, cudaStream_t st) {
   const bool adj_in_ws = adj_bits == nullptr;
-  CodebookLayout L = codebook_layout(cfg, b, adj_in_ws);
+  const Tuning tune = current_tuning();
+  const bool bf = Gamma.dtype == SPINDLEKV_BF16;
+  const bool tc = bf && sim_tc_available();   // bf16: tensor-core similarity (TMA + tcgen05)
+  CodebookLayout L = codebook_layout(cfg, b, adj_in_ws, tc ? min(tune.rec_per_tile, kDefaultRecPerTile) : 0);
   if (ws_bytes < L.total) return SPINDLEKV_WORKSPACE_TOO_SMALL;
   if ((size_t)(b.max_len + 2) * 4 > 200 * 1024) return SPINDLEKV_UNSUPPORTED;
   const int units = b.n_layers * b.n_seqs * cfg.n_kv_heads;
   if (units > 65535) return SPINDLEKV_UNSUPPORTED;
+  const bool records = L.rec_per_tile > 0;    // candidate records first, the bit matrix for units that overflow
   char* w = reinterpret_cast<char*>(ws);
   CodebookParams p;
   p.G = make_view(Gamma);
@@ -866,19 +1157,53 @@ spindlekv_status codebook_shallow_impl(const spindlekv_config& cfg, const spindl
   p.ref = ref;
   p.centre_idx = centre_idx;
   p.n_entries = n_entries;
+  p.rec = reinterpret_cast<const uint2*>(w + L.rec);
+  p.rec_cnt = reinterpret_cast<const int32_t*>(w + L.rec_cnt);
+  p.ovf = reinterpret_cast<int32_t*>(w + L.ovf);
+  p.rec_per_tile = L.rec_per_tile;
+  p.n_blocks = L.n_blocks;
+  p.unit_rec_cap = records ? rec_unit_capacity(L.n_blocks / 2, L.rec_per_tile) : 0;
+  p.csr = reinterpret_cast<int32_t*>(w + L.csr);
+  p.lbase = reinterpret_cast<int32_t*>(w + L.lbase);
+  p.long_cap = L.long_cap;
+  p.spin_limit = tune.spin_limit;
+  p.round_cap = tune.round_cap;
   if (cudaMemsetAsync(w, 0, kHeaderBytes, st) != cudaSuccess) return SPINDLEKV_CUDA;
-  const bool bf = Gamma.dtype == SPINDLEKV_BF16;
-  const bool tc = bf && sim_tc_available();   // bf16: tensor-core similarity (TMA + tcgen05)
+  // overflow flags and record counts: all zero on the record path; without records every unit counts as overflowed
+  if (cudaMemsetAsync(w + L.ovf, records ? 0 : 1, L.lbase - L.ovf, st) != cudaSuccess) return SPINDLEKV_CUDA;
   p.ext = tc ? reinterpret_cast<__nv_bfloat16*>(w + L.ext) : nullptr;
   if (cfg.head_dim == 64) {
     if (bf) launch_norms<__nv_bfloat16, 64>(p, st); else launch_norms<float, 64>(p, st);
   } else {
     if (bf) launch_norms<__nv_bfloat16, 128>(p, st); else launch_norms<float, 128>(p, st);
   }
+  const size_t flag_words = (size_t)(p.row_words / 2) * p.row_words;
   if (tc) {
-    // the similarity kernel writes only the flag words that hold a set bit
-    if (cudaMemsetAsync(p.flags, 0, (size_t)units * (p.row_words / 2) * p.row_words * 4, st) != cudaSuccess) return SPINDLEKV_CUDA;
-    spindlekv_status rs = launch_sim_tc(Gamma, b, cfg.n_kv_heads, cfg.head_dim, p.ext, p.adj, p.flags, p.hdr, adj_in_ws, st);
+    SimRecordPool pool{reinterpret_cast<uint2*>(w + L.rec), reinterpret_cast<int32_t*>(w + L.rec_cnt), p.ovf, L.rec_per_tile};
+    if (records) {
+      if (!adj_in_ws &&
+          cudaMemsetAsync(adj_bits, 0, (size_t)units * b.max_len * p.row_words * 4, st) != cudaSuccess) return SPINDLEKV_CUDA;
+      spindlekv_status rs = launch_sim_tc(Gamma, b, cfg.n_kv_heads, cfg.head_dim, p.ext, p.adj, p.flags, p.hdr, adj_in_ws, &pool,
+                                          true, tune.mbar_wait_cycles, st);
+      if (rs != SPINDLEKV_OK) return rs;
+      static PerDeviceOnce once;
+      const int dev0 = PerDeviceOnce::current();
+      if (dev0 < 0) return SPINDLEKV_CUDA;
+      if (!once.done[dev0]) {
+        if (cudaFuncSetAttribute(build_lists_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 49152 * 4) != cudaSuccess)
+          return SPINDLEKV_CUDA;
+        once.done[dev0] = true;
+      }
+      LaunchScope ls(KC_DEGREE, st);
+      build_lists_kernel<<<units, kBuildThreads, (size_t)p.row_words * 32 * 4, st>>>(p);
+    }
+    // units without usable records (all of them when the record path is off): bit matrix, occupancy flags, extraction
+    {
+      LaunchScope ls(KC_DEGREE, st);
+      clear_flags_kernel<<<dim3((unsigned)std::min<size_t>((flag_words + 255) / 256, 64), units), 256, 0, st>>>(p);
+    }
+    spindlekv_status rs = launch_sim_tc(Gamma, b, cfg.n_kv_heads, cfg.head_dim, p.ext, p.adj, p.flags, p.hdr, adj_in_ws, &pool,
+                                        false, tune.mbar_wait_cycles, st);
     if (rs != SPINDLEKV_OK) return rs;
   } else if (cfg.head_dim == 64) {
     if (bf) launch_sim_simt<__nv_bfloat16, 64>(p, b, st); else launch_sim_simt<float, 64>(p, b, st);
@@ -887,12 +1212,15 @@ spindlekv_status codebook_shallow_impl(const spindlekv_config& cfg, const spindl
   }
   if (!tc) {
     // the CUDA-core similarity kernel writes no occupancy flags: every chunk counts as occupied
-    if (cudaMemsetAsync(p.flags, 0xFF, (size_t)units * (p.row_words / 2) * p.row_words * 4, st) != cudaSuccess)
-      return SPINDLEKV_CUDA;
+    if (cudaMemsetAsync(p.flags, 0xFF, (size_t)units * flag_words * 4, st) != cudaSuccess) return SPINDLEKV_CUDA;
   }
   {
     LaunchScope ls(KC_DEGREE, st);
     extract_kernel<<<(unsigned)(((size_t)units * p.row_words * 32 + 255) / 256), 256, 0, st>>>(p);
+  }
+  if (records && !adj_in_ws) {
+    LaunchScope ls(KC_DEGREE, st);
+    expand_records_kernel<<<units, kBuildThreads, 0, st>>>(p, adj_bits);
   }
   // cooperative launch: as many blocks as can be resident at once
   static int coop_blocks_dev[kMaxDevices] = {};

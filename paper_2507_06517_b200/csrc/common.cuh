@@ -10,12 +10,13 @@
 namespace skv {
 
 // ---- status block at the start of every workspace -------------------------------------------
-// word 0: device status, 1: greedy rounds used, 2: live tokens left, 3: unused,
+// word 0: device status, 1: greedy rounds used, 2: live tokens left, 3: units whose neighbour lists came from a bit matrix,
 // words 8..: barrier and counters of the cooperative greedy kernel.
 constexpr int kHeaderBytes = 256;
 constexpr int kHdrStatus = 0;
 constexpr int kHdrRounds = 1;
 constexpr int kHdrLive = 2;
+constexpr int kHdrBitUnits = 3;
 constexpr int kHdrBarrier = 8;
 constexpr int kHdrLiveCnt0 = 9;   // two slots, alternated by round parity
 constexpr int kHdrLiveCnt1 = 10;
@@ -82,6 +83,26 @@ __device__ __forceinline__ void load8(const __nv_bfloat16* p, float* out) {
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 __host__ __device__ inline int row_words_for(int max_len) { return 4 * ((max_len + 127) / 128); }
+
+// ---- candidate records of the similarity kernel ------------------------------------------------------
+// A record is one non-zero word of the strict upper triangle of the adjacency: .x = row << kRecRowShift |
+// word column (32 columns per word), .y = the word's bits.
+constexpr int kRecRowShift = 11;   // word columns < 2048, i.e. sequences of fewer than 65536 tokens
+// Record pool of a unit: the similarity kernel's row block `blk` of pair p = blk / 2 computes the tiles p .. T-1 (T tiles of 256
+// columns for the call's longest sequence), so its region holds rec_per_tile * (T - p) records and
+// starts after those of the blocks before it.
+__host__ __device__ inline long long rec_region_offset(int blk, int T, int rec_per_tile) {
+  const long long p = blk >> 1, r = blk & 1;
+  return (long long)rec_per_tile * (2 * p * T - p * (p - 1) + r * (T - p));
+}
+__host__ __device__ inline long long rec_unit_capacity(int T, int rec_per_tile) { return (long long)rec_per_tile * T * (T + 1); }
+
+struct SimRecordPool {   // device buffers of the candidate records of one CodeBook call
+  uint2* rec;            // [units][rec_unit_capacity]
+  int32_t* rec_cnt;      // [units][row blocks]
+  int32_t* ovf;          // [units]
+  int rec_per_tile;
+};
 
 // 32x32 bit transpose across a warp: in: lane r holds bits (r, c) at bit c; out: lane c holds bit r.
 // Five butterfly stages (j = 16, 8, 4, 2, 1): a lane takes from its partner the half of every 2j-bit
@@ -152,6 +173,18 @@ struct PerDeviceOnce {
     return cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < kMaxDevices ? dev : -1;
   }
 };
+
+// ---- limits that tests may tighten (host) -----------------------------------------------------------
+constexpr int kDefaultRecPerTile = 512;             // candidate records per 128 x 256 tile of a row block's region
+constexpr uint32_t kDefaultSpinLimit = 4u << 20;    // polls of a grid barrier
+constexpr long long kDefaultMbarWaitCycles = 4000000000ll;   // about two seconds of SM clock
+struct Tuning {
+  int rec_per_tile;          // 0: no candidate records, every unit goes through the bit matrix
+  uint32_t spin_limit;
+  int round_cap;             // greedy rounds (never more than the sequence length)
+  long long mbar_wait_cycles;
+};
+Tuning current_tuning();
 
 // ---- launch bookkeeping (host) ---------------------------------------------------------------
 void note_launch(int kclass, cudaStream_t st, bool before);

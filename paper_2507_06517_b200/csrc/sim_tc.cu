@@ -32,6 +32,18 @@
 // exactly one writer: the rows' own block for chunks at or right of the block's own columns, the
 // block that mirrors into the rows for chunks left of them.  The caller clears the flag words; only
 // words with a set bit are written.
+//
+// Candidate emission (the first choice; the bit matrix above is the bounded fallback).  Graphs of real
+// caches are sparse: a token is similar to a handful of others.  In this form a warp, after collecting
+// the sign words of its 32 x 128 piece of a tile, keeps the pairs with a < b only and writes nothing but
+// the non-zero words, as records (row, word column, 32 bits): a ballot counts them, one shared-memory
+// atomic reserves room in the block's own region of the unit's record pool, and the lanes store their
+// records side by side.  No transpose, no staging, no barrier between warps: the next kernel mirrors the
+// pairs when it builds the neighbour lists.  A block's region holds `rec_per_tile` records per tile it
+// computes; a block that runs out of room raises the unit's overflow flag, and such units are computed
+// again as a bit matrix by the other instantiation of this kernel (which returns at once for all other
+// units).  The order of the records inside a region depends on warp timing; everything derived from them
+// is independent of that order.
 #include "common.cuh"
 #include "sm100_ptx.cuh"
 
@@ -44,6 +56,13 @@ struct SimTcParams {
   uint32_t* flags;     // [units][row_words][row_words / 2]
   uint32_t* hdr;
   int skip_empty;      // mirrored chunks without a set bit are not stored (their flag bit stays 0)
+  // candidate emission
+  uint2* rec;          // [units][unit_rec_cap] records: .x = row << kRecRowShift | word column, .y = bits (pairs a < b only)
+  int32_t* rec_cnt;    // [units][blocks] records written by each row block (cleared by the caller)
+  int32_t* ovf;        // [units] != 0: the unit does not fit the record pool and is computed as a bit matrix
+  int rec_per_tile;    // a block's region holds rec_per_tile records per tile it computes
+  long long unit_rec_cap;
+  long long wait_cycles;   // bound of every mbarrier wait, in SM clock cycles
 };
 
 constexpr int kBM = 128;          // rows of the resident block (UMMA M)
@@ -150,12 +169,15 @@ __device__ __forceinline__ void umma_commit_pair(uint64_t* bar) {
                ::"r"(ptx::smem_u32(bar)), "h"((uint16_t)3) : "memory");
 }
 
-template <int D>
+// kEmit: candidate records for every unit; otherwise the bit matrix, for the units whose overflow flag is set
+// (all units when the caller passes no flags).
+template <int D, bool kEmit>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kSimThreads, 1) sim_tc_kernel(const __grid_constant__ CUtensorMap tmap,
                                                                 const __grid_constant__ CUtensorMap emap,
                                                                 SimTcParams p) {
   using L = SimSmem<D>;
   const int unit = blockIdx.y;
+  if (!kEmit && p.ovf && !p.ovf[unit]) return;   // both CTAs of a pair: the unit's records were enough
   const int j = unit % p.n_kv_heads;
   const int ls = unit / p.n_kv_heads;
   const int s = ls % p.batch.n_seqs;
@@ -185,6 +207,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kSimThreads, 1) sim_
   uint64_t* acc_empty = acc_full + 2;           // [2]
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(acc_empty + 3);
+  int* rec_used = reinterpret_cast<int*>(acc_empty + 3) + 1;   // records this block has reserved
+  const long long wait_cycles = p.wait_cycles;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
@@ -192,6 +216,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kSimThreads, 1) sim_
     for (int i = 0; i < kStages; ++i) { ptx::mbar_init(b_full + i, 1); ptx::mbar_init(b_empty + i, 1); }
     for (int i = 0; i < 2; ++i) { ptx::mbar_init(acc_full + i, 1); ptx::mbar_init(acc_empty + i, 2 * kTeamWarps); }
     *abort_flag = 0;
+    *rec_used = 0;
     ptx::fence_barrier_init();
   }
   if (warp == 1) {
@@ -216,7 +241,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kSimThreads, 1) sim_
       tma_load_4d_pair(sEA, &emap, a_full, 0, row0, unit, 0);
       for (int it = 0; tile0 + it < n_tiles; ++it) {
         const int st = it % kStages;
-        if (!ptx::mbar_wait(b_empty + st, ((it / kStages) & 1) ^ 1, abort_flag)) break;
+        if (!ptx::mbar_wait(b_empty + st, ((it / kStages) & 1) ^ 1, abort_flag, wait_cycles)) break;
         if (rank == 0) ptx::mbar_expect_tx(b_full + st, 2 * (L::B_BYTES + L::EB_BYTES));
         uint8_t* dst = sB + st * L::B_BYTES;
         const int brow = (tile0 + it) * kBN + rank * kBH;   // this CTA's half of the tile
@@ -231,11 +256,11 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kSimThreads, 1) sim_
       constexpr uint32_t idesc_pos = ptx::idesc_bf16_f32(2 * kBM, kBN, false);
       const uint32_t a_addr = ptx::smem_u32(sA);
       const uint64_t dea = ptx::smem_desc_sw32(ptx::smem_u32(sEA));
-      bool ok = ptx::mbar_wait(a_full, 0, abort_flag);
+      bool ok = ptx::mbar_wait(a_full, 0, abort_flag, wait_cycles);
       for (int it = 0; ok && tile0 + it < n_tiles; ++it) {
         const int st = it % kStages, as = it & 1;
-        if (!ptx::mbar_wait(b_full + st, (it / kStages) & 1, abort_flag)) break;
-        if (!ptx::mbar_wait(acc_empty + as, ((it >> 1) & 1) ^ 1, abort_flag)) break;
+        if (!ptx::mbar_wait(b_full + st, (it / kStages) & 1, abort_flag, wait_cycles)) break;
+        if (!ptx::mbar_wait(acc_empty + as, ((it >> 1) & 1) ^ 1, abort_flag, wait_cycles)) break;
         ptx::tc_fence_after();
         const uint32_t b_addr = ptx::smem_u32(sB + st * L::B_BYTES);
 #pragma unroll
@@ -249,6 +274,88 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kSimThreads, 1) sim_
         umma_bf16_pair(tmem_base + as * kBN, dea, ptx::smem_desc_sw32(ptx::smem_u32(sEB + st * L::EB_BYTES)), idesc_pos, 1u);
         umma_commit_pair(b_empty + st);   // both CTAs: the stage may be refilled
         umma_commit_pair(acc_full + as);  // both CTAs: accumulator ready for the epilogue
+      }
+    }
+  } else if constexpr (kEmit) {
+    // ---- candidate emission ----
+    const int q = warp & 3;               // TMEM lane quarter this warp may read
+    const int team = (warp - 2) >> 3;     // which TMEM stage this warp serves
+    const int cg = ((warp - 2) >> 2) & 1; // which half of the tile's columns
+    const int R = row0 + q * 32;          // first row of this warp's 32-row strip
+    const int row = R + lane;
+    const bool live_block = row0 < l;     // the second CTA of a sequence's last pair may own no row at all
+    const uint32_t tcol = tmem_base + ((uint32_t)(q * 32) << 16) + team * kBN + cg * kColsPerWarp;
+    const uint32_t below = (1u << lane) - 1u;
+    const uint32_t key_row = (uint32_t)row << kRecRowShift;
+#pragma unroll 1
+    for (int it = team; tile0 + it < n_tiles; it += 2) {
+      const int c0 = (tile0 + it) * kBN;
+      bool ok = __all_sync(0xffffffffu, ptx::mbar_wait(acc_full + team, (it >> 1) & 1, abort_flag, wait_cycles));
+      if (!ok) break;                     // nobody waits for this warp: it may leave its loop
+      if (!live_block) {
+        if (lane == 0) mbar_arrive_leader(acc_empty + team);
+        continue;
+      }
+      ptx::tc_fence_after();
+      uint32_t words[kChunks];
+      words[0] = words[1] = words[2] = words[3] = 0u;
+      // This loop must stay a loop: unrolled, every pass gets 32 registers of its own for its accumulators
+      // and the thread (96 registers with twenty warps in the block) spills, which costs more than all the rest.
+#pragma unroll 1
+      for (int ch = 0; ch < kChunks; ++ch) {
+        uint32_t acc[32];
+        ptx::tmem_ld_32x32_sync(tcol + ch * 32, acc);   // load and wait in one statement
+        const uint32_t w = sign_word(acc);
+        words[0] = ch == 0 ? w : words[0];
+        words[1] = ch == 1 ? w : words[1];
+        words[2] = ch == 2 ? w : words[2];
+        words[3] = ch == 3 ? w : words[3];
+      }
+      ptx::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_leader(acc_empty + team);
+      const int wc0 = (c0 + cg * kColsPerWarp) >> 5;   // word column of this warp's first 32 columns
+      if (c0 + kBN > l || R + 32 > l) {
+        // ragged edge: columns and rows that do not exist carry no bits
+#pragma unroll
+        for (int ch = 0; ch < kChunks; ++ch) {
+          const int nvalid = l - (wc0 + ch) * 32;
+          if (nvalid < 32) words[ch] &= nvalid > 0 ? ((1u << nvalid) - 1u) : 0u;
+          if (row >= l) words[ch] = 0;
+        }
+      }
+      if (c0 < row0 + kBM) {
+        // the tile that holds the diagonal: only pairs a < b are kept (the rest is their mirror image)
+#pragma unroll
+        for (int ch = 0; ch < kChunks; ++ch) {
+          const int col0 = (wc0 + ch) * 32;
+          if (col0 + 32 <= R) words[ch] = 0u;
+          else if (col0 == R) words[ch] &= lane == 31 ? 0u : (0xFFFFFFFFu << (lane + 1));
+        }
+      }
+      uint32_t m[kChunks];
+      int n = 0;
+#pragma unroll
+      for (int ch = 0; ch < kChunks; ++ch) {
+        m[ch] = __ballot_sync(0xffffffffu, words[ch] != 0u);
+        n += __popc(m[ch]);
+      }
+      if (n == 0) continue;
+      int at = 0;
+      if (lane == 0) at = atomicAdd(rec_used, n);
+      at = __shfl_sync(0xffffffffu, at, 0);
+      // the block's region of the unit's record pool (worked out here, where it is needed, to keep registers free)
+      const int T_max = (p.batch.max_len + kBN - 1) / kBN;
+      const int cap = p.rec_per_tile * (T_max - (int)(blockIdx.x >> 1));
+      uint2* rec_blk = p.rec + (long long)unit * p.unit_rec_cap + rec_region_offset((int)blockIdx.x, T_max, p.rec_per_tile);
+      if (at + n > cap) {
+        if (lane == 0) p.ovf[unit] = 1;   // the unit is computed again as a bit matrix
+        continue;
+      }
+#pragma unroll
+      for (int ch = 0; ch < kChunks; ++ch) {
+        if (words[ch]) rec_blk[at + __popc(m[ch] & below)] = make_uint2(key_row | (uint32_t)(wc0 + ch), words[ch]);
+        at += __popc(m[ch]);
       }
     }
   } else {
@@ -291,7 +398,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kSimThreads, 1) sim_
       const int slot = (tile >> 1) & 1;        // which of the team's two tiles of the four-tile span
       uint32_t* sdbuf = sD_team + ((tile >> 2) & 1) * (kBM * kDPitch);
       uint32_t* sdw = sdbuf + rl * kDPitch + slot * kTileWords + cg * kChunks;
-      bool ok = __all_sync(0xffffffffu, ptx::mbar_wait(acc_full + team, (it >> 1) & 1, abort_flag));
+      bool ok = __all_sync(0xffffffffu, ptx::mbar_wait(acc_full + team, (it >> 1) & 1, abort_flag, wait_cycles));
       if (ok && !live_block) {
         if (lane == 0) mbar_arrive_leader(acc_empty + team);
         ok = false;
@@ -397,6 +504,10 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kSimThreads, 1) sim_
   __syncwarp();
   ptx::tc_fence_before();
   __syncthreads();
+  if (kEmit && threadIdx.x == 0) {
+    const int cap = p.rec_per_tile * ((p.batch.max_len + kBN - 1) / kBN - (int)(blockIdx.x >> 1));
+    p.rec_cnt[(long long)unit * gridDim.x + blockIdx.x] = min(*rec_used, cap);
+  }
   if (*abort_flag) {
     if (threadIdx.x == 0) atomicExch(&p.hdr[kHdrStatus], (uint32_t)SPINDLEKV_TIMEOUT);
     __nanosleep(100000);  // let any bulk copy still in flight land before the block retires
@@ -406,6 +517,32 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kSimThreads, 1) sim_
     ptx::tc_fence_after();
     tmem_dealloc_pair(tmem_base, 512);
   }
+}
+
+// Self-test of the bounded mbarrier wait: nobody ever arrives on the barrier, so the wait must run out
+// after `wait_cycles`, and the block reports TIMEOUT the way the kernels above do.
+__global__ void mbar_selftest_kernel(uint32_t* hdr, long long wait_cycles) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_sh;
+  volatile int* abort_flag = &abort_sh;
+  if (threadIdx.x == 0) {
+    ptx::mbar_init(&bar, 1);
+    abort_sh = 0;
+    ptx::fence_barrier_init();
+  }
+  __syncthreads();
+  const bool ok = ptx::mbar_wait(&bar, 0, abort_flag, wait_cycles);   // every thread waits; the first to give up releases the rest
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    if (*abort_flag) atomicExch(&hdr[kHdrStatus], (uint32_t)SPINDLEKV_TIMEOUT);
+    if (ok) hdr[kHdrLive] = 0xBADu;   // must not happen
+  }
+}
+
+spindlekv_status selftest_mbarrier_impl(uint32_t* hdr, long long wait_cycles, cudaStream_t st) {
+  if (cudaMemsetAsync(hdr, 0, kHeaderBytes, st) != cudaSuccess) return SPINDLEKV_CUDA;
+  mbar_selftest_kernel<<<1, 64, 0, st>>>(hdr, wait_cycles);
+  return cudaGetLastError() == cudaSuccess ? SPINDLEKV_OK : SPINDLEKV_CUDA;
 }
 
 // ---- host -----------------------------------------------------------------------------------------
@@ -496,13 +633,32 @@ bool sim_tc_available() {
   return ok[dev] == 1;
 }
 
+template <int D, bool kEmit>
+static spindlekv_status launch_sim_tc_one(const CUtensorMap& map, const CUtensorMap& emap, const SimTcParams& p, dim3 grid,
+                                          cudaStream_t st) {
+  static PerDeviceOnce once;
+  const int dev = PerDeviceOnce::current();
+  if (dev < 0) return SPINDLEKV_CUDA;
+  if (!once.done[dev]) {
+    if (cudaFuncSetAttribute(sim_tc_kernel<D, kEmit>, cudaFuncAttributeMaxDynamicSharedMemorySize, SimSmem<D>::TOTAL) != cudaSuccess)
+      return SPINDLEKV_CUDA;
+    once.done[dev] = true;
+  }
+  sim_tc_kernel<D, kEmit><<<grid, kSimThreads, SimSmem<D>::TOTAL, st>>>(map, emap, p);
+  return SPINDLEKV_OK;
+}
+
+// `pool`: where candidate records go.  emit = true: every unit's candidates are written as records (units that do
+// not fit raise their overflow flag).  emit = false: the bit matrix, for the units whose overflow flag is set, or,
+// without a pool, for every unit.
 spindlekv_status launch_sim_tc(const spindlekv_tensor& Gamma, const spindlekv_batch& b, int n_kv_heads, int head_dim,
                                const void* ext, uint32_t* adj, uint32_t* flags, uint32_t* hdr, bool skip_empty,
-                               cudaStream_t st) {
+                               const SimRecordPool* pool, bool emit, long long wait_cycles, cudaStream_t st) {
   const int units = b.n_layers * b.n_seqs * n_kv_heads;
   CUtensorMap map, emap;
   if (!make_tensor_map_bf16(&map, Gamma, b, n_kv_heads, head_dim, 128)) return SPINDLEKV_CUDA;
   if (!make_ext_map(&emap, ext, units, row_words_for(b.max_len) * 32)) return SPINDLEKV_CUDA;
+  if (emit && !pool) return SPINDLEKV_INVALID_ARG;
   SimTcParams p;
   p.batch = make_batch(b);
   p.n_kv_heads = n_kv_heads;
@@ -511,29 +667,18 @@ spindlekv_status launch_sim_tc(const spindlekv_tensor& Gamma, const spindlekv_ba
   p.flags = flags;
   p.hdr = hdr;
   p.skip_empty = skip_empty ? 1 : 0;
+  p.rec = pool ? pool->rec : nullptr;
+  p.rec_cnt = pool ? pool->rec_cnt : nullptr;
+  p.ovf = pool ? pool->ovf : nullptr;
+  p.rec_per_tile = pool ? pool->rec_per_tile : 0;
+  p.unit_rec_cap = pool ? rec_unit_capacity(ceil_div(b.max_len, kBN), pool->rec_per_tile) : 0;
+  p.wait_cycles = wait_cycles;
   dim3 grid(2 * ceil_div(b.max_len, 2 * kBM), units);   // whole pairs
   LaunchScope ls(KC_SIM, st);
-  if (head_dim == 128) {
-    static PerDeviceOnce once;
-    const int dev = PerDeviceOnce::current();
-    if (dev < 0) return SPINDLEKV_CUDA;
-    if (!once.done[dev]) {
-      if (cudaFuncSetAttribute(sim_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, SimSmem<128>::TOTAL) != cudaSuccess)
-        return SPINDLEKV_CUDA;
-      once.done[dev] = true;
-    }
-    sim_tc_kernel<128><<<grid, kSimThreads, SimSmem<128>::TOTAL, st>>>(map, emap, p);
-  } else {
-    static PerDeviceOnce once;
-    const int dev = PerDeviceOnce::current();
-    if (dev < 0) return SPINDLEKV_CUDA;
-    if (!once.done[dev]) {
-      if (cudaFuncSetAttribute(sim_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, SimSmem<64>::TOTAL) != cudaSuccess)
-        return SPINDLEKV_CUDA;
-      once.done[dev] = true;
-    }
-    sim_tc_kernel<64><<<grid, kSimThreads, SimSmem<64>::TOTAL, st>>>(map, emap, p);
-  }
+  spindlekv_status rs;
+  if (head_dim == 128) rs = emit ? launch_sim_tc_one<128, true>(map, emap, p, grid, st) : launch_sim_tc_one<128, false>(map, emap, p, grid, st);
+  else rs = emit ? launch_sim_tc_one<64, true>(map, emap, p, grid, st) : launch_sim_tc_one<64, false>(map, emap, p, grid, st);
+  if (rs != SPINDLEKV_OK) return rs;
   return cudaGetLastError() == cudaSuccess ? SPINDLEKV_OK : SPINDLEKV_CUDA;
 }
 

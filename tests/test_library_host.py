@@ -12,9 +12,13 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
 def _declared():
-    text = open(os.path.join(ROOT, "include", "spindlekv.h")).read()
-    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\b(spindlekv_[a-z_]+)\s*\(", text)))
+    names = set()
+    inc = os.path.join(ROOT, "include")
+    for fn in sorted(os.listdir(inc)):
+        if fn.endswith(".h"):
+            text = re.sub(r"/\*.*?\*/", "", open(os.path.join(inc, fn)).read(), flags=re.S)
+            names |= set(re.findall(r"\b(spindlekv_[a-z_]+)\s*\(", text))
+    return sorted(names)
 
 
 def test_library_exports_every_declared_symbol():
@@ -147,3 +151,25 @@ def test_allocation_free_entry_point_checks_its_arguments_like_the_ordinary_one(
     assert B.spindlekv_workspace_bytes(B.Config(4, 8, 2, 128, 32, 2, budget_tokens=300.0),
                                        B.Batch(16, 1, 16384, 16384), B.WS_EVICT) > B.NOALLOC_SCRATCH_BYTES
     assert call(K=f32, Q=f32, b=big) == B.WORKSPACE_TOO_SMALL
+
+
+def test_limits_can_be_tightened_and_restored():
+    from paper_2507_06517_b200 import binding as B
+    defaults = [B.spindlekv_get_tuning(k) for k in range(4)]
+    assert defaults[B.TUNE_RECORDS_PER_TILE] == 512
+    try:
+        B.spindlekv_set_tuning(B.TUNE_RECORDS_PER_TILE, 7)
+        B.spindlekv_set_tuning(B.TUNE_GREEDY_ROUND_CAP, 1)
+        assert B.spindlekv_get_tuning(B.TUNE_RECORDS_PER_TILE) == 7 and B.spindlekv_get_tuning(B.TUNE_GREEDY_ROUND_CAP) == 1
+        B.spindlekv_set_tuning(B.TUNE_RECORDS_PER_TILE, 100000)      # never above what the workspace is sized for
+        assert B.spindlekv_get_tuning(B.TUNE_RECORDS_PER_TILE) == 512
+        with pytest.raises(B.SpindleKVError):
+            B.spindlekv_set_tuning(99, 1)
+        assert B.spindlekv_get_tuning(99) == -1
+    finally:
+        for k in range(4):
+            B.spindlekv_set_tuning(k, -1)
+    assert [B.spindlekv_get_tuning(k) for k in range(4)] == defaults
+    # the self-tests check their arguments before launching anything
+    assert B._lib.spindlekv_selftest_grid_barrier_timeout(None, 100, None) == B.INVALID_ARG
+    assert B._lib.spindlekv_selftest_mbarrier_timeout(256, 0, None) == B.INVALID_ARG

@@ -80,7 +80,7 @@ def test_noalloc_on_the_tensor_core_kernel_and_its_status_word():
         _both_ways(wl)
         status, _ = B.spindlekv_poll_status(None)
         assert status == B.OK
-    many = wl.replace(n_layers=12, seq_lens=(6000,), name="noalloc-tc-12")   # row statistics of 12 such layers would not fit 8 MiB
+    many = wl.replace(n_layers=12, seq_lens=(6000,), budget_tokens=1200.0, name="noalloc-tc-12")   # row statistics of 12 such layers would not fit 8 MiB
     assert B.spindlekv_workspace_bytes(make_config(many), B.Batch(12, 1, 6000, 6000), B.WS_EVICT) > B.NOALLOC_SCRATCH_BYTES
     _both_ways(many)
     assert B.spindlekv_poll_status(None)[0] == B.OK
