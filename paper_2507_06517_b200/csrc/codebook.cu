@@ -35,8 +35,8 @@ struct CodebookParams {
   int32_t* owner;        // [units][max_len]
   int32_t* pickdeg;      // [units][max_len], -1 = not a centre
   int32_t* rank;         // [units][max_len] entry number of a centre
-  int32_t* ell;          // [kEll][units][max_len] neighbour lists of rows with few neighbours, entry-major
-  int32_t* ell_cnt;      // [units][max_len] list length; -1: use the bit row; -1 - n (n > kEll): the n neighbours are in `csr`
+  int32_t* lists;        // [units][list_cap] neighbour lists, one contiguous run per row, starting at lbase[row]
+  int32_t* ell_cnt;      // [units][max_len] list length n <= kEll; -1: use the bit row; -1 - n: a list of n > kEll neighbours
   int32_t* dense_rows;   // rows (unit * max_len + token) with more than kEll neighbours; count in the header
   uint32_t* flags;       // [units][row_words][row_words/2] bit r of word [w][c]: chunk c (64 columns) of row 32w+r may hold a bit
   uint32_t* hdr;
@@ -49,9 +49,8 @@ struct CodebookParams {
   int32_t* ovf;          // [units] != 0: the unit goes through the bit matrix (records did not fit, or no records at all)
   int rec_per_tile, n_blocks;
   long long unit_rec_cap;
-  int32_t* csr;          // [units][long_cap] neighbour lists of rows with more than kEll neighbours (record path)
-  int32_t* lbase;        // [units][max_len] start of such a row's list within its unit's part of `csr`
-  int long_cap;
+  int32_t* lbase;        // [units][max_len] start of a row's list within its unit's part of `lists`
+  int list_cap;          // entries per unit (at least kEll per row: the bit-matrix path gives every row kEll slots)
   uint32_t spin_limit;   // polls after which a grid barrier gives up
   int round_cap;         // rounds after which the greedy cover gives up
 };
@@ -243,8 +242,8 @@ __device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long v)
 // chunks, eight per lane, and transposes them into per-row occupancy words); only those chunks of the bit
 // row are read, several at a time.  Written per row:
 // the initial degree (Eq. (10)) and key, and, for rows with at most kEll neighbours (the row itself
-// not counted), the ascending list of those neighbours, stored entry-major (`ell[k][row]`) so that
-// the threads of a warp read consecutive words.  Rows with more neighbours keep using their bit row
+// not counted), the ascending list of those neighbours in the row's kEll slots of `lists`.
+// Rows with more neighbours keep using their bit row
 // and are appended to a list of dense rows.  A token with no neighbour at all is settled here: it is
 // a centre with pick degree 1 (Algorithm 1 reaches it with exactly that degree, whenever it does).
 constexpr int kEll = 32;
@@ -264,10 +263,10 @@ __global__ void __launch_bounds__(256, 5) extract_kernel(CodebookParams p) {
   const int l = seq_len(p.batch, layer, s, j);
   const bool exists = u < l;
   const int64_t idx = (int64_t)unit * ML + (exists ? u : 0);
-  const int64_t n_rows = (int64_t)p.n_units * ML;
   const int own = u >> 6;   // the chunk that holds the token's own bit
   const uint32_t* fl = p.flags + ((int64_t)unit * RW + (u >> 5)) * NC;
   const uint2* row2 = reinterpret_cast<const uint2*>(p.adj + idx * RW);
+  int32_t* my_list = p.lists + (int64_t)unit * p.list_cap + (int64_t)(exists ? u : 0) * kEll;   // kEll slots per row
   TransposeLane tr;
   tr.init(lane);
   int cnt = 1, k = 0;
@@ -315,7 +314,7 @@ __global__ void __launch_bounds__(256, 5) extract_kernel(CodebookParams p) {
           while (m && k < kEll) {
             const int b = __ffs(m) - 1;
             m &= m - 1;
-            p.ell[(int64_t)k * n_rows + idx] = cs[i] * 64 + q * 32 + b;
+            my_list[k] = cs[i] * 64 + q * 32 + b;
             ++k;
           }
         }
@@ -327,6 +326,7 @@ __global__ void __launch_bounds__(256, 5) extract_kernel(CodebookParams p) {
     p.deg[idx] = cnt;
     p.key[idx] = ((unsigned long long)(uint32_t)cnt << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)u);
     p.ell_cnt[idx] = cnt - 1 <= kEll ? cnt - 1 : -1;
+    p.lbase[idx] = u * kEll;
     p.pickdeg[idx] = cnt == 1 ? 1 : -1;   // -1: not a centre (until the greedy cover picks it)
     if (cnt == 1) {
       p.owner[idx] = u;
@@ -345,15 +345,17 @@ __global__ void __launch_bounds__(256, 5) extract_kernel(CodebookParams p) {
 
 // ---- neighbour lists from candidate records ------------------------------------------------------
 // One block per unit that fitted its record pool.  A record is a non-zero word of the strict upper
-// triangle: every set bit is a pair (a, b), a < b, and is entered into both tokens' lists.  Degrees are
-// counted in shared memory (a word per token: neighbours in the low half, fill cursor in the high half),
-// then the pairs are entered: tokens with at most kEll neighbours into the entry-major lists that the
-// greedy kernels read (`ell`), the others into one contiguous list each (`csr`).  The order of a list
-// depends on the order in which the atomics land; nothing downstream depends on it (maxima, counts and
-// ownership by the single centre within reach are all independent of it).  Everything else the bit-matrix
-// path's extraction pass leaves behind is written here too: degree, key, live masks, settled isolated
-// tokens, the list of rows with many neighbours.  A unit whose long lists do not fit `long_cap` raises its
-// overflow flag and goes through the bit matrix instead.
+// triangle: every set bit is a pair (a, b), a < b, and is entered into both tokens' lists.  First the
+// degrees are counted in shared memory (one word per token), then a prefix sum turns the counts into the
+// start of every token's list within the unit's part of `lists`, then the pairs are entered, the shared
+// word of a token serving as its fill cursor.  The lists of a unit are contiguous and small (two entries
+// per pair), so the scattered 4-byte stores of the last step meet in the L2 cache.  The order inside a
+// list depends on the order in which the atomics land; nothing downstream depends on it (maxima, counts
+// and ownership by the single centre within reach are all independent of it).  Everything else the
+// bit-matrix path's extraction pass leaves behind is written here too: degree, key, live masks, settled
+// isolated tokens, the list of rows with more than kEll neighbours (which the greedy kernels walk a warp
+// per row).  A unit whose lists do not fit `list_cap` raises its overflow flag and goes through the bit
+// matrix instead.
 constexpr int kBuildThreads = 1024;
 
 template <typename F>
@@ -379,19 +381,17 @@ __device__ __forceinline__ void for_each_record(const CodebookParams& p, int uni
 }
 
 __global__ void __launch_bounds__(kBuildThreads) build_lists_kernel(CodebookParams p) {
-  extern __shared__ uint32_t cur[];   // [row_words * 32]
-  __shared__ int long_total, long_used;
+  extern __shared__ uint32_t cur[];   // [row_words * 32]: degree, then start of the list, then fill cursor
+  __shared__ int warp_total[32];
   const int unit = blockIdx.x;
   if (p.ovf[unit]) return;
   int layer, s, j;
   cb_decode(p, unit, layer, s, j);
   const int l = seq_len(p.batch, layer, s, j);
   const int RW = p.row_words, NP = RW * 32, ML = p.batch.max_len;
-  const int64_t n_rows = (int64_t)p.n_units * ML;
   const int64_t row0 = (int64_t)unit * ML;
-  const int tid = threadIdx.x, lane = tid & 31;
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   for (int u = tid; u < NP; u += kBuildThreads) cur[u] = 0u;
-  if (tid == 0) { long_total = 0; long_used = 0; }
   __syncthreads();
   // Eq. (10) without the token itself: both ends of every pair
   for_each_record(p, unit, [&](int a, int b0, uint32_t bits) {
@@ -402,63 +402,67 @@ __global__ void __launch_bounds__(kBuildThreads) build_lists_kernel(CodebookPara
     }
   });
   __syncthreads();
+  // prefix sum of the degrees: warp w owns the rows [w * seg, (w + 1) * seg) and walks them 32 at a time;
+  // first the warps' totals (and the decision whether the lists fit), then the starts and all per-row outputs
+  const int seg = ((NP + 1023) / 1024) * 32;   // rows per warp, a multiple of 32
+  const int u_end = min((wid + 1) * seg, NP);
   {
-    int mine = 0;
-    for (int u = tid; u < l; u += kBuildThreads) {
-      const int d = (int)cur[u];
-      if (d > kEll) mine += d;
-    }
+    int run = 0;
+    for (int u0 = wid * seg; u0 < u_end; u0 += 32) run += (int)cur[u0 + lane];
 #pragma unroll
-    for (int o = 16; o >= 1; o >>= 1) mine += __shfl_xor_sync(0xffffffffu, mine, o);
-    if (lane == 0 && mine) atomicAdd(&long_total, mine);
+    for (int o = 16; o >= 1; o >>= 1) run += __shfl_xor_sync(0xffffffffu, run, o);
+    if (lane == 0) warp_total[wid] = run;
   }
   __syncthreads();
-  if (long_total > p.long_cap) {
+  int run = 0, total = 0;
+  for (int w = 0; w < 32; ++w) {
+    const int t = warp_total[w];
+    if (w < wid) run += t;
+    total += t;
+  }
+  if (total > p.list_cap) {            // the same decision in every thread
     if (tid == 0) p.ovf[unit] = 1;
     return;
   }
-  for (int u = tid; u < NP; u += kBuildThreads) {
+  for (int u0 = wid * seg; u0 < u_end; u0 += 32) {
+    const int u = u0 + lane;
     const bool exists = u < l;
-    const int d = exists ? (int)cur[u] : 0;
+    const int d = (int)cur[u];         // 0 beyond the sequence
+    int inc = d;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int n = __shfl_up_sync(0xffffffffu, inc, o);
+      if (lane >= o) inc += n;
+    }
+    const int start = run + inc - d;
+    run += __shfl_sync(0xffffffffu, inc, 31);
+    cur[u] = (uint32_t)start;
     const int64_t idx = row0 + u;
-    bool live = false;
     if (exists) {
       const int cnt = d + 1;
       p.deg[idx] = cnt;
       p.key[idx] = ((unsigned long long)(uint32_t)cnt << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)u);
       p.ell_cnt[idx] = d <= kEll ? d : -1 - d;
+      p.lbase[idx] = start;
       p.pickdeg[idx] = cnt == 1 ? 1 : -1;   // a token without a neighbour is a centre of pick degree 1
-      if (cnt == 1) {
-        p.owner[idx] = u;
-      } else {
-        live = true;
-        if (d > kEll) {
-          p.lbase[idx] = atomicAdd(&long_used, d);
-          p.dense_rows[atomicAdd(&p.hdr[kHdrDenseCnt], 1u)] = (int32_t)idx;
-        }
-      }
+      if (cnt == 1) p.owner[idx] = u;
+      if (d > kEll) p.dense_rows[atomicAdd(&p.hdr[kHdrDenseCnt], 1u)] = (int32_t)idx;
     }
-    const uint32_t word = __ballot_sync(0xffffffffu, live);
+    const uint32_t word = __ballot_sync(0xffffffffu, exists && d > 0);   // tokens with a neighbour start live
     if (lane == 0) {
-      p.live0[(int64_t)unit * RW + (u >> 5)] = word;
-      p.live1[(int64_t)unit * RW + (u >> 5)] = word;
+      p.live0[(int64_t)unit * RW + (u0 >> 5)] = word;
+      p.live1[(int64_t)unit * RW + (u0 >> 5)] = word;
     }
   }
-  __syncthreads();   // lbase of this unit's long rows is complete (read back below through L2)
-  int32_t* csr = p.csr + (int64_t)unit * p.long_cap;
-  auto enter = [&](int a, int b, uint32_t old) {
-    const int d = (int)(old & 0xFFFFu), k = (int)(old >> 16);
-    if (d <= kEll) p.ell[(int64_t)k * n_rows + row0 + a] = b;
-    else csr[__ldcg(&p.lbase[row0 + a]) + k] = b;
-  };
+  __syncthreads();
+  int32_t* lists = p.lists + (int64_t)unit * p.list_cap;
   for_each_record(p, unit, [&](int a, int b0, uint32_t bits) {
-    uint32_t old_a = atomicAdd(&cur[a], (uint32_t)__popc(bits) << 16);
+    uint32_t at_a = atomicAdd(&cur[a], (uint32_t)__popc(bits));
     while (bits) {
       const int b = b0 + __ffs(bits) - 1;
       bits &= bits - 1;
-      enter(a, b, old_a);
-      old_a += 1u << 16;
-      enter(b, a, atomicAdd(&cur[b], 1u << 16));
+      lists[at_a++] = b;
+      lists[atomicAdd(&cur[b], 1u)] = a;
     }
   });
 }
@@ -509,9 +513,13 @@ __device__ __forceinline__ bool chunk_flagged(const uint32_t* fr, int chunk, int
 // Eight entries of a row's neighbour list at a time: the loads of one batch do not depend on each
 // other, so a row costs a few memory round trips instead of one per neighbour.
 constexpr int kBatch = 8;
-__device__ __forceinline__ void load_batch(const int32_t* ell_row, int64_t n_rows, int k0, int ec, int (&v)[kBatch]) {
+__device__ __forceinline__ void load_batch(const int32_t* list, int k0, int ec, int (&v)[kBatch]) {
 #pragma unroll
-  for (int i = 0; i < kBatch; ++i) v[i] = k0 + i < ec ? ell_row[(int64_t)(k0 + i) * n_rows] : -1;
+  for (int i = 0; i < kBatch; ++i) v[i] = k0 + i < ec ? list[k0 + i] : -1;
+}
+// a row's neighbour list
+__device__ __forceinline__ const int32_t* list_of(const CodebookParams& p, int unit, int64_t idx) {
+  return p.lists + (int64_t)unit * p.list_cap + p.lbase[idx];
 }
 // keeps only the entries that are live (others become -1)
 __device__ __forceinline__ void keep_live(const uint32_t* lv, int (&v)[kBatch]) {
@@ -529,7 +537,6 @@ __device__ __forceinline__ void keep_live(const uint32_t* lv, int (&v)[kBatch]) 
 template <bool kAllLive>
 __device__ __forceinline__ void max_of_listed_rows(const CodebookParams& p, const uint32_t* live, int64_t w, int lane) {
   const int ML = p.batch.max_len, RW = p.row_words;
-  const int64_t n_rows = (int64_t)p.n_units * ML;
   const uint32_t lvw = live[w];
   if (!((lvw >> lane) & 1u)) return;
   const int unit = (int)(w / RW), u = (int)(w - (int64_t)unit * RW) * 32 + lane;
@@ -538,10 +545,11 @@ __device__ __forceinline__ void max_of_listed_rows(const CodebookParams& p, cons
   if (ec < 0) return;                             // dense rows: separately
   const uint32_t* lv = live + (int64_t)unit * RW;
   const unsigned long long* key = p.key + (int64_t)unit * ML;
+  const int32_t* list = list_of(p, unit, idx);
   unsigned long long best = key[u];               // the token itself belongs to its closed neighbourhood
   for (int k0 = 0; k0 < ec; k0 += kBatch) {
     int v[kBatch];
-    load_batch(p.ell + idx, n_rows, k0, ec, v);
+    load_batch(list, k0, ec, v);
     if (!kAllLive) keep_live(lv, v);
     unsigned long long kv[kBatch];
 #pragma unroll
@@ -582,7 +590,6 @@ template <bool kAllLive>
 __device__ __forceinline__ void pick_listed_rows(const CodebookParams& p, const uint32_t* live, uint32_t* next, int64_t w,
                                                  int lane) {
   const int ML = p.batch.max_len, RW = p.row_words;
-  const int64_t n_rows = (int64_t)p.n_units * ML;
   const uint32_t lvw = live[w];
   if (!((lvw >> lane) & 1u)) return;
   const int unit = (int)(w / RW), u = (int)(w - (int64_t)unit * RW) * 32 + lane;
@@ -593,10 +600,11 @@ __device__ __forceinline__ void pick_listed_rows(const CodebookParams& p, const 
   if (p.m1[idx] != mykey) return;
   const uint32_t* lv = live + (int64_t)unit * RW;
   const unsigned long long* m1 = p.m1 + (int64_t)unit * ML;
+  const int32_t* list = list_of(p, unit, idx);
   bool ok = true;
   for (int k0 = 0; k0 < ec && ok; k0 += kBatch) {
     int v[kBatch];
-    load_batch(p.ell + idx, n_rows, k0, ec, v);
+    load_batch(list, k0, ec, v);
     if (!kAllLive) keep_live(lv, v);
     unsigned long long mv[kBatch];
 #pragma unroll
@@ -609,7 +617,7 @@ __device__ __forceinline__ void pick_listed_rows(const CodebookParams& p, const 
   uint32_t* nx = next + (int64_t)unit * RW;
   for (int k0 = 0; k0 < ec; k0 += kBatch) {
     int v[kBatch];
-    load_batch(p.ell + idx, n_rows, k0, ec, v);
+    load_batch(list, k0, ec, v);
     if (!kAllLive) keep_live(lv, v);
 #pragma unroll
     for (int i = 0; i < kBatch; ++i)
@@ -659,18 +667,15 @@ __device__ __forceinline__ void pick_dense_row(const CodebookParams& p, const ui
   }
 }
 
-// The same three steps for a row whose `n` neighbours (more than kEll) are listed in `csr` (record path): a warp
-// walks the list, 32 entries at a time.
-__device__ __forceinline__ const int32_t* long_list(const CodebookParams& p, int unit, int64_t idx) {
-  return p.csr + (int64_t)unit * p.long_cap + p.lbase[idx];
-}
+// The same three steps for a row whose `n` neighbours (more than kEll) are listed (record path): a warp walks
+// the list, 32 entries at a time.
 
 __device__ __forceinline__ void degree_of_long_row(const CodebookParams& p, const uint32_t* live, int64_t idx, int n, int lane) {
   const int ML = p.batch.max_len, RW = p.row_words;
   const int unit = (int)(idx / ML), u = (int)(idx - (int64_t)unit * ML);
   const uint32_t* lv = live + (int64_t)unit * RW;
   if (!is_live(lv, u)) return;
-  const int32_t* list = long_list(p, unit, idx);
+  const int32_t* list = list_of(p, unit, idx);
   int cnt = 0;
   for (int k = lane; k < n; k += 32) cnt += is_live(lv, list[k]) ? 1 : 0;
 #pragma unroll
@@ -687,7 +692,7 @@ __device__ __forceinline__ void max_of_long_row(const CodebookParams& p, const u
   const uint32_t* lv = live + (int64_t)unit * RW;
   if (!is_live(lv, u)) return;
   const unsigned long long* key = p.key + (int64_t)unit * ML;
-  const int32_t* list = long_list(p, unit, idx);
+  const int32_t* list = list_of(p, unit, idx);
   unsigned long long best = lane == 0 ? key[u] : 0ull;   // the token itself belongs to its closed neighbourhood
   for (int k = lane; k < n; k += 32) {
     const int v = list[k];
@@ -711,7 +716,7 @@ __device__ __forceinline__ void pick_long_row(const CodebookParams& p, const uin
   const unsigned long long* m1 = p.m1 + (int64_t)unit * ML;
   int32_t* owner = p.owner + (int64_t)unit * ML;
   uint32_t* nx = next + (int64_t)unit * RW;
-  const int32_t* list = long_list(p, unit, idx);
+  const int32_t* list = list_of(p, unit, idx);
   bool ok = true;
   for (int k = lane; k < n; k += 32) {
     const int v = list[k];
@@ -775,7 +780,6 @@ __global__ void __launch_bounds__(512) greedy_kernel(CodebookParams p) {
   const int64_t nwarps = (int64_t)gridDim.x * warps_per_block;
   const int64_t gthread = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   const int ML = p.batch.max_len, RW = p.row_words, RW4 = RW >> 2;
-  const int64_t n_rows = (int64_t)p.n_units * ML;
   const int64_t n_words = (int64_t)p.n_units * RW;
   const int n_dense = (int)*reinterpret_cast<volatile uint32_t*>(&p.hdr[kHdrDenseCnt]);
   uint32_t target = 0;
@@ -802,10 +806,11 @@ __global__ void __launch_bounds__(512) greedy_kernel(CodebookParams p) {
         const int ec = p.ell_cnt[idx];
         if (ec < 0) continue;                       // dense rows: below
         const uint32_t* lv = live + (int64_t)unit * RW;
+        const int32_t* list = list_of(p, unit, idx);
         int cnt = 1;
         for (int k0 = 0; k0 < ec; k0 += kBatch) {
           int v[kBatch];
-          load_batch(p.ell + idx, n_rows, k0, ec, v);
+          load_batch(list, k0, ec, v);
           keep_live(lv, v);
 #pragma unroll
           for (int i = 0; i < kBatch; ++i) cnt += v[i] >= 0 ? 1 : 0;
@@ -1051,12 +1056,13 @@ __global__ void __launch_bounds__(kFinalThreads) finalize_kernel(CodebookParams 
 
 struct CodebookLayout {
   size_t ext, ell, ell_cnt, dense_rows, flags, adj, deg, key, m1, live0, live1, owner, pickdeg, rank, total;
-  size_t ovf, rec_cnt, lbase, csr, rec;   // candidate records (tensor-core path)
-  int rec_per_tile, n_blocks, long_cap;
+  size_t ovf, rec_cnt, lbase, rec;   // candidate records (tensor-core path)
+  int rec_per_tile, n_blocks, list_cap;
 };
 
-// Neighbour-list entries per unit that the record path may spend on rows with more than kEll neighbours.
-static int long_list_capacity(int max_len) { return 64 * max_len; }
+// Neighbour-list entries per unit: the bit-matrix path gives every row kEll slots; the record path may spend
+// twice that on the whole unit, however the entries are spread over the rows.
+static int list_capacity(int max_len) { return 2 * kEll * max_len; }
 // The record path counts degrees in one 32-bit word per token in shared memory.
 static bool record_path_fits(int max_len) { return row_words_for(max_len) * 32 <= 49152; }
 
@@ -1075,18 +1081,17 @@ static CodebookLayout codebook_layout(const spindlekv_config& cfg, const spindle
   L.pickdeg = take(units * ML * 4);
   L.rank = take(units * ML * 4);
   L.ext = take(2 * units * RW * 32 * 16 * 2);
-  L.ell = take(units * ML * 32 * 4);
+  L.list_cap = list_capacity(b.max_len);
+  L.ell = take(units * (size_t)L.list_cap * 4);
   L.ell_cnt = take(units * ML * 4);
   L.dense_rows = take(units * ML * 4);
   L.flags = take(units * (RW / 2) * RW * 4);
   // candidate records: the overflow flags and the per-block counts sit side by side (one clearing pass)
   L.rec_per_tile = record_path_fits(b.max_len) ? rec_per_tile : 0;
   L.n_blocks = 2 * ceil_div(b.max_len, 256);
-  L.long_cap = long_list_capacity(b.max_len);
   L.ovf = take(units * 4);
   L.rec_cnt = take(units * L.n_blocks * 4);
   L.lbase = take(units * ML * 4);
-  L.csr = take(L.rec_per_tile ? units * (size_t)L.long_cap * 4 : 0);
   L.rec = take(L.rec_per_tile ? units * (size_t)rec_unit_capacity(L.n_blocks / 2, L.rec_per_tile) * 8 : 0);
   L.adj = off;
   if (adj_in_ws) take(units * ML * RW * 4);
@@ -1149,7 +1154,7 @@ spindlekv_status codebook_shallow_impl(const spindlekv_config& cfg, const spindl
   p.owner = reinterpret_cast<int32_t*>(w + L.owner);
   p.pickdeg = reinterpret_cast<int32_t*>(w + L.pickdeg);
   p.rank = reinterpret_cast<int32_t*>(w + L.rank);
-  p.ell = reinterpret_cast<int32_t*>(w + L.ell);
+  p.lists = reinterpret_cast<int32_t*>(w + L.ell);
   p.ell_cnt = reinterpret_cast<int32_t*>(w + L.ell_cnt);
   p.dense_rows = reinterpret_cast<int32_t*>(w + L.dense_rows);
   p.flags = reinterpret_cast<uint32_t*>(w + L.flags);
@@ -1163,9 +1168,8 @@ spindlekv_status codebook_shallow_impl(const spindlekv_config& cfg, const spindl
   p.rec_per_tile = L.rec_per_tile;
   p.n_blocks = L.n_blocks;
   p.unit_rec_cap = records ? rec_unit_capacity(L.n_blocks / 2, L.rec_per_tile) : 0;
-  p.csr = reinterpret_cast<int32_t*>(w + L.csr);
   p.lbase = reinterpret_cast<int32_t*>(w + L.lbase);
-  p.long_cap = L.long_cap;
+  p.list_cap = L.list_cap;
   p.spin_limit = tune.spin_limit;
   p.round_cap = tune.round_cap;
   if (cudaMemsetAsync(w, 0, kHeaderBytes, st) != cudaSuccess) return SPINDLEKV_CUDA;
