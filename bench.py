@@ -80,9 +80,14 @@ def workload_config(wl, extra=None):
 
 # ---- CPU baseline: the checker, as it stands, on a bounded sample ------------------------------
 
-def oracle_sample_seconds(wl):
-    """Times the CPU checker on (shallow layer 0, head 0: K and V CodeBooks) and on one deep layer
-    (all heads) of sequence 0, and scales by unit counts to one whole step."""
+def oracle_sample_seconds(wl, gpu=None):
+    """Times the CPU checker on the K and V CodeBooks of two heads of shallow layer 0 and on one deep layer
+    (all heads) of sequence 0, and scales by unit counts to one whole step.
+
+    ``gpu`` (optional, only looked at outside the timed sections): the GPU's adjacency of the same CodeBook units
+    and its kept positions of the same deep layer; when given, the decisions that fall inside the 1e-4 margin
+    are counted against the checker's and everything outside the margin must agree.
+    """
     from oracle import spindlekv_oracle as O
     try:
         from threadpoolctl import threadpool_info
@@ -90,35 +95,64 @@ def oracle_sample_seconds(wl):
     except Exception:
         cores = os.cpu_count() or 1
     ns, nd = wl.n_shallow, wl.n_layers - wl.n_shallow
-    units = wl.batch * wl.n_kv_heads
     total = 0.0
     parts = []
+    margins = {"rel_margin": 1e-4}
     scale_len = wl.total_tokens / (wl.seq_lens[0])  # sequences other than 0: scaled by length
     if ns:
-        k, v = synth.unit_kv(wl, 0, 0, 0)
-        t0 = time.perf_counter()
-        O.codebook_shallow(k.astype(np.float64), wl.theta_k)
-        t1 = time.perf_counter()
-        O.codebook_shallow(v.astype(np.float64), wl.theta_v)
-        t2 = time.perf_counter()
+        heads = list(range(min(2, wl.n_kv_heads)))
+        spent = 0.0
+        near = {"K": 0, "V": 0}
+        flips = {"K": 0, "V": 0}
+        pairs = 0
+        for j in heads:
+            k, v = synth.unit_kv(wl, 0, 0, j)
+            for name, gamma, theta in (("K", k, wl.theta_k), ("V", v, wl.theta_v)):
+                t0 = time.perf_counter()
+                r = O.codebook_shallow(gamma.astype(np.float64), theta)
+                spent += time.perf_counter() - t0
+                m = np.triu(O.threshold_margin_mask(r["S"], theta, 1e-4), k=1)
+                near[name] += int(m.sum())
+                pairs += gamma.shape[0] * (gamma.shape[0] - 1) // 2
+                if gpu is not None:
+                    diff = np.triu(gpu["adj"][(name, j)] != r["G"], k=1)
+                    if np.any(diff & ~m):
+                        raise RuntimeError(f"adjacency of layer 0 head {j} {name} differs from the checker outside the 1e-4 margin")
+                    flips[name] += int(diff.sum())
         # cost grows with the square of the length; other sequences are scaled accordingly
         sq = sum(float(l) ** 2 for l in wl.seq_lens) / float(wl.seq_lens[0]) ** 2
-        total += ((t1 - t0) + (t2 - t1)) * ns * wl.n_kv_heads * sq
-        parts.append(f"layer 0 head 0 K+V CodeBooks ({t2 - t0:.1f} s)")
+        total += spent / len(heads) * ns * wl.n_kv_heads * sq
+        parts.append(f"layer 0 heads {heads} K+V CodeBooks ({spent:.1f} s)")
+        margins["similarity"] = {"units": [f"layer 0 head {j}" for j in heads], "pairs_per_gamma": pairs // 2,
+                                 "pairs_within_margin_of_theta": near,
+                                 "decided_differently_from_checker": flips if gpu is not None else None}
     if nd:
         lam = ns
         ks = np.stack([synth.unit_kv(wl, lam, 0, j)[0] for j in range(wl.n_kv_heads)])
         q = synth.window_queries(wl, lam, 0, list(ks))
         _, _, kplan = O.plan_layers(wl.n_layers, ns, wl.seq_lens, wl.window, wl.beta,
                                     reserve_ratio=wl.budget_frac, budget_tokens=wl.budget_tokens)
+        kk = int(kplan[lam, 0])
         t0 = time.perf_counter()
-        res = O.evict_deep(q.astype(np.float64), ks.astype(np.float64), int(kplan[lam, 0]))
+        res = O.evict_deep(q.astype(np.float64), ks.astype(np.float64), kk)
         for j in range(wl.n_kv_heads):
             O.gather_rows(ks[j], res["keep"][j])
         t1 = time.perf_counter()
         total += (t1 - t0) * nd * scale_len
         parts.append(f"layer {lam} all heads eviction ({t1 - t0:.1f} s)")
-    return total, cores, "extrapolated by unit count from: " + "; ".join(parts)
+        near_k, differ = 0, 0
+        for j in range(wl.n_kv_heads):
+            m = O.topk_margin_mask(res["scores"][j], kk, 1e-4)
+            near_k += int(m.sum())
+            if gpu is not None:
+                d = np.setxor1d(gpu["keep"][j][:kk], res["keep"][j][:kk])
+                if not np.all(m[d]):
+                    raise RuntimeError(f"kept set of layer {lam} head {j} differs from the checker outside the 1e-4 margin")
+                differ += int(d.size)
+        margins["top_k"] = {"unit": f"layer {lam}, sequence 0, {wl.n_kv_heads} heads", "k": kk,
+                            "positions_within_margin_of_kth_score": near_k,
+                            "kept_differently_from_checker": differ if gpu is not None else None}
+    return total, cores, "extrapolated by unit count from: " + "; ".join(parts), margins
 
 
 def run_reference(args, wl):
@@ -129,7 +163,7 @@ def run_reference(args, wl):
     sample = ""
     cores = 1
     for i in range(args.warmup + args.steps):
-        t, cores, sample = oracle_sample_seconds(wl)
+        t, cores, sample, _ = oracle_sample_seconds(wl)
         if i >= args.warmup:
             times.append(t)
         if sum(times) > 0 and (time.perf_counter() - T_START) > 240:
@@ -139,7 +173,7 @@ def run_reference(args, wl):
     line = {"metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": len(times),
             "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f64", "data": "synthetic", "impl": "reference",
-            "config": workload_config(wl),
+            "config": workload_config(wl, {"parallelism": f"replicas x{args.gpus}"}),
             "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
             "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
@@ -170,6 +204,13 @@ class ClockSampler:
     def _read(self):
         for line in self.proc.stdout:
             self.rows.append((time.perf_counter(), line.strip()))
+
+    def wait_until_sampling(self, timeout=5.0):
+        """Blocks until the first samples have arrived (the tool needs a moment to start), so that a short timed
+        region is not over before the first one."""
+        t_end = time.perf_counter() + timeout
+        while self.proc is not None and len(self.rows) < 2 and time.perf_counter() < t_end:
+            time.sleep(0.02)
 
     def stop(self, t0, t1):
         if self.proc is None:
@@ -250,8 +291,13 @@ def run_literal(args, wl):
     nk, nv = p.cb["K"]["n_entries"].cpu().numpy(), p.cb["V"]["n_entries"].cpu().numpy()
     kept = p.kept_host[:, 0].astype(np.float64)       # tokens kept per head (per query head when unfolded)
     heads = wl.n_q_heads if args.repeat else wl.n_kv_heads   # Eq. (15): h_g = h after a repeat
-    r1 = kept / wl.max_len
-    r2 = (nk[:, 0].sum(axis=1) + nv[:, 0].sum(axis=1)) / (2.0 * heads * kept)
+    # Eq. (15) per layer, evaluated by the library.  After a repeat h is the number of query heads: the CodeBooks of a
+    # KV head then stand for all its query heads, whose slots in the per-head arrays beyond the first stay empty.
+    pad = np.zeros(heads - wl.n_kv_heads, dtype=np.int32)
+    rr = [B.spindlekv_reserve_ratio(wl.max_len, int(kept[lam]), np.concatenate([nk[lam, 0], pad]),
+                                    np.concatenate([nv[lam, 0], pad])) for lam in range(wl.n_layers)]
+    r1 = np.array([x[0] for x in rr])
+    r2 = np.array([x[1] for x in rr])
     line = {"metric": METRIC + (", composition as written, GQA unfolded" if args.repeat else ", composition as written"), "value": wl.total_tokens * args.steps / (ms * 1e-3),
             "unit": UNIT, "n_gpus": 1, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic",
@@ -260,6 +306,33 @@ def run_literal(args, wl):
             "reserve_ratio": {"r1_mean": float(r1.mean()), "r2_mean": float(r2.mean()), "r1_r2_mean": float((r1 * r2).mean()),
                               "kept_first_last": [int(kept[0]), int(kept[-1])]}}
     print(json.dumps(line))
+
+
+def sampled_gpu_decisions(wl, p, dK, dV, dtype, dev):
+    """The GPU's adjacency of the CodeBook units and its kept positions of the evicting layer that the CPU-baseline
+    leg runs the checker on (outside every timed region)."""
+    from paper_2507_06517_b200 import binding as B
+    from paper_2507_06517_b200.pipeline import SpindleKVPass
+    out = {"adj": {}, "keep": None}
+    ns = wl.n_shallow
+    if ns:
+        l = wl.seq_lens[0]
+        one = B.Config(n_layers=1, n_q_heads=1, n_kv_heads=1, head_dim=wl.head_dim, window=1, n_shallow=1,
+                       budget_tokens=float(l), theta_k=wl.theta_k, theta_v=wl.theta_v)
+        q = SpindleKVPass(one, [l], dtype, device=dev, keep_adjacency=True)
+        for j in range(min(2, wl.n_kv_heads)):
+            for name, src in (("K", dK), ("V", dV)):
+                rows = (src[0, :l, j] if wl.packed else src[0, 0, j]).contiguous().reshape(1, 1, 1, l, wl.head_dim)
+                q.codebook(rows, name)
+                if q.device_status()["codebook"][0] != 0:
+                    raise RuntimeError("device status in the sampled CodeBook unit")
+                words = q.adj[0, :l].cpu().numpy().view(np.uint32)
+                bits = np.unpackbits(words.view(np.uint8), axis=1, bitorder="little")[:, :l].astype(bool)
+                out["adj"][(name, j)] = bits
+        del q
+    if wl.n_layers > ns:
+        out["keep"] = p.keep_idx[0, :, : wl.seq_lens[0]].cpu().numpy()
+    return out
 
 
 def run_native(args, wl):
@@ -324,6 +397,10 @@ def run_native(args, wl):
         if v[0] != 0:
             raise RuntimeError(f"device status {v} in {k}")
     sampler = ClockSampler(local_rank) if rank == 0 else None
+    if sampler:
+        sampler.wait_until_sampling()
+        for _ in range(3):   # the part is under load again when the timed region starts
+            step()
     B.spindlekv_launch_count(True)
     t0 = time.perf_counter()
     ms = timed(step, args.steps)
@@ -331,6 +408,17 @@ def run_native(args, wl):
     job_tokens = timed.tokens
     launches = B.spindlekv_launch_count(True)
     clocks = sampler.stop(t0, t1) if sampler else None
+
+    # the same steps once more, each with its own event pair: the median beside the mean
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    barrier()
+    for a, b in evs:
+        a.record()
+        step()
+        b.record()
+    barrier()
+    per_step = sorted(a.elapsed_time(b) for a, b in evs)
+    ms_median = sharding.aggregate(wl.total_tokens, statistics.median(per_step), dist, dev)[1]
 
     e2e = None
     if not args.no_e2e:
@@ -362,6 +450,17 @@ def run_native(args, wl):
     torch.cuda.synchronize(dev)
     kt = B.spindlekv_timing_read()
     B.spindlekv_timing_enable(False)
+
+    # counters of the CodeBook graph stage, per Gamma: the status block of a call holds its rounds, the units that went
+    # through the bit matrix and the neighbour-list entries built from candidate records
+    graph = {}
+    if p.n_shallow:
+        for g, src in (("K", dK), ("V", dV)):
+            p.codebook(src[:p.n_shallow], g)
+            stat, det = p.device_status()["codebook"]
+            if stat != 0:
+                raise RuntimeError(f"device status {stat} in the {g} CodeBook call")
+            graph[g] = {"greedy_rounds": det[0], "units_through_bit_matrix": det[2], "list_entries": det[3]}
 
     if rank != 0:
         if dist is not None:
@@ -401,29 +500,60 @@ def run_native(args, wl):
         rate = exps / (kernels["window_score"]["ms_per_step"] * 1e-3)
         kernels["window_score"]["exp_unit"] = {"exponentials_per_step": exps, "achieved_per_s": rate,
                                                "peak_per_s": peak, "frac": rate / peak, "sm_mhz": mhz}
+    if ns and graph:
+        # Graph stage, bytes that must move at least once per step (K and V calls together).  List building: the
+        # candidate records (8 bytes per similar pair, read), the lists (4 bytes per entry, written), and per token
+        # degree, key, list start and length, pick degree and live bit (24 bytes, written).  Greedy cover: every list
+        # entry read with the 8-byte key or neighbourhood maximum it points to, per-token key, maximum, owner and
+        # pick degree (24 bytes).  Numbering: pick degree, owner, rank, reference and centre position per token (20).
+        rows = 2 * ns * Hk * tok
+        ent = sum(v["list_entries"] for v in graph.values())
+        for name, nbytes in (("degree", ent // 2 * 8 + ent * 4 + rows * 24), ("greedy", ent * 12 + rows * 24),
+                             ("finalise", rows * 20)):
+            if name in kernels and kernels[name]["ms_per_step"] > 0:
+                gbs = nbytes / (kernels[name]["ms_per_step"] * 1e-3) / 1e9
+                kernels[name].update({"bound": "hbm (in fact: latency of dependent gathers; see profiles/)",
+                                      "algorithmic_bytes": nbytes, "achieved_gbs": gbs, "frac_of_hbm_peak": gbs / pk["hbm_gbs"]})
+        kernels["greedy"]["rounds"] = {g: v["greedy_rounds"] for g, v in graph.items()}
+        kernels["degree"]["units_through_bit_matrix"] = {g: v["units_through_bit_matrix"] for g, v in graph.items()}
+        kernels["degree"]["list_entries"] = {g: v["list_entries"] for g, v in graph.items()}
     roof = None
     if p.n_shallow and kt["similarity"][1]:
         sim_ms, sim_n = kt["similarity"]
         units_per_launch = 2 * wl.n_shallow * wl.n_kv_heads * wl.batch / (sim_n / args.steps)
         flops_per_step = sum(float(l) * (l - 1) * wl.head_dim for l in wl.seq_lens) * 2 * wl.n_shallow * wl.n_kv_heads
         achieved = flops_per_step * args.steps / (sim_ms * 1e-3) / 1e12
-        peak = pk["bf16_tflops_sustained"] if wl.dtype == "bf16" else pk["bf16_tflops_sustained"] / 32.0
+        mhz = (clocks or {}).get("sm_mhz") or 1965.0
+        if wl.dtype == "bf16":
+            bound, peak, peak_name = "tensor", pk["bf16_tflops_sustained"], "cuBLAS bf16 GEMM, sustained loop (MEASURED_PEAKS.json)"
+        else:
+            # fp32 inputs take the CUDA-core kernel: 128 fused multiply-adds per clock and SM, 148 SMs, sampled clock
+            bound, peak, peak_name = "alu", 2.0 * 128 * 148 * mhz * 1e6 / 1e12, "fp32 FMA rate at the sampled SM clock"
         traffic = None
         if not wl.packed and wl.max_len in SIMILARITY_TRAFFIC_BYTES_PER_UNIT and wl.head_dim == 128:
             traffic = SIMILARITY_TRAFFIC_BYTES_PER_UNIT[wl.max_len] * units_per_launch
-        roof = {"kernel": "similarity (Eq. 4, 9)", "bound": "tensor", "achieved": achieved, "peak": peak,
-                "unit": "TFLOP/s", "frac": achieved / peak, "traffic": traffic, "peak_source": pk_src,
+        roof = {"kernel": "similarity (Eq. 4, 9)", "bound": bound, "achieved": achieved, "peak": peak,
+                "unit": "TFLOP/s", "frac": achieved / peak, "traffic": traffic, "peak_source": pk_src, "peak_is": peak_name,
                 "avg_launch_ms": sim_ms / sim_n, "algorithmic_flops_per_launch": flops_per_step * args.steps / sim_n}
+        if wl.dtype == "bf16":
+            # the same achieved rate against the other denominators one may want: the cuBLAS burst figure, and the
+            # tensor pipe itself at the clock sampled during the run (nominal 2250 TFLOP/s dense bf16 at 1965 MHz)
+            roof["frac_of_cublas_sustained"] = achieved / pk["bf16_tflops_sustained"]
+            roof["frac_of_cublas_burst"] = achieved / pk["bf16_tflops"]
+            roof["frac_of_pipe_at_sampled_clock"] = achieved / (2250.0 * mhz / 1965.0)
+            roof["executed_over_useful"] = 9.0 / 8.0   # one K-step in nine carries the threshold
     line = {"metric": METRIC, "value": sharding.throughput(job_tokens, args.steps, ms), "unit": UNIT,
             "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps,
+            "ms_per_step_median": ms_median,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": wl.dtype,
             "data": "synthetic", "config": workload_config(wl, {"parallelism": f"replicas x{world}"}),
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roof, "kernels": kernels,
             "greedy_rounds": st.get("codebook", (0, [0]))[1][0]}
     if not args.no_cpu_baseline and world == 1:
-        sec, cores, sample = oracle_sample_seconds(wl)
+        sec, cores, sample, margins = oracle_sample_seconds(wl, sampled_gpu_decisions(wl, p, dK, dV, dtype, dev))
         line["cpu_baseline"] = {"value": wl.total_tokens / sec, "unit": UNIT, "cores": cores, "kind": "oracle",
                                 "sample": sample}
+        line["near_threshold"] = margins
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()

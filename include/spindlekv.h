@@ -111,6 +111,18 @@ typedef struct {
 spindlekv_status spindlekv_plan_layers(const spindlekv_config* cfg, int32_t n_seqs, const int32_t* seq_lens,
                                        int32_t* layer_mode, double* r_c_layer, int32_t* k_ctx);
 
+/*
+ * Reserve ratios of one layer, host only (Eq. (15) without its storage-type factor r3):
+ *   r1 = kept K and V tokens over all K and V tokens      = (2 h kept) / (2 h l)
+ *   r2 = CodeBook entries of K and V over kept K and V tokens = (sum_j |C_K,j| + sum_j |C_V,j|) / (2 h kept)
+ * with h = n_heads heads (the KV heads; the query heads when GQA was unfolded), l = seq_len tokens per head
+ * before the pass and `kept` tokens per head after eviction.  The layer keeps r1 * r2 of its cache rows.
+ *   entries_k, entries_v  host [n_heads]: CodeBook sizes per head
+ * INVALID_ARG for null pointers or non-positive sizes.
+ */
+spindlekv_status spindlekv_reserve_ratio(int32_t n_heads, int32_t seq_len, int32_t kept, const int32_t* entries_k,
+                                         const int32_t* entries_v, double* r1, double* r2);
+
 /* Bytes of device scratch the given call kind (SPINDLEKV_WS_*) needs for `batch`.  0 on bad arguments. */
 size_t spindlekv_workspace_bytes(const spindlekv_config* cfg, const spindlekv_batch* batch, int32_t which);
 
@@ -280,7 +292,8 @@ spindlekv_status spindlekv_reconstruct(const spindlekv_batch* batch, int32_t n_h
  *   device_status host out: SPINDLEKV_OK or SPINDLEKV_TIMEOUT
  *   detail        host out, optional [4]: {greedy rounds used, live tokens left, units of the call whose
  *                 adjacency was computed as a bit matrix (all of them for fp32 input; for bf16 input only
- *                 those whose candidate pairs did not fit the record pool), 0}
+ *                 those whose candidate pairs did not fit the record pool), neighbour-list entries built
+ *                 from candidate records (two per similar pair) over the other units}
  */
 spindlekv_status spindlekv_poll_status(const void* ws, int32_t* device_status, int32_t* detail);
 

@@ -54,6 +54,8 @@ def _load() -> C.CDLL:
     lib.spindlekv_status_string.argtypes = [C.c_int32]
     lib.spindlekv_plan_layers.restype = C.c_int32
     lib.spindlekv_plan_layers.argtypes = [C.POINTER(_Config), C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+    lib.spindlekv_reserve_ratio.restype = C.c_int32
+    lib.spindlekv_reserve_ratio.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
     lib.spindlekv_workspace_bytes.restype = C.c_size_t
     lib.spindlekv_workspace_bytes.argtypes = [C.POINTER(_Config), C.POINTER(_Batch), C.c_int32]
     lib.spindlekv_evict_deep.restype = C.c_int32
@@ -192,6 +194,16 @@ def spindlekv_plan_layers(cfg: Config, seq_lens: Sequence[int]):
     return mode, ratio, k_ctx
 
 
+def spindlekv_reserve_ratio(seq_len: int, kept: int, entries_k: Sequence[int], entries_v: Sequence[int]):
+    """Eq. (15)'s ``(r1, r2)`` of one layer from the CodeBook sizes per head (host arithmetic in the library)."""
+    ek = np.ascontiguousarray(entries_k, dtype=np.int32)
+    ev = np.ascontiguousarray(entries_v, dtype=np.int32)
+    r1, r2 = C.c_double(0.0), C.c_double(0.0)
+    st = _lib.spindlekv_reserve_ratio(int(ek.shape[0]), seq_len, kept, ek.ctypes.data, ev.ctypes.data, C.byref(r1), C.byref(r2))
+    _check(st, "spindlekv_reserve_ratio")
+    return float(r1.value), float(r2.value)
+
+
 def spindlekv_workspace_bytes(cfg: Config, batch: Batch, which: int) -> int:
     cc, bb = cfg.c(), batch.c()
     return int(_lib.spindlekv_workspace_bytes(C.byref(cc), C.byref(bb), which))
@@ -285,7 +297,7 @@ def spindlekv_reconstruct(batch: Batch, n_heads: int, head_dim: int, Cb: _Tensor
 
 
 def spindlekv_poll_status(ws: Optional[torch.Tensor]):
-    """Device status word of a workspace and ``[greedy rounds, live tokens left, units done as a bit matrix, 0]``.  ``None`` reads the
+    """Device status word of a workspace and ``[greedy rounds, live tokens left, units done as a bit matrix, list entries built from records]``.  ``None`` reads the
     built-in scratch of ``spindlekv_evict_deep_noalloc`` on the current device."""
     status = C.c_int32(0)
     detail = (C.c_int32 * 4)()

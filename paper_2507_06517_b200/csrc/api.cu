@@ -147,6 +147,19 @@ spindlekv_status spindlekv_plan_layers(const spindlekv_config* cfg, int32_t n_se
   return SPINDLEKV_OK;
 }
 
+spindlekv_status spindlekv_reserve_ratio(int32_t n_heads, int32_t seq_len, int32_t kept, const int32_t* entries_k,
+                                         const int32_t* entries_v, double* r1, double* r2) {
+  if (n_heads <= 0 || seq_len <= 0 || kept <= 0 || !entries_k || !entries_v || !r1 || !r2) return SPINDLEKV_INVALID_ARG;
+  double sum_k = 0.0, sum_v = 0.0;
+  for (int j = 0; j < n_heads; ++j) {
+    sum_k += (double)entries_k[j];
+    sum_v += (double)entries_v[j];
+  }
+  *r1 = (2.0 * (double)n_heads * (double)kept) / (2.0 * (double)n_heads * (double)seq_len);
+  *r2 = (sum_k + sum_v) / (2.0 * (double)n_heads * (double)kept);
+  return SPINDLEKV_OK;
+}
+
 size_t spindlekv_workspace_bytes(const spindlekv_config* cfg, const spindlekv_batch* batch, int32_t which) {
   if (!cfg_ok(cfg) || !batch_ok(batch, cfg->window)) return 0;
   if (which == SPINDLEKV_WS_EVICT) return evict_workspace_bytes(*cfg, *batch);
@@ -256,10 +269,10 @@ spindlekv_status spindlekv_poll_status(const void* ws, int32_t* device_status, i
   if (!device_status) return SPINDLEKV_INVALID_ARG;
   if (!ws) ws = noalloc_scratch_of_current_device();   // NULL: the built-in scratch of the allocation-free entry point
   if (!ws) return SPINDLEKV_INVALID_ARG;
-  int32_t h[4];
+  int32_t h[8];
   if (cudaMemcpy(h, ws, sizeof(h), cudaMemcpyDeviceToHost) != cudaSuccess) return SPINDLEKV_CUDA;
   *device_status = h[kHdrStatus];
-  if (detail) { detail[0] = h[kHdrRounds]; detail[1] = h[kHdrLive]; detail[2] = h[kHdrBitUnits]; detail[3] = 0; }
+  if (detail) { detail[0] = h[kHdrRounds]; detail[1] = h[kHdrLive]; detail[2] = h[kHdrBitUnits]; detail[3] = h[kHdrListEntries]; }
   return SPINDLEKV_OK;
 }
 

@@ -424,6 +424,7 @@ __global__ void __launch_bounds__(kBuildThreads) build_lists_kernel(CodebookPara
     if (tid == 0) p.ovf[unit] = 1;
     return;
   }
+  if (tid == 0) atomicAdd(&p.hdr[kHdrListEntries], (uint32_t)total);
   for (int u0 = wid * seg; u0 < u_end; u0 += 32) {
     const int u = u0 + lane;
     const bool exists = u < l;

@@ -11,12 +11,14 @@ namespace skv {
 
 // ---- status block at the start of every workspace -------------------------------------------
 // word 0: device status, 1: greedy rounds used, 2: live tokens left, 3: units whose neighbour lists came from a bit matrix,
+// 4: neighbour-list entries built from candidate records (both directions of every pair),
 // words 8..: barrier and counters of the cooperative greedy kernel.
 constexpr int kHeaderBytes = 256;
 constexpr int kHdrStatus = 0;
 constexpr int kHdrRounds = 1;
 constexpr int kHdrLive = 2;
 constexpr int kHdrBitUnits = 3;
+constexpr int kHdrListEntries = 4;
 constexpr int kHdrBarrier = 8;
 constexpr int kHdrLiveCnt0 = 9;   // two slots, alternated by round parity
 constexpr int kHdrLiveCnt1 = 10;

@@ -173,3 +173,16 @@ def test_limits_can_be_tightened_and_restored():
     # the self-tests check their arguments before launching anything
     assert B._lib.spindlekv_selftest_grid_barrier_timeout(None, 100, None) == B.INVALID_ARG
     assert B._lib.spindlekv_selftest_mbarrier_timeout(256, 0, None) == B.INVALID_ARG
+
+
+def test_reserve_ratio_matches_checker():
+    from paper_2507_06517_b200 import binding as B
+    rng = np.random.default_rng(5)
+    for _ in range(100):
+        h = int(rng.integers(1, 33))
+        l = int(rng.integers(64, 40000))
+        kept = int(rng.integers(1, l + 1))
+        ek, ev = rng.integers(1, kept + 1, size=h), rng.integers(1, kept + 1, size=h)
+        assert B.spindlekv_reserve_ratio(l, kept, ek, ev) == O.reserve_ratio_layer(l, kept, ek, ev)
+    with pytest.raises(B.SpindleKVError):
+        B.spindlekv_reserve_ratio(100, 0, [1], [1])
