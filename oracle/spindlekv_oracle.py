@@ -33,6 +33,14 @@ Readings taken where the text is silent, garbled or inconsistent:
 * Eq. (11): ``argmax`` ties go to the lower index; a CodeBook entry is the
   unit vector of the centre token (no averaging).
 * Zero vectors get ``gamma_hat = 0`` and therefore an entry of their own.
+* Rotary position embedding (the matrix R of Eq. (1), which the paper does not spell out): the
+  convention of the LLaMA / Mistral models the paper evaluates, i.e. element ``i < d_h/2`` is paired
+  with element ``i + d_h/2`` and the pair is rotated by the angle ``p * base**(-2 i / d_h)`` at
+  position ``p``.
+* Attention over the replaced cache at decode time (Section 3.4, after Eq. (14)): K is rebuilt as
+  ``C_K[r_K] (x) m_K`` from CodeBooks of pre-RoPE keys, rotated at each token's original position,
+  and scored against the rotated query; V is rebuilt as ``C_V[r_V] (x) m_V``; every cached token is
+  visible to the new query.
 * The shallow/deep split is an argument: layers ``< n_shallow`` build
   CodeBooks over all tokens, layers ``>= n_shallow`` evict, with the pyramid
   of Eq. (5)(6) laid over the evicting layers only.
@@ -452,3 +460,52 @@ def codebook_extend(C: np.ndarray, gamma_new: np.ndarray, theta: float,
         out_ref[left] = C.shape[0] + sub["ref"]
         C_ext = np.concatenate([C, sub["C"]], axis=0)
     return {"ref": out_ref, "mag": magnitudes(gamma_new), "C": C_ext, "S": S, "left": left, "sub": sub}
+
+
+# --------------------------------------------------------------------------
+# Decode-time attention over the replaced cache (Eq. (14), Eq. (1), Section 3.4 last paragraph)
+# --------------------------------------------------------------------------
+
+def rope_frequencies(d: int, base: float = 10000.0) -> np.ndarray:
+    """Angular steps ``omega_i = base**(-2 i / d)`` for ``i = 0 .. d/2 - 1``."""
+    return np.asarray(base, dtype=np.float64) ** (-2.0 * np.arange(d // 2, dtype=np.float64) / float(d))
+
+
+def rope(x: np.ndarray, positions: np.ndarray, base: float = 10000.0) -> np.ndarray:
+    """Rotary position embedding (the matrix R of Eq. (1)) of rows ``x[t]`` at positions ``positions[t]``.
+
+    Element ``i`` and element ``i + d/2`` form a pair that is rotated by ``positions[t] * omega_i``:
+    ``(a, b) -> (a cos - b sin, b cos + a sin)``.
+    """
+    x = np.asarray(x, dtype=np.float64)
+    d = x.shape[-1]
+    h = d // 2
+    ang = np.asarray(positions, dtype=np.float64)[..., None] * rope_frequencies(d, base)
+    c, s_ = np.cos(ang), np.sin(ang)
+    a, b = x[..., :h], x[..., h:]
+    return np.concatenate([a * c - b * s_, b * c + a * s_], axis=-1)
+
+
+def decode_attention(q: np.ndarray, pos_q: int, C_K: np.ndarray, r_K: np.ndarray, m_K: np.ndarray,
+                     C_V: np.ndarray, r_V: np.ndarray, m_V: np.ndarray, positions: Optional[np.ndarray] = None,
+                     base: float = 10000.0) -> Dict[str, np.ndarray]:
+    """One decode step of the query heads of a GQA group over the replaced cache of their KV head.
+
+    ``q`` is ``[h_n, d]``: the pre-RoPE queries of the new token at position ``pos_q``.  The CodeBooks were
+    built from pre-RoPE keys (Section 3.4), so: ``K = C_K[r_K] (x) m_K`` (Eq. (14)), rotated at each cached
+    token's own position (``positions[t]``, default ``t``); the query is rotated at ``pos_q``;
+    ``A = softmax(q K^T / sqrt(d))`` over all cached tokens (Eq. (1); every cached token precedes the
+    query); ``V = C_V[r_V] (x) m_V``; output ``A V``.  Returns ``out [h_n, d]`` and ``A [h_n, n]``.
+    """
+    q = np.asarray(q, dtype=np.float64)
+    n = np.asarray(r_K).shape[0]
+    d = q.shape[1]
+    positions = np.arange(n) if positions is None else np.asarray(positions)
+    K = rope(reconstruct(C_K, r_K, m_K), positions, base)
+    V = reconstruct(C_V, r_V, m_V)
+    qr = rope(q, np.full(q.shape[0], pos_q), base)
+    s = (qr @ K.T) / math.sqrt(d)
+    s = s - s.max(axis=1, keepdims=True)
+    e = np.exp(s)
+    A = e / e.sum(axis=1, keepdims=True)
+    return {"out": A @ V, "A": A}

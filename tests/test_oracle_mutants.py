@@ -12,6 +12,7 @@ from oracle import spindlekv_oracle as O
 
 import test_oracle_codebook
 import test_oracle_compose
+import test_oracle_decode
 import test_oracle_evict
 import test_oracle_plan
 
@@ -320,11 +321,52 @@ def _extend_without_offset(C, gamma_new, theta, ref_override=None, G_override=No
     return out
 
 
+def _rope(kind):
+    def rope(x, positions, base=10000.0):
+        x = np.asarray(x, dtype=np.float64)
+        d = x.shape[-1]
+        h = d // 2
+        ang = np.asarray(positions, dtype=np.float64)[..., None] * O.rope_frequencies(d, base)
+        c, s_ = np.cos(ang), np.sin(ang)
+        if kind == "clockwise":
+            s_ = -s_
+        if kind == "neighbouring_pairs":               # (2i, 2i+1) instead of (i, i + d/2)
+            a, b = x[..., 0::2], x[..., 1::2]
+            out = np.empty_like(x)
+            out[..., 0::2], out[..., 1::2] = a * c - b * s_, b * c + a * s_
+            return out
+        a, b = x[..., :h], x[..., h:]
+        return np.concatenate([a * c - b * s_, b * c + a * s_], axis=-1)
+    return rope
+
+
+def _frequencies_of_half_the_dimension(d, base=10000.0):
+    return np.asarray(base, dtype=np.float64) ** (-1.0 * np.arange(d // 2, dtype=np.float64) / float(d))
+
+
+def _decode(kind):
+    def decode_attention(q, pos_q, C_K, r_K, m_K, C_V, r_V, m_V, positions=None, base=10000.0):
+        q = np.asarray(q, dtype=np.float64)
+        n, d = np.asarray(r_K).shape[0], q.shape[1]
+        positions = np.arange(n) if (positions is None or kind == "positions_ignored") else np.asarray(positions)
+        K = O.reconstruct(C_K, r_K, np.ones(n) if kind == "key_magnitude_dropped" else m_K)
+        K = K if kind == "keys_not_rotated" else O.rope(K, positions, base)
+        V = O.reconstruct(C_V, r_V, np.ones(n) if kind == "value_magnitude_dropped" else m_V)
+        qr = q if kind == "query_not_rotated" else O.rope(q, np.full(q.shape[0], pos_q), base)
+        s = (qr @ K.T) / (1.0 if kind == "no_scale" else math.sqrt(d))
+        s = s - s.max(axis=1, keepdims=True)
+        e = np.exp(s)
+        A = e / e.sum(axis=1, keepdims=True)
+        return {"out": A @ V, "A": A}
+    return decode_attention
+
+
 _ORIGINAL = {"plan_layers": O.plan_layers, "codebook_extend": O.codebook_extend}
 
 _EVICT = (test_oracle_evict, test_oracle_compose)
 _CODEBOOK = (test_oracle_codebook, test_oracle_compose)
 _PLAN = (test_oracle_plan, test_oracle_compose)
+_DECODE = (test_oracle_decode,)
 
 MUTANTS = [
     ("logits not scaled by 1/sqrt(d)", "window_attention", _attention(scale=False), _EVICT),
@@ -365,11 +407,21 @@ MUTANTS = [
     ("reconstruction with a shared magnitude", "reconstruct", _reconstruct_centre_magnitude, _CODEBOOK),
     ("first suitable entry instead of the most similar", "match_entries", _match("first_suitable"), _CODEBOOK),
     ("last of equally similar entries", "match_entries", _match("last_max"), _CODEBOOK),
+    ("rotation clockwise", "rope", _rope("clockwise"), _DECODE),
+    ("rotation pairs neighbouring elements", "rope", _rope("neighbouring_pairs"), _DECODE),
+    ("frequencies base**(-i/d)", "rope_frequencies", _frequencies_of_half_the_dimension, _DECODE),
+    ("query not rotated", "decode_attention", _decode("query_not_rotated"), _DECODE),
+    ("rebuilt keys not rotated", "decode_attention", _decode("keys_not_rotated"), _DECODE),
+    ("cached tokens rotated at their list index", "decode_attention", _decode("positions_ignored"), _DECODE),
+    ("key magnitudes dropped", "decode_attention", _decode("key_magnitude_dropped"), _DECODE),
+    ("value magnitudes dropped", "decode_attention", _decode("value_magnitude_dropped"), _DECODE),
+    ("decode scores not scaled by 1/sqrt(d)", "decode_attention", _decode("no_scale"), _DECODE),
 ]
 
 
 def test_pins_pass_on_the_checker_as_it_stands():
-    assert _failing_pins((test_oracle_evict, test_oracle_codebook, test_oracle_plan, test_oracle_compose)) == []
+    assert _failing_pins((test_oracle_evict, test_oracle_codebook, test_oracle_plan, test_oracle_compose,
+                          test_oracle_decode)) == []
 
 
 @pytest.mark.parametrize("what,attr,replacement,modules", MUTANTS, ids=[m[0] for m in MUTANTS])
