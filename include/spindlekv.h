@@ -285,6 +285,42 @@ spindlekv_status spindlekv_reconstruct(const spindlekv_batch* batch, int32_t n_h
                                        void* stream);
 
 /*
+ * Decode-time attention of one new token over the replaced cache (Section 3.4: Eq. (14) inside Eq. (1)).  The
+ * CodeBooks hold pre-RoPE keys, so the rotary embedding is applied again after reconstruction: for every
+ * (layer, seq, KV head) and each of its h_n query heads g,
+ *     K_t = RoPE(C_K[ref_K[t]] * mag_K[t], position of t),   V_t = C_V[ref_V[t]] * mag_V[t],
+ *     out_g = softmax_t( RoPE(q_g, pos_q) . K_t / sqrt(d_h) ) V
+ * over all cached tokens t (all of them precede the new token).  Rotary embedding as in the LLaMA / Mistral
+ * models: element i < d_h/2 is paired with element i + d_h/2, angle = position * base^(-2 i / d_h).  The rebuilt
+ * rows are never written to memory: CodeBook rows are gathered, scaled and rotated on the fly.
+ *
+ * spindlekv_rope_table fills the table of cosines and sines the call reads: float2 (cos, sin)
+ * [n_positions][head_dim/2], computed in double precision; spindlekv_rope_table_bytes is its size.
+ *
+ * spindlekv_decode_attend
+ *   batch       describes the cached tokens (max_len, or layer_lens per layer or per head; no cu_seqlens)
+ *   q           device, [layer][seq][q head][d] pre-RoPE queries of the new token (stride_tok unused)
+ *   pos_q       device [B]: position of the new token of every sequence
+ *   C_K, C_V    device, CodeBook rows [layer][seq][kv head][entry][d] (spindlekv_compact with divide_by = mag)
+ *   ref_*, mag_* device [n_layers][n_kv_heads][T]: outputs of spindlekv_codebook_shallow for K and for V
+ *   positions   device [n_layers][n_kv_heads][T] int32: original position of every cached token (the kept
+ *               positions when the CodeBooks were built from an evicted cache), or NULL: token t is at position t
+ *   rope_table, table_positions: the table and its number of positions; positions beyond it are clamped
+ *   out         device [n_layers][B][n_q_heads][d] fp32
+ *   ws          device scratch of spindlekv_decode_workspace_bytes bytes, 256-byte aligned
+ * At most 8 query heads per KV head; q, C_K and C_V share one dtype.
+ */
+size_t spindlekv_rope_table_bytes(int32_t head_dim, int32_t n_positions);
+spindlekv_status spindlekv_rope_table(int32_t head_dim, int32_t n_positions, double base, void* table, void* stream);
+size_t spindlekv_decode_workspace_bytes(const spindlekv_batch* batch, int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim);
+spindlekv_status spindlekv_decode_attend(const spindlekv_batch* batch, int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim,
+                                         spindlekv_tensor q, const int32_t* pos_q,
+                                         spindlekv_tensor C_K, const int32_t* ref_K, const float* mag_K,
+                                         spindlekv_tensor C_V, const int32_t* ref_V, const float* mag_V,
+                                         const int32_t* positions, const void* rope_table, int32_t table_positions,
+                                         float* out, void* ws, size_t ws_bytes, void* stream);
+
+/*
  * Reads the device status word of a workspace (blocking copy; synchronise the stream first).
  *   ws            the workspace of the call in question; NULL: the built-in scratch that
  *                 spindlekv_evict_deep_noalloc uses on the current device (INVALID_ARG before the first

@@ -86,6 +86,16 @@ def _load() -> C.CDLL:
     lib.spindlekv_reconstruct.restype = C.c_int32
     lib.spindlekv_reconstruct.argtypes = [C.POINTER(_Batch), C.c_int32, C.c_int32, _Tensor, C.c_void_p, C.c_void_p,
                                           _Tensor, C.c_void_p]
+    lib.spindlekv_rope_table_bytes.restype = C.c_size_t
+    lib.spindlekv_rope_table_bytes.argtypes = [C.c_int32, C.c_int32]
+    lib.spindlekv_rope_table.restype = C.c_int32
+    lib.spindlekv_rope_table.argtypes = [C.c_int32, C.c_int32, C.c_double, C.c_void_p, C.c_void_p]
+    lib.spindlekv_decode_workspace_bytes.restype = C.c_size_t
+    lib.spindlekv_decode_workspace_bytes.argtypes = [C.POINTER(_Batch), C.c_int32, C.c_int32, C.c_int32]
+    lib.spindlekv_decode_attend.restype = C.c_int32
+    lib.spindlekv_decode_attend.argtypes = [C.POINTER(_Batch), C.c_int32, C.c_int32, C.c_int32, _Tensor, C.c_void_p,
+                                            _Tensor, C.c_void_p, C.c_void_p, _Tensor, C.c_void_p, C.c_void_p,
+                                            C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
     lib.spindlekv_poll_status.restype = C.c_int32
     lib.spindlekv_poll_status.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
     lib.spindlekv_set_tuning.restype = C.c_int32
@@ -294,6 +304,32 @@ def spindlekv_reconstruct(batch: Batch, n_heads: int, head_dim: int, Cb: _Tensor
     bb = batch.c()
     st = _lib.spindlekv_reconstruct(C.byref(bb), n_heads, head_dim, Cb, _ptr(ref), _ptr(mag), dst, _stream(stream))
     _check(st, "spindlekv_reconstruct")
+
+
+def spindlekv_rope_table_bytes(head_dim: int, n_positions: int) -> int:
+    return int(_lib.spindlekv_rope_table_bytes(head_dim, n_positions))
+
+
+def spindlekv_rope_table(head_dim: int, n_positions: int, base: float, table: torch.Tensor, stream=None) -> None:
+    """Fills ``table`` (``[n_positions, head_dim/2, 2]`` fp32: cos, sin) for ``spindlekv_decode_attend``."""
+    _check(_lib.spindlekv_rope_table(head_dim, n_positions, base, _ptr(table), _stream(stream)), "spindlekv_rope_table")
+
+
+def spindlekv_decode_workspace_bytes(batch: Batch, n_q_heads: int, n_kv_heads: int, head_dim: int) -> int:
+    bb = batch.c()
+    return int(_lib.spindlekv_decode_workspace_bytes(C.byref(bb), n_q_heads, n_kv_heads, head_dim))
+
+
+def spindlekv_decode_attend(batch: Batch, n_q_heads: int, n_kv_heads: int, head_dim: int, q: _Tensor, pos_q: torch.Tensor,
+                            C_K: _Tensor, ref_K: torch.Tensor, mag_K: torch.Tensor, C_V: _Tensor, ref_V: torch.Tensor,
+                            mag_V: torch.Tensor, positions: Optional[torch.Tensor], rope_table: torch.Tensor,
+                            out: torch.Tensor, ws: torch.Tensor, stream=None) -> None:
+    """One decode step over the replaced cache; ``rope_table`` is ``[n_positions, head_dim/2, 2]`` fp32."""
+    bb = batch.c()
+    st = _lib.spindlekv_decode_attend(C.byref(bb), n_q_heads, n_kv_heads, head_dim, q, _ptr(pos_q), C_K, _ptr(ref_K),
+                                      _ptr(mag_K), C_V, _ptr(ref_V), _ptr(mag_V), _ptr(positions), _ptr(rope_table),
+                                      rope_table.shape[0], _ptr(out), _ptr(ws), ws.numel() * ws.element_size(), _stream(stream))
+    _check(st, "spindlekv_decode_attend")
 
 
 def spindlekv_poll_status(ws: Optional[torch.Tensor]):

@@ -10,7 +10,7 @@ ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libspindlekv.so")
 
-SOURCES = ["api.cu", "evict.cu", "codebook.cu", "compact.cu", "sim_tc.cu", "win_tc.cu", "extend.cu", "noalloc.cu"]
+SOURCES = ["api.cu", "evict.cu", "codebook.cu", "compact.cu", "sim_tc.cu", "win_tc.cu", "extend.cu", "noalloc.cu", "decode.cu"]
 HEADERS = ["args.cuh", "common.cuh", "simt_tile.cuh", "sm100_ptx.cuh"]
 
 

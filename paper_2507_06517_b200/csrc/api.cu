@@ -34,6 +34,15 @@ spindlekv_status union_lists_impl(int n_layers, int n_seqs, int n_heads, int n_l
 
 const void* noalloc_scratch_of_current_device();
 
+spindlekv_status rope_table_impl(int head_dim, int n_pos, double base, void* table, cudaStream_t st);
+size_t decode_workspace_bytes(const spindlekv_batch& b, int n_q_heads, int n_kv_heads, int head_dim);
+spindlekv_status decode_attend_impl(const spindlekv_batch& b, int n_q_heads, int n_kv_heads, int head_dim,
+                                    const spindlekv_tensor& q, const int32_t* pos_q, const spindlekv_tensor& CK,
+                                    const int32_t* ref_k, const float* mag_k, const spindlekv_tensor& CV,
+                                    const int32_t* ref_v, const float* mag_v, const int32_t* positions,
+                                    const void* table, int table_positions, float* out, void* ws, size_t ws_bytes,
+                                    cudaStream_t st);
+
 size_t match_workspace_bytes(const spindlekv_batch& b, int n_heads);
 spindlekv_status match_impl(const spindlekv_batch& b, int n_heads, int head_dim, const spindlekv_tensor& G,
                             const spindlekv_tensor& C, const int32_t* n_entries, int c_rows, float theta, float* mag,
@@ -263,6 +272,46 @@ spindlekv_status spindlekv_reconstruct(const spindlekv_batch* batch, int32_t n_h
   if (C.dtype != dst.dtype) return SPINDLEKV_UNSUPPORTED;
   if (head_dim != 64 && head_dim != 128) return SPINDLEKV_UNSUPPORTED;
   return reconstruct_impl(*batch, n_heads, head_dim, C, ref, mag, dst, (cudaStream_t)stream);
+}
+
+size_t spindlekv_rope_table_bytes(int32_t head_dim, int32_t n_positions) {
+  if ((head_dim != 64 && head_dim != 128) || n_positions <= 0) return 0;
+  return (size_t)n_positions * (head_dim / 2) * sizeof(float) * 2;
+}
+
+spindlekv_status spindlekv_rope_table(int32_t head_dim, int32_t n_positions, double base, void* table, void* stream) {
+  if (!table || n_positions <= 0 || !(base > 1.0) || reinterpret_cast<uintptr_t>(table) % 16) return SPINDLEKV_INVALID_ARG;
+  if (head_dim != 64 && head_dim != 128) return SPINDLEKV_UNSUPPORTED;
+  return rope_table_impl(head_dim, n_positions, base, table, (cudaStream_t)stream);
+}
+
+static bool decode_batch_ok(const spindlekv_batch* b) {
+  if (!b || b->n_layers <= 0 || b->n_seqs <= 0 || b->max_len <= 0 || b->cu_seqlens) return false;
+  return (int64_t)b->total_len == (int64_t)b->n_seqs * b->max_len;
+}
+
+size_t spindlekv_decode_workspace_bytes(const spindlekv_batch* batch, int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim) {
+  if (!decode_batch_ok(batch) || n_q_heads <= 0 || n_kv_heads <= 0 || n_q_heads % n_kv_heads) return 0;
+  if (head_dim != 64 && head_dim != 128) return 0;
+  return decode_workspace_bytes(*batch, n_q_heads, n_kv_heads, head_dim);
+}
+
+spindlekv_status spindlekv_decode_attend(const spindlekv_batch* batch, int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim,
+                                         spindlekv_tensor q, const int32_t* pos_q,
+                                         spindlekv_tensor C_K, const int32_t* ref_K, const float* mag_K,
+                                         spindlekv_tensor C_V, const int32_t* ref_V, const float* mag_V,
+                                         const int32_t* positions, const void* rope_table, int32_t table_positions,
+                                         float* out, void* ws, size_t ws_bytes, void* stream) {
+  if (!decode_batch_ok(batch) || n_q_heads <= 0 || n_kv_heads <= 0 || n_q_heads % n_kv_heads) return SPINDLEKV_INVALID_ARG;
+  if (!tensor_ok(q) || !tensor_ok(C_K) || !tensor_ok(C_V) || !pos_q || !ref_K || !mag_K || !ref_V || !mag_V || !rope_table ||
+      table_positions <= 0 || !out || !ws)
+    return SPINDLEKV_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(ws) % 256 || reinterpret_cast<uintptr_t>(rope_table) % 16) return SPINDLEKV_INVALID_ARG;
+  if (q.dtype != C_K.dtype || q.dtype != C_V.dtype) return SPINDLEKV_UNSUPPORTED;
+  if (head_dim != 64 && head_dim != 128) return SPINDLEKV_UNSUPPORTED;
+  if (n_q_heads / n_kv_heads > 8) return SPINDLEKV_UNSUPPORTED;
+  return decode_attend_impl(*batch, n_q_heads, n_kv_heads, head_dim, q, pos_q, C_K, ref_K, mag_K, C_V, ref_V, mag_V, positions,
+                            rope_table, table_positions, out, ws, ws_bytes, (cudaStream_t)stream);
 }
 
 spindlekv_status spindlekv_poll_status(const void* ws, int32_t* device_status, int32_t* detail) {

@@ -407,3 +407,25 @@ class SpindleKVDecodeMerge:
                                      self.ws_codebook, self.adj, stream)
         B.spindlekv_codebook_append(self.batch, H, d, ld, o["mag"], o["ref"], o["centre_idx"], o["n_entries"],
                                     self.left_idx, self.left_cnt, cd, self.c_rows, n_entries, self.ref_new, stream)
+
+
+class SpindleKVDecodeAttention:
+    """Buffers for ``spindlekv_decode_attend``: the table of rotary cosines and sines, the scratch of the split
+    pass and the output ``[L, B, H_q, d]`` (fp32).  ``batch`` describes the cached tokens.  Call order only."""
+
+    def __init__(self, batch: B.Batch, n_q_heads: int, n_kv_heads: int, head_dim: int, n_positions: int,
+                 rope_base: float = 10000.0, device="cuda"):
+        self.batch, self.Hq, self.Hkv, self.d = batch, n_q_heads, n_kv_heads, head_dim
+        dev = torch.device(device)
+        self.table = torch.empty((n_positions, head_dim // 2, 2), dtype=torch.float32, device=dev)
+        B.spindlekv_rope_table(head_dim, n_positions, rope_base, self.table)
+        self.ws = torch.empty(B.spindlekv_decode_workspace_bytes(batch, n_q_heads, n_kv_heads, head_dim), dtype=torch.uint8, device=dev)
+        self.out = torch.zeros((batch.n_layers, batch.n_seqs, n_q_heads, head_dim), dtype=torch.float32, device=dev)
+
+    def run(self, q: torch.Tensor, pos_q: torch.Tensor, cb_k: Dict[str, torch.Tensor], cb_v: Dict[str, torch.Tensor],
+            positions: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+        """``q``: ``[L, B, H_q, 1, d]`` pre-RoPE queries; ``cb_k`` / ``cb_v``: the ``C``, ``ref``, ``mag`` a CodeBook pass left."""
+        B.spindlekv_decode_attend(self.batch, self.Hq, self.Hkv, self.d, B.desc_bhnd(q), pos_q, B.desc_bhnd(cb_k["C"]),
+                                  cb_k["ref"], cb_k["mag"], B.desc_bhnd(cb_v["C"]), cb_v["ref"], cb_v["mag"], positions,
+                                  self.table, self.out, self.ws, stream)
+        return self.out

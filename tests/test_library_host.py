@@ -186,3 +186,29 @@ def test_reserve_ratio_matches_checker():
         assert B.spindlekv_reserve_ratio(l, kept, ek, ev) == O.reserve_ratio_layer(l, kept, ek, ev)
     with pytest.raises(B.SpindleKVError):
         B.spindlekv_reserve_ratio(100, 0, [1], [1])
+
+
+def test_decode_entry_points_check_their_arguments():
+    import ctypes as C
+    from paper_2507_06517_b200 import binding as B
+    lib = B._lib
+    batch = B._Batch(1, 1, 1024, 1024, None, None, 0)
+    packed = B._Batch(1, 1, 1024, 1024, 256, None, 0)
+    good, f32 = B._Tensor(256, B.BF16, 8, 8, 8, 8), B._Tensor(256, B.F32, 8, 8, 8, 8)
+    p = C.c_void_p(256)
+
+    def call(b=batch, hq=8, hkv=2, d=128, q=good, ck=good, cv=good, table=p, npos=64, ws=p):
+        return lib.spindlekv_decode_attend(C.byref(b), hq, hkv, d, q, p, ck, p, p, cv, p, p, None, table, npos, p, ws, 1 << 20, None)
+
+    assert call(b=packed) == B.INVALID_ARG            # equal-length form only
+    assert call(hq=7) == B.INVALID_ARG                # query heads must divide over the KV heads
+    assert call(table=None) == B.INVALID_ARG
+    assert call(ws=C.c_void_p(260)) == B.INVALID_ARG
+    assert call(ck=f32) == B.UNSUPPORTED              # one dtype for q and both CodeBooks
+    assert call(d=96) == B.UNSUPPORTED
+    assert call(hq=32, hkv=2) == B.UNSUPPORTED        # more than 8 query heads per KV head
+    assert B.spindlekv_rope_table_bytes(128, 4096) == 4096 * 64 * 8
+    assert B.spindlekv_rope_table_bytes(100, 4096) == 0
+    assert lib.spindlekv_rope_table(128, 0, 10000.0, p, None) == B.INVALID_ARG
+    assert lib.spindlekv_decode_workspace_bytes(C.byref(packed), 8, 2, 128) == 0
+    assert lib.spindlekv_decode_workspace_bytes(C.byref(batch), 8, 2, 128) >= 4 * 130 * 4 * 2
