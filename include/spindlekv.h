@@ -79,6 +79,10 @@ typedef struct {
   float theta_k;          /* similarity thresholds of Eq. (9) */
   float theta_v;
   int32_t score_norm;     /* 0: divide by (l - a) as Eq. (2) prints; 1: plain window sum (not in the paper) */
+  int32_t per_query_head; /* 0: scores are the group mean of Eq. (3) and every KV head selects once;
+                             1: the GQA "repeat" alternative of Section 3.3: the KV vectors count once per query head,
+                             every query head i selects with its own ac_i of Eq. (2); the per-head outputs of
+                             spindlekv_evict_deep (scores, keep_idx, keep_cnt) are then indexed by query head */
 } spindlekv_config;
 
 /* Which layers and sequences one device call covers. */
@@ -139,6 +143,8 @@ size_t spindlekv_workspace_bytes(const spindlekv_config* cfg, const spindlekv_ba
  *   keep_cnt device out [n_layers][B][n_kv_heads] = k + l_w
  *   scores   device out [n_layers][n_kv_heads][T] fp32: ac' of Eq. (3) for context positions
  *            (window columns are left untouched); may not be NULL
+ * With cfg->per_query_head = 1 the three outputs have n_q_heads in place of n_kv_heads (query head h_n*j + g reads
+ * KV head j), scores hold ac_i of Eq. (2), and every query head keeps its own k_ctx positions.
  */
 spindlekv_status spindlekv_evict_deep(const spindlekv_config* cfg, const spindlekv_batch* batch,
                                       spindlekv_tensor K, spindlekv_tensor Qwin, const int32_t* k_ctx,
@@ -227,10 +233,12 @@ spindlekv_status spindlekv_compact(const spindlekv_batch* batch, int32_t n_heads
  * pass 0, then of pass 1, ...; out count = sum of the counts (clipped to seq_out).  Equal-length batches only.
  *   idx_in  device [n_lists][n_layers][n_heads][t_in], sequence s starting at column s * seq_in
  *   cnt_in  device [n_lists][n_layers][n_seqs][n_heads]
+ *           (lists_inner = 1: [n_layers][n_heads][n_lists][t_in] and [n_layers][n_seqs][n_heads][n_lists], i.e. the
+ *           per-query-head outputs of one spindlekv_evict_deep call with per_query_head = 1, n_lists = h_n)
  *   idx_out device [n_layers][n_heads][t_out], sequence s starting at column s * seq_out
  *   cnt_out device [n_layers][n_seqs][n_heads]
  */
-spindlekv_status spindlekv_union_lists(int32_t n_layers, int32_t n_seqs, int32_t n_heads, int32_t n_lists,
+spindlekv_status spindlekv_union_lists(int32_t n_layers, int32_t n_seqs, int32_t n_heads, int32_t n_lists, int32_t lists_inner,
                                        int32_t t_in, int32_t seq_in, const int32_t* idx_in, const int32_t* cnt_in,
                                        int32_t t_out, int32_t seq_out, int32_t* idx_out, int32_t* cnt_out, void* stream);
 

@@ -37,7 +37,8 @@ class _Config(C.Structure):
     _fields_ = [("n_layers", C.c_int32), ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32),
                 ("head_dim", C.c_int32), ("window", C.c_int32), ("n_shallow", C.c_int32),
                 ("reserve_ratio", C.c_double), ("budget_tokens", C.c_double), ("beta", C.c_double),
-                ("theta_k", C.c_float), ("theta_v", C.c_float), ("score_norm", C.c_int32)]
+                ("theta_k", C.c_float), ("theta_v", C.c_float), ("score_norm", C.c_int32),
+                ("per_query_head", C.c_int32)]
 
 
 class _Batch(C.Structure):
@@ -72,7 +73,7 @@ def _load() -> C.CDLL:
     lib.spindlekv_compact.argtypes = [C.POINTER(_Batch), C.c_int32, C.c_int32, _Tensor, C.c_void_p, C.c_void_p,
                                       C.c_void_p, _Tensor, C.c_void_p, C.c_void_p]
     lib.spindlekv_union_lists.restype = C.c_int32
-    lib.spindlekv_union_lists.argtypes = [C.c_int32] * 6 + [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_void_p,
+    lib.spindlekv_union_lists.argtypes = [C.c_int32] * 7 + [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_void_p,
                                                             C.c_void_p, C.c_void_p]
     lib.spindlekv_match_workspace_bytes.restype = C.c_size_t
     lib.spindlekv_match_workspace_bytes.argtypes = [C.POINTER(_Batch), C.c_int32]
@@ -133,10 +134,12 @@ class Config:
     theta_k: float = 0.98
     theta_v: float = 0.95
     score_norm: int = 0
+    per_query_head: int = 0
 
     def c(self) -> _Config:
         return _Config(self.n_layers, self.n_q_heads, self.n_kv_heads, self.head_dim, self.window, self.n_shallow,
-                       self.reserve_ratio, self.budget_tokens, self.beta, self.theta_k, self.theta_v, self.score_norm)
+                       self.reserve_ratio, self.budget_tokens, self.beta, self.theta_k, self.theta_v, self.score_norm,
+                       self.per_query_head)
 
 
 @dataclasses.dataclass
@@ -266,10 +269,14 @@ def spindlekv_compact(batch: Batch, n_heads: int, head_dim: int, src: _Tensor, i
 
 
 def spindlekv_union_lists(n_layers: int, n_seqs: int, n_heads: int, idx_in: torch.Tensor, cnt_in: torch.Tensor,
-                          seq_in: int, idx_out: torch.Tensor, cnt_out: torch.Tensor, seq_out: int, stream=None) -> None:
-    """``idx_in [n_lists, L, H, t_in]``, ``cnt_in [n_lists, L, B, H]`` -> ``idx_out [L, H, t_out]``, ``cnt_out [L, B, H]``."""
-    st = _lib.spindlekv_union_lists(n_layers, n_seqs, n_heads, idx_in.shape[0], idx_in.shape[-1], seq_in, _ptr(idx_in),
-                                    _ptr(cnt_in), idx_out.shape[-1], seq_out, _ptr(idx_out), _ptr(cnt_out), _stream(stream))
+                          seq_in: int, idx_out: torch.Tensor, cnt_out: torch.Tensor, seq_out: int, stream=None,
+                          lists_inner: bool = False) -> None:
+    """``idx_in [n_lists, L, H, t_in]``, ``cnt_in [n_lists, L, B, H]`` (``lists_inner``: ``[L, H, n_lists, t_in]`` and
+    ``[L, B, H, n_lists]``) -> ``idx_out [L, H, t_out]``, ``cnt_out [L, B, H]``."""
+    n_lists = idx_in.shape[2] if lists_inner else idx_in.shape[0]
+    st = _lib.spindlekv_union_lists(n_layers, n_seqs, n_heads, n_lists, 1 if lists_inner else 0, idx_in.shape[-1], seq_in,
+                                    _ptr(idx_in), _ptr(cnt_in), idx_out.shape[-1], seq_out, _ptr(idx_out), _ptr(cnt_out),
+                                    _stream(stream))
     _check(st, "spindlekv_union_lists")
 
 

@@ -28,7 +28,7 @@ spindlekv_status compact_impl(const spindlekv_batch& b, int n_heads, int head_di
 spindlekv_status reconstruct_impl(const spindlekv_batch& b, int n_heads, int head_dim, const spindlekv_tensor& C,
                                   const int32_t* ref, const float* mag, const spindlekv_tensor& dst, cudaStream_t st);
 
-spindlekv_status union_lists_impl(int n_layers, int n_seqs, int n_heads, int n_lists, int t_in, int seq_in,
+spindlekv_status union_lists_impl(int n_layers, int n_seqs, int n_heads, int n_lists, int lists_inner, int t_in, int seq_in,
                                   const int32_t* idx_in, const int32_t* cnt_in, int t_out, int seq_out,
                                   int32_t* idx_out, int32_t* cnt_out, cudaStream_t st);
 
@@ -212,14 +212,14 @@ spindlekv_status spindlekv_compact(const spindlekv_batch* batch, int32_t n_heads
   return compact_impl(*batch, n_heads, head_dim, src, idx, cnt, divide_by, dst, dst_cu_seqlens, (cudaStream_t)stream);
 }
 
-spindlekv_status spindlekv_union_lists(int32_t n_layers, int32_t n_seqs, int32_t n_heads, int32_t n_lists,
+spindlekv_status spindlekv_union_lists(int32_t n_layers, int32_t n_seqs, int32_t n_heads, int32_t n_lists, int32_t lists_inner,
                                        int32_t t_in, int32_t seq_in, const int32_t* idx_in, const int32_t* cnt_in,
                                        int32_t t_out, int32_t seq_out, int32_t* idx_out, int32_t* cnt_out, void* stream) {
   if (n_layers <= 0 || n_seqs <= 0 || n_heads <= 0 || n_lists <= 0 || t_in <= 0 || t_out <= 0) return SPINDLEKV_INVALID_ARG;
   if (seq_in <= 0 || seq_out <= 0 || (int64_t)n_seqs * seq_in > t_in || (int64_t)n_seqs * seq_out > t_out) return SPINDLEKV_INVALID_ARG;
   if (!idx_in || !cnt_in || !idx_out || !cnt_out) return SPINDLEKV_INVALID_ARG;
   if ((int64_t)n_layers * n_seqs * n_heads > 0x7FFFFFFF) return SPINDLEKV_UNSUPPORTED;
-  return union_lists_impl(n_layers, n_seqs, n_heads, n_lists, t_in, seq_in, idx_in, cnt_in, t_out, seq_out, idx_out,
+  return union_lists_impl(n_layers, n_seqs, n_heads, n_lists, lists_inner, t_in, seq_in, idx_in, cnt_in, t_out, seq_out, idx_out,
                           cnt_out, (cudaStream_t)stream);
 }
 

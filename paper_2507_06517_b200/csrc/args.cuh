@@ -40,7 +40,8 @@ inline spindlekv_status evict_args_status(const spindlekv_config* cfg, const spi
   if (!tensor_ok(K) || !tensor_ok(Qwin) || !k_ctx || !keep_idx || !keep_cnt || !scores) return SPINDLEKV_INVALID_ARG;
   if (K.dtype != Qwin.dtype) return SPINDLEKV_UNSUPPORTED;
   if (cfg->head_dim != 64 && cfg->head_dim != 128) return SPINDLEKV_UNSUPPORTED;
-  if ((int64_t)batch->n_layers * batch->n_seqs * cfg->n_kv_heads > 65535) return SPINDLEKV_UNSUPPORTED;
+  const int64_t out_heads = cfg->per_query_head ? cfg->n_q_heads : cfg->n_kv_heads;   // heads that select on their own
+  if ((int64_t)batch->n_layers * batch->n_seqs * out_heads > 65535) return SPINDLEKV_UNSUPPORTED;
   return SPINDLEKV_OK;
 }
 

@@ -151,6 +151,7 @@ spindlekv_status reconstruct_impl(const spindlekv_batch& b, int n_heads, int hea
 // pass 0, then pass 1, ...; its count is the sum of the counts.
 struct UnionParams {
   int n_layers, n_seqs, n_heads, n_lists;
+  int lists_inner;             // 0: idx_in [n_lists][layers][H][t_in]; 1: [layers][H][n_lists][t_in] (cnt alike)
   int t_in, t_out;             // row length of one (layer, head) in idx_in / idx_out
   int seq_in, seq_out;         // start of sequence s within a row: s * seq_in, s * seq_out
   const int32_t* idx_in;       // [n_lists][layers][H][t_in]
@@ -172,18 +173,20 @@ __global__ void __launch_bounds__(256) union_lists_kernel(UnionParams p) {
   const int64_t cnt_at = ((int64_t)layer * p.n_seqs + s) * p.n_heads + h;
   int base = 0;
   for (int g = 0; g < p.n_lists; ++g) {
-    const int n = p.cnt_in[g * per_list_cnt + cnt_at];
-    const int32_t* src = p.idx_in + g * per_list_idx + in_row;
+    const int n = p.lists_inner ? p.cnt_in[cnt_at * p.n_lists + g] : p.cnt_in[g * per_list_cnt + cnt_at];
+    const int32_t* src = p.lists_inner
+        ? p.idx_in + (((int64_t)layer * p.n_heads + h) * p.n_lists + g) * p.t_in + (int64_t)s * p.seq_in
+        : p.idx_in + g * per_list_idx + in_row;
     for (int r = threadIdx.x; r < n && base + r < p.seq_out; r += blockDim.x) p.idx_out[out_row + base + r] = src[r];
     base += n;
   }
   if (threadIdx.x == 0) p.cnt_out[cnt_at] = min(base, p.seq_out);
 }
 
-spindlekv_status union_lists_impl(int n_layers, int n_seqs, int n_heads, int n_lists, int t_in, int seq_in,
+spindlekv_status union_lists_impl(int n_layers, int n_seqs, int n_heads, int n_lists, int lists_inner, int t_in, int seq_in,
                                   const int32_t* idx_in, const int32_t* cnt_in, int t_out, int seq_out,
                                   int32_t* idx_out, int32_t* cnt_out, cudaStream_t st) {
-  UnionParams p{n_layers, n_seqs, n_heads, n_lists, t_in, t_out, seq_in, seq_out, idx_in, cnt_in, idx_out, cnt_out};
+  UnionParams p{n_layers, n_seqs, n_heads, n_lists, lists_inner, t_in, t_out, seq_in, seq_out, idx_in, cnt_in, idx_out, cnt_out};
   LaunchScope ls(KC_GATHER, st);
   union_lists_kernel<<<n_layers * n_seqs * n_heads, 256, 0, st>>>(p);
   return cudaGetLastError() == cudaSuccess ? SPINDLEKV_OK : SPINDLEKV_CUDA;

@@ -18,7 +18,8 @@ namespace skv {
 struct EvictParams {
   View K, Q;
   Batch batch;
-  int n_q_heads, n_kv_heads, window, h_n;
+  int n_q_heads, n_kv_heads, window, h_n;   // n_kv_heads: heads that get a score row; h_n: query heads summed into one
+  int kv_div;           // head j reads KV head j / kv_div (1, or h_n when every query head has its own row)
   int n_tiles;          // key tiles per unit = ceil(max_len / 64)
   int score_norm;
   float scale;          // 1 / sqrt(d_h)
@@ -38,7 +39,7 @@ __device__ __forceinline__ void decode_unit(const EvictParams& p, int unit, int&
 template <typename T, int D>
 __device__ __forceinline__ void logits_tile(const EvictParams& p, TileSmem& sm, int layer, int s, int j, int l,
                                             int row0, int key0, float (&acc)[4][4]) {
-  const T* kbase = reinterpret_cast<const T*>(p.K.ptr) + unit_offset(p.K, p.batch, layer, s, j);
+  const T* kbase = reinterpret_cast<const T*>(p.K.ptr) + unit_offset(p.K, p.batch, layer, s, j / p.kv_div);
   const T* qbase = reinterpret_cast<const T*>(p.Q.ptr) + (int64_t)layer * p.Q.sl + (int64_t)s * p.Q.ss;
   const int M = p.h_n * p.window;
   auto row_q = [&](int r) -> const T* {
@@ -368,17 +369,21 @@ spindlekv_status evict_deep_impl(const spindlekv_config& cfg, const spindlekv_ba
                                  const spindlekv_tensor& Q, const int32_t* k_ctx, int32_t* keep_idx,
                                  int32_t* keep_cnt, float* scores, void* ws, size_t ws_bytes, cudaStream_t st) {
   if (ws_bytes < evict_scratch_needed(cfg, b, K.dtype)) return SPINDLEKV_WORKSPACE_TOO_SMALL;
-  const int units = b.n_layers * b.n_seqs * cfg.n_kv_heads;
-  const int h_n = cfg.n_q_heads / cfg.n_kv_heads;
+  // per_query_head: every query head is a unit of its own (one head per "group") that reads its group's KV head
+  const bool per_head = cfg.per_query_head != 0;
+  const int out_heads = per_head ? cfg.n_q_heads : cfg.n_kv_heads;
+  const int units = b.n_layers * b.n_seqs * out_heads;
+  const int h_n = per_head ? 1 : cfg.n_q_heads / cfg.n_kv_heads;
   const size_t M = (size_t)h_n * cfg.window;
   EvictParams p;
   p.K = make_view(K);
   p.Q = make_view(Q);
   p.batch = make_batch(b);
   p.n_q_heads = cfg.n_q_heads;
-  p.n_kv_heads = cfg.n_kv_heads;
+  p.n_kv_heads = out_heads;
   p.window = cfg.window;
   p.h_n = h_n;
+  p.kv_div = per_head ? cfg.n_q_heads / cfg.n_kv_heads : 1;
   p.n_tiles = ceil_div(b.max_len, kTile);
   p.score_norm = cfg.score_norm;
   p.scale = 1.0f / sqrtf((float)cfg.head_dim);
@@ -399,7 +404,7 @@ spindlekv_status evict_deep_impl(const spindlekv_config& cfg, const spindlekv_ba
   }
   TopkParams t;
   t.batch = p.batch;
-  t.n_kv_heads = cfg.n_kv_heads;
+  t.n_kv_heads = out_heads;
   t.window = cfg.window;
   t.scores = scores;
   t.k_ctx = k_ctx;

@@ -30,6 +30,7 @@ struct WinTcParams {
   int n_kv_heads, h_n, window;
   int m_rows;            // h_n * window
   int score_norm;
+  int per_head;          // 1: one score row per query head (Eq. (2)), no group mean; scores are then [layers][H_q][T]
   float c;               // log2(e) / sqrt(d_h)
   float* scores;         // [layers][H_kv][T]
   uint32_t* hdr;
@@ -309,21 +310,43 @@ __global__ void __launch_bounds__(WinShape<QB>::THREADS, 1) win_tc_kernel(const 
     ptx::fence_proxy_async();
     __syncwarp();
     if (lane == 0) ptx::mbar_arrive(ext_full);
-    // ---- pass B: this thread's key, summed over all query rows ----
+    // ---- pass B: this thread's key, summed over all query rows (group mean) or over each head's rows ----
     const float inv_hn = 1.0f / (float)p.h_n;
-    float* out = p.scores + ((int64_t)layer * p.n_kv_heads + j) * p.batch.total_len + tok_base(p.batch, s);
+    const bool per_head = p.per_head != 0;
+    const int out_heads = per_head ? p.n_kv_heads * p.h_n : p.n_kv_heads;
+    float* out = p.scores + ((int64_t)layer * out_heads + (per_head ? p.h_n * j : j)) * p.batch.total_len + tok_base(p.batch, s);
+    const int cph = p.window >= 32 ? p.window / 32 : 1;   // 32-column chunks per query head (a window of 16: two heads per chunk)
     // the first pass-B item whose stage belongs to this group
     for (int i = T + ((eg - T % G + G) % G); ok && i < T + Tc; i += G) {
       const int as = i % AS;
       const uint32_t tlane = tquarter + as * AS_COLS;
       if (!__all_sync(0xffffffffu, ptx::mbar_wait(acc_full + as, (i / AS) & 1, abort_flag))) break;
       ptx::tc_fence_after();
-      float colsum = 0.f;
-      auto chunk_b = [&](const uint32_t (&raw)[32]) {
-        float part = 0.f;
+      const int a = (i - T) * kWinTile + q * 32 + lane;
+      float colsum = 0.f, headsum = 0.f;
+      // Eq. (2) for one query head: its window rows summed, divided by the distance to the end
+      auto write_head = [&](int g, float v) {
+        if (g < p.h_n && a < l_c) out[(int64_t)g * p.batch.total_len + a] = p.score_norm == 0 ? v / (float)(l - a) : v;
+      };
+      auto chunk_b = [&](const uint32_t (&raw)[32], int ch) {
+        float lo = 0.f, hi = 0.f;
 #pragma unroll
-        for (int e = 0; e < 32; ++e) part += ex2_approx(__uint_as_float(raw[e]) * c);
-        colsum += part;
+        for (int e = 0; e < 16; ++e) lo += ex2_approx(__uint_as_float(raw[e]) * c);
+#pragma unroll
+        for (int e = 16; e < 32; ++e) hi += ex2_approx(__uint_as_float(raw[e]) * c);
+        colsum += lo + hi;
+        if (per_head) {
+          if (p.window == 16) {
+            write_head(2 * ch, lo);
+            write_head(2 * ch + 1, hi);
+          } else {
+            headsum += lo + hi;
+            if ((ch + 1) % cph == 0) {
+              write_head(ch / cph, headsum);
+              headsum = 0.f;
+            }
+          }
+        }
       };
       if constexpr (QB == 1) {
         // eighteen warps share the register file: one load at a time, the other warps of the scheduler fill in
@@ -332,7 +355,7 @@ __global__ void __launch_bounds__(WinShape<QB>::THREADS, 1) win_tc_kernel(const 
           uint32_t raw[32];
           ptx::tmem_ld_32x32(tlane + ch * 32, raw);
           ptx::tmem_ld_wait(raw);
-          chunk_b(raw);
+          chunk_b(raw, ch);
         }
       } else {
         // groups of four chunks in straight-line code, the next 32 columns on their way while these are worked on:
@@ -345,18 +368,17 @@ __global__ void __launch_bounds__(WinShape<QB>::THREADS, 1) win_tc_kernel(const 
           for (int ch = 0; ch < 4; ch += 2) {
             ptx::tmem_ld_wait(r0);
             ptx::tmem_ld_32x32(tlane + g * 128 + (ch + 1) * 32, r1);
-            chunk_b(r0);
+            chunk_b(r0, g * 4 + ch);
             ptx::tmem_ld_wait(r1);
             if (ch + 2 < 4) ptx::tmem_ld_32x32(tlane + g * 128 + (ch + 2) * 32, r0);
-            chunk_b(r1);
+            chunk_b(r1, g * 4 + ch + 1);
           }
         }
       }
       ptx::tc_fence_before();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(acc_empty + as);
-      const int a = (i - T) * kWinTile + q * 32 + lane;
-      if (a < l_c) {
+      if (!per_head && a < l_c) {
         float v = colsum * inv_hn;
         if (p.score_norm == 0) v = v / (float)(l - a);
         out[a] = v;
@@ -424,6 +446,7 @@ spindlekv_status launch_win_tc(const spindlekv_config& cfg, const spindlekv_batc
   p.window = cfg.window;
   p.m_rows = p.h_n * cfg.window;
   p.score_norm = cfg.score_norm;
+  p.per_head = cfg.per_query_head ? 1 : 0;
   p.c = 1.4426950408889634f / sqrtf((float)cfg.head_dim);
   p.scores = scores;
   p.hdr = hdr;

@@ -293,7 +293,7 @@ class SpindleKVRepeatPass:
     its query heads kept, listed one head after the other, where a token kept by several heads
     appears several times and collapses into one entry (cosine similarity 1).  ``cfg.n_shallow`` must
     be -1; equal-length sequences.  ``K``, ``V``: ``[L, B, H_kv, N, d]``; ``Q``: ``[L, B, H_q, w, d]``.
-    Buffers and call order only.
+    One eviction call with ``per_query_head`` set serves all query heads.  Buffers and call order only.
     """
 
     def __init__(self, cfg: B.Config, seq_lens: Sequence[int], dtype: torch.dtype, device="cuda",
@@ -305,17 +305,16 @@ class SpindleKVRepeatPass:
         self.cfg = cfg
         self.device = dev = torch.device(device)
         self.h_n = cfg.n_q_heads // cfg.n_kv_heads
-        L, nB, H, d, N = cfg.n_layers, len(seq_lens), cfg.n_kv_heads, cfg.head_dim, int(seq_lens[0])
+        L, nB, H, Hq, d, N = cfg.n_layers, len(seq_lens), cfg.n_kv_heads, cfg.n_q_heads, cfg.head_dim, int(seq_lens[0])
         self.n_seqs, self.max_len = nB, N
-        # one eviction call per position g in the group: query heads g, h_n + g, ... against the KV heads
-        self.ecfg = dataclasses.replace(cfg, n_q_heads=H, n_shallow=0)
+        self.ecfg = dataclasses.replace(cfg, n_shallow=0, per_query_head=1)
         self.mode, self.ratio, self.k_ctx_host = B.spindlekv_plan_layers(cfg, list(seq_lens))
         self.k_ctx = torch.from_numpy(np.ascontiguousarray(self.k_ctx_host)).to(dev)
         self.ev_batch = B.Batch(L, nB, N, nB * N)
         i32 = dict(dtype=torch.int32, device=dev)
-        self.keep_idx = torch.zeros((self.h_n, L, H, nB * N), **i32)
-        self.keep_cnt = torch.zeros((self.h_n, L, nB, H), **i32)
-        self.scores = torch.zeros((self.h_n, L, H, nB * N), dtype=torch.float32, device=dev)
+        self.keep_idx = torch.zeros((L, Hq, nB * N), **i32)              # per query head
+        self.keep_cnt = torch.zeros((L, nB, Hq), **i32)
+        self.scores = torch.zeros((L, Hq, nB * N), dtype=torch.float32, device=dev)
         self.ws_evict = torch.empty(B.spindlekv_workspace_bytes(self.ecfg, self.ev_batch, B.WS_EVICT), dtype=torch.uint8, device=dev)
         self.kept_host = (self.k_ctx_host + cfg.window).astype(np.int32)                     # per query head
         self.union_host = (self.h_n * self.kept_host).astype(np.int32)                       # per KV head
@@ -325,7 +324,6 @@ class SpindleKVRepeatPass:
         self.union_idx = torch.zeros((L, H, T), **i32)
         self.union_cnt = torch.zeros((L, nB, H), **i32)
         self.cb_batch = B.Batch(L, nB, self.max_union, T, None, self.layer_lens)
-        self.gather_batch = B.Batch(L, nB, N, nB * N)
         self.ws_codebook = torch.empty(B.spindlekv_workspace_bytes(cfg, self.cb_batch, B.WS_CODEBOOK), dtype=torch.uint8, device=dev)
         self.rep = {g: torch.zeros((L, nB, H, self.max_union, d), dtype=dtype, device=dev) for g in ("K", "V")}
         self.cb: Dict[str, Dict[str, torch.Tensor]] = {}
@@ -341,11 +339,13 @@ class SpindleKVRepeatPass:
 
     def run(self, K: torch.Tensor, V: torch.Tensor, Q: torch.Tensor, which=("K", "V"), stream=None) -> None:
         cfg, H, d = self.cfg, self.cfg.n_kv_heads, self.cfg.head_dim
-        for g in range(self.h_n):
-            B.spindlekv_evict_deep(self.ecfg, self.ev_batch, B.desc_bhnd(K), B.desc_bhnd(Q[:, :, g::self.h_n]), self.k_ctx,
-                                   self.keep_idx[g], self.keep_cnt[g], self.scores[g], self.ws_evict, stream)
-        B.spindlekv_union_lists(cfg.n_layers, self.n_seqs, H, self.keep_idx, self.keep_cnt, self.max_len,
-                                self.union_idx, self.union_cnt, self.max_union, stream)
+        B.spindlekv_evict_deep(self.ecfg, self.ev_batch, B.desc_bhnd(K), B.desc_bhnd(Q), self.k_ctx, self.keep_idx,
+                               self.keep_cnt, self.scores, self.ws_evict, stream)
+        # query head h_n*j + g is list g of KV head j: the per-query-head outputs are [L][H][h_n][...] as they stand
+        L = cfg.n_layers
+        B.spindlekv_union_lists(L, self.n_seqs, H, self.keep_idx.view(L, H, self.h_n, -1),
+                                self.keep_cnt.view(L, self.n_seqs, H, self.h_n), self.max_len,
+                                self.union_idx, self.union_cnt, self.max_union, stream, lists_inner=True)
         for g in which:
             src, rep, o = (K if g == "K" else V), self.rep[g], self.cb[g]
             # rows of the union list, gathered from the KV head (the union list is laid out per max_union tokens,

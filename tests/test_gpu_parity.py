@@ -240,7 +240,7 @@ def test_gqa_repeat_variant():
         p.run(K, V, Q, which=(g,))
         st = p.device_status()
         assert st["evict"][0] == 0 and st["codebook"][0] == 0 and st["codebook"][1][1] == 0
-        keep, cnt, scores = p.keep_idx.cpu().numpy(), p.keep_cnt.cpu().numpy(), p.scores.cpu().numpy()
+        keep, cnt, scores = p.keep_idx.cpu().numpy(), p.keep_cnt.cpu().numpy(), p.scores.cpu().numpy()   # per query head
         union, ucnt = p.union_idx.cpu().numpy(), p.union_cnt.cpu().numpy()
         o = {k: (v.float() if k == "C" else v).cpu().numpy() for k, v in p.cb[g].items()}
         adj = p.adj.cpu().numpy()
@@ -249,10 +249,12 @@ def test_gqa_repeat_variant():
             n = k_ctx + w
             Ks = np.stack([host[lam][0][0, j] for j in range(H)])
             for gq in range(h_n):
-                check_evict_unit(one, host[lam][2][0][gq::h_n], Ks, k_ctx, scores[gq, lam], keep[gq, lam], cnt[gq, lam, 0])
+                # the query heads at position gq of every group, each against its own KV head: a group of one
+                sel = np.arange(gq, wl.n_q_heads, h_n)
+                check_evict_unit(one, host[lam][2][0][sel], Ks, k_ctx, scores[lam][sel], keep[lam][sel], cnt[lam, 0][sel])
             for j in range(H):
                 assert ucnt[lam, 0, j] == h_n * n
-                want_union = np.concatenate([keep[gq, lam, j, :n] for gq in range(h_n)])
+                want_union = np.concatenate([keep[lam, h_n * j + gq, :n] for gq in range(h_n)])
                 assert np.array_equal(union[lam, j, : h_n * n], want_union)
                 gamma = host[lam][idx][0, j][want_union]
                 check_codebook_unit(gamma, theta, adj[lam * H + j], o["mag"][lam, j, : h_n * n], o["ref"][lam, j, : h_n * n],
@@ -262,6 +264,42 @@ def test_gqa_repeat_variant():
                 ref = o["ref"][lam, j, : h_n * n]
                 for tok in np.unique(want_union):
                     assert len(set(ref[want_union == tok])) == 1
+
+
+def test_per_query_head_eviction_on_every_window_shape():
+    # Section 3.3's alternative to the group mean, one call: every query head gets its own score row (Eq. (2)) and its
+    # own kept set; windows of 16 (two heads per 32-column chunk), 32, 64 (two chunks per head), 256 query rows per
+    # KV head, and the fp32 CUDA-core kernels
+    from paper_2507_06517_b200 import binding as B
+    cases = [
+        synth.Workload("pq_w32", 2, 0, 8, 2, 128, "bf16", 32, (900,), 20, (0.05, 0.3), 2, "recency", budget_tokens=200.0, seed=111),
+        synth.Workload("pq_w16", 1, 0, 16, 4, 64, "bf16", 16, (640,), 20, 0.2, 2, "recency", budget_tokens=100.0, seed=112),
+        synth.Workload("pq_w64", 1, 0, 8, 2, 128, "bf16", 64, (1100,), 30, (0.05, 0.3), 4, "recency", budget_tokens=300.0, seed=113),
+        synth.Workload("pq_qb2", 1, 0, 16, 2, 64, "bf16", 32, (700,), 30, (0.05, 0.3), 4, "recency", budget_tokens=200.0, seed=114),
+        synth.Workload("pq_f32", 1, 0, 4, 2, 64, "f32", 32, (333,), 8, 0.1, 2, "gauss", budget_tokens=80.0, seed=115),
+    ]
+    for wl in cases:
+        host = generate(wl)
+        layers = list(range(wl.n_layers))
+        K, Q = stack_layers(wl, host, layers, "K"), stack_layers(wl, host, layers, "Q")
+        cfg = make_config(wl, per_query_head=1)
+        L, Hq, H, N, w, h_n = wl.n_layers, wl.n_q_heads, wl.n_kv_heads, wl.max_len, wl.window, wl.group
+        batch = B.Batch(L, 1, N, N)
+        _, _, k_plan = B.spindlekv_plan_layers(cfg, wl.seq_lens)
+        k_dev = torch.from_numpy(np.ascontiguousarray(k_plan)).cuda()
+        keep = torch.full((L, Hq, N), -1, dtype=torch.int32, device="cuda")
+        cnt = torch.zeros((L, 1, Hq), dtype=torch.int32, device="cuda")
+        scores = torch.zeros((L, Hq, N), dtype=torch.float32, device="cuda")
+        ws = torch.empty(B.spindlekv_workspace_bytes(cfg, batch, B.WS_EVICT), dtype=torch.uint8, device="cuda")
+        B.spindlekv_evict_deep(cfg, batch, B.desc_bhnd(K), B.desc_bhnd(Q), k_dev, keep, cnt, scores, ws)
+        torch.cuda.synchronize()
+        assert B.spindlekv_poll_status(ws)[0] == 0
+        keep, cnt, scores = keep.cpu().numpy(), cnt.cpu().numpy(), scores.cpu().numpy()
+        one = wl.replace(n_q_heads=1, n_kv_heads=1)
+        for lam in layers:
+            for i in range(Hq):
+                check_evict_unit(one, host[lam][2][0][i:i + 1], host[lam][0][0][i // h_n:i // h_n + 1], int(k_plan[lam, 0]),
+                                 scores[lam, i:i + 1], keep[lam, i:i + 1], cnt[lam, 0, i:i + 1])
 
 
 def test_decode_time_merge_into_existing_codebooks():

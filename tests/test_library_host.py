@@ -112,8 +112,8 @@ def test_device_entry_points_reject_bad_arguments_before_touching_the_gpu():
     assert lib.spindlekv_compact(C.byref(batch), 2, 128, good, p, p, None, f32, None, None) == B.UNSUPPORTED
     assert lib.spindlekv_reconstruct(C.byref(batch), 2, 128, good, None, p, good, None) == B.INVALID_ARG
     assert lib.spindlekv_reconstruct(C.byref(batch), 2, 96, good, p, p, good, None) == B.UNSUPPORTED
-    assert lib.spindlekv_union_lists(1, 2, 2, 4, 100, 60, p, p, 400, 200, p, p, None) == B.INVALID_ARG   # 2 x 60 > 100
-    assert lib.spindlekv_union_lists(1, 1, 2, 4, 100, 100, None, p, 400, 400, p, p, None) == B.INVALID_ARG
+    assert lib.spindlekv_union_lists(1, 2, 2, 4, 0, 100, 60, p, p, 400, 200, p, p, None) == B.INVALID_ARG   # 2 x 60 > 100
+    assert lib.spindlekv_union_lists(1, 1, 2, 4, 1, 100, 100, None, p, 400, 400, p, p, None) == B.INVALID_ARG
     assert lib.spindlekv_match_workspace_bytes(C.byref(both), 2) == 0
     assert lib.spindlekv_match_workspace_bytes(C.byref(batch), 2) >= 8 * 2 * 1024
     assert lib.spindlekv_codebook_match(C.byref(batch), 2, 128, good, good, p, 0, 0.98, p, p, p, p, p, 1 << 20, None) == B.INVALID_ARG
