@@ -103,8 +103,6 @@ def _load() -> C.CDLL:
     lib.spindlekv_set_tuning.argtypes = [C.c_int32, C.c_int64]
     lib.spindlekv_get_tuning.restype = C.c_int64
     lib.spindlekv_get_tuning.argtypes = [C.c_int32]
-    lib.spindlekv_selftest_grid_barrier_timeout.restype = C.c_int32
-    lib.spindlekv_selftest_grid_barrier_timeout.argtypes = [C.c_void_p, C.c_int64, C.c_void_p]
     lib.spindlekv_selftest_mbarrier_timeout.restype = C.c_int32
     lib.spindlekv_selftest_mbarrier_timeout.argtypes = [C.c_void_p, C.c_int64, C.c_void_p]
     lib.spindlekv_launch_count.restype = C.c_int64
@@ -349,7 +347,7 @@ def spindlekv_poll_status(ws: Optional[torch.Tensor]):
     return int(status.value), [int(x) for x in detail]
 
 
-TUNE_RECORDS_PER_TILE, TUNE_SPIN_LIMIT, TUNE_GREEDY_ROUND_CAP, TUNE_MBAR_WAIT_CYCLES = range(4)
+TUNE_RECORDS_PER_TILE, TUNE_GREEDY_ROUND_CAP, TUNE_MBAR_WAIT_CYCLES = range(3)
 
 
 def spindlekv_set_tuning(key: int, value: int) -> None:
@@ -359,11 +357,6 @@ def spindlekv_set_tuning(key: int, value: int) -> None:
 
 def spindlekv_get_tuning(key: int) -> int:
     return int(_lib.spindlekv_get_tuning(key))
-
-
-def spindlekv_selftest_grid_barrier_timeout(ws: torch.Tensor, limit: int, stream=None) -> None:
-    """Test hook: a grid-wide barrier that cannot complete; must leave TIMEOUT in the status word of ``ws``."""
-    _check(_lib.spindlekv_selftest_grid_barrier_timeout(_ptr(ws), limit, _stream(stream)), "spindlekv_selftest_grid_barrier_timeout")
 
 
 def spindlekv_selftest_mbarrier_timeout(ws: torch.Tensor, limit: int, stream=None) -> None:

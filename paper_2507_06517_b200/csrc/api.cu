@@ -52,12 +52,11 @@ spindlekv_status append_impl(const spindlekv_batch& b, int n_heads, int head_dim
                              const int32_t* n_left_entries, const int32_t* left_idx, const int32_t* left_cnt,
                              const spindlekv_tensor& C, int c_rows, int32_t* n_entries, int32_t* ref_new, cudaStream_t st);
 
-spindlekv_status selftest_grid_barrier_impl(uint32_t* hdr, uint32_t spin_limit, cudaStream_t st);
 spindlekv_status selftest_mbarrier_impl(uint32_t* hdr, long long wait_cycles, cudaStream_t st);
 
 // ---- limits that tests may tighten --------------------------------------------------------------
 static std::mutex g_tune_mu;
-static Tuning g_tuning{kDefaultRecPerTile, kDefaultSpinLimit, 0x7FFFFFFF, kDefaultMbarWaitCycles};
+static Tuning g_tuning{kDefaultRecPerTile, 0x7FFFFFFF, kDefaultMbarWaitCycles};
 Tuning current_tuning() {
   std::lock_guard<std::mutex> lk(g_tune_mu);
   return g_tuning;
@@ -331,9 +330,6 @@ spindlekv_status spindlekv_set_tuning(int32_t key, int64_t value) {
     case SPINDLEKV_TUNE_RECORDS_PER_TILE:
       g_tuning.rec_per_tile = value < 0 ? kDefaultRecPerTile : (int)std::min<int64_t>(value, kDefaultRecPerTile);
       return SPINDLEKV_OK;
-    case SPINDLEKV_TUNE_SPIN_LIMIT:
-      g_tuning.spin_limit = value < 0 ? kDefaultSpinLimit : (uint32_t)std::min<int64_t>(value, 0xFFFFFFFFll);
-      return SPINDLEKV_OK;
     case SPINDLEKV_TUNE_GREEDY_ROUND_CAP:
       g_tuning.round_cap = value < 0 ? 0x7FFFFFFF : (int)std::min<int64_t>(value, 0x7FFFFFFF);
       return SPINDLEKV_OK;
@@ -349,16 +345,10 @@ int64_t spindlekv_get_tuning(int32_t key) {
   const Tuning t = current_tuning();
   switch (key) {
     case SPINDLEKV_TUNE_RECORDS_PER_TILE: return t.rec_per_tile;
-    case SPINDLEKV_TUNE_SPIN_LIMIT: return t.spin_limit;
     case SPINDLEKV_TUNE_GREEDY_ROUND_CAP: return t.round_cap;
     case SPINDLEKV_TUNE_MBAR_WAIT_CYCLES: return t.mbar_wait_cycles;
     default: return -1;
   }
-}
-
-spindlekv_status spindlekv_selftest_grid_barrier_timeout(void* ws, int64_t limit, void* stream) {
-  if (!ws || reinterpret_cast<uintptr_t>(ws) % 256 || limit < 1 || limit > (int64_t)kDefaultSpinLimit) return SPINDLEKV_INVALID_ARG;
-  return selftest_grid_barrier_impl(reinterpret_cast<uint32_t*>(ws), (uint32_t)limit, (cudaStream_t)stream);
 }
 
 spindlekv_status spindlekv_selftest_mbarrier_timeout(void* ws, int64_t limit, void* stream) {

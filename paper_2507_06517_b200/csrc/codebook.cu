@@ -37,7 +37,8 @@ struct CodebookParams {
   int32_t* rank;         // [units][max_len] entry number of a centre
   int32_t* lists;        // [units][list_cap] neighbour lists, one contiguous run per row, starting at lbase[row]
   int32_t* ell_cnt;      // [units][max_len] list length n <= kEll; -1: use the bit row; -1 - n: a list of n > kEll neighbours
-  int32_t* dense_rows;   // rows (unit * max_len + token) with more than kEll neighbours; count in the header
+  int32_t* dense_rows;   // [units][max_len] tokens with more than kEll neighbours, in no particular order
+  int32_t* dense_cnt;    // [units] how many
   uint32_t* flags;       // [units][row_words][row_words/2] bit r of word [w][c]: chunk c (64 columns) of row 32w+r may hold a bit
   uint32_t* hdr;
   int32_t* ref;          // [layers][H][T]
@@ -51,7 +52,6 @@ struct CodebookParams {
   long long unit_rec_cap;
   int32_t* lbase;        // [units][max_len] start of a row's list within its unit's part of `lists`
   int list_cap;          // entries per unit (at least kEll per row: the bit-matrix path gives every row kEll slots)
-  uint32_t spin_limit;   // polls after which a grid barrier gives up
   int round_cap;         // rounds after which the greedy cover gives up
 };
 
@@ -182,50 +182,7 @@ __global__ void __launch_bounds__(256) sim_simt_kernel(CodebookParams p) {
   }
 }
 
-// ---- grid-wide barrier and warp helpers of the cooperative greedy kernel ------------------------
-
-// Grid-wide barrier on a monotonically increasing counter.  Every wait is bounded: when it gives up
-// (after `spin_limit` polls) it raises the TIMEOUT status, and every block that sees a non-zero status
-// leaves the kernel.
-__device__ __forceinline__ bool grid_barrier(uint32_t* hdr, uint32_t& target, uint32_t spin_limit) {
-  __shared__ int ok_sh;
-  __syncthreads();
-  target += gridDim.x;
-  if (threadIdx.x == 0) {
-    int ok = 1;
-    __threadfence();
-    atomicAdd(&hdr[kHdrBarrier], 1u);
-    uint32_t spins = 0;
-    while (true) {
-      uint32_t v = *reinterpret_cast<volatile uint32_t*>(&hdr[kHdrBarrier]);
-      if (v >= target) break;
-      if (*reinterpret_cast<volatile uint32_t*>(&hdr[kHdrStatus]) != 0u || ++spins > spin_limit) {
-        atomicExch(&hdr[kHdrStatus], (uint32_t)SPINDLEKV_TIMEOUT);
-        ok = 0;
-        break;
-      }
-      __nanosleep(64);
-    }
-    __threadfence();
-    ok_sh = ok;
-  }
-  __syncthreads();
-  return ok_sh != 0;
-}
-
-// Self-test of the bounded barrier: the blocks of this launch are one short of the arrivals the barrier
-// expects, so the wait must run out, raise TIMEOUT in the status word and let every block return.
-__global__ void barrier_selftest_kernel(uint32_t* hdr, uint32_t spin_limit) {
-  uint32_t target = 1;   // one arrival more than the grid will ever deliver
-  const bool ok = grid_barrier(hdr, target, spin_limit);
-  if (ok && threadIdx.x == 0) hdr[kHdrLive] = 0xBADu;   // must not happen
-}
-
-spindlekv_status selftest_grid_barrier_impl(uint32_t* hdr, uint32_t spin_limit, cudaStream_t st) {
-  if (cudaMemsetAsync(hdr, 0, kHeaderBytes, st) != cudaSuccess) return SPINDLEKV_CUDA;
-  barrier_selftest_kernel<<<2, 64, 0, st>>>(hdr, spin_limit);
-  return cudaGetLastError() == cudaSuccess ? SPINDLEKV_OK : SPINDLEKV_CUDA;
-}
+// ---- warp helpers of the greedy kernels ------------------------------------------------------------
 
 __device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long v) {
 #pragma unroll
@@ -332,7 +289,7 @@ __global__ void __launch_bounds__(256, 5) extract_kernel(CodebookParams p) {
       p.owner[idx] = u;
     } else {
       live = true;
-      if (cnt - 1 > kEll) p.dense_rows[atomicAdd(&p.hdr[kHdrDenseCnt], 1u)] = (int32_t)idx;
+      if (cnt - 1 > kEll) p.dense_rows[(int64_t)unit * ML + atomicAdd(&p.dense_cnt[unit], 1)] = u;
     }
   }
   // all tokens that still have a neighbour start live (both copies of the mask)
@@ -447,7 +404,7 @@ __global__ void __launch_bounds__(kBuildThreads) build_lists_kernel(CodebookPara
       p.lbase[idx] = start;
       p.pickdeg[idx] = cnt == 1 ? 1 : -1;   // a token without a neighbour is a centre of pick degree 1
       if (cnt == 1) p.owner[idx] = u;
-      if (d > kEll) p.dense_rows[atomicAdd(&p.hdr[kHdrDenseCnt], 1u)] = (int32_t)idx;
+      if (d > kEll) p.dense_rows[row0 + atomicAdd(&p.dense_cnt[unit], 1)] = u;
     }
     const uint32_t word = __ballot_sync(0xffffffffu, exists && d > 0);   // tokens with a neighbour start live
     if (lane == 0) {
@@ -750,122 +707,123 @@ __device__ __forceinline__ void pick_big_row(const CodebookParams& p, const uint
   else pick_long_row(p, live, next, idx, -1 - ec, lane);
 }
 
-// Round 0 as two ordinary launches: every row is still live, so the phases run with one warp per word of
-// the live mask over the whole grid (far more threads in flight than the cooperative kernel can keep
-// resident); the last kDenseBlocks blocks walk the list of dense rows.  `phase` 2: neighbourhood maxima,
-// 3: picks.
-constexpr int kDenseBlocks = 148;
+// Phase 1 for the 32 rows of live-mask word w: live degrees (Eq. (10)) and keys of the rows with a list.
+__device__ __forceinline__ void degrees_of_listed_rows(const CodebookParams& p, const uint32_t* live, int64_t w, uint32_t lvw,
+                                                       int lane) {
+  if (!((lvw >> lane) & 1u)) return;
+  const int ML = p.batch.max_len, RW = p.row_words;
+  const int unit = (int)(w / RW), u = (int)(w - (int64_t)unit * RW) * 32 + lane;
+  const int64_t idx = (int64_t)unit * ML + u;
+  const int ec = p.ell_cnt[idx];
+  if (ec < 0) return;                             // rows with many neighbours: separately
+  const uint32_t* lv = live + (int64_t)unit * RW;
+  const int32_t* list = list_of(p, unit, idx);
+  int cnt = 1;
+  for (int k0 = 0; k0 < ec; k0 += kBatch) {
+    int v[kBatch];
+    load_batch(list, k0, ec, v);
+    keep_live(lv, v);
+#pragma unroll
+    for (int i = 0; i < kBatch; ++i) cnt += v[i] >= 0 ? 1 : 0;
+  }
+  p.deg[idx] = cnt;
+  p.key[idx] = ((unsigned long long)(uint32_t)cnt << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)u);
+}
 
-__global__ void __launch_bounds__(256) greedy_first_round_kernel(CodebookParams p, int phase, int word_blocks) {
-  const int lane = threadIdx.x & 31;
-  if ((int)blockIdx.x < word_blocks) {
-    const int64_t w = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    if (w >= (int64_t)p.n_units * p.row_words) return;
-    if (phase == 2) max_of_listed_rows<true>(p, p.live0, w, lane);
-    else pick_listed_rows<true>(p, p.live0, p.live1, w, lane);
-  } else {
-    const int n_dense = (int)p.hdr[kHdrDenseCnt];
-    const int nw = kDenseBlocks * (blockDim.x >> 5);
-    for (int d = ((int)blockIdx.x - word_blocks) * (blockDim.x >> 5) + (threadIdx.x >> 5); d < n_dense; d += nw) {
-      if (phase == 2) max_of_big_row(p, p.live0, p.dense_rows[d], lane);
-      else pick_big_row(p, p.live0, p.live1, p.dense_rows[d], lane);
-    }
+// Phase 1 for one row that uses its bit row.
+__device__ __forceinline__ void degree_of_dense_row(const CodebookParams& p, const uint32_t* live, int64_t idx, int lane) {
+  const int ML = p.batch.max_len, RW = p.row_words, RW4 = RW >> 2;
+  const int unit = (int)(idx / ML), u = (int)(idx - (int64_t)unit * ML);
+  const uint32_t* lv = live + (int64_t)unit * RW;
+  if (!is_live(lv, u)) return;
+  const uint4* row4 = reinterpret_cast<const uint4*>(p.adj + idx * RW);
+  const uint4* lv4 = reinterpret_cast<const uint4*>(lv);
+  const uint32_t* fr = flag_row(p, unit, u);
+  int cnt = 0;
+  for (int w4 = lane; w4 < RW4; w4 += 32) {
+    const uint4 a = row4[w4], b = lv4[w4];
+    if (chunk_flagged(fr, 2 * w4, u)) cnt += __popc(a.x & b.x) + __popc(a.y & b.y);
+    if (chunk_flagged(fr, 2 * w4 + 1, u)) cnt += __popc(a.z & b.z) + __popc(a.w & b.w);
+  }
+#pragma unroll
+  for (int o = 16; o >= 1; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+  if (lane == 0) {
+    p.deg[idx] = cnt;
+    p.key[idx] = ((unsigned long long)(uint32_t)cnt << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)u);
   }
 }
 
-// Rounds 1, 2, ...: few rows are left, one cooperative launch runs them to the end.
-__global__ void __launch_bounds__(512) greedy_kernel(CodebookParams p) {
-  const int lane = threadIdx.x & 31;
-  const int warps_per_block = blockDim.x >> 5;
-  const int64_t gwarp = (int64_t)blockIdx.x * warps_per_block + (threadIdx.x >> 5);
-  const int64_t nwarps = (int64_t)gridDim.x * warps_per_block;
-  const int64_t gthread = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  const int ML = p.batch.max_len, RW = p.row_words, RW4 = RW >> 2;
-  const int64_t n_words = (int64_t)p.n_units * RW;
-  const int n_dense = (int)*reinterpret_cast<volatile uint32_t*>(&p.hdr[kHdrDenseCnt]);
-  uint32_t target = 0;
+// The greedy cover of one unit, all rounds, by one block: units are independent graphs, so the three phases of a
+// round are separated by block barriers only, and a unit stops as soon as it has no live token left, whatever the
+// other units still do.  Round 0 finds every token with a neighbour live and its degree known from the list
+// building; later rounds first recount the degrees of the tokens that are left.  A warp takes the 32 rows of one
+// word of the unit's live mask (empty words cost one load); rows with more than kEll neighbours come from the
+// unit's own list of such rows, a warp per row.
+constexpr int kCoverThreads = 1024;
 
+__global__ void __launch_bounds__(kCoverThreads) cover_kernel(CodebookParams p) {
+  __shared__ int live_total;
+  const int unit = blockIdx.x;
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  constexpr int NW = kCoverThreads / 32;
+  const int ML = p.batch.max_len, RW = p.row_words;
+  const int64_t w0 = (int64_t)unit * RW;
+  const int32_t* big = p.dense_rows + (int64_t)unit * ML;
+  const int n_big = p.dense_cnt[unit];
   const int round_cap = min(ML, p.round_cap);
-  int round = 1;
-  for (; round <= round_cap; ++round) {
+  int round = 0;
+  bool gave_up = false;
+  for (;; ++round) {
     uint32_t* live = (round & 1) ? p.live1 : p.live0;
     uint32_t* next = (round & 1) ? p.live0 : p.live1;
-    const int slot = (round & 1) ? kHdrLiveCnt1 : kHdrLiveCnt0;
-    const int other = (round & 1) ? kHdrLiveCnt0 : kHdrLiveCnt1;
-    {
-      // phase 1: live degrees (Eq. (10)) and keys; `next` becomes a copy of `live`.
-      if (gthread == 0) p.hdr[other] = 0;
+    if (round > 0) {
+      if (round > round_cap) { gave_up = true; break; }
+      // phase 1: live degrees and keys; `next` becomes a copy of `live`
+      if (tid == 0) live_total = 0;
+      __syncthreads();
       int my_live = 0;
-      for (int64_t w = gwarp; w < n_words; w += nwarps) {
-        const uint32_t lvw = live[w];
-        if (lane == 0) next[w] = lvw;
+      for (int w = wid; w < RW; w += NW) {
+        const uint32_t lvw = live[w0 + w];
+        if (lane == 0) next[w0 + w] = lvw;
         if (!lvw) continue;
         my_live += __popc(lvw);
-        if (!((lvw >> lane) & 1u)) continue;
-        const int unit = (int)(w / RW), u = (int)(w - (int64_t)unit * RW) * 32 + lane;
-        const int64_t idx = (int64_t)unit * ML + u;
+        degrees_of_listed_rows(p, live, w0 + w, lvw, lane);
+      }
+      for (int d = wid; d < n_big; d += NW) {
+        const int64_t idx = (int64_t)unit * ML + big[d];
         const int ec = p.ell_cnt[idx];
-        if (ec < 0) continue;                       // dense rows: below
-        const uint32_t* lv = live + (int64_t)unit * RW;
-        const int32_t* list = list_of(p, unit, idx);
-        int cnt = 1;
-        for (int k0 = 0; k0 < ec; k0 += kBatch) {
-          int v[kBatch];
-          load_batch(list, k0, ec, v);
-          keep_live(lv, v);
-#pragma unroll
-          for (int i = 0; i < kBatch; ++i) cnt += v[i] >= 0 ? 1 : 0;
-        }
-        p.deg[idx] = cnt;
-        p.key[idx] = ((unsigned long long)(uint32_t)cnt << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)u);
+        if (ec == -1) degree_of_dense_row(p, live, idx, lane);
+        else degree_of_long_row(p, live, idx, -1 - ec, lane);
       }
-      for (int64_t d = gwarp; d < n_dense; d += nwarps) {
-        const int64_t idx = p.dense_rows[d];
-        const int ec_big = p.ell_cnt[idx];
-        if (ec_big != -1) {
-          degree_of_long_row(p, live, idx, -1 - ec_big, lane);
-          continue;
-        }
-        const int unit = (int)(idx / ML), u = (int)(idx - (int64_t)unit * ML);
-        const uint32_t* lv = live + (int64_t)unit * RW;
-        if (!is_live(lv, u)) continue;
-        const uint4* row4 = reinterpret_cast<const uint4*>(p.adj + idx * RW);
-        const uint4* lv4 = reinterpret_cast<const uint4*>(lv);
-        const uint32_t* fr = flag_row(p, unit, u);
-        int cnt = 0;
-        for (int w4 = lane; w4 < RW4; w4 += 32) {
-          const uint4 a = row4[w4], b = lv4[w4];
-          if (chunk_flagged(fr, 2 * w4, u)) cnt += __popc(a.x & b.x) + __popc(a.y & b.y);
-          if (chunk_flagged(fr, 2 * w4 + 1, u)) cnt += __popc(a.z & b.z) + __popc(a.w & b.w);
-        }
-#pragma unroll
-        for (int o = 16; o >= 1; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
-        if (lane == 0) {
-          p.deg[idx] = cnt;
-          p.key[idx] = ((unsigned long long)(uint32_t)cnt << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)u);
-        }
-      }
-      if (lane == 0 && my_live) atomicAdd(&p.hdr[slot], (uint32_t)my_live);
-      if (!grid_barrier(p.hdr, target, p.spin_limit)) return;
-      const uint32_t total_live = *reinterpret_cast<volatile uint32_t*>(&p.hdr[slot]);
-      if (total_live == 0) break;
+      if (lane == 0 && my_live) atomicAdd(&live_total, my_live);
+      __syncthreads();
+      if (live_total == 0) break;
     }
-
     // phase 2: largest key in each closed live neighbourhood
-    for (int64_t w = gwarp; w < n_words; w += nwarps) max_of_listed_rows<false>(p, live, w, lane);
-    for (int64_t d = gwarp; d < n_dense; d += nwarps) max_of_big_row(p, live, p.dense_rows[d], lane);
-    if (!grid_barrier(p.hdr, target, p.spin_limit)) return;
-
-    // phase 3: picks
-    for (int64_t w = gwarp; w < n_words; w += nwarps) pick_listed_rows<false>(p, live, next, w, lane);
-    for (int64_t d = gwarp; d < n_dense; d += nwarps) pick_big_row(p, live, next, p.dense_rows[d], lane);
-    if (!grid_barrier(p.hdr, target, p.spin_limit)) return;
+    for (int w = wid; w < RW; w += NW) {
+      if (round == 0) max_of_listed_rows<true>(p, live, w0 + w, lane);
+      else max_of_listed_rows<false>(p, live, w0 + w, lane);
+    }
+    for (int d = wid; d < n_big; d += NW) max_of_big_row(p, live, (int64_t)unit * ML + big[d], lane);
+    __syncthreads();
+    // phase 3: picks (Eq. (11)-(13))
+    for (int w = wid; w < RW; w += NW) {
+      if (round == 0) pick_listed_rows<true>(p, live, next, w0 + w, lane);
+      else pick_listed_rows<false>(p, live, next, w0 + w, lane);
+    }
+    for (int d = wid; d < n_big; d += NW) pick_big_row(p, live, next, (int64_t)unit * ML + big[d], lane);
+    __syncthreads();
   }
-  if (gthread == 0) {
-    p.hdr[kHdrRounds] = (uint32_t)round;
-    uint32_t left = *reinterpret_cast<volatile uint32_t*>(&p.hdr[(round & 1) ? kHdrLiveCnt1 : kHdrLiveCnt0]);
-    p.hdr[kHdrLive] = round > round_cap ? max(left, 1u) : left;
-    if (round > round_cap) atomicExch(&p.hdr[kHdrStatus], (uint32_t)SPINDLEKV_TIMEOUT);
+  if (tid == 0) {
+    atomicMax(&p.hdr[kHdrRounds], (uint32_t)round);
+    if (gave_up) {
+      // the round that was not run: its live tokens are the ones left without a centre
+      const uint32_t* live = (round & 1) ? p.live1 : p.live0;
+      uint32_t left = 0;
+      for (int w = 0; w < RW; ++w) left += __popc(live[w0 + w]);
+      atomicAdd(&p.hdr[kHdrLive], max(left, 1u));
+      atomicExch(&p.hdr[kHdrStatus], (uint32_t)SPINDLEKV_TIMEOUT);
+    }
   }
 }
 
@@ -1057,7 +1015,7 @@ __global__ void __launch_bounds__(kFinalThreads) finalize_kernel(CodebookParams 
 
 struct CodebookLayout {
   size_t ext, ell, ell_cnt, dense_rows, flags, adj, deg, key, m1, live0, live1, owner, pickdeg, rank, total;
-  size_t ovf, rec_cnt, lbase, rec;   // candidate records (tensor-core path)
+  size_t ovf, rec_cnt, dense_cnt, lbase, rec;   // candidate records (tensor-core path)
   int rec_per_tile, n_blocks, list_cap;
 };
 
@@ -1092,6 +1050,7 @@ static CodebookLayout codebook_layout(const spindlekv_config& cfg, const spindle
   L.n_blocks = 2 * ceil_div(b.max_len, 256);
   L.ovf = take(units * 4);
   L.rec_cnt = take(units * L.n_blocks * 4);
+  L.dense_cnt = take(units * 4);
   L.lbase = take(units * ML * 4);
   L.rec = take(L.rec_per_tile ? units * (size_t)rec_unit_capacity(L.n_blocks / 2, L.rec_per_tile) * 8 : 0);
   L.adj = off;
@@ -1158,6 +1117,7 @@ spindlekv_status codebook_shallow_impl(const spindlekv_config& cfg, const spindl
   p.lists = reinterpret_cast<int32_t*>(w + L.ell);
   p.ell_cnt = reinterpret_cast<int32_t*>(w + L.ell_cnt);
   p.dense_rows = reinterpret_cast<int32_t*>(w + L.dense_rows);
+  p.dense_cnt = reinterpret_cast<int32_t*>(w + L.dense_cnt);
   p.flags = reinterpret_cast<uint32_t*>(w + L.flags);
   p.hdr = reinterpret_cast<uint32_t*>(w);
   p.ref = ref;
@@ -1171,11 +1131,12 @@ spindlekv_status codebook_shallow_impl(const spindlekv_config& cfg, const spindl
   p.unit_rec_cap = records ? rec_unit_capacity(L.n_blocks / 2, L.rec_per_tile) : 0;
   p.lbase = reinterpret_cast<int32_t*>(w + L.lbase);
   p.list_cap = L.list_cap;
-  p.spin_limit = tune.spin_limit;
   p.round_cap = tune.round_cap;
   if (cudaMemsetAsync(w, 0, kHeaderBytes, st) != cudaSuccess) return SPINDLEKV_CUDA;
-  // overflow flags and record counts: all zero on the record path; without records every unit counts as overflowed
-  if (cudaMemsetAsync(w + L.ovf, records ? 0 : 1, L.lbase - L.ovf, st) != cudaSuccess) return SPINDLEKV_CUDA;
+  // overflow flags and record counts: all zero on the record path; without records every unit counts as overflowed;
+  // the per-unit counts of rows with many neighbours start at zero
+  if (cudaMemsetAsync(w + L.ovf, records ? 0 : 1, L.dense_cnt - L.ovf, st) != cudaSuccess) return SPINDLEKV_CUDA;
+  if (cudaMemsetAsync(w + L.dense_cnt, 0, L.lbase - L.dense_cnt, st) != cudaSuccess) return SPINDLEKV_CUDA;
   p.ext = tc ? reinterpret_cast<__nv_bfloat16*>(w + L.ext) : nullptr;
   if (cfg.head_dim == 64) {
     if (bf) launch_norms<__nv_bfloat16, 64>(p, st); else launch_norms<float, 64>(p, st);
@@ -1227,28 +1188,11 @@ spindlekv_status codebook_shallow_impl(const spindlekv_config& cfg, const spindl
     LaunchScope ls(KC_DEGREE, st);
     expand_records_kernel<<<units, kBuildThreads, 0, st>>>(p, adj_bits);
   }
-  // cooperative launch: as many blocks as can be resident at once
-  static int coop_blocks_dev[kMaxDevices] = {};
   const int dev = PerDeviceOnce::current();
   if (dev < 0) return SPINDLEKV_CUDA;
-  if (coop_blocks_dev[dev] == 0) {
-    int sms = 0, per_sm = 0;
-    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return SPINDLEKV_CUDA;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, greedy_kernel, 512, 0) != cudaSuccess) return SPINDLEKV_CUDA;
-    if (per_sm < 1) return SPINDLEKV_CUDA;
-    coop_blocks_dev[dev] = sms * per_sm;
-  }
-  const int coop_blocks = coop_blocks_dev[dev];
-  for (int phase = 2; phase <= 3; ++phase) {
-    const int word_blocks = (int)(((size_t)units * p.row_words * 32 + 255) / 256);
-    LaunchScope ls(KC_GREEDY, st);
-    greedy_first_round_kernel<<<word_blocks + kDenseBlocks, 256, 0, st>>>(p, phase, word_blocks);
-  }
   {
     LaunchScope ls(KC_GREEDY, st);
-    void* args[] = {&p};
-    if (cudaLaunchCooperativeKernel((const void*)greedy_kernel, dim3(coop_blocks), dim3(512), args, 0, st) != cudaSuccess)
-      return SPINDLEKV_CUDA;
+    cover_kernel<<<units, kCoverThreads, 0, st>>>(p);
   }
   {
     size_t smem = (size_t)(b.max_len + 2) * 4;

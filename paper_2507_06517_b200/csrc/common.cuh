@@ -12,17 +12,13 @@ namespace skv {
 // ---- status block at the start of every workspace -------------------------------------------
 // word 0: device status, 1: greedy rounds used, 2: live tokens left, 3: units whose neighbour lists came from a bit matrix,
 // 4: neighbour-list entries built from candidate records (both directions of every pair),
-// words 8..: barrier and counters of the cooperative greedy kernel.
+// the rest is unused.
 constexpr int kHeaderBytes = 256;
 constexpr int kHdrStatus = 0;
 constexpr int kHdrRounds = 1;
 constexpr int kHdrLive = 2;
 constexpr int kHdrBitUnits = 3;
 constexpr int kHdrListEntries = 4;
-constexpr int kHdrBarrier = 8;
-constexpr int kHdrLiveCnt0 = 9;   // two slots, alternated by round parity
-constexpr int kHdrLiveCnt1 = 10;
-constexpr int kHdrDenseCnt = 11;  // rows with too many neighbours for a list
 
 // kernel classes for launch counting / timing
 enum KernelClass { KC_WINDOW = 0, KC_TOPK, KC_NORMS, KC_SIM, KC_DEGREE, KC_GREEDY, KC_FINAL, KC_GATHER, KC_COUNT };
@@ -178,11 +174,9 @@ struct PerDeviceOnce {
 
 // ---- limits that tests may tighten (host) -----------------------------------------------------------
 constexpr int kDefaultRecPerTile = 512;             // candidate records per 128 x 256 tile of a row block's region
-constexpr uint32_t kDefaultSpinLimit = 4u << 20;    // polls of a grid barrier
 constexpr long long kDefaultMbarWaitCycles = 4000000000ll;   // about two seconds of SM clock
 struct Tuning {
   int rec_per_tile;          // 0: no candidate records, every unit goes through the bit matrix
-  uint32_t spin_limit;
   int round_cap;             // greedy rounds (never more than the sequence length)
   long long mbar_wait_cycles;
 };

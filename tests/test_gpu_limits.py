@@ -17,7 +17,7 @@ pytestmark = pytest.mark.gpu
 def _restore_limits():
     from paper_2507_06517_b200 import binding as B
     yield
-    for k in range(4):
+    for k in range(3):
         B.spindlekv_set_tuning(k, -1)
 
 
@@ -107,10 +107,6 @@ def test_dense_graph_goes_through_the_bit_matrix_by_itself():
 def test_bounded_waits_run_out_and_report_timeout():
     from paper_2507_06517_b200 import binding as B
     ws = torch.zeros(4096, dtype=torch.uint8, device="cuda")
-    B.spindlekv_selftest_grid_barrier_timeout(ws, 2000)
-    torch.cuda.synchronize()
-    status, detail = B.spindlekv_poll_status(ws)
-    assert status == B.TIMEOUT and detail[1] == 0         # both blocks gave up and returned; nobody got through
     B.spindlekv_selftest_mbarrier_timeout(ws, 20000)      # about ten microseconds of SM clock
     torch.cuda.synchronize()
     status, detail = B.spindlekv_poll_status(ws)
