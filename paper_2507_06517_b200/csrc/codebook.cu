@@ -28,10 +28,7 @@ struct CodebookParams {
                          // ([0]: theta*|gamma|, [1]: |gamma|, each in three bf16 pieces; zero beyond the sequence)
   uint32_t* adj;         // [units][max_len][row_words]
   int32_t* deg;          // [units][max_len]
-  unsigned long long* key;  // [units][max_len]
-  unsigned long long* m1;   // [units][max_len]
-  uint32_t* live0;       // [units][row_words]
-  uint32_t* live1;
+  uint32_t* live0;       // [units][row_words] tokens that have a neighbour: live when the greedy cover starts
   int32_t* owner;        // [units][max_len]
   int32_t* pickdeg;      // [units][max_len], -1 = not a centre
   int32_t* rank;         // [units][max_len] entry number of a centre
@@ -182,23 +179,12 @@ __global__ void __launch_bounds__(256) sim_simt_kernel(CodebookParams p) {
   }
 }
 
-// ---- warp helpers of the greedy kernels ------------------------------------------------------------
-
-__device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long v) {
-#pragma unroll
-  for (int o = 16; o >= 1; o >>= 1) {
-    unsigned long long n = __shfl_xor_sync(0xffffffffu, v, o);
-    v = n > v ? n : v;
-  }
-  return v;
-}
-
 // ---- neighbour lists ------------------------------------------------------------------------------
 // One thread per row.  The similarity kernel left one bit per (row, 64-column chunk) that says
 // whether the chunk may hold a set bit (a word holds the bits of 32 rows: a warp reads the words of 256
 // chunks, eight per lane, and transposes them into per-row occupancy words); only those chunks of the bit
 // row are read, several at a time.  Written per row:
-// the initial degree (Eq. (10)) and key, and, for rows with at most kEll neighbours (the row itself
+// the initial degree (Eq. (10)), and, for rows with at most kEll neighbours (the row itself
 // not counted), the ascending list of those neighbours in the row's kEll slots of `lists`.
 // Rows with more neighbours keep using their bit row
 // and are appended to a list of dense rows.  A token with no neighbour at all is settled here: it is
@@ -281,7 +267,6 @@ __global__ void __launch_bounds__(256, 5) extract_kernel(CodebookParams p) {
   bool live = false;
   if (exists) {
     p.deg[idx] = cnt;
-    p.key[idx] = ((unsigned long long)(uint32_t)cnt << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)u);
     p.ell_cnt[idx] = cnt - 1 <= kEll ? cnt - 1 : -1;
     p.lbase[idx] = u * kEll;
     p.pickdeg[idx] = cnt == 1 ? 1 : -1;   // -1: not a centre (until the greedy cover picks it)
@@ -292,12 +277,9 @@ __global__ void __launch_bounds__(256, 5) extract_kernel(CodebookParams p) {
       if (cnt - 1 > kEll) p.dense_rows[(int64_t)unit * ML + atomicAdd(&p.dense_cnt[unit], 1)] = u;
     }
   }
-  // all tokens that still have a neighbour start live (both copies of the mask)
+  // all tokens that still have a neighbour start live
   const uint32_t word = __ballot_sync(0xffffffffu, live);
-  if (lane == 0) {
-    p.live0[(int64_t)unit * RW + (u >> 5)] = word;
-    p.live1[(int64_t)unit * RW + (u >> 5)] = word;
-  }
+  if (lane == 0) p.live0[(int64_t)unit * RW + (u >> 5)] = word;
 }
 
 // ---- neighbour lists from candidate records ------------------------------------------------------
@@ -309,7 +291,7 @@ __global__ void __launch_bounds__(256, 5) extract_kernel(CodebookParams p) {
 // per pair), so the scattered 4-byte stores of the last step meet in the L2 cache.  The order inside a
 // list depends on the order in which the atomics land; nothing downstream depends on it (maxima, counts
 // and ownership by the single centre within reach are all independent of it).  Everything else the
-// bit-matrix path's extraction pass leaves behind is written here too: degree, key, live masks, settled
+// bit-matrix path's extraction pass leaves behind is written here too: degree, live mask, settled
 // isolated tokens, the list of rows with more than kEll neighbours (which the greedy kernels walk a warp
 // per row).  A unit whose lists do not fit `list_cap` raises its overflow flag and goes through the bit
 // matrix instead.
@@ -399,7 +381,6 @@ __global__ void __launch_bounds__(kBuildThreads) build_lists_kernel(CodebookPara
     if (exists) {
       const int cnt = d + 1;
       p.deg[idx] = cnt;
-      p.key[idx] = ((unsigned long long)(uint32_t)cnt << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)u);
       p.ell_cnt[idx] = d <= kEll ? d : -1 - d;
       p.lbase[idx] = start;
       p.pickdeg[idx] = cnt == 1 ? 1 : -1;   // a token without a neighbour is a centre of pick degree 1
@@ -407,10 +388,7 @@ __global__ void __launch_bounds__(kBuildThreads) build_lists_kernel(CodebookPara
       if (d > kEll) p.dense_rows[row0 + atomicAdd(&p.dense_cnt[unit], 1)] = u;
     }
     const uint32_t word = __ballot_sync(0xffffffffu, exists && d > 0);   // tokens with a neighbour start live
-    if (lane == 0) {
-      p.live0[(int64_t)unit * RW + (u0 >> 5)] = word;
-      p.live1[(int64_t)unit * RW + (u0 >> 5)] = word;
-    }
+    if (lane == 0) p.live0[(int64_t)unit * RW + (u0 >> 5)] = word;
   }
   __syncthreads();
   int32_t* lists = p.lists + (int64_t)unit * p.list_cap;
@@ -456,9 +434,18 @@ __global__ void __launch_bounds__(kBuildThreads) expand_records_kernel(CodebookP
   });
 }
 
-// ---- greedy cover, cooperative kernel over all units of the call --------------------------------
-// Rows with a neighbour list are handled one per thread (a warp takes the 32 rows of one word of the
-// live mask and skips words that are empty), dense rows one per warp from their list.
+// ---- greedy cover: one block per unit, its state on chip ----------------------------------------------
+// Units are independent graphs, so a block runs all rounds of its unit with block barriers between the three
+// phases of a round and stops as soon as the unit has no live token left, whatever the other units still do.
+// What the phases gather from at random sits in shared memory: the two live masks, the key of every token
+// (live degree in the high half, 0xFFFF - index in the low half: larger degree first, lower index on ties) and,
+// per token, the index of the largest key in its closed live neighbourhood.  What stays in global memory is
+// read once per row and phase: the row's list (or, on the bit-matrix path, its bit row).
+//
+// Round 0 finds every token with a neighbour live and its degree known from the list building; the rounds after
+// it first collect the tokens that are left into a list (as a rule a few per cent) and work on that list, one
+// thread per token, instead of sweeping the live mask.  Rows with more than kEll neighbours are taken a warp
+// per row from the unit's list of such rows.
 __device__ __forceinline__ bool is_live(const uint32_t* lv, int v) { return (lv[v >> 5] >> (v & 31)) & 1u; }
 
 // The flag words of token u's group of 32 rows, one per 64-column chunk.  A chunk of a bit row whose flag bit is
@@ -475,104 +462,80 @@ __device__ __forceinline__ void load_batch(const int32_t* list, int k0, int ec, 
 #pragma unroll
   for (int i = 0; i < kBatch; ++i) v[i] = k0 + i < ec ? list[k0 + i] : -1;
 }
-// a row's neighbour list
-__device__ __forceinline__ const int32_t* list_of(const CodebookParams& p, int unit, int64_t idx) {
-  return p.lists + (int64_t)unit * p.list_cap + p.lbase[idx];
-}
 // keeps only the entries that are live (others become -1)
 __device__ __forceinline__ void keep_live(const uint32_t* lv, int (&v)[kBatch]) {
-  uint32_t w[kBatch];
-#pragma unroll
-  for (int i = 0; i < kBatch; ++i) w[i] = v[i] >= 0 ? lv[v[i] >> 5] : 0u;
 #pragma unroll
   for (int i = 0; i < kBatch; ++i)
-    if (!((w[i] >> (v[i] & 31)) & 1u)) v[i] = -1;
+    if (v[i] >= 0 && !is_live(lv, v[i])) v[i] = -1;
 }
 
-// Phase 2 for the 32 rows of live-mask word w: largest key in each closed live neighbourhood.
-// `kAllLive`: every listed neighbour is known to be live (round 0: a token with a neighbour is live),
-// so the live mask need not be consulted per neighbour.
+struct CoverState {        // shared memory of one unit's block
+  uint32_t* key;           // [tokens] (live degree << 16) | (0xFFFF - token)
+  uint16_t* best;          // [tokens] token with the largest key in the closed live neighbourhood
+  uint32_t* live0;         // [row_words] live masks: rounds alternate between the two
+  uint32_t* live1;
+  uint16_t* left;          // [kLeftCap] tokens still live at the start of a round
+};
+constexpr int kLeftCap = 4096;
+constexpr int kCoverMaxTokens = 32768;   // 16-bit token numbers, and 6 bytes of shared memory per token
+
+__device__ __forceinline__ uint32_t make_key(int cnt, int u) { return ((uint32_t)cnt << 16) | (uint32_t)(0xFFFF - u); }
+__device__ __forceinline__ int key_token(uint32_t k) { return 0xFFFF - (int)(k & 0xFFFFu); }
+
+// ---- rows with a list of at most kEll neighbours, one thread per row --------------------------------
+// phase 1: live degree (Eq. (10)) and key
+__device__ __forceinline__ void degree_of_row(const CodebookParams& p, const CoverState& st, const uint32_t* lv, int64_t row0, int u) {
+  const int ec = p.ell_cnt[row0 + u];
+  if (ec < 0) return;                             // rows with many neighbours: separately
+  const int32_t* list = p.lists + p.lbase[row0 + u];
+  int cnt = 1;
+  for (int k0 = 0; k0 < ec; k0 += kBatch) {
+    int v[kBatch];
+    load_batch(list, k0, ec, v);
+    keep_live(lv, v);
+#pragma unroll
+    for (int i = 0; i < kBatch; ++i) cnt += v[i] >= 0 ? 1 : 0;
+  }
+  st.key[u] = make_key(cnt, u);
+}
+
+// phase 2: largest key in the closed live neighbourhood.  `kAllLive`: every listed neighbour is known to be live
+// (round 0: a token with a neighbour is live).
 template <bool kAllLive>
-__device__ __forceinline__ void max_of_listed_rows(const CodebookParams& p, const uint32_t* live, int64_t w, int lane) {
-  const int ML = p.batch.max_len, RW = p.row_words;
-  const uint32_t lvw = live[w];
-  if (!((lvw >> lane) & 1u)) return;
-  const int unit = (int)(w / RW), u = (int)(w - (int64_t)unit * RW) * 32 + lane;
-  const int64_t idx = (int64_t)unit * ML + u;
-  const int ec = p.ell_cnt[idx];
-  if (ec < 0) return;                             // dense rows: separately
-  const uint32_t* lv = live + (int64_t)unit * RW;
-  const unsigned long long* key = p.key + (int64_t)unit * ML;
-  const int32_t* list = list_of(p, unit, idx);
-  unsigned long long best = key[u];               // the token itself belongs to its closed neighbourhood
+__device__ __forceinline__ void best_of_row(const CodebookParams& p, const CoverState& st, const uint32_t* lv, int64_t row0, int u) {
+  const int ec = p.ell_cnt[row0 + u];
+  if (ec < 0) return;
+  const int32_t* list = p.lists + p.lbase[row0 + u];
+  uint32_t best = st.key[u];                      // the token itself belongs to its closed neighbourhood
   for (int k0 = 0; k0 < ec; k0 += kBatch) {
     int v[kBatch];
     load_batch(list, k0, ec, v);
     if (!kAllLive) keep_live(lv, v);
-    unsigned long long kv[kBatch];
 #pragma unroll
-    for (int i = 0; i < kBatch; ++i) kv[i] = v[i] >= 0 ? key[v[i]] : 0ull;
-#pragma unroll
-    for (int i = 0; i < kBatch; ++i) best = kv[i] > best ? kv[i] : best;
+    for (int i = 0; i < kBatch; ++i) best = max(best, v[i] >= 0 ? st.key[v[i]] : 0u);
   }
-  p.m1[idx] = best;
+  st.best[u] = (uint16_t)key_token(best);
 }
 
-// Phase 2 for one dense row, a warp on its bit row.
-__device__ __forceinline__ void max_of_dense_row(const CodebookParams& p, const uint32_t* live, int64_t idx, int lane) {
-  const int ML = p.batch.max_len, RW = p.row_words;
-  const int unit = (int)(idx / ML), u = (int)(idx - (int64_t)unit * ML);
-  const uint32_t* lv = live + (int64_t)unit * RW;
-  if (!is_live(lv, u)) return;
-  const unsigned long long* key = p.key + (int64_t)unit * ML;
-  const uint32_t* row = p.adj + idx * RW;
-  const uint32_t* fr = flag_row(p, unit, u);
-  unsigned long long best = 0ull;
-  for (int w = lane; w < RW; w += 32) {
-    uint32_t m = chunk_flagged(fr, w >> 1, u) ? row[w] & lv[w] : 0u;
-    while (m) {
-      int b = __ffs(m) - 1;
-      m &= m - 1;
-      unsigned long long kv = key[w * 32 + b];
-      best = kv > best ? kv : best;
-    }
-  }
-  best = warp_max_u64(best);
-  if (lane == 0) p.m1[idx] = best;
-}
-
-// Phase 3 for the 32 rows of live-mask word w: a node that is the maximum of every neighbour's
-// neighbourhood is a centre (Eq. (11)); its live neighbours take it as owner (Eq. (12)) and leave the
-// graph (Eq. (13)).
+// phase 3: a token that is the maximum of every live neighbour's neighbourhood is a centre (Eq. (11)); its live
+// neighbours take it as owner (Eq. (12)) and leave the graph (Eq. (13))
 template <bool kAllLive>
-__device__ __forceinline__ void pick_listed_rows(const CodebookParams& p, const uint32_t* live, uint32_t* next, int64_t w,
-                                                 int lane) {
-  const int ML = p.batch.max_len, RW = p.row_words;
-  const uint32_t lvw = live[w];
-  if (!((lvw >> lane) & 1u)) return;
-  const int unit = (int)(w / RW), u = (int)(w - (int64_t)unit * RW) * 32 + lane;
-  const int64_t idx = (int64_t)unit * ML + u;
-  const int ec = p.ell_cnt[idx];
+__device__ __forceinline__ void pick_row(const CodebookParams& p, const CoverState& st, const uint32_t* lv, uint32_t* nx, int64_t row0,
+                                         int u) {
+  const int ec = p.ell_cnt[row0 + u];
   if (ec < 0) return;
-  const unsigned long long mykey = p.key[idx];
-  if (p.m1[idx] != mykey) return;
-  const uint32_t* lv = live + (int64_t)unit * RW;
-  const unsigned long long* m1 = p.m1 + (int64_t)unit * ML;
-  const int32_t* list = list_of(p, unit, idx);
+  if (st.best[u] != (uint16_t)u) return;
+  const int32_t* list = p.lists + p.lbase[row0 + u];
   bool ok = true;
   for (int k0 = 0; k0 < ec && ok; k0 += kBatch) {
     int v[kBatch];
     load_batch(list, k0, ec, v);
     if (!kAllLive) keep_live(lv, v);
-    unsigned long long mv[kBatch];
 #pragma unroll
-    for (int i = 0; i < kBatch; ++i) mv[i] = v[i] >= 0 ? m1[v[i]] : mykey;
-#pragma unroll
-    for (int i = 0; i < kBatch; ++i) ok = ok && mv[i] == mykey;
+    for (int i = 0; i < kBatch; ++i) ok = ok && (v[i] < 0 || st.best[v[i]] == (uint16_t)u);
   }
   if (!ok) return;
-  int32_t* owner = p.owner + (int64_t)unit * ML;
-  uint32_t* nx = next + (int64_t)unit * RW;
+  int32_t* owner = p.owner + row0;
   for (int k0 = 0; k0 < ec; k0 += kBatch) {
     int v[kBatch];
     load_batch(list, k0, ec, v);
@@ -584,247 +547,181 @@ __device__ __forceinline__ void pick_listed_rows(const CodebookParams& p, const 
         atomicAnd(&nx[v[i] >> 5], ~(1u << (v[i] & 31)));
       }
   }
-  p.pickdeg[idx] = p.deg[idx];
+  p.pickdeg[row0 + u] = (int)(st.key[u] >> 16);
   owner[u] = u;
   atomicAnd(&nx[u >> 5], ~(1u << (u & 31)));
 }
 
-// Phase 3 for one dense row.
-__device__ __forceinline__ void pick_dense_row(const CodebookParams& p, const uint32_t* live, uint32_t* next, int64_t idx,
-                                               int lane) {
-  const int ML = p.batch.max_len, RW = p.row_words;
-  const int unit = (int)(idx / ML), u = (int)(idx - (int64_t)unit * ML);
-  const uint32_t* lv = live + (int64_t)unit * RW;
-  if (!is_live(lv, u)) return;
-  const unsigned long long mykey = p.key[idx];
-  if (p.m1[idx] != mykey) return;
-  const unsigned long long* m1 = p.m1 + (int64_t)unit * ML;
-  int32_t* owner = p.owner + (int64_t)unit * ML;
-  uint32_t* nx = next + (int64_t)unit * RW;
-  const uint32_t* row = p.adj + idx * RW;
-  const uint32_t* fr = flag_row(p, unit, u);
-  bool ok = true;
-  for (int w = lane; w < RW; w += 32) {
-    uint32_t m = chunk_flagged(fr, w >> 1, u) ? row[w] & lv[w] : 0u;
-    while (m) {
-      int b = __ffs(m) - 1;
-      m &= m - 1;
-      if (m1[w * 32 + b] != mykey) ok = false;
+// ---- rows with more than kEll neighbours, one warp per row: the neighbours come from the row's list (record
+// path, ell_cnt = -1 - n) or from its bit row masked by the occupancy flags (bit-matrix path, ell_cnt = -1) ----
+template <typename F>
+__device__ __forceinline__ void for_each_live_neighbour(const CodebookParams& p, const uint32_t* lv, int unit, int64_t row0, int u,
+                                                        int lane, F f) {
+  const int ec = p.ell_cnt[row0 + u];
+  if (ec == -1) {
+    const int RW = p.row_words;
+    const uint32_t* row = p.adj + (row0 + u) * RW;
+    const uint32_t* fr = flag_row(p, unit, u);
+    for (int w = lane; w < RW; w += 32) {
+      uint32_t m = chunk_flagged(fr, w >> 1, u) ? row[w] & lv[w] : 0u;
+      while (m) {
+        const int b = __ffs(m) - 1;
+        m &= m - 1;
+        if (w * 32 + b != u) f(w * 32 + b);
+      }
     }
-  }
-  if (!__all_sync(0xffffffffu, ok)) return;
-  if (lane == 0) p.pickdeg[idx] = p.deg[idx];
-  for (int w = lane; w < RW; w += 32) {
-    uint32_t m = chunk_flagged(fr, w >> 1, u) ? row[w] & lv[w] : 0u;
-    if (m) atomicAnd(&nx[w], ~m);
-    while (m) {
-      int b = __ffs(m) - 1;
-      m &= m - 1;
-      owner[w * 32 + b] = u;
+  } else {
+    const int n = -1 - ec;
+    const int32_t* list = p.lists + p.lbase[row0 + u];
+    for (int k = lane; k < n; k += 32) {
+      const int v = list[k];
+      if (is_live(lv, v)) f(v);
     }
   }
 }
 
-// The same three steps for a row whose `n` neighbours (more than kEll) are listed (record path): a warp walks
-// the list, 32 entries at a time.
-
-__device__ __forceinline__ void degree_of_long_row(const CodebookParams& p, const uint32_t* live, int64_t idx, int n, int lane) {
-  const int ML = p.batch.max_len, RW = p.row_words;
-  const int unit = (int)(idx / ML), u = (int)(idx - (int64_t)unit * ML);
-  const uint32_t* lv = live + (int64_t)unit * RW;
+__device__ __forceinline__ void degree_of_big_row(const CodebookParams& p, const CoverState& st, const uint32_t* lv, int unit,
+                                                  int64_t row0, int u, int lane) {
   if (!is_live(lv, u)) return;
-  const int32_t* list = list_of(p, unit, idx);
   int cnt = 0;
-  for (int k = lane; k < n; k += 32) cnt += is_live(lv, list[k]) ? 1 : 0;
+  for_each_live_neighbour(p, lv, unit, row0, u, lane, [&](int) { ++cnt; });
 #pragma unroll
   for (int o = 16; o >= 1; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
-  if (lane == 0) {
-    p.deg[idx] = cnt + 1;
-    p.key[idx] = ((unsigned long long)(uint32_t)(cnt + 1) << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)u);
-  }
+  if (lane == 0) st.key[u] = make_key(cnt + 1, u);
 }
 
-__device__ __forceinline__ void max_of_long_row(const CodebookParams& p, const uint32_t* live, int64_t idx, int n, int lane) {
-  const int ML = p.batch.max_len, RW = p.row_words;
-  const int unit = (int)(idx / ML), u = (int)(idx - (int64_t)unit * ML);
-  const uint32_t* lv = live + (int64_t)unit * RW;
+__device__ __forceinline__ void best_of_big_row(const CodebookParams& p, const CoverState& st, const uint32_t* lv, int unit,
+                                                int64_t row0, int u, int lane) {
   if (!is_live(lv, u)) return;
-  const unsigned long long* key = p.key + (int64_t)unit * ML;
-  const int32_t* list = list_of(p, unit, idx);
-  unsigned long long best = lane == 0 ? key[u] : 0ull;   // the token itself belongs to its closed neighbourhood
-  for (int k = lane; k < n; k += 32) {
-    const int v = list[k];
-    if (is_live(lv, v)) {
-      const unsigned long long kv = key[v];
-      best = kv > best ? kv : best;
-    }
-  }
-  best = warp_max_u64(best);
-  if (lane == 0) p.m1[idx] = best;
+  uint32_t best = lane == 0 ? st.key[u] : 0u;
+  for_each_live_neighbour(p, lv, unit, row0, u, lane, [&](int v) { best = max(best, st.key[v]); });
+#pragma unroll
+  for (int o = 16; o >= 1; o >>= 1) best = max(best, __shfl_xor_sync(0xffffffffu, best, o));
+  if (lane == 0) st.best[u] = (uint16_t)key_token(best);
 }
 
-__device__ __forceinline__ void pick_long_row(const CodebookParams& p, const uint32_t* live, uint32_t* next, int64_t idx, int n,
-                                              int lane) {
-  const int ML = p.batch.max_len, RW = p.row_words;
-  const int unit = (int)(idx / ML), u = (int)(idx - (int64_t)unit * ML);
-  const uint32_t* lv = live + (int64_t)unit * RW;
+__device__ __forceinline__ void pick_big_row(const CodebookParams& p, const CoverState& st, const uint32_t* lv, uint32_t* nx, int unit,
+                                             int64_t row0, int u, int lane) {
   if (!is_live(lv, u)) return;
-  const unsigned long long mykey = p.key[idx];
-  if (p.m1[idx] != mykey) return;
-  const unsigned long long* m1 = p.m1 + (int64_t)unit * ML;
-  int32_t* owner = p.owner + (int64_t)unit * ML;
-  uint32_t* nx = next + (int64_t)unit * RW;
-  const int32_t* list = list_of(p, unit, idx);
+  if (st.best[u] != (uint16_t)u) return;
   bool ok = true;
-  for (int k = lane; k < n; k += 32) {
-    const int v = list[k];
-    if (is_live(lv, v) && m1[v] != mykey) ok = false;
-  }
+  for_each_live_neighbour(p, lv, unit, row0, u, lane, [&](int v) { ok = ok && st.best[v] == (uint16_t)u; });
   if (!__all_sync(0xffffffffu, ok)) return;
-  for (int k = lane; k < n; k += 32) {
-    const int v = list[k];
-    if (is_live(lv, v)) {
-      owner[v] = u;
-      atomicAnd(&nx[v >> 5], ~(1u << (v & 31)));
-    }
-  }
+  int32_t* owner = p.owner + row0;
+  for_each_live_neighbour(p, lv, unit, row0, u, lane, [&](int v) {
+    owner[v] = u;
+    atomicAnd(&nx[v >> 5], ~(1u << (v & 31)));
+  });
   if (lane == 0) {
-    p.pickdeg[idx] = p.deg[idx];
+    p.pickdeg[row0 + u] = (int)(st.key[u] >> 16);
     owner[u] = u;
     atomicAnd(&nx[u >> 5], ~(1u << (u & 31)));
   }
 }
 
-// A row with more than kEll neighbours: its bit row (ell_cnt == -1) or its list (ell_cnt == -1 - n).
-__device__ __forceinline__ void max_of_big_row(const CodebookParams& p, const uint32_t* live, int64_t idx, int lane) {
-  const int ec = p.ell_cnt[idx];
-  if (ec == -1) max_of_dense_row(p, live, idx, lane);
-  else max_of_long_row(p, live, idx, -1 - ec, lane);
-}
-__device__ __forceinline__ void pick_big_row(const CodebookParams& p, const uint32_t* live, uint32_t* next, int64_t idx, int lane) {
-  const int ec = p.ell_cnt[idx];
-  if (ec == -1) pick_dense_row(p, live, next, idx, lane);
-  else pick_long_row(p, live, next, idx, -1 - ec, lane);
-}
-
-// Phase 1 for the 32 rows of live-mask word w: live degrees (Eq. (10)) and keys of the rows with a list.
-__device__ __forceinline__ void degrees_of_listed_rows(const CodebookParams& p, const uint32_t* live, int64_t w, uint32_t lvw,
-                                                       int lane) {
-  if (!((lvw >> lane) & 1u)) return;
-  const int ML = p.batch.max_len, RW = p.row_words;
-  const int unit = (int)(w / RW), u = (int)(w - (int64_t)unit * RW) * 32 + lane;
-  const int64_t idx = (int64_t)unit * ML + u;
-  const int ec = p.ell_cnt[idx];
-  if (ec < 0) return;                             // rows with many neighbours: separately
-  const uint32_t* lv = live + (int64_t)unit * RW;
-  const int32_t* list = list_of(p, unit, idx);
-  int cnt = 1;
-  for (int k0 = 0; k0 < ec; k0 += kBatch) {
-    int v[kBatch];
-    load_batch(list, k0, ec, v);
-    keep_live(lv, v);
-#pragma unroll
-    for (int i = 0; i < kBatch; ++i) cnt += v[i] >= 0 ? 1 : 0;
-  }
-  p.deg[idx] = cnt;
-  p.key[idx] = ((unsigned long long)(uint32_t)cnt << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)u);
-}
-
-// Phase 1 for one row that uses its bit row.
-__device__ __forceinline__ void degree_of_dense_row(const CodebookParams& p, const uint32_t* live, int64_t idx, int lane) {
-  const int ML = p.batch.max_len, RW = p.row_words, RW4 = RW >> 2;
-  const int unit = (int)(idx / ML), u = (int)(idx - (int64_t)unit * ML);
-  const uint32_t* lv = live + (int64_t)unit * RW;
-  if (!is_live(lv, u)) return;
-  const uint4* row4 = reinterpret_cast<const uint4*>(p.adj + idx * RW);
-  const uint4* lv4 = reinterpret_cast<const uint4*>(lv);
-  const uint32_t* fr = flag_row(p, unit, u);
-  int cnt = 0;
-  for (int w4 = lane; w4 < RW4; w4 += 32) {
-    const uint4 a = row4[w4], b = lv4[w4];
-    if (chunk_flagged(fr, 2 * w4, u)) cnt += __popc(a.x & b.x) + __popc(a.y & b.y);
-    if (chunk_flagged(fr, 2 * w4 + 1, u)) cnt += __popc(a.z & b.z) + __popc(a.w & b.w);
-  }
-#pragma unroll
-  for (int o = 16; o >= 1; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
-  if (lane == 0) {
-    p.deg[idx] = cnt;
-    p.key[idx] = ((unsigned long long)(uint32_t)cnt << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)u);
-  }
-}
-
-// The greedy cover of one unit, all rounds, by one block: units are independent graphs, so the three phases of a
-// round are separated by block barriers only, and a unit stops as soon as it has no live token left, whatever the
-// other units still do.  Round 0 finds every token with a neighbour live and its degree known from the list
-// building; later rounds first recount the degrees of the tokens that are left.  A warp takes the 32 rows of one
-// word of the unit's live mask (empty words cost one load); rows with more than kEll neighbours come from the
-// unit's own list of such rows, a warp per row.
 constexpr int kCoverThreads = 1024;
 
 __global__ void __launch_bounds__(kCoverThreads) cover_kernel(CodebookParams p) {
-  __shared__ int live_total;
+  extern __shared__ uint32_t cover_sm[];
+  __shared__ int n_left;
   const int unit = blockIdx.x;
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   constexpr int NW = kCoverThreads / 32;
-  const int ML = p.batch.max_len, RW = p.row_words;
-  const int64_t w0 = (int64_t)unit * RW;
-  const int32_t* big = p.dense_rows + (int64_t)unit * ML;
+  const int ML = p.batch.max_len, RW = p.row_words, NP = RW * 32;
+  const int64_t row0 = (int64_t)unit * ML;
+  CoverState st;
+  st.key = cover_sm;
+  st.live0 = st.key + NP;
+  st.live1 = st.live0 + RW;
+  st.best = reinterpret_cast<uint16_t*>(st.live1 + RW);
+  st.left = st.best + NP;
+  {
+    int layer, s, j;
+    cb_decode(p, unit, layer, s, j);
+    const int l = seq_len(p.batch, layer, s, j);
+    for (int u = tid; u < NP; u += kCoverThreads) st.key[u] = make_key(u < l ? p.deg[row0 + u] : 0, u);
+    for (int w = tid; w < RW; w += kCoverThreads) st.live0[w] = st.live1[w] = p.live0[(int64_t)unit * RW + w];
+  }
+  // the lists of this unit are addressed from the unit's part of the list buffer
+  p.lists += (int64_t)unit * p.list_cap;
+  const int32_t* big = p.dense_rows + row0;
   const int n_big = p.dense_cnt[unit];
   const int round_cap = min(ML, p.round_cap);
+  __syncthreads();
   int round = 0;
   bool gave_up = false;
   for (;; ++round) {
-    uint32_t* live = (round & 1) ? p.live1 : p.live0;
-    uint32_t* next = (round & 1) ? p.live0 : p.live1;
+    const uint32_t* lv = (round & 1) ? st.live1 : st.live0;
+    uint32_t* nx = (round & 1) ? st.live0 : st.live1;
+    bool listed = false;                 // the live tokens of this round are in st.left
     if (round > 0) {
       if (round > round_cap) { gave_up = true; break; }
-      // phase 1: live degrees and keys; `next` becomes a copy of `live`
-      if (tid == 0) live_total = 0;
+      // phase 1: `next` becomes a copy of `live`; the tokens that are left, their number, their live degrees
+      if (tid == 0) n_left = 0;
       __syncthreads();
-      int my_live = 0;
       for (int w = wid; w < RW; w += NW) {
-        const uint32_t lvw = live[w0 + w];
-        if (lane == 0) next[w0 + w] = lvw;
+        const uint32_t lvw = lv[w];
+        if (lane == 0) nx[w] = lvw;
         if (!lvw) continue;
-        my_live += __popc(lvw);
-        degrees_of_listed_rows(p, live, w0 + w, lvw, lane);
+        int at = 0;
+        if (lane == 0) at = atomicAdd(&n_left, __popc(lvw));
+        at = __shfl_sync(0xffffffffu, at, 0) + __popc(lvw & ((1u << lane) - 1u));
+        if (((lvw >> lane) & 1u) && at < kLeftCap) st.left[at] = (uint16_t)(w * 32 + lane);
       }
-      for (int d = wid; d < n_big; d += NW) {
-        const int64_t idx = (int64_t)unit * ML + big[d];
-        const int ec = p.ell_cnt[idx];
-        if (ec == -1) degree_of_dense_row(p, live, idx, lane);
-        else degree_of_long_row(p, live, idx, -1 - ec, lane);
-      }
-      if (lane == 0 && my_live) atomicAdd(&live_total, my_live);
       __syncthreads();
-      if (live_total == 0) break;
+      const int nl = n_left;
+      if (nl == 0) break;
+      listed = nl <= kLeftCap;
+      if (listed) {
+        for (int i = tid; i < nl; i += kCoverThreads) degree_of_row(p, st, lv, row0, st.left[i]);
+      } else {
+        for (int w = wid; w < RW; w += NW)
+          if ((lv[w] >> lane) & 1u) degree_of_row(p, st, lv, row0, w * 32 + lane);
+      }
+      for (int d = wid; d < n_big; d += NW) degree_of_big_row(p, st, lv, unit, row0, big[d], lane);
+      __syncthreads();
     }
     // phase 2: largest key in each closed live neighbourhood
-    for (int w = wid; w < RW; w += NW) {
-      if (round == 0) max_of_listed_rows<true>(p, live, w0 + w, lane);
-      else max_of_listed_rows<false>(p, live, w0 + w, lane);
+    if (round == 0) {
+      for (int w = wid; w < RW; w += NW)
+        if ((lv[w] >> lane) & 1u) best_of_row<true>(p, st, lv, row0, w * 32 + lane);
+    } else if (listed) {
+      for (int i = tid; i < n_left; i += kCoverThreads) best_of_row<false>(p, st, lv, row0, st.left[i]);
+    } else {
+      for (int w = wid; w < RW; w += NW)
+        if ((lv[w] >> lane) & 1u) best_of_row<false>(p, st, lv, row0, w * 32 + lane);
     }
-    for (int d = wid; d < n_big; d += NW) max_of_big_row(p, live, (int64_t)unit * ML + big[d], lane);
+    for (int d = wid; d < n_big; d += NW) best_of_big_row(p, st, lv, unit, row0, big[d], lane);
     __syncthreads();
-    // phase 3: picks (Eq. (11)-(13))
-    for (int w = wid; w < RW; w += NW) {
-      if (round == 0) pick_listed_rows<true>(p, live, next, w0 + w, lane);
-      else pick_listed_rows<false>(p, live, next, w0 + w, lane);
+    // phase 3: picks
+    if (round == 0) {
+      for (int w = wid; w < RW; w += NW)
+        if ((lv[w] >> lane) & 1u) pick_row<true>(p, st, lv, nx, row0, w * 32 + lane);
+    } else if (listed) {
+      for (int i = tid; i < n_left; i += kCoverThreads) pick_row<false>(p, st, lv, nx, row0, st.left[i]);
+    } else {
+      for (int w = wid; w < RW; w += NW)
+        if ((lv[w] >> lane) & 1u) pick_row<false>(p, st, lv, nx, row0, w * 32 + lane);
     }
-    for (int d = wid; d < n_big; d += NW) pick_big_row(p, live, next, (int64_t)unit * ML + big[d], lane);
+    for (int d = wid; d < n_big; d += NW) pick_big_row(p, st, lv, nx, unit, row0, big[d], lane);
     __syncthreads();
   }
   if (tid == 0) {
     atomicMax(&p.hdr[kHdrRounds], (uint32_t)round);
     if (gave_up) {
       // the round that was not run: its live tokens are the ones left without a centre
-      const uint32_t* live = (round & 1) ? p.live1 : p.live0;
+      const uint32_t* lv = (round & 1) ? st.live1 : st.live0;
       uint32_t left = 0;
-      for (int w = 0; w < RW; ++w) left += __popc(live[w0 + w]);
+      for (int w = 0; w < RW; ++w) left += __popc(lv[w]);
       atomicAdd(&p.hdr[kHdrLive], max(left, 1u));
       atomicExch(&p.hdr[kHdrStatus], (uint32_t)SPINDLEKV_TIMEOUT);
     }
   }
+}
+
+static size_t cover_smem_bytes(int row_words) {
+  const size_t NP = (size_t)row_words * 32;
+  return NP * 4 + 2 * (size_t)row_words * 4 + NP * 2 + kLeftCap * 2;
 }
 
 // ---- entry numbering ------------------------------------------------------------------------------
@@ -1014,7 +911,7 @@ __global__ void __launch_bounds__(kFinalThreads) finalize_kernel(CodebookParams 
 // ---- host side ----------------------------------------------------------------------------------
 
 struct CodebookLayout {
-  size_t ext, ell, ell_cnt, dense_rows, flags, adj, deg, key, m1, live0, live1, owner, pickdeg, rank, total;
+  size_t ext, ell, ell_cnt, dense_rows, flags, adj, deg, live0, owner, pickdeg, rank, total;
   size_t ovf, rec_cnt, dense_cnt, lbase, rec;   // candidate records (tensor-core path)
   int rec_per_tile, n_blocks, list_cap;
 };
@@ -1032,10 +929,7 @@ static CodebookLayout codebook_layout(const spindlekv_config& cfg, const spindle
   size_t off = kHeaderBytes;
   auto take = [&](size_t bytes) { size_t o = off; off += align_up(bytes, 256); return o; };
   L.deg = take(units * ML * 4);
-  L.key = take(units * ML * 8);
-  L.m1 = take(units * ML * 8);
   L.live0 = take(units * RW * 4);
-  L.live1 = take(units * RW * 4);
   L.owner = take(units * ML * 4);
   L.pickdeg = take(units * ML * 4);
   L.rank = take(units * ML * 4);
@@ -1092,7 +986,7 @@ spindlekv_status codebook_shallow_impl(const spindlekv_config& cfg, const spindl
   const bool tc = bf && sim_tc_available();   // bf16: tensor-core similarity (TMA + tcgen05)
   CodebookLayout L = codebook_layout(cfg, b, adj_in_ws, tc ? min(tune.rec_per_tile, kDefaultRecPerTile) : 0);
   if (ws_bytes < L.total) return SPINDLEKV_WORKSPACE_TOO_SMALL;
-  if ((size_t)(b.max_len + 2) * 4 > 200 * 1024) return SPINDLEKV_UNSUPPORTED;
+  if (row_words_for(b.max_len) * 32 > kCoverMaxTokens) return SPINDLEKV_UNSUPPORTED;   // the cover keeps a unit's state on chip
   const int units = b.n_layers * b.n_seqs * cfg.n_kv_heads;
   if (units > 65535) return SPINDLEKV_UNSUPPORTED;
   const bool records = L.rec_per_tile > 0;    // candidate records first, the bit matrix for units that overflow
@@ -1107,10 +1001,7 @@ spindlekv_status codebook_shallow_impl(const spindlekv_config& cfg, const spindl
   p.mag = mag;
   p.adj = adj_in_ws ? reinterpret_cast<uint32_t*>(w + L.adj) : adj_bits;
   p.deg = reinterpret_cast<int32_t*>(w + L.deg);
-  p.key = reinterpret_cast<unsigned long long*>(w + L.key);
-  p.m1 = reinterpret_cast<unsigned long long*>(w + L.m1);
   p.live0 = reinterpret_cast<uint32_t*>(w + L.live0);
-  p.live1 = reinterpret_cast<uint32_t*>(w + L.live1);
   p.owner = reinterpret_cast<int32_t*>(w + L.owner);
   p.pickdeg = reinterpret_cast<int32_t*>(w + L.pickdeg);
   p.rank = reinterpret_cast<int32_t*>(w + L.rank);
@@ -1191,8 +1082,14 @@ spindlekv_status codebook_shallow_impl(const spindlekv_config& cfg, const spindl
   const int dev = PerDeviceOnce::current();
   if (dev < 0) return SPINDLEKV_CUDA;
   {
+    static PerDeviceOnce once;
+    if (!once.done[dev]) {
+      if (cudaFuncSetAttribute(cover_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)cover_smem_bytes(kCoverMaxTokens / 32)) != cudaSuccess)
+        return SPINDLEKV_CUDA;
+      once.done[dev] = true;
+    }
     LaunchScope ls(KC_GREEDY, st);
-    cover_kernel<<<units, kCoverThreads, 0, st>>>(p);
+    cover_kernel<<<units, kCoverThreads, cover_smem_bytes(p.row_words), st>>>(p);
   }
   {
     size_t smem = (size_t)(b.max_len + 2) * 4;
