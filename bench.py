@@ -503,12 +503,13 @@ def run_native(args, wl):
     if ns and graph:
         # Graph stage, bytes that must move at least once per step (K and V calls together).  List building: the
         # candidate records (8 bytes per similar pair, read), the lists (4 bytes per entry, written), and per token
-        # degree, key, list start and length, pick degree and live bit (24 bytes, written).  Greedy cover: every list
-        # entry read with the 8-byte key or neighbourhood maximum it points to, per-token key, maximum, owner and
-        # pick degree (24 bytes).  Numbering: pick degree, owner, rank, reference and centre position per token (20).
+        # degree, list start and length, pick degree and live bit (16 bytes, written).  Greedy cover (keys and
+        # neighbourhood maxima live in shared memory): every list entry read once, per-token degree, list start and
+        # length read, owner and pick degree written (20 bytes).  Numbering: pick degree, owner, rank, reference and
+        # centre position per token (20 bytes).
         rows = 2 * ns * Hk * tok
         ent = sum(v["list_entries"] for v in graph.values())
-        for name, nbytes in (("degree", ent // 2 * 8 + ent * 4 + rows * 24), ("greedy", ent * 12 + rows * 24),
+        for name, nbytes in (("degree", ent // 2 * 8 + ent * 4 + rows * 16), ("greedy", ent * 4 + rows * 20),
                              ("finalise", rows * 20)):
             if name in kernels and kernels[name]["ms_per_step"] > 0:
                 gbs = nbytes / (kernels[name]["ms_per_step"] * 1e-3) / 1e9

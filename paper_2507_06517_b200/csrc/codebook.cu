@@ -403,6 +403,21 @@ __global__ void __launch_bounds__(kBuildThreads) build_lists_kernel(CodebookPara
   });
 }
 
+// The units whose overflow flag is set, in ascending order, for the bit-matrix pass of the similarity kernel.
+__global__ void __launch_bounds__(1024) list_overflowed_kernel(const int32_t* ovf, int n_units, int32_t* work_list, int32_t* n_work) {
+  __shared__ int warp_sums[33];
+  int base = 0;
+  for (int u0 = 0; u0 < n_units; u0 += 1024) {
+    const int u = u0 + threadIdx.x;
+    const int flag = (u < n_units && ovf[u]) ? 1 : 0;
+    int total;
+    const int at = block_exclusive_scan(flag, warp_sums, total);
+    if (flag) work_list[base + at] = u;
+    base += total;
+  }
+  if (threadIdx.x == 0) *n_work = base;
+}
+
 // Flag words of the units that go through the bit matrix start at zero (the similarity kernel writes only
 // the words that hold a set bit).
 __global__ void __launch_bounds__(256) clear_flags_kernel(CodebookParams p) {
@@ -912,7 +927,7 @@ __global__ void __launch_bounds__(kFinalThreads) finalize_kernel(CodebookParams 
 
 struct CodebookLayout {
   size_t ext, ell, ell_cnt, dense_rows, flags, adj, deg, live0, owner, pickdeg, rank, total;
-  size_t ovf, rec_cnt, dense_cnt, lbase, rec;   // candidate records (tensor-core path)
+  size_t ovf, rec_cnt, dense_cnt, work_list, lbase, rec;   // candidate records (tensor-core path)
   int rec_per_tile, n_blocks, list_cap;
 };
 
@@ -945,6 +960,7 @@ static CodebookLayout codebook_layout(const spindlekv_config& cfg, const spindle
   L.ovf = take(units * 4);
   L.rec_cnt = take(units * L.n_blocks * 4);
   L.dense_cnt = take(units * 4);
+  L.work_list = take((units + 1) * 4);
   L.lbase = take(units * ML * 4);
   L.rec = take(L.rec_per_tile ? units * (size_t)rec_unit_capacity(L.n_blocks / 2, L.rec_per_tile) * 8 : 0);
   L.adj = off;
@@ -1027,7 +1043,7 @@ spindlekv_status codebook_shallow_impl(const spindlekv_config& cfg, const spindl
   // overflow flags and record counts: all zero on the record path; without records every unit counts as overflowed;
   // the per-unit counts of rows with many neighbours start at zero
   if (cudaMemsetAsync(w + L.ovf, records ? 0 : 1, L.dense_cnt - L.ovf, st) != cudaSuccess) return SPINDLEKV_CUDA;
-  if (cudaMemsetAsync(w + L.dense_cnt, 0, L.lbase - L.dense_cnt, st) != cudaSuccess) return SPINDLEKV_CUDA;
+  if (cudaMemsetAsync(w + L.dense_cnt, 0, L.work_list - L.dense_cnt, st) != cudaSuccess) return SPINDLEKV_CUDA;
   p.ext = tc ? reinterpret_cast<__nv_bfloat16*>(w + L.ext) : nullptr;
   if (cfg.head_dim == 64) {
     if (bf) launch_norms<__nv_bfloat16, 64>(p, st); else launch_norms<float, 64>(p, st);
@@ -1036,7 +1052,8 @@ spindlekv_status codebook_shallow_impl(const spindlekv_config& cfg, const spindl
   }
   const size_t flag_words = (size_t)(p.row_words / 2) * p.row_words;
   if (tc) {
-    SimRecordPool pool{reinterpret_cast<uint2*>(w + L.rec), reinterpret_cast<int32_t*>(w + L.rec_cnt), p.ovf, L.rec_per_tile};
+    SimRecordPool pool{reinterpret_cast<uint2*>(w + L.rec), reinterpret_cast<int32_t*>(w + L.rec_cnt), p.ovf, L.rec_per_tile,
+                       reinterpret_cast<int32_t*>(w + L.work_list) + 1, reinterpret_cast<int32_t*>(w + L.work_list)};
     if (records) {
       if (!adj_in_ws &&
           cudaMemsetAsync(adj_bits, 0, (size_t)units * b.max_len * p.row_words * 4, st) != cudaSuccess) return SPINDLEKV_CUDA;
@@ -1055,6 +1072,10 @@ spindlekv_status codebook_shallow_impl(const spindlekv_config& cfg, const spindl
       build_lists_kernel<<<units, kBuildThreads, (size_t)p.row_words * 32 * 4, st>>>(p);
     }
     // units without usable records (all of them when the record path is off): bit matrix, occupancy flags, extraction
+    if (records) {
+      LaunchScope ls(KC_DEGREE, st);
+      list_overflowed_kernel<<<1, 1024, 0, st>>>(p.ovf, units, pool.work_list, pool.n_work);
+    }
     {
       LaunchScope ls(KC_DEGREE, st);
       clear_flags_kernel<<<dim3((unsigned)std::min<size_t>((flag_words + 255) / 256, 64), units), 256, 0, st>>>(p);

@@ -100,7 +100,10 @@ struct SimRecordPool {   // device buffers of the candidate records of one CodeB
   int32_t* rec_cnt;      // [units][row blocks]
   int32_t* ovf;          // [units]
   int rec_per_tile;
+  int32_t* work_list;    // [units] the units whose overflow flag is set, ascending (written before the bit-matrix pass)
+  int32_t* n_work;       // [1] how many
 };
+constexpr int kFallbackSlots = 16;   // pairs of blocks per row span that the bit-matrix pass behind a record pool launches
 
 // 32x32 bit transpose across a warp: in: lane r holds bits (r, c) at bit c; out: lane c holds bit r.
 // Five butterfly stages (j = 16, 8, 4, 2, 1): a lane takes from its partner the half of every 2j-bit

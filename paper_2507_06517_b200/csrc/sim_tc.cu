@@ -44,6 +44,8 @@
 // again as a bit matrix by the other instantiation of this kernel (which returns at once for all other
 // units).  The order of the records inside a region depends on warp timing; everything derived from them
 // is independent of that order.
+#include <algorithm>
+
 #include "common.cuh"
 #include "sm100_ptx.cuh"
 
@@ -63,6 +65,11 @@ struct SimTcParams {
   int rec_per_tile;    // a block's region holds rec_per_tile records per tile it computes
   long long unit_rec_cap;
   long long wait_cycles;   // bound of every mbarrier wait, in SM clock cycles
+  // bit-matrix instantiation behind a record pool: the units to compute (those that overflowed), in ascending
+  // order, and their number; a pair of blocks with blockIdx.y = k takes the units work_list[k], work_list[k +
+  // gridDim.y], ...  Null: blockIdx.y is the unit.
+  const int32_t* work_list;
+  const int32_t* n_work;
 };
 
 constexpr int kBM = 128;          // rows of the resident block (UMMA M)
@@ -176,18 +183,28 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kSimThreads, 1) sim_
                                                                 const __grid_constant__ CUtensorMap emap,
                                                                 SimTcParams p) {
   using L = SimSmem<D>;
-  const int unit = blockIdx.y;
-  if (!kEmit && p.ovf && !p.ovf[unit]) return;   // both CTAs of a pair: the unit's records were enough
-  const int j = unit % p.n_kv_heads;
-  const int ls = unit / p.n_kv_heads;
-  const int s = ls % p.batch.n_seqs;
-  const int layer = ls / p.batch.n_seqs;
-  const int l = seq_len(p.batch, layer, s, j);
+  const int n_work = p.work_list ? *p.n_work : (int)gridDim.y;
+  if ((int)blockIdx.y >= n_work) return;     // both CTAs of a pair: nothing to compute
   const int row0 = blockIdx.x * kBM;
   const int rank = (int)cluster_ctarank();   // = blockIdx.x & 1
-  if ((row0 & ~(kBN - 1)) >= l) return;      // both CTAs of a pair: the whole 256-row span lies beyond the sequence
-  const int n_tiles = (l + kBN - 1) / kBN;   // tiles of this sequence: columns beyond its end are never produced
   const int tile0 = row0 / kBN;   // the tile that holds the pair's diagonal; earlier tiles are mirrored by other pairs
+  // What a pair has to do for its k-th unit.  Every role of both CTAs walks the same units in the same order and
+  // counts the tiles done so far (`base`) and the units that had any (`ua`): ring stages, accumulator stages and
+  // barrier phases carry on from one unit to the next.
+  struct UnitWork { int unit, j, s, layer, l, n_tiles, nt; };
+  auto unit_work = [&](int k) {
+    UnitWork w;
+    w.unit = p.work_list ? p.work_list[k] : k;
+    w.j = w.unit % p.n_kv_heads;
+    const int ls = w.unit / p.n_kv_heads;
+    w.s = ls % p.batch.n_seqs;
+    w.layer = ls / p.batch.n_seqs;
+    w.l = seq_len(p.batch, w.layer, w.s, w.j);
+    w.n_tiles = (w.l + kBN - 1) / kBN;         // tiles of this sequence: columns beyond its end are never produced
+    // nothing when the whole 256-row span lies beyond the sequence
+    w.nt = (row0 & ~(kBN - 1)) >= w.l ? 0 : w.n_tiles - tile0;
+    return w;
+  };
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -208,11 +225,13 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kSimThreads, 1) sim_
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(acc_empty + 3);
   int* rec_used = reinterpret_cast<int*>(acc_empty + 3) + 1;   // records this block has reserved
+  uint64_t* a_empty = acc_empty + 4;            // both CTAs: the MMAs of a unit have read its resident block
   const long long wait_cycles = p.wait_cycles;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
     ptx::mbar_init(a_full, 1);
+    ptx::mbar_init(a_empty, 1);
     for (int i = 0; i < kStages; ++i) { ptx::mbar_init(b_full + i, 1); ptx::mbar_init(b_empty + i, 1); }
     for (int i = 0; i < 2; ++i) { ptx::mbar_init(acc_full + i, 1); ptx::mbar_init(acc_empty + i, 2 * kTeamWarps); }
     *abort_flag = 0;
@@ -228,26 +247,35 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kSimThreads, 1) sim_
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  const int tok0 = p.batch.cu ? p.batch.cu[s] : 0;
-  const int sdim = p.batch.cu ? 0 : s;
-
   if (warp == 0) {
     if (lane == 0) {
       ptx::prefetch_tensormap(&tmap);
       ptx::prefetch_tensormap(&emap);
-      if (rank == 0) ptx::mbar_expect_tx(a_full, 2 * (L::A_BYTES + L::EA_BYTES));
-      for (int kh = 0; kh < L::KH; ++kh)
-        tma_load_5d_pair(sA + kh * kBM * 128, &tmap, a_full, kh * 64, tok0 + row0, j, sdim, layer);
-      tma_load_4d_pair(sEA, &emap, a_full, 0, row0, unit, 0);
-      for (int it = 0; tile0 + it < n_tiles; ++it) {
-        const int st = it % kStages;
-        if (!ptx::mbar_wait(b_empty + st, ((it / kStages) & 1) ^ 1, abort_flag, wait_cycles)) break;
-        if (rank == 0) ptx::mbar_expect_tx(b_full + st, 2 * (L::B_BYTES + L::EB_BYTES));
-        uint8_t* dst = sB + st * L::B_BYTES;
-        const int brow = (tile0 + it) * kBN + rank * kBH;   // this CTA's half of the tile
+      int base = 0, ua = 0;
+      bool ok = true;
+      for (int k = blockIdx.y; ok && k < n_work; k += gridDim.y) {
+        const UnitWork w = unit_work(k);
+        if (w.nt == 0) continue;
+        const int tok0 = p.batch.cu ? p.batch.cu[w.s] : 0;
+        const int sdim = p.batch.cu ? 0 : w.s;
+        // the resident block of the previous unit must have been read by all of its MMAs
+        if (ua > 0 && !ptx::mbar_wait(a_empty, (ua - 1) & 1, abort_flag, wait_cycles)) break;
+        if (rank == 0) ptx::mbar_expect_tx(a_full, 2 * (L::A_BYTES + L::EA_BYTES));
         for (int kh = 0; kh < L::KH; ++kh)
-          tma_load_5d_pair(dst + kh * kBH * 128, &tmap, b_full + st, kh * 64, tok0 + brow, j, sdim, layer);
-        tma_load_4d_pair(sEB + st * L::EB_BYTES, &emap, b_full + st, 0, brow, unit, 1);
+          tma_load_5d_pair(sA + kh * kBM * 128, &tmap, a_full, kh * 64, tok0 + row0, w.j, sdim, w.layer);
+        tma_load_4d_pair(sEA, &emap, a_full, 0, row0, w.unit, 0);
+        for (int it = 0; it < w.nt; ++it) {
+          const int gi = base + it, st = gi % kStages;
+          if (!ptx::mbar_wait(b_empty + st, ((gi / kStages) & 1) ^ 1, abort_flag, wait_cycles)) { ok = false; break; }
+          if (rank == 0) ptx::mbar_expect_tx(b_full + st, 2 * (L::B_BYTES + L::EB_BYTES));
+          uint8_t* dst = sB + st * L::B_BYTES;
+          const int brow = (tile0 + it) * kBN + rank * kBH;   // this CTA's half of the tile
+          for (int kh = 0; kh < L::KH; ++kh)
+            tma_load_5d_pair(dst + kh * kBH * 128, &tmap, b_full + st, kh * 64, tok0 + brow, w.j, sdim, w.layer);
+          tma_load_4d_pair(sEB + st * L::EB_BYTES, &emap, b_full + st, 0, brow, w.unit, 1);
+        }
+        base += w.nt;
+        ++ua;
       }
     }
   } else if (warp == 1) {
@@ -256,24 +284,33 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kSimThreads, 1) sim_
       constexpr uint32_t idesc_pos = ptx::idesc_bf16_f32(2 * kBM, kBN, false);
       const uint32_t a_addr = ptx::smem_u32(sA);
       const uint64_t dea = ptx::smem_desc_sw32(ptx::smem_u32(sEA));
-      bool ok = ptx::mbar_wait(a_full, 0, abort_flag, wait_cycles);
-      for (int it = 0; ok && tile0 + it < n_tiles; ++it) {
-        const int st = it % kStages, as = it & 1;
-        if (!ptx::mbar_wait(b_full + st, (it / kStages) & 1, abort_flag, wait_cycles)) break;
-        if (!ptx::mbar_wait(acc_empty + as, ((it >> 1) & 1) ^ 1, abort_flag, wait_cycles)) break;
-        ptx::tc_fence_after();
-        const uint32_t b_addr = ptx::smem_u32(sB + st * L::B_BYTES);
+      int base = 0, ua = 0;
+      bool ok = true;
+      for (int k = blockIdx.y; ok && k < n_work; k += gridDim.y) {
+        const UnitWork w = unit_work(k);
+        if (w.nt == 0) continue;
+        ok = ptx::mbar_wait(a_full, ua & 1, abort_flag, wait_cycles);
+        for (int it = 0; ok && it < w.nt; ++it) {
+          const int gi = base + it, st = gi % kStages, as = gi & 1;
+          if (!ptx::mbar_wait(b_full + st, (gi / kStages) & 1, abort_flag, wait_cycles)) { ok = false; break; }
+          if (!ptx::mbar_wait(acc_empty + as, ((gi >> 1) & 1) ^ 1, abort_flag, wait_cycles)) { ok = false; break; }
+          ptx::tc_fence_after();
+          const uint32_t b_addr = ptx::smem_u32(sB + st * L::B_BYTES);
 #pragma unroll
-        for (int k = 0; k < D / 16; ++k) {
-          const int kh = k >> 2, kk = k & 3;
-          uint64_t da = ptx::smem_desc_sw128(a_addr + kh * kBM * 128 + kk * 32);
-          uint64_t db = ptx::smem_desc_sw128(b_addr + kh * kBH * 128 + kk * 32);
-          umma_bf16_pair(tmem_base + as * kBN, da, db, idesc_neg, k > 0 ? 1u : 0u);
+          for (int kk16 = 0; kk16 < D / 16; ++kk16) {
+            const int kh = kk16 >> 2, kk = kk16 & 3;
+            uint64_t da = ptx::smem_desc_sw128(a_addr + kh * kBM * 128 + kk * 32);
+            uint64_t db = ptx::smem_desc_sw128(b_addr + kh * kBH * 128 + kk * 32);
+            umma_bf16_pair(tmem_base + as * kBN, da, db, idesc_neg, kk16 > 0 ? 1u : 0u);
+          }
+          // + theta * |a| * |b|
+          umma_bf16_pair(tmem_base + as * kBN, dea, ptx::smem_desc_sw32(ptx::smem_u32(sEB + st * L::EB_BYTES)), idesc_pos, 1u);
+          umma_commit_pair(b_empty + st);   // both CTAs: the stage may be refilled
+          umma_commit_pair(acc_full + as);  // both CTAs: accumulator ready for the epilogue
         }
-        // + theta * |a| * |b|
-        umma_bf16_pair(tmem_base + as * kBN, dea, ptx::smem_desc_sw32(ptx::smem_u32(sEB + st * L::EB_BYTES)), idesc_pos, 1u);
-        umma_commit_pair(b_empty + st);   // both CTAs: the stage may be refilled
-        umma_commit_pair(acc_full + as);  // both CTAs: accumulator ready for the epilogue
+        if (ok) umma_commit_pair(a_empty);  // both CTAs: the resident block may be replaced
+        base += w.nt;
+        ++ua;
       }
     }
   } else if constexpr (kEmit) {
@@ -283,12 +320,15 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kSimThreads, 1) sim_
     const int cg = ((warp - 2) >> 2) & 1; // which half of the tile's columns
     const int R = row0 + q * 32;          // first row of this warp's 32-row strip
     const int row = R + lane;
-    const bool live_block = row0 < l;     // the second CTA of a sequence's last pair may own no row at all
     const uint32_t tcol = tmem_base + ((uint32_t)(q * 32) << 16) + team * kBN + cg * kColsPerWarp;
     const uint32_t below = (1u << lane) - 1u;
     const uint32_t key_row = (uint32_t)row << kRecRowShift;
+    // records are counted per block and unit: this instantiation is launched with one unit per pair of blocks
+    const UnitWork w = unit_work(blockIdx.y);
+    const int unit = w.unit, l = w.l;
+    const bool live_block = row0 < l;     // the second CTA of a sequence's last pair may own no row at all
 #pragma unroll 1
-    for (int it = team; tile0 + it < n_tiles; it += 2) {
+    for (int it = team; it < w.nt; it += 2) {
       const int c0 = (tile0 + it) * kBN;
       bool ok = __all_sync(0xffffffffu, ptx::mbar_wait(acc_full + team, (it >> 1) & 1, abort_flag, wait_cycles));
       if (!ok) break;                     // nobody waits for this warp: it may leave its loop
@@ -366,138 +406,147 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kSimThreads, 1) sim_
     const int rl = q * 32 + lane;         // row within the block
     const int R = row0 + q * 32;          // first row of this warp's 32-row strip
     const int row = R + lane;
-    const int RW = p.row_words;
-    uint32_t* adj_unit = p.adj + (int64_t)unit * p.batch.max_len * RW;
-    const int NC = RW >> 1;               // 64-column chunks per row
-    const int blk = blockIdx.x;
-    uint32_t* funit = p.flags + (int64_t)unit * NC * RW;
-    // the second CTA of a sequence's last pair may own no row at all: it still loads its half tiles and
-    // keeps the barrier protocol going, but reads and writes nothing
-    const bool live_block = row0 < l;
-    if (lane == 0 && live_block) {
-      // The two chunks that hold the block's own 128 columns are flagged as occupied without looking:
-      // for the block's rows (diagonal bit, and words mirrored inside the block), and, from an even
-      // block, for the rows of the next block, which its diagonal tile mirrors into piecemeal.
-      const int chunk = 2 * blk + cg;
-      const int wb = (row0 >> 5) + team * 4 + q;   // team 0: own rows; team 1: the next block's rows
-      if (chunk < NC && wb < RW && (team == 0 || !(blk & 1))) funit[(int64_t)wb * NC + chunk] = 0xFFFFFFFFu;
-    }
     TransposeLane tr;
     tr.init(lane);
-    uint32_t* sD_team = sD + team * (2 * kBM * kDPitch);
-    // mirrored rows: thread tt of the team writes row c0 + tt, 16 bytes at the block's column
-    const uint32_t tcol = tmem_base + ((uint32_t)(q * 32) << 16) + team * kBN + cg * kColsPerWarp;
-    uint32_t* tq = sT + (team * 4 + q) * kBN + cg * kColsPerWarp + lane;
-    const uint32_t* tr0 = sT + team * 4 * kBN + tt;
-    // No early exit from this loop: after a wait that gave up (every later wait then returns at once)
-    // the warp still meets its partners at each barrier, with nothing to do in between.
-    for (int it = team; tile0 + it < n_tiles; it += 2) {
-      const int tile = tile0 + it;
-      const int c0 = tile * kBN;
-      const bool fast = c0 >= row0 + kBM;      // whole tile strictly above the diagonal
-      const int slot = (tile >> 1) & 1;        // which of the team's two tiles of the four-tile span
-      uint32_t* sdbuf = sD_team + ((tile >> 2) & 1) * (kBM * kDPitch);
-      uint32_t* sdw = sdbuf + rl * kDPitch + slot * kTileWords + cg * kChunks;
-      bool ok = __all_sync(0xffffffffu, ptx::mbar_wait(acc_full + team, (it >> 1) & 1, abort_flag, wait_cycles));
-      if (ok && !live_block) {
-        if (lane == 0) mbar_arrive_leader(acc_empty + team);
-        ok = false;
+    int base = 0;
+    // Every unit of the pair, also after a wait that gave up (every later wait then returns at once): the warps of
+    // a team meet at named barriers inside, so none may leave early.
+    for (int k = blockIdx.y; k < n_work; k += gridDim.y) {
+      const UnitWork w = unit_work(k);
+      if (w.nt == 0) continue;
+      const int unit = w.unit, l = w.l, n_tiles = w.n_tiles;
+      const int RW = p.row_words;
+      uint32_t* adj_unit = p.adj + (int64_t)unit * p.batch.max_len * RW;
+      const int NC = RW >> 1;               // 64-column chunks per row
+      const int blk = blockIdx.x;
+      uint32_t* funit = p.flags + (int64_t)unit * NC * RW;
+      // the second CTA of a sequence's last pair may own no row at all: it still loads its half tiles and
+      // keeps the barrier protocol going, but reads and writes nothing
+      const bool live_block = row0 < l;
+      if (lane == 0 && live_block) {
+        // The two chunks that hold the block's own 128 columns are flagged as occupied without looking:
+        // for the block's rows (diagonal bit, and words mirrored inside the block), and, from an even
+        // block, for the rows of the next block, which its diagonal tile mirrors into piecemeal.
+        const int chunk = 2 * blk + cg;
+        const int wb = (row0 >> 5) + team * 4 + q;   // team 0: own rows; team 1: the next block's rows
+        if (chunk < NC && wb < RW && (team == 0 || !(blk & 1))) funit[(int64_t)wb * NC + chunk] = 0xFFFFFFFFu;
       }
-      if (ok) {
-        ptx::tc_fence_after();
-        uint32_t words[kChunks];
-#pragma unroll
-        for (int ch = 0; ch < kChunks; ++ch) {
-          uint32_t acc[32];
-          ptx::tmem_ld_32x32(tcol + ch * 32, acc);
-          ptx::tmem_ld_wait(acc);
-          words[ch] = sign_word(acc);
+      uint32_t* sD_team = sD + team * (2 * kBM * kDPitch);
+      // mirrored rows: thread tt of the team writes row c0 + tt, 16 bytes at the block's column
+      const uint32_t tcol = tmem_base + ((uint32_t)(q * 32) << 16) + team * kBN + cg * kColsPerWarp;
+      uint32_t* tq = sT + (team * 4 + q) * kBN + cg * kColsPerWarp + lane;
+      const uint32_t* tr0 = sT + team * 4 * kBN + tt;
+      // No early exit from this loop: after a wait that gave up (every later wait then returns at once)
+      // the warp still meets its partners at each barrier, with nothing to do in between.
+      for (int it = (team ^ base) & 1; it < w.nt; it += 2) {
+        const int tile = tile0 + it;
+        const int c0 = tile * kBN;
+        const bool fast = c0 >= row0 + kBM;      // whole tile strictly above the diagonal
+        const int slot = (tile >> 1) & 1;        // which of the team's two tiles of the four-tile span
+        uint32_t* sdbuf = sD_team + ((tile >> 2) & 1) * (kBM * kDPitch);
+        uint32_t* sdw = sdbuf + rl * kDPitch + slot * kTileWords + cg * kChunks;
+        bool ok = __all_sync(0xffffffffu, ptx::mbar_wait(acc_full + team, ((base + it) >> 1) & 1, abort_flag, wait_cycles));
+        if (ok && !live_block) {
+          if (lane == 0) mbar_arrive_leader(acc_empty + team);
+          ok = false;
         }
-        ptx::tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive_leader(acc_empty + team);
-        if (c0 + kBN > l || R + 32 > l) {
-          // ragged edge: columns and rows that do not exist carry no bits
-#pragma unroll
+        if (ok) {
+          ptx::tc_fence_after();
+          uint32_t words[kChunks];
+  #pragma unroll
           for (int ch = 0; ch < kChunks; ++ch) {
-            const int nvalid = l - (c0 + cg * kColsPerWarp + ch * 32);
-            if (nvalid < 32) words[ch] &= nvalid > 0 ? ((1u << nvalid) - 1u) : 0u;
-            if (row >= l) words[ch] = 0;
+            uint32_t acc[32];
+            ptx::tmem_ld_32x32(tcol + ch * 32, acc);
+            ptx::tmem_ld_wait(acc);
+            words[ch] = sign_word(acc);
           }
-        }
-        if (c0 + cg * kColsPerWarp >= row0 + kBM) {
-          // this warp's two 64-column chunks lie right of the block's own columns: their flags for the strip
-          const uint32_t f0 = __ballot_sync(0xffffffffu, (words[0] | words[1]) != 0u);
-          const uint32_t f1 = __ballot_sync(0xffffffffu, (words[2] | words[3]) != 0u);
-          const int chunk = tile * 4 + cg * 2 + lane;
-          const uint32_t fw = lane ? f1 : f0;   // the flag words start at zero: only occupied ones are written
-          if (lane < 2 && chunk < NC && fw) funit[(int64_t)(R >> 5) * NC + chunk] = fw;
-        }
-        if (fast) {
-          *reinterpret_cast<uint2*>(sdw) = make_uint2(words[0], words[1]);
-          *reinterpret_cast<uint2*>(sdw + 2) = make_uint2(words[2], words[3]);
-          // most 32 x 32 sub-blocks of a sparse graph are empty: their mirror image is too
-#pragma unroll
-          for (int ch = 0; ch < kChunks; ++ch)
-            tq[ch * 32] = __any_sync(0xffffffffu, words[ch] != 0u) ? tr.apply(words[ch]) : 0u;
-        } else {
-#pragma unroll
-          for (int ch = 0; ch < kChunks; ++ch) {
-            const int col0 = c0 + cg * kColsPerWarp + ch * 32;
-            if (col0 + 32 <= R) continue;                      // below the diagonal: another block mirrors it
-            if (col0 == R) {
-              // diagonal sub-block: upper triangle as computed, lower triangle mirrored from it, unit diagonal
-              const uint32_t upper = lane == 31 ? 0u : (0xFFFFFFFFu << (lane + 1));
-              const uint32_t wu = words[ch] & upper;
-              const uint32_t wt = tr.apply(wu);
-              sdw[ch] = row < l ? (wu | wt | (1u << lane)) : 0u;
-            } else {
-              sdw[ch] = words[ch];
-              const uint32_t wt = tr.apply(words[ch]);
-              if (col0 + lane < l) adj_unit[(int64_t)(col0 + lane) * RW + (R >> 5)] = wt;
+          ptx::tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive_leader(acc_empty + team);
+          if (c0 + kBN > l || R + 32 > l) {
+            // ragged edge: columns and rows that do not exist carry no bits
+  #pragma unroll
+            for (int ch = 0; ch < kChunks; ++ch) {
+              const int nvalid = l - (c0 + cg * kColsPerWarp + ch * 32);
+              if (nvalid < 32) words[ch] &= nvalid > 0 ? ((1u << nvalid) - 1u) : 0u;
+              if (row >= l) words[ch] = 0;
+            }
+          }
+          if (c0 + cg * kColsPerWarp >= row0 + kBM) {
+            // this warp's two 64-column chunks lie right of the block's own columns: their flags for the strip
+            const uint32_t f0 = __ballot_sync(0xffffffffu, (words[0] | words[1]) != 0u);
+            const uint32_t f1 = __ballot_sync(0xffffffffu, (words[2] | words[3]) != 0u);
+            const int chunk = tile * 4 + cg * 2 + lane;
+            const uint32_t fw = lane ? f1 : f0;   // the flag words start at zero: only occupied ones are written
+            if (lane < 2 && chunk < NC && fw) funit[(int64_t)(R >> 5) * NC + chunk] = fw;
+          }
+          if (fast) {
+            *reinterpret_cast<uint2*>(sdw) = make_uint2(words[0], words[1]);
+            *reinterpret_cast<uint2*>(sdw + 2) = make_uint2(words[2], words[3]);
+            // most 32 x 32 sub-blocks of a sparse graph are empty: their mirror image is too
+  #pragma unroll
+            for (int ch = 0; ch < kChunks; ++ch)
+              tq[ch * 32] = __any_sync(0xffffffffu, words[ch] != 0u) ? tr.apply(words[ch]) : 0u;
+          } else {
+  #pragma unroll
+            for (int ch = 0; ch < kChunks; ++ch) {
+              const int col0 = c0 + cg * kColsPerWarp + ch * 32;
+              if (col0 + 32 <= R) continue;                      // below the diagonal: another block mirrors it
+              if (col0 == R) {
+                // diagonal sub-block: upper triangle as computed, lower triangle mirrored from it, unit diagonal
+                const uint32_t upper = lane == 31 ? 0u : (0xFFFFFFFFu << (lane + 1));
+                const uint32_t wu = words[ch] & upper;
+                const uint32_t wt = tr.apply(wu);
+                sdw[ch] = row < l ? (wu | wt | (1u << lane)) : 0u;
+              } else {
+                sdw[ch] = words[ch];
+                const uint32_t wt = tr.apply(words[ch]);
+                if (col0 + lane < l) adj_unit[(int64_t)(col0 + lane) * RW + (R >> 5)] = wt;
+              }
             }
           }
         }
-      }
-      // the team's mirrored words of this tile are in shared memory
-      epi_bar_n(2 + team, 32 * kTeamWarps);
-      if (ok && fast) {
-        const int b = c0 + tt;
-        bool occ_lo = false, occ_hi = false;
-        if (b < l) {
-          const uint4 mv = make_uint4(tr0[0], tr0[kBN], tr0[2 * kBN], tr0[3 * kBN]);
-          occ_lo = (mv.x | mv.y) != 0u;
-          occ_hi = (mv.z | mv.w) != 0u;
-          uint32_t* dst = adj_unit + (int64_t)b * RW + (row0 >> 5);
-          if (!p.skip_empty) {
-            *reinterpret_cast<uint4*>(dst) = mv;
-          } else {
-            // a reader consults the chunk's flag bit first: empty chunks need not reach memory
-            if (occ_lo) *reinterpret_cast<uint2*>(dst) = make_uint2(mv.x, mv.y);
-            if (occ_hi) *reinterpret_cast<uint2*>(dst + 2) = make_uint2(mv.z, mv.w);
+        // the team's mirrored words of this tile are in shared memory
+        epi_bar_n(2 + team, 32 * kTeamWarps);
+        if (ok && fast) {
+          const int b = c0 + tt;
+          bool occ_lo = false, occ_hi = false;
+          if (b < l) {
+            const uint4 mv = make_uint4(tr0[0], tr0[kBN], tr0[2 * kBN], tr0[3 * kBN]);
+            occ_lo = (mv.x | mv.y) != 0u;
+            occ_hi = (mv.z | mv.w) != 0u;
+            uint32_t* dst = adj_unit + (int64_t)b * RW + (row0 >> 5);
+            if (!p.skip_empty) {
+              *reinterpret_cast<uint4*>(dst) = mv;
+            } else {
+              // a reader consults the chunk's flag bit first: empty chunks need not reach memory
+              if (occ_lo) *reinterpret_cast<uint2*>(dst) = make_uint2(mv.x, mv.y);
+              if (occ_hi) *reinterpret_cast<uint2*>(dst + 2) = make_uint2(mv.z, mv.w);
+            }
+          }
+          const uint32_t flo = __ballot_sync(0xffffffffu, occ_lo), fhi = __ballot_sync(0xffffffffu, occ_hi);
+          const uint32_t fw = lane ? fhi : flo;
+          if (lane < 2 && (b >> 5) < RW && fw) funit[(int64_t)(b >> 5) * NC + 2 * blk + lane] = fw;
+        }
+        if (slot == 1 || tile + 2 >= n_tiles) {
+          // the two warps of the team that share this 32-row strip have staged their direct words of the
+          // team's (up to) two tiles of this four-tile span: two 32-byte pieces per row, sixteen rows per
+          // warp, two rows per store; words left of the strip's diagonal sub-block belong to mirrored writes
+          epi_bar_n(4 + team * 4 + q, 64);
+          const int half = lane >> 4, wl = lane & 15;           // row of the pair, word of the row's 16
+          const int wtile = (tile & ~3) + (tile & 1) + 2 * (wl >> 3);   // the tile this word belongs to
+          const int wi = wtile * kTileWords + (wl & 7);
+          const int r0 = q * 32 + cg * 16 + half;
+          if (wi >= (R >> 5) && wi < RW && wtile < n_tiles) {   // words of tiles beyond the sequence hold nothing of this unit
+            uint32_t* dst = adj_unit + (int64_t)(row0 + r0) * RW + wi;
+            const uint32_t* src = sdbuf + r0 * kDPitch + wl;
+  #pragma unroll
+            for (int i = 0; i < 16; i += 2)
+              if (row0 + r0 + i < l) dst[(int64_t)i * RW] = src[i * kDPitch];
           }
         }
-        const uint32_t flo = __ballot_sync(0xffffffffu, occ_lo), fhi = __ballot_sync(0xffffffffu, occ_hi);
-        const uint32_t fw = lane ? fhi : flo;
-        if (lane < 2 && (b >> 5) < RW && fw) funit[(int64_t)(b >> 5) * NC + 2 * blk + lane] = fw;
       }
-      if (slot == 1 || tile + 2 >= n_tiles) {
-        // the two warps of the team that share this 32-row strip have staged their direct words of the
-        // team's (up to) two tiles of this four-tile span: two 32-byte pieces per row, sixteen rows per
-        // warp, two rows per store; words left of the strip's diagonal sub-block belong to mirrored writes
-        epi_bar_n(4 + team * 4 + q, 64);
-        const int half = lane >> 4, wl = lane & 15;           // row of the pair, word of the row's 16
-        const int wtile = (tile & ~3) + (tile & 1) + 2 * (wl >> 3);   // the tile this word belongs to
-        const int wi = wtile * kTileWords + (wl & 7);
-        const int r0 = q * 32 + cg * 16 + half;
-        if (wi >= (R >> 5) && wi < RW) {
-          uint32_t* dst = adj_unit + (int64_t)(row0 + r0) * RW + wi;
-          const uint32_t* src = sdbuf + r0 * kDPitch + wl;
-#pragma unroll
-          for (int i = 0; i < 16; i += 2)
-            if (row0 + r0 + i < l) dst[(int64_t)i * RW] = src[i * kDPitch];
-        }
-      }
+      base += w.nt;
     }
   }
   // teardown: every role ends here, also after a wait that gave up
@@ -506,7 +555,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kSimThreads, 1) sim_
   __syncthreads();
   if (kEmit && threadIdx.x == 0) {
     const int cap = p.rec_per_tile * ((p.batch.max_len + kBN - 1) / kBN - (int)(blockIdx.x >> 1));
-    p.rec_cnt[(long long)unit * gridDim.x + blockIdx.x] = min(*rec_used, cap);
+    p.rec_cnt[(long long)blockIdx.y * gridDim.x + blockIdx.x] = min(*rec_used, cap);
   }
   if (*abort_flag) {
     if (threadIdx.x == 0) atomicExch(&p.hdr[kHdrStatus], (uint32_t)SPINDLEKV_TIMEOUT);
@@ -673,7 +722,11 @@ spindlekv_status launch_sim_tc(const spindlekv_tensor& Gamma, const spindlekv_ba
   p.rec_per_tile = pool ? pool->rec_per_tile : 0;
   p.unit_rec_cap = pool ? rec_unit_capacity(ceil_div(b.max_len, kBN), pool->rec_per_tile) : 0;
   p.wait_cycles = wait_cycles;
-  dim3 grid(2 * ceil_div(b.max_len, 2 * kBM), units);   // whole pairs
+  // behind a record pool the bit-matrix pass computes the overflowed units only: a few slots of blocks walk their list
+  const bool listed = !emit && pool && pool->rec_per_tile > 0;
+  p.work_list = listed ? pool->work_list : nullptr;
+  p.n_work = listed ? pool->n_work : nullptr;
+  dim3 grid(2 * ceil_div(b.max_len, 2 * kBM), listed ? std::min(units, kFallbackSlots) : units);   // whole pairs
   LaunchScope ls(KC_SIM, st);
   spindlekv_status rs;
   if (head_dim == 128) rs = emit ? launch_sim_tc_one<128, true>(map, emap, p, grid, st) : launch_sim_tc_one<128, false>(map, emap, p, grid, st);

@@ -93,6 +93,39 @@ def test_some_units_in_the_pool_and_some_through_the_bit_matrix_in_one_call():
                                 int(o["n_entries"][li, 0, j]), o["C"][li, 0, j], 1e-2)
 
 
+def test_more_overflowed_units_than_the_bit_matrix_pass_has_slots():
+    # 48 units of two different lengths all overflow a tiny pool: every pair of blocks of the bit-matrix pass then
+    # works through several units one after the other (ring stages and barrier phases carry on from unit to unit)
+    from paper_2507_06517_b200 import binding as B
+    from paper_2507_06517_b200.pipeline import SpindleKVPass
+    wl = synth.Workload("many", 3, 3, 16, 8, 128, "bf16", 32, (700, 390), 100, (0.05, 0.3), 2, "recency",
+                        budget_frac=1.0, seed=94)
+    host = generate(wl)
+    G = stack_layers(wl, host, [0, 1, 2], "V")
+    units = wl.n_shallow * wl.batch * wl.n_kv_heads
+    outs = []
+    for cap in (-1, 2):
+        B.spindlekv_set_tuning(B.TUNE_RECORDS_PER_TILE, cap)
+        p = SpindleKVPass(make_config(wl), wl.seq_lens, torch_dtype(wl), keep_adjacency=True)
+        p.ws_codebook.fill_(0x5A)
+        p.codebook(G, "V")
+        status, detail = p.device_status()["codebook"]
+        assert status == 0 and detail[2] == (0 if cap < 0 else units)
+        outs.append([p.cb["V"][k].clone() for k in ("ref", "n_entries", "mag")] + [p.adj.clone()])
+    for a, b in zip(*outs):
+        assert torch.equal(a, b)
+    # and the result is the checker's (one unit of each length)
+    o = {k: (v.float() if k == "C" else v).cpu().numpy() for k, v in p.cb["V"].items()}
+    adj = outs[1][3].cpu().numpy()
+    cu = synth.cu_seqlens(wl)
+    for li, s_, j in ((0, 0, 0), (2, 1, 7)):
+        l = wl.seq_lens[s_]
+        unit = (li * wl.batch + s_) * wl.n_kv_heads + j
+        gamma = host[li][1][cu[s_]:cu[s_ + 1], j]
+        check_codebook_unit(gamma, wl.theta_v, adj[unit], o["mag"][li, j, cu[s_]:cu[s_] + l], o["ref"][li, j, cu[s_]:cu[s_] + l],
+                            o["centre_idx"][li, j, cu[s_]:cu[s_] + l], int(o["n_entries"][li, s_, j]), None, 1e-2)
+
+
 def test_dense_graph_goes_through_the_bit_matrix_by_itself():
     # three big clusters: rows with hundreds of neighbours, whose lists do not fit the record path's budget
     wl = synth.Workload("dense", 1, 1, 2, 2, 128, "bf16", 8, (700,), 3, (0.02, 0.1), 2, "gauss",
