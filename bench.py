@@ -52,6 +52,8 @@ def parse_args():
                     help="the paper's own composition: every layer evicts, then builds CodeBooks of what it kept")
     ap.add_argument("--repeat", action="store_true",
                     help="with --literal: unfold GQA, every query head selects its own tokens (Section 3.3)")
+    ap.add_argument("--decode", action="store_true",
+                    help="one decode step of attention over the replaced cache of every layer (Eq. 14 with RoPE re-applied)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--e2e-chunk", type=int, default=4, help="CodeBook layers per upload/compute/download group")
@@ -305,6 +307,60 @@ def run_literal(args, wl):
             "gpu_launches": int(launches),
             "reserve_ratio": {"r1_mean": float(r1.mean()), "r2_mean": float(r2.mean()), "r1_r2_mean": float((r1 * r2).mean()),
                               "kept_first_last": [int(kept[0]), int(kept[-1])]}}
+    print(json.dumps(line))
+
+
+def run_decode(args, wl):
+    """CodeBooks of every layer (all tokens), then decode steps: the queries of one new token attend to the replaced
+    cache of all layers.  Reports the time of a step and the bytes it has to read (CodeBook rows once, reference and
+    magnitude per token) beside the bytes of the dense cache it stands for."""
+    from paper_2507_06517_b200 import binding as B
+    from paper_2507_06517_b200.pipeline import SpindleKVDecodeAttention, SpindleKVPass
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the reduction pass has no CPU fallback")
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    wl = wl.replace(n_shallow=wl.n_layers, budget_tokens=None, budget_frac=1.0)
+    hK, hV, _ = host_inputs(wl)
+    cfg = B.Config(n_layers=wl.n_layers, n_q_heads=wl.n_q_heads, n_kv_heads=wl.n_kv_heads, head_dim=wl.head_dim,
+                   window=wl.window, n_shallow=wl.n_layers, beta=wl.beta, theta_k=wl.theta_k, theta_v=wl.theta_v, reserve_ratio=1.0)
+    p = SpindleKVPass(cfg, wl.seq_lens, hK.dtype, device=dev, layers_per_codebook_call=min(8, wl.n_layers))
+    p.run(hK.to(dev), hV.to(dev), None)
+    if p.device_status()["codebook"][0]:
+        raise RuntimeError("device status in the CodeBook pass")
+    n, d, e = wl.max_len, wl.head_dim, hK.element_size()
+    att = SpindleKVDecodeAttention(p.cb_batch if p.cb_layers_per_call == wl.n_layers else B.Batch(wl.n_layers, wl.batch, n, wl.batch * n),
+                                   wl.n_q_heads, wl.n_kv_heads, d, n + 64)
+    g = torch.Generator(device="cpu").manual_seed(wl.seed)
+    q = torch.randn((wl.n_layers, wl.batch, wl.n_q_heads, 1, d), generator=g).to(hK.dtype).to(dev)
+    pos_q = torch.full((wl.batch,), n, dtype=torch.int32, device=dev)
+    step = lambda: att.run(q, pos_q, p.cb["K"], p.cb["V"])
+    for _ in range(max(args.warmup, 3)):
+        step()
+    B.spindlekv_launch_count(True)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize(dev)
+    ev0.record()
+    for _ in range(args.steps):
+        step()
+    ev1.record()
+    torch.cuda.synchronize(dev)
+    ms = ev0.elapsed_time(ev1) / args.steps
+    launches = B.spindlekv_launch_count(True)
+    entries = int(p.cb["K"]["n_entries"].sum().item()) + int(p.cb["V"]["n_entries"].sum().item())
+    units = wl.n_layers * wl.batch * wl.n_kv_heads
+    alg = entries * d * e + units * n * 16                  # CodeBook rows once; reference and magnitude of K and of V per token
+    dense = units * n * 2 * d * e
+    pk, pk_src = peaks()
+    line = {"metric": "decode steps/s over the replaced cache of all layers (Eq. 14, RoPE re-applied)", "value": 1e3 / ms, "unit": "steps/s",
+            "n_gpus": 1, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic",
+            "config": workload_config(wl, {"cached_tokens_per_head": n, "query_heads_per_kv_head": wl.group}),
+            "gpu_launches": int(launches),
+            "roofline": {"kernel": "decode attention over CodeBooks", "bound": "hbm", "achieved": alg / (ms * 1e-3) / 1e9,
+                         "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": alg / (ms * 1e-3) / 1e9 / pk["hbm_gbs"], "traffic": None,
+                         "peak_source": pk_src, "algorithmic_bytes": alg, "dense_cache_bytes": dense,
+                         "codebook_entries_over_tokens": entries / (2.0 * units * n)}}
     print(json.dumps(line))
 
 
@@ -570,6 +626,8 @@ if __name__ == "__main__":
                       name=f"{w.name}[{a.layers} layers]")
     if a.impl == "reference":
         run_reference(a, w)
+    elif a.decode:
+        run_decode(a, w)
     elif a.literal:
         run_literal(a, w)
     else:

@@ -348,7 +348,8 @@ int64_t spindlekv_launch_count(int32_t reset);
  * Optional per-kernel timing with CUDA events recorded on the caller's stream around each launch.
  * spindlekv_timing_enable(1) starts collecting (costs two event records per launch);
  * spindlekv_timing_read synchronises the recorded events and returns, for kernel class `which`
- * (0 window-score, 1 top-k, 2 norms, 3 similarity, 4 degree, 5 greedy, 6 finalise, 7 gather),
+ * (0 window-score, 1 top-k, 2 norms, 3 similarity, 4 neighbour lists, 5 greedy cover, 6 entry numbering, 7 gather,
+ * 8 the bit-matrix pass of the similarity kernel over units that overflowed their record pool, 9 decode attention),
  * the summed milliseconds and the number of launches since the last spindlekv_timing_enable call.
  */
 void spindlekv_timing_enable(int32_t on);

@@ -19,7 +19,8 @@ OK, INVALID_ARG, BUDGET, WORKSPACE_TOO_SMALL, CAPACITY, UNSUPPORTED, CUDA_ERROR,
 F32, BF16 = 0, 1
 MODE_EVICT, MODE_CODEBOOK = 1, 2
 WS_EVICT, WS_CODEBOOK = 0, 1
-KERNEL_CLASSES = ("window_score", "topk", "norms", "similarity", "degree", "greedy", "finalise", "gather")
+KERNEL_CLASSES = ("window_score", "topk", "norms", "similarity", "degree", "greedy", "finalise", "gather",
+                  "similarity_fallback", "decode")
 
 
 class SpindleKVError(RuntimeError):

@@ -21,7 +21,7 @@ constexpr int kHdrBitUnits = 3;
 constexpr int kHdrListEntries = 4;
 
 // kernel classes for launch counting / timing
-enum KernelClass { KC_WINDOW = 0, KC_TOPK, KC_NORMS, KC_SIM, KC_DEGREE, KC_GREEDY, KC_FINAL, KC_GATHER, KC_COUNT };
+enum KernelClass { KC_WINDOW = 0, KC_TOPK, KC_NORMS, KC_SIM, KC_DEGREE, KC_GREEDY, KC_FINAL, KC_GATHER, KC_SIM_FALLBACK, KC_DECODE, KC_COUNT };
 
 struct View {  // device-side copy of spindlekv_tensor
   const void* ptr;

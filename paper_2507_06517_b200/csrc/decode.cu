@@ -11,9 +11,9 @@
 //      token's magnitude, rotate it, and form the dot products with the rotated queries (kept in shared
 //      memory); the 16 partial sums meet through shuffles.  Scores of the chunk stay in shared memory.
 //   2. the chunk's maximum and exp-sum per query head (fixed-order block reductions);
-//   3. values: every thread owns one pair of output elements of one query head and walks the chunk's
-//      tokens in order, adding weight * magnitude * CodeBook row; the row pieces of a token are read by
-//      consecutive threads.
+//   3. values: every thread owns one pair of output elements for all query heads and a share of the chunk's
+//      tokens, adding weight * magnitude * CodeBook row; the row pieces of a token are read by consecutive
+//      threads, once for the whole group; the shares are then added up in a fixed order.
 // A second kernel merges the chunks of a unit (log-sum-exp weights) in chunk order.  All sums run in a
 // fixed order: the result is bit-reproducible from run to run.
 #include <math_constants.h>
@@ -22,7 +22,7 @@
 
 namespace skv {
 
-constexpr int kDecChunk = 1024;    // tokens per block
+constexpr int kDecChunk = 512;     // tokens per block
 constexpr int kDecThreads = 256;
 constexpr int kDecMaxGroup = 8;    // query heads per KV head
 
@@ -115,45 +115,53 @@ __global__ void __launch_bounds__(kDecThreads) decode_chunk_kernel(DecodeParams 
     smv[t] = p.mag_v[orow + t0 + t];
   }
   __syncthreads();
-  // ---- 1. scores ----
+  // ---- 1. scores: two tokens per 16-thread group and sweep, all their loads in flight before any is used ----
   {
+    constexpr int kTok = 2;
     const int sub = tid & 15, grp = tid >> 4;     // 16 token groups per sweep
-    for (int tb = 0; tb < nt; tb += kDecThreads / 16) {
-      const int t = tb + grp;
-      float acc[kDecMaxGroup];
+    for (int tb = 0; tb < nt; tb += kTok * (kDecThreads / 16)) {
+      float lo[kTok][PPT], hi[kTok][PPT], m[kTok];
+      float2 cs[kTok][PPT];
+      int tk[kTok];
 #pragma unroll
-      for (int g = 0; g < kDecMaxGroup; ++g) acc[g] = 0.f;
-      if (t < nt) {
-        const int r = p.ref_k[orow + t0 + t];
-        const float m = p.mag_k[orow + t0 + t];
-        const int pos = p.positions ? p.positions[orow + t0 + t] : t0 + t;
+      for (int x = 0; x < kTok; ++x) {
+        const int t = tb + x * (kDecThreads / 16) + grp;
+        tk[x] = t;
+        const bool has = t < nt;
+        const int r = has ? p.ref_k[orow + t0 + t] : 0;
+        m[x] = has ? p.mag_k[orow + t0 + t] : 0.f;
+        const int pos = (has && p.positions) ? p.positions[orow + t0 + t] : t0 + t;
         const float2* tab = p.table + (int64_t)min(max(pos, 0), p.table_positions - 1) * H + sub * PPT;
         const T* row = ck + (int64_t)r * p.CK.st;
-        float lo[PPT], hi[PPT];
-        load_row_piece<T, PPT>(row + sub * PPT, lo);
-        load_row_piece<T, PPT>(row + H + sub * PPT, hi);
-        float2 cs[PPT];
+        load_row_piece<T, PPT>(row + sub * PPT, lo[x]);
+        load_row_piece<T, PPT>(row + H + sub * PPT, hi[x]);
 #pragma unroll
         for (int k = 0; k < PPT; k += 2) {
           const float4 v = *reinterpret_cast<const float4*>(tab + k);
-          cs[k] = make_float2(v.x, v.y);
-          cs[k + 1] = make_float2(v.z, v.w);
+          cs[x][k] = make_float2(v.x, v.y);
+          cs[x][k + 1] = make_float2(v.z, v.w);
         }
+      }
+#pragma unroll
+      for (int x = 0; x < kTok; ++x) {
+        float acc[kDecMaxGroup];
+#pragma unroll
+        for (int g = 0; g < kDecMaxGroup; ++g) acc[g] = 0.f;
 #pragma unroll
         for (int k = 0; k < PPT; ++k) {
-          const float a = lo[k] * m, b = hi[k] * m;               // Eq. (14)
-          const float ra = a * cs[k].x - b * cs[k].y, rb = b * cs[k].x + a * cs[k].y;
+          const float a = lo[x][k] * m[x], b = hi[x][k] * m[x];               // Eq. (14)
+          const float ra = a * cs[x][k].x - b * cs[x][k].y, rb = b * cs[x][k].x + a * cs[x][k].y;
 #pragma unroll
           for (int g = 0; g < kDecMaxGroup; ++g)
             if (g < h_n) acc[g] = fmaf(sq[g * D + sub * PPT + k], ra, fmaf(sq[g * D + H + sub * PPT + k], rb, acc[g]));
         }
-      }
 #pragma unroll
-      for (int g = 0; g < kDecMaxGroup; ++g) {
-        if (g < h_n) {
+        for (int g = 0; g < kDecMaxGroup; ++g) {
+          if (g < h_n) {
 #pragma unroll
-          for (int o = 8; o >= 1; o >>= 1) acc[g] += __shfl_xor_sync(0xffffffffu, acc[g], o);
-          if (sub == 0 && t < nt) sc[g * kDecChunk + t] = acc[g] * p.scale;
+            for (int o = 8; o >= 1; o >>= 1) acc[g] += __shfl_xor_sync(0xffffffffu, acc[g], o);
+            if (sub == 0 && tk[x] < nt) sc[g * kDecChunk + tk[x]] = acc[g] * p.scale;
+          }
         }
       }
     }
@@ -182,18 +190,20 @@ __global__ void __launch_bounds__(kDecThreads) decode_chunk_kernel(DecodeParams 
     }
   }
   __syncthreads();
-  // ---- 3. values: slot = (query head, pair of output elements) ----
-  for (int slot = tid; slot < h_n * H; slot += kDecThreads) {
-    const int g = slot / H, pr = slot - g * H;
-    const float* wgt = sc + g * kDecChunk;
-    float o0 = 0.f, o1 = 0.f;
-    for (int tb = 0; tb < nt; tb += 4) {
-      float x[4][2];
-      float wv[4];
+  // ---- 3. values: a thread owns one pair of output elements for all query heads and every kParts-th token, so a
+  // CodeBook row piece is loaded once for the whole group; the kParts partial sums meet in shared memory ----
+  {
+    constexpr int kParts = kDecThreads / H;
+    constexpr int kUnroll = 8;
+    const int pr = tid % H, tq = tid / H;
+    float o[kDecMaxGroup][2];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const int t = tb + i;
-        wv[i] = t < nt ? wgt[t] : 0.f;
+    for (int g = 0; g < kDecMaxGroup; ++g) o[g][0] = o[g][1] = 0.f;
+    for (int tb = tq; tb < nt; tb += kParts * kUnroll) {
+      float x[kUnroll][2];
+#pragma unroll
+      for (int i = 0; i < kUnroll; ++i) {
+        const int t = tb + i * kParts;
         const int r = t < nt ? srv[t] : 0;
         if constexpr (sizeof(T) == 4) {
           const float2 v = *reinterpret_cast<const float2*>(cv + (int64_t)r * p.CV.st + 2 * pr);
@@ -204,13 +214,33 @@ __global__ void __launch_bounds__(kDecThreads) decode_chunk_kernel(DecodeParams 
         }
       }
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        o0 = fmaf(wv[i], x[i][0], o0);
-        o1 = fmaf(wv[i], x[i][1], o1);
+      for (int i = 0; i < kUnroll; ++i) {
+        const int t = tb + i * kParts;
+        if (t >= nt) continue;
+#pragma unroll
+        for (int g = 0; g < kDecMaxGroup; ++g)
+          if (g < h_n) {
+            const float wv = sc[g * kDecChunk + t];
+            o[g][0] = fmaf(wv, x[i][0], o[g][0]);
+            o[g][1] = fmaf(wv, x[i][1], o[g][1]);
+          }
       }
     }
-    part[g * (D + 2) + 2 + 2 * pr] = o0;
-    part[g * (D + 2) + 2 + 2 * pr + 1] = o1;
+    __syncthreads();                         // every thread is done with the weights: their place takes the partial sums
+    float* ps = sc;                          // [kParts][h_n][D]
+#pragma unroll
+    for (int g = 0; g < kDecMaxGroup; ++g)
+      if (g < h_n) {
+        ps[(tq * h_n + g) * D + 2 * pr] = o[g][0];
+        ps[(tq * h_n + g) * D + 2 * pr + 1] = o[g][1];
+      }
+    __syncthreads();
+    for (int i = tid; i < h_n * D; i += kDecThreads) {
+      float sum = 0.f;
+#pragma unroll
+      for (int q = 0; q < kParts; ++q) sum += ps[q * h_n * D + i];   // fixed order
+      part[(i / D) * (D + 2) + 2 + (i % D)] = sum;
+    }
   }
   if (tid < h_n) {
     part[tid * (D + 2)] = red[tid * 2];
@@ -282,8 +312,8 @@ static spindlekv_status launch_decode(const DecodeParams& p, int units, cudaStre
       return SPINDLEKV_CUDA;
     once.done[dev] = true;
   }
-  { LaunchScope ls(KC_GATHER, st); decode_chunk_kernel<T, D><<<dim3(p.n_chunks, units), kDecThreads, smem, st>>>(p); }
-  { LaunchScope ls(KC_GATHER, st); decode_merge_kernel<D><<<units, kDecThreads, 0, st>>>(p); }
+  { LaunchScope ls(KC_DECODE, st); decode_chunk_kernel<T, D><<<dim3(p.n_chunks, units), kDecThreads, smem, st>>>(p); }
+  { LaunchScope ls(KC_DECODE, st); decode_merge_kernel<D><<<units, kDecThreads, 0, st>>>(p); }
   return cudaGetLastError() == cudaSuccess ? SPINDLEKV_OK : SPINDLEKV_CUDA;
 }
 

@@ -727,7 +727,7 @@ spindlekv_status launch_sim_tc(const spindlekv_tensor& Gamma, const spindlekv_ba
   p.work_list = listed ? pool->work_list : nullptr;
   p.n_work = listed ? pool->n_work : nullptr;
   dim3 grid(2 * ceil_div(b.max_len, 2 * kBM), listed ? std::min(units, kFallbackSlots) : units);   // whole pairs
-  LaunchScope ls(KC_SIM, st);
+  LaunchScope ls(listed ? KC_SIM_FALLBACK : KC_SIM, st);
   spindlekv_status rs;
   if (head_dim == 128) rs = emit ? launch_sim_tc_one<128, true>(map, emap, p, grid, st) : launch_sim_tc_one<128, false>(map, emap, p, grid, st);
   else rs = emit ? launch_sim_tc_one<64, true>(map, emap, p, grid, st) : launch_sim_tc_one<64, false>(map, emap, p, grid, st);
