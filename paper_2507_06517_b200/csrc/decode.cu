@@ -67,7 +67,8 @@ __device__ __forceinline__ void load_row_piece(const T* p, float (&out)[N]) {
   }
 }
 
-template <typename T, int D>
+// HN: query heads per KV head the instantiation is unrolled for (the group's actual size h_n <= HN)
+template <typename T, int D, int HN>
 __global__ void __launch_bounds__(kDecThreads) decode_chunk_kernel(DecodeParams p) {
   constexpr int H = D / 2;            // rotation pairs
   constexpr int PPT = D / 32;         // pairs per thread of a 16-thread token group
@@ -119,6 +120,15 @@ __global__ void __launch_bounds__(kDecThreads) decode_chunk_kernel(DecodeParams 
   {
     constexpr int kTok = 2;
     const int sub = tid & 15, grp = tid >> 4;     // 16 token groups per sweep
+    // this thread's part of the rotated queries stays in registers for the whole chunk
+    float qlo[HN][PPT], qhi[HN][PPT];
+#pragma unroll
+    for (int g = 0; g < HN; ++g)
+#pragma unroll
+      for (int k = 0; k < PPT; ++k) {
+        qlo[g][k] = g < h_n ? sq[g * D + sub * PPT + k] : 0.f;
+        qhi[g][k] = g < h_n ? sq[g * D + H + sub * PPT + k] : 0.f;
+      }
     for (int tb = 0; tb < nt; tb += kTok * (kDecThreads / 16)) {
       float lo[kTok][PPT], hi[kTok][PPT], m[kTok];
       float2 cs[kTok][PPT];
@@ -144,19 +154,19 @@ __global__ void __launch_bounds__(kDecThreads) decode_chunk_kernel(DecodeParams 
       }
 #pragma unroll
       for (int x = 0; x < kTok; ++x) {
-        float acc[kDecMaxGroup];
+        float acc[HN];
 #pragma unroll
-        for (int g = 0; g < kDecMaxGroup; ++g) acc[g] = 0.f;
+        for (int g = 0; g < HN; ++g) acc[g] = 0.f;
 #pragma unroll
         for (int k = 0; k < PPT; ++k) {
           const float a = lo[x][k] * m[x], b = hi[x][k] * m[x];               // Eq. (14)
           const float ra = a * cs[x][k].x - b * cs[x][k].y, rb = b * cs[x][k].x + a * cs[x][k].y;
 #pragma unroll
-          for (int g = 0; g < kDecMaxGroup; ++g)
-            if (g < h_n) acc[g] = fmaf(sq[g * D + sub * PPT + k], ra, fmaf(sq[g * D + H + sub * PPT + k], rb, acc[g]));
+          for (int g = 0; g < HN; ++g)
+            if (g < h_n) acc[g] = fmaf(qlo[g][k], ra, fmaf(qhi[g][k], rb, acc[g]));
         }
 #pragma unroll
-        for (int g = 0; g < kDecMaxGroup; ++g) {
+        for (int g = 0; g < HN; ++g) {
           if (g < h_n) {
 #pragma unroll
             for (int o = 8; o >= 1; o >>= 1) acc[g] += __shfl_xor_sync(0xffffffffu, acc[g], o);
@@ -196,9 +206,9 @@ __global__ void __launch_bounds__(kDecThreads) decode_chunk_kernel(DecodeParams 
     constexpr int kParts = kDecThreads / H;
     constexpr int kUnroll = 8;
     const int pr = tid % H, tq = tid / H;
-    float o[kDecMaxGroup][2];
+    float o[HN][2];
 #pragma unroll
-    for (int g = 0; g < kDecMaxGroup; ++g) o[g][0] = o[g][1] = 0.f;
+    for (int g = 0; g < HN; ++g) o[g][0] = o[g][1] = 0.f;
     for (int tb = tq; tb < nt; tb += kParts * kUnroll) {
       float x[kUnroll][2];
 #pragma unroll
@@ -218,7 +228,7 @@ __global__ void __launch_bounds__(kDecThreads) decode_chunk_kernel(DecodeParams 
         const int t = tb + i * kParts;
         if (t >= nt) continue;
 #pragma unroll
-        for (int g = 0; g < kDecMaxGroup; ++g)
+        for (int g = 0; g < HN; ++g)
           if (g < h_n) {
             const float wv = sc[g * kDecChunk + t];
             o[g][0] = fmaf(wv, x[i][0], o[g][0]);
@@ -229,7 +239,7 @@ __global__ void __launch_bounds__(kDecThreads) decode_chunk_kernel(DecodeParams 
     __syncthreads();                         // every thread is done with the weights: their place takes the partial sums
     float* ps = sc;                          // [kParts][h_n][D]
 #pragma unroll
-    for (int g = 0; g < kDecMaxGroup; ++g)
+    for (int g = 0; g < HN; ++g)
       if (g < h_n) {
         ps[(tq * h_n + g) * D + 2 * pr] = o[g][0];
         ps[(tq * h_n + g) * D + 2 * pr + 1] = o[g][1];
@@ -301,20 +311,28 @@ static size_t decode_smem_bytes(int head_dim) {
   return (size_t)(kDecMaxGroup * head_dim + kDecMaxGroup * kDecChunk + 2 * kDecChunk + kDecMaxGroup * 8) * 4;
 }
 
-template <typename T, int D>
-static spindlekv_status launch_decode(const DecodeParams& p, int units, cudaStream_t st) {
+template <typename T, int D, int HN>
+static spindlekv_status launch_decode_hn(const DecodeParams& p, int units, cudaStream_t st) {
   static PerDeviceOnce once;
   const int dev = PerDeviceOnce::current();
   if (dev < 0) return SPINDLEKV_CUDA;
   const size_t smem = decode_smem_bytes(D);
   if (!once.done[dev]) {
-    if (cudaFuncSetAttribute(decode_chunk_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+    if (cudaFuncSetAttribute(decode_chunk_kernel<T, D, HN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
       return SPINDLEKV_CUDA;
     once.done[dev] = true;
   }
-  { LaunchScope ls(KC_DECODE, st); decode_chunk_kernel<T, D><<<dim3(p.n_chunks, units), kDecThreads, smem, st>>>(p); }
+  { LaunchScope ls(KC_DECODE, st); decode_chunk_kernel<T, D, HN><<<dim3(p.n_chunks, units), kDecThreads, smem, st>>>(p); }
   { LaunchScope ls(KC_DECODE, st); decode_merge_kernel<D><<<units, kDecThreads, 0, st>>>(p); }
   return cudaGetLastError() == cudaSuccess ? SPINDLEKV_OK : SPINDLEKV_CUDA;
+}
+
+template <typename T, int D>
+static spindlekv_status launch_decode(const DecodeParams& p, int units, cudaStream_t st) {
+  if (p.h_n <= 1) return launch_decode_hn<T, D, 1>(p, units, st);
+  if (p.h_n <= 2) return launch_decode_hn<T, D, 2>(p, units, st);
+  if (p.h_n <= 4) return launch_decode_hn<T, D, 4>(p, units, st);
+  return launch_decode_hn<T, D, kDecMaxGroup>(p, units, st);
 }
 
 spindlekv_status decode_attend_impl(const spindlekv_batch& b, int n_q_heads, int n_kv_heads, int head_dim,
