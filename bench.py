@@ -36,7 +36,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # dram__bytes_read.sum + dram__bytes_write.sum of the similarity kernel per unit (one head's K or V of one
 # layer), by sequence length, from the ncu capture summarised under profiles/ (8 units per launch there;
 # traffic grows in proportion to the units of a launch).  Lengths without a capture report null.
-SIMILARITY_TRAFFIC_BYTES_PER_UNIT = {16384: 19.7e6}
+SIMILARITY_TRAFFIC_BYTES_PER_UNIT = {16384: 5.27e6}
 
 
 def parse_args():
