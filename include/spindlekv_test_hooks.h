@@ -24,8 +24,11 @@ enum {
                                            records, every unit is computed as a bit matrix */
   SPINDLEKV_TUNE_GREEDY_ROUND_CAP = 1,  /* rounds after which the greedy cover gives up (default: the sequence length,
                                            which an exact run can never exceed) */
-  SPINDLEKV_TUNE_MBAR_WAIT_CYCLES = 2   /* SM clock cycles after which a wait on a shared-memory barrier of the
+  SPINDLEKV_TUNE_MBAR_WAIT_CYCLES = 2,  /* SM clock cycles after which a wait on a shared-memory barrier of the
                                            tensor-core kernels gives up */
+  SPINDLEKV_TUNE_SIM_BLOCK_PAIRS = 3    /* pairs of blocks the candidate-record similarity kernel runs on (default 0:
+                                           as many as the device holds at once); fewer make every pair walk more
+                                           (unit, row span) items one after the other */
 };
 
 /* Sets one limit; value < 0 restores its default.  INVALID_ARG for an unknown key. */

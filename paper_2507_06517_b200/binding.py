@@ -348,7 +348,7 @@ def spindlekv_poll_status(ws: Optional[torch.Tensor]):
     return int(status.value), [int(x) for x in detail]
 
 
-TUNE_RECORDS_PER_TILE, TUNE_GREEDY_ROUND_CAP, TUNE_MBAR_WAIT_CYCLES = range(3)
+TUNE_RECORDS_PER_TILE, TUNE_GREEDY_ROUND_CAP, TUNE_MBAR_WAIT_CYCLES, TUNE_SIM_BLOCK_PAIRS = range(4)
 
 
 def spindlekv_set_tuning(key: int, value: int) -> None:

@@ -56,7 +56,7 @@ spindlekv_status selftest_mbarrier_impl(uint32_t* hdr, long long wait_cycles, cu
 
 // ---- limits that tests may tighten --------------------------------------------------------------
 static std::mutex g_tune_mu;
-static Tuning g_tuning{kDefaultRecPerTile, 0x7FFFFFFF, kDefaultMbarWaitCycles};
+static Tuning g_tuning{kDefaultRecPerTile, 0x7FFFFFFF, kDefaultMbarWaitCycles, 0};
 Tuning current_tuning() {
   std::lock_guard<std::mutex> lk(g_tune_mu);
   return g_tuning;
@@ -336,6 +336,9 @@ spindlekv_status spindlekv_set_tuning(int32_t key, int64_t value) {
     case SPINDLEKV_TUNE_MBAR_WAIT_CYCLES:
       g_tuning.mbar_wait_cycles = value < 0 ? kDefaultMbarWaitCycles : value;
       return SPINDLEKV_OK;
+    case SPINDLEKV_TUNE_SIM_BLOCK_PAIRS:
+      g_tuning.sim_block_pairs = value < 0 ? 0 : (int)std::min<int64_t>(value, 1 << 20);
+      return SPINDLEKV_OK;
     default:
       return SPINDLEKV_INVALID_ARG;
   }
@@ -347,6 +350,7 @@ int64_t spindlekv_get_tuning(int32_t key) {
     case SPINDLEKV_TUNE_RECORDS_PER_TILE: return t.rec_per_tile;
     case SPINDLEKV_TUNE_GREEDY_ROUND_CAP: return t.round_cap;
     case SPINDLEKV_TUNE_MBAR_WAIT_CYCLES: return t.mbar_wait_cycles;
+    case SPINDLEKV_TUNE_SIM_BLOCK_PAIRS: return t.sim_block_pairs;
     default: return -1;
   }
 }

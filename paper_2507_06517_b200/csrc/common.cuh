@@ -182,6 +182,7 @@ struct Tuning {
   int rec_per_tile;          // 0: no candidate records, every unit goes through the bit matrix
   int round_cap;             // greedy rounds (never more than the sequence length)
   long long mbar_wait_cycles;
+  int sim_block_pairs;       // pairs of blocks the candidate-record kernel runs on; 0: as many as the device holds
 };
 Tuning current_tuning();
 

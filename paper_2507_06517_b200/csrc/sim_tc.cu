@@ -70,6 +70,7 @@ struct SimTcParams {
   // gridDim.y], ...  Null: blockIdx.y is the unit.
   const int32_t* work_list;
   const int32_t* n_work;
+  int n_units;         // units of the call
 };
 
 constexpr int kBM = 128;          // rows of the resident block (UMMA M)
@@ -80,23 +81,30 @@ constexpr int kEpiWarps = 16;                         // two teams of eight; tea
 constexpr int kTeamWarps = kEpiWarps / 2;
 constexpr int kColsPerWarp = kBN / (kTeamWarps / 4);  // tile columns handled by one epilogue warp
 constexpr int kChunks = kColsPerWarp / 32;
-constexpr int kSimThreads = 32 * (2 + kEpiWarps);
+constexpr int kEmitCols = kBN / (kEpiWarps / 4);     // columns of a tile per warp when all warps share every tile
+constexpr int kEmitChunks = kEmitCols / 32;
+static_assert(kEmitChunks == 2, "the record epilogue keeps two words per lane");
+constexpr int kIssueWarp2 = 2 + kEpiWarps;            // the warp of the second MMA-issuing thread
+constexpr int kSimThreads = 32 * (3 + kEpiWarps);   // loads, MMAs of even tiles, epilogue warps, MMAs of odd tiles
 constexpr int kTileWords = kBN / 32;                  // words of a row per tile
 constexpr int kDPitch = 2 * kTileWords + 2;           // staging pitch: a team's two tiles of a four-tile span
 static_assert(kChunks == 4 && kTileWords == 8, "epilogue layout assumes 128 columns per warp");
 
-template <int D>
+// kEmit: two resident blocks (the next one loads while the MMAs read the current one) and no staging of
+// bit-matrix words; otherwise one resident block and the staging areas.
+template <int D, bool kEmit>
 struct SimSmem {
   static constexpr int KH = D / 64;                  // 64-element (128-byte) swizzle atoms along head_dim
+  static constexpr int NA = kEmit ? 2 : 1;           // resident blocks in shared memory
   static constexpr int A_BYTES = KH * kBM * 128;
   static constexpr int B_BYTES = KH * kBH * 128;     // this CTA's half of a streamed tile
   static constexpr int EA_BYTES = kBM * 32;          // threshold rows of the block (one 16-element K-step)
   static constexpr int EB_BYTES = kBH * 32;          // magnitude rows of this CTA's half tile
-  static constexpr int T_BYTES = 2 * 4 * kBN * 4;    // mirrored words [slot][row quarter][tile column]
-  static constexpr int D_BYTES = 2 * 2 * kBM * kDPitch * 4;  // direct words [team][slot][row][word]
-  static constexpr int OFF_B = A_BYTES;
+  static constexpr int T_BYTES = kEmit ? 0 : 2 * 4 * kBN * 4;    // mirrored words [slot][row quarter][tile column]
+  static constexpr int D_BYTES = kEmit ? 0 : 2 * 2 * kBM * kDPitch * 4;  // direct words [team][slot][row][word]
+  static constexpr int OFF_B = NA * A_BYTES;
   static constexpr int OFF_EA = OFF_B + kStages * B_BYTES;
-  static constexpr int OFF_EB = OFF_EA + EA_BYTES;
+  static constexpr int OFF_EB = OFF_EA + NA * EA_BYTES;
   static constexpr int OFF_T = OFF_EB + kStages * EB_BYTES;
   static constexpr int OFF_D = OFF_T + T_BYTES;
   static constexpr int OFF_BAR = OFF_D + D_BYTES;
@@ -110,6 +118,21 @@ struct SimSmem {
 // the two warps of a team that share a 32-row strip (64 threads).
 __device__ __forceinline__ void epi_bar_n(int id, int nthreads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
+
+// Waits until the shared counter `turn` reaches `want`; gives up like a barrier wait (false, abort flag set).
+__device__ __forceinline__ bool wait_turn(volatile int* turn, int want, volatile int* abort_flag, long long limit_cycles) {
+  if (*turn == want) return true;
+  const long long t0 = clock64();
+  for (uint32_t i = 0;; ++i) {
+    if (*turn == want) return true;
+    if ((i & 63u) == 63u) {
+      if (*abort_flag) return false;
+      if (clock64() - t0 > limit_cycles) break;
+    }
+  }
+  *abort_flag = 1;
+  return false;
 }
 
 // sign bits of 32 accumulators -> one word, bit c = sign of column c
@@ -182,18 +205,28 @@ template <int D, bool kEmit>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kSimThreads, 1) sim_tc_kernel(const __grid_constant__ CUtensorMap tmap,
                                                                 const __grid_constant__ CUtensorMap emap,
                                                                 SimTcParams p) {
-  using L = SimSmem<D>;
-  const int n_work = p.work_list ? *p.n_work : (int)gridDim.y;
-  if ((int)blockIdx.y >= n_work) return;     // both CTAs of a pair: nothing to compute
-  const int row0 = blockIdx.x * kBM;
+  using L = SimSmem<D, kEmit>;
+  const int n_work = p.work_list ? *p.n_work : p.n_units;
   const int rank = (int)cluster_ctarank();   // = blockIdx.x & 1
-  const int tile0 = row0 / kBN;   // the tile that holds the pair's diagonal; earlier tiles are mirrored by other pairs
-  // What a pair has to do for its k-th unit.  Every role of both CTAs walks the same units in the same order and
-  // counts the tiles done so far (`base`) and the units that had any (`ua`): ring stages, accumulator stages and
-  // barrier phases carry on from one unit to the next.
-  struct UnitWork { int unit, j, s, layer, l, n_tiles, nt; };
-  auto unit_work = [&](int k) {
-    UnitWork w;
+  // Work of a pair of blocks, walked in the same order by every role of both CTAs.  The roles count the tiles done
+  // so far (`base`) and the pieces that had any (`ua`): ring stages, accumulator stages, resident blocks and barrier
+  // phases carry on from one piece to the next.
+  //  Bit matrix: a piece is (unit, the pair's own 256-row span blockIdx.x / 2); the pair takes the units with list
+  //  index blockIdx.y, blockIdx.y + gridDim.y, ...
+  //  Candidate records: the grid is a fixed number of pairs; item i = (unit i / F, fold f = i % F) holds the spans
+  //  f and n_tiles - 1 - f of the unit, which together always cost n_tiles + 1 tiles, and the pair takes the items
+  //  blockIdx.x / 2, + gridDim.x / 2, ...: neighbouring pairs work on the same few units at any time.
+  constexpr int kHalves = kEmit ? 2 : 1;
+  const int F = kEmit ? ((p.batch.max_len + kBN - 1) / kBN + 1) / 2 : 1;
+  const int item0 = kEmit ? (int)(blockIdx.x >> 1) : (int)blockIdx.y;
+  const int item_step = kEmit ? (int)(gridDim.x >> 1) : (int)gridDim.y;
+  const int n_items = n_work * F;
+  if (item0 >= n_items) return;              // both CTAs of a pair: nothing to compute
+  struct Piece { int unit, j, s, layer, l, n_tiles, nt, span; };
+  auto piece = [&](int i, int h) {
+    Piece w;
+    const int k = kEmit ? i / F : i;
+    const int f = kEmit ? i - k * F : (int)(blockIdx.x >> 1);
     w.unit = p.work_list ? p.work_list[k] : k;
     w.j = w.unit % p.n_kv_heads;
     const int ls = w.unit / p.n_kv_heads;
@@ -201,10 +234,16 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kSimThreads, 1) sim_
     w.layer = ls / p.batch.n_seqs;
     w.l = seq_len(p.batch, w.layer, w.s, w.j);
     w.n_tiles = (w.l + kBN - 1) / kBN;         // tiles of this sequence: columns beyond its end are never produced
-    // nothing when the whole 256-row span lies beyond the sequence
-    w.nt = (row0 & ~(kBN - 1)) >= w.l ? 0 : w.n_tiles - tile0;
+    w.span = h == 0 ? f : w.n_tiles - 1 - f;
+    // a fold has work while its first span is not beyond its second (a sequence shorter than the longest has
+    // fewer folds); the second span counts only where it is another one than the first
+    const bool any = kEmit ? (h == 0 ? 2 * f <= w.n_tiles - 1 : 2 * f < w.n_tiles - 1) : w.span < w.n_tiles;
+    w.nt = any ? w.n_tiles - w.span : 0;
     return w;
   };
+  // bit matrix only: the pair's fixed rows
+  const int row0 = blockIdx.x * kBM;
+  const int tile0 = row0 / kBN;   // the tile that holds the pair's diagonal; earlier tiles are mirrored by other pairs
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -217,25 +256,26 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kSimThreads, 1) sim_
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::OFF_BAR);
   // a_full, b_full and acc_empty are used in the leader (rank 0) only: both CTAs' loads and both CTAs'
   // epilogue warps signal them there; b_empty and acc_full are signalled in both CTAs by the leader's commits
-  uint64_t* a_full = bars + 0;
-  uint64_t* b_full = bars + 1;                  // [kStages]
-  uint64_t* b_empty = bars + 1 + kStages;       // [kStages]
-  uint64_t* acc_full = bars + 1 + 2 * kStages;  // [2]
+  uint64_t* a_full = bars + 0;                  // [2]
+  uint64_t* b_full = bars + 2;                  // [kStages]
+  uint64_t* b_empty = bars + 2 + kStages;       // [kStages]
+  uint64_t* acc_full = bars + 2 + 2 * kStages;  // [2]
   uint64_t* acc_empty = acc_full + 2;           // [2]
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(acc_empty + 3);
-  int* rec_used = reinterpret_cast<int*>(acc_empty + 3) + 1;   // records this block has reserved
-  uint64_t* a_empty = acc_empty + 4;            // both CTAs: the MMAs of a unit have read its resident block
+  uint64_t* a_empty = acc_empty + 4;            // [2] both CTAs: the MMAs of a piece have read its resident block
+  int* rec_used = reinterpret_cast<int*>(acc_empty + 6);   // [2] records reserved for a piece; pieces alternate
+  volatile int* turn = reinterpret_cast<volatile int*>(acc_empty + 7);   // the tile whose MMAs may be issued now
   const long long wait_cycles = p.wait_cycles;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
-    ptx::mbar_init(a_full, 1);
-    ptx::mbar_init(a_empty, 1);
+    for (int i = 0; i < 2; ++i) { ptx::mbar_init(a_full + i, 1); ptx::mbar_init(a_empty + i, 2); }
     for (int i = 0; i < kStages; ++i) { ptx::mbar_init(b_full + i, 1); ptx::mbar_init(b_empty + i, 1); }
-    for (int i = 0; i < 2; ++i) { ptx::mbar_init(acc_full + i, 1); ptx::mbar_init(acc_empty + i, 2 * kTeamWarps); }
+    for (int i = 0; i < 2; ++i) { ptx::mbar_init(acc_full + i, 1); ptx::mbar_init(acc_empty + i, kEmit ? 2 * kEpiWarps : 2 * kTeamWarps); }
     *abort_flag = 0;
-    *rec_used = 0;
+    rec_used[0] = rec_used[1] = 0;
+    *turn = 0;
     ptx::fence_barrier_init();
   }
   if (warp == 1) {
@@ -253,149 +293,183 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kSimThreads, 1) sim_
       ptx::prefetch_tensormap(&emap);
       int base = 0, ua = 0;
       bool ok = true;
-      for (int k = blockIdx.y; ok && k < n_work; k += gridDim.y) {
-        const UnitWork w = unit_work(k);
-        if (w.nt == 0) continue;
-        const int tok0 = p.batch.cu ? p.batch.cu[w.s] : 0;
-        const int sdim = p.batch.cu ? 0 : w.s;
-        // the resident block of the previous unit must have been read by all of its MMAs
-        if (ua > 0 && !ptx::mbar_wait(a_empty, (ua - 1) & 1, abort_flag, wait_cycles)) break;
-        if (rank == 0) ptx::mbar_expect_tx(a_full, 2 * (L::A_BYTES + L::EA_BYTES));
-        for (int kh = 0; kh < L::KH; ++kh)
-          tma_load_5d_pair(sA + kh * kBM * 128, &tmap, a_full, kh * 64, tok0 + row0, w.j, sdim, w.layer);
-        tma_load_4d_pair(sEA, &emap, a_full, 0, row0, w.unit, 0);
-        for (int it = 0; it < w.nt; ++it) {
-          const int gi = base + it, st = gi % kStages;
-          if (!ptx::mbar_wait(b_empty + st, ((gi / kStages) & 1) ^ 1, abort_flag, wait_cycles)) { ok = false; break; }
-          if (rank == 0) ptx::mbar_expect_tx(b_full + st, 2 * (L::B_BYTES + L::EB_BYTES));
-          uint8_t* dst = sB + st * L::B_BYTES;
-          const int brow = (tile0 + it) * kBN + rank * kBH;   // this CTA's half of the tile
+      for (int i = item0; ok && i < n_items; i += item_step) {
+        for (int h = 0; ok && h < kHalves; ++h) {
+          const Piece w = piece(i, h);
+          if (w.nt == 0) continue;
+          const int tok0 = p.batch.cu ? p.batch.cu[w.s] : 0;
+          const int sdim = p.batch.cu ? 0 : w.s;
+          const int ab = ua % L::NA;
+          // the piece that used this resident block before must have been read by all of its MMAs
+          if (ua >= L::NA && !ptx::mbar_wait(a_empty + ab, ((ua / L::NA) & 1) ^ 1, abort_flag, wait_cycles)) { ok = false; break; }
+          if (rank == 0) ptx::mbar_expect_tx(a_full + ab, 2 * (L::A_BYTES + L::EA_BYTES));
+          const int arow = w.span * kBN + rank * kBM;
           for (int kh = 0; kh < L::KH; ++kh)
-            tma_load_5d_pair(dst + kh * kBH * 128, &tmap, b_full + st, kh * 64, tok0 + brow, w.j, sdim, w.layer);
-          tma_load_4d_pair(sEB + st * L::EB_BYTES, &emap, b_full + st, 0, brow, w.unit, 1);
+            tma_load_5d_pair(sA + ab * L::A_BYTES + kh * kBM * 128, &tmap, a_full + ab, kh * 64, tok0 + arow, w.j, sdim, w.layer);
+          tma_load_4d_pair(sEA + ab * L::EA_BYTES, &emap, a_full + ab, 0, arow, w.unit, 0);
+          for (int it = 0; it < w.nt; ++it) {
+            const int gi = base + it, st = gi % kStages;
+            if (!ptx::mbar_wait(b_empty + st, ((gi / kStages) & 1) ^ 1, abort_flag, wait_cycles)) { ok = false; break; }
+            if (rank == 0) ptx::mbar_expect_tx(b_full + st, 2 * (L::B_BYTES + L::EB_BYTES));
+            uint8_t* dst = sB + st * L::B_BYTES;
+            const int brow = (w.span + it) * kBN + rank * kBH;   // this CTA's half of the tile
+            for (int kh = 0; kh < L::KH; ++kh)
+              tma_load_5d_pair(dst + kh * kBH * 128, &tmap, b_full + st, kh * 64, tok0 + brow, w.j, sdim, w.layer);
+            tma_load_4d_pair(sEB + st * L::EB_BYTES, &emap, b_full + st, 0, brow, w.unit, 1);
+          }
+          base += w.nt;
+          ++ua;
         }
-        base += w.nt;
-        ++ua;
       }
     }
-  } else if (warp == 1) {
+  } else if (warp == 1 || warp == kIssueWarp2) {
+    // Two threads of the leader issue the MMAs, one the even tiles (first accumulator), one the odd tiles (second
+    // accumulator), taking turns tile by tile.  Issuing an MMA holds its thread for about as long as the MMA runs,
+    // and the commits and barrier waits around a tile come on top: with one thread the tensor cores sat idle over
+    // those.  Here a thread does its waits while the other issues, takes the turn, issues its nine MMAs, hands the
+    // turn on and only then commits.  (MMAs of two tiles issued in alternation ran far slower: hence the turns.)
     if (lane == 0 && rank == 0) {
+      const int me = warp == 1 ? 0 : 1;
       constexpr uint32_t idesc_neg = ptx::idesc_bf16_f32(2 * kBM, kBN, true);
       constexpr uint32_t idesc_pos = ptx::idesc_bf16_f32(2 * kBM, kBN, false);
-      const uint32_t a_addr = ptx::smem_u32(sA);
-      const uint64_t dea = ptx::smem_desc_sw32(ptx::smem_u32(sEA));
       int base = 0, ua = 0;
       bool ok = true;
-      for (int k = blockIdx.y; ok && k < n_work; k += gridDim.y) {
-        const UnitWork w = unit_work(k);
-        if (w.nt == 0) continue;
-        ok = ptx::mbar_wait(a_full, ua & 1, abort_flag, wait_cycles);
-        for (int it = 0; ok && it < w.nt; ++it) {
-          const int gi = base + it, st = gi % kStages, as = gi & 1;
-          if (!ptx::mbar_wait(b_full + st, (gi / kStages) & 1, abort_flag, wait_cycles)) { ok = false; break; }
-          if (!ptx::mbar_wait(acc_empty + as, ((gi >> 1) & 1) ^ 1, abort_flag, wait_cycles)) { ok = false; break; }
-          ptx::tc_fence_after();
-          const uint32_t b_addr = ptx::smem_u32(sB + st * L::B_BYTES);
+      for (int i = item0; ok && i < n_items; i += item_step) {
+        for (int h = 0; ok && h < kHalves; ++h) {
+          const Piece w = piece(i, h);
+          if (w.nt == 0) continue;
+          const int ab = ua % L::NA;
+          const uint32_t a_addr = ptx::smem_u32(sA + ab * L::A_BYTES);
+          const uint64_t dea = ptx::smem_desc_sw32(ptx::smem_u32(sEA + ab * L::EA_BYTES));
+          ok = ptx::mbar_wait(a_full + ab, (ua / L::NA) & 1, abort_flag, wait_cycles);
+          for (int it = (me ^ base) & 1; ok && it < w.nt; it += 2) {
+            const int gi = base + it, st = gi % kStages;   // gi & 1 == me: the accumulator of this thread
+            if (!ptx::mbar_wait(b_full + st, (gi / kStages) & 1, abort_flag, wait_cycles)) { ok = false; break; }
+            if (!ptx::mbar_wait(acc_empty + me, ((gi >> 1) & 1) ^ 1, abort_flag, wait_cycles)) { ok = false; break; }
+            if (!wait_turn(turn, gi, abort_flag, wait_cycles)) { ok = false; break; }
+            ptx::tc_fence_after();
+            const uint32_t b_addr = ptx::smem_u32(sB + st * L::B_BYTES);
 #pragma unroll
-          for (int kk16 = 0; kk16 < D / 16; ++kk16) {
-            const int kh = kk16 >> 2, kk = kk16 & 3;
-            uint64_t da = ptx::smem_desc_sw128(a_addr + kh * kBM * 128 + kk * 32);
-            uint64_t db = ptx::smem_desc_sw128(b_addr + kh * kBH * 128 + kk * 32);
-            umma_bf16_pair(tmem_base + as * kBN, da, db, idesc_neg, kk16 > 0 ? 1u : 0u);
+            for (int kk16 = 0; kk16 < D / 16; ++kk16) {
+              const int kh = kk16 >> 2, kk = kk16 & 3;
+              uint64_t da = ptx::smem_desc_sw128(a_addr + kh * kBM * 128 + kk * 32);
+              uint64_t db = ptx::smem_desc_sw128(b_addr + kh * kBH * 128 + kk * 32);
+              umma_bf16_pair(tmem_base + me * kBN, da, db, idesc_neg, kk16 > 0 ? 1u : 0u);
+            }
+            // + theta * |a| * |b|
+            umma_bf16_pair(tmem_base + me * kBN, dea, ptx::smem_desc_sw32(ptx::smem_u32(sEB + st * L::EB_BYTES)), idesc_pos, 1u);
+            *turn = gi + 1;                   // the other thread may issue the next tile
+            umma_commit_pair(b_empty + st);   // both CTAs: the stage may be refilled
+            umma_commit_pair(acc_full + me);  // both CTAs: accumulator ready for the epilogue
           }
-          // + theta * |a| * |b|
-          umma_bf16_pair(tmem_base + as * kBN, dea, ptx::smem_desc_sw32(ptx::smem_u32(sEB + st * L::EB_BYTES)), idesc_pos, 1u);
-          umma_commit_pair(b_empty + st);   // both CTAs: the stage may be refilled
-          umma_commit_pair(acc_full + as);  // both CTAs: accumulator ready for the epilogue
+          // both CTAs: the resident block may be replaced once both threads' MMAs of the piece have read it (a
+          // thread without a tile in the piece arrives at once)
+          if (ok) umma_commit_pair(a_empty + ab);
+          base += w.nt;
+          ++ua;
         }
-        if (ok) umma_commit_pair(a_empty);  // both CTAs: the resident block may be replaced
-        base += w.nt;
-        ++ua;
       }
     }
   } else if constexpr (kEmit) {
     // ---- candidate emission ----
+    // All sixteen warps work on every tile: a warp reads 64 columns of its 32 accumulator rows, so that an
+    // accumulator is handed back to the MMAs well within the time the other one takes to fill.
     const int q = warp & 3;               // TMEM lane quarter this warp may read
-    const int team = (warp - 2) >> 3;     // which TMEM stage this warp serves
-    const int cg = ((warp - 2) >> 2) & 1; // which half of the tile's columns
-    const int R = row0 + q * 32;          // first row of this warp's 32-row strip
-    const int row = R + lane;
-    const uint32_t tcol = tmem_base + ((uint32_t)(q * 32) << 16) + team * kBN + cg * kColsPerWarp;
+    const int cg = (warp - 2) >> 2;       // which quarter of the tile's columns
+    const uint32_t tcol = tmem_base + ((uint32_t)(q * 32) << 16) + cg * kEmitCols;
     const uint32_t below = (1u << lane) - 1u;
-    const uint32_t key_row = (uint32_t)row << kRecRowShift;
-    // records are counted per block and unit: this instantiation is launched with one unit per pair of blocks
-    const UnitWork w = unit_work(blockIdx.y);
-    const int unit = w.unit, l = w.l;
-    const bool live_block = row0 < l;     // the second CTA of a sequence's last pair may own no row at all
+    const int T_max = (p.batch.max_len + kBN - 1) / kBN;
+    int base = 0, ui = 0;
+    // every piece of the pair, also after a wait that gave up: the warps meet at a barrier at the end of each
+    for (int i = item0; i < n_items; i += item_step) {
+      for (int h = 0; h < kHalves; ++h) {
+        const Piece w = piece(i, h);
+        if (w.nt == 0) continue;
+        const int unit = w.unit, l = w.l;
+        const int blk = 2 * w.span + rank;             // the 128-row block of the sequence this CTA holds
+        const int R = blk * kBM + q * 32;              // first row of this warp's 32-row strip
+        const int row = R + lane;
+        const uint32_t key_row = (uint32_t)row << kRecRowShift;
+        const int cap = p.rec_per_tile * (T_max - w.span);   // records the block's region holds
+        int* used = rec_used + (ui & 1);               // pieces alternate between two counters
+        const bool live_block = blk * kBM < l;         // the second CTA of a sequence's last span may own no row at all
 #pragma unroll 1
-    for (int it = team; it < w.nt; it += 2) {
-      const int c0 = (tile0 + it) * kBN;
-      bool ok = __all_sync(0xffffffffu, ptx::mbar_wait(acc_full + team, (it >> 1) & 1, abort_flag, wait_cycles));
-      if (!ok) break;                     // nobody waits for this warp: it may leave its loop
-      if (!live_block) {
-        if (lane == 0) mbar_arrive_leader(acc_empty + team);
-        continue;
-      }
-      ptx::tc_fence_after();
-      uint32_t words[kChunks];
-      words[0] = words[1] = words[2] = words[3] = 0u;
-      // This loop must stay a loop: unrolled, every pass gets 32 registers of its own for its accumulators
-      // and the thread (96 registers with twenty warps in the block) spills, which costs more than all the rest.
+        for (int it = 0; it < w.nt; ++it) {
+          const int c0 = (w.span + it) * kBN;
+          const int as = (base + it) & 1;              // accumulator stage of this tile
+          bool ok = __all_sync(0xffffffffu, ptx::mbar_wait(acc_full + as, ((base + it) >> 1) & 1, abort_flag, wait_cycles));
+          if (!ok) break;                     // the barrier at the end of the piece is still met
+          if (!live_block) {
+            if (lane == 0) mbar_arrive_leader(acc_empty + as);
+            continue;
+          }
+          ptx::tc_fence_after();
+          uint32_t words[kEmitChunks];
+          words[0] = words[1] = 0u;
+          // This loop must stay a loop: unrolled, every pass gets 32 registers of its own for its accumulators
+          // and the thread (96 registers with twenty warps in the block) spills, which costs more than all the rest.
 #pragma unroll 1
-      for (int ch = 0; ch < kChunks; ++ch) {
-        uint32_t acc[32];
-        ptx::tmem_ld_32x32_sync(tcol + ch * 32, acc);   // load and wait in one statement
-        const uint32_t w = sign_word(acc);
-        words[0] = ch == 0 ? w : words[0];
-        words[1] = ch == 1 ? w : words[1];
-        words[2] = ch == 2 ? w : words[2];
-        words[3] = ch == 3 ? w : words[3];
-      }
-      ptx::tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive_leader(acc_empty + team);
-      const int wc0 = (c0 + cg * kColsPerWarp) >> 5;   // word column of this warp's first 32 columns
-      if (c0 + kBN > l || R + 32 > l) {
-        // ragged edge: columns and rows that do not exist carry no bits
+          for (int ch = 0; ch < kEmitChunks; ++ch) {
+            uint32_t acc[32];
+            ptx::tmem_ld_32x32_sync(tcol + as * kBN + ch * 32, acc);   // load and wait in one statement
+            const uint32_t sw = sign_word(acc);
+            words[0] = ch == 0 ? sw : words[0];
+            words[1] = ch == 1 ? sw : words[1];
+          }
+          ptx::tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive_leader(acc_empty + as);
+          const int wc0 = (c0 + cg * kEmitCols) >> 5;   // word column of this warp's first 32 columns
+          if (c0 + kBN > l || R + 32 > l) {
+            // ragged edge: columns and rows that do not exist carry no bits
 #pragma unroll
-        for (int ch = 0; ch < kChunks; ++ch) {
-          const int nvalid = l - (wc0 + ch) * 32;
-          if (nvalid < 32) words[ch] &= nvalid > 0 ? ((1u << nvalid) - 1u) : 0u;
-          if (row >= l) words[ch] = 0;
+            for (int ch = 0; ch < kEmitChunks; ++ch) {
+              const int nvalid = l - (wc0 + ch) * 32;
+              if (nvalid < 32) words[ch] &= nvalid > 0 ? ((1u << nvalid) - 1u) : 0u;
+              if (row >= l) words[ch] = 0;
+            }
+          }
+          if (it == 0) {
+            // the tile that holds the diagonal: only pairs a < b are kept (the rest is their mirror image)
+#pragma unroll
+            for (int ch = 0; ch < kEmitChunks; ++ch) {
+              const int col0 = (wc0 + ch) * 32;
+              if (col0 + 32 <= R) words[ch] = 0u;
+              else if (col0 == R) words[ch] &= lane == 31 ? 0u : (0xFFFFFFFFu << (lane + 1));
+            }
+          }
+          uint32_t m[kEmitChunks];
+          int n = 0;
+#pragma unroll
+          for (int ch = 0; ch < kEmitChunks; ++ch) {
+            m[ch] = __ballot_sync(0xffffffffu, words[ch] != 0u);
+            n += __popc(m[ch]);
+          }
+          if (n == 0) continue;
+          int at = 0;
+          if (lane == 0) at = atomicAdd(used, n);
+          at = __shfl_sync(0xffffffffu, at, 0);
+          if (at + n > cap) {
+            if (lane == 0) p.ovf[unit] = 1;   // the unit is computed again as a bit matrix
+            continue;
+          }
+          // the block's region of the unit's record pool (worked out here, where it is needed, to keep registers free)
+          uint2* rec_blk = p.rec + (long long)unit * p.unit_rec_cap + rec_region_offset(blk, T_max, p.rec_per_tile);
+#pragma unroll
+          for (int ch = 0; ch < kEmitChunks; ++ch) {
+            if (words[ch]) rec_blk[at + __popc(m[ch] & below)] = make_uint2(key_row | (uint32_t)(wc0 + ch), words[ch]);
+            at += __popc(m[ch]);
+          }
         }
-      }
-      if (c0 < row0 + kBM) {
-        // the tile that holds the diagonal: only pairs a < b are kept (the rest is their mirror image)
-#pragma unroll
-        for (int ch = 0; ch < kChunks; ++ch) {
-          const int col0 = (wc0 + ch) * 32;
-          if (col0 + 32 <= R) words[ch] = 0u;
-          else if (col0 == R) words[ch] &= lane == 31 ? 0u : (0xFFFFFFFFu << (lane + 1));
+        // all warps have reserved and written this piece's records: publish the count, clear the counter for the
+        // piece after next
+        epi_bar_n(2, 32 * kEpiWarps);
+        if (warp == 2 && lane == 0) {
+          p.rec_cnt[(long long)unit * (2 * T_max) + blk] = min(*used, cap);
+          *used = 0;
         }
-      }
-      uint32_t m[kChunks];
-      int n = 0;
-#pragma unroll
-      for (int ch = 0; ch < kChunks; ++ch) {
-        m[ch] = __ballot_sync(0xffffffffu, words[ch] != 0u);
-        n += __popc(m[ch]);
-      }
-      if (n == 0) continue;
-      int at = 0;
-      if (lane == 0) at = atomicAdd(rec_used, n);
-      at = __shfl_sync(0xffffffffu, at, 0);
-      // the block's region of the unit's record pool (worked out here, where it is needed, to keep registers free)
-      const int T_max = (p.batch.max_len + kBN - 1) / kBN;
-      const int cap = p.rec_per_tile * (T_max - (int)(blockIdx.x >> 1));
-      uint2* rec_blk = p.rec + (long long)unit * p.unit_rec_cap + rec_region_offset((int)blockIdx.x, T_max, p.rec_per_tile);
-      if (at + n > cap) {
-        if (lane == 0) p.ovf[unit] = 1;   // the unit is computed again as a bit matrix
-        continue;
-      }
-#pragma unroll
-      for (int ch = 0; ch < kChunks; ++ch) {
-        if (words[ch]) rec_blk[at + __popc(m[ch] & below)] = make_uint2(key_row | (uint32_t)(wc0 + ch), words[ch]);
-        at += __popc(m[ch]);
+        base += w.nt;
+        ++ui;
       }
     }
   } else {
@@ -411,8 +485,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kSimThreads, 1) sim_
     int base = 0;
     // Every unit of the pair, also after a wait that gave up (every later wait then returns at once): the warps of
     // a team meet at named barriers inside, so none may leave early.
-    for (int k = blockIdx.y; k < n_work; k += gridDim.y) {
-      const UnitWork w = unit_work(k);
+    for (int i = item0; i < n_items; i += item_step) {
+      const Piece w = piece(i, 0);
       if (w.nt == 0) continue;
       const int unit = w.unit, l = w.l, n_tiles = w.n_tiles;
       const int RW = p.row_words;
@@ -553,10 +627,6 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kSimThreads, 1) sim_
   __syncwarp();
   ptx::tc_fence_before();
   __syncthreads();
-  if (kEmit && threadIdx.x == 0) {
-    const int cap = p.rec_per_tile * ((p.batch.max_len + kBN - 1) / kBN - (int)(blockIdx.x >> 1));
-    p.rec_cnt[(long long)blockIdx.y * gridDim.x + blockIdx.x] = min(*rec_used, cap);
-  }
   if (*abort_flag) {
     if (threadIdx.x == 0) atomicExch(&p.hdr[kHdrStatus], (uint32_t)SPINDLEKV_TIMEOUT);
     __nanosleep(100000);  // let any bulk copy still in flight land before the block retires
@@ -683,17 +753,53 @@ bool sim_tc_available() {
 }
 
 template <int D, bool kEmit>
-static spindlekv_status launch_sim_tc_one(const CUtensorMap& map, const CUtensorMap& emap, const SimTcParams& p, dim3 grid,
-                                          cudaStream_t st) {
+static bool sim_tc_prepare() {
   static PerDeviceOnce once;
   const int dev = PerDeviceOnce::current();
-  if (dev < 0) return SPINDLEKV_CUDA;
+  if (dev < 0) return false;
   if (!once.done[dev]) {
-    if (cudaFuncSetAttribute(sim_tc_kernel<D, kEmit>, cudaFuncAttributeMaxDynamicSharedMemorySize, SimSmem<D>::TOTAL) != cudaSuccess)
-      return SPINDLEKV_CUDA;
+    if (cudaFuncSetAttribute(sim_tc_kernel<D, kEmit>, cudaFuncAttributeMaxDynamicSharedMemorySize, SimSmem<D, kEmit>::TOTAL) != cudaSuccess)
+      return false;
     once.done[dev] = true;
   }
-  sim_tc_kernel<D, kEmit><<<grid, kSimThreads, SimSmem<D>::TOTAL, st>>>(map, emap, p);
+  return true;
+}
+
+// Pairs of blocks of the candidate-record kernel that the device holds at once (one block per SM).
+template <int D>
+static int resident_pairs() {
+  static int pairs[kMaxDevices] = {};
+  const int dev = PerDeviceOnce::current();
+  if (dev < 0 || !sim_tc_prepare<D, true>()) return 0;
+  if (pairs[dev] == 0) {
+    int sms = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 2) return 0;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * (sms / 2), 1, 1);
+    cfg.blockDim = dim3(kSimThreads, 1, 1);
+    cfg.dynamicSmemBytes = SimSmem<D, true>::TOTAL;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = 2;
+    attr.val.clusterDim.y = 1;
+    attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, sim_tc_kernel<D, true>, &cfg) != cudaSuccess || n <= 0) {
+      (void)cudaGetLastError();
+      n = sms / 2;
+    }
+    pairs[dev] = std::min(n, sms / 2);
+  }
+  return pairs[dev];
+}
+
+template <int D, bool kEmit>
+static spindlekv_status launch_sim_tc_one(const CUtensorMap& map, const CUtensorMap& emap, const SimTcParams& p, dim3 grid,
+                                          cudaStream_t st) {
+  if (!sim_tc_prepare<D, kEmit>()) return SPINDLEKV_CUDA;
+  sim_tc_kernel<D, kEmit><<<grid, kSimThreads, SimSmem<D, kEmit>::TOTAL, st>>>(map, emap, p);
   return SPINDLEKV_OK;
 }
 
@@ -726,7 +832,18 @@ spindlekv_status launch_sim_tc(const spindlekv_tensor& Gamma, const spindlekv_ba
   const bool listed = !emit && pool && pool->rec_per_tile > 0;
   p.work_list = listed ? pool->work_list : nullptr;
   p.n_work = listed ? pool->n_work : nullptr;
-  dim3 grid(2 * ceil_div(b.max_len, 2 * kBM), listed ? std::min(units, kFallbackSlots) : units);   // whole pairs
+  p.n_units = units;
+  const int spans = ceil_div(b.max_len, 2 * kBM);
+  dim3 grid(2 * spans, listed ? std::min(units, kFallbackSlots) : units);   // whole pairs
+  if (emit) {
+    // as many pairs as the device runs at once, each walking its share of the (unit, fold) items
+    int pairs = head_dim == 128 ? resident_pairs<128>() : resident_pairs<64>();
+    if (pairs <= 0) return SPINDLEKV_CUDA;
+    const Tuning tune = current_tuning();
+    if (tune.sim_block_pairs > 0) pairs = std::min(pairs, tune.sim_block_pairs);
+    const long long items = (long long)units * ((spans + 1) / 2);
+    grid = dim3(2 * (unsigned)std::min<long long>(pairs, items), 1);
+  }
   LaunchScope ls(listed ? KC_SIM_FALLBACK : KC_SIM, st);
   spindlekv_status rs;
   if (head_dim == 128) rs = emit ? launch_sim_tc_one<128, true>(map, emap, p, grid, st) : launch_sim_tc_one<128, false>(map, emap, p, grid, st);

@@ -17,7 +17,7 @@ pytestmark = pytest.mark.gpu
 def _restore_limits():
     from paper_2507_06517_b200 import binding as B
     yield
-    for k in range(3):
+    for k in range(4):
         B.spindlekv_set_tuning(k, -1)
 
 
@@ -124,6 +124,33 @@ def test_more_overflowed_units_than_the_bit_matrix_pass_has_slots():
         gamma = host[li][1][cu[s_]:cu[s_ + 1], j]
         check_codebook_unit(gamma, wl.theta_v, adj[unit], o["mag"][li, j, cu[s_]:cu[s_] + l], o["ref"][li, j, cu[s_]:cu[s_] + l],
                             o["centre_idx"][li, j, cu[s_]:cu[s_] + l], int(o["n_entries"][li, s_, j]), None, 1e-2)
+
+
+def test_few_block_pairs_walk_every_unit_and_row_span():
+    # The candidate-record kernel runs a fixed number of block pairs that share out the (unit, pair of row spans) items.
+    # With 1, 2 or 3 pairs every pair walks many items of sequences of different lengths (odd and even numbers of
+    # 256-row spans, a last span with one live block only) and must give what the full grid gives.
+    from paper_2507_06517_b200 import binding as B
+    wl = synth.Workload("walk", 4, 2, 8, 2, 128, "bf16", 32, (1100, 300, 1537, 700), 120, (0.05, 0.3), 4, "recency",
+                        budget_frac=0.3, seed=95)
+    _, ref_out, n_bits = _codebooks(wl, "K")     # the full grid (checked against the oracle by the parity tests)
+    assert n_bits == 0
+    for pairs in (1, 2, 3):
+        B.spindlekv_set_tuning(B.TUNE_SIM_BLOCK_PAIRS, pairs)
+        assert B.spindlekv_get_tuning(B.TUNE_SIM_BLOCK_PAIRS) == pairs
+        _, out, n_bits = _codebooks(wl, "K", poison=True)
+        assert n_bits == 0
+        for k in ("mag", "ref", "n_entries"):
+            assert np.array_equal(out[k], ref_out[k]), (pairs, k)
+        cu = synth.cu_seqlens(wl)
+        for li in range(wl.n_shallow):
+            for s_ in range(len(wl.seq_lens)):
+                for j in range(wl.n_kv_heads):
+                    m = int(ref_out["n_entries"][li, s_, j])
+                    assert np.array_equal(out["centre_idx"][li, j, cu[s_]:cu[s_] + m], ref_out["centre_idx"][li, j, cu[s_]:cu[s_] + m])
+        for u in range(ref_out["adj"].shape[0]):
+            lu = wl.seq_lens[(u // wl.n_kv_heads) % len(wl.seq_lens)]
+            assert np.array_equal(out["adj"][u, :lu, :(lu + 31) // 32], ref_out["adj"][u, :lu, :(lu + 31) // 32]), (pairs, u)
 
 
 def test_dense_graph_goes_through_the_bit_matrix_by_itself():
