@@ -499,13 +499,18 @@ def run_native(args, wl):
                "codebook_layers_per_group": args.e2e_chunk}
         del p2
 
-    # per-kernel times: one more pass with event pairs around every launch
+    # per-kernel times: one more pass with event pairs around every launch, the three calls one after the other on
+    # one stream (in the timed steps above they run side by side on three streams, where a kernel's span holds its
+    # neighbours' time too)
+    side = p.side_by_side
+    p.side_by_side = False
     B.spindlekv_timing_enable(True)
     for _ in range(args.steps):
         step()
     torch.cuda.synchronize(dev)
     kt = B.spindlekv_timing_read()
     B.spindlekv_timing_enable(False)
+    p.side_by_side = side
 
     # counters of the CodeBook graph stage, per Gamma: the status block of a call holds its rounds, the units that went
     # through the bit matrix and the neighbour-list entries built from candidate records
@@ -603,7 +608,10 @@ def run_native(args, wl):
             "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps,
             "ms_per_step_median": ms_median,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": wl.dtype,
-            "data": "synthetic", "config": workload_config(wl, {"parallelism": f"replicas x{world}"}),
+            "data": "synthetic",
+            "config": workload_config(wl, {"parallelism": f"replicas x{world}",
+                                           "streams": "K CodeBooks, V CodeBooks and eviction side by side on three streams; "
+                                                      "per-kernel times from a serial pass"}),
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roof, "kernels": kernels,
             "greedy_rounds": st.get("codebook", (0, [0]))[1][0]}
     if not args.no_cpu_baseline and world == 1:

@@ -112,8 +112,10 @@ __global__ void __launch_bounds__(256) norms_kernel(CodebookParams p) {
     p.mag[cb_out_row(p, layer, s, j) + block_row0 + threadIdx.x] = sm_m[threadIdx.x];
   if (p.ext) {
     // Operand [op] of the extra K-step, row `row`: slots 0..8 hold the pieces so that the nine products of
-    // an A row with a B row add up to theta*|a| * |b|.  A zero vector takes magnitude 1: its dot
-    // products are 0, so the accumulator keeps the sign of theta, as "0 > theta" demands.
+    // an A row with a B row add up to -theta*|a| * |b|: the similarity kernel negates operand A in every MMA
+    // (one instruction descriptor for the whole tile), which turns a.b into -a.b and this into +theta*|a|*|b|.
+    // A zero vector takes magnitude 1: its dot products are 0, so the accumulator keeps the sign of theta, as
+    // "0 > theta" demands.
     for (int t = threadIdx.x; t < ROWS * 4; t += 256) {
       const int op = t / (ROWS * 2), r = (t % (ROWS * 2)) >> 1, hi = t & 1;
       const int row = block_row0 + r;
@@ -121,7 +123,7 @@ __global__ void __launch_bounds__(256) norms_kernel(CodebookParams p) {
       const float m = sm_m[r];
       const float n = m > 0.f ? m : 1.f;
       __nv_bfloat16 pc[3];
-      split3_bf16(op == 0 ? p.theta * n : n, pc);
+      split3_bf16(op == 0 ? -(p.theta * n) : n, pc);
       __align__(16) __nv_bfloat16 out[8];
 #pragma unroll
       for (int i = 0; i < 8; ++i) {

@@ -3,47 +3,54 @@
 // The adjacency is symmetric, so only pairs (a, b) with a < b are computed and each decision is
 // written twice: into row a and, mirrored, into row b.
 //
-// One CTA owns a block of 128 token rows of one (layer, sequence, head) unit: the block is loaded
-// once by TMA and stays in shared memory as operand A; tiles of 256 token rows, from the tile that
-// holds the diagonal onwards, stream through a ring as operand B.  Two CTAs (a cluster) own the two
-// blocks of a 256-row span and share one MMA stream: each loads only its half of every streamed tile,
-// and one elected thread of the first CTA issues tcgen05.mma.cta_group::2 (256 x 256 x 16, fp32
-// accumulation in both CTAs' TMEM, 128 rows each), which halves the operand traffic per SM.
+// A pair of CTAs (a cluster) works on a 256-row span of one (layer, sequence, head) unit: each CTA's
+// block of 128 token rows is loaded once by TMA and stays in shared memory as operand A; tiles of 256
+// token rows, from the tile that holds the diagonal onwards, stream through a ring as operand B.  The
+// two CTAs share one MMA stream: each loads only its half of every streamed tile, and threads of the
+// first CTA issue tcgen05.mma.cta_group::2 (256 x 256 x 16, fp32 accumulation in both CTAs' TMEM, 128
+// rows each), which halves the operand traffic per SM.
 //
-// The threshold is part of the contraction.  The main K-steps run with the negate-A flag and
+// The threshold is part of the contraction.  Every K-step runs with the negate-A flag: the main ones
 // accumulate -gamma_a . gamma_b; one more K-step multiplies two 16-element rows prepared by the
-// magnitude kernel: theta*|gamma_a| and |gamma_b|, each split into three bf16 pieces, laid out so
-// that the nine cross products add up to theta*|gamma_a|*|gamma_b| (exact up to the fp32
+// magnitude kernel: -theta*|gamma_a| and |gamma_b|, each split into three bf16 pieces, laid out so
+// that the nine cross products add up to -theta*|gamma_a|*|gamma_b| (exact up to the fp32
 // accumulation).  The accumulator then holds  theta*|a||b| - a.b , whose sign bit is the decision
 // a.b / (|a||b|) > theta.  The epilogue therefore only collects sign bits: no per-column operand,
 // no floating-point instruction.
 //
-// Sixteen epilogue warps in two teams of eight read the accumulators back with tcgen05.ld; team e
-// serves TMEM stage e, i.e. every other tile, so that two tiles are in the epilogue at once while the
-// tensor cores fill the stage that was released first.  Inside a team a warp owns a 32-row strip and
-// half of the tile's columns; a thread owns one row a and shifts the sign bits of 32 columns into a
-// word.  Direct words are staged in shared memory and leave in 32-byte pieces, two per row, after the
-// team's two tiles of a four-tile span (the two warps of a strip meet for that); a 32x32 bit transpose
-// across the warp turns the words of a sub-block into the words of the mirrored rows, which are
-// staged too and written 16 bytes per row by the whole team.  Nothing but bits leaves the SM:
-// N*N/8 bytes per unit, plus one bit per (row, 64-column chunk) that says whether the chunk may hold
-// a set bit (0: certainly empty), so that the next kernel reads only the occupied part of a sparse
-// graph.  The flags of 32 consecutive rows and one chunk form a word (`flags[row / 32][chunk]`) with
-// exactly one writer: the rows' own block for chunks at or right of the block's own columns, the
-// block that mirrors into the rows for chunks left of them.  The caller clears the flag words; only
-// words with a set bit are written.
+// Two threads issue the MMAs, one the even tiles into the first accumulator, one the odd tiles into the
+// second, taking turns tile by tile; while one issues, the other does the commits of its last tile and
+// the barrier waits of its next one (with a single thread the tensor cores idled over those).
 //
-// Candidate emission (the first choice; the bit matrix above is the bounded fallback).  Graphs of real
-// caches are sparse: a token is similar to a handful of others.  In this form a warp, after collecting
-// the sign words of its 32 x 128 piece of a tile, keeps the pairs with a < b only and writes nothing but
+// Candidate emission (the first choice; the bit matrix below is the bounded fallback).  Graphs of real
+// caches are sparse: a token is similar to a handful of others.  The launch is a fixed number of CTA
+// pairs, as many as the device holds; they share out the items (unit, fold), a fold being the row spans
+// f and n_tiles - 1 - f of a unit, which together always cost n_tiles + 1 tiles, and walk them with two
+// resident blocks in shared memory, so that the next block loads while the current one is in use and
+// rings, accumulators and barrier phases carry on from item to item.  All sixteen epilogue warps read
+// every tile back with tcgen05.ld (a warp: 32 rows x 64 columns); a thread owns one row a and shifts the
+// sign bits of 32 columns into a word.  A warp keeps the pairs with a < b only and writes nothing but
 // the non-zero words, as records (row, word column, 32 bits): a ballot counts them, one shared-memory
 // atomic reserves room in the block's own region of the unit's record pool, and the lanes store their
-// records side by side.  No transpose, no staging, no barrier between warps: the next kernel mirrors the
-// pairs when it builds the neighbour lists.  A block's region holds `rec_per_tile` records per tile it
-// computes; a block that runs out of room raises the unit's overflow flag, and such units are computed
-// again as a bit matrix by the other instantiation of this kernel (which returns at once for all other
-// units).  The order of the records inside a region depends on warp timing; everything derived from them
-// is independent of that order.
+// records side by side.  No transpose, no staging: the next kernel mirrors the pairs when it builds
+// the neighbour lists.  A block's region holds `rec_per_tile` records per tile it computes; a block
+// that runs out of room raises the unit's overflow flag, and such units are computed again as a bit
+// matrix.  The order of the records inside a region depends on warp timing; everything derived from
+// them is independent of that order.
+//
+// Bit matrix (units that overflowed their record pool, or every unit when the caller passes no pool).
+// One pair of CTAs per row span and slot; a slot walks the listed units with its fixed span.  Sixteen
+// epilogue warps in two teams of eight; team e serves TMEM stage e, i.e. every other tile.  Inside a
+// team a warp owns a 32-row strip and half of the tile's columns.  Direct words are staged in shared
+// memory and leave in 32-byte pieces, two per row, after the team's two tiles of a four-tile span (the
+// two warps of a strip meet for that); a 32x32 bit transpose across the warp turns the words of a
+// sub-block into the words of the mirrored rows, which are staged too and written 16 bytes per row by
+// the whole team.  Nothing but bits leaves the SM: N*N/8 bytes per unit, plus one bit per (row,
+// 64-column chunk) that says whether the chunk may hold a set bit (0: certainly empty), so that the
+// next kernel reads only the occupied part of a sparse graph.  The flags of 32 consecutive rows and
+// one chunk form a word (`flags[row / 32][chunk]`) with exactly one writer: the rows' own block for
+// chunks at or right of the block's own columns, the block that mirrors into the rows for chunks left
+// of them.  The caller clears the flag words; only words with a set bit are written.
 #include <algorithm>
 
 #include "common.cuh"
@@ -331,7 +338,6 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kSimThreads, 1) sim_
     if (lane == 0 && rank == 0) {
       const int me = warp == 1 ? 0 : 1;
       constexpr uint32_t idesc_neg = ptx::idesc_bf16_f32(2 * kBM, kBN, true);
-      constexpr uint32_t idesc_pos = ptx::idesc_bf16_f32(2 * kBM, kBN, false);
       int base = 0, ua = 0;
       bool ok = true;
       for (int i = item0; ok && i < n_items; i += item_step) {
@@ -356,8 +362,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kSimThreads, 1) sim_
               uint64_t db = ptx::smem_desc_sw128(b_addr + kh * kBH * 128 + kk * 32);
               umma_bf16_pair(tmem_base + me * kBN, da, db, idesc_neg, kk16 > 0 ? 1u : 0u);
             }
-            // + theta * |a| * |b|
-            umma_bf16_pair(tmem_base + me * kBN, dea, ptx::smem_desc_sw32(ptx::smem_u32(sEB + st * L::EB_BYTES)), idesc_pos, 1u);
+            // + theta * |a| * |b|: the threshold rows of operand A are stored negated, so the same descriptor serves
+            // (a change of descriptor between MMAs cost about twenty cycles each time)
+            umma_bf16_pair(tmem_base + me * kBN, dea, ptx::smem_desc_sw32(ptx::smem_u32(sEB + st * L::EB_BYTES)), idesc_neg, 1u);
             *turn = gi + 1;                   // the other thread may issue the next tile
             umma_commit_pair(b_empty + st);   // both CTAs: the stage may be refilled
             umma_commit_pair(acc_full + me);  // both CTAs: accumulator ready for the epilogue

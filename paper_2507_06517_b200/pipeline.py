@@ -23,8 +23,14 @@ class SpindleKVPass:
     """
 
     def __init__(self, cfg: B.Config, seq_lens: Sequence[int], dtype: torch.dtype, device="cuda",
-                 layers_per_codebook_call: Optional[int] = None, keep_adjacency: bool = False):
+                 layers_per_codebook_call: Optional[int] = None, keep_adjacency: bool = False,
+                 side_by_side: bool = True):
         self.cfg = cfg
+        # run(): the K CodeBooks, the V CodeBooks and the eviction are independent; on three streams the short
+        # kernels of one (norms, lists, cover, top-k, gathers: a block per unit, far from filling the device) run
+        # beside those of the others.  Costs a second CodeBook workspace.  Off when the adjacency is kept (one
+        # buffer for both calls).
+        self.side_by_side = side_by_side and not keep_adjacency
         self.seq_lens = [int(x) for x in seq_lens]
         self.dtype = dtype
         self.device = torch.device(device)
@@ -113,11 +119,38 @@ class SpindleKVPass:
     def run(self, K: torch.Tensor, V: torch.Tensor, Q: torch.Tensor, stream=None) -> None:
         """All layers of one prompt batch (``K``/``V`` hold every layer)."""
         ns = self.n_shallow
+        if self.side_by_side and ns:
+            return self._run_side_by_side(K, V, Q, stream)
         if self.n_deep:
             self.evict(K[ns:], V[ns:], Q, stream)
         if ns:
             self.codebook(K[:ns], "K", stream)
             self.codebook(V[:ns], "V", stream)
+
+    def _run_side_by_side(self, K, V, Q, stream=None) -> None:
+        """``run`` on three streams: K CodeBooks on the caller's stream, V CodeBooks and the eviction on two side
+        streams that start after the work already queued on the caller's stream and are joined before returning."""
+        dev, ns = self.device, self.n_shallow
+        cur = stream if stream is not None else torch.cuda.current_stream(dev)
+        if not hasattr(self, "_side"):
+            self._side = [torch.cuda.Stream(dev) for _ in range(2)]
+            self._ws_codebook_v = torch.empty_like(self.ws_codebook)
+        sV, sE = self._side
+        ev = torch.cuda.Event()
+        ev.record(cur)
+        sV.wait_event(ev)
+        self.codebook(K[:ns], "K", cur)
+        ws = self.ws_codebook
+        self.ws_codebook = self._ws_codebook_v
+        try:
+            self.codebook(V[:ns], "V", sV)
+        finally:
+            self.ws_codebook = ws
+        if self.n_deep:
+            sE.wait_event(ev)
+            self.evict(K[ns:], V[ns:], Q, sE)
+            cur.wait_stream(sE)
+        cur.wait_stream(sV)
 
     # -- the same pass fed from host memory ----------------------------------------------------
     def host_outputs(self) -> Dict[str, torch.Tensor]:
@@ -222,6 +255,8 @@ class SpindleKVPass:
             out["evict"] = B.spindlekv_poll_status(self.ws_evict)
         if self.n_shallow:
             out["codebook"] = B.spindlekv_poll_status(self.ws_codebook)
+            if hasattr(self, "_ws_codebook_v"):   # the V call of the last side-by-side run
+                out["codebook_v"] = B.spindlekv_poll_status(self._ws_codebook_v)
         return out
 
 

@@ -182,6 +182,49 @@ def test_host_fed_pass_equals_resident_pass():
                 assert torch.equal(out["V_kept"][li, 0, j, :m], p.V_kept.cpu()[li, 0, j, :m])
 
 
+def test_three_streams_give_what_one_stream_gives():
+    # run() puts the K CodeBooks, the V CodeBooks and the eviction on three streams (two CodeBook workspaces);
+    # every output must equal that of the three calls one after the other on one stream
+    wl = synth.Workload("streams", 6, 3, 8, 2, 128, "bf16", 32, (700, 1300, 420), 30, (0.05, 0.3), 2, "recency",
+                        budget_frac=0.3, seed=43)
+    host = generate(wl)
+    layers = list(range(wl.n_layers))
+    K, V = stack_layers(wl, host, layers, "K"), stack_layers(wl, host, layers, "V")
+    Q = stack_layers(wl, host, layers[wl.n_shallow:], "Q")
+    serial = _pass(wl)
+    serial.side_by_side = False
+    serial.run(K, V, Q)
+    side = _pass(wl)
+    assert side.side_by_side
+    for _ in range(2):   # the second run reuses the side streams and the second workspace
+        side.run(K, V, Q)
+        st = side.device_status()
+        assert st["evict"][0] == 0 and st["codebook"][0] == 0 and st["codebook_v"][0] == 0
+        for g in ("K", "V"):
+            n = serial.cb[g]["n_entries"].cpu()
+            assert torch.equal(side.cb[g]["n_entries"].cpu(), n)
+            assert torch.equal(side.cb[g]["ref"], serial.cb[g]["ref"])
+            assert torch.equal(side.cb[g]["mag"], serial.cb[g]["mag"])
+            cu = synth.cu_seqlens(wl)
+            for li in range(wl.n_shallow):
+                for s_ in range(len(wl.seq_lens)):
+                    for j in range(wl.n_kv_heads):
+                        m = int(n[li, s_, j])
+                        a, b = int(cu[s_]), int(cu[s_]) + m
+                        assert torch.equal(side.cb[g]["centre_idx"][li, j, a:b], serial.cb[g]["centre_idx"][li, j, a:b])
+                        assert torch.equal(side.cb[g]["C"][li, a:b, j], serial.cb[g]["C"][li, a:b, j])
+        assert torch.equal(side.keep_cnt, serial.keep_cnt)
+        cnt = serial.keep_cnt.cpu()
+        for li in range(wl.n_layers - wl.n_shallow):
+            for s_ in range(len(wl.seq_lens)):
+                for j in range(wl.n_kv_heads):
+                    m = int(cnt[li, s_, j])
+                    a, b = int(cu[s_]), int(cu[s_]) + m
+                    assert torch.equal(side.keep_idx[li, j, a:b], serial.keep_idx[li, j, a:b])
+                    assert torch.equal(side.K_kept[li, a:b, j], serial.K_kept[li, a:b, j])
+                    assert torch.equal(side.V_kept[li, a:b, j], serial.V_kept[li, a:b, j])
+
+
 def test_composition_as_written_evict_then_codebooks_of_the_kept_tokens():
     # every layer evicts under the pyramid over all layers, then builds K and V CodeBooks of what it kept
     # (different counts per layer, passed to the CodeBook call as per-layer lengths)
