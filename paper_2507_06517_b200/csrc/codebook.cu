@@ -746,16 +746,18 @@ static size_t cover_smem_bytes(int row_words) {
 // a counting sort on the degree, stable in the index.  hist[] lives in dynamic shared memory.
 // Centres of degree 1 are placed by all threads (ballots and a block scan); centres of larger degree by
 // one warp that walks, in index order, only the 32-token chunks that hold one.
-constexpr int kFinalThreads = 1024;
+constexpr int kFinalThreads = 512;     // two blocks fit an SM: the K and the V call of a pass run side by side
+constexpr int kFinalWarps = kFinalThreads / 32;
 constexpr int kFinalBatch = 16;        // tokens per thread loaded together
 constexpr int kFinalChunkWords = 64;   // chunk map for 64 * 32 * 32 = 65536 tokens (longer sequences: every chunk is visited)
 
-__global__ void __launch_bounds__(kFinalThreads) finalize_kernel(CodebookParams p) {
+__global__ void __launch_bounds__(kFinalThreads, 2) finalize_kernel(CodebookParams p) {
   extern __shared__ int hist[];  // [l + 2]
   __shared__ int warp_sums[33];
   __shared__ uint32_t busy[kFinalChunkWords];   // bit per 32-token chunk: holds a centre of pick degree >= 2
   __shared__ uint16_t busy_list[kFinalChunkWords * 32];
-  __shared__ int cnt_sh[kFinalBatch * 32];
+  __shared__ int cnt_sh[kFinalBatch * kFinalWarps];
+  static_assert(kFinalBatch * kFinalWarps <= kFinalThreads, "one thread per count in the scan");
   const int unit = blockIdx.x;
   int layer, s, j;
   cb_decode(p, unit, layer, s, j);
@@ -828,22 +830,22 @@ __global__ void __launch_bounds__(kFinalThreads) finalize_kernel(CodebookParams 
 #pragma unroll
       for (int i = 0; i < kFinalBatch; ++i) {
         ones[i] = __ballot_sync(0xffffffffu, dr[i] == 1);
-        if (lane == 0) cnt_sh[i * 32 + (tid >> 5)] = __popc(ones[i]);   // in token order: sweep i, warp w
+        if (lane == 0) cnt_sh[i * kFinalWarps + (tid >> 5)] = __popc(ones[i]);   // in token order: sweep i, warp w
       }
       __syncthreads();
       int tot;
       {
-        // exclusive scan of the kFinalBatch * 32 counts (entries beyond them count 0)
-        const int v = tid < kFinalBatch * 32 ? cnt_sh[tid] : 0;
+        // exclusive scan of the kFinalBatch * kFinalWarps counts (threads beyond them count 0)
+        const int v = tid < kFinalBatch * kFinalWarps ? cnt_sh[tid] : 0;
         const int ex = block_exclusive_scan(v, warp_sums, tot);
-        if (tid < kFinalBatch * 32) cnt_sh[tid] = ex;
+        if (tid < kFinalBatch * kFinalWarps) cnt_sh[tid] = ex;
         __syncthreads();
       }
 #pragma unroll
       for (int i = 0; i < kFinalBatch; ++i) {
         if (dr[i] == 1) {
           const int u = base0 + i * kFinalThreads + tid;
-          const int pos = before + cnt_sh[i * 32 + (tid >> 5)] + __popc(ones[i] & ((1u << lane) - 1u));
+          const int pos = before + cnt_sh[i * kFinalWarps + (tid >> 5)] + __popc(ones[i] & ((1u << lane) - 1u));
           rank[u] = pos;
           p.centre_idx[orow + pos] = u;
         }

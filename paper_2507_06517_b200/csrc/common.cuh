@@ -146,7 +146,7 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int* warp_sums, int& 
   if (lane == 31) warp_sums[wid] = inc;
   __syncthreads();
   if (wid == 0) {
-    int ws = warp_sums[lane];
+    int ws = lane < (int)((blockDim.x + 31) >> 5) ? warp_sums[lane] : 0;   // blocks of fewer than 32 warps
     int winc = ws;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
