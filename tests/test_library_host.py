@@ -155,21 +155,23 @@ def test_allocation_free_entry_point_checks_its_arguments_like_the_ordinary_one(
 
 def test_limits_can_be_tightened_and_restored():
     from paper_2507_06517_b200 import binding as B
-    defaults = [B.spindlekv_get_tuning(k) for k in range(3)]
-    assert defaults[B.TUNE_RECORDS_PER_TILE] == 512
+    defaults = [B.spindlekv_get_tuning(k) for k in range(4)]
+    assert defaults[B.TUNE_RECORDS_PER_TILE] == 512 and defaults[B.TUNE_SIM_BLOCK_PAIRS] == 0
     try:
         B.spindlekv_set_tuning(B.TUNE_RECORDS_PER_TILE, 7)
         B.spindlekv_set_tuning(B.TUNE_GREEDY_ROUND_CAP, 1)
         assert B.spindlekv_get_tuning(B.TUNE_RECORDS_PER_TILE) == 7 and B.spindlekv_get_tuning(B.TUNE_GREEDY_ROUND_CAP) == 1
+        B.spindlekv_set_tuning(B.TUNE_SIM_BLOCK_PAIRS, 3)
+        assert B.spindlekv_get_tuning(B.TUNE_SIM_BLOCK_PAIRS) == 3
         B.spindlekv_set_tuning(B.TUNE_RECORDS_PER_TILE, 100000)      # never above what the workspace is sized for
         assert B.spindlekv_get_tuning(B.TUNE_RECORDS_PER_TILE) == 512
         with pytest.raises(B.SpindleKVError):
             B.spindlekv_set_tuning(99, 1)
         assert B.spindlekv_get_tuning(99) == -1
     finally:
-        for k in range(3):
+        for k in range(4):
             B.spindlekv_set_tuning(k, -1)
-    assert [B.spindlekv_get_tuning(k) for k in range(3)] == defaults
+    assert [B.spindlekv_get_tuning(k) for k in range(4)] == defaults
     # the self-tests check their arguments before launching anything
     assert B._lib.spindlekv_selftest_mbarrier_timeout(None, 100, None) == B.INVALID_ARG
     assert B._lib.spindlekv_selftest_mbarrier_timeout(256, 0, None) == B.INVALID_ARG
