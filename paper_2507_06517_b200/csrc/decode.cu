@@ -7,13 +7,16 @@
 // One unit is (layer, sequence, KV head); the h_n query heads of its GQA group are served together, so a
 // key is rebuilt and rotated once for all of them.  A unit's tokens are split into chunks of kDecChunk;
 // one block per (chunk, unit):
-//   1. scores: 16 threads per token gather the token's CodeBook row (16-byte pieces), scale it by the
-//      token's magnitude, rotate it, and form the dot products with the rotated queries (kept in shared
-//      memory); the 16 partial sums meet through shuffles.  Scores of the chunk stay in shared memory.
-//   2. the chunk's maximum and exp-sum per query head (fixed-order block reductions);
-//   3. values: every thread owns one pair of output elements for all query heads and a share of the chunk's
-//      tokens, adding weight * magnitude * CodeBook row; the row pieces of a token are read by consecutive
-//      threads, once for the whole group; the shares are then added up in a fixed order.
+//   0. the chunk's references, magnitudes and positions are copied into shared memory, so that no row load
+//      waits for the load of its own address;
+//   1. scores: 16 threads per token gather the token's CodeBook row, scale it by the token's magnitude, rotate
+//      it, and form the dot products with the rotated queries (each thread's part of them in registers); the
+//      16 partial sums meet through shuffles.  Scores of the chunk stay in shared memory.
+//   2. the chunk's maximum and exp-sum per query head (fixed-order reductions);
+//   3. values: a 16-byte piece of a CodeBook row per thread and token (the threads of a row side by side, the
+//      chunk's tokens dealt out over the rows of threads), weight * magnitude * piece added for all query heads
+//      at once; the partial sums meet by shuffles inside a warp and through shared memory across warps, in a
+//      fixed order.
 // A second kernel merges the chunks of a unit (log-sum-exp weights) in chunk order.  All sums run in a
 // fixed order: the result is bit-reproducible from run to run.
 #include <math_constants.h>
@@ -67,9 +70,58 @@ __device__ __forceinline__ void load_row_piece(const T* p, float (&out)[N]) {
   }
 }
 
+// Sum of acc[g] over the 16 threads of a token, for all HN heads at once: at every step a thread keeps half of its
+// values and hands the other half to its partner, so HN heads cost HN - 1 + (4 - log2 HN) shuffles instead of
+// 4 HN.  Returns the total of head `head` in the threads whose low 4 - log2(HN) bits of `sub` are zero (all
+// threads of the token hold some head's total; those are the ones that store it).  Fixed order of additions.
+template <int HN>
+__device__ __forceinline__ float reduce_heads(const float (&acc)[HN], int sub, int& head) {
+  float v[HN];
+#pragma unroll
+  for (int g = 0; g < HN; ++g) v[g] = acc[g];
+  head = 0;
+  int n = HN;
+#pragma unroll
+  for (int bit = 8; bit >= 1; bit >>= 1) {
+    if (n > 1) {
+      const bool up = (sub & bit) != 0;
+      const int half = n >> 1;
+#pragma unroll
+      for (int i = 0; i < HN / 2; ++i) {
+        if (i < half) {
+          const float keep = up ? v[half + i] : v[i];
+          const float send = up ? v[i] : v[half + i];
+          v[i] = keep + __shfl_xor_sync(0xffffffffu, send, bit);
+        }
+      }
+      head += up ? half : 0;
+      n = half;
+    } else {
+      v[0] += __shfl_xor_sync(0xffffffffu, v[0], bit);
+    }
+  }
+  return v[0];
+}
+
+template <int HN>
+__device__ __forceinline__ void load_heads(const float* p, float (&w)[HN]) {
+  if constexpr (HN == 1) {
+    w[0] = p[0];
+  } else if constexpr (HN == 2) {
+    const float2 v = *reinterpret_cast<const float2*>(p);
+    w[0] = v.x; w[1] = v.y;
+  } else {
+#pragma unroll
+    for (int i = 0; i < HN; i += 4) {
+      const float4 v = *reinterpret_cast<const float4*>(p + i);
+      w[i] = v.x; w[i + 1] = v.y; w[i + 2] = v.z; w[i + 3] = v.w;
+    }
+  }
+}
+
 // HN: query heads per KV head the instantiation is unrolled for (the group's actual size h_n <= HN)
 template <typename T, int D, int HN>
-__global__ void __launch_bounds__(kDecThreads) decode_chunk_kernel(DecodeParams p) {
+__global__ void __launch_bounds__(kDecThreads, HN <= 4 ? 4 : 2) decode_chunk_kernel(DecodeParams p) {
   constexpr int H = D / 2;            // rotation pairs
   constexpr int PPT = D / 32;         // pairs per thread of a 16-thread token group
   extern __shared__ float sm[];
@@ -90,10 +142,14 @@ __global__ void __launch_bounds__(kDecThreads) decode_chunk_kernel(DecodeParams 
   }
   const int nt = min(kDecChunk, n - t0);
   float* sq = sm;                                 // [h_n][D] rotated queries
-  float* sc = sq + kDecMaxGroup * D;              // [h_n][kDecChunk] scores, then weights
-  int32_t* srv = reinterpret_cast<int32_t*>(sc + kDecMaxGroup * kDecChunk);   // [kDecChunk] value references
+  float* sc = sq + h_n * D;                       // [kDecChunk][HN] scores, then weights (a token's heads side by side)
+  int32_t* srv = reinterpret_cast<int32_t*>(sc + HN * kDecChunk);             // [kDecChunk] value references
   float* smv = reinterpret_cast<float*>(srv + kDecChunk);                     // [kDecChunk] value magnitudes
-  float* red = smv + kDecChunk;                   // [kDecMaxGroup][8] reduction scratch
+  int32_t* srk = reinterpret_cast<int32_t*>(smv + kDecChunk);                 // [kDecChunk] key references
+  float* smk = reinterpret_cast<float*>(srk + kDecChunk);                     // [kDecChunk] key magnitudes
+  int32_t* spos = reinterpret_cast<int32_t*>(smk + kDecChunk);                // [kDecChunk] positions, clamped to the table
+  float* red = reinterpret_cast<float*>(spos + kDecChunk);                    // [2][warps][HN] reduction scratch
+  float* ps = red + 2 * kDecMaxGroup * (kDecThreads / 32);             // [warps][h_n][D] partial value sums
   const int64_t orow = ((int64_t)layer * p.n_kv_heads + j) * p.batch.total_len + tok_base(p.batch, s);
   const T* ck = reinterpret_cast<const T*>(p.CK.ptr) + unit_offset(p.CK, p.batch, layer, s, j);
   const T* cv = reinterpret_cast<const T*>(p.CV.ptr) + unit_offset(p.CV, p.batch, layer, s, j);
@@ -114,147 +170,207 @@ __global__ void __launch_bounds__(kDecThreads) decode_chunk_kernel(DecodeParams 
   for (int t = tid; t < nt; t += kDecThreads) {
     srv[t] = p.ref_v[orow + t0 + t];
     smv[t] = p.mag_v[orow + t0 + t];
+    srk[t] = p.ref_k[orow + t0 + t];
+    smk[t] = p.mag_k[orow + t0 + t];
+    spos[t] = min(max(p.positions ? p.positions[orow + t0 + t] : t0 + t, 0), p.table_positions - 1);
   }
   __syncthreads();
   // ---- 1. scores: two tokens per 16-thread group and sweep, all their loads in flight before any is used ----
   {
     constexpr int kTok = 2;
     const int sub = tid & 15, grp = tid >> 4;     // 16 token groups per sweep
-    // this thread's part of the rotated queries stays in registers for the whole chunk
-    float qlo[HN][PPT], qhi[HN][PPT];
+    // this thread's part of the rotated queries stays in registers for the whole chunk, two pairs to a register
+    // pair: the arithmetic below is packed (two fp32 lanes per instruction)
+    static_assert(PPT % 2 == 0, "pairs are handled two at a time");
+    float2 qlo[HN][PPT / 2], qhi[HN][PPT / 2];
 #pragma unroll
     for (int g = 0; g < HN; ++g)
 #pragma unroll
-      for (int k = 0; k < PPT; ++k) {
-        qlo[g][k] = g < h_n ? sq[g * D + sub * PPT + k] : 0.f;
-        qhi[g][k] = g < h_n ? sq[g * D + H + sub * PPT + k] : 0.f;
+      for (int k = 0; k < PPT / 2; ++k) {
+        const float* q0 = sq + g * D + sub * PPT + 2 * k;
+        qlo[g][k] = g < h_n ? make_float2(q0[0], q0[1]) : make_float2(0.f, 0.f);
+        qhi[g][k] = g < h_n ? make_float2(q0[H], q0[H + 1]) : make_float2(0.f, 0.f);
       }
     for (int tb = 0; tb < nt; tb += kTok * (kDecThreads / 16)) {
       float lo[kTok][PPT], hi[kTok][PPT], m[kTok];
-      float2 cs[kTok][PPT];
+      float4 cs[kTok][PPT / 2];          // (cos, sin) of two pairs
       int tk[kTok];
 #pragma unroll
       for (int x = 0; x < kTok; ++x) {
         const int t = tb + x * (kDecThreads / 16) + grp;
         tk[x] = t;
         const bool has = t < nt;
-        const int r = has ? p.ref_k[orow + t0 + t] : 0;
-        m[x] = has ? p.mag_k[orow + t0 + t] : 0.f;
-        const int pos = (has && p.positions) ? p.positions[orow + t0 + t] : t0 + t;
-        const float2* tab = p.table + (int64_t)min(max(pos, 0), p.table_positions - 1) * H + sub * PPT;
+        const int r = has ? srk[t] : 0;
+        m[x] = has ? smk[t] : 0.f;
+        const float2* tab = p.table + (int64_t)(has ? spos[t] : 0) * H + sub * PPT;
         const T* row = ck + (int64_t)r * p.CK.st;
         load_row_piece<T, PPT>(row + sub * PPT, lo[x]);
         load_row_piece<T, PPT>(row + H + sub * PPT, hi[x]);
 #pragma unroll
-        for (int k = 0; k < PPT; k += 2) {
-          const float4 v = *reinterpret_cast<const float4*>(tab + k);
-          cs[x][k] = make_float2(v.x, v.y);
-          cs[x][k + 1] = make_float2(v.z, v.w);
-        }
+        for (int k = 0; k < PPT / 2; ++k) cs[x][k] = *reinterpret_cast<const float4*>(tab + 2 * k);
       }
 #pragma unroll
       for (int x = 0; x < kTok; ++x) {
-        float acc[HN];
+        float2 acc2[HN];
 #pragma unroll
-        for (int g = 0; g < HN; ++g) acc[g] = 0.f;
+        for (int g = 0; g < HN; ++g) acc2[g] = make_float2(0.f, 0.f);
+        const float2 m2 = make_float2(m[x], m[x]);
 #pragma unroll
-        for (int k = 0; k < PPT; ++k) {
-          const float a = lo[x][k] * m[x], b = hi[x][k] * m[x];               // Eq. (14)
-          const float ra = a * cs[x][k].x - b * cs[x][k].y, rb = b * cs[x][k].x + a * cs[x][k].y;
+        for (int k = 0; k < PPT / 2; ++k) {
+          const float2 c2 = make_float2(cs[x][k].x, cs[x][k].z), s2 = make_float2(cs[x][k].y, cs[x][k].w);
+          const float2 a2 = __fmul2_rn(make_float2(lo[x][2 * k], lo[x][2 * k + 1]), m2);    // Eq. (14)
+          const float2 b2 = __fmul2_rn(make_float2(hi[x][2 * k], hi[x][2 * k + 1]), m2);
+          // (a, b) -> (a cos - b sin, b cos + a sin)
+          const float2 ra = __ffma2_rn(make_float2(-b2.x, -b2.y), s2, __fmul2_rn(a2, c2));
+          const float2 rb = __ffma2_rn(a2, s2, __fmul2_rn(b2, c2));
 #pragma unroll
           for (int g = 0; g < HN; ++g)
-            if (g < h_n) acc[g] = fmaf(qlo[g][k], ra, fmaf(qhi[g][k], rb, acc[g]));
+            if (g < h_n) acc2[g] = __ffma2_rn(qlo[g][k], ra, __ffma2_rn(qhi[g][k], rb, acc2[g]));
         }
+        float acc[HN];
 #pragma unroll
-        for (int g = 0; g < HN; ++g) {
-          if (g < h_n) {
-#pragma unroll
-            for (int o = 8; o >= 1; o >>= 1) acc[g] += __shfl_xor_sync(0xffffffffu, acc[g], o);
-            if (sub == 0 && tk[x] < nt) sc[g * kDecChunk + tk[x]] = acc[g] * p.scale;
-          }
-        }
+        for (int g = 0; g < HN; ++g) acc[g] = acc2[g].x + acc2[g].y;
+        int head;
+        const float total = reduce_heads<HN>(acc, sub, head);
+        if ((sub & (16 / HN - 1)) == 0 && head < h_n && tk[x] < nt) sc[tk[x] * HN + head] = total * p.scale;
       }
     }
   }
   __syncthreads();
-  // ---- 2. maximum and exp-sum per query head: warp w of eight takes head w (and w + 8 never: h_n <= 8) ----
+  // ---- 2. maximum and exp-sum per query head: a thread takes every kDecThreads-th token with all its heads; the
+  // partial results meet by shuffles inside a warp and through shared memory across the warps, in a fixed order ----
   {
     const int w = tid >> 5, lane = tid & 31;
-    if (w < h_n) {
-      float mx = -CUDART_INF_F;
-      for (int t = lane; t < nt; t += 32) mx = fmaxf(mx, sc[w * kDecChunk + t]);
+    constexpr int NW = kDecThreads / 32;
+    float mx[HN];
 #pragma unroll
-      for (int o = 16; o >= 1; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-      float sum = 0.f;
-      for (int t = lane; t < nt; t += 32) {
-        const float e = expf(sc[w * kDecChunk + t] - mx);
-        sc[w * kDecChunk + t] = e * smv[t];          // weight of the CodeBook row: probability share times magnitude
-        sum += e;
-      }
+    for (int g = 0; g < HN; ++g) mx[g] = -CUDART_INF_F;
+    for (int t = tid; t < nt; t += kDecThreads) {
+      float v[HN];
+      load_heads<HN>(sc + t * HN, v);
 #pragma unroll
-      for (int o = 16; o >= 1; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-      if (lane == 0) {
-        red[w * 2] = mx;
-        red[w * 2 + 1] = sum;
+      for (int g = 0; g < HN; ++g) mx[g] = fmaxf(mx[g], v[g]);
+    }
+#pragma unroll
+    for (int g = 0; g < HN; ++g) {
+#pragma unroll
+      for (int o = 16; o >= 1; o >>= 1) mx[g] = fmaxf(mx[g], __shfl_xor_sync(0xffffffffu, mx[g], o));
+      if (lane == 0) red[w * HN + g] = mx[g];
+    }
+    __syncthreads();
+#pragma unroll
+    for (int g = 0; g < HN; ++g) {
+      float v = red[g];
+#pragma unroll
+      for (int q = 1; q < NW; ++q) v = fmaxf(v, red[q * HN + g]);
+      mx[g] = v;
+    }
+    float sum[HN];
+#pragma unroll
+    for (int g = 0; g < HN; ++g) sum[g] = 0.f;
+    for (int t = tid; t < nt; t += kDecThreads) {
+      float v[HN];
+      load_heads<HN>(sc + t * HN, v);
+      const float mv = smv[t];
+#pragma unroll
+      for (int g = 0; g < HN; ++g) {
+        const float e = g < h_n ? expf(v[g] - mx[g]) : 0.f;
+        sum[g] += e;
+        sc[t * HN + g] = e * mv;                   // weight of the CodeBook row: probability share times magnitude
       }
+    }
+#pragma unroll
+    for (int g = 0; g < HN; ++g) {
+#pragma unroll
+      for (int o = 16; o >= 1; o >>= 1) sum[g] += __shfl_xor_sync(0xffffffffu, sum[g], o);
+      if (lane == 0) red[kDecMaxGroup * NW + w * HN + g] = sum[g];
+    }
+    __syncthreads();
+    if (tid < h_n) {
+      float vm = red[tid], v = 0.f;
+#pragma unroll
+      for (int q = 1; q < NW; ++q) vm = fmaxf(vm, red[q * HN + tid]);
+#pragma unroll
+      for (int q = 0; q < NW; ++q) v += red[kDecMaxGroup * NW + q * HN + tid];     // fixed order
+      part[tid * (D + 2)] = vm;
+      part[tid * (D + 2) + 1] = v;
     }
   }
-  __syncthreads();
-  // ---- 3. values: a thread owns one pair of output elements for all query heads and every kParts-th token, so a
-  // CodeBook row piece is loaded once for the whole group; the kParts partial sums meet in shared memory ----
+  // ---- 3. values: TPR threads side by side read a CodeBook row in 16-byte pieces, once for the whole group; the
+  // chunk's tokens are dealt out over the kDecThreads / TPR rows of threads ----
   {
-    constexpr int kParts = kDecThreads / H;
-    constexpr int kUnroll = 8;
-    const int pr = tid % H, tq = tid / H;
-    float o[HN][2];
-#pragma unroll
-    for (int g = 0; g < HN; ++g) o[g][0] = o[g][1] = 0.f;
-    for (int tb = tq; tb < nt; tb += kParts * kUnroll) {
-      float x[kUnroll][2];
-#pragma unroll
-      for (int i = 0; i < kUnroll; ++i) {
-        const int t = tb + i * kParts;
-        const int r = t < nt ? srv[t] : 0;
-        if constexpr (sizeof(T) == 4) {
-          const float2 v = *reinterpret_cast<const float2*>(cv + (int64_t)r * p.CV.st + 2 * pr);
-          x[i][0] = v.x; x[i][1] = v.y;
-        } else {
-          const uint32_t v = *reinterpret_cast<const uint32_t*>(cv + (int64_t)r * p.CV.st + 2 * pr);
-          x[i][0] = __uint_as_float(v << 16); x[i][1] = __uint_as_float(v & 0xFFFF0000u);
-        }
-      }
-#pragma unroll
-      for (int i = 0; i < kUnroll; ++i) {
-        const int t = tb + i * kParts;
-        if (t >= nt) continue;
-#pragma unroll
-        for (int g = 0; g < HN; ++g)
-          if (g < h_n) {
-            const float wv = sc[g * kDecChunk + t];
-            o[g][0] = fmaf(wv, x[i][0], o[g][0]);
-            o[g][1] = fmaf(wv, x[i][1], o[g][1]);
-          }
-      }
-    }
-    __syncthreads();                         // every thread is done with the weights: their place takes the partial sums
-    float* ps = sc;                          // [kParts][h_n][D]
+    constexpr int EPT = 16 / (int)sizeof(T);     // elements per piece
+    constexpr int TPR = D / EPT;                 // threads per row
+    constexpr int G = kDecThreads / TPR;         // rows of threads
+    constexpr int kUnroll = 4;
+    static_assert(TPR <= 32 && 32 % TPR == 0, "a row of threads lies inside a warp");
+    const int sub = tid % TPR, grp = tid / TPR;
+    float2 o[HN][EPT / 2];
 #pragma unroll
     for (int g = 0; g < HN; ++g)
-      if (g < h_n) {
-        ps[(tq * h_n + g) * D + 2 * pr] = o[g][0];
-        ps[(tq * h_n + g) * D + 2 * pr + 1] = o[g][1];
+#pragma unroll
+      for (int e = 0; e < EPT / 2; ++e) o[g][e] = make_float2(0.f, 0.f);
+    for (int tb = grp; tb < nt; tb += G * kUnroll) {
+      uint4 raw[kUnroll];
+#pragma unroll
+      for (int i = 0; i < kUnroll; ++i) {
+        const int t = tb + i * G;
+        const int r = t < nt ? srv[t] : 0;
+        raw[i] = *reinterpret_cast<const uint4*>(cv + (int64_t)r * p.CV.st + sub * EPT);
       }
+#pragma unroll
+      for (int i = 0; i < kUnroll; ++i) {
+        const int t = tb + i * G;
+        if (t >= nt) continue;
+        float x[EPT];
+        if constexpr (sizeof(T) == 4) {
+          x[0] = __uint_as_float(raw[i].x); x[1] = __uint_as_float(raw[i].y);
+          x[2] = __uint_as_float(raw[i].z); x[3] = __uint_as_float(raw[i].w);
+        } else {
+          const uint32_t w4[4] = {raw[i].x, raw[i].y, raw[i].z, raw[i].w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            x[2 * e] = __uint_as_float(w4[e] << 16);
+            x[2 * e + 1] = __uint_as_float(w4[e] & 0xFFFF0000u);
+          }
+        }
+        float wv[HN];
+        load_heads<HN>(sc + t * HN, wv);
+#pragma unroll
+        for (int g = 0; g < HN; ++g) {
+          const float2 w2 = make_float2(wv[g], wv[g]);
+#pragma unroll
+          for (int e = 0; e < EPT / 2; ++e) o[g][e] = __ffma2_rn(w2, make_float2(x[2 * e], x[2 * e + 1]), o[g][e]);
+        }
+      }
+    }
+    // the rows of threads of a warp first (lanes that hold the same piece), then the warps in order
+#pragma unroll
+    for (int off = TPR; off < 32; off <<= 1)
+#pragma unroll
+      for (int g = 0; g < HN; ++g)
+#pragma unroll
+        for (int e = 0; e < EPT / 2; ++e) {
+          o[g][e].x += __shfl_xor_sync(0xffffffffu, o[g][e].x, off);
+          o[g][e].y += __shfl_xor_sync(0xffffffffu, o[g][e].y, off);
+        }
+    const int wp = tid >> 5, lane = tid & 31;
+    if (lane < TPR) {
+#pragma unroll
+      for (int g = 0; g < HN; ++g)
+        if (g < h_n) {
+#pragma unroll
+          for (int e = 0; e < EPT / 2; ++e)
+            *reinterpret_cast<float2*>(ps + (wp * h_n + g) * D + sub * EPT + 2 * e) = o[g][e];
+        }
+    }
     __syncthreads();
     for (int i = tid; i < h_n * D; i += kDecThreads) {
       float sum = 0.f;
 #pragma unroll
-      for (int q = 0; q < kParts; ++q) sum += ps[q * h_n * D + i];   // fixed order
+      for (int q = 0; q < kDecThreads / 32; ++q) sum += ps[q * h_n * D + i];   // fixed order
       part[(i / D) * (D + 2) + 2 + (i % D)] = sum;
     }
-  }
-  if (tid < h_n) {
-    part[tid * (D + 2)] = red[tid * 2];
-    part[tid * (D + 2) + 1] = red[tid * 2 + 1];
   }
 }
 
@@ -307,8 +423,10 @@ size_t decode_workspace_bytes(const spindlekv_batch& b, int n_q_heads, int n_kv_
   return align_up(units * chunks * (size_t)(n_q_heads / n_kv_heads) * (head_dim + 2) * sizeof(float), 256);
 }
 
-static size_t decode_smem_bytes(int head_dim) {
-  return (size_t)(kDecMaxGroup * head_dim + kDecMaxGroup * kDecChunk + 2 * kDecChunk + kDecMaxGroup * 8) * 4;
+// hn_slots: the group size the kernel instantiation is unrolled for (a token's scores take that many floats)
+static size_t decode_smem_bytes(int head_dim, int h_n, int hn_slots) {
+  // rotated queries, scores, five per-token arrays, reduction scratch, per-warp partial value sums
+  return (size_t)(h_n * head_dim + hn_slots * kDecChunk + 5 * kDecChunk + 2 * kDecMaxGroup * (kDecThreads / 32) + (kDecThreads / 32) * h_n * head_dim) * 4;
 }
 
 template <typename T, int D, int HN>
@@ -316,9 +434,9 @@ static spindlekv_status launch_decode_hn(const DecodeParams& p, int units, cudaS
   static PerDeviceOnce once;
   const int dev = PerDeviceOnce::current();
   if (dev < 0) return SPINDLEKV_CUDA;
-  const size_t smem = decode_smem_bytes(D);
+  const size_t smem = decode_smem_bytes(D, p.h_n, HN);
   if (!once.done[dev]) {
-    if (cudaFuncSetAttribute(decode_chunk_kernel<T, D, HN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+    if (cudaFuncSetAttribute(decode_chunk_kernel<T, D, HN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)decode_smem_bytes(D, HN, HN)) != cudaSuccess)
       return SPINDLEKV_CUDA;
     once.done[dev] = true;
   }

@@ -64,6 +64,29 @@ def test_decode_attention_over_codebooks_of_whole_sequences(dtype, d, tol):
     assert torch.equal(again, out)                       # fixed summation order: the same bits every time
 
 
+@pytest.mark.parametrize("d", [128, 64])
+def test_decode_attention_for_every_group_size(d):
+    # 1, 2, 3, 4 and 8 query heads per KV head: the kernel is unrolled for 1, 2, 4 and 8 (three heads run in the
+    # form for four with one slot idle) and sums a token's partial dot products for all heads of the group at once;
+    # one chunk plus a ragged second one
+    from paper_2507_06517_b200.pipeline import SpindleKVDecodeAttention, SpindleKVPass
+    wl = synth.Workload("decg", 1, 1, 16, 2, d, "bf16", 8, (700,), 60, (0.05, 0.3), 4, "gauss", budget_tokens=700.0, seed=103)
+    host = generate(wl)
+    p = SpindleKVPass(make_config(wl), wl.seq_lens, torch_dtype(wl))
+    K, V = stack_layers(wl, host, [0], "K"), stack_layers(wl, host, [0], "V")
+    p.run(K, V, None)
+    assert p.device_status()["codebook"][0] == 0
+    rng = np.random.default_rng(11)
+    pos_q = np.array([700], dtype=np.int32)
+    for h_n in (1, 2, 3, 4, 8):
+        hq = h_n * wl.n_kv_heads
+        q = torch.from_numpy(rng.standard_normal((1, 1, hq, 1, d)).astype(np.float32)).to(torch_dtype(wl)).cuda()
+        att = SpindleKVDecodeAttention(p.cb_batch, hq, wl.n_kv_heads, d, 1024)
+        out = att.run(q, torch.from_numpy(pos_q).cuda(), p.cb["K"], p.cb["V"]).clone()
+        torch.cuda.synchronize()
+        _check(wl.replace(n_q_heads=hq), out, q, pos_q, p.cb["K"], p.cb["V"], None, 10000.0, 1e-2)
+
+
 def test_decode_attention_over_an_evicted_and_replaced_cache():
     # the composition as written: every layer keeps k + w tokens (different per layer) and replaces them; the cached
     # tokens keep their original positions (the kept indices), which the rotation must use
