@@ -300,17 +300,32 @@ class SpindleKVLiteralPass:
         if keep_adjacency:
             self.adj = torch.zeros((L * nB * H, self.max_keep, B.row_words(self.max_keep)), **i32)
 
-    def run(self, K: torch.Tensor, V: torch.Tensor, Q: torch.Tensor, which=("K", "V"), stream=None) -> None:
+    def _codebook(self, g: str, ws: torch.Tensor, stream) -> None:
         cfg = self.cfg
+        kept = (self.ev.K_kept if g == "K" else self.ev.V_kept)[:, :, :, : self.max_keep]
+        o = self.cb[g]
+        B.spindlekv_codebook_shallow(cfg, self.cb_batch, B.desc_bhnd(kept), cfg.theta_k if g == "K" else cfg.theta_v,
+                                     o["mag"], o["ref"], o["centre_idx"], o["n_entries"], ws, self.adj, stream)
+        B.spindlekv_compact(self.cb_batch, cfg.n_kv_heads, cfg.head_dim, B.desc_bhnd(kept), o["centre_idx"],
+                            o["n_entries"], B.desc_bhnd(o["C"]), o["mag"], None, stream)
+
+    def run(self, K: torch.Tensor, V: torch.Tensor, Q: torch.Tensor, which=("K", "V"), stream=None) -> None:
         self.ev.evict(K, V, Q, stream)
+        if self.adj is None and tuple(which) == ("K", "V"):
+            # the two CodeBook calls are independent: the V call runs on a side stream with a workspace of its own
+            cur = stream if stream is not None else torch.cuda.current_stream(self.device)
+            if not hasattr(self, "_side"):
+                self._side = torch.cuda.Stream(self.device)
+                self._ws_codebook_v = torch.empty_like(self.ws_codebook)
+            ev = torch.cuda.Event()
+            ev.record(cur)
+            self._side.wait_event(ev)
+            self._codebook("K", self.ws_codebook, cur)
+            self._codebook("V", self._ws_codebook_v, self._side)
+            cur.wait_stream(self._side)
+            return
         for g in which:
-            kept = (self.ev.K_kept if g == "K" else self.ev.V_kept)[:, :, :, : self.max_keep]
-            o = self.cb[g]
-            B.spindlekv_codebook_shallow(cfg, self.cb_batch, B.desc_bhnd(kept), cfg.theta_k if g == "K" else cfg.theta_v,
-                                         o["mag"], o["ref"], o["centre_idx"], o["n_entries"], self.ws_codebook,
-                                         self.adj, stream)
-            B.spindlekv_compact(self.cb_batch, cfg.n_kv_heads, cfg.head_dim, B.desc_bhnd(kept), o["centre_idx"],
-                                o["n_entries"], B.desc_bhnd(o["C"]), o["mag"], None, stream)
+            self._codebook(g, self.ws_codebook, stream)
 
     def entry_counts(self):
         """Host copies of the CodeBook sizes ``[L, B, H]`` for K and V (synchronises)."""
@@ -318,7 +333,10 @@ class SpindleKVLiteralPass:
 
     def device_status(self):
         torch.cuda.synchronize(self.device)
-        return {"evict": B.spindlekv_poll_status(self.ev.ws_evict), "codebook": B.spindlekv_poll_status(self.ws_codebook)}
+        out = {"evict": B.spindlekv_poll_status(self.ev.ws_evict), "codebook": B.spindlekv_poll_status(self.ws_codebook)}
+        if hasattr(self, "_ws_codebook_v"):
+            out["codebook_v"] = B.spindlekv_poll_status(self._ws_codebook_v)
+        return out
 
 
 class SpindleKVRepeatPass:
@@ -381,16 +399,31 @@ class SpindleKVRepeatPass:
         B.spindlekv_union_lists(L, self.n_seqs, H, self.keep_idx.view(L, H, self.h_n, -1),
                                 self.keep_cnt.view(L, self.n_seqs, H, self.h_n), self.max_len,
                                 self.union_idx, self.union_cnt, self.max_union, stream, lists_inner=True)
-        for g in which:
+        def codebook(g, ws, st):
             src, rep, o = (K if g == "K" else V), self.rep[g], self.cb[g]
             # rows of the union list, gathered from the KV head (the union list is laid out per max_union tokens,
             # the source per max_len tokens: two batches describe the two sides)
-            self._gather(src, rep, stream)
+            self._gather(src, rep, st)
             B.spindlekv_codebook_shallow(cfg, self.cb_batch, B.desc_bhnd(rep), cfg.theta_k if g == "K" else cfg.theta_v,
-                                         o["mag"], o["ref"], o["centre_idx"], o["n_entries"], self.ws_codebook,
-                                         self.adj, stream)
+                                         o["mag"], o["ref"], o["centre_idx"], o["n_entries"], ws, self.adj, st)
             B.spindlekv_compact(self.cb_batch, H, d, B.desc_bhnd(rep), o["centre_idx"], o["n_entries"],
-                                B.desc_bhnd(o["C"]), o["mag"], None, stream)
+                                B.desc_bhnd(o["C"]), o["mag"], None, st)
+
+        if self.adj is None and tuple(which) == ("K", "V"):
+            # the two CodeBook calls are independent: the V call runs on a side stream with a workspace of its own
+            cur = stream if stream is not None else torch.cuda.current_stream(self.device)
+            if not hasattr(self, "_side"):
+                self._side = torch.cuda.Stream(self.device)
+                self._ws_codebook_v = torch.empty_like(self.ws_codebook)
+            ev = torch.cuda.Event()
+            ev.record(cur)
+            self._side.wait_event(ev)
+            codebook("K", self.ws_codebook, cur)
+            codebook("V", self._ws_codebook_v, self._side)
+            cur.wait_stream(self._side)
+            return
+        for g in which:
+            codebook(g, self.ws_codebook, stream)
 
     def _gather(self, src: torch.Tensor, rep: torch.Tensor, stream=None) -> None:
         # index rows are [L][H][B * max_union]; the compaction call addresses source rows through the batch's
@@ -402,7 +435,10 @@ class SpindleKVRepeatPass:
 
     def device_status(self):
         torch.cuda.synchronize(self.device)
-        return {"evict": B.spindlekv_poll_status(self.ws_evict), "codebook": B.spindlekv_poll_status(self.ws_codebook)}
+        out = {"evict": B.spindlekv_poll_status(self.ws_evict), "codebook": B.spindlekv_poll_status(self.ws_codebook)}
+        if hasattr(self, "_ws_codebook_v"):
+            out["codebook_v"] = B.spindlekv_poll_status(self._ws_codebook_v)
+        return out
 
 
 class SpindleKVDecodeMerge:

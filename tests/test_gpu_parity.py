@@ -225,6 +225,35 @@ def test_three_streams_give_what_one_stream_gives():
                     assert torch.equal(side.V_kept[li, a:b, j], serial.V_kept[li, a:b, j])
 
 
+def test_side_stream_of_the_composition_as_written_changes_nothing():
+    # the literal and the repeat pass build the V CodeBooks on a side stream while the K CodeBooks are built on the
+    # caller's: same outputs as one Gamma after the other
+    from paper_2507_06517_b200.pipeline import SpindleKVLiteralPass, SpindleKVRepeatPass
+    wl = synth.Workload("lits", 3, -1, 8, 2, 128, "bf16", 32, (900, 900), 30, (0.05, 0.3), 2, "recency",
+                        budget_frac=0.3, seed=47)
+    host = generate(wl)
+    layers = list(range(wl.n_layers))
+    K, V, Q = (stack_layers(wl, host, layers, x) for x in ("K", "V", "Q"))
+    for cls in (SpindleKVLiteralPass, SpindleKVRepeatPass):
+        a = cls(make_config(wl), wl.seq_lens, torch_dtype(wl))
+        a.run(K, V, Q)                                   # K on the caller's stream, V on the side stream
+        st = a.device_status()
+        assert st["codebook"][0] == 0 and st["codebook_v"][0] == 0
+        b = cls(make_config(wl), wl.seq_lens, torch_dtype(wl))
+        b.run(K, V, Q, which=("K",))
+        b.run(K, V, Q, which=("V",))
+        torch.cuda.synchronize()
+        for g in ("K", "V"):
+            n = b.cb[g]["n_entries"].cpu()
+            assert torch.equal(a.cb[g]["n_entries"].cpu(), n)
+            assert torch.equal(a.cb[g]["ref"], b.cb[g]["ref"]) and torch.equal(a.cb[g]["mag"], b.cb[g]["mag"])
+            for li in range(wl.n_layers):
+                for s_ in range(len(wl.seq_lens)):
+                    for j in range(wl.n_kv_heads):
+                        m = int(n[li, s_, j])
+                        assert torch.equal(a.cb[g]["C"][li, s_, j, :m], b.cb[g]["C"][li, s_, j, :m])
+
+
 def test_composition_as_written_evict_then_codebooks_of_the_kept_tokens():
     # every layer evicts under the pyramid over all layers, then builds K and V CodeBooks of what it kept
     # (different counts per layer, passed to the CodeBook call as per-layer lengths)
