@@ -202,6 +202,10 @@ spindlekv_status spindlekv_evict_deep_noalloc(const spindlekv_config* cfg, const
  *              bit (b & 31) of word b >> 5 of row a is G[a][b]; rows and words beyond a sequence's own
  *              length are not written; 16-byte aligned, else INVALID_ARG.  With NULL the matrix in the
  *              workspace is sparse: 64-column chunks of a row without a set bit may be left unwritten
+ * Limits: sequences of at most 32768 tokens and at most 65535 (layer, sequence, head) units per call, else
+ * UNSUPPORTED; two calls may run at the same time on different streams when each has a workspace of its own.
+ * A bounded device wait that gave up, or a greedy cover that exceeded its round limit, leaves TIMEOUT in the
+ * workspace's status word (spindlekv_poll_status), never an endless wait.
  */
 spindlekv_status spindlekv_codebook_shallow(const spindlekv_config* cfg, const spindlekv_batch* batch,
                                             spindlekv_tensor Gamma, float theta,
