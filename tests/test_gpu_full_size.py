@@ -27,14 +27,14 @@ MAX_MARGIN_KEPT_POSITIONS = 16
 
 
 def _record_margins(name, units_evict, kept_positions, units_codebook, adjacency_bits):
-    """Asserts the bounds and leaves one line per workload in ``gpurun_out/margin_counts.jsonl`` (scratch output of a
-    GPU run; the committed summary under ``profiles/`` is copied from it)."""
+    """Asserts the bounds and, where the run's scratch output folder exists, leaves one line per workload in its
+    ``margin_counts.jsonl`` (the committed summary under ``profiles/`` is copied from such a run)."""
     import json
     import os
     assert kept_positions <= MAX_MARGIN_KEPT_POSITIONS * max(1, units_evict)
     assert adjacency_bits <= MAX_MARGIN_ADJACENCY_BITS * max(1, units_codebook)
     root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
-    out = os.path.join(root, "gpurun_out")
+    out = os.path.join(root, os.environ.get("SPINDLEKV_TEST_OUT", "gpurun_out"))
     if os.path.isdir(out):
         with open(os.path.join(out, "margin_counts.jsonl"), "a") as f:
             f.write(json.dumps({"workload": name, "sampled_evicting_units": units_evict,
