@@ -119,8 +119,8 @@ class SpindleKVPass:
     def run(self, K: torch.Tensor, V: torch.Tensor, Q: torch.Tensor, stream=None) -> None:
         """All layers of one prompt batch (``K``/``V`` hold every layer)."""
         ns = self.n_shallow
-        if self.side_by_side and ns:
-            return self._run_side_by_side(K, V, Q, stream)
+        if self.side_by_side and ns and (stream is None or isinstance(stream, torch.cuda.Stream)):
+            return self._run_side_by_side(K, V, Q, stream)   # (a raw stream handle cannot be joined with: one stream then)
         if self.n_deep:
             self.evict(K[ns:], V[ns:], Q, stream)
         if ns:
@@ -311,7 +311,7 @@ class SpindleKVLiteralPass:
 
     def run(self, K: torch.Tensor, V: torch.Tensor, Q: torch.Tensor, which=("K", "V"), stream=None) -> None:
         self.ev.evict(K, V, Q, stream)
-        if self.adj is None and tuple(which) == ("K", "V"):
+        if self.adj is None and tuple(which) == ("K", "V") and (stream is None or isinstance(stream, torch.cuda.Stream)):
             # the two CodeBook calls are independent: the V call runs on a side stream with a workspace of its own
             cur = stream if stream is not None else torch.cuda.current_stream(self.device)
             if not hasattr(self, "_side"):
@@ -409,7 +409,7 @@ class SpindleKVRepeatPass:
             B.spindlekv_compact(self.cb_batch, H, d, B.desc_bhnd(rep), o["centre_idx"], o["n_entries"],
                                 B.desc_bhnd(o["C"]), o["mag"], None, st)
 
-        if self.adj is None and tuple(which) == ("K", "V"):
+        if self.adj is None and tuple(which) == ("K", "V") and (stream is None or isinstance(stream, torch.cuda.Stream)):
             # the two CodeBook calls are independent: the V call runs on a side stream with a workspace of its own
             cur = stream if stream is not None else torch.cuda.current_stream(self.device)
             if not hasattr(self, "_side"):
