@@ -127,6 +127,22 @@ class SpindleKVPass:
             self.codebook(K[:ns], "K", stream)
             self.codebook(V[:ns], "V", stream)
 
+    def capture(self, K: torch.Tensor, V: torch.Tensor, Q: torch.Tensor) -> "torch.cuda.CUDAGraph":
+        """Records one ``run`` on these tensors (side streams included) as a CUDA graph and returns it; ``replay()``
+        on the result repeats the pass on whatever the same tensors hold by then, with one launch from the host.
+        ``run`` is called once outside the capture first, so that everything that is set up on first use (kernel
+        attributes, side streams, the second workspace) exists before the recording starts."""
+        warm = torch.cuda.Stream(self.device)
+        warm.wait_stream(torch.cuda.current_stream(self.device))
+        with torch.cuda.stream(warm):
+            self.run(K, V, Q)
+        torch.cuda.current_stream(self.device).wait_stream(warm)
+        torch.cuda.synchronize(self.device)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            self.run(K, V, Q)
+        return graph
+
     def _run_side_by_side(self, K, V, Q, stream=None) -> None:
         """``run`` on three streams: K CodeBooks on the caller's stream, V CodeBooks and the eviction on two side
         streams that start after the work already queued on the caller's stream and are joined before returning."""

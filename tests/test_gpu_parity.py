@@ -225,6 +225,44 @@ def test_three_streams_give_what_one_stream_gives():
                     assert torch.equal(side.V_kept[li, a:b, j], serial.V_kept[li, a:b, j])
 
 
+def test_a_pass_replayed_from_a_cuda_graph_gives_the_same_outputs():
+    # run() recorded once (three streams, memsets and all kernels) and replayed on new contents of the same input tensors
+    wl = synth.Workload("graph", 4, 2, 8, 2, 128, "bf16", 32, (900,), 30, (0.05, 0.3), 2, "recency",
+                        budget_frac=0.3, seed=44)
+    other = wl.replace(seed=45)
+    layers = list(range(wl.n_layers))
+    def tensors(w):
+        host = generate(w)
+        return (stack_layers(w, host, layers, "K"), stack_layers(w, host, layers, "V"),
+                stack_layers(w, host, layers[w.n_shallow:], "Q"))
+    K, V, Q = tensors(wl)
+    K2, V2, Q2 = tensors(other)
+    direct = _pass(wl)
+    direct.run(K2, V2, Q2)
+    p = _pass(wl)
+    graph = p.capture(K, V, Q)
+    K.copy_(K2); V.copy_(V2); Q.copy_(Q2)
+    for _ in range(2):
+        graph.replay()
+        st = p.device_status()
+        assert st["evict"][0] == 0 and st["codebook"][0] == 0 and st["codebook_v"][0] == 0
+        for g in ("K", "V"):
+            n = direct.cb[g]["n_entries"].cpu()
+            assert torch.equal(p.cb[g]["n_entries"].cpu(), n)
+            assert torch.equal(p.cb[g]["ref"], direct.cb[g]["ref"]) and torch.equal(p.cb[g]["mag"], direct.cb[g]["mag"])
+            for li in range(wl.n_shallow):
+                for j in range(wl.n_kv_heads):
+                    m = int(n[li, 0, j])
+                    assert torch.equal(p.cb[g]["C"][li, 0, j, :m], direct.cb[g]["C"][li, 0, j, :m])
+        assert torch.equal(p.keep_cnt, direct.keep_cnt)
+        cnt = direct.keep_cnt.cpu()
+        for li in range(wl.n_layers - wl.n_shallow):
+            for j in range(wl.n_kv_heads):
+                m = int(cnt[li, 0, j])
+                assert torch.equal(p.keep_idx[li, j, :m], direct.keep_idx[li, j, :m])
+                assert torch.equal(p.K_kept[li, 0, j, :m], direct.K_kept[li, 0, j, :m])
+
+
 def test_side_stream_of_the_composition_as_written_changes_nothing():
     # the literal and the repeat pass build the V CodeBooks on a side stream while the K CodeBooks are built on the
     # caller's: same outputs as one Gamma after the other
