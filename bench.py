@@ -258,6 +258,20 @@ def host_inputs(wl):
     return K, V, Q
 
 
+def recorded(fn, dev):
+    """``fn`` as a replay of its CUDA graph (one launch from the host per step) and the number of kernels a replay
+    stands for; ``fn`` itself and 0 where recording is not possible."""
+    from paper_2507_06517_b200 import binding as B
+    from paper_2507_06517_b200.pipeline import record_graph
+    B.spindlekv_launch_count(True)
+    try:
+        graph = record_graph(fn, dev)
+        return graph.replay, B.spindlekv_launch_count(True) // 2    # the recording runs fn twice
+    except Exception as exc:   # noqa: BLE001
+        print(f"[bench] CUDA graph capture failed ({exc}); direct calls", file=sys.stderr)
+        return fn, 0
+
+
 def run_literal(args, wl):
     """Every layer evicts under the pyramid over all layers, then builds K and V CodeBooks of the kept
     tokens (Section 3 as written).  Single GPU; reports throughput and the reserve ratios of Eq. (15)."""
@@ -275,21 +289,22 @@ def run_literal(args, wl):
                    reserve_ratio=wl.budget_frac if wl.budget_frac is not None else -1.0)
     p = (SpindleKVRepeatPass if args.repeat else SpindleKVLiteralPass)(cfg, wl.seq_lens, hK.dtype, device=dev)
     dK, dV, dQ = hK.to(dev), hV.to(dev), hQ.to(dev)
+    step, per_replay = recorded(lambda: p.run(dK, dV, dQ), dev)
     for _ in range(max(args.warmup, 3)):
-        p.run(dK, dV, dQ)
+        step()
     st = p.device_status()
-    if st["evict"][0] or st["codebook"][0]:
+    if any(v[0] for v in st.values()):
         raise RuntimeError(f"device status {st}")
     B.spindlekv_launch_count(True)
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     torch.cuda.synchronize(dev)
     ev0.record()
     for _ in range(args.steps):
-        p.run(dK, dV, dQ)
+        step()
     ev1.record()
     torch.cuda.synchronize(dev)
     ms = ev0.elapsed_time(ev1)
-    launches = B.spindlekv_launch_count(True)
+    launches = B.spindlekv_launch_count(True) + per_replay * args.steps
     nk, nv = p.cb["K"]["n_entries"].cpu().numpy(), p.cb["V"]["n_entries"].cpu().numpy()
     kept = p.kept_host[:, 0].astype(np.float64)       # tokens kept per head (per query head when unfolded)
     heads = wl.n_q_heads if args.repeat else wl.n_kv_heads   # Eq. (15): h_g = h after a repeat
@@ -334,7 +349,7 @@ def run_decode(args, wl):
     g = torch.Generator(device="cpu").manual_seed(wl.seed)
     q = torch.randn((wl.n_layers, wl.batch, wl.n_q_heads, 1, d), generator=g).to(hK.dtype).to(dev)
     pos_q = torch.full((wl.batch,), n, dtype=torch.int32, device=dev)
-    step = lambda: att.run(q, pos_q, p.cb["K"], p.cb["V"])
+    step, per_replay = recorded(lambda: att.run(q, pos_q, p.cb["K"], p.cb["V"]), dev)
     for _ in range(max(args.warmup, 3)):
         step()
     B.spindlekv_launch_count(True)
@@ -346,7 +361,7 @@ def run_decode(args, wl):
     ev1.record()
     torch.cuda.synchronize(dev)
     ms = ev0.elapsed_time(ev1) / args.steps
-    launches = B.spindlekv_launch_count(True)
+    launches = B.spindlekv_launch_count(True) + per_replay * args.steps
     entries = int(p.cb["K"]["n_entries"].sum().item()) + int(p.cb["V"]["n_entries"].sum().item())
     units = wl.n_layers * wl.batch * wl.n_kv_heads
     alg = entries * d * e + units * n * 16                  # CodeBook rows once; reference and magnitude of K and of V per token
@@ -448,15 +463,8 @@ def run_native(args, wl):
     run_direct = lambda: p.run(dK, dV, dQ)
     # the timed steps replay one recorded pass (a CUDA graph: one launch from the host per step); direct calls where
     # recording is not possible, and for the per-kernel pass further down
-    B.spindlekv_launch_count(True)
-    try:
-        graph = p.capture(dK, dV, dQ)
-        launches_per_replay = B.spindlekv_launch_count(True) // 2   # capture() runs the pass twice
-        step = graph.replay
-    except Exception as exc:   # noqa: BLE001
-        print(f"[bench] CUDA graph capture failed ({exc}); direct calls", file=sys.stderr)
-        graph, launches_per_replay = None, 0
-        step = run_direct
+    step, launches_per_replay = recorded(run_direct, dev)
+    graph = step if step is not run_direct else None
     for _ in range(max(args.warmup, 3)):
         step()
     st = p.device_status()

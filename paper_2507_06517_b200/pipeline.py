@@ -13,6 +13,24 @@ import torch
 from . import binding as B
 
 
+def record_graph(fn, device="cuda") -> "torch.cuda.CUDAGraph":
+    """Records what ``fn()`` enqueues (calls of this library on the current stream and on streams forked from it) as a
+    CUDA graph; ``replay()`` on the result repeats it with one launch from the host.  ``fn`` runs once outside the
+    recording first, so that whatever is set up on first use (kernel attributes, side streams, workspaces) exists
+    before the recording starts; the tensors it uses must stay where they are."""
+    dev = torch.device(device)
+    warm = torch.cuda.Stream(dev)
+    warm.wait_stream(torch.cuda.current_stream(dev))
+    with torch.cuda.stream(warm):
+        fn()
+    torch.cuda.current_stream(dev).wait_stream(warm)
+    torch.cuda.synchronize(dev)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        fn()
+    return graph
+
+
 class SpindleKVPass:
     """Buffers and call sequence for one prompt batch.
 
@@ -129,19 +147,8 @@ class SpindleKVPass:
 
     def capture(self, K: torch.Tensor, V: torch.Tensor, Q: torch.Tensor) -> "torch.cuda.CUDAGraph":
         """Records one ``run`` on these tensors (side streams included) as a CUDA graph and returns it; ``replay()``
-        on the result repeats the pass on whatever the same tensors hold by then, with one launch from the host.
-        ``run`` is called once outside the capture first, so that everything that is set up on first use (kernel
-        attributes, side streams, the second workspace) exists before the recording starts."""
-        warm = torch.cuda.Stream(self.device)
-        warm.wait_stream(torch.cuda.current_stream(self.device))
-        with torch.cuda.stream(warm):
-            self.run(K, V, Q)
-        torch.cuda.current_stream(self.device).wait_stream(warm)
-        torch.cuda.synchronize(self.device)
-        graph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(graph):
-            self.run(K, V, Q)
-        return graph
+        on the result repeats the pass on whatever the same tensors hold by then, with one launch from the host."""
+        return record_graph(lambda: self.run(K, V, Q), self.device)
 
     def _run_side_by_side(self, K, V, Q, stream=None) -> None:
         """``run`` on three streams: K CodeBooks on the caller's stream, V CodeBooks and the eviction on two side
