@@ -26,7 +26,8 @@ def record_graph(fn, device="cuda") -> "torch.cuda.CUDAGraph":
     torch.cuda.current_stream(dev).wait_stream(warm)
     torch.cuda.synchronize(dev)
     graph = torch.cuda.CUDAGraph()
-    with torch.cuda.graph(graph):
+    # only this thread's calls belong to the recording (a communication library's watchdog thread may poll its events meanwhile)
+    with torch.cuda.graph(graph, capture_error_mode="thread_local"):
         fn()
     return graph
 
