@@ -143,12 +143,11 @@ __global__ void __launch_bounds__(kDecThreads, HN <= 4 ? 4 : 2) decode_chunk_ker
   const int nt = min(kDecChunk, n - t0);
   float* sq = sm;                                 // [h_n][D] rotated queries
   float* sc = sq + h_n * D;                       // [kDecChunk][HN] scores, then weights (a token's heads side by side)
-  int32_t* srv = reinterpret_cast<int32_t*>(sc + HN * kDecChunk);             // [kDecChunk] value references
-  float* smv = reinterpret_cast<float*>(srv + kDecChunk);                     // [kDecChunk] value magnitudes
-  int32_t* srk = reinterpret_cast<int32_t*>(smv + kDecChunk);                 // [kDecChunk] key references
-  float* smk = reinterpret_cast<float*>(srk + kDecChunk);                     // [kDecChunk] key magnitudes
-  int32_t* spos = reinterpret_cast<int32_t*>(smk + kDecChunk);                // [kDecChunk] positions, clamped to the table
-  float* red = reinterpret_cast<float*>(spos + kDecChunk);                    // [2][warps][HN] reduction scratch
+  // per token, read with one 16-byte load: key reference, key magnitude (bits), position clamped to the table,
+  // value reference
+  int4* stok = reinterpret_cast<int4*>(sc + HN * kDecChunk);                  // [kDecChunk]
+  float* smv = reinterpret_cast<float*>(stok + kDecChunk);                    // [kDecChunk] value magnitudes
+  float* red = smv + kDecChunk;                                               // [2][warps][HN] reduction scratch
   float* ps = red + 2 * kDecMaxGroup * (kDecThreads / 32);             // [warps][h_n][D] partial value sums
   const int64_t orow = ((int64_t)layer * p.n_kv_heads + j) * p.batch.total_len + tok_base(p.batch, s);
   const T* ck = reinterpret_cast<const T*>(p.CK.ptr) + unit_offset(p.CK, p.batch, layer, s, j);
@@ -168,11 +167,10 @@ __global__ void __launch_bounds__(kDecThreads, HN <= 4 ? 4 : 2) decode_chunk_ker
     }
   }
   for (int t = tid; t < nt; t += kDecThreads) {
-    srv[t] = p.ref_v[orow + t0 + t];
     smv[t] = p.mag_v[orow + t0 + t];
-    srk[t] = p.ref_k[orow + t0 + t];
-    smk[t] = p.mag_k[orow + t0 + t];
-    spos[t] = min(max(p.positions ? p.positions[orow + t0 + t] : t0 + t, 0), p.table_positions - 1);
+    stok[t] = make_int4(p.ref_k[orow + t0 + t], __float_as_int(p.mag_k[orow + t0 + t]),
+                        min(max(p.positions ? p.positions[orow + t0 + t] : t0 + t, 0), p.table_positions - 1),
+                        p.ref_v[orow + t0 + t]);
   }
   __syncthreads();
   // ---- 1. scores: two tokens per 16-thread group and sweep, all their loads in flight before any is used ----
@@ -200,9 +198,10 @@ __global__ void __launch_bounds__(kDecThreads, HN <= 4 ? 4 : 2) decode_chunk_ker
         const int t = tb + x * (kDecThreads / 16) + grp;
         tk[x] = t;
         const bool has = t < nt;
-        const int r = has ? srk[t] : 0;
-        m[x] = has ? smk[t] : 0.f;
-        const float2* tab = p.table + (int64_t)(has ? spos[t] : 0) * H + sub * PPT;
+        const int4 tk4 = has ? stok[t] : make_int4(0, 0, 0, 0);
+        const int r = tk4.x;
+        m[x] = __int_as_float(tk4.y);
+        const float2* tab = p.table + (int64_t)tk4.z * H + sub * PPT;
         const T* row = ck + (int64_t)r * p.CK.st;
         load_row_piece<T, PPT>(row + sub * PPT, lo[x]);
         load_row_piece<T, PPT>(row + H + sub * PPT, hi[x]);
@@ -315,7 +314,7 @@ __global__ void __launch_bounds__(kDecThreads, HN <= 4 ? 4 : 2) decode_chunk_ker
 #pragma unroll
       for (int i = 0; i < kUnroll; ++i) {
         const int t = tb + i * G;
-        const int r = t < nt ? srv[t] : 0;
+        const int r = t < nt ? stok[t].w : 0;
         raw[i] = *reinterpret_cast<const uint4*>(cv + (int64_t)r * p.CV.st + sub * EPT);
       }
 #pragma unroll
